@@ -1,0 +1,330 @@
+"""fp64 CPU oracle for the MGRIT solve of the GRU recurrence (forward and adjoint).
+
+THIS IS TEST INFRASTRUCTURE, NOT THE PRODUCT.  It is a plain, slow, NumPy float64
+restatement of the method, written from the paper's equations and algorithms in
+their own order and notation, so that it can be checked against the paper by eye.
+It shares no code with the CUDA path and must never be imported by it; only the
+tests, the smoke check and the benchmark's CPU-baseline leg call it.
+
+What pins each function (see tests/test_oracle_*.py):
+  * classic cell / serial sweep / BPTT ........ torch.nn.GRU in float64 (Eq. "gru")
+  * implicit cell ............................. algebraic identity of Eq. "gru-implicit",
+                                                limits z->1 and gamma->0, model-problem decay
+  * adjoint step coefficients ................. central finite differences
+  * MGRIT cycle (forward and adjoint) ......... fixed point, exactness after T/c_f (F) and
+                                                T/(2 c_f) (FCF) two-level cycles, prefix
+                                                exactness, monotone residual, hand-unrolled
+                                                brute force on T=8, dense two-level error
+                                                propagator for the linear adjoint problem,
+                                                hierarchy sizes quoted in the paper
+  * loss head ................................. torch.nn.functional.cross_entropy float64
+  * values after a FEW cycles (2-3) ........... parity unpinned by the paper (an iteration's
+                                                intermediate iterates have no closed form);
+                                                they are covered only indirectly by the pins
+                                                above, which any wrong step of the cycle breaks.
+
+Array conventions (row-major, time-major): x[T,B,I], gi[T,B,3H], h[T,B,H] with h[k] the
+paper's h_{k+1}; h_0 is passed separately.  Gate order along 3H is r | z | n.
+"""
+from __future__ import annotations
+
+import numpy as np
+
+CELL_CLASSIC = 0   # explicit Euler propagator, Eq. "gru-classic"
+CELL_IMPLICIT = 1  # Implicit GRU propagator, Eq. "gru-imap"
+RELAX_F = 0
+RELAX_FCF = 1
+
+
+# --------------------------------------------------------------------------- cell
+def sigmoid(a):
+    return 1.0 / (1.0 + np.exp(-a))
+
+
+def input_projection(W_ih, b_ih, x):
+    """gi_t = W_i x_t + b_i for every t (input half of Eq. "gru"); computed once on the
+    fine grid and reused by every level and by the adjoint (Appendix, feature reuse)."""
+    return x @ W_ih.T + b_ih
+
+
+def gates(W_hh, b_hh, gi, h_prev):
+    """r, z, n of Eq. "gru" from the pre-computed input part gi and the previous state.
+    Also returns gh_n = W_hn h + b_hn, which the adjoint needs."""
+    H = h_prev.shape[-1]
+    gh = h_prev @ W_hh.T + b_hh
+    r = sigmoid(gi[..., 0:H] + gh[..., 0:H])
+    z = sigmoid(gi[..., H:2 * H] + gh[..., H:2 * H])
+    n = np.tanh(gi[..., 2 * H:3 * H] + r * gh[..., 2 * H:3 * H])
+    return r, z, n, gh[..., 2 * H:3 * H]
+
+
+def phi(W_hh, b_hh, gi, h_prev, gamma, cell):
+    """Propagator Phi_gamma(x_t, h_{t-1}).
+
+    classic  (Eq. "gru-classic"): h + gamma * ( -(1-z) h + (1-z) n )
+    implicit (Eq. "gru-imap")   : (1 + gamma (1-z))^-1 * ( h + gamma (1-z) n )
+    """
+    r, z, n, _ = gates(W_hh, b_hh, gi, h_prev)
+    q = gamma * (1.0 - z)
+    if cell == CELL_CLASSIC:
+        return h_prev + q * (n - h_prev)
+    if cell == CELL_IMPLICIT:
+        return (h_prev + q * n) / (1.0 + q)
+    raise ValueError("cell")
+
+
+def adjoint_coefficients(W_hh, b_hh, gi, h_prev, gamma, cell):
+    """Entries of the transposed Jacobian of one Phi_gamma step (discrete adjoint of
+    Eq. "gru-imap" / "gru-classic").  With lambda the sensitivity of the step's output:
+
+        lambda_prev = a*lambda + [c_r*lambda | c_z*lambda | c_n*lambda] W_hh
+        d(gi)       =            [c_r*lambda | c_z*lambda | c_np*lambda]
+
+    Returns a, c_r, c_z, c_n, c_np  (c_n = c_np * r: the n-gate path seen through gh_n).
+    """
+    r, z, n, gh_n = gates(W_hh, b_hh, gi, h_prev)
+    q = gamma * (1.0 - z)
+    if cell == CELL_IMPLICIT:
+        D = 1.0 + q
+        a = 1.0 / D
+        dPhi_dn = q / D
+        dPhi_dz = -gamma * (n - h_prev) / (D * D)
+    elif cell == CELL_CLASSIC:
+        a = 1.0 - q
+        dPhi_dn = q
+        dPhi_dz = -gamma * (n - h_prev)
+    else:
+        raise ValueError("cell")
+    c_np = dPhi_dn * (1.0 - n * n)
+    c_n = c_np * r
+    c_r = c_np * gh_n * r * (1.0 - r)
+    c_z = dPhi_dz * z * (1.0 - z)
+    return a, c_r, c_z, c_n, c_np
+
+
+# --------------------------------------------------------------------------- serial sweep
+def serial_forward(W_ih, W_hh, b_ih, b_hh, x, h0, cell=CELL_IMPLICIT, dt=1.0):
+    """h_t = Phi_dt(x_t, h_{t-1}), t = 1..T: the solution of f(h) = 0 (Eq. "fine-res")."""
+    T = x.shape[0]
+    gi = input_projection(W_ih, b_ih, x)
+    h = np.empty((T,) + h0.shape)
+    prev = h0
+    for t in range(T):
+        prev = phi(W_hh, b_hh, gi[t], prev, dt, cell)
+        h[t] = prev
+    return h
+
+
+def weight_gradients(W_ih, W_hh, b_ih, b_hh, x, h0, h, lam, cell=CELL_IMPLICIT, dt=1.0, want_dx=True):
+    """g_i = w_i d(h_i)/d(Theta) for every fine step (Algorithm "MGRITTraining", gradient
+    line): one time-parallel pass with given states h and sensitivities lam (lam[k] = dL/dh_{k+1})."""
+    T = x.shape[0]
+    gi = input_projection(W_ih, b_ih, x)
+    hprev = np.concatenate([h0[None], h[:-1]], axis=0)           # h_{t-1} for t = 1..T
+    a, c_r, c_z, c_n, c_np = adjoint_coefficients(W_hh, b_hh, gi, hprev, dt, cell)
+    dA_h = np.concatenate([c_r * lam, c_z * lam, c_n * lam], axis=-1)    # [T,B,3H]
+    dA_i = np.concatenate([c_r * lam, c_z * lam, c_np * lam], axis=-1)
+    G3 = dA_h.shape[-1]
+    out = {
+        "dW_hh": dA_h.reshape(-1, G3).T @ hprev.reshape(-1, hprev.shape[-1]),
+        "dW_ih": dA_i.reshape(-1, G3).T @ x.reshape(-1, x.shape[-1]),
+        "db_hh": dA_h.reshape(-1, G3).sum(axis=0),
+        "db_ih": dA_i.reshape(-1, G3).sum(axis=0),
+    }
+    if want_dx:
+        out["dx"] = dA_i @ W_ih
+    return out
+
+
+def serial_backward(W_ih, W_hh, b_ih, b_hh, x, h0, h, dh_seed, cell=CELL_IMPLICIT, dt=1.0):
+    """Exact back-propagation through time for the serial sweep.
+
+    dh_seed[k] is the direct derivative of the loss with respect to h_{k+1} (zero except the
+    last slice for a loss on h_T).  Returns the total sensitivities lam[k] = dL/dh_{k+1},
+    lam0 = dL/dh_0 and the parameter / input gradients."""
+    T = x.shape[0]
+    gi = input_projection(W_ih, b_ih, x)
+    lam = np.empty_like(h)
+    cur = dh_seed[T - 1].copy()
+    for t in range(T, 0, -1):                       # paper index t: step h_{t-1} -> h_t
+        lam[t - 1] = cur
+        hprev = h[t - 2] if t >= 2 else h0
+        a, c_r, c_z, c_n, _ = adjoint_coefficients(W_hh, b_hh, gi[t - 1], hprev, dt, cell)
+        back = a * cur + np.concatenate([c_r * cur, c_z * cur, c_n * cur], axis=-1) @ W_hh
+        cur = back + (dh_seed[t - 2] if t >= 2 else 0.0)
+    lam0 = cur
+    grads = weight_gradients(W_ih, W_hh, b_ih, b_hh, x, h0, h, lam, cell, dt)
+    return lam, lam0, grads
+
+
+# --------------------------------------------------------------------------- MGRIT cycle
+def level_sizes(T, cf, levels):
+    """N_l = T / c_f^l (e.g. 128/32/8 for c_f = 4 and three levels)."""
+    if cf < 2 or levels < 1:
+        raise ValueError("cf >= 2 and levels >= 1 required")
+    if T % (cf ** (levels - 1)) != 0:
+        raise ValueError("T must be divisible by cf^(levels-1)")
+    return [T // cf ** l for l in range(levels)]
+
+
+def fas_vcycle(step, N, cf, relax, u, g, l=0, resnorm=None):
+    """One multigrid cycle on level l (Algorithm "MGProp" with the recursive coarse solve of
+    the remark "Beyond Two-Level"), for the level-l system
+
+        u_j = step(l, j, u_{j-1}) + g_j ,  j = 1..N_l ,   u_0 fixed.
+
+    step(l, j, u_prev): j is an integer array of target points, u_prev their predecessors'
+    states; all entries are independent (the "ParallelFor" of Algorithm "F-relaxation").
+    u[l], g[l]: arrays [N_l+1, ...].  relax[l] in {RELAX_F, RELAX_FCF}.  Modifies u in place.
+    """
+    Nl = N[l]
+    ul, gl = u[l], g[l]
+    L = len(N)
+    if l == L - 1:
+        # coarsest level: serial propagation resolves the level's system exactly
+        for j in range(1, Nl + 1):
+            ul[j] = step(l, np.array([j]), ul[j - 1:j])[0] + gl[j]
+        return
+
+    def f_relax():
+        # from every C-point fill the F-points up to the next C-point, exclusive
+        for s in range(1, cf):
+            j = np.arange(0, Nl, cf) + s
+            ul[j] = step(l, j, ul[j - 1]) + gl[j]
+
+    def c_relax():
+        # one more step from the last F-point of each interval onto the next C-point
+        j = np.arange(cf, Nl + 1, cf)
+        ul[j] = step(l, j, ul[j - 1]) + gl[j]
+
+    # relax the current guess
+    f_relax()
+    if relax[l] == RELAX_FCF:
+        c_relax()
+        f_relax()
+
+    # residual at the C-points, restricted by injection:  r_c = R(f(h')),  h'_c = R(h')
+    jc = np.arange(cf, Nl + 1, cf)
+    v = step(l, jc, ul[jc - 1]) + gl[jc]
+    r_c = ul[jc] - v
+    if resnorm is not None and l == 0:
+        resnorm.append(float(np.sqrt(np.sum(r_c * r_c))))
+    Uc = np.concatenate([ul[0:1], ul[jc]], axis=0)            # U'_0 .. U'_{N_{l+1}}
+
+    # coarse equation f_c(h_c*) = f_c(h'_c) - r_c, i.e.  U_k = step(l+1,k,U_{k-1}) + G_k  with
+    # G_k = U'_k - step(l+1,k,U'_{k-1}) - r_k = v_k - step(l+1,k,U'_{k-1})
+    k = np.arange(1, N[l + 1] + 1)
+    G = np.zeros_like(Uc)
+    G[k] = v - step(l + 1, k, Uc[k - 1])
+    u[l + 1] = Uc.copy()                                       # initial guess = restricted state
+    g[l + 1] = G
+    fas_vcycle(step, N, cf, relax, u, g, l + 1, resnorm)
+
+    # h'' = h' + P(h_c* - h'_c): only the C-point values are read afterwards
+    ul[jc] = u[l + 1][1:]
+    # final F-relaxation spreads the correction over the F-points
+    f_relax()
+
+
+def _relax_list(levels, relax_fine, relax_coarse):
+    return [relax_fine] + [relax_coarse] * (levels - 1)
+
+
+def mgrit_forward(W_ih, W_hh, b_ih, b_hh, x, h0, cf, levels, iters, cell=CELL_IMPLICIT,
+                  relax_fine=RELAX_F, relax_coarse=RELAX_FCF, dt=1.0, h_init=None):
+    """Forward propagation by `iters` MGRIT cycles from the zero initial guess
+    (Algorithm "MGRITTraining", forward block).  Level l uses the same cell with time step
+    gamma = c_f^l * dt and, for its point j, the input of fine step c_f^l * j.
+
+    Returns h[T,B,H] and the list of level-0 C-point residual 2-norms, one per cycle, each
+    measured after that cycle's pre-relaxation."""
+    T = x.shape[0]
+    N = level_sizes(T, cf, levels)
+    gi = input_projection(W_ih, b_ih, x)
+
+    def step(l, j, u_prev):
+        m = cf ** l
+        return phi(W_hh, b_hh, gi[m * j - 1], u_prev, m * dt, cell)
+
+    u = [None] * levels
+    g = [None] * levels
+    u[0] = np.zeros((T + 1,) + h0.shape)
+    u[0][0] = h0
+    if h_init is not None:
+        u[0][1:] = h_init
+    g[0] = np.zeros_like(u[0])
+    relax = _relax_list(levels, relax_fine, relax_coarse)
+    resnorm = []
+    if levels == 1:
+        fas_vcycle(step, N, cf, relax, u, g, 0, None)
+        return u[0][1:].copy(), resnorm
+    for _ in range(iters):
+        fas_vcycle(step, N, cf, relax, u, g, 0, resnorm)
+    return u[0][1:].copy(), resnorm
+
+
+def mgrit_adjoint(W_ih, W_hh, b_ih, b_hh, x, h0, h, dh_seed, cf, levels, iters, cell=CELL_IMPLICIT,
+                  relax_fine=RELAX_F, relax_coarse=RELAX_FCF, dt=1.0, want_dx=True):
+    """Backward propagation by MGRIT on the adjoint recurrence, time reversed
+    (Algorithm "MGRITTraining", backward block; Appendix "Training With MGRIT").
+
+    Reversed index s = N_l - j: the level-l unknown mu_s approximates lambda at forward
+    point N_l - s.  mu_0 = lambda_T is fixed; the step arriving at s applies the transposed
+    Jacobian of forward step j = N_l - s + 1 of level l, linearised at the GIVEN states h
+    (restricted by injection) with gamma = c_f^l dt.  The fine-level source is the direct
+    loss derivative dh_seed at that time.  Zero initial guess.
+
+    Returns lam[T,B,H] (lam[k] = dL/dh_{k+1}), lam0, gradients (one time-parallel pass with
+    the final lam and h) and the residual norms."""
+    T = x.shape[0]
+    N = level_sizes(T, cf, levels)
+    gi = input_projection(W_ih, b_ih, x)
+    hfull = np.concatenate([h0[None], h], axis=0)                 # h_0 .. h_T
+
+    def step(l, s, mu_prev):
+        m = cf ** l
+        j = N[l] - s + 1
+        a, c_r, c_z, c_n, _ = adjoint_coefficients(W_hh, b_hh, gi[m * j - 1], hfull[m * (j - 1)],
+                                                   m * dt, cell)
+        return a * mu_prev + np.concatenate([c_r * mu_prev, c_z * mu_prev, c_n * mu_prev], axis=-1) @ W_hh
+
+    u = [None] * levels
+    g = [None] * levels
+    u[0] = np.zeros((T + 1,) + h0.shape)
+    u[0][0] = dh_seed[T - 1]
+    g[0] = np.zeros_like(u[0])
+    for s in range(1, T):
+        g[0][s] = dh_seed[T - s - 1]                               # seed at forward point T-s
+    relax = _relax_list(levels, relax_fine, relax_coarse)
+    resnorm = []
+    if levels == 1:
+        fas_vcycle(step, N, cf, relax, u, g, 0, None)
+    else:
+        for _ in range(iters):
+            fas_vcycle(step, N, cf, relax, u, g, 0, resnorm)
+    lam = np.ascontiguousarray(u[0][0:T][::-1])                    # lam[k] = mu_{T-1-k}
+    lam0 = u[0][T].copy()
+    grads = weight_gradients(W_ih, W_hh, b_ih, b_hh, x, h0, h, lam, cell, dt, want_dx)
+    return lam, lam0, grads, resnorm
+
+
+# --------------------------------------------------------------------------- head / update
+def xent_head(hT, W_c, b_c, labels):
+    """Linear classifier on h_T with mean softmax cross-entropy; returns the loss and
+    w_T = grad_{h_T} L (the seed of the backward block) plus the head's own gradients."""
+    B = hT.shape[0]
+    logits = hT @ W_c.T + b_c
+    m = logits.max(axis=1, keepdims=True)
+    e = np.exp(logits - m)
+    p = e / e.sum(axis=1, keepdims=True)
+    logp = (logits - m) - np.log(e.sum(axis=1, keepdims=True))
+    loss = -np.mean(logp[np.arange(B), labels])
+    dlogits = p.copy()
+    dlogits[np.arange(B), labels] -= 1.0
+    dlogits /= B
+    return loss, dlogits @ W_c, dlogits.T @ hT, dlogits.sum(axis=0)
+
+
+def sgd_update(p, g, lr):
+    """Theta <- Theta - l_r g (last line of Algorithm "MGRITTraining")."""
+    return p - lr * g

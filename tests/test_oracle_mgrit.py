@@ -1,0 +1,215 @@
+"""Pins for the oracle's MGRIT cycle, forward and adjoint (CPU only)."""
+import os
+
+import numpy as np
+import pytest
+
+from oracle import mgrit_gru_oracle as O
+from tests.helpers import f64_inputs, tiny_workload
+
+GOLDEN = os.path.join(os.path.dirname(__file__), "golden")
+
+
+def test_hierarchy_sizes_quoted_in_the_paper():
+    # Appendix, residual-convergence study: c_f=4 -> 128/32/8; c_f=2 -> 128..4; c_f=8 -> 128/16
+    assert O.level_sizes(128, 4, 3) == [128, 32, 8]
+    assert O.level_sizes(128, 2, 6) == [128, 64, 32, 16, 8, 4]
+    assert O.level_sizes(128, 8, 2) == [128, 16]
+    with pytest.raises(ValueError):
+        O.level_sizes(100, 8, 3)
+
+
+def test_serial_solution_is_a_fixed_point():
+    # f(h*) = 0: the cycle applied to the serial solution returns it, residual zero
+    w = tiny_workload()
+    P, x, h0, _ = f64_inputs(w)
+    hs = O.serial_forward(*P, x, h0)
+    for levels, rf, rc in ((2, 0, 1), (3, 1, 1), (3, 0, 0)):
+        h, res = O.mgrit_forward(*P, x, h0, cf=4, levels=levels, iters=1, relax_fine=rf,
+                                 relax_coarse=rc, h_init=hs)
+        assert np.max(np.abs(h - hs)) < 1e-14
+        assert res[0] < 1e-13
+
+
+@pytest.mark.parametrize("relax,need", [(O.RELAX_F, 16), (O.RELAX_FCF, 8)])
+def test_two_level_is_exact_after_T_over_cf_cycles(relax, need):
+    # two-level MGRIT is a direct method: exact after T/c_f cycles with F-relaxation and
+    # after T/(2 c_f) with FCF-relaxation -- and not before.
+    w = tiny_workload()
+    P, x, h0, _ = f64_inputs(w)
+    hs = O.serial_forward(*P, x, h0)
+    h, _ = O.mgrit_forward(*P, x, h0, cf=4, levels=2, iters=need, relax_fine=relax)
+    assert np.max(np.abs(h - hs)) < 1e-13
+    h, _ = O.mgrit_forward(*P, x, h0, cf=4, levels=2, iters=need - 2, relax_fine=relax)
+    assert np.max(np.abs(h - hs)) > 1e-11          # converging, but not yet a direct solve
+
+
+def test_prefix_exactness():
+    # after k two-level F cycles h_t is exact for t < (k+1) c_f; a multilevel V-cycle is exact
+    # at least for t <= k c_f
+    w = tiny_workload()
+    P, x, h0, _ = f64_inputs(w)
+    hs = O.serial_forward(*P, x, h0)
+    for k in (1, 2, 5):
+        h, _ = O.mgrit_forward(*P, x, h0, cf=4, levels=2, iters=k, relax_fine=O.RELAX_F)
+        n_exact = (k + 1) * 4 - 1                      # paper indices 1 .. (k+1)cf - 1
+        assert np.max(np.abs(h[:n_exact] - hs[:n_exact])) < 1e-14
+        assert np.max(np.abs(h[n_exact:] - hs[n_exact:])) > 1e-6
+        h, _ = O.mgrit_forward(*P, x, h0, cf=4, levels=3, iters=k, relax_fine=O.RELAX_F,
+                               relax_coarse=O.RELAX_FCF)
+        assert np.max(np.abs(h[:k * 4] - hs[:k * 4])) < 1e-14
+
+
+def test_residual_decreases_monotonically_and_limit_is_serial():
+    w = tiny_workload()
+    P, x, h0, _ = f64_inputs(w)
+    hs = O.serial_forward(*P, x, h0)
+    for levels, cf, rf in ((2, 4, 0), (2, 4, 1), (3, 4, 0), (3, 2, 1), (2, 8, 0)):
+        h, res = O.mgrit_forward(*P, x, h0, cf=cf, levels=levels, iters=10, relax_fine=rf)
+        res = [r for r in res if r > 1e-13]
+        assert all(b < a for a, b in zip(res, res[1:])), (levels, cf, rf, res)
+        assert np.max(np.abs(h - hs)) < 1e-4, (levels, cf, rf)
+
+
+def test_explicit_coarse_propagator_is_unstable_implicit_is_not():
+    # Section "Coarse Grid Propagators": forward Euler with step c_f^l > 2 amplifies, the
+    # implicit propagator does not.  Measured on the error before the exactness iteration.
+    w = tiny_workload()
+    P, x, h0, _ = f64_inputs(w)
+    hs_i = O.serial_forward(*P, x, h0, cell=O.CELL_IMPLICIT)
+    hs_e = O.serial_forward(*P, x, h0, cell=O.CELL_CLASSIC)
+    h_i, _ = O.mgrit_forward(*P, x, h0, cf=8, levels=2, iters=3, cell=O.CELL_IMPLICIT)
+    h_e, _ = O.mgrit_forward(*P, x, h0, cf=8, levels=2, iters=3, cell=O.CELL_CLASSIC)
+    assert np.max(np.abs(h_i - hs_i)) < 0.1
+    assert np.max(np.abs(h_e - hs_e)) > 10 * np.max(np.abs(h_i - hs_i))
+
+
+def test_one_cycle_against_hand_unrolled_T4_cf2():
+    # Algorithm "MGProp" written out statement by statement for T=4, c_f=2, two levels,
+    # F-relaxation, zero initial guess; Phi evaluated one point at a time.
+    w = tiny_workload(T=4, B=1, I=3, H=5)
+    P, x, h0, _ = f64_inputs(w)
+    h0 = np.random.default_rng(3).standard_normal(h0.shape) * 0.5
+    gi = O.input_projection(P[0], P[2], x)
+    f = lambda t, hp: O.phi(P[1], P[3], gi[t - 1], hp, 1.0, O.CELL_IMPLICIT)   # fine step into t
+    c = lambda t, hp: O.phi(P[1], P[3], gi[t - 1], hp, 2.0, O.CELL_IMPLICIT)   # coarse step into t
+    z = np.zeros_like(h0)
+    u0, u1, u2, u3, u4 = h0, z, z, z, z
+    u1 = f(1, u0); u3 = f(3, u2)                       # F-relaxation
+    v2 = f(2, u1); v4 = f(4, u3)                       # residual at C-points
+    r2 = u2 - v2; r4 = u4 - v4
+    G2 = v2 - c(2, u0); G4 = v4 - c(4, u2)             # coarse right-hand side
+    U2 = c(2, u0) + G2; U4 = c(4, U2) + G4             # serial coarse solve
+    u2, u4 = U2, U4                                    # correction
+    u1 = f(1, u0); u3 = f(3, u2)                       # final F-relaxation
+    h, res = O.mgrit_forward(*P, x, h0, cf=2, levels=2, iters=1, relax_fine=O.RELAX_F)
+    assert np.max(np.abs(h - np.stack([u1, u2, u3, u4]))) < 1e-15
+    assert abs(res[0] - np.sqrt(np.sum(r2 * r2) + np.sum(r4 * r4))) < 1e-14
+
+
+# ------------------------------------------------------------------ adjoint
+def _adjoint_setup(T=16, B=1, H=5, I=3, seed_all=False):
+    w = tiny_workload(T=T, B=B, I=I, H=H)
+    P, x, h0, _ = f64_inputs(w)
+    rng = np.random.default_rng(9)
+    h0 = rng.standard_normal(h0.shape) * 0.4
+    h = O.serial_forward(*P, x, h0)
+    seed = np.zeros_like(h)
+    seed[-1] = rng.standard_normal(seed[-1].shape)
+    if seed_all:
+        seed += rng.standard_normal(seed.shape)
+    return P, x, h0, h, seed
+
+
+@pytest.mark.parametrize("seed_all", [False, True])
+def test_adjoint_two_level_exact_after_T_over_cf(seed_all):
+    P, x, h0, h, seed = _adjoint_setup(T=32, B=2, seed_all=seed_all)
+    lam_s, lam0_s, g_s = O.serial_backward(*P, x, h0, h, seed)
+    lam, lam0, g, res = O.mgrit_adjoint(*P, x, h0, h, seed, cf=4, levels=2, iters=8, relax_fine=O.RELAX_F)
+    assert np.max(np.abs(lam - lam_s)) < 1e-13
+    assert np.max(np.abs(lam0 - lam0_s)) < 1e-13
+    for k in g_s:
+        assert np.max(np.abs(g[k] - g_s[k])) < 1e-12, k
+    res = [r for r in res if r > 1e-14]
+    assert all(b < a for a, b in zip(res, res[1:]))
+    lam, _, _, _ = O.mgrit_adjoint(*P, x, h0, h, seed, cf=4, levels=3, iters=12, relax_fine=O.RELAX_FCF)
+    assert np.max(np.abs(lam - lam_s)) < 1e-9
+
+
+@pytest.mark.parametrize("relax", [O.RELAX_F, O.RELAX_FCF])
+def test_adjoint_cycle_equals_dense_two_level_error_propagator(relax):
+    # The adjoint recurrence is linear, so one two-level cycle maps the C-point error e to
+    # (I - B^-1 A) e with F-relaxation and (I - B^-1 A)(I - A) e with FCF-relaxation, where A is
+    # the Schur complement of the fine system on the C-points (products of c_f fine step
+    # matrices) and B the coarse-grid operator (two-level MGRIT theory the paper cites).
+    T, cf, H = 16, 4, 5
+    P, x, h0, h, seed = _adjoint_setup(T=T, B=1, H=H)
+    W_hh, b_hh = P[1], P[3]
+    gi = O.input_projection(P[0], P[2], x)
+    hfull = np.concatenate([h0[None], h], 0)
+
+    def step_matrix(j, m):                 # column-vector matrix of the adjoint step of forward step j, level stride m
+        a, c_r, c_z, c_n, _ = O.adjoint_coefficients(W_hh, b_hh, gi[m * j - 1], hfull[m * (j - 1)], float(m), O.CELL_IMPLICIT)
+        M = np.diag(a[0])
+        for gidx, cg in enumerate((c_r, c_z, c_n)):
+            M = M + W_hh[gidx * H:(gidx + 1) * H].T @ np.diag(cg[0])
+        return M
+
+    Nc = T // cf
+    A = np.eye(Nc * H)
+    Bm = np.eye(Nc * H)
+    for k in range(1, Nc + 1):             # coarse reversed point k; fine reversed points cf(k-1)+1 .. cf k
+        prod = np.eye(H)
+        for s in range(cf * (k - 1) + 1, cf * k + 1):
+            prod = step_matrix(T - s + 1, 1) @ prod
+        Mc = step_matrix(Nc - k + 1, cf)
+        if k >= 2:
+            A[(k - 1) * H:k * H, (k - 2) * H:(k - 1) * H] = -prod
+            Bm[(k - 1) * H:k * H, (k - 2) * H:(k - 1) * H] = -Mc
+    lam_s, lam0_s, _ = O.serial_backward(*P, x, h0, h, seed)
+    mu_exact = np.concatenate([lam_s[::-1], lam0_s[None]], 0)          # mu_0 .. mu_T
+    e0 = -np.concatenate([mu_exact[cf * k, 0] for k in range(1, Nc + 1)])   # zero initial guess
+    E = np.eye(Nc * H) - np.linalg.solve(Bm, A)
+    if relax == O.RELAX_FCF:
+        E = E @ (np.eye(Nc * H) - A)
+    lam, lam0, _, _ = O.mgrit_adjoint(*P, x, h0, h, seed, cf=cf, levels=2, iters=1, relax_fine=relax)
+    mu = np.concatenate([lam[::-1], lam0[None]], 0)
+    e1 = np.concatenate([(mu - mu_exact)[cf * k, 0] for k in range(1, Nc + 1)])
+    assert np.max(np.abs(e1 - E @ e0)) < 1e-13 * max(1.0, np.max(np.abs(e0)))
+    assert np.max(np.abs(e1)) > 1e-9       # the check is not vacuous
+
+
+def test_toy_ode_two_level_convergence_shape():
+    # Supplementary demo: two-level MGRIT on  h' = -h/2 + sigmoid(A h + B d + b), dimension 10,
+    # 128 steps.  The printed run (golden file) loses 1.5-2.3 decades of error per cycle and
+    # reaches rounding in 8 cycles with residual and error of similar size; weights are random,
+    # so only that shape is pinned.  Reading (the demo's discretisation is not given): step 0.1 on the
+    # fine grid, decay term implicit, FCF relaxation, c_f = 4.
+    rows = [l.split() for l in open(os.path.join(GOLDEN, "toy_ode_two_level.txt")) if not l.startswith("#")]
+    paper_err = np.array([float(r[0]) for r in rows]); paper_res = np.array([float(r[1]) for r in rows])
+    paper_rate = np.log10(paper_err[0] / paper_err[-1]) / (len(paper_err) - 1)
+    rng = np.random.default_rng(0)
+    n, T, cf = 10, 128, 4
+    Am = rng.standard_normal((n, n)) / np.sqrt(n); Bd = rng.standard_normal((n, n)) / np.sqrt(n)
+    b = rng.standard_normal(n); d = rng.standard_normal((T + 1, n))
+
+    def step(l, j, up):
+        dtl = 0.1 * float(cf ** l)
+        dj = d[(cf ** l) * j]
+        # implicit treatment of the linear decay keeps the coarse level stable
+        return (up + dtl * O.sigmoid(up @ Am.T + dj @ Bd.T + b)) / (1 + 0.5 * dtl)
+
+    exact = np.zeros((T + 1, n))
+    for j in range(1, T + 1):
+        exact[j] = step(0, np.array([j]), exact[j - 1:j])[0]
+    u = [np.zeros((T + 1, n)), None]; g = [np.zeros((T + 1, n)), None]
+    errs, ress = [], []
+    for _ in range(8):
+        res = []
+        O.fas_vcycle(step, [T, T // cf], cf, [O.RELAX_FCF, O.RELAX_FCF], u, g, 0, res)
+        ress.append(res[0]); errs.append(np.max(np.abs(u[0] - exact)))
+    rate = np.log10(errs[0] / max(errs[-1], 1e-16)) / 7
+    assert errs[-1] < 1e-10 and rate > 0.6 * paper_rate
+    assert all(b_ < a_ for a_, b_ in zip(errs, errs[1:]) if a_ > 1e-13)
+    # residual and error of similar size, as in the printed run (ratio ~0.7)
+    assert 0.05 < paper_res[0] / paper_err[0] < 2
