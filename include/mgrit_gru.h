@@ -1,0 +1,152 @@
+/* mgrit_gru.h -- C ABI of the B200 (sm_100a) MGRIT solver for the GRU hidden-state recurrence.
+ *
+ * The library implements, as CUDA kernels only (there is no CPU fallback), the parallel-in-time
+ * training path of "Parallel Training of GRU Networks with a Multi-Grid Solver for Long
+ * Sequences": the input projection, the multigrid-reduction-in-time (MGRIT) cycle for the
+ * forward recurrence h_t = Phi(x_t, h_{t-1}) and for its adjoint, the time-parallel weight
+ * gradients, a classifier/loss head, the SGD update, and the exact serial sweep it converges to.
+ *
+ * Conventions
+ *  - Every data pointer is a DEVICE pointer owned by the caller, 16-byte aligned, fp32, row-major,
+ *    time-major: x[T,B,I], gi[T,B,3H], h[T,B,H]; h[k] is the paper's h_{k+1}, h_0 is passed
+ *    separately.  Gate order along 3H is r | z | n (Eq. "gru").
+ *  - cfg, resnorm and the size outputs are HOST pointers.
+ *  - The library never allocates or frees device memory: scratch is a caller-provided workspace
+ *    (device, 256-byte aligned) of at least the size reported by mgrit_gru_workspace_bytes().
+ *  - Calls enqueue work on `stream` and return without synchronising, except that a non-NULL
+ *    `resnorm` makes the call synchronise the stream before it returns.
+ *  - Return value: MGRIT_OK (0) or a negative error code; outputs are undefined after an error.
+ *    Nothing aborts the process.  Device-side waits are bounded: a wait that runs out makes the
+ *    next synchronising call (or mgrit_gru_last_device_status) report MGRIT_DEVICE_TIMEOUT.
+ *  - One GPU, the current device.  Calls that share a workspace must not overlap on the GPU.
+ */
+#ifndef MGRIT_GRU_H_
+#define MGRIT_GRU_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef struct CUstream_st* mgrit_stream_t; /* a cudaStream_t */
+
+enum {
+  MGRIT_OK = 0,
+  MGRIT_INVALID_ARG = -1,        /* NULL pointer, non-positive size, unknown enum value */
+  MGRIT_NOT_DIVISIBLE = -2,      /* T is not a multiple of cf^(levels-1) */
+  MGRIT_WORKSPACE_TOO_SMALL = -3,
+  MGRIT_UNSUPPORTED = -4,        /* shape outside what the selected operand mode supports */
+  MGRIT_CUDA_ERROR = -5,         /* a CUDA runtime/driver call failed */
+  MGRIT_DEVICE_TIMEOUT = -6      /* a bounded device-side wait ran out */
+};
+
+enum { MGRIT_CELL_CLASSIC = 0, MGRIT_CELL_IMPLICIT = 1 };
+enum { MGRIT_RELAX_F = 0, MGRIT_RELAX_FCF = 1 };
+enum { MGRIT_OPERANDS_FP32 = 0, MGRIT_OPERANDS_BF16 = 2 };
+enum { MGRIT_FLAG_SKIP_DUPLICATE_FRELAX = 1 };
+
+/* Problem and cycle description (Algorithm "MGProp", remark "Beyond Two-Level", Section
+ * "Coarse Grid Propagators").  Level l has N_l = T / cf^l points and time step cf^l * dt. */
+typedef struct {
+  int32_t T, B, I, H;   /* sequence length, batch, input width, hidden width; H % 8 == 0, I % 8 == 0 */
+  int32_t cf;           /* coarsening factor c_f >= 2 */
+  int32_t levels;       /* >= 1; 1 = plain serial sweep; needs T % cf^(levels-1) == 0 */
+  int32_t iters;        /* number of MGRIT cycles (ForwardIters / BackwardIters of Algorithm "MGRITTraining") */
+  int32_t cell;         /* MGRIT_CELL_CLASSIC: Eq. "gru-classic"; MGRIT_CELL_IMPLICIT: Eq. "gru-imap"; same on all levels */
+  int32_t relax_fine;   /* relaxation on level 0: MGRIT_RELAX_F or MGRIT_RELAX_FCF (Eq. "fcf-relax") */
+  int32_t relax_coarse; /* relaxation on levels 1 .. levels-2 */
+  int32_t operands;     /* MGRIT_OPERANDS_FP32: FFMA everywhere; MGRIT_OPERANDS_BF16: bf16 tensor-core
+                           operands with fp32 accumulation; states, gates and gradients stay fp32 */
+  int32_t flags;        /* MGRIT_FLAG_SKIP_DUPLICATE_FRELAX: a cycle after the first starts from C-points
+                           whose F-points the previous cycle's final F-relaxation already filled; skip
+                           re-doing it (results are identical) */
+  float dt;             /* fine time step (1.0 in every experiment of the paper) */
+} mgrit_gru_cfg;
+
+/* GRU parameters of Eq. "gru", PyTorch layout: rows r | z | n. */
+typedef struct {
+  const float* W_ih; /* [3H, I] */
+  const float* W_hh; /* [3H, H] */
+  const float* b_ih; /* [3H] */
+  const float* b_hh; /* [3H] */
+} gru_params;
+
+/* Parameter gradients; overwritten, not accumulated. */
+typedef struct {
+  float* dW_ih; /* [3H, I] */
+  float* dW_hh; /* [3H, H] */
+  float* db_ih; /* [3H] */
+  float* db_hh; /* [3H] */
+} gru_grads;
+
+/* Workspace sizes in bytes for this cfg.  fwd_bytes serves gru_input_projection,
+ * mgrit_gru_forward and gru_serial_forward; adj_bytes serves mgrit_gru_adjoint and
+ * gru_serial_backward.  Either output may be NULL. */
+int mgrit_gru_workspace_bytes(const mgrit_gru_cfg* cfg, size_t* fwd_bytes, size_t* adj_bytes);
+
+/* gi[t] = W_ih x_t + b_ih for all t (input half of Eq. "gru"); computed once on the fine grid
+ * and reused by every level and by the adjoint.  x[T,B,I] -> gi[T,B,3H]. */
+int gru_input_projection(const mgrit_gru_cfg* cfg, const gru_params* p, const float* x, float* gi,
+                         void* ws, size_t ws_bytes, mgrit_stream_t stream);
+
+/* Forward propagation by cfg->iters MGRIT cycles from the zero initial guess (Algorithm
+ * "MGRITTraining", forward block; Algorithm "MGProp"): relaxation, residual restriction,
+ * FAS coarse equation, recursive / serial coarse solve, correction, final F-relaxation.
+ *   x[T,B,I], h0[B,H]  -> gi[T,B,3H] (written: the projection, kept for the adjoint), h[T,B,H].
+ *   resnorm: HOST array of cfg->iters floats or NULL; entry i = 2-norm of the level-0 C-point
+ *   residual measured in cycle i after its pre-relaxation.  levels == 1 runs the serial sweep. */
+int mgrit_gru_forward(const mgrit_gru_cfg* cfg, const gru_params* p, const float* x, const float* h0,
+                      float* gi, float* h, float* resnorm, void* ws, size_t ws_bytes,
+                      mgrit_stream_t stream);
+
+/* Backward propagation by cfg->iters MGRIT cycles on the adjoint recurrence, time reversed
+ * (Algorithm "MGRITTraining", backward block; Appendix "Training With MGRIT"), linearised at the
+ * GIVEN states h (the possibly inexact forward result), followed by the time-parallel gradient
+ * pass g_i = w_i dh_i/dTheta.
+ *   dh_seed[T,B,H] or NULL: direct loss derivative w.r.t. every h_t (stacked layers);
+ *   dhT[B,H] or NULL: direct loss derivative w.r.t. h_T, added to dh_seed[T-1]; one of the two
+ *   must be given.  Outputs: dh[T,B,H] total dL/dh_t, dh0[B,H], dx[T,B,I] or NULL, grads.
+ *   gi is the projection written by the forward call for the same x and parameters. */
+int mgrit_gru_adjoint(const mgrit_gru_cfg* cfg, const gru_params* p, const float* x, const float* h0,
+                      const float* gi, const float* h, const float* dh_seed, const float* dhT,
+                      float* dh, float* dh0, float* dx, const gru_grads* grads, float* resnorm,
+                      void* ws, size_t ws_bytes, mgrit_stream_t stream);
+
+/* Exact serial sweep h_t = Phi_dt(x_t, h_{t-1}), t = 1..T (the solution of Eq. "fine-res"), with
+ * the same cell as level 0 of the MGRIT solve; also writes gi. cf/levels/iters are ignored. */
+int gru_serial_forward(const mgrit_gru_cfg* cfg, const gru_params* p, const float* x, const float* h0,
+                       float* gi, float* h, void* ws, size_t ws_bytes, mgrit_stream_t stream);
+
+/* Exact back-propagation through time for the serial sweep; arguments as mgrit_gru_adjoint. */
+int gru_serial_backward(const mgrit_gru_cfg* cfg, const gru_params* p, const float* x, const float* h0,
+                        const float* gi, const float* h, const float* dh_seed, const float* dhT,
+                        float* dh, float* dh0, float* dx, const gru_grads* grads,
+                        void* ws, size_t ws_bytes, mgrit_stream_t stream);
+
+/* Classifier head on h_T with mean softmax cross-entropy (the loss whose gradient seeds the
+ * backward block: w_T = grad_{h_T} L).  hT[B,H], Wc[C,H], bc[C], labels[B] (int32, device)
+ * -> loss[1] (device), dhT[B,H], dWc[C,H], dbc[C].  ws: device scratch of at least
+ * xent_head_workspace_bytes(B, C) bytes. */
+size_t xent_head_workspace_bytes(int32_t B, int32_t C);
+int xent_head_fwd_bwd(int32_t B, int32_t H, int32_t C, const float* hT, const float* Wc, const float* bc,
+                      const int32_t* labels, float* loss, float* dhT, float* dWc, float* dbc,
+                      void* ws, size_t ws_bytes, mgrit_stream_t stream);
+
+/* Theta <- Theta - lr * g (last line of Algorithm "MGRITTraining"); n fp32 elements. */
+int sgd_update(float* p, const float* g, size_t n, float lr, mgrit_stream_t stream);
+
+/* Status word written by bounded device-side waits since the library was loaded (0 = none ran out).
+ * Synchronises the device. */
+int mgrit_gru_last_device_status(void);
+
+/* Number of kernels this library has launched since it was loaded (all streams). */
+unsigned long long mgrit_gru_kernel_launches(void);
+
+const char* mgrit_gru_strerror(int code);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* MGRIT_GRU_H_ */

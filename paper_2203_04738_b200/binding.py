@@ -1,0 +1,205 @@
+"""Thin ctypes binding of the C ABI in include/mgrit_gru.h: argument marshalling only.
+
+Tensors are torch CUDA tensors (fp32, contiguous); outputs and the workspace are allocated with
+torch; work is enqueued on torch's current stream.  Every step of the path runs in the
+library's kernels -- if the library has not been built, importing this module raises.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+from dataclasses import dataclass
+
+import torch
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_HERE, "libmgrit_gru.so")
+if not os.path.exists(LIB_PATH):
+    raise ImportError(f"{LIB_PATH} is missing: build it with `python -m paper_2203_04738_b200.build` "
+                      "(there is no CPU or PyTorch fallback)")
+lib = ctypes.CDLL(LIB_PATH)
+
+OK = 0
+CELL_CLASSIC, CELL_IMPLICIT = 0, 1
+RELAX_F, RELAX_FCF = 0, 1
+OPERANDS_FP32, OPERANDS_BF16 = 0, 2
+FLAG_SKIP_DUPLICATE_FRELAX = 1
+
+
+class Cfg(ctypes.Structure):
+    _fields_ = [(n, ctypes.c_int32) for n in
+                ("T", "B", "I", "H", "cf", "levels", "iters", "cell", "relax_fine", "relax_coarse", "operands", "flags")] + \
+               [("dt", ctypes.c_float)]
+
+
+class _Params(ctypes.Structure):
+    _fields_ = [(n, ctypes.c_void_p) for n in ("W_ih", "W_hh", "b_ih", "b_hh")]
+
+
+class _Grads(ctypes.Structure):
+    _fields_ = [(n, ctypes.c_void_p) for n in ("dW_ih", "dW_hh", "db_ih", "db_hh")]
+
+
+_vp, _sz, _i32 = ctypes.c_void_p, ctypes.c_size_t, ctypes.c_int32
+lib.mgrit_gru_workspace_bytes.argtypes = [ctypes.POINTER(Cfg), ctypes.POINTER(_sz), ctypes.POINTER(_sz)]
+lib.gru_input_projection.argtypes = [ctypes.POINTER(Cfg), ctypes.POINTER(_Params), _vp, _vp, _vp, _sz, _vp]
+lib.mgrit_gru_forward.argtypes = [ctypes.POINTER(Cfg), ctypes.POINTER(_Params), _vp, _vp, _vp, _vp,
+                                  ctypes.POINTER(ctypes.c_float), _vp, _sz, _vp]
+lib.gru_serial_forward.argtypes = [ctypes.POINTER(Cfg), ctypes.POINTER(_Params), _vp, _vp, _vp, _vp, _vp, _sz, _vp]
+lib.mgrit_gru_adjoint.argtypes = [ctypes.POINTER(Cfg), ctypes.POINTER(_Params), _vp, _vp, _vp, _vp, _vp, _vp, _vp, _vp, _vp,
+                                  ctypes.POINTER(_Grads), ctypes.POINTER(ctypes.c_float), _vp, _sz, _vp]
+lib.gru_serial_backward.argtypes = [ctypes.POINTER(Cfg), ctypes.POINTER(_Params), _vp, _vp, _vp, _vp, _vp, _vp, _vp, _vp, _vp,
+                                    ctypes.POINTER(_Grads), _vp, _sz, _vp]
+lib.xent_head_workspace_bytes.argtypes = [_i32, _i32]
+lib.xent_head_workspace_bytes.restype = _sz
+lib.xent_head_fwd_bwd.argtypes = [_i32, _i32, _i32, _vp, _vp, _vp, _vp, _vp, _vp, _vp, _vp, _vp, _sz, _vp]
+lib.sgd_update.argtypes = [_vp, _vp, _sz, ctypes.c_float, _vp]
+lib.mgrit_gru_last_device_status.restype = ctypes.c_int
+lib.mgrit_gru_kernel_launches.restype = ctypes.c_ulonglong
+lib.mgrit_gru_strerror.argtypes = [ctypes.c_int]
+lib.mgrit_gru_strerror.restype = ctypes.c_char_p
+
+
+class MgritError(RuntimeError):
+    def __init__(self, code):
+        self.code = code
+        super().__init__(f"mgrit_gru error {code}: {lib.mgrit_gru_strerror(code).decode()}")
+
+
+def _check(rc):
+    if rc != OK:
+        raise MgritError(rc)
+
+
+def make_cfg(T, B, I, H, cf=4, levels=2, iters=2, cell=CELL_IMPLICIT, relax_fine=RELAX_F, relax_coarse=RELAX_FCF,
+             operands=OPERANDS_FP32, flags=0, dt=1.0) -> Cfg:
+    return Cfg(T, B, I, H, cf, levels, iters, cell, relax_fine, relax_coarse, operands, flags, dt)
+
+
+def _ptr(t):
+    if t is None:
+        return None
+    assert t.is_cuda and t.is_contiguous(), "CUDA contiguous tensor required"
+    return ctypes.c_void_p(t.data_ptr())
+
+
+def _f32(t):
+    assert t is None or t.dtype == torch.float32
+    return _ptr(t)
+
+
+def _stream():
+    return ctypes.c_void_p(torch.cuda.current_stream().cuda_stream)
+
+
+def _params(p):
+    return _Params(*[p[n].data_ptr() for n in ("W_ih", "W_hh", "b_ih", "b_hh")])
+
+
+def workspace_bytes(cfg: Cfg):
+    f, a = _sz(0), _sz(0)
+    _check(lib.mgrit_gru_workspace_bytes(ctypes.byref(cfg), ctypes.byref(f), ctypes.byref(a)))
+    return f.value, a.value
+
+
+def _ws(nbytes, ws, dev):
+    if ws is None or ws.numel() < nbytes:
+        ws = torch.empty(nbytes, dtype=torch.uint8, device=dev)
+    return ws
+
+
+def gru_input_projection(cfg, p, x, gi=None, ws=None):
+    gi = torch.empty(cfg.T, cfg.B, 3 * cfg.H, device=x.device) if gi is None else gi
+    ws = _ws(workspace_bytes(cfg)[0], ws, x.device)
+    _check(lib.gru_input_projection(ctypes.byref(cfg), ctypes.byref(_params(p)), _f32(x), _f32(gi), _ptr(ws), ws.numel(), _stream()))
+    return gi
+
+
+def mgrit_gru_forward(cfg, p, x, h0, want_resnorm=False, gi=None, h=None, ws=None):
+    """-> (h[T,B,H], gi[T,B,3H], resnorm list or None)"""
+    dev = x.device
+    gi = torch.empty(cfg.T, cfg.B, 3 * cfg.H, device=dev) if gi is None else gi
+    h = torch.empty(cfg.T, cfg.B, cfg.H, device=dev) if h is None else h
+    ws = _ws(workspace_bytes(cfg)[0], ws, dev)
+    rn = (ctypes.c_float * max(cfg.iters, 1))() if want_resnorm else None
+    _check(lib.mgrit_gru_forward(ctypes.byref(cfg), ctypes.byref(_params(p)), _f32(x), _f32(h0), _f32(gi), _f32(h), rn,
+                                 _ptr(ws), ws.numel(), _stream()))
+    return h, gi, (list(rn)[:cfg.iters] if want_resnorm else None)
+
+
+def gru_serial_forward(cfg, p, x, h0, gi=None, h=None, ws=None):
+    dev = x.device
+    gi = torch.empty(cfg.T, cfg.B, 3 * cfg.H, device=dev) if gi is None else gi
+    h = torch.empty(cfg.T, cfg.B, cfg.H, device=dev) if h is None else h
+    ws = _ws(workspace_bytes(cfg)[0], ws, dev)
+    _check(lib.gru_serial_forward(ctypes.byref(cfg), ctypes.byref(_params(p)), _f32(x), _f32(h0), _f32(gi), _f32(h),
+                                  _ptr(ws), ws.numel(), _stream()))
+    return h, gi
+
+
+@dataclass
+class AdjointResult:
+    dh: torch.Tensor
+    dh0: torch.Tensor
+    dx: torch.Tensor | None
+    dW_ih: torch.Tensor
+    dW_hh: torch.Tensor
+    db_ih: torch.Tensor
+    db_hh: torch.Tensor
+    resnorm: list | None = None
+
+
+def _adjoint(fn, serial, cfg, p, x, h0, gi, h, dh_seed, dhT, want_dx, want_resnorm, ws, out):
+    dev = x.device
+    o = out or AdjointResult(
+        dh=torch.empty(cfg.T, cfg.B, cfg.H, device=dev), dh0=torch.empty(cfg.B, cfg.H, device=dev),
+        dx=torch.empty(cfg.T, cfg.B, cfg.I, device=dev) if want_dx else None,
+        dW_ih=torch.empty(3 * cfg.H, cfg.I, device=dev), dW_hh=torch.empty(3 * cfg.H, cfg.H, device=dev),
+        db_ih=torch.empty(3 * cfg.H, device=dev), db_hh=torch.empty(3 * cfg.H, device=dev))
+    ws = _ws(workspace_bytes(cfg)[1], ws, dev)
+    g = _Grads(o.dW_ih.data_ptr(), o.dW_hh.data_ptr(), o.db_ih.data_ptr(), o.db_hh.data_ptr())
+    args = [ctypes.byref(cfg), ctypes.byref(_params(p)), _f32(x), _f32(h0), _f32(gi), _f32(h), _f32(dh_seed), _f32(dhT),
+            _f32(o.dh), _f32(o.dh0), _f32(o.dx), ctypes.byref(g)]
+    if not serial:
+        rn = (ctypes.c_float * max(cfg.iters, 1))() if want_resnorm else None
+        args.append(rn)
+    args += [_ptr(ws), ws.numel(), _stream()]
+    _check(fn(*args))
+    if not serial and want_resnorm:
+        o.resnorm = list(rn)[:cfg.iters]
+    return o
+
+
+def mgrit_gru_adjoint(cfg, p, x, h0, gi, h, dh_seed=None, dhT=None, want_dx=True, want_resnorm=False, ws=None, out=None):
+    return _adjoint(lib.mgrit_gru_adjoint, False, cfg, p, x, h0, gi, h, dh_seed, dhT, want_dx, want_resnorm, ws, out)
+
+
+def gru_serial_backward(cfg, p, x, h0, gi, h, dh_seed=None, dhT=None, want_dx=True, ws=None, out=None):
+    return _adjoint(lib.gru_serial_backward, True, cfg, p, x, h0, gi, h, dh_seed, dhT, want_dx, False, ws, out)
+
+
+def xent_head_fwd_bwd(hT, Wc, bc, labels, ws=None):
+    """-> (loss[1], dhT[B,H], dWc[C,H], dbc[C]) device tensors"""
+    B, H = hT.shape
+    C = Wc.shape[0]
+    dev = hT.device
+    assert labels.dtype == torch.int32
+    loss = torch.empty(1, device=dev)
+    dhT, dWc, dbc = torch.empty(B, H, device=dev), torch.empty(C, H, device=dev), torch.empty(C, device=dev)
+    ws = _ws(lib.xent_head_workspace_bytes(B, C), ws, dev)
+    _check(lib.xent_head_fwd_bwd(B, H, C, _f32(hT), _f32(Wc), _f32(bc), _ptr(labels), _f32(loss), _f32(dhT), _f32(dWc),
+                                 _f32(dbc), _ptr(ws), ws.numel(), _stream()))
+    return loss, dhT, dWc, dbc
+
+
+def sgd_update(p, g, lr):
+    _check(lib.sgd_update(_f32(p), _f32(g), p.numel(), ctypes.c_float(lr), _stream()))
+    return p
+
+
+def last_device_status() -> int:
+    return lib.mgrit_gru_last_device_status()
+
+
+def kernel_launches() -> int:
+    return int(lib.mgrit_gru_kernel_launches())

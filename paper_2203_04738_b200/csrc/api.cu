@@ -1,0 +1,437 @@
+// C ABI, argument validation, workspace layout and the host side of the multigrid cycle.
+// The cycle logic is written once over an abstract "step" and instantiated for the forward
+// recurrence and for its adjoint; every step, transfer and reduction is a kernel launch.
+#include <math.h>
+#include <stdio.h>
+#include <string.h>
+
+#include "common.cuh"
+#include "umma_engine.cuh"
+
+namespace mg {
+
+unsigned long long g_kernel_launches = 0;
+
+namespace {
+
+constexpr int kMaxLevels = 16;
+
+struct Ws {  // bump allocator over the caller's workspace; base == nullptr only counts bytes
+  char* base; size_t size; size_t off;
+  template <class T> T* take(size_t n) {
+    size_t bytes = (n * sizeof(T) + 255) & ~(size_t)255;
+    T* p = base ? reinterpret_cast<T*>(base + off) : nullptr;
+    off += bytes;
+    return p;
+  }
+  bool fits() const { return base == nullptr || off <= size; }
+};
+
+struct Hier {
+  int L; int N[kMaxLevels]; i64 stride_t[kMaxLevels]; float gamma[kMaxLevels];
+};
+
+int check_cfg(const mgrit_gru_cfg* c, Hier* hr) {
+  if (!c) return MGRIT_INVALID_ARG;
+  if (c->T <= 0 || c->B <= 0 || c->I <= 0 || c->H <= 0 || c->levels < 1 || c->levels > kMaxLevels) return MGRIT_INVALID_ARG;
+  if (c->levels > 1 && (c->cf < 2 || c->iters < 0)) return MGRIT_INVALID_ARG;
+  if (c->cell != MGRIT_CELL_CLASSIC && c->cell != MGRIT_CELL_IMPLICIT) return MGRIT_INVALID_ARG;
+  if (c->relax_fine != MGRIT_RELAX_F && c->relax_fine != MGRIT_RELAX_FCF) return MGRIT_INVALID_ARG;
+  if (c->relax_coarse != MGRIT_RELAX_F && c->relax_coarse != MGRIT_RELAX_FCF) return MGRIT_INVALID_ARG;
+  if (c->operands != MGRIT_OPERANDS_FP32 && c->operands != MGRIT_OPERANDS_BF16) return MGRIT_INVALID_ARG;
+  if (!(c->dt > 0.f)) return MGRIT_INVALID_ARG;
+  if (c->H % 8 != 0 || c->I % 8 != 0) return MGRIT_UNSUPPORTED;
+  i64 m = 1;
+  hr->L = c->levels;
+  for (int l = 0; l < c->levels; ++l) {
+    if (c->T % m != 0) return MGRIT_NOT_DIVISIBLE;
+    hr->N[l] = (int)(c->T / m);
+    hr->stride_t[l] = m;
+    hr->gamma[l] = (float)m * c->dt;
+    if (l + 1 < c->levels) {
+      m *= c->cf;
+      if (m > c->T) return MGRIT_NOT_DIVISIBLE;
+    }
+  }
+  if (c->operands == MGRIT_OPERANDS_BF16) {
+    int rc = umma_supported(c);
+    if (rc != MGRIT_OK) return rc;
+  }
+  return MGRIT_OK;
+}
+
+struct FwdWs {
+  float* U[kMaxLevels]; float* G[kMaxLevels]; double* res_acc; UmmaFwdWs um;
+};
+struct AdjWs {
+  float* U[kMaxLevels]; float* G[kMaxLevels];
+  float *a[kMaxLevels], *cr[kMaxLevels], *cz[kMaxLevels], *cn[kMaxLevels], *cnp;
+  float *dA_h, *dA_i; double* res_acc; UmmaAdjWs um;
+};
+
+void plan_fwd(const mgrit_gru_cfg* c, const Hier& hr, Ws& w, FwdWs* o) {
+  size_t BH = (size_t)c->B * c->H;
+  for (int l = 0; l < hr.L; ++l) {
+    o->U[l] = w.take<float>((size_t)(hr.N[l] + 1) * BH);
+    o->G[l] = l == 0 ? nullptr : w.take<float>((size_t)(hr.N[l] + 1) * BH);
+  }
+  o->res_acc = w.take<double>((size_t)(c->iters > 0 ? c->iters : 1));
+  if (c->operands == MGRIT_OPERANDS_BF16) umma_plan_fwd(c, hr.N, hr.L, w.base, &w.off, &o->um);
+}
+
+void plan_adj(const mgrit_gru_cfg* c, const Hier& hr, Ws& w, AdjWs* o) {
+  size_t BH = (size_t)c->B * c->H;
+  for (int l = 0; l < hr.L; ++l) {
+    o->U[l] = w.take<float>((size_t)(hr.N[l] + 1) * BH);
+    o->G[l] = w.take<float>((size_t)(hr.N[l] + 1) * BH);
+    o->a[l] = w.take<float>((size_t)hr.N[l] * BH);
+    o->cr[l] = w.take<float>((size_t)hr.N[l] * BH);
+    o->cz[l] = w.take<float>((size_t)hr.N[l] * BH);
+    o->cn[l] = w.take<float>((size_t)hr.N[l] * BH);
+  }
+  o->cnp = w.take<float>((size_t)hr.N[0] * BH);
+  o->res_acc = w.take<double>((size_t)(c->iters > 0 ? c->iters : 1));
+  if (c->operands == MGRIT_OPERANDS_BF16) {
+    o->dA_h = o->dA_i = nullptr;
+    umma_plan_adj(c, hr.N, hr.L, w.base, &w.off, &o->um);
+  } else {
+    o->dA_h = w.take<float>((size_t)c->T * BH * 3);
+    o->dA_i = w.take<float>((size_t)c->T * BH * 3);
+  }
+}
+
+// One launch of "advance nk*B rows by one step of level l".
+struct StepDesc {
+  int l, nk;
+  int in_slot, in_stride;                 // source slots in U[l]
+  float* out; int out_slot, out_stride;   // destination array (slot-major [.,B,H]) and slots
+  const float* gadd; int gadd_slot, gadd_stride;
+  int tgt_slot, tgt_stride;               // level-l point the step arrives at (selects input / coefficients)
+  int mode;
+};
+
+// The multigrid cycle (Algorithm "MGProp" with the recursive coarse solve of the remark
+// "Beyond Two-Level"), FAS form: level l solves u_j = step_l(u_{j-1}) + g_j.
+struct Cycle {
+  const mgrit_gru_cfg* c; Hier hr; cudaStream_t s;
+  float** U; float** G; double* res_acc; int cycle_idx = 0;
+  size_t BH;
+  virtual void step(const StepDesc& d) = 0;
+  virtual ~Cycle() {}
+
+  void frelax(int l) {
+    int cf = c->cf, nki = hr.N[l] / cf;
+    for (int sI = 1; sI < cf; ++sI)
+      step(StepDesc{l, nki, sI - 1, cf, U[l], sI, cf, G[l], sI, cf, sI, cf, 0});
+  }
+  void crelax(int l) {
+    int cf = c->cf, nki = hr.N[l] / cf;
+    step(StepDesc{l, nki, cf - 1, cf, U[l], cf, cf, G[l], cf, cf, cf, cf, 0});
+  }
+  void vcycle(int l) {
+    int cf = c->cf, N = hr.N[l];
+    if (l == hr.L - 1) {  // coarsest level: serial propagation
+      for (int j = 1; j <= N; ++j) step(StepDesc{l, 1, j - 1, 1, U[l], j, 1, G[l], j, 1, j, 1, 0});
+      return;
+    }
+    int relax = l == 0 ? c->relax_fine : c->relax_coarse;
+    bool dup = l == 0 && cycle_idx > 0 && (c->flags & MGRIT_FLAG_SKIP_DUPLICATE_FRELAX);
+    if (!dup) frelax(l);
+    if (relax == MGRIT_RELAX_FCF) { crelax(l); frelax(l); }
+    int nc = N / cf;
+    // v_k = step_l(u_{cf k - 1}) + g_{cf k}  ->  G[l+1][k]
+    step(StepDesc{l, nc, cf - 1, cf, G[l + 1], 1, 1, G[l], cf, cf, cf, cf, 0});
+    // r_k = u_{cf k} - v_k ; U'_k = u_{cf k}
+    stream_restrict_residual(U[l], cf, G[l + 1], U[l + 1], nc, (i64)BH, l == 0 ? res_acc + cycle_idx : nullptr, s);
+    // G_k = v_k - step_{l+1}(U'_{k-1})
+    step(StepDesc{l + 1, nc, 0, 1, G[l + 1], 1, 1, nullptr, 0, 0, 1, 1, 1});
+    vcycle(l + 1);
+    stream_correct(U[l], cf, U[l + 1], nc, (i64)BH, s);
+    frelax(l);
+  }
+  void solve() {
+    if (hr.L == 1) { vcycle(0); return; }
+    cudaMemsetAsync(res_acc, 0, sizeof(double) * (size_t)(c->iters > 0 ? c->iters : 1), s);
+    for (cycle_idx = 0; cycle_idx < c->iters; ++cycle_idx) vcycle(0);
+  }
+};
+
+struct FwdCycle : Cycle {
+  const gru_params* p; const float* gi; UmmaFwdWs* um;
+  void step(const StepDesc& d) override {
+    FwdStepArgs a;
+    a.M = d.nk * c->B; a.B = c->B; a.H = c->H;
+    a.hin = U[d.l] + (size_t)d.in_slot * BH; a.hin_ks = (i64)d.in_stride * BH;
+    a.hout = d.out + (size_t)d.out_slot * BH; a.hout_ks = (i64)d.out_stride * BH;
+    i64 st = hr.stride_t[d.l];
+    a.gi = gi + ((i64)st * d.tgt_slot - 1) * (i64)BH * 3; a.gi_ks = st * d.tgt_stride * (i64)BH * 3;
+    a.gadd = d.gadd ? d.gadd + (size_t)d.gadd_slot * BH : nullptr; a.gadd_ks = (i64)d.gadd_stride * BH;
+    a.W_hh = p->W_hh; a.b_hh = p->b_hh; a.gamma = hr.gamma[d.l]; a.cell = c->cell; a.mode = d.mode;
+    if (c->operands == MGRIT_OPERANDS_BF16) umma_fwd_step(a, um, s); else simt_fwd_step(a, s);
+  }
+};
+
+struct AdjCycle : Cycle {
+  const gru_params* p; AdjWs* w;
+  void step(const StepDesc& d) override {
+    AdjStepArgs a;
+    a.M = d.nk * c->B; a.B = c->B; a.H = c->H;
+    a.lin = U[d.l] + (size_t)d.in_slot * BH; a.lin_ks = (i64)d.in_stride * BH;
+    a.lout = d.out + (size_t)d.out_slot * BH; a.lout_ks = (i64)d.out_stride * BH;
+    a.gadd = d.gadd ? d.gadd + (size_t)d.gadd_slot * BH : nullptr; a.gadd_ks = (i64)d.gadd_stride * BH;
+    // the step arriving at reversed point s applies forward step j = N_l - s + 1, stored at row N_l - s
+    i64 row0 = (i64)(hr.N[d.l] - d.tgt_slot) * BH;
+    a.a = w->a[d.l] + row0; a.cr = w->cr[d.l] + row0; a.cz = w->cz[d.l] + row0; a.cn = w->cn[d.l] + row0;
+    a.coef_ks = -(i64)d.tgt_stride * BH;
+    a.W_hh = p->W_hh; a.mode = d.mode;
+    if (c->operands == MGRIT_OPERANDS_BF16) umma_adj_step(a, &w->um, s); else simt_adj_step(a, s);
+  }
+};
+
+int finish(cudaStream_t s, bool sync) {
+  if (sync && cudaStreamSynchronize(s) != cudaSuccess) return MGRIT_CUDA_ERROR;
+  cudaError_t e = cudaGetLastError();
+  if (e != cudaSuccess) { fprintf(stderr, "mgrit_gru: CUDA error: %s\n", cudaGetErrorString(e)); return MGRIT_CUDA_ERROR; }
+  if (sync && umma_device_status() != 0) return MGRIT_DEVICE_TIMEOUT;
+  return MGRIT_OK;
+}
+
+int fetch_resnorm(const double* acc, float* resnorm, int iters, cudaStream_t s) {
+  double tmp[64];
+  for (int base = 0; base < iters; base += 64) {
+    int n = iters - base < 64 ? iters - base : 64;
+    if (cudaMemcpyAsync(tmp, acc + base, sizeof(double) * n, cudaMemcpyDeviceToHost, s) != cudaSuccess) return MGRIT_CUDA_ERROR;
+    if (cudaStreamSynchronize(s) != cudaSuccess) return MGRIT_CUDA_ERROR;
+    for (int i = 0; i < n; ++i) resnorm[base + i] = (float)sqrt(tmp[i]);
+  }
+  return MGRIT_OK;
+}
+
+int forward_impl(const mgrit_gru_cfg* cfg_in, bool serial, const gru_params* p, const float* x, const float* h0, float* gi,
+                 float* h, float* resnorm, void* ws, size_t ws_bytes, cudaStream_t s) {
+  if (!cfg_in || !p || !x || !h0 || !gi || !h || !ws || !p->W_ih || !p->W_hh || !p->b_ih || !p->b_hh) return MGRIT_INVALID_ARG;
+  mgrit_gru_cfg c = *cfg_in;
+  if (serial) { c.levels = 1; c.iters = 1; c.cf = 2; }
+  Hier hr;
+  int rc = check_cfg(&c, &hr);
+  if (rc) return rc;
+  Ws w{(char*)ws, ws_bytes, 0};
+  FwdWs fw;
+  plan_fwd(&c, hr, w, &fw);
+  if (!w.fits()) return MGRIT_WORKSPACE_TOO_SMALL;
+  size_t BH = (size_t)c.B * c.H;
+
+  if (c.operands == MGRIT_OPERANDS_BF16) {
+    rc = umma_prepare_fwd(&c, p, x, gi, &fw.um, s);
+    if (rc) return rc;
+  } else {
+    simt_project(x, p->W_ih, p->b_ih, gi, c.T * c.B, c.I, 3 * c.H, s);
+  }
+  cudaMemsetAsync(fw.U[0] + BH, 0, sizeof(float) * (size_t)c.T * BH, s);
+  for (int l = 0; l < hr.L; ++l) cudaMemcpyAsync(fw.U[l], h0, sizeof(float) * BH, cudaMemcpyDeviceToDevice, s);
+
+  FwdCycle cy;
+  cy.c = &c; cy.hr = hr; cy.s = s; cy.U = fw.U; cy.G = fw.G; cy.res_acc = fw.res_acc; cy.BH = BH;
+  cy.p = p; cy.gi = gi; cy.um = &fw.um;
+  cy.solve();
+  cudaMemcpyAsync(h, fw.U[0] + BH, sizeof(float) * (size_t)c.T * BH, cudaMemcpyDeviceToDevice, s);
+  if (resnorm && hr.L > 1 && c.iters > 0) {
+    rc = fetch_resnorm(fw.res_acc, resnorm, c.iters, s);
+    if (rc) return rc;
+    return finish(s, true);
+  }
+  return finish(s, false);
+}
+
+int adjoint_impl(const mgrit_gru_cfg* cfg_in, bool serial, const gru_params* p, const float* x, const float* h0,
+                 const float* gi, const float* h, const float* dh_seed, const float* dhT, float* dh, float* dh0, float* dx,
+                 const gru_grads* g, float* resnorm, void* ws, size_t ws_bytes, cudaStream_t s) {
+  if (!cfg_in || !p || !x || !h0 || !gi || !h || !dh || !dh0 || !g || !ws) return MGRIT_INVALID_ARG;
+  if (!dh_seed && !dhT) return MGRIT_INVALID_ARG;
+  if (!p->W_ih || !p->W_hh || !p->b_ih || !p->b_hh || !g->dW_ih || !g->dW_hh || !g->db_ih || !g->db_hh) return MGRIT_INVALID_ARG;
+  mgrit_gru_cfg c = *cfg_in;
+  if (serial) { c.levels = 1; c.iters = 1; c.cf = 2; }
+  Hier hr;
+  int rc = check_cfg(&c, &hr);
+  if (rc) return rc;
+  Ws w{(char*)ws, ws_bytes, 0};
+  AdjWs aw;
+  plan_adj(&c, hr, w, &aw);
+  if (!w.fits()) return MGRIT_WORKSPACE_TOO_SMALL;
+  size_t BH = (size_t)c.B * c.H;
+  const int T = c.T;
+  const bool bf16 = c.operands == MGRIT_OPERANDS_BF16;
+
+  if (bf16) {
+    rc = umma_prepare_adj(&c, p, &aw.um, s);
+    if (rc) return rc;
+  }
+  // adjoint coefficients of every level's steps at the given states (restricted by injection)
+  for (int l = 0; l < hr.L; ++l) {
+    LinArgs a;
+    a.M = hr.N[l] * c.B; a.B = c.B; a.H = c.H; a.h0 = h0; a.h = h; a.stride_t = hr.stride_t[l]; a.gi = gi;
+    a.W_hh = p->W_hh; a.b_hh = p->b_hh; a.gamma = hr.gamma[l]; a.cell = c.cell;
+    a.a = aw.a[l]; a.cr = aw.cr[l]; a.cz = aw.cz[l]; a.cn = aw.cn[l]; a.cnp = l == 0 ? aw.cnp : nullptr;
+    if (bf16) umma_linearise(a, &aw.um, s); else simt_linearise(a, s);
+  }
+  // mu_0 = lambda_T; zero initial guess elsewhere; fine-level source = reversed dh_seed
+  cudaMemsetAsync(aw.U[0], 0, sizeof(float) * (size_t)(T + 1) * BH, s);
+  if (dh_seed) {
+    cudaMemcpyAsync(aw.U[0], dh_seed + (size_t)(T - 1) * BH, sizeof(float) * BH, cudaMemcpyDeviceToDevice, s);
+    if (dhT) stream_add_rows(aw.U[0], dhT, (i64)BH, s);
+    cudaMemsetAsync(aw.G[0], 0, sizeof(float) * BH, s);
+    cudaMemsetAsync(aw.G[0] + (size_t)T * BH, 0, sizeof(float) * BH, s);
+    if (T > 1) stream_gather_rows(aw.G[0] + BH, (i64)BH, dh_seed + (size_t)(T - 2) * BH, -(i64)BH, T - 1, (i64)BH, s);
+  } else {
+    cudaMemcpyAsync(aw.U[0], dhT, sizeof(float) * BH, cudaMemcpyDeviceToDevice, s);
+  }
+  for (int l = 1; l < hr.L; ++l) cudaMemcpyAsync(aw.U[l], aw.U[0], sizeof(float) * BH, cudaMemcpyDeviceToDevice, s);
+
+  float* Gl[kMaxLevels];
+  for (int l = 0; l < hr.L; ++l) Gl[l] = aw.G[l];
+  if (!dh_seed) Gl[0] = nullptr;
+  AdjCycle cy;
+  cy.c = &c; cy.hr = hr; cy.s = s; cy.U = aw.U; cy.G = Gl; cy.res_acc = aw.res_acc; cy.BH = BH;
+  cy.p = p; cy.w = &aw;
+  cy.solve();
+
+  // dh[k] = lambda_{k+1} = mu_{T-1-k};  dh0 = lambda_0 = mu_T
+  stream_gather_rows(dh, (i64)BH, aw.U[0] + (size_t)(T - 1) * BH, -(i64)BH, T, (i64)BH, s);
+  cudaMemcpyAsync(dh0, aw.U[0] + (size_t)T * BH, sizeof(float) * BH, cudaMemcpyDeviceToDevice, s);
+
+  // gradient pass g = w * dh/dTheta over all fine steps at once
+  if (bf16) {
+    rc = umma_gradients(&c, p, x, h0, h, dh, aw.cr[0], aw.cz[0], aw.cn[0], aw.cnp, dx, g, &aw.um, s);
+    if (rc) return rc;
+  } else {
+    i64 M = (i64)T * c.B;
+    stream_form_dA(dh, aw.cr[0], aw.cz[0], aw.cn[0], aw.cnp, aw.dA_h, aw.dA_i, M, c.H, s);
+    simt_wgrad(aw.dA_h, (int)M, 3 * c.H, h0, c.B, h, c.H, g->dW_hh, s);
+    simt_wgrad(aw.dA_i, (int)M, 3 * c.H, nullptr, 0, x, c.I, g->dW_ih, s);
+    stream_colsum(aw.dA_h, M, 3 * c.H, g->db_hh, s);
+    stream_colsum(aw.dA_i, M, 3 * c.H, g->db_ih, s);
+    if (dx) simt_dgrad(aw.dA_i, (int)M, 3 * c.H, p->W_ih, c.I, dx, s);
+  }
+  if (resnorm && hr.L > 1 && c.iters > 0) {
+    rc = fetch_resnorm(aw.res_acc, resnorm, c.iters, s);
+    if (rc) return rc;
+    return finish(s, true);
+  }
+  return finish(s, false);
+}
+
+}  // namespace
+}  // namespace mg
+
+using namespace mg;
+
+extern "C" {
+
+int mgrit_gru_workspace_bytes(const mgrit_gru_cfg* cfg, size_t* fwd_bytes, size_t* adj_bytes) {
+  Hier hr;
+  int rc = check_cfg(cfg, &hr);
+  if (rc) return rc;
+  // the serial entry points run the same cfg with levels = 1: take the larger of the two plans
+  mgrit_gru_cfg c1 = *cfg; c1.levels = 1; c1.iters = 1; c1.cf = 2;
+  Hier h1;
+  rc = check_cfg(&c1, &h1);
+  if (rc) return rc;
+  if (fwd_bytes) {
+    Ws w{nullptr, 0, 0}; FwdWs f; plan_fwd(cfg, hr, w, &f);
+    Ws w1{nullptr, 0, 0}; FwdWs f1; plan_fwd(&c1, h1, w1, &f1);
+    *fwd_bytes = (w.off > w1.off ? w.off : w1.off) + 256;
+  }
+  if (adj_bytes) {
+    Ws w{nullptr, 0, 0}; AdjWs a; plan_adj(cfg, hr, w, &a);
+    Ws w1{nullptr, 0, 0}; AdjWs a1; plan_adj(&c1, h1, w1, &a1);
+    *adj_bytes = (w.off > w1.off ? w.off : w1.off) + 256;
+  }
+  return MGRIT_OK;
+}
+
+int gru_input_projection(const mgrit_gru_cfg* cfg, const gru_params* p, const float* x, float* gi, void* ws, size_t ws_bytes,
+                         mgrit_stream_t stream) {
+  if (!cfg || !p || !x || !gi || !p->W_ih || !p->b_ih) return MGRIT_INVALID_ARG;
+  Hier hr;
+  int rc = check_cfg(cfg, &hr);
+  if (rc) return rc;
+  cudaStream_t s = (cudaStream_t)stream;
+  if (cfg->operands == MGRIT_OPERANDS_BF16) {
+    if (!ws) return MGRIT_INVALID_ARG;
+    Ws w{(char*)ws, ws_bytes, 0};
+    FwdWs fw;
+    plan_fwd(cfg, hr, w, &fw);
+    if (!w.fits()) return MGRIT_WORKSPACE_TOO_SMALL;
+    rc = umma_prepare_fwd(cfg, p, x, gi, &fw.um, s);
+    if (rc) return rc;
+  } else {
+    simt_project(x, p->W_ih, p->b_ih, gi, cfg->T * cfg->B, cfg->I, 3 * cfg->H, s);
+  }
+  return finish(s, false);
+}
+
+int mgrit_gru_forward(const mgrit_gru_cfg* cfg, const gru_params* p, const float* x, const float* h0, float* gi, float* h,
+                      float* resnorm, void* ws, size_t ws_bytes, mgrit_stream_t stream) {
+  return forward_impl(cfg, false, p, x, h0, gi, h, resnorm, ws, ws_bytes, (cudaStream_t)stream);
+}
+
+int gru_serial_forward(const mgrit_gru_cfg* cfg, const gru_params* p, const float* x, const float* h0, float* gi, float* h,
+                       void* ws, size_t ws_bytes, mgrit_stream_t stream) {
+  return forward_impl(cfg, true, p, x, h0, gi, h, nullptr, ws, ws_bytes, (cudaStream_t)stream);
+}
+
+int mgrit_gru_adjoint(const mgrit_gru_cfg* cfg, const gru_params* p, const float* x, const float* h0, const float* gi,
+                      const float* h, const float* dh_seed, const float* dhT, float* dh, float* dh0, float* dx,
+                      const gru_grads* grads, float* resnorm, void* ws, size_t ws_bytes, mgrit_stream_t stream) {
+  return adjoint_impl(cfg, false, p, x, h0, gi, h, dh_seed, dhT, dh, dh0, dx, grads, resnorm, ws, ws_bytes, (cudaStream_t)stream);
+}
+
+int gru_serial_backward(const mgrit_gru_cfg* cfg, const gru_params* p, const float* x, const float* h0, const float* gi,
+                        const float* h, const float* dh_seed, const float* dhT, float* dh, float* dh0, float* dx,
+                        const gru_grads* grads, void* ws, size_t ws_bytes, mgrit_stream_t stream) {
+  return adjoint_impl(cfg, true, p, x, h0, gi, h, dh_seed, dhT, dh, dh0, dx, grads, nullptr, ws, ws_bytes, (cudaStream_t)stream);
+}
+
+size_t xent_head_workspace_bytes(int32_t B, int32_t C) {
+  if (B <= 0 || C <= 0) return 0;
+  return (((size_t)B * C * sizeof(float)) + 255) & ~(size_t)255;
+}
+
+int xent_head_fwd_bwd(int32_t B, int32_t H, int32_t C, const float* hT, const float* Wc, const float* bc, const int32_t* labels,
+                      float* loss, float* dhT, float* dWc, float* dbc, void* ws, size_t ws_bytes, mgrit_stream_t stream) {
+  if (B <= 0 || H <= 0 || C <= 0 || !hT || !Wc || !bc || !labels || !loss || !dhT || !dWc || !dbc || !ws) return MGRIT_INVALID_ARG;
+  if (C > 8192) return MGRIT_UNSUPPORTED;
+  if (ws_bytes < xent_head_workspace_bytes(B, C)) return MGRIT_WORKSPACE_TOO_SMALL;
+  stream_xent(B, H, C, hT, Wc, bc, labels, loss, dhT, dWc, dbc, (float*)ws, (cudaStream_t)stream);
+  return finish((cudaStream_t)stream, false);
+}
+
+int sgd_update(float* p, const float* g, size_t n, float lr, mgrit_stream_t stream) {
+  if (!p || !g) return MGRIT_INVALID_ARG;
+  if (n == 0) return MGRIT_OK;
+  if (((uintptr_t)p | (uintptr_t)g) & 15) return MGRIT_INVALID_ARG;
+  stream_sgd(p, g, n, lr, (cudaStream_t)stream);
+  return finish((cudaStream_t)stream, false);
+}
+
+int mgrit_gru_last_device_status(void) {
+  if (cudaDeviceSynchronize() != cudaSuccess) return MGRIT_CUDA_ERROR;
+  return umma_device_status() != 0 ? MGRIT_DEVICE_TIMEOUT : MGRIT_OK;
+}
+
+unsigned long long mgrit_gru_kernel_launches(void) { return g_kernel_launches; }
+
+const char* mgrit_gru_strerror(int code) {
+  switch (code) {
+    case MGRIT_OK: return "ok";
+    case MGRIT_INVALID_ARG: return "invalid argument";
+    case MGRIT_NOT_DIVISIBLE: return "T is not divisible by cf^(levels-1)";
+    case MGRIT_WORKSPACE_TOO_SMALL: return "workspace too small";
+    case MGRIT_UNSUPPORTED: return "shape not supported by the selected operand mode";
+    case MGRIT_CUDA_ERROR: return "CUDA error";
+    case MGRIT_DEVICE_TIMEOUT: return "a bounded device-side wait ran out";
+    default: return "unknown error";
+  }
+}
+
+}  // extern "C"

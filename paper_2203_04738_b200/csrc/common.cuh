@@ -1,0 +1,84 @@
+// Shared declarations of the library's translation units (host launchers and argument structs).
+#pragma once
+#include <cuda_runtime.h>
+#include <cuda_bf16.h>
+#include <stdint.h>
+#include <stddef.h>
+
+#include "../../include/mgrit_gru.h"
+
+namespace mg {
+
+typedef long long i64;
+
+// Every launch goes through this counter (reported by mgrit_gru_kernel_launches()).
+extern unsigned long long g_kernel_launches;
+inline void count_launch(int n = 1) { g_kernel_launches += (unsigned long long)n; }
+
+// ---- one forward cell evaluation for M = nk*B rows (Eq. "gru" + Eq. "gru-classic"/"gru-imap") ----
+// Row m = (k, b): k = m / B, b = m % B.  All *_ks are strides per k in ELEMENTS (may be negative).
+struct FwdStepArgs {
+  int M, B, H;
+  const float* hin;  i64 hin_ks;    // previous state rows      hin  + k*hin_ks  + b*H
+  float* hout;       i64 hout_ks;   // result rows              hout + k*hout_ks + b*H
+  const float* gi;   i64 gi_ks;     // input projection rows    gi   + k*gi_ks   + b*3H
+  const float* gadd; i64 gadd_ks;   // optional FAS term rows (same shape as hout) or nullptr
+  const float* W_hh;                // [3H,H] fp32
+  const float* b_hh;                // [3H]
+  float gamma;                      // time step of the level: cf^l * dt
+  int cell;                         // MGRIT_CELL_*
+  int mode;                         // 0: hout = Phi + gadd ; 1: hout = hout - Phi   (FAS right-hand side)
+};
+
+// ---- adjoint coefficients of every step of one level (discrete adjoint of the cell) ----
+// Row m = (j-1, b) for forward steps j = 1..N_l.  Outputs are [N_l*B, H] each.
+struct LinArgs {
+  int M, B, H;
+  const float* h0;                  // [B,H]   state at level point 0
+  const float* h;                   // [T,B,H] fine states (h[k] = h_{k+1})
+  i64 stride_t;                     // fine steps per level step: cf^l
+  const float* gi;                  // [T,B,3H]
+  const float* W_hh; const float* b_hh;
+  float gamma; int cell;
+  float *a, *cr, *cz, *cn, *cnp;    // cnp may be nullptr (only level 0 needs it)
+};
+
+// ---- one adjoint step for M = nk*B rows:  out = a*lam + [cr*lam | cz*lam | cn*lam] W_hh (+ gadd) ----
+struct AdjStepArgs {
+  int M, B, H;
+  const float* lin;  i64 lin_ks;    // incoming sensitivity rows
+  float* lout;       i64 lout_ks;
+  const float* gadd; i64 gadd_ks;   // optional source / FAS term, same shape as lout
+  const float *a, *cr, *cz, *cn; i64 coef_ks;   // coefficient rows (+k*coef_ks + b*H), already offset to k = 0
+  const float* W_hh;                // [3H,H] fp32
+  int mode;                         // as FwdStepArgs
+};
+
+// SIMT (fp32 FFMA) engine
+void simt_project(const float* x, const float* W_ih, const float* b_ih, float* gi, int M, int I, int H3, cudaStream_t s);
+void simt_fwd_step(const FwdStepArgs& a, cudaStream_t s);
+void simt_linearise(const LinArgs& a, cudaStream_t s);
+void simt_adj_step(const AdjStepArgs& a, cudaStream_t s);
+// dW[n3, c] = sum_m dA[m, n3] * R[m, c],  R rows: m < B ? first[m] : rest[m-B]   (first may be nullptr with B = 0)
+void simt_wgrad(const float* dA, int M, int H3, const float* first, int Bfirst, const float* rest, int C, float* dW, cudaStream_t s);
+// dx[m, c] = sum_n3 dA[m, n3] * W[n3, c]
+void simt_dgrad(const float* dA, int M, int H3, const float* W, int C, float* dx, cudaStream_t s);
+
+// streaming kernels
+// r = uC - v at the C-points, sum of squares into *acc (double, device), copy of the C-point state
+// to the coarse level:   uc[k] = uf[cf*k],  k = 1..nc   (rows of rowlen = B*H floats)
+void stream_restrict_residual(const float* uf, int cf, const float* v, float* uc, int nc, i64 rowlen, double* acc, cudaStream_t s);
+void stream_correct(float* uf, int cf, const float* uc, int nc, i64 rowlen, cudaStream_t s);
+// dst[k] = src[k*src_ks], k = 0..nk-1, rows of rowlen floats (src_ks in elements, may be negative)
+void stream_gather_rows(float* dst, i64 dst_ks, const float* src, i64 src_ks, int nk, i64 rowlen, cudaStream_t s);
+void stream_add_rows(float* dst, const float* src, i64 n, cudaStream_t s);
+// dA_h = [cr*lam | cz*lam | cn*lam], dA_i = [cr*lam | cz*lam | cnp*lam]  for M rows of H
+void stream_form_dA(const float* lam, const float* cr, const float* cz, const float* cn, const float* cnp,
+                    float* dA_h, float* dA_i, i64 M, int H, cudaStream_t s);
+void stream_colsum(const float* A, i64 M, int N, float* out, cudaStream_t s);
+void stream_sqrt_to_float(const double* acc, float* out, int n, cudaStream_t s);
+void stream_xent(int B, int H, int C, const float* hT, const float* Wc, const float* bc, const int32_t* labels,
+                 float* loss, float* dhT, float* dWc, float* dbc, float* dlogits, cudaStream_t s);
+void stream_sgd(float* p, const float* g, size_t n, float lr, cudaStream_t s);
+
+}  // namespace mg

@@ -1,0 +1,255 @@
+// Streaming (HBM-bound) kernels: grid transfers of the multigrid cycle, operand forming for the
+// gradient pass, column sums, the classifier head and the SGD update.  float4 accesses,
+// coalesced along the hidden dimension; grids sized in multiples of the SM count.
+#include "common.cuh"
+
+namespace mg {
+
+namespace {
+
+constexpr int kSMs = 148;
+constexpr int kThreads = 256;
+
+inline int stream_grid(i64 work_items, int per_block = kThreads) {
+  i64 blocks = (work_items + per_block - 1) / per_block;
+  i64 cap = (i64)kSMs * 8;
+  if (blocks > cap) blocks = cap;
+  if (blocks < 1) blocks = 1;
+  return (int)blocks;
+}
+
+__device__ __forceinline__ float warp_sum(float v) {
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
+  return v;
+}
+
+// Residual at the C-points (r = u_C - v), its squared norm, and restriction by injection
+// (Algorithm "MGProp": r_c = R(f(h')), h'_c = R(h');  Eq. "restrict").
+__global__ void __launch_bounds__(kThreads) restrict_residual_kernel(const float4* __restrict__ uf, int cf,
+                                                                     const float4* __restrict__ v,
+                                                                     float4* __restrict__ uc, int nc, i64 row4,
+                                                                     double* acc) {
+  i64 total = (i64)nc * row4;
+  float s = 0.f;
+  for (i64 e = (i64)blockIdx.x * blockDim.x + threadIdx.x; e < total; e += (i64)gridDim.x * blockDim.x) {
+    i64 k = e / row4 + 1, c = e % row4;
+    float4 u = uf[(k * cf) * row4 + c];
+    float4 w = v[k * row4 + c];
+    float4 r = make_float4(u.x - w.x, u.y - w.y, u.z - w.z, u.w - w.w);
+    s += r.x * r.x + r.y * r.y + r.z * r.z + r.w * r.w;
+    uc[k * row4 + c] = u;
+  }
+  __shared__ float part[kThreads / 32];
+  s = warp_sum(s);
+  if ((threadIdx.x & 31) == 0) part[threadIdx.x >> 5] = s;
+  __syncthreads();
+  if (threadIdx.x < 32) {
+    float t = threadIdx.x < kThreads / 32 ? part[threadIdx.x] : 0.f;
+    t = warp_sum(t);
+    if (threadIdx.x == 0 && acc) atomicAdd(acc, (double)t);
+  }
+}
+
+// Correction h'' = h' + P(h_c* - h'_c): only C-points are read afterwards, so u_{cf k} <- U_k.
+__global__ void __launch_bounds__(kThreads) correct_kernel(float4* __restrict__ uf, int cf, const float4* __restrict__ uc,
+                                                           int nc, i64 row4) {
+  i64 total = (i64)nc * row4;
+  for (i64 e = (i64)blockIdx.x * blockDim.x + threadIdx.x; e < total; e += (i64)gridDim.x * blockDim.x) {
+    i64 k = e / row4 + 1, c = e % row4;
+    uf[(k * cf) * row4 + c] = uc[k * row4 + c];
+  }
+}
+
+__global__ void __launch_bounds__(kThreads) gather_rows_kernel(float4* __restrict__ dst, i64 dst_ks4,
+                                                               const float4* __restrict__ src, i64 src_ks4, int nk,
+                                                               i64 row4) {
+  i64 total = (i64)nk * row4;
+  for (i64 e = (i64)blockIdx.x * blockDim.x + threadIdx.x; e < total; e += (i64)gridDim.x * blockDim.x) {
+    i64 k = e / row4, c = e % row4;
+    dst[k * dst_ks4 + c] = src[k * src_ks4 + c];
+  }
+}
+
+__global__ void __launch_bounds__(kThreads) add_rows_kernel(float4* __restrict__ dst, const float4* __restrict__ src, i64 n4) {
+  for (i64 e = (i64)blockIdx.x * blockDim.x + threadIdx.x; e < n4; e += (i64)gridDim.x * blockDim.x) {
+    float4 a = dst[e], b = src[e];
+    dst[e] = make_float4(a.x + b.x, a.y + b.y, a.z + b.z, a.w + b.w);
+  }
+}
+
+__global__ void __launch_bounds__(kThreads) form_dA_kernel(const float4* __restrict__ lam, const float4* __restrict__ cr,
+                                                           const float4* __restrict__ cz, const float4* __restrict__ cn,
+                                                           const float4* __restrict__ cnp, float4* __restrict__ dA_h,
+                                                           float4* __restrict__ dA_i, i64 M, int H4) {
+  i64 total = M * H4;
+  for (i64 e = (i64)blockIdx.x * blockDim.x + threadIdx.x; e < total; e += (i64)gridDim.x * blockDim.x) {
+    i64 m = e / H4, c = e % H4;
+    float4 l = lam[e], r = cr[e], z = cz[e], n = cn[e], p = cnp[e];
+    i64 o = m * 3 * H4 + c;
+    float4 vr = make_float4(r.x * l.x, r.y * l.y, r.z * l.z, r.w * l.w);
+    float4 vz = make_float4(z.x * l.x, z.y * l.y, z.z * l.z, z.w * l.w);
+    dA_h[o] = vr; dA_i[o] = vr;
+    dA_h[o + H4] = vz; dA_i[o + H4] = vz;
+    dA_h[o + 2 * H4] = make_float4(n.x * l.x, n.y * l.y, n.z * l.z, n.w * l.w);
+    dA_i[o + 2 * H4] = make_float4(p.x * l.x, p.y * l.y, p.z * l.z, p.w * l.w);
+  }
+}
+
+// out[n] = sum_m A[m, n]; one block per 32 columns, deterministic.
+__global__ void __launch_bounds__(1024) colsum_kernel(const float* __restrict__ A, i64 M, int N, float* __restrict__ out) {
+  __shared__ float part[32][33];
+  int n = blockIdx.x * 32 + threadIdx.x;
+  float s = 0.f;
+  if (n < N)
+    for (i64 m = threadIdx.y; m < M; m += 32) s += A[m * N + n];
+  part[threadIdx.y][threadIdx.x] = s;
+  __syncthreads();
+  if (threadIdx.y == 0 && n < N) {
+    float t = 0.f;
+#pragma unroll
+    for (int i = 0; i < 32; ++i) t += part[i][threadIdx.x];
+    out[n] = t;
+  }
+}
+
+__global__ void sqrt_to_float_kernel(const double* acc, float* out, int n) {
+  int i = blockIdx.x * blockDim.x + threadIdx.x;
+  if (i < n) out[i] = (float)sqrt(acc[i]);
+}
+
+// Classifier head, pass 1: one block per batch row: logits, softmax, loss term, dlogits = (p - onehot)/B.
+__global__ void __launch_bounds__(kThreads) xent_rows_kernel(int B, int H, int C, const float* __restrict__ hT,
+                                                             const float* __restrict__ Wc, const float* __restrict__ bc,
+                                                             const int32_t* __restrict__ labels, float* loss,
+                                                             float* __restrict__ dlogits) {
+  extern __shared__ float logit[];  // C floats
+  int b = blockIdx.x;
+  int warp = threadIdx.x >> 5, lane = threadIdx.x & 31, nw = blockDim.x >> 5;
+  for (int c = warp; c < C; c += nw) {
+    float s = 0.f;
+    for (int i = lane; i < H; i += 32) s += hT[(i64)b * H + i] * Wc[(i64)c * H + i];
+    s = warp_sum(s);
+    if (lane == 0) logit[c] = s + bc[c];
+  }
+  __syncthreads();
+  if (warp == 0) {
+    float mx = -INFINITY;
+    for (int c = lane; c < C; c += 32) mx = fmaxf(mx, logit[c]);
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, o));
+    float se = 0.f;
+    for (int c = lane; c < C; c += 32) se += __expf(logit[c] - mx);
+    se = warp_sum(se);
+    int lab = labels[b];
+    float invB = 1.0f / (float)B;
+    for (int c = lane; c < C; c += 32) {
+      float p = __expf(logit[c] - mx) / se;
+      dlogits[(i64)b * C + c] = (p - (c == lab ? 1.f : 0.f)) * invB;
+    }
+    if (lane == 0) atomicAdd(loss, -((logit[lab] - mx) - logf(se)) * invB);
+  }
+}
+
+// pass 2: dhT = dlogits Wc ; dWc = dlogits^T hT ; dbc = column sums of dlogits.
+__global__ void __launch_bounds__(kThreads) xent_grads_kernel(int B, int H, int C, const float* __restrict__ hT,
+                                                              const float* __restrict__ Wc,
+                                                              const float* __restrict__ dlogits, float* __restrict__ dhT,
+                                                              float* __restrict__ dWc, float* __restrict__ dbc) {
+  i64 nBH = (i64)B * H, nCH = (i64)C * H;
+  for (i64 e = (i64)blockIdx.x * blockDim.x + threadIdx.x; e < nBH + nCH + C; e += (i64)gridDim.x * blockDim.x) {
+    if (e < nBH) {
+      int b = e / H, i = e % H;
+      float s = 0.f;
+      for (int c = 0; c < C; ++c) s += dlogits[(i64)b * C + c] * Wc[(i64)c * H + i];
+      dhT[e] = s;
+    } else if (e < nBH + nCH) {
+      i64 f = e - nBH;
+      int c = f / H, i = f % H;
+      float s = 0.f;
+      for (int b = 0; b < B; ++b) s += dlogits[(i64)b * C + c] * hT[(i64)b * H + i];
+      dWc[f] = s;
+    } else {
+      int c = (int)(e - nBH - nCH);
+      float s = 0.f;
+      for (int b = 0; b < B; ++b) s += dlogits[(i64)b * C + c];
+      dbc[c] = s;
+    }
+  }
+}
+
+__global__ void __launch_bounds__(kThreads) sgd_kernel(float* __restrict__ p, const float* __restrict__ g, size_t n, float lr) {
+  size_t n4 = n / 4;
+  float4* p4 = reinterpret_cast<float4*>(p);
+  const float4* g4 = reinterpret_cast<const float4*>(g);
+  size_t stride = (size_t)gridDim.x * blockDim.x, t = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
+  for (size_t e = t; e < n4; e += stride) {
+    float4 a = p4[e], b = g4[e];
+    p4[e] = make_float4(a.x - lr * b.x, a.y - lr * b.y, a.z - lr * b.z, a.w - lr * b.w);
+  }
+  for (size_t e = n4 * 4 + t; e < n; e += stride) p[e] -= lr * g[e];
+}
+
+}  // namespace
+
+void stream_restrict_residual(const float* uf, int cf, const float* v, float* uc, int nc, i64 rowlen, double* acc,
+                              cudaStream_t s) {
+  i64 row4 = rowlen / 4;
+  restrict_residual_kernel<<<stream_grid((i64)nc * row4), kThreads, 0, s>>>(
+      reinterpret_cast<const float4*>(uf), cf, reinterpret_cast<const float4*>(v), reinterpret_cast<float4*>(uc), nc, row4, acc);
+  count_launch();
+}
+
+void stream_correct(float* uf, int cf, const float* uc, int nc, i64 rowlen, cudaStream_t s) {
+  i64 row4 = rowlen / 4;
+  correct_kernel<<<stream_grid((i64)nc * row4), kThreads, 0, s>>>(reinterpret_cast<float4*>(uf), cf,
+                                                                  reinterpret_cast<const float4*>(uc), nc, row4);
+  count_launch();
+}
+
+void stream_gather_rows(float* dst, i64 dst_ks, const float* src, i64 src_ks, int nk, i64 rowlen, cudaStream_t s) {
+  if (nk <= 0) return;
+  i64 row4 = rowlen / 4;
+  gather_rows_kernel<<<stream_grid((i64)nk * row4), kThreads, 0, s>>>(reinterpret_cast<float4*>(dst), dst_ks / 4,
+                                                                      reinterpret_cast<const float4*>(src), src_ks / 4, nk, row4);
+  count_launch();
+}
+
+void stream_add_rows(float* dst, const float* src, i64 n, cudaStream_t s) {
+  add_rows_kernel<<<stream_grid(n / 4), kThreads, 0, s>>>(reinterpret_cast<float4*>(dst), reinterpret_cast<const float4*>(src), n / 4);
+  count_launch();
+}
+
+void stream_form_dA(const float* lam, const float* cr, const float* cz, const float* cn, const float* cnp, float* dA_h,
+                    float* dA_i, i64 M, int H, cudaStream_t s) {
+  form_dA_kernel<<<stream_grid(M * (H / 4)), kThreads, 0, s>>>(
+      reinterpret_cast<const float4*>(lam), reinterpret_cast<const float4*>(cr), reinterpret_cast<const float4*>(cz),
+      reinterpret_cast<const float4*>(cn), reinterpret_cast<const float4*>(cnp), reinterpret_cast<float4*>(dA_h),
+      reinterpret_cast<float4*>(dA_i), M, H / 4);
+  count_launch();
+}
+
+void stream_colsum(const float* A, i64 M, int N, float* out, cudaStream_t s) {
+  colsum_kernel<<<(N + 31) / 32, dim3(32, 32), 0, s>>>(A, M, N, out);
+  count_launch();
+}
+
+void stream_sqrt_to_float(const double* acc, float* out, int n, cudaStream_t s) {
+  sqrt_to_float_kernel<<<(n + 63) / 64, 64, 0, s>>>(acc, out, n);
+  count_launch();
+}
+
+void stream_xent(int B, int H, int C, const float* hT, const float* Wc, const float* bc, const int32_t* labels, float* loss,
+                 float* dhT, float* dWc, float* dbc, float* dlogits, cudaStream_t s) {
+  cudaMemsetAsync(loss, 0, sizeof(float), s);
+  xent_rows_kernel<<<B, kThreads, (size_t)C * sizeof(float), s>>>(B, H, C, hT, Wc, bc, labels, loss, dlogits);
+  xent_grads_kernel<<<stream_grid((i64)B * H + (i64)C * H + C), kThreads, 0, s>>>(B, H, C, hT, Wc, dlogits, dhT, dWc, dbc);
+  count_launch(2);
+}
+
+void stream_sgd(float* p, const float* g, size_t n, float lr, cudaStream_t s) {
+  sgd_kernel<<<stream_grid((i64)(n / 4 + 1)), kThreads, 0, s>>>(p, g, n, lr);
+  count_launch();
+}
+
+}  // namespace mg

@@ -1,0 +1,42 @@
+// Interface of the tensor-core (tcgen05 / TMA, bf16 operands, fp32 accumulation) engine.
+#pragma once
+#include "common.cuh"
+
+namespace mg {
+
+struct UmmaFwdWs {
+  __nv_bfloat16* W_hh;   // [3H,H]
+  __nv_bfloat16* W_ih;   // [3H,I]
+  __nv_bfloat16* xb;     // [T*B,I]
+  __nv_bfloat16* Apack;  // [maxM,H]  A operand of one step (rows gathered from the level state)
+  size_t maxM;
+};
+
+struct UmmaAdjWs {
+  __nv_bfloat16* W_hh;    // [3H,H]   (linearisation)
+  __nv_bfloat16* W_hhT;   // [H,3H]   (adjoint step: B operand, K = 3H contiguous)
+  __nv_bfloat16* W_ihT;   // [I,3H]   (dx = dA_i W_ih)
+  __nv_bfloat16* Apack;   // [maxM,3H]
+  __nv_bfloat16* dAhT;    // [3H,T*B]
+  __nv_bfloat16* dAiT;    // [3H,T*B]
+  __nv_bfloat16* dAi;     // [T*B,3H]
+  __nv_bfloat16* hprevT;  // [H,T*B]
+  __nv_bfloat16* xT;      // [I,T*B]
+  float* dbpart;          // partial column sums
+  size_t maxM;
+};
+
+int umma_supported(const mgrit_gru_cfg* c);
+void umma_plan_fwd(const mgrit_gru_cfg* c, const int* N, int L, char* base, size_t* off, UmmaFwdWs* o);
+void umma_plan_adj(const mgrit_gru_cfg* c, const int* N, int L, char* base, size_t* off, UmmaAdjWs* o);
+int umma_prepare_fwd(const mgrit_gru_cfg* c, const gru_params* p, const float* x, float* gi, UmmaFwdWs* w, cudaStream_t s);
+int umma_prepare_adj(const mgrit_gru_cfg* c, const gru_params* p, UmmaAdjWs* w, cudaStream_t s);
+void umma_fwd_step(const FwdStepArgs& a, UmmaFwdWs* w, cudaStream_t s);
+void umma_linearise(const LinArgs& a, UmmaAdjWs* w, cudaStream_t s);
+void umma_adj_step(const AdjStepArgs& a, UmmaAdjWs* w, cudaStream_t s);
+int umma_gradients(const mgrit_gru_cfg* c, const gru_params* p, const float* x, const float* h0, const float* h,
+                   const float* lam, const float* cr, const float* cz, const float* cn, const float* cnp, float* dx,
+                   const gru_grads* g, UmmaAdjWs* w, cudaStream_t s);
+int umma_device_status();
+
+}  // namespace mg
