@@ -1,14 +1,489 @@
+// Tensor-core engine: bf16 operands, fp32 accumulation in tensor memory, fp32 states and gates.
+// Host launchers, operand-packing kernels and the fused epilogues of the tcgen05 GEMM.
+#include <stdio.h>
+
+#include "cell.cuh"
 #include "umma_engine.cuh"
+#include "umma_gemm.cuh"
+
 namespace mg {
-int umma_supported(const mgrit_gru_cfg*) { return MGRIT_UNSUPPORTED; }
-void umma_plan_fwd(const mgrit_gru_cfg*, const int*, int, char*, size_t*, UmmaFwdWs*) {}
-void umma_plan_adj(const mgrit_gru_cfg*, const int*, int, char*, size_t*, UmmaAdjWs*) {}
-int umma_prepare_fwd(const mgrit_gru_cfg*, const gru_params*, const float*, float*, UmmaFwdWs*, cudaStream_t) { return MGRIT_UNSUPPORTED; }
-int umma_prepare_adj(const mgrit_gru_cfg*, const gru_params*, UmmaAdjWs*, cudaStream_t) { return MGRIT_UNSUPPORTED; }
-void umma_fwd_step(const FwdStepArgs&, UmmaFwdWs*, cudaStream_t) {}
-void umma_linearise(const LinArgs&, UmmaAdjWs*, cudaStream_t) {}
-void umma_adj_step(const AdjStepArgs&, UmmaAdjWs*, cudaStream_t) {}
-int umma_gradients(const mgrit_gru_cfg*, const gru_params*, const float*, const float*, const float*, const float*, const float*,
-                   const float*, const float*, const float*, float*, const gru_grads*, UmmaAdjWs*, cudaStream_t) { return MGRIT_UNSUPPORTED; }
-int umma_device_status() { return 0; }
+
+namespace {
+
+using namespace umma;
+typedef __nv_bfloat16 bf16;
+
+__device__ int g_umma_status = 0;   // first error code of a bounded wait that ran out (0 = none)
+int* g_status_ptr = nullptr;
+
+constexpr int kSMs = 148;
+
+// ---------------------------------------------------------------- tensor maps
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*, const cuuint64_t*,
+                                  const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave, CUtensorMapSwizzle,
+                                  CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+EncodeTiledFn g_encode = nullptr;
+
+bool ensure_driver() {
+  if (g_encode && g_status_ptr) return true;
+  if (!g_encode) {
+    void* fn = nullptr;
+    cudaDriverEntryPointQueryResult q;
+    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &fn, cudaEnableDefault, &q) != cudaSuccess || !fn) return false;
+    g_encode = (EncodeTiledFn)fn;
+  }
+  if (!g_status_ptr) {
+    if (cudaGetSymbolAddress((void**)&g_status_ptr, g_umma_status) != cudaSuccess) return false;
+  }
+  return true;
 }
+
+// bf16 matrix [rows, inner] with row pitch `pitch` elements; box = 64 x box_rows, 128-byte swizzle
+bool make_map(CUtensorMap* m, const bf16* base, uint64_t inner, uint64_t rows, uint64_t pitch, uint32_t box_rows) {
+  cuuint64_t dims[2] = {inner, rows};
+  cuuint64_t strides[1] = {pitch * sizeof(bf16)};
+  cuuint32_t box[2] = {(cuuint32_t)BK, box_rows};
+  cuuint32_t estr[2] = {1, 1};
+  CUresult r = g_encode(m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, (void*)base, dims, strides, box, estr,
+                        CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                        CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  if (r != CUDA_SUCCESS) fprintf(stderr, "mgrit_gru: cuTensorMapEncodeTiled failed (%d)\n", (int)r);
+  return r == CUDA_SUCCESS;
+}
+
+template <int BN, bool GATES, class Epi>
+bool launch_gemm(const bf16* A, i64 lda, const bf16* Bm, i64 ldb, int M, int N, int K, int gate_rows, int b_rows, Epi epi,
+                 cudaStream_t s) {
+  using C = Cfg<BN, GATES>;
+  if (M <= 0 || N <= 0) return true;
+  if (!ensure_driver()) return false;
+  static bool attr_set = false;
+  auto kern = umma_gemm_kernel<BN, GATES, Epi>;
+  if (!attr_set) {
+    if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, C::kSmemBytes) != cudaSuccess) return false;
+    attr_set = true;
+  }
+  CUtensorMap ta, tb;
+  if (!make_map(&ta, A, (uint64_t)K, (uint64_t)M, (uint64_t)lda, BM)) return false;
+  if (!make_map(&tb, Bm, (uint64_t)K, (uint64_t)b_rows, (uint64_t)ldb, GATES ? BN / 3 : BN)) return false;
+  GemmShape sh{M, N, K, gate_rows};
+  int m_tiles = (M + BM - 1) / BM, n_tiles = (N + C::kNPerTile - 1) / C::kNPerTile;
+  int tiles = m_tiles * n_tiles;
+  int grid = tiles < kSMs ? tiles : kSMs;
+  kern<<<grid, kThreads, C::kSmemBytes, s>>>(ta, tb, sh, epi, g_status_ptr);
+  count_launch();
+  return true;
+}
+
+// ---------------------------------------------------------------- epilogues (one output row per thread)
+__device__ __forceinline__ float4 ld4(const float* p) { return *reinterpret_cast<const float4*>(p); }
+__device__ __forceinline__ void st4(float* p, float a, float b, float c, float d) {
+  *reinterpret_cast<float4*>(p) = make_float4(a, b, c, d);
+}
+
+struct EpiBias {  // out[m, n] = acc + bias[n]      (input projection)
+  float* out; i64 ld; const float* bias; int M, N;
+  __device__ void operator()(uint32_t taddr, int row, int n0) const {
+    const bool valid = row < M;
+    float* o = out + (i64)row * ld + n0;
+    for (int c0 = 0; c0 < 256 && n0 + c0 < N; c0 += 16) {
+      float v[16];
+      tmem_ld16(taddr + c0, v);
+      tmem_ld_wait();
+      if (valid) {
+#pragma unroll
+        for (int i = 0; i < 16; i += 4) {
+          float4 b = __ldg(reinterpret_cast<const float4*>(bias + n0 + c0 + i));
+          st4(o + c0 + i, v[i] + b.x, v[i + 1] + b.y, v[i + 2] + b.z, v[i + 3] + b.w);
+        }
+      }
+    }
+  }
+};
+
+struct EpiStore {  // out[m, n] = acc            (weight / input gradients)
+  float* out; i64 ld; int M, N;
+  __device__ void operator()(uint32_t taddr, int row, int n0) const {
+    const bool valid = row < M;
+    float* o = out + (i64)row * ld + n0;
+    for (int c0 = 0; c0 < 256 && n0 + c0 < N; c0 += 16) {
+      float v[16];
+      tmem_ld16(taddr + c0, v);
+      tmem_ld_wait();
+      if (valid) {
+#pragma unroll
+        for (int i = 0; i < 16; i += 4) st4(o + c0 + i, v[i], v[i + 1], v[i + 2], v[i + 3]);
+      }
+    }
+  }
+};
+
+struct EpiFwd {  // GRU cell on the r|z|n accumulator columns of 64 hidden units
+  FwdStepArgs a;
+  __device__ void operator()(uint32_t taddr, int row, int u0) const {
+    const bool valid = row < a.M;
+    const int k = valid ? row / a.B : 0, b = valid ? row % a.B : 0;
+    const float* gi = a.gi + (i64)k * a.gi_ks + (i64)b * 3 * a.H + u0;
+    const float* hp = a.hin + (i64)k * a.hin_ks + (i64)b * a.H + u0;
+    float* ho = a.hout + (i64)k * a.hout_ks + (i64)b * a.H + u0;
+    const float* ga = a.gadd ? a.gadd + (i64)k * a.gadd_ks + (i64)b * a.H + u0 : nullptr;
+    const float* bh = a.b_hh + u0;
+    for (int c0 = 0; c0 < 64; c0 += 16) {
+      float r[16], z[16], n[16];
+      tmem_ld16(taddr + c0, r);
+      tmem_ld16(taddr + 64 + c0, z);
+      tmem_ld16(taddr + 128 + c0, n);
+      tmem_ld_wait();
+      if (valid) {
+#pragma unroll
+        for (int i = 0; i < 16; i += 4) {
+          const int c = c0 + i;
+          float4 gr = ld4(gi + c), gz = ld4(gi + a.H + c), gn = ld4(gi + 2 * a.H + c), h4 = ld4(hp + c);
+          float4 br = __ldg(reinterpret_cast<const float4*>(bh + c));
+          float4 bz = __ldg(reinterpret_cast<const float4*>(bh + a.H + c));
+          float4 bn = __ldg(reinterpret_cast<const float4*>(bh + 2 * a.H + c));
+          float o0 = cell_forward(gr.x, gz.x, gn.x, r[i] + br.x, z[i] + bz.x, n[i] + bn.x, h4.x, a.gamma, a.cell);
+          float o1 = cell_forward(gr.y, gz.y, gn.y, r[i + 1] + br.y, z[i + 1] + bz.y, n[i + 1] + bn.y, h4.y, a.gamma, a.cell);
+          float o2 = cell_forward(gr.z, gz.z, gn.z, r[i + 2] + br.z, z[i + 2] + bz.z, n[i + 2] + bn.z, h4.z, a.gamma, a.cell);
+          float o3 = cell_forward(gr.w, gz.w, gn.w, r[i + 3] + br.w, z[i + 3] + bz.w, n[i + 3] + bn.w, h4.w, a.gamma, a.cell);
+          if (a.mode == 0) {
+            if (ga) { float4 g4 = ld4(ga + c); o0 += g4.x; o1 += g4.y; o2 += g4.z; o3 += g4.w; }
+            st4(ho + c, o0, o1, o2, o3);
+          } else {
+            float4 p4 = ld4(ho + c);
+            st4(ho + c, p4.x - o0, p4.y - o1, p4.z - o2, p4.w - o3);
+          }
+        }
+      }
+    }
+  }
+};
+
+struct EpiLin {  // adjoint coefficients of every step of a level
+  LinArgs a;
+  __device__ void operator()(uint32_t taddr, int row, int u0) const {
+    const bool valid = row < a.M;
+    const int j1 = valid ? row / a.B : 0, b = valid ? row % a.B : 0;
+    const float* gi = a.gi + (((i64)(j1 + 1) * a.stride_t - 1) * a.B + b) * 3 * a.H + u0;
+    const float* hp = (j1 == 0 ? a.h0 + (i64)b * a.H : a.h + (((i64)j1 * a.stride_t - 1) * a.B + b) * a.H) + u0;
+    const i64 o = (i64)row * a.H + u0;
+    const float* bh = a.b_hh + u0;
+    for (int c0 = 0; c0 < 64; c0 += 16) {
+      float r[16], z[16], n[16];
+      tmem_ld16(taddr + c0, r);
+      tmem_ld16(taddr + 64 + c0, z);
+      tmem_ld16(taddr + 128 + c0, n);
+      tmem_ld_wait();
+      if (valid) {
+#pragma unroll
+        for (int i = 0; i < 16; i += 4) {
+          const int c = c0 + i;
+          float gr[4], gz[4], gn[4], h4[4], br[4], bz[4], bn[4];
+          *reinterpret_cast<float4*>(gr) = ld4(gi + c);
+          *reinterpret_cast<float4*>(gz) = ld4(gi + a.H + c);
+          *reinterpret_cast<float4*>(gn) = ld4(gi + 2 * a.H + c);
+          *reinterpret_cast<float4*>(h4) = ld4(hp + c);
+          *reinterpret_cast<float4*>(br) = __ldg(reinterpret_cast<const float4*>(bh + c));
+          *reinterpret_cast<float4*>(bz) = __ldg(reinterpret_cast<const float4*>(bh + a.H + c));
+          *reinterpret_cast<float4*>(bn) = __ldg(reinterpret_cast<const float4*>(bh + 2 * a.H + c));
+          float oa[4], ocr[4], ocz[4], ocn[4], ocp[4];
+#pragma unroll
+          for (int e = 0; e < 4; ++e) {
+            CellLin L = cell_linearise(gr[e], gz[e], gn[e], r[i + e] + br[e], z[i + e] + bz[e], n[i + e] + bn[e], h4[e],
+                                       a.gamma, a.cell);
+            oa[e] = L.a; ocr[e] = L.cr; ocz[e] = L.cz; ocn[e] = L.cn; ocp[e] = L.cnp;
+          }
+          st4(a.a + o + c, oa[0], oa[1], oa[2], oa[3]);
+          st4(a.cr + o + c, ocr[0], ocr[1], ocr[2], ocr[3]);
+          st4(a.cz + o + c, ocz[0], ocz[1], ocz[2], ocz[3]);
+          st4(a.cn + o + c, ocn[0], ocn[1], ocn[2], ocn[3]);
+          if (a.cnp) st4(a.cnp + o + c, ocp[0], ocp[1], ocp[2], ocp[3]);
+        }
+      }
+    }
+  }
+};
+
+struct EpiAdj {  // lambda_prev = a*lambda + acc (+ source)
+  AdjStepArgs a;
+  __device__ void operator()(uint32_t taddr, int row, int n0) const {
+    const bool valid = row < a.M;
+    const int k = valid ? row / a.B : 0, b = valid ? row % a.B : 0;
+    const float* li = a.lin + (i64)k * a.lin_ks + (i64)b * a.H + n0;
+    const float* ca = a.a + (i64)k * a.coef_ks + (i64)b * a.H + n0;
+    float* lo = a.lout + (i64)k * a.lout_ks + (i64)b * a.H + n0;
+    const float* ga = a.gadd ? a.gadd + (i64)k * a.gadd_ks + (i64)b * a.H + n0 : nullptr;
+    for (int c0 = 0; c0 < 256 && n0 + c0 < a.H; c0 += 16) {
+      float v[16];
+      tmem_ld16(taddr + c0, v);
+      tmem_ld_wait();
+      if (valid) {
+#pragma unroll
+        for (int i = 0; i < 16; i += 4) {
+          const int c = c0 + i;
+          float4 l4 = ld4(li + c), a4 = ld4(ca + c);
+          float o0 = a4.x * l4.x + v[i], o1 = a4.y * l4.y + v[i + 1], o2 = a4.z * l4.z + v[i + 2], o3 = a4.w * l4.w + v[i + 3];
+          if (a.mode == 0) {
+            if (ga) { float4 g4 = ld4(ga + c); o0 += g4.x; o1 += g4.y; o2 += g4.z; o3 += g4.w; }
+            st4(lo + c, o0, o1, o2, o3);
+          } else {
+            float4 p4 = ld4(lo + c);
+            st4(lo + c, p4.x - o0, p4.y - o1, p4.z - o2, p4.w - o3);
+          }
+        }
+      }
+    }
+  }
+};
+
+// ---------------------------------------------------------------- operand packing (HBM streams)
+constexpr int kPT = 256;
+inline int pgrid(i64 items) {
+  i64 b = (items + kPT - 1) / kPT, cap = (i64)kSMs * 8;
+  return (int)(b < 1 ? 1 : (b > cap ? cap : b));
+}
+__device__ __forceinline__ uint2 pack4(float4 v) {
+  __nv_bfloat162 lo = __floats2bfloat162_rn(v.x, v.y), hi = __floats2bfloat162_rn(v.z, v.w);
+  uint2 o;
+  o.x = *reinterpret_cast<uint32_t*>(&lo);
+  o.y = *reinterpret_cast<uint32_t*>(&hi);
+  return o;
+}
+
+__global__ void __launch_bounds__(kPT) convert_kernel(const float4* __restrict__ src, uint2* __restrict__ dst, i64 n4) {
+  for (i64 e = (i64)blockIdx.x * blockDim.x + threadIdx.x; e < n4; e += (i64)gridDim.x * blockDim.x) dst[e] = pack4(src[e]);
+}
+
+// dst[m, :] = bf16(src row (k, b)),  m = k*B + b
+__global__ void __launch_bounds__(kPT) pack_rows_kernel(const float* __restrict__ src, i64 ks, int B, int H4, i64 M,
+                                                        uint2* __restrict__ dst) {
+  i64 total = M * H4;
+  for (i64 e = (i64)blockIdx.x * blockDim.x + threadIdx.x; e < total; e += (i64)gridDim.x * blockDim.x) {
+    i64 m = e / H4; int c = (int)(e % H4);
+    i64 k = m / B; int b = (int)(m % B);
+    dst[e] = pack4(*reinterpret_cast<const float4*>(src + k * ks + ((i64)b * H4 + c) * 4));
+  }
+}
+
+// dst[m, g*H + i] = bf16(c_g[m, i] * lam[m, i])
+__global__ void __launch_bounds__(kPT) pack_adj_kernel(const float* __restrict__ lin, i64 lin_ks, const float* __restrict__ cr,
+                                                       const float* __restrict__ cz, const float* __restrict__ cn, i64 coef_ks,
+                                                       int B, int H4, i64 M, uint2* __restrict__ dst) {
+  i64 total = M * H4;
+  for (i64 e = (i64)blockIdx.x * blockDim.x + threadIdx.x; e < total; e += (i64)gridDim.x * blockDim.x) {
+    i64 m = e / H4; int c = (int)(e % H4);
+    i64 k = m / B; int b = (int)(m % B);
+    i64 ro = ((i64)b * H4 + c) * 4;
+    float4 l = *reinterpret_cast<const float4*>(lin + k * lin_ks + ro);
+    float4 r = *reinterpret_cast<const float4*>(cr + k * coef_ks + ro);
+    float4 z = *reinterpret_cast<const float4*>(cz + k * coef_ks + ro);
+    float4 n = *reinterpret_cast<const float4*>(cn + k * coef_ks + ro);
+    i64 o = m * 3 * H4 + c;
+    dst[o] = pack4(make_float4(r.x * l.x, r.y * l.y, r.z * l.z, r.w * l.w));
+    dst[o + H4] = pack4(make_float4(z.x * l.x, z.y * l.y, z.z * l.z, z.w * l.w));
+    dst[o + 2 * H4] = pack4(make_float4(n.x * l.x, n.y * l.y, n.z * l.z, n.w * l.w));
+  }
+}
+
+// dst[c * dst_ld + col0 + r] = bf16(src[r * C + c]),  src [R, C] fp32
+__global__ void __launch_bounds__(1024) transpose_kernel(const float* __restrict__ src, i64 R, int C, bf16* __restrict__ dst,
+                                                         i64 dst_ld, i64 col0) {
+  __shared__ float tile[32][33];
+  i64 r0 = (i64)blockIdx.x * 32; int c0 = blockIdx.y * 32;
+  i64 r = r0 + threadIdx.y; int c = c0 + threadIdx.x;
+  tile[threadIdx.y][threadIdx.x] = (r < R && c < C) ? src[r * C + c] : 0.f;
+  __syncthreads();
+  i64 rr = r0 + threadIdx.x; int cc = c0 + threadIdx.y;
+  if (rr < R && cc < C) dst[(i64)cc * dst_ld + col0 + rr] = __float2bfloat16(tile[threadIdx.x][threadIdx.y]);
+}
+
+// Gradient-pass operands from the final sensitivities: dA_h = [cr|cz|cn]*lam, dA_i = [cr|cz|cnp]*lam.
+// Writes dA_h^T, dA_i^T ([3H, M] bf16), optionally dA_i ([M, 3H] bf16), and adds the fp32 column sums
+// (bias gradients) of 32-row x 32-unit tiles into db_hh / db_ih.
+__global__ void __launch_bounds__(1024) form_dA_T_kernel(const float* __restrict__ lam, const float* __restrict__ cr,
+                                                         const float* __restrict__ cz, const float* __restrict__ cn,
+                                                         const float* __restrict__ cnp, i64 M, int H, bf16* __restrict__ dAhT,
+                                                         bf16* __restrict__ dAiT, bf16* __restrict__ dAi,
+                                                         float* __restrict__ db_hh, float* __restrict__ db_ih, int row_tiles) {
+  __shared__ float t[4][32][33];
+  const int tx = threadIdx.x, ty = threadIdx.y;
+  const int i = blockIdx.y * 32 + tx;
+  float s[4] = {0.f, 0.f, 0.f, 0.f};
+  for (int rt = 0; rt < row_tiles; ++rt) {
+    i64 m0 = ((i64)blockIdx.x * row_tiles + rt) * 32;
+    if (m0 >= M) break;
+    i64 m = m0 + ty;
+    float v[4] = {0.f, 0.f, 0.f, 0.f};
+    if (m < M && i < H) {
+      i64 e = m * H + i;
+      float l = lam[e];
+      v[0] = cr[e] * l; v[1] = cz[e] * l; v[2] = cn[e] * l; v[3] = cnp[e] * l;
+      if (dAi) {
+        i64 o = m * 3 * H + i;
+        dAi[o] = __float2bfloat16(v[0]); dAi[o + H] = __float2bfloat16(v[1]); dAi[o + 2 * H] = __float2bfloat16(v[3]);
+      }
+    }
+#pragma unroll
+    for (int g = 0; g < 4; ++g) { t[g][ty][tx] = v[g]; s[g] += v[g]; }
+    __syncthreads();
+    i64 mm = m0 + tx; int ii = blockIdx.y * 32 + ty;
+    if (mm < M && ii < H) {
+      bf16 r_ = __float2bfloat16(t[0][tx][ty]), z_ = __float2bfloat16(t[1][tx][ty]);
+      dAhT[(i64)ii * M + mm] = r_;            dAiT[(i64)ii * M + mm] = r_;
+      dAhT[((i64)H + ii) * M + mm] = z_;      dAiT[((i64)H + ii) * M + mm] = z_;
+      dAhT[((i64)2 * H + ii) * M + mm] = __float2bfloat16(t[2][tx][ty]);
+      dAiT[((i64)2 * H + ii) * M + mm] = __float2bfloat16(t[3][tx][ty]);
+    }
+    __syncthreads();
+  }
+  // column sums over this block's rows
+#pragma unroll
+  for (int g = 0; g < 4; ++g) t[g][ty][tx] = s[g];
+  __syncthreads();
+  if (ty < 4 && i < H) {
+    float acc = 0.f;
+#pragma unroll
+    for (int r = 0; r < 32; ++r) acc += t[ty][r][tx];
+    if (ty == 0) { atomicAdd(db_hh + i, acc); atomicAdd(db_ih + i, acc); }
+    else if (ty == 1) { atomicAdd(db_hh + H + i, acc); atomicAdd(db_ih + H + i, acc); }
+    else if (ty == 2) atomicAdd(db_hh + 2 * H + i, acc);
+    else atomicAdd(db_ih + 2 * H + i, acc);
+  }
+}
+
+void convert(const float* src, bf16* dst, i64 n, cudaStream_t s) {
+  convert_kernel<<<pgrid(n / 4), kPT, 0, s>>>(reinterpret_cast<const float4*>(src), reinterpret_cast<uint2*>(dst), n / 4);
+  count_launch();
+}
+void transpose(const float* src, i64 R, int C, bf16* dst, i64 dst_ld, i64 col0, cudaStream_t s) {
+  if (R <= 0) return;
+  transpose_kernel<<<dim3((unsigned)((R + 31) / 32), (C + 31) / 32), dim3(32, 32), 0, s>>>(src, R, C, dst, dst_ld, col0);
+  count_launch();
+}
+
+inline size_t round_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
+template <class T> T* take(char* base, size_t* off, size_t n) {
+  T* p = base ? reinterpret_cast<T*>(base + *off) : nullptr;
+  *off += round_up(n * sizeof(T), 256);
+  return p;
+}
+size_t max_step_rows(const mgrit_gru_cfg* c, const int* N, int L) {
+  size_t m = (size_t)c->B;
+  for (int l = 0; l + 1 < L; ++l) {
+    size_t r = (size_t)(N[l] / c->cf) * c->B;   // relaxation / residual / FAS right-hand side rows
+    if (r > m) m = r;
+  }
+  return m;
+}
+
+}  // namespace
+
+int umma_supported(const mgrit_gru_cfg* c) {
+  if (c->H % 64 != 0 || c->I % 16 != 0 || ((i64)c->T * c->B) % 8 != 0) return MGRIT_UNSUPPORTED;
+  return MGRIT_OK;
+}
+
+void umma_plan_fwd(const mgrit_gru_cfg* c, const int* N, int L, char* base, size_t* off, UmmaFwdWs* o) {
+  o->maxM = max_step_rows(c, N, L);
+  o->W_hh = take<bf16>(base, off, (size_t)3 * c->H * c->H);
+  o->W_ih = take<bf16>(base, off, (size_t)3 * c->H * c->I);
+  o->xb = take<bf16>(base, off, (size_t)c->T * c->B * c->I);
+  o->Apack = take<bf16>(base, off, o->maxM * c->H);
+}
+
+void umma_plan_adj(const mgrit_gru_cfg* c, const int* N, int L, char* base, size_t* off, UmmaAdjWs* o) {
+  size_t TB = (size_t)c->T * c->B, H = c->H, I = c->I;
+  o->maxM = max_step_rows(c, N, L);
+  o->W_hh = take<bf16>(base, off, 3 * H * H);
+  o->W_hhT = take<bf16>(base, off, 3 * H * H);
+  o->W_ihT = take<bf16>(base, off, 3 * H * I);
+  size_t apack = o->maxM * 3 * H;
+  if (TB * H > apack) apack = TB * H;     // the linearisation packs all T*B rows of a level at once
+  o->Apack = take<bf16>(base, off, apack);
+  o->dAhT = take<bf16>(base, off, 3 * H * TB);
+  o->dAiT = take<bf16>(base, off, 3 * H * TB);
+  o->dAi = take<bf16>(base, off, 3 * H * TB);
+  o->hprevT = take<bf16>(base, off, H * TB);
+  o->xT = take<bf16>(base, off, I * TB);
+  o->dbpart = nullptr;
+}
+
+int umma_prepare_fwd(const mgrit_gru_cfg* c, const gru_params* p, const float* x, float* gi, UmmaFwdWs* w, cudaStream_t s) {
+  const int H = c->H, I = c->I;
+  const i64 TB = (i64)c->T * c->B;
+  convert(p->W_hh, w->W_hh, (i64)3 * H * H, s);
+  convert(p->W_ih, w->W_ih, (i64)3 * H * I, s);
+  convert(x, w->xb, TB * I, s);
+  // gi = x W_ih^T + b_ih :  M = T*B, N = 3H, K = I
+  if (!launch_gemm<256, false>(w->xb, I, w->W_ih, I, (int)TB, 3 * H, I, 0, 3 * H, EpiBias{gi, 3 * H, p->b_ih, (int)TB, 3 * H}, s))
+    return MGRIT_CUDA_ERROR;
+  return MGRIT_OK;
+}
+
+int umma_prepare_adj(const mgrit_gru_cfg* c, const gru_params* p, UmmaAdjWs* w, cudaStream_t s) {
+  const int H = c->H, I = c->I;
+  convert(p->W_hh, w->W_hh, (i64)3 * H * H, s);
+  transpose(p->W_hh, 3 * H, H, w->W_hhT, 3 * H, 0, s);   // [H, 3H]
+  transpose(p->W_ih, 3 * H, I, w->W_ihT, 3 * H, 0, s);   // [I, 3H]
+  return ensure_driver() ? MGRIT_OK : MGRIT_CUDA_ERROR;
+}
+
+void umma_fwd_step(const FwdStepArgs& a, UmmaFwdWs* w, cudaStream_t s) {
+  pack_rows_kernel<<<pgrid((i64)a.M * (a.H / 4)), kPT, 0, s>>>(a.hin, a.hin_ks, a.B, a.H / 4, a.M, reinterpret_cast<uint2*>(w->Apack));
+  count_launch();
+  launch_gemm<192, true>(w->Apack, a.H, w->W_hh, a.H, a.M, a.H, a.H, a.H, 3 * a.H, EpiFwd{a}, s);
+}
+
+void umma_linearise(const LinArgs& a, UmmaAdjWs* w, cudaStream_t s) {
+  // rows (j-1, b): state entering forward step j of the level = h_{stride*(j-1)}
+  const i64 BH = (i64)a.B * a.H;
+  pack_rows_kernel<<<pgrid((i64)a.B * (a.H / 4)), kPT, 0, s>>>(a.h0, 0, a.B, a.H / 4, a.B, reinterpret_cast<uint2*>(w->Apack));
+  count_launch();
+  if (a.M > a.B) {
+    pack_rows_kernel<<<pgrid((i64)(a.M - a.B) * (a.H / 4)), kPT, 0, s>>>(a.h + (a.stride_t - 1) * BH, a.stride_t * BH, a.B, a.H / 4,
+                                                                         a.M - a.B, reinterpret_cast<uint2*>(w->Apack + BH));
+    count_launch();
+  }
+  launch_gemm<192, true>(w->Apack, a.H, w->W_hh, a.H, a.M, a.H, a.H, a.H, 3 * a.H, EpiLin{a}, s);
+}
+
+void umma_adj_step(const AdjStepArgs& a, UmmaAdjWs* w, cudaStream_t s) {
+  pack_adj_kernel<<<pgrid((i64)a.M * (a.H / 4)), kPT, 0, s>>>(a.lin, a.lin_ks, a.cr, a.cz, a.cn, a.coef_ks, a.B, a.H / 4, a.M,
+                                                              reinterpret_cast<uint2*>(w->Apack));
+  count_launch();
+  launch_gemm<256, false>(w->Apack, 3 * a.H, w->W_hhT, 3 * a.H, a.M, a.H, 3 * a.H, 0, a.H, EpiAdj{a}, s);
+}
+
+int umma_gradients(const mgrit_gru_cfg* c, const gru_params* p, const float* x, const float* h0, const float* h, const float* lam,
+                   const float* cr, const float* cz, const float* cn, const float* cnp, float* dx, const gru_grads* g,
+                   UmmaAdjWs* w, cudaStream_t s) {
+  const int H = c->H, I = c->I, B = c->B;
+  const i64 M = (i64)c->T * B;
+  cudaMemsetAsync(g->db_hh, 0, sizeof(float) * 3 * H, s);
+  cudaMemsetAsync(g->db_ih, 0, sizeof(float) * 3 * H, s);
+  const int row_tiles = 16;
+  dim3 grid((unsigned)((M + 32 * row_tiles - 1) / (32 * row_tiles)), (H + 31) / 32);
+  form_dA_T_kernel<<<grid, dim3(32, 32), 0, s>>>(lam, cr, cz, cn, cnp, M, H, w->dAhT, w->dAiT, dx ? w->dAi : nullptr, g->db_hh,
+                                                 g->db_ih, row_tiles);
+  count_launch();
+  // h_{t-1} for t = 1..T, transposed: columns (t, b)
+  transpose(h0, B, H, w->hprevT, M, 0, s);
+  transpose(h, M - B, H, w->hprevT, M, B, s);
+  transpose(x, M, I, w->xT, M, 0, s);
+  bool ok = true;
+  // dW_hh[3H, H] = dA_h^T h_prev ;  dW_ih[3H, I] = dA_i^T x    (K = T*B)
+  ok = ok && launch_gemm<256, false>(w->dAhT, M, w->hprevT, M, 3 * H, H, (int)M, 0, H, EpiStore{g->dW_hh, H, 3 * H, H}, s);
+  ok = ok && launch_gemm<256, false>(w->dAiT, M, w->xT, M, 3 * H, I, (int)M, 0, I, EpiStore{g->dW_ih, I, 3 * H, I}, s);
+  // dx[T*B, I] = dA_i W_ih   (K = 3H)
+  if (dx) ok = ok && launch_gemm<256, false>(w->dAi, 3 * H, w->W_ihT, 3 * H, (int)M, I, 3 * H, 0, I, EpiStore{dx, I, (int)M, I}, s);
+  return ok ? MGRIT_OK : MGRIT_CUDA_ERROR;
+}
+
+int umma_device_status() {
+  if (!g_status_ptr) return 0;
+  int v = 0;
+  if (cudaMemcpy(&v, g_status_ptr, sizeof(int), cudaMemcpyDeviceToHost) != cudaSuccess) return -1;
+  return v;
+}
+
+}  // namespace mg
