@@ -1,0 +1,293 @@
+#!/usr/bin/env python
+"""Benchmark of the MGRIT-GRU hot path on B200:  python bench.py --gpus N --steps K --warmup W
+
+One step = one pass of the whole path over one batch of seeded synthetic per-frame features:
+input projections, MGRIT forward of every layer, loss head, MGRIT adjoint of every layer,
+time-parallel weight gradients, SGD update.  Metric: timesteps x batch per second (T*B / step time),
+summed over the N independent replicas (the path does not shard across GPUs: replicas only).
+
+Prints ONE JSON line.  `--impl reference` times the fp64 CPU oracle on a bounded sample instead.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import subprocess
+import sys
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+sys.path.insert(0, ROOT)
+
+METRIC = "MGRIT-GRU fwd+adjoint timesteps*batch/sec"
+UNIT = "timesteps*batch/s"
+# DRAM bytes (read + write) per launch of the forward relaxation-step GEMM, from the ncu capture
+# summarised in profiles/ (per workload); None where no capture exists.
+NCU_TRAFFIC_BYTES_PER_LAUNCH = {}
+
+
+def measured_peaks():
+    try:
+        with open(os.path.join(ROOT, "MEASURED_PEAKS.json")) as f:
+            d = json.load(f)
+        return d, "measured"
+    except Exception:
+        return {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}, "fallback"
+
+
+# ------------------------------------------------------------------------------------------ CPU oracle leg
+def oracle_step(w, d, T, Bsz):
+    """The same training step computed by the fp64 oracle (as it stands) on a T x Bsz sample."""
+    import numpy as np
+    from oracle import mgrit_gru_oracle as O
+    f64 = lambda a: a.astype(np.float64)
+    layers = [[f64(l[n]) for n in ("W_ih", "W_hh", "b_ih", "b_hh")] for l in d["layers"]]
+    x, h0 = f64(d["x"]), f64(d["h0"])
+    kw = dict(cf=w.cf, levels=w.levels, cell=w.cell, relax_fine=w.relax_fine, relax_coarse=w.relax_coarse)
+    hs, inp = [], x
+    for P in layers:
+        h, _ = O.mgrit_forward(*P, inp, h0, iters=w.iters_fwd, **kw)
+        hs.append(h)
+        inp = h
+    loss, dhT, dWc, dbc = O.xent_head(hs[-1][-1], f64(d["W_c"]), f64(d["b_c"]), d["labels"])
+    seed = np.zeros_like(hs[-1])
+    seed[-1] = dhT
+    for l in range(len(layers) - 1, -1, -1):
+        inp = x if l == 0 else hs[l - 1]
+        lam, lam0, g, _ = O.mgrit_adjoint(*layers[l], inp, h0, hs[l], seed, iters=w.iters_adj, want_dx=l > 0, **kw)
+        for i, n in enumerate(("dW_ih", "dW_hh", "db_ih", "db_hh")):
+            layers[l][i] = O.sgd_update(layers[l][i], g[n], 1e-3)
+        seed = g.get("dx")
+    return loss
+
+
+def cpu_sample_shape(w):
+    """A bounded sample of the workload: same widths, levels and cycle counts, shorter and narrower batch."""
+    unit = w.cf ** (w.levels - 1)
+    T = min(w.T, max(unit * 4, 256 if w.H >= 512 else w.T))
+    T = (T // unit) * unit
+    Bsz = min(w.B, 8 if w.H >= 512 else w.B)
+    return T, Bsz
+
+
+def time_oracle(w, steps=1, warmup=0):
+    from paper_2203_04738_b200.synthetic import make_inputs
+    T, Bsz = cpu_sample_shape(w)
+    d = make_inputs(w, T=T, B=Bsz)
+    for _ in range(warmup):
+        oracle_step(w, d, T, Bsz)
+    ts = []
+    for _ in range(max(1, steps)):
+        t0 = time.perf_counter()
+        oracle_step(w, d, T, Bsz)
+        ts.append(time.perf_counter() - t0)
+    sec = sum(ts) / len(ts)
+    try:
+        import threadpoolctl
+        cores = max([p.get("num_threads", 1) for p in threadpoolctl.threadpool_info()] or [1])
+    except Exception:
+        cores = os.cpu_count() or 1
+    return {"value": T * Bsz / sec, "unit": UNIT, "cores": cores, "kind": "oracle",
+            "sample": f"same step on T={T}, B={Bsz} of workload '{w.name}' (fp64 NumPy, {len(ts)} run(s), {sec:.2f} s each)"}, sec
+
+
+# ------------------------------------------------------------------------------------------ clocks
+class ClockSampler:
+    Q = "clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown," \
+        "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap"
+
+    def __init__(self, index):
+        self.p = None
+        try:
+            self.p = subprocess.Popen(["nvidia-smi", f"--query-gpu={self.Q}", "--format=csv,noheader,nounits", "-lms", "100",
+                                       "-i", str(index)], stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+        except Exception:
+            self.p = None
+
+    def stop(self):
+        if self.p is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": []}
+        self.p.terminate()
+        try:
+            out, _ = self.p.communicate(timeout=5)
+        except Exception:
+            self.p.kill()
+            out = ""
+        sm, mx, reasons = [], [], set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for line in out.strip().splitlines():
+            f = [s.strip() for s in line.split(",")]
+            if len(f) < 7:
+                continue
+            try:
+                sm.append(float(f[0])); mx.append(float(f[1]))
+            except ValueError:
+                continue
+            for n, v in zip(names, f[3:7]):
+                if v.lower().startswith("active"):
+                    reasons.add(n)
+        return {"sm_mhz": statistics.median(sm) if sm else None, "sm_max_mhz": max(mx) if mx else None,
+                "reasons": sorted(reasons), "samples": len(sm)}
+
+
+# ------------------------------------------------------------------------------------------ main
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=5)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--workload", default="train")
+    ap.add_argument("--T", type=int, default=None, help="override the sequence length (sweeps)")
+    ap.add_argument("--serial", action="store_true", help="time the GPU serial sweep + exact BPTT instead of MGRIT")
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-e2e", action="store_true")
+    args = ap.parse_args()
+
+    from paper_2203_04738_b200.synthetic import WORKLOADS, make_inputs
+    w = WORKLOADS[args.workload]
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    T = args.T or w.T
+    config = {"workload": f"{w.name}: {w.layers}-layer GRU I={w.I} H={w.H} B={w.B} T={T}, cf={w.cf}, levels={w.levels}, "
+                          f"iters fwd/adj={w.iters_fwd}/{w.iters_adj}, relax fine/coarse={'FCF' if w.relax_fine else 'F'}/"
+                          f"{'FCF' if w.relax_coarse else 'F'}, implicit cell, {w.classes}-class xent on h_T, SGD",
+              "solver": "serial sweep + BPTT" if args.serial else "MGRIT",
+              "l2": "inputs larger than L2 (x, gi and states are re-streamed from HBM every step)",
+              "parallelism": f"replicas x{args.gpus} (no sharding, no collective)"}
+
+    if args.impl == "reference":
+        if rank != 0:
+            return
+        cb, sec = time_oracle(w, steps=args.steps, warmup=min(args.warmup, 1))
+        print(json.dumps({"metric": METRIC, "value": cb["value"], "unit": UNIT, "n_gpus": args.gpus, "steps": args.steps,
+                          "warmup": args.warmup, "ms_per_step": sec * 1e3, "higher_is_better": True, "scaling": "weak",
+                          "vs_baseline": None, "dtype": "f64", "data": "synthetic", "config": config, "impl": "reference",
+                          "cpu_baseline": cb, "gpu_launches": 0,
+                          "e2e": {"value": cb["value"], "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0}}))
+        return
+
+    import torch
+    import torch.distributed as dist
+    from paper_2203_04738_b200 import binding as B
+    from paper_2203_04738_b200.train_step import alloc_buffers, training_step
+
+    torch.cuda.set_device(local_rank)
+    dev = torch.device("cuda", local_rank)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=dev)
+
+    d = make_inputs(w, T=T)
+    up = lambda a: torch.from_numpy(a).to(dev)
+    layers = [{n: up(l[n]) for n in ("W_ih", "W_hh", "b_ih", "b_hh")} for l in d["layers"]]
+    W_c, b_c, labels, h0 = up(d["W_c"]), up(d["b_c"]), up(d["labels"]), up(d["h0"])
+    x_host = torch.from_numpy(d["x"]).pin_memory()
+    x = x_host.to(dev)
+    buf = alloc_buffers(w, T, w.B, dev, serial=args.serial)
+    loss_host = torch.empty(1).pin_memory()
+
+    def step():
+        return training_step(w, layers, W_c, b_c, x, h0, labels, buf)
+
+    def barrier():
+        torch.cuda.synchronize()
+        if world > 1:
+            dist.barrier()
+            torch.cuda.synchronize()
+
+    for _ in range(max(args.warmup, 3)):
+        step()
+    barrier()
+    sampler = ClockSampler(local_rank) if rank == 0 else None
+    l0 = B.kernel_launches()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    barrier()
+    e0.record()
+    for _ in range(args.steps):
+        loss = step()
+    e1.record()
+    barrier()
+    ms = e0.elapsed_time(e1)
+    launches = B.kernel_launches() - l0
+    clocks = sampler.stop() if sampler else None
+    if world > 1:
+        t = torch.tensor([ms], device=dev)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        ms = float(t.item())
+    ms_step = ms / args.steps
+    value = world * T * w.B / (ms_step * 1e-3)
+
+    # end to end: inputs start in pinned host memory, the loss is read back, every step
+    e2e = None
+    if not args.no_e2e:
+        barrier()
+        e0.record()
+        for _ in range(args.steps):
+            x.copy_(x_host, non_blocking=True)
+            loss = step()
+            loss_host.copy_(loss, non_blocking=True)
+            torch.cuda.current_stream().synchronize()
+        e1.record()
+        barrier()
+        ms2 = e0.elapsed_time(e1)
+        if world > 1:
+            t = torch.tensor([ms2], device=dev)
+            dist.all_reduce(t, op=dist.ReduceOp.MAX)
+            ms2 = float(t.item())
+        e2e = {"value": world * T * w.B / (ms2 / args.steps * 1e-3), "unit": UNIT,
+               "h2d_bytes_per_step": x_host.numel() * 4, "d2h_bytes_per_step": 4}
+
+    # per-kernel timing pass (CUDA events around every GEMM-shaped launch; outside the timed region so
+    # that the event records do not perturb it)
+    roofline, breakdown = None, None
+    if rank == 0:
+        torch.cuda.synchronize()
+        B.profile_enable(True)
+        nprof = 2
+        for _ in range(nprof):
+            step()
+        prof = B.profile_read()
+        B.profile_enable(False)
+        peaks, pk = measured_peaks()
+        bf16 = w.operands == 2
+        breakdown = {k: {"ms_per_step": v[0] / nprof, "launches_per_step": v[1] // nprof,
+                         "tflops": (v[2] / (v[0] * 1e-3) / 1e12) if v[0] > 0 else None} for k, v in prof.items()}
+        dom = max(prof.items(), key=lambda kv: kv[1][0])
+        name, (tms, n, fl) = dom
+        if tms > 0 and n > 0:
+            achieved = fl / (tms * 1e-3) / 1e12
+            if bf16:
+                peak = float(peaks.get("bf16_tflops_sustained", peaks["bf16_tflops"]))
+                bound, note = "tensor", f"bf16 dense, sustained cuBLAS figure ({pk})"
+            else:
+                # fp32 FFMA: 148 SMs x 128 lanes x 2 flop x max SM clock
+                peak = 148 * 128 * 2 * float(peaks.get("sm_max_mhz", 1965.0)) * 1e6 / 1e12
+                bound, note = "alu", "fp32 FFMA: 148 SMs x 128 lanes x 2 flop x max SM clock"
+            roofline = {"kernel": name, "bound": bound, "achieved": achieved, "peak": peak, "unit": "TFLOP/s",
+                        "frac": achieved / peak, "traffic": NCU_TRAFFIC_BYTES_PER_LAUNCH.get(w.name),
+                        "avg_launch_us": tms / n * 1e3, "launches_per_step": n // nprof,
+                        "share_of_gemm_time": tms / max(sum(v[0] for v in prof.values()), 1e-9), "peak_source": note}
+
+    if rank != 0:
+        if world > 1:
+            dist.destroy_process_group()
+        return
+    cpu = None
+    if world == 1 and not args.no_cpu_baseline:
+        cpu, _ = time_oracle(w)
+    status = B.last_device_status()
+    out = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": max(args.warmup, 3),
+           "ms_per_step": ms_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+           "dtype": "bf16" if w.operands == 2 else "f32", "data": "synthetic", "config": config, "clocks": clocks,
+           "e2e": e2e, "gpu_launches": int(launches), "roofline": roofline, "cpu_baseline": cpu,
+           "kernel_breakdown": breakdown, "loss": float(loss.item()), "device_status": status}
+    print(json.dumps(out))
+    if world > 1:
+        dist.destroy_process_group()
+
+
+if __name__ == "__main__":
+    main()

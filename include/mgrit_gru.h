@@ -144,6 +144,15 @@ int mgrit_gru_last_device_status(void);
 /* Number of kernels this library has launched since it was loaded (all streams). */
 unsigned long long mgrit_gru_kernel_launches(void);
 
+/* Measurement aid (no counterpart in the paper): while enabled, every launch of a GEMM-shaped
+ * kernel is bracketed by CUDA events on its stream.  mgrit_gru_profile_enable(1) clears earlier
+ * records and starts recording, (0) stops.  mgrit_gru_profile_read synchronises the device and
+ * returns, for one kernel class, the summed launch durations (ms), the number of launches and
+ * their algorithmic flops (2*M*N*K).  Classes: 0 input projection, 1 forward relaxation step,
+ * 2 adjoint linearisation, 3 adjoint relaxation step, 4 weight/input gradient GEMMs. */
+int mgrit_gru_profile_enable(int on);
+int mgrit_gru_profile_read(int kernel_class, double* total_ms, unsigned long long* launches, double* flops);
+
 const char* mgrit_gru_strerror(int code);
 
 #ifdef __cplusplus

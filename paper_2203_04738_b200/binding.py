@@ -56,6 +56,9 @@ lib.xent_head_fwd_bwd.argtypes = [_i32, _i32, _i32, _vp, _vp, _vp, _vp, _vp, _vp
 lib.sgd_update.argtypes = [_vp, _vp, _sz, ctypes.c_float, _vp]
 lib.mgrit_gru_last_device_status.restype = ctypes.c_int
 lib.mgrit_gru_kernel_launches.restype = ctypes.c_ulonglong
+lib.mgrit_gru_profile_enable.argtypes = [ctypes.c_int]
+lib.mgrit_gru_profile_read.argtypes = [ctypes.c_int, ctypes.POINTER(ctypes.c_double), ctypes.POINTER(ctypes.c_ulonglong),
+                                       ctypes.POINTER(ctypes.c_double)]
 lib.mgrit_gru_strerror.argtypes = [ctypes.c_int]
 lib.mgrit_gru_strerror.restype = ctypes.c_char_p
 
@@ -203,3 +206,20 @@ def last_device_status() -> int:
 
 def kernel_launches() -> int:
     return int(lib.mgrit_gru_kernel_launches())
+
+
+KERNEL_CLASSES = ("input_projection", "forward_step", "adjoint_linearise", "adjoint_step", "gradient_gemms")
+
+
+def profile_enable(on: bool) -> None:
+    _check(lib.mgrit_gru_profile_enable(1 if on else 0))
+
+
+def profile_read():
+    """-> {class name: (total ms, launches, algorithmic flops)} for the launches recorded since profile_enable(True)."""
+    out = {}
+    for i, name in enumerate(KERNEL_CLASSES):
+        ms, n, fl = ctypes.c_double(0), ctypes.c_ulonglong(0), ctypes.c_double(0)
+        _check(lib.mgrit_gru_profile_read(i, ctypes.byref(ms), ctypes.byref(n), ctypes.byref(fl)))
+        out[name] = (ms.value, int(n.value), fl.value)
+    return out

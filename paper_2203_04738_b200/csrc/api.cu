@@ -5,12 +5,38 @@
 #include <stdio.h>
 #include <string.h>
 
+#include <vector>
+
 #include "common.cuh"
 #include "umma_engine.cuh"
 
 namespace mg {
 
 unsigned long long g_kernel_launches = 0;
+bool g_prof_on = false;
+
+namespace {
+struct ProfRec { int kc; double flops; cudaEvent_t e0, e1; };
+std::vector<ProfRec> g_prof_recs;
+std::vector<cudaEvent_t> g_prof_pool;
+cudaEvent_t prof_event() {
+  cudaEvent_t e = nullptr;
+  if (!g_prof_pool.empty()) { e = g_prof_pool.back(); g_prof_pool.pop_back(); }
+  else cudaEventCreate(&e);
+  return e;
+}
+}  // namespace
+
+void prof_begin(int kc, double flops, cudaStream_t s) {
+  if (!g_prof_on) return;
+  ProfRec r{kc, flops, prof_event(), prof_event()};
+  cudaEventRecord(r.e0, s);
+  g_prof_recs.push_back(r);
+}
+void prof_end(cudaStream_t s) {
+  if (!g_prof_on || g_prof_recs.empty()) return;
+  cudaEventRecord(g_prof_recs.back().e1, s);
+}
 
 namespace {
 
@@ -420,6 +446,29 @@ int mgrit_gru_last_device_status(void) {
 }
 
 unsigned long long mgrit_gru_kernel_launches(void) { return g_kernel_launches; }
+
+int mgrit_gru_profile_enable(int on) {
+  for (auto& r : g_prof_recs) { g_prof_pool.push_back(r.e0); g_prof_pool.push_back(r.e1); }
+  g_prof_recs.clear();
+  g_prof_on = on != 0;
+  return MGRIT_OK;
+}
+
+int mgrit_gru_profile_read(int kernel_class, double* total_ms, unsigned long long* launches, double* flops) {
+  if (kernel_class < 0 || kernel_class >= KC_COUNT) return MGRIT_INVALID_ARG;
+  if (cudaDeviceSynchronize() != cudaSuccess) return MGRIT_CUDA_ERROR;
+  double ms = 0, fl = 0; unsigned long long n = 0;
+  for (auto& r : g_prof_recs) {
+    if (r.kc != kernel_class) continue;
+    float t = 0.f;
+    if (cudaEventElapsedTime(&t, r.e0, r.e1) != cudaSuccess) return MGRIT_CUDA_ERROR;
+    ms += t; fl += r.flops; ++n;
+  }
+  if (total_ms) *total_ms = ms;
+  if (launches) *launches = n;
+  if (flops) *flops = fl;
+  return MGRIT_OK;
+}
 
 const char* mgrit_gru_strerror(int code) {
   switch (code) {

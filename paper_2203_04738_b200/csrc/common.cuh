@@ -15,6 +15,12 @@ typedef long long i64;
 extern unsigned long long g_kernel_launches;
 inline void count_launch(int n = 1) { g_kernel_launches += (unsigned long long)n; }
 
+// Optional per-launch timing of the GEMM-shaped kernels (CUDA events on the launching stream).
+enum KernelClass { KC_PROJ = 0, KC_FWD_STEP, KC_LINEARISE, KC_ADJ_STEP, KC_WGRAD, KC_COUNT };
+extern bool g_prof_on;
+void prof_begin(int kc, double flops, cudaStream_t s);
+void prof_end(cudaStream_t s);
+
 // ---- one forward cell evaluation for M = nk*B rows (Eq. "gru" + Eq. "gru-classic"/"gru-imap") ----
 // Row m = (k, b): k = m / B, b = m % B.  All *_ks are strides per k in ELEMENTS (may be negative).
 struct FwdStepArgs {

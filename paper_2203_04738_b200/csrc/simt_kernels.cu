@@ -70,10 +70,12 @@ __global__ void __launch_bounds__(NT) simt_gemm_kernel(int M, int N, int K, AL a
 }
 
 template <int NG, bool AKC, bool BKC, class AL, class BL, class Epi>
-void launch(int M, int N, int K, AL al, BL bl, Epi epi, cudaStream_t s) {
+void launch(int kc, int M, int N, int K, AL al, BL bl, Epi epi, cudaStream_t s) {
   if (M <= 0 || N <= 0) return;
   dim3 grid((M + BM - 1) / BM, (N + BN - 1) / BN);
+  prof_begin(kc, 2.0 * M * N * NG * K, s);
   simt_gemm_kernel<NG, AKC, BKC><<<grid, NT, 0, s>>>(M, N, K, al, bl, epi);
+  prof_end(s);
   count_launch();
 }
 
@@ -182,29 +184,29 @@ struct AdjEpi {
 }  // namespace
 
 void simt_project(const float* x, const float* W_ih, const float* b_ih, float* gi, int M, int I, int H3, cudaStream_t s) {
-  launch<1, true, true>(M, H3, I, DenseA{x, I}, DenseB{W_ih, I}, BiasEpi{gi, H3, b_ih}, s);
+  launch<1, true, true>(KC_PROJ, M, H3, I, DenseA{x, I}, DenseB{W_ih, I}, BiasEpi{gi, H3, b_ih}, s);
 }
 
 void simt_fwd_step(const FwdStepArgs& a, cudaStream_t s) {
-  launch<3, true, true>(a.M, a.H, a.H, StridedRowsA{a.hin, a.hin_ks, a.B, a.H}, GateW{a.W_hh, a.H, a.H}, FwdEpi{a}, s);
+  launch<3, true, true>(KC_FWD_STEP, a.M, a.H, a.H, StridedRowsA{a.hin, a.hin_ks, a.B, a.H}, GateW{a.W_hh, a.H, a.H}, FwdEpi{a}, s);
 }
 
 void simt_linearise(const LinArgs& a, cudaStream_t s) {
-  launch<3, true, true>(a.M, a.H, a.H, LinA{a.h0, a.h, a.stride_t, a.B, a.H}, GateW{a.W_hh, a.H, a.H}, LinEpi{a}, s);
+  launch<3, true, true>(KC_LINEARISE, a.M, a.H, a.H, LinA{a.h0, a.h, a.stride_t, a.B, a.H}, GateW{a.W_hh, a.H, a.H}, LinEpi{a}, s);
 }
 
 void simt_adj_step(const AdjStepArgs& a, cudaStream_t s) {
-  launch<1, true, false>(a.M, a.H, 3 * a.H, AdjA{a.lin, a.lin_ks, a.cr, a.cz, a.cn, a.coef_ks, a.B, a.H},
+  launch<1, true, false>(KC_ADJ_STEP, a.M, a.H, 3 * a.H, AdjA{a.lin, a.lin_ks, a.cr, a.cz, a.cn, a.coef_ks, a.B, a.H},
                          DenseBT{a.W_hh, a.H}, AdjEpi{a}, s);
 }
 
 void simt_wgrad(const float* dA, int M, int H3, const float* first, int Bfirst, const float* rest, int C, float* dW,
                 cudaStream_t s) {
-  launch<1, false, false>(H3, C, M, DenseAT{dA, H3}, FirstRestBT{first, Bfirst, rest, C}, StoreEpi{dW, C}, s);
+  launch<1, false, false>(KC_WGRAD, H3, C, M, DenseAT{dA, H3}, FirstRestBT{first, Bfirst, rest, C}, StoreEpi{dW, C}, s);
 }
 
 void simt_dgrad(const float* dA, int M, int H3, const float* W, int C, float* dx, cudaStream_t s) {
-  launch<1, true, false>(M, C, H3, DenseA{dA, H3}, DenseBT{W, C}, StoreEpi{dx, C}, s);
+  launch<1, true, false>(KC_WGRAD, M, C, H3, DenseA{dA, H3}, DenseBT{W, C}, StoreEpi{dx, C}, s);
 }
 
 }  // namespace mg

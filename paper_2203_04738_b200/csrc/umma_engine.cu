@@ -52,7 +52,7 @@ bool make_map(CUtensorMap* m, const bf16* base, uint64_t inner, uint64_t rows, u
 }
 
 template <int BN, bool GATES, class Epi>
-bool launch_gemm(const bf16* A, i64 lda, const bf16* Bm, i64 ldb, int M, int N, int K, int gate_rows, int b_rows, Epi epi,
+bool launch_gemm(int kc, const bf16* A, i64 lda, const bf16* Bm, i64 ldb, int M, int N, int K, int gate_rows, int b_rows, Epi epi,
                  cudaStream_t s) {
   using C = Cfg<BN, GATES>;
   if (M <= 0 || N <= 0) return true;
@@ -70,7 +70,9 @@ bool launch_gemm(const bf16* A, i64 lda, const bf16* Bm, i64 ldb, int M, int N, 
   int m_tiles = (M + BM - 1) / BM, n_tiles = (N + C::kNPerTile - 1) / C::kNPerTile;
   int tiles = m_tiles * n_tiles;
   int grid = tiles < kSMs ? tiles : kSMs;
+  prof_begin(kc, 2.0 * M * (GATES ? 3.0 * N : (double)N) * K, s);
   kern<<<grid, kThreads, C::kSmemBytes, s>>>(ta, tb, sh, epi, g_status_ptr);
+  prof_end(s);
   count_launch();
   return true;
 }
@@ -415,7 +417,7 @@ int umma_prepare_fwd(const mgrit_gru_cfg* c, const gru_params* p, const float* x
   convert(p->W_ih, w->W_ih, (i64)3 * H * I, s);
   convert(x, w->xb, TB * I, s);
   // gi = x W_ih^T + b_ih :  M = T*B, N = 3H, K = I
-  if (!launch_gemm<256, false>(w->xb, I, w->W_ih, I, (int)TB, 3 * H, I, 0, 3 * H, EpiBias{gi, 3 * H, p->b_ih, (int)TB, 3 * H}, s))
+  if (!launch_gemm<256, false>(KC_PROJ, w->xb, I, w->W_ih, I, (int)TB, 3 * H, I, 0, 3 * H, EpiBias{gi, 3 * H, p->b_ih, (int)TB, 3 * H}, s))
     return MGRIT_CUDA_ERROR;
   return MGRIT_OK;
 }
@@ -431,7 +433,7 @@ int umma_prepare_adj(const mgrit_gru_cfg* c, const gru_params* p, UmmaAdjWs* w, 
 void umma_fwd_step(const FwdStepArgs& a, UmmaFwdWs* w, cudaStream_t s) {
   pack_rows_kernel<<<pgrid((i64)a.M * (a.H / 4)), kPT, 0, s>>>(a.hin, a.hin_ks, a.B, a.H / 4, a.M, reinterpret_cast<uint2*>(w->Apack));
   count_launch();
-  launch_gemm<192, true>(w->Apack, a.H, w->W_hh, a.H, a.M, a.H, a.H, a.H, 3 * a.H, EpiFwd{a}, s);
+  launch_gemm<192, true>(KC_FWD_STEP, w->Apack, a.H, w->W_hh, a.H, a.M, a.H, a.H, a.H, 3 * a.H, EpiFwd{a}, s);
 }
 
 void umma_linearise(const LinArgs& a, UmmaAdjWs* w, cudaStream_t s) {
@@ -444,14 +446,14 @@ void umma_linearise(const LinArgs& a, UmmaAdjWs* w, cudaStream_t s) {
                                                                          a.M - a.B, reinterpret_cast<uint2*>(w->Apack + BH));
     count_launch();
   }
-  launch_gemm<192, true>(w->Apack, a.H, w->W_hh, a.H, a.M, a.H, a.H, a.H, 3 * a.H, EpiLin{a}, s);
+  launch_gemm<192, true>(KC_LINEARISE, w->Apack, a.H, w->W_hh, a.H, a.M, a.H, a.H, a.H, 3 * a.H, EpiLin{a}, s);
 }
 
 void umma_adj_step(const AdjStepArgs& a, UmmaAdjWs* w, cudaStream_t s) {
   pack_adj_kernel<<<pgrid((i64)a.M * (a.H / 4)), kPT, 0, s>>>(a.lin, a.lin_ks, a.cr, a.cz, a.cn, a.coef_ks, a.B, a.H / 4, a.M,
                                                               reinterpret_cast<uint2*>(w->Apack));
   count_launch();
-  launch_gemm<256, false>(w->Apack, 3 * a.H, w->W_hhT, 3 * a.H, a.M, a.H, 3 * a.H, 0, a.H, EpiAdj{a}, s);
+  launch_gemm<256, false>(KC_ADJ_STEP, w->Apack, 3 * a.H, w->W_hhT, 3 * a.H, a.M, a.H, 3 * a.H, 0, a.H, EpiAdj{a}, s);
 }
 
 int umma_gradients(const mgrit_gru_cfg* c, const gru_params* p, const float* x, const float* h0, const float* h, const float* lam,
@@ -472,10 +474,10 @@ int umma_gradients(const mgrit_gru_cfg* c, const gru_params* p, const float* x, 
   transpose(x, M, I, w->xT, M, 0, s);
   bool ok = true;
   // dW_hh[3H, H] = dA_h^T h_prev ;  dW_ih[3H, I] = dA_i^T x    (K = T*B)
-  ok = ok && launch_gemm<256, false>(w->dAhT, M, w->hprevT, M, 3 * H, H, (int)M, 0, H, EpiStore{g->dW_hh, H, 3 * H, H}, s);
-  ok = ok && launch_gemm<256, false>(w->dAiT, M, w->xT, M, 3 * H, I, (int)M, 0, I, EpiStore{g->dW_ih, I, 3 * H, I}, s);
+  ok = ok && launch_gemm<256, false>(KC_WGRAD, w->dAhT, M, w->hprevT, M, 3 * H, H, (int)M, 0, H, EpiStore{g->dW_hh, H, 3 * H, H}, s);
+  ok = ok && launch_gemm<256, false>(KC_WGRAD, w->dAiT, M, w->xT, M, 3 * H, I, (int)M, 0, I, EpiStore{g->dW_ih, I, 3 * H, I}, s);
   // dx[T*B, I] = dA_i W_ih   (K = 3H)
-  if (dx) ok = ok && launch_gemm<256, false>(w->dAi, 3 * H, w->W_ihT, 3 * H, (int)M, I, 3 * H, 0, I, EpiStore{dx, I, (int)M, I}, s);
+  if (dx) ok = ok && launch_gemm<256, false>(KC_WGRAD, w->dAi, 3 * H, w->W_ihT, 3 * H, (int)M, I, 3 * H, 0, I, EpiStore{dx, I, (int)M, I}, s);
   return ok ? MGRIT_OK : MGRIT_CUDA_ERROR;
 }
 

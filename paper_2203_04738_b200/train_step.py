@@ -1,0 +1,78 @@
+"""One training step of a stacked GRU whose layers are each solved by MGRIT: a fixed sequence
+of C-ABI calls (no arithmetic here).  Layer l+1 reads layer l's (inexact) hidden states; in the
+backward direction layer l+1's input gradient is layer l's direct loss derivative dh_seed."""
+from __future__ import annotations
+
+from dataclasses import dataclass, field
+
+import torch
+
+from . import binding as B
+from .synthetic import Workload
+
+
+@dataclass
+class StepBuffers:
+    """Device buffers reused across steps (allocated once; the library itself never allocates)."""
+    cfgs_fwd: list
+    cfgs_adj: list
+    ws_fwd: torch.Tensor
+    ws_adj: torch.Tensor
+    ws_head: torch.Tensor
+    gi: list
+    h: list
+    adj: list
+    serial: bool = False
+
+
+def make_cfgs(w: Workload, T: int, Bsz: int, serial: bool = False, flags: int = 0):
+    fw, ad = [], []
+    for l in range(w.layers):
+        I = w.I if l == 0 else w.H
+        kw = dict(cf=w.cf, levels=1 if serial else w.levels, cell=w.cell, relax_fine=w.relax_fine,
+                  relax_coarse=w.relax_coarse, operands=w.operands, flags=flags)
+        fw.append(B.make_cfg(T, Bsz, I, w.H, iters=w.iters_fwd, **kw))
+        ad.append(B.make_cfg(T, Bsz, I, w.H, iters=w.iters_adj, **kw))
+    return fw, ad
+
+
+def alloc_buffers(w: Workload, T: int, Bsz: int, device, serial: bool = False, flags: int = 0) -> StepBuffers:
+    fw, ad = make_cfgs(w, T, Bsz, serial, flags)
+    nf = max(B.workspace_bytes(c)[0] for c in fw)
+    na = max(B.workspace_bytes(c)[1] for c in ad)
+    mk = lambda *s: torch.empty(*s, device=device)
+    adj = []
+    for l, c in enumerate(ad):
+        adj.append(B.AdjointResult(dh=mk(T, Bsz, w.H), dh0=mk(Bsz, w.H), dx=mk(T, Bsz, c.I) if l > 0 else None,
+                                   dW_ih=mk(3 * w.H, c.I), dW_hh=mk(3 * w.H, w.H), db_ih=mk(3 * w.H), db_hh=mk(3 * w.H)))
+    return StepBuffers(fw, ad, torch.empty(nf, dtype=torch.uint8, device=device), torch.empty(na, dtype=torch.uint8, device=device),
+                       torch.empty(B.lib.xent_head_workspace_bytes(Bsz, w.classes), dtype=torch.uint8, device=device),
+                       [mk(T, Bsz, 3 * w.H) for _ in fw], [mk(T, Bsz, w.H) for _ in fw], adj, serial)
+
+
+def training_step(w: Workload, layers, W_c, b_c, x, h0, labels, buf: StepBuffers, lr: float = 1e-3, update: bool = True):
+    """Forward (all layers) -> loss head -> adjoint (top layer first) -> weight gradients -> SGD.
+    layers: list of dicts W_ih, W_hh, b_ih, b_hh (device fp32).  Returns the loss tensor (device)."""
+    inp = x
+    for l, p in enumerate(layers):
+        if buf.serial:
+            B.gru_serial_forward(buf.cfgs_fwd[l], p, inp, h0, gi=buf.gi[l], h=buf.h[l], ws=buf.ws_fwd)
+        else:
+            B.mgrit_gru_forward(buf.cfgs_fwd[l], p, inp, h0, gi=buf.gi[l], h=buf.h[l], ws=buf.ws_fwd)
+        inp = buf.h[l]
+    loss, dhT, dWc, dbc = B.xent_head_fwd_bwd(buf.h[-1][-1], W_c, b_c, labels, ws=buf.ws_head)
+    seed = None
+    for l in range(len(layers) - 1, -1, -1):
+        inp = x if l == 0 else buf.h[l - 1]
+        fn = B.gru_serial_backward if buf.serial else B.mgrit_gru_adjoint
+        fn(buf.cfgs_adj[l], layers[l], inp, h0, buf.gi[l], buf.h[l], dh_seed=seed, dhT=dhT if seed is None else None,
+           want_dx=l > 0, ws=buf.ws_adj, out=buf.adj[l])
+        seed = buf.adj[l].dx
+    if update:
+        for l, p in enumerate(layers):
+            a = buf.adj[l]
+            for name, g in (("W_ih", a.dW_ih), ("W_hh", a.dW_hh), ("b_ih", a.db_ih), ("b_hh", a.db_hh)):
+                B.sgd_update(p[name], g, lr)
+        B.sgd_update(W_c, dWc, lr)
+        B.sgd_update(b_c, dbc, lr)
+    return loss

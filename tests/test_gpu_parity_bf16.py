@@ -1,0 +1,166 @@
+"""GPU parity, bf16 tensor-core operand mode (tcgen05 GEMMs, fp32 accumulation, fp32 state), against the
+fp64 oracle at the same cycle count.  Tolerance: 2e-2 norm-relative (||a-b||_inf / ||b||_inf) on h, on
+every gradient and on dh; 1e-2 relative on residual norms.
+
+Small shapes are compared element by element over everything.  The full-size configurations are compared
+on sampled batch rows (rows of a batch never interact in the forward or adjoint recurrences, so the oracle
+can compute a few rows exactly as the full problem would) in the launch configuration the benchmark times.
+"""
+import numpy as np
+import pytest
+import torch
+
+from oracle import mgrit_gru_oracle as O
+from paper_2203_04738_b200.synthetic import WORKLOADS, Workload, make_inputs
+from tests.gpu_util import NAMES, max_abs, oracle_params, rel_inf, to_dev, upload
+
+pytestmark = pytest.mark.gpu
+TOL = 2e-2
+
+
+@pytest.fixture(scope="module")
+def B():
+    from paper_2203_04738_b200 import binding
+    return binding
+
+
+def _cfg(B, w, iters, T=None, Bsz=None, flags=0):
+    return B.make_cfg(T or w.T, Bsz or w.B, w.I, w.H, cf=w.cf, levels=w.levels, iters=iters, cell=w.cell,
+                      relax_fine=w.relax_fine, relax_coarse=w.relax_coarse, operands=B.OPERANDS_BF16, flags=flags)
+
+
+def _full_case(B, w, check_grads=True):
+    d = make_inputs(w)
+    p, x, h0 = upload(d)
+    P = oracle_params(d)
+    xr, h0r = d["x"].astype(np.float64), d["h0"].astype(np.float64)
+    kw = dict(cf=w.cf, levels=w.levels, relax_fine=w.relax_fine, relax_coarse=w.relax_coarse)
+    cfg = _cfg(B, w, w.iters_fwd)
+    h, gi, rn = B.mgrit_gru_forward(cfg, p, x, h0, want_resnorm=True)
+    href, rref = O.mgrit_forward(*P, xr, h0r, iters=w.iters_fwd, **kw)
+    assert rel_inf(gi.cpu().numpy(), O.input_projection(P[0], P[2], xr)) < TOL
+    assert rel_inf(h.cpu().numpy(), href) < TOL
+    for a, b in zip(rn, rref):
+        assert abs(a - b) <= 1e-2 * b
+    hs, _ = B.gru_serial_forward(cfg, p, x, h0)
+    assert rel_inf(hs.cpu().numpy(), O.serial_forward(*P, xr, h0r)) < TOL
+    if not check_grads:
+        return
+    loss, dhT, dWc, dbc = B.xent_head_fwd_bwd(h[-1].contiguous(), to_dev(d["W_c"]), to_dev(d["b_c"]), to_dev(d["labels"]))
+    hn = h.cpu().numpy().astype(np.float64)
+    rng = np.random.default_rng(3)
+    seed = (rng.standard_normal(hn.shape) * 1e-3).astype(np.float32)
+    seed64 = seed.astype(np.float64)
+    seed64[-1] += dhT.cpu().numpy()
+    cfga = _cfg(B, w, w.iters_adj)
+    r = B.mgrit_gru_adjoint(cfga, p, x, h0, gi, h, dh_seed=to_dev(seed), dhT=dhT, want_resnorm=True)
+    gi64 = None
+    lam, lam0, g, rref = O.mgrit_adjoint(*P, xr, h0r, hn, seed64, iters=w.iters_adj, **kw)
+    for a, b in zip(r.resnorm, rref):
+        assert abs(a - b) <= 1e-2 * b
+    assert rel_inf(r.dh.cpu().numpy(), lam) < TOL
+    assert max_abs(r.dh0.cpu().numpy(), lam0) / np.max(np.abs(lam)) < TOL
+    for k in ("dx", "dW_ih", "dW_hh", "db_ih", "db_hh"):
+        assert rel_inf(getattr(r, k).cpu().numpy(), g[k]) < TOL, k
+    # exact BPTT of the serial sweep
+    rs = B.gru_serial_backward(cfga, p, x, h0, gi, h, dh_seed=to_dev(seed), dhT=dhT)
+    lam_s, lam0_s, g_s = O.serial_backward(*P, xr, h0r, hn, seed64)
+    assert rel_inf(rs.dh.cpu().numpy(), lam_s) < TOL
+    for k in ("dx", "dW_ih", "dW_hh", "db_ih", "db_hh"):
+        assert rel_inf(getattr(rs, k).cpu().numpy(), g_s[k]) < TOL, k
+
+
+def test_small_two_level(B):
+    _full_case(B, Workload("s2", T=64, B=8, I=128, H=128, cf=4, levels=2, iters_fwd=2, iters_adj=2, relax_fine=0, relax_coarse=1,
+                           operands=2, classes=8, relu=True, seed=7))
+
+
+def test_small_ragged_three_level_fcf(B):
+    # rows per step 48*24 = 1152 (nine 128-row tiles, batch rows straddling tiles), H = 192 (three unit tiles,
+    # one partial 256-column tile in the adjoint GEMM), I = 80 (K tail of 16 in the projection)
+    _full_case(B, Workload("s3", T=96, B=24, I=80, H=192, cf=2, levels=3, iters_fwd=2, iters_adj=3, relax_fine=1, relax_coarse=1,
+                           operands=2, classes=8, relu=True, seed=8))
+
+
+def test_small_single_level_and_tiny_batch(B):
+    _full_case(B, Workload("s1", T=24, B=8, I=16, H=64, cf=2, levels=4, iters_fwd=3, iters_adj=1, relax_fine=0, relax_coarse=0,
+                           operands=2, classes=8, relu=False, seed=9))
+
+
+def test_medium_full(B):
+    # third configuration, everything compared: I=1024 H=512 B=32 T=1024, cf=4, 3 levels, 2 + 2 cycles
+    _full_case(B, WORKLOADS["medium"])
+
+
+def _sampled_rows_case(B, w, rows):
+    """Full-size run on the GPU; the oracle recomputes the batch rows `rows` of every layer."""
+    from paper_2203_04738_b200.train_step import alloc_buffers, training_step
+    d = make_inputs(w)
+    dev = torch.device("cuda")
+    layers = [{n: to_dev(l[n]) for n in NAMES} for l in d["layers"]]
+    W_c, b_c, labels, h0, x = to_dev(d["W_c"]), to_dev(d["b_c"]), to_dev(d["labels"]), to_dev(d["h0"]), to_dev(d["x"])
+    buf = alloc_buffers(w, w.T, w.B, dev)
+    training_step(w, layers, W_c, b_c, x, h0, labels, buf, update=False)
+    torch.cuda.synchronize()
+    assert B.last_device_status() == 0
+    kw = dict(cf=w.cf, levels=w.levels, relax_fine=w.relax_fine, relax_coarse=w.relax_coarse)
+    inp = d["x"][:, rows].astype(np.float64)
+    h0r = d["h0"][rows].astype(np.float64)
+    hs_gpu = []
+    for l in range(w.layers):
+        P = oracle_params(d, l)
+        href, _ = O.mgrit_forward(*P, inp, h0r, iters=w.iters_fwd, **kw)
+        hg = buf.h[l][:, rows].cpu().numpy()
+        assert rel_inf(hg, href) < TOL, ("h", l)
+        hs_gpu.append(hg.astype(np.float64))
+        inp = hs_gpu[-1]          # the next layer is fed what the GPU fed it
+    # adjoint of the sampled rows, linearised at the GPU's states, seeded with the GPU's loss gradient
+    # (which couples the rows through the batch mean only by a constant factor already inside dhT)
+    loss, dhT, dWc, dbc = B.xent_head_fwd_bwd(buf.h[-1][-1], W_c, b_c, labels)
+    lr, dh_r, _, _ = O.xent_head(buf.h[-1][-1].cpu().numpy().astype(np.float64), d["W_c"].astype(np.float64),
+                                 d["b_c"].astype(np.float64), d["labels"])
+    assert abs(loss.item() - lr) < 1e-4 and rel_inf(dhT.cpu().numpy(), dh_r) < 1e-3
+    seed = np.zeros_like(hs_gpu[-1])
+    seed[-1] = dhT[rows].cpu().numpy()
+    for l in range(w.layers - 1, -1, -1):
+        P = oracle_params(d, l)
+        inp = d["x"][:, rows].astype(np.float64) if l == 0 else hs_gpu[l - 1]
+        lam, lam0, g, _ = O.mgrit_adjoint(*P, inp, h0r, hs_gpu[l], seed, iters=w.iters_adj, want_dx=l > 0, **kw)
+        assert rel_inf(buf.adj[l].dh[:, rows].cpu().numpy(), lam) < TOL, ("dh", l)
+        if l > 0:
+            dxg = buf.adj[l].dx[:, rows].cpu().numpy()
+            assert rel_inf(dxg, g["dx"]) < TOL, ("dx", l)
+            seed = dxg.astype(np.float64)
+    for l in range(w.layers):
+        for k in ("dW_ih", "dW_hh", "db_ih", "db_hh"):
+            assert torch.isfinite(getattr(buf.adj[l], k)).all()
+
+
+def test_long_sampled_rows(B):
+    # fourth configuration at full size: I=2048 H=1024 B=8 T=4096, cf=8, 4 levels, 3 + 3 cycles
+    _sampled_rows_case(B, WORKLOADS["long"], [0, 5])
+
+
+def test_train_sampled_rows(B):
+    # fifth configuration at full size: 2 stacked layers, I=2048 H=1024 B=32 T=2048, cf=4, 3 levels, 2 + 2 cycles
+    _sampled_rows_case(B, WORKLOADS["train"], [3])
+
+
+def test_prefix_exactness_and_convergence_at_full_size(B):
+    # properties that hold at any size: after k cycles the first k*cf states equal the serial sweep, the residual
+    # falls from cycle to cycle, and more cycles approach the GPU's own serial sweep
+    w = WORKLOADS["long"]
+    d = make_inputs(w, T=1024)
+    p, x, h0 = upload(d)
+    cfg = _cfg(B, w, 3, T=1024)
+    h, gi, rn = B.mgrit_gru_forward(cfg, p, x, h0, want_resnorm=True)
+    hs, _ = B.gru_serial_forward(cfg, p, x, h0)
+    k = 3 * w.cf
+    assert rel_inf(h[:k].cpu().numpy(), hs[:k].cpu().numpy()) < 1e-2
+    assert rn[0] > rn[1] > rn[2]
+    e3 = rel_inf(h.cpu().numpy(), hs.cpu().numpy())
+    h8, _, _ = B.mgrit_gru_forward(_cfg(B, w, 8, T=1024), p, x, h0)
+    e8 = rel_inf(h8.cpu().numpy(), hs.cpu().numpy())
+    assert e8 < e3 and e8 < 2e-2
+    h_dup, _, _ = B.mgrit_gru_forward(_cfg(B, w, 3, T=1024, flags=B.FLAG_SKIP_DUPLICATE_FRELAX), p, x, h0)
+    assert torch.equal(h, h_dup)
