@@ -144,6 +144,7 @@ def main():
     ap.add_argument("--serial", action="store_true", help="time the GPU serial sweep + exact BPTT instead of MGRIT")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
+    ap.add_argument("--no-kernel-timing", action="store_true", help="skip the per-kernel CUDA-event pass")
     args = ap.parse_args()
 
     from paper_2203_04738_b200.synthetic import WORKLOADS, make_inputs
@@ -243,7 +244,7 @@ def main():
     # per-kernel timing pass (CUDA events around every GEMM-shaped launch; outside the timed region so
     # that the event records do not perturb it)
     roofline, breakdown = None, None
-    if rank == 0:
+    if rank == 0 and not args.no_kernel_timing:
         torch.cuda.synchronize()
         B.profile_enable(True)
         nprof = 2
