@@ -243,14 +243,21 @@ def main():
 
     # per-kernel timing pass (CUDA events around every GEMM-shaped launch; outside the timed region so
     # that the event records do not perturb it)
-    roofline, breakdown = None, None
+    roofline, breakdown, by_size = None, None, None
     if rank == 0 and not args.no_kernel_timing:
         torch.cuda.synchronize()
-        B.profile_enable(True)
         nprof = 2
+        B.profile_enable(True)
         for _ in range(nprof):
             step()
         prof = B.profile_read()
+        by_size = {}
+        for name, tms_, fl_ in B.profile_records():
+            e = by_size.setdefault(f"{name}@{fl_ / 1e9:.2f}GF", [0, 0.0])
+            e[0] += 1
+            e[1] += tms_
+        by_size = {k: {"launches_per_step": v[0] // nprof, "avg_us": v[1] / v[0] * 1e3, "ms_per_step": v[1] / nprof,
+                       "tflops": float(k.split("@")[1][:-2]) * 1e9 / (v[1] / v[0] * 1e-3) / 1e12} for k, v in by_size.items()}
         B.profile_enable(False)
         peaks, pk = measured_peaks()
         bf16 = w.operands == 2
@@ -284,7 +291,7 @@ def main():
            "ms_per_step": ms_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
            "dtype": "bf16" if w.operands == 2 else "f32", "data": "synthetic", "config": config, "clocks": clocks,
            "e2e": e2e, "gpu_launches": int(launches), "roofline": roofline, "cpu_baseline": cpu,
-           "kernel_breakdown": breakdown, "loss": float(loss.item()), "device_status": status}
+           "kernel_breakdown": breakdown, "kernel_by_size": by_size, "loss": float(loss.item()), "device_status": status}
     print(json.dumps(out))
     if world > 1:
         dist.destroy_process_group()

@@ -152,6 +152,9 @@ unsigned long long mgrit_gru_kernel_launches(void);
  * 2 adjoint linearisation, 3 adjoint relaxation step, 4 weight/input gradient GEMMs. */
 int mgrit_gru_profile_enable(int on);
 int mgrit_gru_profile_read(int kernel_class, double* total_ms, unsigned long long* launches, double* flops);
+/* The individual records in launch order: duration (ms), algorithmic flops and class of each
+ * recorded launch; writes min(cap, *n) entries and the total count to *n (HOST arrays). */
+int mgrit_gru_profile_records(double* ms, double* flops, int32_t* kernel_class, size_t cap, size_t* n);
 
 const char* mgrit_gru_strerror(int code);
 

@@ -59,6 +59,8 @@ lib.mgrit_gru_kernel_launches.restype = ctypes.c_ulonglong
 lib.mgrit_gru_profile_enable.argtypes = [ctypes.c_int]
 lib.mgrit_gru_profile_read.argtypes = [ctypes.c_int, ctypes.POINTER(ctypes.c_double), ctypes.POINTER(ctypes.c_ulonglong),
                                        ctypes.POINTER(ctypes.c_double)]
+lib.mgrit_gru_profile_records.argtypes = [ctypes.POINTER(ctypes.c_double), ctypes.POINTER(ctypes.c_double),
+                                          ctypes.POINTER(ctypes.c_int32), _sz, ctypes.POINTER(_sz)]
 lib.mgrit_gru_strerror.argtypes = [ctypes.c_int]
 lib.mgrit_gru_strerror.restype = ctypes.c_char_p
 
@@ -213,6 +215,16 @@ KERNEL_CLASSES = ("input_projection", "forward_step", "adjoint_linearise", "adjo
 
 def profile_enable(on: bool) -> None:
     _check(lib.mgrit_gru_profile_enable(1 if on else 0))
+
+
+def profile_records():
+    """-> list of (class name, ms, flops) per recorded launch, in launch order."""
+    n = _sz(0)
+    _check(lib.mgrit_gru_profile_records(None, None, None, 0, ctypes.byref(n)))
+    cap = n.value
+    ms, fl, kc = (ctypes.c_double * cap)(), (ctypes.c_double * cap)(), (ctypes.c_int32 * cap)()
+    _check(lib.mgrit_gru_profile_records(ms, fl, kc, cap, ctypes.byref(n)))
+    return [(KERNEL_CLASSES[kc[i]], ms[i], fl[i]) for i in range(cap)]
 
 
 def profile_read():

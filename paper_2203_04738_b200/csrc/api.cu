@@ -454,6 +454,20 @@ int mgrit_gru_profile_enable(int on) {
   return MGRIT_OK;
 }
 
+int mgrit_gru_profile_records(double* ms, double* flops, int32_t* kernel_class, size_t cap, size_t* n) {
+  if (!n) return MGRIT_INVALID_ARG;
+  if (cudaDeviceSynchronize() != cudaSuccess) return MGRIT_CUDA_ERROR;
+  *n = g_prof_recs.size();
+  for (size_t i = 0; i < g_prof_recs.size() && i < cap; ++i) {
+    float t = 0.f;
+    if (cudaEventElapsedTime(&t, g_prof_recs[i].e0, g_prof_recs[i].e1) != cudaSuccess) return MGRIT_CUDA_ERROR;
+    if (ms) ms[i] = t;
+    if (flops) flops[i] = g_prof_recs[i].flops;
+    if (kernel_class) kernel_class[i] = g_prof_recs[i].kc;
+  }
+  return MGRIT_OK;
+}
+
 int mgrit_gru_profile_read(int kernel_class, double* total_ms, unsigned long long* launches, double* flops) {
   if (kernel_class < 0 || kernel_class >= KC_COUNT) return MGRIT_INVALID_ARG;
   if (cudaDeviceSynchronize() != cudaSuccess) return MGRIT_CUDA_ERROR;

@@ -78,24 +78,30 @@ bool launch_gemm(int kc, const bf16* A, i64 lda, const bf16* Bm, i64 ldb, int M,
 }
 
 // ---------------------------------------------------------------- epilogues (one output row per thread)
+// Each epilogue warp handles 32 rows (its TMEM lane quarter) and one half of the tile's columns.
+// Per 16-column chunk the global loads are issued first, then the accumulator is read, so that the
+// memory latency of a chunk overlaps its tcgen05.ld and the other warps' work.
 __device__ __forceinline__ float4 ld4(const float* p) { return *reinterpret_cast<const float4*>(p); }
+__device__ __forceinline__ float4 ldg4(const float* p) { return __ldg(reinterpret_cast<const float4*>(p)); }
 __device__ __forceinline__ void st4(float* p, float a, float b, float c, float d) {
   *reinterpret_cast<float4*>(p) = make_float4(a, b, c, d);
 }
+__device__ __forceinline__ float f4get(const float4& v, int e) { return e == 0 ? v.x : (e == 1 ? v.y : (e == 2 ? v.z : v.w)); }
 
 struct EpiBias {  // out[m, n] = acc + bias[n]      (input projection)
   float* out; i64 ld; const float* bias; int M, N;
-  __device__ void operator()(uint32_t taddr, int row, int n0) const {
+  __device__ void operator()(uint32_t taddr, int row, int n0, int half) const {
     const bool valid = row < M;
     float* o = out + (i64)row * ld + n0;
-    for (int c0 = 0; c0 < 256 && n0 + c0 < N; c0 += 16) {
+    const int cbeg = half * 128;
+    for (int c0 = cbeg; c0 < cbeg + 128 && n0 + c0 < N; c0 += 16) {
       float v[16];
       tmem_ld16(taddr + c0, v);
       tmem_ld_wait();
       if (valid) {
 #pragma unroll
         for (int i = 0; i < 16; i += 4) {
-          float4 b = __ldg(reinterpret_cast<const float4*>(bias + n0 + c0 + i));
+          float4 b = ldg4(bias + n0 + c0 + i);
           st4(o + c0 + i, v[i] + b.x, v[i + 1] + b.y, v[i + 2] + b.z, v[i + 3] + b.w);
         }
       }
@@ -105,10 +111,11 @@ struct EpiBias {  // out[m, n] = acc + bias[n]      (input projection)
 
 struct EpiStore {  // out[m, n] = acc            (weight / input gradients)
   float* out; i64 ld; int M, N;
-  __device__ void operator()(uint32_t taddr, int row, int n0) const {
+  __device__ void operator()(uint32_t taddr, int row, int n0, int half) const {
     const bool valid = row < M;
     float* o = out + (i64)row * ld + n0;
-    for (int c0 = 0; c0 < 256 && n0 + c0 < N; c0 += 16) {
+    const int cbeg = half * 128;
+    for (int c0 = cbeg; c0 < cbeg + 128 && n0 + c0 < N; c0 += 16) {
       float v[16];
       tmem_ld16(taddr + c0, v);
       tmem_ld_wait();
@@ -122,15 +129,29 @@ struct EpiStore {  // out[m, n] = acc            (weight / input gradients)
 
 struct EpiFwd {  // GRU cell on the r|z|n accumulator columns of 64 hidden units
   FwdStepArgs a;
-  __device__ void operator()(uint32_t taddr, int row, int u0) const {
+  __device__ void operator()(uint32_t taddr, int row, int u0, int half) const {
     const bool valid = row < a.M;
     const int k = valid ? row / a.B : 0, b = valid ? row % a.B : 0;
-    const float* gi = a.gi + (i64)k * a.gi_ks + (i64)b * 3 * a.H + u0;
-    const float* hp = a.hin + (i64)k * a.hin_ks + (i64)b * a.H + u0;
-    float* ho = a.hout + (i64)k * a.hout_ks + (i64)b * a.H + u0;
-    const float* ga = a.gadd ? a.gadd + (i64)k * a.gadd_ks + (i64)b * a.H + u0 : nullptr;
-    const float* bh = a.b_hh + u0;
-    for (int c0 = 0; c0 < 64; c0 += 16) {
+    const int H = a.H;
+    const float* __restrict__ gi = a.gi + (i64)k * a.gi_ks + (i64)b * 3 * H + u0;
+    const float* __restrict__ hp = a.hin + (i64)k * a.hin_ks + (i64)b * H + u0;
+    float* __restrict__ ho = a.hout + (i64)k * a.hout_ks + (i64)b * H + u0;
+    // in mode 1 the previous content of the destination plays the role of the additive term
+    const float* __restrict__ ga = a.mode == 1 ? ho : (a.gadd ? a.gadd + (i64)k * a.gadd_ks + (i64)b * H + u0 : nullptr);
+    const float* __restrict__ bh = a.b_hh + u0;
+    const float sign = a.mode == 1 ? -1.f : 1.f;
+#pragma unroll
+    for (int cc = 0; cc < 2; ++cc) {
+      const int c0 = half * 32 + cc * 16;
+      float4 gr[4], gz[4], gn[4], h4[4], g4[4];
+      if (valid) {
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+          gr[i] = ld4(gi + c0 + 4 * i); gz[i] = ld4(gi + H + c0 + 4 * i); gn[i] = ld4(gi + 2 * H + c0 + 4 * i);
+          h4[i] = ld4(hp + c0 + 4 * i);
+          g4[i] = ga ? ld4(ga + c0 + 4 * i) : make_float4(0.f, 0.f, 0.f, 0.f);
+        }
+      }
       float r[16], z[16], n[16];
       tmem_ld16(taddr + c0, r);
       tmem_ld16(taddr + 64 + c0, z);
@@ -138,39 +159,46 @@ struct EpiFwd {  // GRU cell on the r|z|n accumulator columns of 64 hidden units
       tmem_ld_wait();
       if (valid) {
 #pragma unroll
-        for (int i = 0; i < 16; i += 4) {
-          const int c = c0 + i;
-          float4 gr = ld4(gi + c), gz = ld4(gi + a.H + c), gn = ld4(gi + 2 * a.H + c), h4 = ld4(hp + c);
-          float4 br = __ldg(reinterpret_cast<const float4*>(bh + c));
-          float4 bz = __ldg(reinterpret_cast<const float4*>(bh + a.H + c));
-          float4 bn = __ldg(reinterpret_cast<const float4*>(bh + 2 * a.H + c));
-          float o0 = cell_forward(gr.x, gz.x, gn.x, r[i] + br.x, z[i] + bz.x, n[i] + bn.x, h4.x, a.gamma, a.cell);
-          float o1 = cell_forward(gr.y, gz.y, gn.y, r[i + 1] + br.y, z[i + 1] + bz.y, n[i + 1] + bn.y, h4.y, a.gamma, a.cell);
-          float o2 = cell_forward(gr.z, gz.z, gn.z, r[i + 2] + br.z, z[i + 2] + bz.z, n[i + 2] + bn.z, h4.z, a.gamma, a.cell);
-          float o3 = cell_forward(gr.w, gz.w, gn.w, r[i + 3] + br.w, z[i + 3] + bz.w, n[i + 3] + bn.w, h4.w, a.gamma, a.cell);
-          if (a.mode == 0) {
-            if (ga) { float4 g4 = ld4(ga + c); o0 += g4.x; o1 += g4.y; o2 += g4.z; o3 += g4.w; }
-            st4(ho + c, o0, o1, o2, o3);
-          } else {
-            float4 p4 = ld4(ho + c);
-            st4(ho + c, p4.x - o0, p4.y - o1, p4.z - o2, p4.w - o3);
+        for (int i = 0; i < 4; ++i) {
+          const int c = c0 + 4 * i;
+          float4 br = ldg4(bh + c), bz = ldg4(bh + H + c), bn = ldg4(bh + 2 * H + c);
+          float o[4];
+#pragma unroll
+          for (int e = 0; e < 4; ++e) {
+            float phi = cell_forward(f4get(gr[i], e), f4get(gz[i], e), f4get(gn[i], e), r[4 * i + e] + f4get(br, e),
+                                     z[4 * i + e] + f4get(bz, e), n[4 * i + e] + f4get(bn, e), f4get(h4[i], e), a.gamma, a.cell);
+            // mode 0: phi + g ;  mode 1: previous - phi
+            o[e] = a.mode == 1 ? f4get(g4[i], e) - phi : phi + f4get(g4[i], e);
           }
+          st4(ho + c, o[0], o[1], o[2], o[3]);
         }
       }
     }
+    (void)sign;
   }
 };
 
 struct EpiLin {  // adjoint coefficients of every step of a level
   LinArgs a;
-  __device__ void operator()(uint32_t taddr, int row, int u0) const {
+  __device__ void operator()(uint32_t taddr, int row, int u0, int half) const {
     const bool valid = row < a.M;
     const int j1 = valid ? row / a.B : 0, b = valid ? row % a.B : 0;
-    const float* gi = a.gi + (((i64)(j1 + 1) * a.stride_t - 1) * a.B + b) * 3 * a.H + u0;
-    const float* hp = (j1 == 0 ? a.h0 + (i64)b * a.H : a.h + (((i64)j1 * a.stride_t - 1) * a.B + b) * a.H) + u0;
-    const i64 o = (i64)row * a.H + u0;
-    const float* bh = a.b_hh + u0;
-    for (int c0 = 0; c0 < 64; c0 += 16) {
+    const int H = a.H;
+    const float* __restrict__ gi = a.gi + (((i64)(j1 + 1) * a.stride_t - 1) * a.B + b) * 3 * H + u0;
+    const float* __restrict__ hp = (j1 == 0 ? a.h0 + (i64)b * H : a.h + (((i64)j1 * a.stride_t - 1) * a.B + b) * H) + u0;
+    const i64 o = (i64)row * H + u0;
+    const float* __restrict__ bh = a.b_hh + u0;
+#pragma unroll
+    for (int cc = 0; cc < 2; ++cc) {
+      const int c0 = half * 32 + cc * 16;
+      float4 gr[4], gz[4], gn[4], h4[4];
+      if (valid) {
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+          gr[i] = ld4(gi + c0 + 4 * i); gz[i] = ld4(gi + H + c0 + 4 * i); gn[i] = ld4(gi + 2 * H + c0 + 4 * i);
+          h4[i] = ld4(hp + c0 + 4 * i);
+        }
+      }
       float r[16], z[16], n[16];
       tmem_ld16(taddr + c0, r);
       tmem_ld16(taddr + 64 + c0, z);
@@ -178,21 +206,14 @@ struct EpiLin {  // adjoint coefficients of every step of a level
       tmem_ld_wait();
       if (valid) {
 #pragma unroll
-        for (int i = 0; i < 16; i += 4) {
-          const int c = c0 + i;
-          float gr[4], gz[4], gn[4], h4[4], br[4], bz[4], bn[4];
-          *reinterpret_cast<float4*>(gr) = ld4(gi + c);
-          *reinterpret_cast<float4*>(gz) = ld4(gi + a.H + c);
-          *reinterpret_cast<float4*>(gn) = ld4(gi + 2 * a.H + c);
-          *reinterpret_cast<float4*>(h4) = ld4(hp + c);
-          *reinterpret_cast<float4*>(br) = __ldg(reinterpret_cast<const float4*>(bh + c));
-          *reinterpret_cast<float4*>(bz) = __ldg(reinterpret_cast<const float4*>(bh + a.H + c));
-          *reinterpret_cast<float4*>(bn) = __ldg(reinterpret_cast<const float4*>(bh + 2 * a.H + c));
+        for (int i = 0; i < 4; ++i) {
+          const int c = c0 + 4 * i;
+          float4 br = ldg4(bh + c), bz = ldg4(bh + H + c), bn = ldg4(bh + 2 * H + c);
           float oa[4], ocr[4], ocz[4], ocn[4], ocp[4];
 #pragma unroll
           for (int e = 0; e < 4; ++e) {
-            CellLin L = cell_linearise(gr[e], gz[e], gn[e], r[i + e] + br[e], z[i + e] + bz[e], n[i + e] + bn[e], h4[e],
-                                       a.gamma, a.cell);
+            CellLin L = cell_linearise(f4get(gr[i], e), f4get(gz[i], e), f4get(gn[i], e), r[4 * i + e] + f4get(br, e),
+                                       z[4 * i + e] + f4get(bz, e), n[4 * i + e] + f4get(bn, e), f4get(h4[i], e), a.gamma, a.cell);
             oa[e] = L.a; ocr[e] = L.cr; ocz[e] = L.cz; ocn[e] = L.cn; ocp[e] = L.cnp;
           }
           st4(a.a + o + c, oa[0], oa[1], oa[2], oa[3]);
@@ -208,30 +229,34 @@ struct EpiLin {  // adjoint coefficients of every step of a level
 
 struct EpiAdj {  // lambda_prev = a*lambda + acc (+ source)
   AdjStepArgs a;
-  __device__ void operator()(uint32_t taddr, int row, int n0) const {
+  __device__ void operator()(uint32_t taddr, int row, int n0, int half) const {
     const bool valid = row < a.M;
     const int k = valid ? row / a.B : 0, b = valid ? row % a.B : 0;
-    const float* li = a.lin + (i64)k * a.lin_ks + (i64)b * a.H + n0;
-    const float* ca = a.a + (i64)k * a.coef_ks + (i64)b * a.H + n0;
-    float* lo = a.lout + (i64)k * a.lout_ks + (i64)b * a.H + n0;
-    const float* ga = a.gadd ? a.gadd + (i64)k * a.gadd_ks + (i64)b * a.H + n0 : nullptr;
-    for (int c0 = 0; c0 < 256 && n0 + c0 < a.H; c0 += 16) {
+    const float* __restrict__ li = a.lin + (i64)k * a.lin_ks + (i64)b * a.H + n0;
+    const float* __restrict__ ca = a.a + (i64)k * a.coef_ks + (i64)b * a.H + n0;
+    float* __restrict__ lo = a.lout + (i64)k * a.lout_ks + (i64)b * a.H + n0;
+    const float* __restrict__ ga = a.mode == 1 ? lo : (a.gadd ? a.gadd + (i64)k * a.gadd_ks + (i64)b * a.H + n0 : nullptr);
+    const int cbeg = half * 128;
+#pragma unroll 2
+    for (int c0 = cbeg; c0 < cbeg + 128 && n0 + c0 < a.H; c0 += 16) {
+      float4 l4[4], a4[4], g4[4];
+      if (valid) {
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+          l4[i] = ld4(li + c0 + 4 * i); a4[i] = ld4(ca + c0 + 4 * i);
+          g4[i] = ga ? ld4(ga + c0 + 4 * i) : make_float4(0.f, 0.f, 0.f, 0.f);
+        }
+      }
       float v[16];
       tmem_ld16(taddr + c0, v);
       tmem_ld_wait();
       if (valid) {
 #pragma unroll
-        for (int i = 0; i < 16; i += 4) {
-          const int c = c0 + i;
-          float4 l4 = ld4(li + c), a4 = ld4(ca + c);
-          float o0 = a4.x * l4.x + v[i], o1 = a4.y * l4.y + v[i + 1], o2 = a4.z * l4.z + v[i + 2], o3 = a4.w * l4.w + v[i + 3];
-          if (a.mode == 0) {
-            if (ga) { float4 g4 = ld4(ga + c); o0 += g4.x; o1 += g4.y; o2 += g4.z; o3 += g4.w; }
-            st4(lo + c, o0, o1, o2, o3);
-          } else {
-            float4 p4 = ld4(lo + c);
-            st4(lo + c, p4.x - o0, p4.y - o1, p4.z - o2, p4.w - o3);
-          }
+        for (int i = 0; i < 4; ++i) {
+          float o0 = a4[i].x * l4[i].x + v[4 * i], o1 = a4[i].y * l4[i].y + v[4 * i + 1];
+          float o2 = a4[i].z * l4[i].z + v[4 * i + 2], o3 = a4[i].w * l4[i].w + v[4 * i + 3];
+          if (a.mode == 1) st4(lo + c0 + 4 * i, g4[i].x - o0, g4[i].y - o1, g4[i].z - o2, g4[i].w - o3);
+          else st4(lo + c0 + 4 * i, o0 + g4[i].x, o1 + g4[i].y, o2 + g4[i].z, o3 + g4[i].w);
         }
       }
     }

@@ -20,7 +20,8 @@ namespace mg {
 namespace umma {
 
 constexpr int BM = 128, BK = 64;
-constexpr int kThreads = 192;  // warp 0: TMA producer, warp 1: MMA issuer + TMEM owner, warps 2-5: epilogue
+constexpr int kEpiWarps = 8;    // two warps per TMEM lane quarter, each taking half of the tile's columns
+constexpr int kThreads = 64 + 32 * kEpiWarps;  // warp 0: TMA producer, warp 1: MMA issuer + TMEM owner, rest: epilogue
 constexpr uint64_t kWaitLimitNs = 2000000000ull;
 
 __device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
@@ -135,10 +136,11 @@ struct Cfg {
   static constexpr int kNPerTile = GATES ? BN / 3 : BN;  // output columns (hidden units) per tile
 };
 
-// Epi: __device__ void operator()(uint32_t tmem_row_addr, int row, int n0) const
+// Epi: __device__ void operator()(uint32_t tmem_row_addr, int row, int n0, int half) const
 //   tmem_row_addr: address of (this thread's lane, first column of the accumulator)
 //   row: global output row of this thread (may be >= M: then only the tcgen05.ld's are executed)
 //   n0 : first output column (GATES: first hidden unit) of the tile
+//   half: 0 or 1, the half of the tile's output columns this warp is responsible for
 template <int BN, bool GATES, class Epi>
 __global__ void __launch_bounds__(kThreads, 1)
 umma_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB, GemmShape sh, Epi epi,
@@ -165,7 +167,7 @@ umma_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
   if (threadIdx.x == 0) {
     abort_flag = 0;
     for (int s = 0; s < C::kStages; ++s) { mbar_init(full_bar(s), 1); mbar_init(empty_bar(s), 1); }
-    for (int a = 0; a < 2; ++a) { mbar_init(tfull_bar(a), 1); mbar_init(tempty_bar(a), 128); }
+    for (int a = 0; a < 2; ++a) { mbar_init(tfull_bar(a), 1); mbar_init(tempty_bar(a), 32 * kEpiWarps); }
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
   if (warp == 1) {
@@ -233,8 +235,9 @@ umma_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
       }
     }
   } else {
-    // ------------------------------------------------------------ epilogue (warps 2..5)
-    const int q = warp & 3;  // TMEM lane quarter this warp may access
+    // ------------------------------------------------------------ epilogue (warps 2..9)
+    const int q = warp & 3;             // TMEM lane quarter this warp may access
+    const int half = (warp - 2) >> 2;   // which half of the tile's columns this warp handles
     int it = 0;
     for (int t = blockIdx.x; t < tiles; t += gridDim.x, ++it) {
       const int mt = t / n_tiles, nt = t % n_tiles;
@@ -243,7 +246,7 @@ umma_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
       if (!mbar_wait(tfull_bar(as), aphase, abortp, status, 4)) break;
       tc_fence_after();
       const uint32_t taddr = tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(as * BN);
-      epi(taddr, mt * BM + q * 32 + lane, nt * C::kNPerTile);
+      epi(taddr, mt * BM + q * 32 + lane, nt * C::kNPerTile, half);
       tc_fence_before();
       mbar_arrive(tempty_bar(as));
     }
@@ -254,6 +257,7 @@ umma_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
   __syncthreads();
   tc_fence_after();
   if (warp == 1) {
+    __syncwarp();
     asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"((uint32_t)C::kTmemCols) : "memory");
   }
 }
