@@ -149,7 +149,8 @@ unsigned long long mgrit_gru_kernel_launches(void);
  * records and starts recording, (0) stops.  mgrit_gru_profile_read synchronises the device and
  * returns, for one kernel class, the summed launch durations (ms), the number of launches and
  * their algorithmic flops (2*M*N*K).  Classes: 0 input projection, 1 forward relaxation step,
- * 2 adjoint linearisation, 3 adjoint relaxation step, 4 weight/input gradient GEMMs. */
+ * 2 adjoint linearisation, 3 adjoint relaxation step, 4 weight/input gradient GEMMs, 5 / 6 forward /
+ * adjoint persistent serial chain (all dependent steps of the coarsest level in one launch). */
 int mgrit_gru_profile_enable(int on);
 int mgrit_gru_profile_read(int kernel_class, double* total_ms, unsigned long long* launches, double* flops);
 /* The individual records in launch order: duration (ms), algorithmic flops and class of each

@@ -210,7 +210,8 @@ def kernel_launches() -> int:
     return int(lib.mgrit_gru_kernel_launches())
 
 
-KERNEL_CLASSES = ("input_projection", "forward_step", "adjoint_linearise", "adjoint_step", "gradient_gemms")
+KERNEL_CLASSES = ("input_projection", "forward_step", "adjoint_linearise", "adjoint_step", "gradient_gemms",
+                  "forward_serial_chain", "adjoint_serial_chain")
 
 
 def profile_enable(on: bool) -> None:

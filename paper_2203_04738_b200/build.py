@@ -8,7 +8,7 @@ import sys
 HERE = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(HERE, "csrc")
 LIB = os.path.join(HERE, "libmgrit_gru.so")
-SOURCES = ["api.cu", "simt_kernels.cu", "stream_kernels.cu", "umma_engine.cu"]
+SOURCES = ["api.cu", "simt_kernels.cu", "stream_kernels.cu", "umma_engine.cu", "serial_kernels.cu"]
 FLAGS = ["-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
          "-Xcompiler", "-fPIC", "-shared"]
 

@@ -8,6 +8,7 @@
 #include <vector>
 
 #include "common.cuh"
+#include "serial_engine.cuh"
 #include "umma_engine.cuh"
 
 namespace mg {
@@ -88,11 +89,13 @@ int check_cfg(const mgrit_gru_cfg* c, Hier* hr) {
 
 struct FwdWs {
   float* U[kMaxLevels]; float* G[kMaxLevels]; double* res_acc; UmmaFwdWs um;
+  __nv_bfloat16* chain_ub; unsigned* chain_bar;   // scratch of the persistent serial-chain kernel
 };
 struct AdjWs {
   float* U[kMaxLevels]; float* G[kMaxLevels];
   float *a[kMaxLevels], *cr[kMaxLevels], *cz[kMaxLevels], *cn[kMaxLevels], *cnp;
   float *dA_h, *dA_i; double* res_acc; UmmaAdjWs um;
+  __nv_bfloat16* chain_dAb; unsigned* chain_bar;
 };
 
 void plan_fwd(const mgrit_gru_cfg* c, const Hier& hr, Ws& w, FwdWs* o) {
@@ -102,7 +105,12 @@ void plan_fwd(const mgrit_gru_cfg* c, const Hier& hr, Ws& w, FwdWs* o) {
     o->G[l] = l == 0 ? nullptr : w.take<float>((size_t)(hr.N[l] + 1) * BH);
   }
   o->res_acc = w.take<double>((size_t)(c->iters > 0 ? c->iters : 1));
-  if (c->operands == MGRIT_OPERANDS_BF16) umma_plan_fwd(c, hr.N, hr.L, w.base, &w.off, &o->um);
+  o->chain_ub = nullptr; o->chain_bar = nullptr;
+  if (c->operands == MGRIT_OPERANDS_BF16) {
+    umma_plan_fwd(c, hr.N, hr.L, w.base, &w.off, &o->um);
+    o->chain_ub = w.take<__nv_bfloat16>(2 * BH);
+    o->chain_bar = w.take<unsigned>(64 + (size_t)c->B / 16);
+  }
 }
 
 void plan_adj(const mgrit_gru_cfg* c, const Hier& hr, Ws& w, AdjWs* o) {
@@ -120,7 +128,10 @@ void plan_adj(const mgrit_gru_cfg* c, const Hier& hr, Ws& w, AdjWs* o) {
   if (c->operands == MGRIT_OPERANDS_BF16) {
     o->dA_h = o->dA_i = nullptr;
     umma_plan_adj(c, hr.N, hr.L, w.base, &w.off, &o->um);
+    o->chain_dAb = w.take<__nv_bfloat16>(6 * BH);
+    o->chain_bar = w.take<unsigned>(64 + (size_t)c->B / 16);
   } else {
+    o->chain_dAb = nullptr; o->chain_bar = nullptr;
     o->dA_h = w.take<float>((size_t)c->T * BH * 3);
     o->dA_i = w.take<float>((size_t)c->T * BH * 3);
   }
@@ -143,6 +154,8 @@ struct Cycle {
   float** U; float** G; double* res_acc; int cycle_idx = 0;
   size_t BH;
   virtual void step(const StepDesc& d) = 0;
+  // all N_l dependent steps of level l in one persistent launch; false = not available here
+  virtual bool chain(int l) { (void)l; return false; }
   virtual ~Cycle() {}
 
   void frelax(int l) {
@@ -157,6 +170,7 @@ struct Cycle {
   void vcycle(int l) {
     int cf = c->cf, N = hr.N[l];
     if (l == hr.L - 1) {  // coarsest level: serial propagation
+      if (chain(l)) return;
       for (int j = 1; j <= N; ++j) step(StepDesc{l, 1, j - 1, 1, U[l], j, 1, G[l], j, 1, j, 1, 0});
       return;
     }
@@ -183,7 +197,17 @@ struct Cycle {
 };
 
 struct FwdCycle : Cycle {
-  const gru_params* p; const float* gi; UmmaFwdWs* um;
+  const gru_params* p; const float* gi; UmmaFwdWs* um; FwdWs* fw;
+  bool chain(int l) override {
+    if (c->operands != MGRIT_OPERANDS_BF16 || !fw->chain_ub) return false;
+    SerialFwdArgs a;
+    a.B = c->B; a.H = c->H; a.nsteps = hr.N[l];
+    a.u = U[l]; a.ub = fw->chain_ub;
+    i64 st = hr.stride_t[l];
+    a.gi = gi + (st - 1) * (i64)BH * 3; a.gi_step = st * (i64)BH * 3;
+    a.g = G[l]; a.W = um->W_hh; a.b_hh = p->b_hh; a.gamma = hr.gamma[l]; a.cell = c->cell; a.bar = fw->chain_bar;
+    return serial_fwd_solve(a, s);
+  }
   void step(const StepDesc& d) override {
     FwdStepArgs a;
     a.M = d.nk * c->B; a.B = c->B; a.H = c->H;
@@ -199,6 +223,17 @@ struct FwdCycle : Cycle {
 
 struct AdjCycle : Cycle {
   const gru_params* p; AdjWs* w;
+  bool chain(int l) override {
+    if (c->operands != MGRIT_OPERANDS_BF16 || !w->chain_dAb) return false;
+    SerialAdjArgs a;
+    a.B = c->B; a.H = c->H; a.nsteps = hr.N[l];
+    a.mu = U[l]; a.dAb = w->chain_dAb;
+    i64 row0 = (i64)(hr.N[l] - 1) * BH;        // step s = 1 applies forward step N_l, stored at row N_l - 1
+    a.a = w->a[l] + row0; a.cr = w->cr[l] + row0; a.cz = w->cz[l] + row0; a.cn = w->cn[l] + row0;
+    a.coef_step = -(i64)BH;
+    a.g = G[l]; a.WT = w->um.W_hhT; a.bar = w->chain_bar;
+    return serial_adj_solve(a, s);
+  }
   void step(const StepDesc& d) override {
     AdjStepArgs a;
     a.M = d.nk * c->B; a.B = c->B; a.H = c->H;
@@ -218,7 +253,7 @@ int finish(cudaStream_t s, bool sync) {
   if (sync && cudaStreamSynchronize(s) != cudaSuccess) return MGRIT_CUDA_ERROR;
   cudaError_t e = cudaGetLastError();
   if (e != cudaSuccess) { fprintf(stderr, "mgrit_gru: CUDA error: %s\n", cudaGetErrorString(e)); return MGRIT_CUDA_ERROR; }
-  if (sync && umma_device_status() != 0) return MGRIT_DEVICE_TIMEOUT;
+  if (sync && (umma_device_status() != 0 || serial_device_status() != 0)) return MGRIT_DEVICE_TIMEOUT;
   return MGRIT_OK;
 }
 
@@ -258,7 +293,7 @@ int forward_impl(const mgrit_gru_cfg* cfg_in, bool serial, const gru_params* p, 
 
   FwdCycle cy;
   cy.c = &c; cy.hr = hr; cy.s = s; cy.U = fw.U; cy.G = fw.G; cy.res_acc = fw.res_acc; cy.BH = BH;
-  cy.p = p; cy.gi = gi; cy.um = &fw.um;
+  cy.p = p; cy.gi = gi; cy.um = &fw.um; cy.fw = &fw;
   cy.solve();
   cudaMemcpyAsync(h, fw.U[0] + BH, sizeof(float) * (size_t)c.T * BH, cudaMemcpyDeviceToDevice, s);
   if (resnorm && hr.L > 1 && c.iters > 0) {
@@ -442,7 +477,7 @@ int sgd_update(float* p, const float* g, size_t n, float lr, mgrit_stream_t stre
 
 int mgrit_gru_last_device_status(void) {
   if (cudaDeviceSynchronize() != cudaSuccess) return MGRIT_CUDA_ERROR;
-  return umma_device_status() != 0 ? MGRIT_DEVICE_TIMEOUT : MGRIT_OK;
+  return (umma_device_status() != 0 || serial_device_status() != 0) ? MGRIT_DEVICE_TIMEOUT : MGRIT_OK;
 }
 
 unsigned long long mgrit_gru_kernel_launches(void) { return g_kernel_launches; }

@@ -16,7 +16,7 @@ extern unsigned long long g_kernel_launches;
 inline void count_launch(int n = 1) { g_kernel_launches += (unsigned long long)n; }
 
 // Optional per-launch timing of the GEMM-shaped kernels (CUDA events on the launching stream).
-enum KernelClass { KC_PROJ = 0, KC_FWD_STEP, KC_LINEARISE, KC_ADJ_STEP, KC_WGRAD, KC_COUNT };
+enum KernelClass { KC_PROJ = 0, KC_FWD_STEP, KC_LINEARISE, KC_ADJ_STEP, KC_WGRAD, KC_FWD_SERIAL, KC_ADJ_SERIAL, KC_COUNT };
 extern bool g_prof_on;
 void prof_begin(int kc, double flops, cudaStream_t s);
 void prof_end(cudaStream_t s);

@@ -1,0 +1,39 @@
+// Interface of the persistent kernels for chains of dependent steps with few rows.
+#pragma once
+#include "common.cuh"
+
+namespace mg {
+
+// u_j = Phi_gamma(gi_j, u_{j-1}) + g_j,  j = 1..nsteps   (slot-major state [nsteps+1][B][H], slot 0 given)
+struct SerialFwdArgs {
+  int B, H, nsteps;
+  float* u;                      // level state; slots 1..nsteps are written
+  __nv_bfloat16* ub;             // [2][B][H] scratch: bf16 copy of the newest state
+  const float* gi; i64 gi_step;  // projection rows of step 1 (+ (j-1)*gi_step for step j), row b at + b*3H
+  const float* g;                // [nsteps+1][B][H] additive term, or nullptr
+  const __nv_bfloat16* W;        // [3H][H]
+  const float* b_hh;
+  float gamma; int cell;
+  unsigned* bar;                 // [ceil(B/16)] barrier counters (scratch)
+};
+
+// mu_s = a_s*mu_{s-1} + ([cr_s|cz_s|cn_s]*mu_{s-1}) W_hh + g_s,  s = 1..nsteps
+struct SerialAdjArgs {
+  int B, H, nsteps;
+  float* mu;                     // [nsteps+1][B][H], slot 0 given
+  __nv_bfloat16* dAb;            // [2][B][3H] scratch
+  const float *a, *cr, *cz, *cn; // coefficient rows of step 1; step s at + (s-1)*coef_step
+  i64 coef_step;
+  const float* g;                // [nsteps+1][B][H] or nullptr
+  const __nv_bfloat16* WT;       // [H][3H] = W_hh^T
+  unsigned* bar;
+};
+
+bool serial_fwd_supported(int B, int H);
+bool serial_adj_supported(int B, int H);
+// false: shape not supported or the cooperative launch failed (the caller then advances step by step)
+bool serial_fwd_solve(const SerialFwdArgs& a, cudaStream_t s);
+bool serial_adj_solve(const SerialAdjArgs& a, cudaStream_t s);
+int serial_device_status();
+
+}  // namespace mg

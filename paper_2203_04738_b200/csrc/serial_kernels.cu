@@ -1,0 +1,388 @@
+// Persistent kernels for chains of DEPENDENT steps with few rows (the serial coarsest-level solve of
+// the multigrid cycle and the exact serial sweep; forward and adjoint).  One launch advances all
+// steps: every CTA keeps its slice of the recurrent weight matrix in shared memory for the whole
+// chain, the state crosses CTAs through L2 once per step as a bf16 operand copy, and the steps are
+// separated by a grid barrier with a bounded wait.  16 batch rows per CTA row group (row groups never
+// interact), bf16 mma.sync m16n8k16 with fp32 accumulation, K split over the 8 warps of a CTA.
+//
+// A wait that runs out writes a non-zero code to the status word; every CTA that sees a non-zero
+// status leaves at its next barrier, so the launch always terminates.
+#include "cell.cuh"
+#include "serial_engine.cuh"
+
+namespace mg {
+
+namespace {
+
+typedef __nv_bfloat16 bf16;
+constexpr int kThreads = 256, kWarps = 8, kRows = 16;
+constexpr uint64_t kWaitLimitNs = 2000000000ull;
+
+__device__ int g_serial_status = 0;
+int* g_serial_status_ptr = nullptr;
+
+__device__ __forceinline__ uint64_t global_ns() {
+  uint64_t t;
+  asm volatile("mov.u64 %0, %globaltimer;" : "=l"(t));
+  return t;
+}
+__device__ __forceinline__ unsigned ld_acquire(const unsigned* p) {
+  unsigned v;
+  asm volatile("ld.acquire.gpu.global.u32 %0, [%1];" : "=r"(v) : "l"(p) : "memory");
+  return v;
+}
+__device__ __forceinline__ int ld_relaxed(const int* p) {
+  int v;
+  asm volatile("ld.relaxed.gpu.global.s32 %0, [%1];" : "=r"(v) : "l"(p) : "memory");
+  return v;
+}
+
+// All CTAs that share `ctr` have finished the step whose arrival count is `target`.
+__device__ __forceinline__ bool grid_barrier(unsigned* ctr, unsigned target, int* status, int* ok_smem) {
+  __syncthreads();
+  if (threadIdx.x == 0) {
+    __threadfence();
+    atomicAdd(ctr, 1u);
+    int ok = 1;
+    unsigned spins = 0;
+    uint64_t t0 = 0;
+    while (ld_acquire(ctr) < target) {
+      if ((++spins & 127u) == 0) {
+        if (t0 == 0) t0 = global_ns();
+        if (ld_relaxed(status) != 0) { ok = 0; break; }
+        if (global_ns() - t0 > kWaitLimitNs) { atomicCAS(status, 0, 5); ok = 0; break; }
+      }
+    }
+    __threadfence();
+    *ok_smem = ok;
+  }
+  __syncthreads();
+  return *ok_smem != 0;
+}
+
+__device__ __forceinline__ void mma16816(float* c, const uint32_t* a, uint32_t b0, uint32_t b1) {
+  asm volatile(
+      "mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
+      : "+f"(c[0]), "+f"(c[1]), "+f"(c[2]), "+f"(c[3])
+      : "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "r"(b0), "r"(b1));
+}
+
+// acc[nt] += As[16, kbeg:kend] * Ws[nt*8 .. nt*8+8, kbeg:kend]^T   (both K-contiguous, row pitch ldk)
+template <int NT>
+__device__ __forceinline__ void warp_gemm(const bf16* As, const bf16* Ws, int ldk, int kbeg, int kend, float (*acc)[4]) {
+  const int lane = threadIdx.x & 31, g = lane >> 2, t = lane & 3;
+  for (int k0 = kbeg; k0 < kend; k0 += 16) {
+    uint32_t a[4];
+    a[0] = *reinterpret_cast<const uint32_t*>(As + g * ldk + k0 + 2 * t);
+    a[1] = *reinterpret_cast<const uint32_t*>(As + (g + 8) * ldk + k0 + 2 * t);
+    a[2] = *reinterpret_cast<const uint32_t*>(As + g * ldk + k0 + 2 * t + 8);
+    a[3] = *reinterpret_cast<const uint32_t*>(As + (g + 8) * ldk + k0 + 2 * t + 8);
+#pragma unroll
+    for (int nt = 0; nt < NT; ++nt) {
+      const bf16* wr = Ws + (nt * 8 + g) * ldk + k0 + 2 * t;
+      mma16816(acc[nt], a, *reinterpret_cast<const uint32_t*>(wr), *reinterpret_cast<const uint32_t*>(wr + 8));
+    }
+  }
+}
+
+// warp partial sums -> red[warp][row][col]   (col < NT*8)
+template <int NT>
+__device__ __forceinline__ void store_partials(float* red, float (*acc)[4]) {
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31, g = lane >> 2, t = lane & 3;
+  constexpr int NC = NT * 8;
+  float* base = red + warp * kRows * NC;
+#pragma unroll
+  for (int nt = 0; nt < NT; ++nt) {
+    base[g * NC + nt * 8 + 2 * t] = acc[nt][0];
+    base[g * NC + nt * 8 + 2 * t + 1] = acc[nt][1];
+    base[(g + 8) * NC + nt * 8 + 2 * t] = acc[nt][2];
+    base[(g + 8) * NC + nt * 8 + 2 * t + 1] = acc[nt][3];
+  }
+}
+template <int NC>
+__device__ __forceinline__ float sum_partials(const float* red, int row, int col) {
+  float s = 0.f;
+#pragma unroll
+  for (int w = 0; w < kWarps; ++w) s += red[(w * kRows + row) * NC + col];
+  return s;
+}
+
+// ------------------------------------------------------------------------------------------------
+// forward chain:  u_j = Phi_gamma(gi_j, u_{j-1}) + g_j ,  j = 1..nsteps
+template <int UNC>
+__global__ void __launch_bounds__(kThreads, 1) serial_fwd_kernel(SerialFwdArgs a, int* status) {
+  constexpr int NW = 3 * UNC, NT = NW / 8, OPT = (kRows * UNC + kThreads - 1) / kThreads;
+  extern __shared__ __align__(16) uint8_t smem[];
+  const int H = a.H, ldk = H + 8;
+  bf16* Ws = reinterpret_cast<bf16*>(smem);                 // [NW][ldk]
+  bf16* As = Ws + NW * ldk;                                 // [16][ldk]
+  float* red = reinterpret_cast<float*>(As + kRows * ldk);  // [8][16][NW]
+  __shared__ int ok_smem;
+  const int tid = threadIdx.x, warp = tid >> 5;
+  const int u0 = blockIdx.x * UNC, rg = blockIdx.y, row0 = rg * kRows;
+  const int nrows = min(kRows, a.B - row0);
+  const unsigned ncta_rg = gridDim.x;
+  const i64 BH = (i64)a.B * H;
+
+  // weights of this CTA's units (rows gate*H + u0 + i), resident for the whole chain
+  for (int e = tid; e < NW * (H / 8); e += kThreads) {
+    int r = e / (H / 8), c = e % (H / 8);
+    int gate = r / UNC, i = r % UNC;
+    *reinterpret_cast<uint4*>(Ws + r * ldk + c * 8) =
+        __ldg(reinterpret_cast<const uint4*>(a.W + ((i64)gate * H + u0 + i) * H + c * 8));
+  }
+  // rows beyond the batch stay zero
+  for (int e = tid; e < kRows * ldk / 2; e += kThreads) reinterpret_cast<uint32_t*>(As)[e] = 0u;
+  __syncthreads();
+  // step 1 reads the fp32 initial state
+  for (int e = tid; e < nrows * (H / 4); e += kThreads) {
+    int r = e / (H / 4), c = e % (H / 4);
+    float4 v = __ldcg(reinterpret_cast<const float4*>(a.u + (i64)(row0 + r) * H + c * 4));
+    __nv_bfloat162 lo = __floats2bfloat162_rn(v.x, v.y), hi = __floats2bfloat162_rn(v.z, v.w);
+    uint2 o; o.x = *reinterpret_cast<uint32_t*>(&lo); o.y = *reinterpret_cast<uint32_t*>(&hi);
+    *reinterpret_cast<uint2*>(As + r * ldk + c * 4) = o;
+  }
+  // outputs owned by this thread: (row, unit) pairs; previous value carried in registers
+  float hp[OPT], pgr[OPT], pgz[OPT], pgn[OPT], pg[OPT];
+  float br[OPT], bz[OPT], bn[OPT];
+#pragma unroll
+  for (int o = 0; o < OPT; ++o) {
+    int idx = tid + o * kThreads, r = idx / UNC, i = idx % UNC;
+    bool v = idx < kRows * UNC && r < nrows;
+    hp[o] = v ? __ldcg(a.u + (i64)(row0 + r) * H + u0 + i) : 0.f;
+    br[o] = a.b_hh[u0 + i]; bz[o] = a.b_hh[H + u0 + i]; bn[o] = a.b_hh[2 * H + u0 + i];
+    const float* gi = a.gi + (i64)(row0 + r) * 3 * H + u0 + i;
+    pgr[o] = v ? gi[0] : 0.f; pgz[o] = v ? gi[H] : 0.f; pgn[o] = v ? gi[2 * H] : 0.f;
+    pg[o] = (v && a.g) ? a.g[BH + (i64)(row0 + r) * H + u0 + i] : 0.f;
+  }
+  __syncthreads();
+
+  const int kw = H / kWarps;
+  for (int j = 1; j <= a.nsteps; ++j) {
+    float acc[NT][4];
+#pragma unroll
+    for (int nt = 0; nt < NT; ++nt) acc[nt][0] = acc[nt][1] = acc[nt][2] = acc[nt][3] = 0.f;
+    warp_gemm<NT>(As, Ws, ldk, warp * kw, (warp + 1) * kw, acc);
+    store_partials<NT>(red, acc);
+    __syncthreads();
+    bf16* ub = a.ub + (i64)(j & 1) * BH;
+#pragma unroll
+    for (int o = 0; o < OPT; ++o) {
+      int idx = tid + o * kThreads, r = idx / UNC, i = idx % UNC;
+      if (idx < kRows * UNC && r < nrows) {
+        float ghr = sum_partials<NW>(red, r, i) + br[o];
+        float ghz = sum_partials<NW>(red, r, UNC + i) + bz[o];
+        float ghn = sum_partials<NW>(red, r, 2 * UNC + i) + bn[o];
+        float val = cell_forward<true>(pgr[o], pgz[o], pgn[o], ghr, ghz, ghn, hp[o], a.gamma, a.cell) + pg[o];
+        hp[o] = val;
+        i64 off = (i64)(row0 + r) * H + u0 + i;
+        a.u[(i64)j * BH + off] = val;
+        ub[off] = __float2bfloat16(val);
+      }
+    }
+    if (j == a.nsteps) break;
+    // operands of the next step that do not depend on other CTAs
+#pragma unroll
+    for (int o = 0; o < OPT; ++o) {
+      int idx = tid + o * kThreads, r = idx / UNC, i = idx % UNC;
+      if (idx < kRows * UNC && r < nrows) {
+        const float* gi = a.gi + (i64)j * a.gi_step + (i64)(row0 + r) * 3 * H + u0 + i;
+        pgr[o] = gi[0]; pgz[o] = gi[H]; pgn[o] = gi[2 * H];
+        if (a.g) pg[o] = a.g[(i64)(j + 1) * BH + (i64)(row0 + r) * H + u0 + i];
+      }
+    }
+    if (!grid_barrier(a.bar + rg, (unsigned)j * ncta_rg, status, &ok_smem)) return;
+    // the full new state of this row group, as the bf16 A operand
+    for (int e = tid; e < nrows * (H / 8); e += kThreads) {
+      int r = e / (H / 8), c = e % (H / 8);
+      *reinterpret_cast<uint4*>(As + r * ldk + c * 8) = __ldcg(reinterpret_cast<const uint4*>(ub + (i64)(row0 + r) * H + c * 8));
+    }
+    __syncthreads();
+  }
+}
+
+// ------------------------------------------------------------------------------------------------
+// adjoint chain:  mu_s = a_s * mu_{s-1} + [cr_s|cz_s|cn_s]*mu_{s-1} W_hh + g_s ,  s = 1..nsteps
+// The bf16 operand copy carries dA_{s+1} = [cr|cz|cn]_{s+1} * mu_s, formed by the CTA that produced mu_s.
+template <int UNC>
+__global__ void __launch_bounds__(kThreads, 1) serial_adj_kernel(SerialAdjArgs a, int* status) {
+  constexpr int NT = UNC / 8, OPT = (kRows * UNC + kThreads - 1) / kThreads;
+  extern __shared__ __align__(16) uint8_t smem[];
+  const int H = a.H, K = 3 * H, ldk = K + 8;
+  bf16* Ws = reinterpret_cast<bf16*>(smem);                 // [UNC][ldk]   rows of W_hh^T
+  bf16* As = Ws + UNC * ldk;                                // [16][ldk]
+  float* red = reinterpret_cast<float*>(As + kRows * ldk);  // [8][16][UNC]
+  __shared__ int ok_smem;
+  const int tid = threadIdx.x, warp = tid >> 5;
+  const int u0 = blockIdx.x * UNC, rg = blockIdx.y, row0 = rg * kRows;
+  const int nrows = min(kRows, a.B - row0);
+  const unsigned ncta_rg = gridDim.x;
+  const i64 BH = (i64)a.B * H;
+
+  for (int e = tid; e < UNC * (K / 8); e += kThreads) {
+    int r = e / (K / 8), c = e % (K / 8);
+    *reinterpret_cast<uint4*>(Ws + r * ldk + c * 8) = __ldg(reinterpret_cast<const uint4*>(a.WT + (i64)(u0 + r) * K + c * 8));
+  }
+  for (int e = tid; e < kRows * ldk / 2; e += kThreads) reinterpret_cast<uint32_t*>(As)[e] = 0u;
+  __syncthreads();
+  // step 1: dA_1 = c_1 * mu_0 for all 3H columns of this row group
+  for (int e = tid; e < nrows * H; e += kThreads) {
+    int r = e / H, i = e % H;
+    i64 off = (i64)(row0 + r) * H + i;
+    float m = __ldcg(a.mu + off);
+    As[r * ldk + i] = __float2bfloat16(a.cr[off] * m);
+    As[r * ldk + H + i] = __float2bfloat16(a.cz[off] * m);
+    As[r * ldk + 2 * H + i] = __float2bfloat16(a.cn[off] * m);
+  }
+  float mp[OPT], pa[OPT], pg[OPT], ncr[OPT], ncz[OPT], ncn[OPT];
+#pragma unroll
+  for (int o = 0; o < OPT; ++o) {
+    int idx = tid + o * kThreads, r = idx / UNC, i = idx % UNC;
+    bool v = idx < kRows * UNC && r < nrows;
+    i64 off = (i64)(row0 + r) * H + u0 + i;
+    mp[o] = v ? __ldcg(a.mu + off) : 0.f;
+    pa[o] = v ? a.a[off] : 0.f;
+    pg[o] = (v && a.g) ? a.g[BH + off] : 0.f;
+    bool more = v && a.nsteps > 1;
+    ncr[o] = more ? a.cr[a.coef_step + off] : 0.f;
+    ncz[o] = more ? a.cz[a.coef_step + off] : 0.f;
+    ncn[o] = more ? a.cn[a.coef_step + off] : 0.f;
+  }
+  __syncthreads();
+
+  const int kw = K / kWarps;
+  for (int s = 1; s <= a.nsteps; ++s) {
+    float acc[NT][4];
+#pragma unroll
+    for (int nt = 0; nt < NT; ++nt) acc[nt][0] = acc[nt][1] = acc[nt][2] = acc[nt][3] = 0.f;
+    warp_gemm<NT>(As, Ws, ldk, warp * kw, (warp + 1) * kw, acc);
+    store_partials<NT>(red, acc);
+    __syncthreads();
+    bf16* dAb = a.dAb + (i64)(s & 1) * 3 * BH;
+#pragma unroll
+    for (int o = 0; o < OPT; ++o) {
+      int idx = tid + o * kThreads, r = idx / UNC, i = idx % UNC;
+      if (idx < kRows * UNC && r < nrows) {
+        float val = pa[o] * mp[o] + sum_partials<UNC>(red, r, i) + pg[o];
+        mp[o] = val;
+        i64 off = (i64)(row0 + r) * H + u0 + i;
+        a.mu[(i64)s * BH + off] = val;
+        if (s < a.nsteps) {
+          bf16* d = dAb + (i64)(row0 + r) * K + u0 + i;
+          d[0] = __float2bfloat16(ncr[o] * val);
+          d[H] = __float2bfloat16(ncz[o] * val);
+          d[2 * H] = __float2bfloat16(ncn[o] * val);
+        }
+      }
+    }
+    if (s == a.nsteps) break;
+#pragma unroll
+    for (int o = 0; o < OPT; ++o) {
+      int idx = tid + o * kThreads, r = idx / UNC, i = idx % UNC;
+      if (idx < kRows * UNC && r < nrows) {
+        i64 off = (i64)(row0 + r) * H + u0 + i;
+        pa[o] = a.a[(i64)s * a.coef_step + off];
+        if (a.g) pg[o] = a.g[(i64)(s + 1) * BH + off];
+        if (s + 1 < a.nsteps) {
+          i64 co = (i64)(s + 1) * a.coef_step + off;
+          ncr[o] = a.cr[co]; ncz[o] = a.cz[co]; ncn[o] = a.cn[co];
+        }
+      }
+    }
+    if (!grid_barrier(a.bar + rg, (unsigned)s * ncta_rg, status, &ok_smem)) return;
+    for (int e = tid; e < nrows * (K / 8); e += kThreads) {
+      int r = e / (K / 8), c = e % (K / 8);
+      *reinterpret_cast<uint4*>(As + r * ldk + c * 8) = __ldcg(reinterpret_cast<const uint4*>(dAb + (i64)(row0 + r) * K + c * 8));
+    }
+    __syncthreads();
+  }
+}
+
+bool ensure_status() {
+  if (g_serial_status_ptr) return true;
+  return cudaGetSymbolAddress((void**)&g_serial_status_ptr, g_serial_status) == cudaSuccess;
+}
+
+constexpr size_t kSmemLimit = 227 * 1024 - 64;
+int g_sm_count = 0;
+int sm_count() {
+  if (g_sm_count == 0) {
+    int dev = 0;
+    cudaGetDevice(&dev);
+    if (cudaDeviceGetAttribute(&g_sm_count, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || g_sm_count <= 0) g_sm_count = 148;
+  }
+  return g_sm_count;
+}
+
+size_t fwd_smem(int unc, int H) { return (size_t)(3 * unc + kRows) * (H + 8) * 2 + (size_t)kWarps * kRows * 3 * unc * 4; }
+size_t adj_smem(int unc, int H) { return (size_t)(unc + kRows) * (3 * H + 8) * 2 + (size_t)kWarps * kRows * unc * 4; }
+
+// smallest units-per-CTA whose grid is co-resident (one CTA per SM) and whose slice fits shared memory
+int pick_unc(int B, int H, bool adj) {
+  if (H % 128 != 0) return 0;
+  int rgs = (B + kRows - 1) / kRows;
+  const int cands[3] = {8, 16, 32};
+  for (int c : cands) {
+    if (H % c != 0) continue;
+    if ((i64)(H / c) * rgs > sm_count()) continue;
+    size_t sm = adj ? adj_smem(c, H) : fwd_smem(c, H);
+    if (sm > kSmemLimit) continue;
+    return c;
+  }
+  return 0;
+}
+
+template <class Args, class Kern>
+bool launch_coop(Kern kern, const Args& a, int unc, size_t smem, cudaStream_t s) {
+  if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess) return false;
+  int rgs = (a.B + kRows - 1) / kRows;
+  if (cudaMemsetAsync(a.bar, 0, sizeof(unsigned) * rgs, s) != cudaSuccess) return false;
+  Args args = a;
+  int* st = g_serial_status_ptr;
+  void* params[2] = {(void*)&args, (void*)&st};
+  dim3 grid(a.H / unc, rgs);
+  if (cudaLaunchCooperativeKernel((const void*)kern, grid, dim3(kThreads), params, smem, s) != cudaSuccess) {
+    cudaGetLastError();
+    return false;
+  }
+  count_launch();
+  return true;
+}
+
+}  // namespace
+
+bool serial_fwd_supported(int B, int H) { return pick_unc(B, H, false) != 0; }
+bool serial_adj_supported(int B, int H) { return pick_unc(B, H, true) != 0; }
+
+bool serial_fwd_solve(const SerialFwdArgs& a, cudaStream_t s) {
+  int unc = pick_unc(a.B, a.H, false);
+  if (unc == 0 || a.nsteps <= 0 || !ensure_status()) return false;
+  size_t smem = fwd_smem(unc, a.H);
+  prof_begin(KC_FWD_SERIAL, 2.0 * a.B * 3.0 * a.H * a.H * a.nsteps, s);
+  bool ok = unc == 8 ? launch_coop(serial_fwd_kernel<8>, a, unc, smem, s)
+          : unc == 16 ? launch_coop(serial_fwd_kernel<16>, a, unc, smem, s)
+                      : launch_coop(serial_fwd_kernel<32>, a, unc, smem, s);
+  prof_end(s);
+  return ok;
+}
+
+bool serial_adj_solve(const SerialAdjArgs& a, cudaStream_t s) {
+  int unc = pick_unc(a.B, a.H, true);
+  if (unc == 0 || a.nsteps <= 0 || !ensure_status()) return false;
+  size_t smem = adj_smem(unc, a.H);
+  prof_begin(KC_ADJ_SERIAL, 2.0 * a.B * 3.0 * a.H * a.H * a.nsteps, s);
+  bool ok = unc == 8 ? launch_coop(serial_adj_kernel<8>, a, unc, smem, s)
+          : unc == 16 ? launch_coop(serial_adj_kernel<16>, a, unc, smem, s)
+                      : launch_coop(serial_adj_kernel<32>, a, unc, smem, s);
+  prof_end(s);
+  return ok;
+}
+
+int serial_device_status() {
+  if (!g_serial_status_ptr) return 0;
+  int v = 0;
+  if (cudaMemcpy(&v, g_serial_status_ptr, sizeof(int), cudaMemcpyDeviceToHost) != cudaSuccess) return -1;
+  return v;
+}
+
+}  // namespace mg

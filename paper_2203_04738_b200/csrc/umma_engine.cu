@@ -139,7 +139,6 @@ struct EpiFwd {  // GRU cell on the r|z|n accumulator columns of 64 hidden units
     // in mode 1 the previous content of the destination plays the role of the additive term
     const float* __restrict__ ga = a.mode == 1 ? ho : (a.gadd ? a.gadd + (i64)k * a.gadd_ks + (i64)b * H + u0 : nullptr);
     const float* __restrict__ bh = a.b_hh + u0;
-    const float sign = a.mode == 1 ? -1.f : 1.f;
 #pragma unroll
     for (int cc = 0; cc < 2; ++cc) {
       const int c0 = half * 32 + cc * 16;
@@ -165,7 +164,7 @@ struct EpiFwd {  // GRU cell on the r|z|n accumulator columns of 64 hidden units
           float o[4];
 #pragma unroll
           for (int e = 0; e < 4; ++e) {
-            float phi = cell_forward(f4get(gr[i], e), f4get(gz[i], e), f4get(gn[i], e), r[4 * i + e] + f4get(br, e),
+            float phi = cell_forward<true>(f4get(gr[i], e), f4get(gz[i], e), f4get(gn[i], e), r[4 * i + e] + f4get(br, e),
                                      z[4 * i + e] + f4get(bz, e), n[4 * i + e] + f4get(bn, e), f4get(h4[i], e), a.gamma, a.cell);
             // mode 0: phi + g ;  mode 1: previous - phi
             o[e] = a.mode == 1 ? f4get(g4[i], e) - phi : phi + f4get(g4[i], e);
@@ -174,7 +173,6 @@ struct EpiFwd {  // GRU cell on the r|z|n accumulator columns of 64 hidden units
         }
       }
     }
-    (void)sign;
   }
 };
 
@@ -212,7 +210,7 @@ struct EpiLin {  // adjoint coefficients of every step of a level
           float oa[4], ocr[4], ocz[4], ocn[4], ocp[4];
 #pragma unroll
           for (int e = 0; e < 4; ++e) {
-            CellLin L = cell_linearise(f4get(gr[i], e), f4get(gz[i], e), f4get(gn[i], e), r[4 * i + e] + f4get(br, e),
+            CellLin L = cell_linearise<true>(f4get(gr[i], e), f4get(gz[i], e), f4get(gn[i], e), r[4 * i + e] + f4get(br, e),
                                        z[4 * i + e] + f4get(bz, e), n[4 * i + e] + f4get(bn, e), f4get(h4[i], e), a.gamma, a.cell);
             oa[e] = L.a; ocr[e] = L.cr; ocz[e] = L.cz; ocn[e] = L.cn; ocp[e] = L.cnp;
           }
