@@ -90,6 +90,7 @@ int check_cfg(const mgrit_gru_cfg* c, Hier* hr) {
 struct FwdWs {
   float* U[kMaxLevels]; float* G[kMaxLevels]; double* res_acc; UmmaFwdWs um;
   __nv_bfloat16* chain_ub; unsigned* chain_bar;   // scratch of the persistent serial-chain kernel
+  __nv_bfloat16* Ub[kMaxLevels];                  // bf16 copies of the level states (tensor-core A operands)
 };
 struct AdjWs {
   float* U[kMaxLevels]; float* G[kMaxLevels];
@@ -106,8 +107,10 @@ void plan_fwd(const mgrit_gru_cfg* c, const Hier& hr, Ws& w, FwdWs* o) {
   }
   o->res_acc = w.take<double>((size_t)(c->iters > 0 ? c->iters : 1));
   o->chain_ub = nullptr; o->chain_bar = nullptr;
+  for (int l = 0; l < kMaxLevels; ++l) o->Ub[l] = nullptr;
   if (c->operands == MGRIT_OPERANDS_BF16) {
     umma_plan_fwd(c, hr.N, hr.L, w.base, &w.off, &o->um);
+    for (int l = 0; l < hr.L; ++l) o->Ub[l] = w.take<__nv_bfloat16>((size_t)(hr.N[l] + 1) * BH);
     o->chain_ub = w.take<__nv_bfloat16>(2 * BH);
     o->chain_bar = w.take<unsigned>(64 + (size_t)c->B / 16);
   }
@@ -152,6 +155,7 @@ struct StepDesc {
 struct Cycle {
   const mgrit_gru_cfg* c; Hier hr; cudaStream_t s;
   float** U; float** G; double* res_acc; int cycle_idx = 0;
+  __nv_bfloat16** Ub = nullptr;   // optional bf16 copies of U (kept in step with every writer)
   size_t BH;
   virtual void step(const StepDesc& d) = 0;
   // all N_l dependent steps of level l in one persistent launch; false = not available here
@@ -182,11 +186,12 @@ struct Cycle {
     // v_k = step_l(u_{cf k - 1}) + g_{cf k}  ->  G[l+1][k]
     step(StepDesc{l, nc, cf - 1, cf, G[l + 1], 1, 1, G[l], cf, cf, cf, cf, 0});
     // r_k = u_{cf k} - v_k ; U'_k = u_{cf k}
-    stream_restrict_residual(U[l], cf, G[l + 1], U[l + 1], nc, (i64)BH, l == 0 ? res_acc + cycle_idx : nullptr, s);
+    stream_restrict_residual(U[l], cf, G[l + 1], U[l + 1], Ub ? Ub[l + 1] : nullptr, nc, (i64)BH,
+                             l == 0 ? res_acc + cycle_idx : nullptr, s);
     // G_k = v_k - step_{l+1}(U'_{k-1})
     step(StepDesc{l + 1, nc, 0, 1, G[l + 1], 1, 1, nullptr, 0, 0, 1, 1, 1});
     vcycle(l + 1);
-    stream_correct(U[l], cf, U[l + 1], nc, (i64)BH, s);
+    stream_correct(U[l], Ub ? Ub[l] : nullptr, cf, U[l + 1], nc, (i64)BH, s);
     frelax(l);
   }
   void solve() {
@@ -213,6 +218,8 @@ struct FwdCycle : Cycle {
     a.M = d.nk * c->B; a.B = c->B; a.H = c->H;
     a.hin = U[d.l] + (size_t)d.in_slot * BH; a.hin_ks = (i64)d.in_stride * BH;
     a.hout = d.out + (size_t)d.out_slot * BH; a.hout_ks = (i64)d.out_stride * BH;
+    a.hin_b = Ub ? Ub[d.l] + (size_t)d.in_slot * BH : nullptr;
+    a.hout_b = (Ub && d.out == U[d.l]) ? Ub[d.l] + (size_t)d.out_slot * BH : nullptr;
     i64 st = hr.stride_t[d.l];
     a.gi = gi + ((i64)st * d.tgt_slot - 1) * (i64)BH * 3; a.gi_ks = st * d.tgt_stride * (i64)BH * 3;
     a.gadd = d.gadd ? d.gadd + (size_t)d.gadd_slot * BH : nullptr; a.gadd_ks = (i64)d.gadd_stride * BH;
@@ -290,10 +297,16 @@ int forward_impl(const mgrit_gru_cfg* cfg_in, bool serial, const gru_params* p, 
   }
   cudaMemsetAsync(fw.U[0] + BH, 0, sizeof(float) * (size_t)c.T * BH, s);
   for (int l = 0; l < hr.L; ++l) cudaMemcpyAsync(fw.U[l], h0, sizeof(float) * BH, cudaMemcpyDeviceToDevice, s);
+  const bool shadows = c.operands == MGRIT_OPERANDS_BF16 && 128 % c.B == 0;
+  if (shadows) {
+    cudaMemsetAsync(fw.Ub[0] + BH, 0, sizeof(__nv_bfloat16) * (size_t)c.T * BH, s);
+    for (int l = 0; l < hr.L; ++l) umma_convert(h0, fw.Ub[l], (i64)BH, s);
+  }
 
   FwdCycle cy;
   cy.c = &c; cy.hr = hr; cy.s = s; cy.U = fw.U; cy.G = fw.G; cy.res_acc = fw.res_acc; cy.BH = BH;
   cy.p = p; cy.gi = gi; cy.um = &fw.um; cy.fw = &fw;
+  cy.Ub = shadows ? fw.Ub : nullptr;
   cy.solve();
   cudaMemcpyAsync(h, fw.U[0] + BH, sizeof(float) * (size_t)c.T * BH, cudaMemcpyDeviceToDevice, s);
   if (resnorm && hr.L > 1 && c.iters > 0) {
@@ -324,7 +337,7 @@ int adjoint_impl(const mgrit_gru_cfg* cfg_in, bool serial, const gru_params* p, 
   const bool bf16 = c.operands == MGRIT_OPERANDS_BF16;
 
   if (bf16) {
-    rc = umma_prepare_adj(&c, p, &aw.um, s);
+    rc = umma_prepare_adj(&c, p, h0, h, &aw.um, s);
     if (rc) return rc;
   }
   // adjoint coefficients of every level's steps at the given states (restricted by injection)

@@ -27,6 +27,8 @@ struct FwdStepArgs {
   int M, B, H;
   const float* hin;  i64 hin_ks;    // previous state rows      hin  + k*hin_ks  + b*H
   float* hout;       i64 hout_ks;   // result rows              hout + k*hout_ks + b*H
+  const __nv_bfloat16* hin_b;       // bf16 copy of the previous state rows (same indexing) or nullptr
+  __nv_bfloat16* hout_b;            // where to write the bf16 copy of the result (same indexing) or nullptr
   const float* gi;   i64 gi_ks;     // input projection rows    gi   + k*gi_ks   + b*3H
   const float* gadd; i64 gadd_ks;   // optional FAS term rows (same shape as hout) or nullptr
   const float* W_hh;                // [3H,H] fp32
@@ -73,8 +75,9 @@ void simt_dgrad(const float* dA, int M, int H3, const float* W, int C, float* dx
 // streaming kernels
 // r = uC - v at the C-points, sum of squares into *acc (double, device), copy of the C-point state
 // to the coarse level:   uc[k] = uf[cf*k],  k = 1..nc   (rows of rowlen = B*H floats)
-void stream_restrict_residual(const float* uf, int cf, const float* v, float* uc, int nc, i64 rowlen, double* acc, cudaStream_t s);
-void stream_correct(float* uf, int cf, const float* uc, int nc, i64 rowlen, cudaStream_t s);
+// ucb / ufb: optional bf16 copies of the written rows (same indexing), nullptr to skip
+void stream_restrict_residual(const float* uf, int cf, const float* v, float* uc, __nv_bfloat16* ucb, int nc, i64 rowlen, double* acc, cudaStream_t s);
+void stream_correct(float* uf, __nv_bfloat16* ufb, int cf, const float* uc, int nc, i64 rowlen, cudaStream_t s);
 // dst[k] = src[k*src_ks], k = 0..nk-1, rows of rowlen floats (src_ks in elements, may be negative)
 void stream_gather_rows(float* dst, i64 dst_ks, const float* src, i64 src_ks, int nk, i64 rowlen, cudaStream_t s);
 void stream_add_rows(float* dst, const float* src, i64 n, cudaStream_t s);

@@ -18,6 +18,14 @@ inline int stream_grid(i64 work_items, int per_block = kThreads) {
   return (int)blocks;
 }
 
+__device__ __forceinline__ uint2 pack_bf16x4(float4 v) {
+  __nv_bfloat162 lo = __floats2bfloat162_rn(v.x, v.y), hi = __floats2bfloat162_rn(v.z, v.w);
+  uint2 o;
+  o.x = *reinterpret_cast<uint32_t*>(&lo);
+  o.y = *reinterpret_cast<uint32_t*>(&hi);
+  return o;
+}
+
 __device__ __forceinline__ float warp_sum(float v) {
 #pragma unroll
   for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
@@ -28,8 +36,8 @@ __device__ __forceinline__ float warp_sum(float v) {
 // (Algorithm "MGProp": r_c = R(f(h')), h'_c = R(h');  Eq. "restrict").
 __global__ void __launch_bounds__(kThreads) restrict_residual_kernel(const float4* __restrict__ uf, int cf,
                                                                      const float4* __restrict__ v,
-                                                                     float4* __restrict__ uc, int nc, i64 row4,
-                                                                     double* acc) {
+                                                                     float4* __restrict__ uc, uint2* __restrict__ ucb,
+                                                                     int nc, i64 row4, double* acc) {
   i64 total = (i64)nc * row4;
   float s = 0.f;
   for (i64 e = (i64)blockIdx.x * blockDim.x + threadIdx.x; e < total; e += (i64)gridDim.x * blockDim.x) {
@@ -39,6 +47,7 @@ __global__ void __launch_bounds__(kThreads) restrict_residual_kernel(const float
     float4 r = make_float4(u.x - w.x, u.y - w.y, u.z - w.z, u.w - w.w);
     s += r.x * r.x + r.y * r.y + r.z * r.z + r.w * r.w;
     uc[k * row4 + c] = u;
+    if (ucb) ucb[k * row4 + c] = pack_bf16x4(u);
   }
   __shared__ float part[kThreads / 32];
   s = warp_sum(s);
@@ -52,12 +61,14 @@ __global__ void __launch_bounds__(kThreads) restrict_residual_kernel(const float
 }
 
 // Correction h'' = h' + P(h_c* - h'_c): only C-points are read afterwards, so u_{cf k} <- U_k.
-__global__ void __launch_bounds__(kThreads) correct_kernel(float4* __restrict__ uf, int cf, const float4* __restrict__ uc,
-                                                           int nc, i64 row4) {
+__global__ void __launch_bounds__(kThreads) correct_kernel(float4* __restrict__ uf, uint2* __restrict__ ufb, int cf,
+                                                           const float4* __restrict__ uc, int nc, i64 row4) {
   i64 total = (i64)nc * row4;
   for (i64 e = (i64)blockIdx.x * blockDim.x + threadIdx.x; e < total; e += (i64)gridDim.x * blockDim.x) {
     i64 k = e / row4 + 1, c = e % row4;
-    uf[(k * cf) * row4 + c] = uc[k * row4 + c];
+    float4 u = uc[k * row4 + c];
+    uf[(k * cf) * row4 + c] = u;
+    if (ufb) ufb[(k * cf) * row4 + c] = pack_bf16x4(u);
   }
 }
 
@@ -192,17 +203,18 @@ __global__ void __launch_bounds__(kThreads) sgd_kernel(float* __restrict__ p, co
 
 }  // namespace
 
-void stream_restrict_residual(const float* uf, int cf, const float* v, float* uc, int nc, i64 rowlen, double* acc,
+void stream_restrict_residual(const float* uf, int cf, const float* v, float* uc, __nv_bfloat16* ucb, int nc, i64 rowlen, double* acc,
                               cudaStream_t s) {
   i64 row4 = rowlen / 4;
   restrict_residual_kernel<<<stream_grid((i64)nc * row4), kThreads, 0, s>>>(
-      reinterpret_cast<const float4*>(uf), cf, reinterpret_cast<const float4*>(v), reinterpret_cast<float4*>(uc), nc, row4, acc);
+      reinterpret_cast<const float4*>(uf), cf, reinterpret_cast<const float4*>(v), reinterpret_cast<float4*>(uc),
+      reinterpret_cast<uint2*>(ucb), nc, row4, acc);
   count_launch();
 }
 
-void stream_correct(float* uf, int cf, const float* uc, int nc, i64 rowlen, cudaStream_t s) {
+void stream_correct(float* uf, __nv_bfloat16* ufb, int cf, const float* uc, int nc, i64 rowlen, cudaStream_t s) {
   i64 row4 = rowlen / 4;
-  correct_kernel<<<stream_grid((i64)nc * row4), kThreads, 0, s>>>(reinterpret_cast<float4*>(uf), cf,
+  correct_kernel<<<stream_grid((i64)nc * row4), kThreads, 0, s>>>(reinterpret_cast<float4*>(uf), reinterpret_cast<uint2*>(ufb), cf,
                                                                   reinterpret_cast<const float4*>(uc), nc, row4);
   count_launch();
 }

@@ -1,0 +1,291 @@
+// Fused "recurrent GEMM + GRU cell" kernel for sm_100a, second form: every operand of the epilogue
+// is staged through shared memory by TMA, so that the only latency-exposed global accesses of the
+// epilogue are its stores.
+//
+//   rows m = (k, b)      k = interval / coarse point, b = batch row, 128 rows per tile = kt k's x B
+//   D[m, gate, u] = sum_j hb[m, j] * W_hh[gate*H + u, j]          (tcgen05, bf16 x bf16 -> fp32 in TMEM)
+//   forward : out[m, u] = Phi_gamma(gi[m, :, u], D + b_hh, h[m, u]) (+ g[m, u])   or   g - Phi   (mode 1)
+//   linearise: a, c_r, c_z, c_n, c_n'[m, u] = transposed-Jacobian coefficients of that step
+//
+// Warp roles (352 threads): 0 = TMA producer of the A/B ring, 1 = MMA issuer and TMEM owner,
+// 2 = TMA producer of the epilogue operands (gi r|z|n, h, g in chunks of 16 hidden units, two
+// buffers), 3..10 = epilogue (two warps per TMEM lane quarter, 8 hidden units per thread and chunk).
+// The A operand (bf16 copy of the state) and the epilogue operands are addressed through 3-D tensor
+// maps {column, batch row, k} whose k-stride is the slot stride of the relaxation, so no gather
+// kernel is needed; the epilogue also writes the bf16 copy of the new state for the next step.
+// Epilogue tiles use the 64-byte swizzle: rows of 16 floats, 16-byte chunk index XOR ((row >> 1) & 3).
+#pragma once
+#include "cell.cuh"
+#include "umma_gemm.cuh"
+
+namespace mg {
+namespace umma {
+
+__device__ __forceinline__ void tma_load_3d(uint32_t dst, const CUtensorMap* map, uint32_t bar, int c0, int c1, int c2) {
+  asm volatile(
+      "cp.async.bulk.tensor.3d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, %5}], [%2];"
+      ::"r"(dst), "l"(map), "r"(bar), "r"(c0), "r"(c1), "r"(c2)
+      : "memory");
+}
+// tcgen05.ld is asynchronous: its destination registers are only valid after tcgen05.wait::ld.  The
+// results are therefore produced directly in their final registers (no copies that the compiler could
+// schedule before the wait), and tmem_ld_wait8 makes every later use depend on the wait.
+__device__ __forceinline__ void tmem_ld8(uint32_t taddr, float* v) {
+  asm volatile("tcgen05.ld.sync.aligned.32x32b.x8.b32 {%0,%1,%2,%3,%4,%5,%6,%7}, [%8];"
+               : "=f"(v[0]), "=f"(v[1]), "=f"(v[2]), "=f"(v[3]), "=f"(v[4]), "=f"(v[5]), "=f"(v[6]), "=f"(v[7])
+               : "r"(taddr));
+}
+__device__ __forceinline__ void tmem_ld_wait8x3(float* a, float* b, float* c) {
+  asm volatile("tcgen05.wait::ld.sync.aligned;"
+               : "+f"(a[0]), "+f"(a[1]), "+f"(a[2]), "+f"(a[3]), "+f"(a[4]), "+f"(a[5]), "+f"(a[6]), "+f"(a[7]),
+                 "+f"(b[0]), "+f"(b[1]), "+f"(b[2]), "+f"(b[3]), "+f"(b[4]), "+f"(b[5]), "+f"(b[6]), "+f"(b[7]),
+                 "+f"(c[0]), "+f"(c[1]), "+f"(c[2]), "+f"(c[3]), "+f"(c[4]), "+f"(c[5]), "+f"(c[6]), "+f"(c[7])
+               :
+               : "memory");
+}
+__device__ __forceinline__ float4 lds4(uint32_t addr) {
+  float4 v;
+  asm volatile("ld.shared.v4.f32 {%0,%1,%2,%3}, [%4];" : "=f"(v.x), "=f"(v.y), "=f"(v.z), "=f"(v.w) : "r"(addr));
+  return v;
+}
+
+struct CellArgs {
+  int M, B, H, kt;                                    // kt = 128 / B
+  float* hout; i64 hout_ks; __nv_bfloat16* hout_b;    // forward: fp32 rows (k, b) and their bf16 copy (or nullptr)
+  float *a, *cr, *cz, *cn, *cnp;                      // linearise: row-major [M, H] (cnp may be nullptr)
+  const float* b_hh; float gamma; int cell; int mode;
+};
+
+namespace cellk {
+constexpr int BN = 192, UN = 64, CH = 16, NCH = UN / CH;
+constexpr int kThreads = 352;
+constexpr int kABytes = BM * BK * 2, kBBytes = BN * BK * 2, kStageBytes = kABytes + kBBytes;
+constexpr int kOpBytes = BM * CH * 4;   // one epilogue operand chunk: 128 rows x 16 floats
+template <bool HAS_G> struct CellCfg {
+  static constexpr int kStages = HAS_G ? 3 : 4;
+  static constexpr int kOps = HAS_G ? 5 : 4;
+  static constexpr int kEpiBytes = kOps * kOpBytes;
+  static constexpr int kSmemBytes = kStages * kStageBytes + 2 * kEpiBytes + 1024 + 256;
+};
+}  // namespace cellk
+
+template <bool LIN, bool HAS_G>
+__global__ void __launch_bounds__(cellk::kThreads, 1)
+umma_cell_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB,
+                 const __grid_constant__ CUtensorMap tmGI, const __grid_constant__ CUtensorMap tmHP,
+                 const __grid_constant__ CUtensorMap tmG, CellArgs p, int* status) {
+  using namespace cellk;
+  using C = CellCfg<HAS_G>;
+  extern __shared__ uint8_t smem_raw[];
+  const uint32_t raw = smem_u32(smem_raw);
+  const uint32_t tiles_base = (raw + 1023u) & ~1023u;
+  const uint32_t epi_base = tiles_base + C::kStages * kStageBytes;
+  const uint32_t bars = epi_base + 2 * C::kEpiBytes;
+  auto full_bar = [&](int s) { return bars + 8u * s; };
+  auto empty_bar = [&](int s) { return bars + 8u * (C::kStages + s); };
+  auto tfull_bar = [&](int a) { return bars + 8u * (2 * C::kStages + a); };
+  auto tempty_bar = [&](int a) { return bars + 8u * (2 * C::kStages + 2 + a); };
+  auto efull_bar = [&](int e) { return bars + 8u * (2 * C::kStages + 4 + e); };
+  auto eempty_bar = [&](int e) { return bars + 8u * (2 * C::kStages + 6 + e); };
+  __shared__ uint32_t tmem_base_smem;
+  __shared__ int abort_flag;
+
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int H = p.H;
+  const int m_tiles = (p.M + BM - 1) / BM, n_tiles = H / UN, tiles = m_tiles * n_tiles;
+  const int k_blocks = (H + BK - 1) / BK;
+
+  if (threadIdx.x == 0) {
+    abort_flag = 0;
+    for (int s = 0; s < C::kStages; ++s) { mbar_init(full_bar(s), 1); mbar_init(empty_bar(s), 1); }
+    for (int a = 0; a < 2; ++a) {
+      mbar_init(tfull_bar(a), 1); mbar_init(tempty_bar(a), 256);
+      mbar_init(efull_bar(a), 1); mbar_init(eempty_bar(a), 256);
+    }
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+  }
+  if (warp == 1) {
+    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&tmem_base_smem)), "r"(512u)
+                 : "memory");
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+  }
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem_base = tmem_base_smem;
+  volatile int* abortp = &abort_flag;
+
+  if (warp == 0) {
+    // ------------------------------------------------------------ A/B producer
+    if (lane == 0) {
+      int stage = 0; uint32_t phase = 0; bool ok = true;
+      for (int t = blockIdx.x; t < tiles && ok; t += gridDim.x) {
+        const int mt = t / n_tiles, nt = t % n_tiles;
+        for (int kb = 0; kb < k_blocks; ++kb) {
+          if (!mbar_wait(empty_bar(stage), phase ^ 1u, abortp, status, 11)) { ok = false; break; }
+          const uint32_t a_dst = tiles_base + stage * kStageBytes, b_dst = a_dst + kABytes;
+          mbar_expect_tx(full_bar(stage), kStageBytes);
+          tma_load_3d(a_dst, &tmA, full_bar(stage), kb * BK, 0, mt * p.kt);
+#pragma unroll
+          for (int g = 0; g < 3; ++g) tma_load_2d(b_dst + g * (kBBytes / 3), &tmB, full_bar(stage), kb * BK, g * H + nt * UN);
+          if (++stage == C::kStages) { stage = 0; phase ^= 1u; }
+        }
+      }
+    }
+  } else if (warp == 1) {
+    // ------------------------------------------------------------ MMA issuer
+    if (lane == 0) {
+      constexpr uint32_t idesc = instr_desc_bf16(BN);
+      int stage = 0; uint32_t phase = 0; int it = 0; bool ok = true;
+      for (int t = blockIdx.x; t < tiles && ok; t += gridDim.x, ++it) {
+        const int as = it & 1;
+        const uint32_t aphase = (uint32_t)(it >> 1) & 1u;
+        if (!mbar_wait(tempty_bar(as), aphase ^ 1u, abortp, status, 12)) { ok = false; break; }
+        tc_fence_after();
+        const uint32_t d_tmem = tmem_base + (uint32_t)(as * BN);
+        for (int kb = 0; kb < k_blocks; ++kb) {
+          if (!mbar_wait(full_bar(stage), phase, abortp, status, 13)) { ok = false; break; }
+          tc_fence_after();
+          const uint32_t a_src = tiles_base + stage * kStageBytes;
+          const uint64_t adesc = smem_desc_sw128(a_src), bdesc = smem_desc_sw128(a_src + kABytes);
+#pragma unroll
+          for (int k = 0; k < BK / 16; ++k)
+            mma_bf16(d_tmem, adesc + (uint64_t)(k * 2), bdesc + (uint64_t)(k * 2), idesc, (kb | k) != 0 ? 1u : 0u);
+          mma_commit(empty_bar(stage));
+          if (++stage == C::kStages) { stage = 0; phase ^= 1u; }
+        }
+        if (ok) mma_commit(tfull_bar(as));
+      }
+    }
+  } else if (warp == 2) {
+    // ------------------------------------------------------------ epilogue-operand producer
+    if (lane == 0) {
+      int eb = 0; uint32_t ephase = 0; bool ok = true;
+      for (int t = blockIdx.x; t < tiles && ok; t += gridDim.x) {
+        const int mt = t / n_tiles, nt = t % n_tiles;
+        for (int c = 0; c < NCH; ++c) {
+          if (!mbar_wait(eempty_bar(eb), ephase ^ 1u, abortp, status, 14)) { ok = false; break; }
+          const uint32_t dst = epi_base + eb * C::kEpiBytes;
+          const int u = nt * UN + c * CH, k0 = mt * p.kt;
+          mbar_expect_tx(efull_bar(eb), C::kEpiBytes);
+          tma_load_3d(dst, &tmGI, efull_bar(eb), u, 0, k0);
+          tma_load_3d(dst + kOpBytes, &tmGI, efull_bar(eb), H + u, 0, k0);
+          tma_load_3d(dst + 2 * kOpBytes, &tmGI, efull_bar(eb), 2 * H + u, 0, k0);
+          tma_load_3d(dst + 3 * kOpBytes, &tmHP, efull_bar(eb), u, 0, k0);
+          if (HAS_G) tma_load_3d(dst + 4 * kOpBytes, &tmG, efull_bar(eb), u, 0, k0);
+          if (++eb == 2) { eb = 0; ephase ^= 1u; }
+        }
+      }
+    }
+  } else {
+    // ------------------------------------------------------------ epilogue (warps 3..10)
+    const int q = warp & 3;              // TMEM lane quarter of this warp
+    const int half = (warp - 3) >> 2;    // which 8 of a chunk's 16 hidden units
+    const int r = q * 32 + lane;         // row inside the tile
+    const uint32_t sw = (uint32_t)((r >> 1) & 3);
+    const uint32_t off0 = (uint32_t)r * 64u + ((((uint32_t)half * 2u) ^ sw) << 4);
+    const uint32_t off1 = (uint32_t)r * 64u + ((((uint32_t)half * 2u + 1u) ^ sw) << 4);
+    int it = 0, eb = 0; uint32_t ephase = 0;
+    bool ok = true;
+    for (int t = blockIdx.x; t < tiles && ok; t += gridDim.x, ++it) {
+      const int mt = t / n_tiles, nt = t % n_tiles;
+      const int as = it & 1;
+      const uint32_t aphase = (uint32_t)(it >> 1) & 1u;
+      const int row = mt * BM + r;
+      const bool valid = row < p.M;
+      const int k = valid ? row / p.B : 0, b = valid ? row % p.B : 0;
+      if (!mbar_wait(tfull_bar(as), aphase, abortp, status, 15)) break;
+      tc_fence_after();
+      const uint32_t taddr = tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(as * BN);
+      for (int c = 0; c < NCH; ++c) {
+        if (!mbar_wait(efull_bar(eb), ephase, abortp, status, 16)) { ok = false; break; }
+        const uint32_t src = epi_base + eb * C::kEpiBytes;
+        float gr[8], gz[8], gn[8], hp[8], gg[8];
+        *reinterpret_cast<float4*>(gr) = lds4(src + off0);                 *reinterpret_cast<float4*>(gr + 4) = lds4(src + off1);
+        *reinterpret_cast<float4*>(gz) = lds4(src + kOpBytes + off0);      *reinterpret_cast<float4*>(gz + 4) = lds4(src + kOpBytes + off1);
+        *reinterpret_cast<float4*>(gn) = lds4(src + 2 * kOpBytes + off0);  *reinterpret_cast<float4*>(gn + 4) = lds4(src + 2 * kOpBytes + off1);
+        *reinterpret_cast<float4*>(hp) = lds4(src + 3 * kOpBytes + off0);  *reinterpret_cast<float4*>(hp + 4) = lds4(src + 3 * kOpBytes + off1);
+        if (HAS_G) {
+          *reinterpret_cast<float4*>(gg) = lds4(src + 4 * kOpBytes + off0); *reinterpret_cast<float4*>(gg + 4) = lds4(src + 4 * kOpBytes + off1);
+        }
+        const int cu = c * CH + half * 8;       // first of this thread's 8 units inside the tile
+        float ar[8], az[8], an[8];
+        tmem_ld8(taddr + cu, ar);
+        tmem_ld8(taddr + UN + cu, az);
+        tmem_ld8(taddr + 2 * UN + cu, an);
+        tmem_ld_wait8x3(ar, az, an);
+        const int eb_done = eb;
+        if (++eb == 2) { eb = 0; ephase ^= 1u; }
+        if (valid) {
+          const int u = nt * UN + cu;
+          float br[8], bz[8], bn[8];
+          *reinterpret_cast<float4*>(br) = __ldg(reinterpret_cast<const float4*>(p.b_hh + u));
+          *reinterpret_cast<float4*>(br + 4) = __ldg(reinterpret_cast<const float4*>(p.b_hh + u + 4));
+          *reinterpret_cast<float4*>(bz) = __ldg(reinterpret_cast<const float4*>(p.b_hh + H + u));
+          *reinterpret_cast<float4*>(bz + 4) = __ldg(reinterpret_cast<const float4*>(p.b_hh + H + u + 4));
+          *reinterpret_cast<float4*>(bn) = __ldg(reinterpret_cast<const float4*>(p.b_hh + 2 * H + u));
+          *reinterpret_cast<float4*>(bn + 4) = __ldg(reinterpret_cast<const float4*>(p.b_hh + 2 * H + u + 4));
+          if (!LIN) {
+            float o[8];
+#pragma unroll
+            for (int e = 0; e < 8; ++e) {
+              float phi = cell_forward<true>(gr[e], gz[e], gn[e], ar[e] + br[e], az[e] + bz[e], an[e] + bn[e], hp[e], p.gamma, p.cell);
+              o[e] = HAS_G ? (p.mode == 1 ? gg[e] - phi : phi + gg[e]) : phi;
+            }
+            const i64 idx = (i64)k * p.hout_ks + (i64)b * H + u;
+            float* ho = p.hout + idx;
+            *reinterpret_cast<float4*>(ho) = make_float4(o[0], o[1], o[2], o[3]);
+            *reinterpret_cast<float4*>(ho + 4) = make_float4(o[4], o[5], o[6], o[7]);
+            if (p.hout_b) {
+              __nv_bfloat162 p0 = __floats2bfloat162_rn(o[0], o[1]), p1 = __floats2bfloat162_rn(o[2], o[3]);
+              __nv_bfloat162 p2 = __floats2bfloat162_rn(o[4], o[5]), p3 = __floats2bfloat162_rn(o[6], o[7]);
+              uint4 pk;
+              pk.x = *reinterpret_cast<uint32_t*>(&p0); pk.y = *reinterpret_cast<uint32_t*>(&p1);
+              pk.z = *reinterpret_cast<uint32_t*>(&p2); pk.w = *reinterpret_cast<uint32_t*>(&p3);
+              *reinterpret_cast<uint4*>(p.hout_b + idx) = pk;
+            }
+          } else {
+            float oa[8], ocr[8], ocz[8], ocn[8], ocp[8];
+#pragma unroll
+            for (int e = 0; e < 8; ++e) {
+              CellLin L = cell_linearise<true>(gr[e], gz[e], gn[e], ar[e] + br[e], az[e] + bz[e], an[e] + bn[e], hp[e], p.gamma, p.cell);
+              oa[e] = L.a; ocr[e] = L.cr; ocz[e] = L.cz; ocn[e] = L.cn; ocp[e] = L.cnp;
+            }
+            const i64 idx = (i64)row * H + u;
+            *reinterpret_cast<float4*>(p.a + idx) = make_float4(oa[0], oa[1], oa[2], oa[3]);
+            *reinterpret_cast<float4*>(p.a + idx + 4) = make_float4(oa[4], oa[5], oa[6], oa[7]);
+            *reinterpret_cast<float4*>(p.cr + idx) = make_float4(ocr[0], ocr[1], ocr[2], ocr[3]);
+            *reinterpret_cast<float4*>(p.cr + idx + 4) = make_float4(ocr[4], ocr[5], ocr[6], ocr[7]);
+            *reinterpret_cast<float4*>(p.cz + idx) = make_float4(ocz[0], ocz[1], ocz[2], ocz[3]);
+            *reinterpret_cast<float4*>(p.cz + idx + 4) = make_float4(ocz[4], ocz[5], ocz[6], ocz[7]);
+            *reinterpret_cast<float4*>(p.cn + idx) = make_float4(ocn[0], ocn[1], ocn[2], ocn[3]);
+            *reinterpret_cast<float4*>(p.cn + idx + 4) = make_float4(ocn[4], ocn[5], ocn[6], ocn[7]);
+            if (p.cnp) {
+              *reinterpret_cast<float4*>(p.cnp + idx) = make_float4(ocp[0], ocp[1], ocp[2], ocp[3]);
+              *reinterpret_cast<float4*>(p.cnp + idx + 4) = make_float4(ocp[4], ocp[5], ocp[6], ocp[7]);
+            }
+          }
+        }
+        // Release the operand buffer only here, after the values read from it have been used: an
+        // mbarrier.arrive issued right after the ld.shared instructions is not ordered behind loads whose
+        // results are still in flight, and the refilling TMA then overwrote rows that had not been read.
+        mbar_arrive(eempty_bar(eb_done));
+      }
+      if (!ok) break;
+      tc_fence_before();
+      mbar_arrive(tempty_bar(as));
+    }
+  }
+
+  // ------------------------------------------------------------ teardown
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  if (warp == 1) {
+    __syncwarp();
+    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(512u) : "memory");
+  }
+}
+
+}  // namespace umma
+}  // namespace mg

@@ -1,9 +1,11 @@
 // Tensor-core engine: bf16 operands, fp32 accumulation in tensor memory, fp32 states and gates.
 // Host launchers, operand-packing kernels and the fused epilogues of the tcgen05 GEMM.
 #include <stdio.h>
+#include <stdlib.h>
 
 #include "cell.cuh"
 #include "umma_engine.cuh"
+#include "umma_cell.cuh"
 #include "umma_gemm.cuh"
 
 namespace mg {
@@ -72,6 +74,56 @@ bool launch_gemm(int kc, const bf16* A, i64 lda, const bf16* Bm, i64 ldb, int M,
   int grid = tiles < kSMs ? tiles : kSMs;
   prof_begin(kc, 2.0 * M * (GATES ? 3.0 * N : (double)N) * K, s);
   kern<<<grid, kThreads, C::kSmemBytes, s>>>(ta, tb, sh, epi, g_status_ptr);
+  prof_end(s);
+  count_launch();
+  return true;
+}
+
+// 3-D map {column, batch row, k}: rows (k, b) at base + k*ks + b*ld, `inner` columns
+bool make_map3(CUtensorMap* m, CUtensorMapDataType dt, size_t esize, const void* base, uint64_t inner, uint64_t B, uint64_t nk,
+               uint64_t ld, i64 ks, uint32_t box_inner, uint32_t box_k, CUtensorMapSwizzle sw) {
+  if (ks <= 0) ks = (i64)(ld * B);       // a single k: any legal stride
+  cuuint64_t dims[3] = {inner, B, nk};
+  cuuint64_t strides[2] = {ld * esize, (cuuint64_t)ks * esize};
+  cuuint32_t box[3] = {box_inner, (cuuint32_t)B, box_k};
+  cuuint32_t estr[3] = {1, 1, 1};
+  CUresult r = g_encode(m, dt, 3, (void*)base, dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE, sw,
+                        CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  if (r != CUDA_SUCCESS) fprintf(stderr, "mgrit_gru: cuTensorMapEncodeTiled (3-D) failed (%d)\n", (int)r);
+  return r == CUDA_SUCCESS;
+}
+
+// Fused recurrent GEMM + cell (forward step or linearisation) with TMA-staged epilogue operands.
+// Rows (k, b), k = 0..nk-1: A rows at A + k*a_ks + b*H (bf16), gi rows at gi + k*gi_ks + b*3H,
+// previous state at hp + k*hp_ks + b*H, optional additive term at g + k*g_ks + b*H.
+template <bool LIN, bool HAS_G>
+bool launch_cell(int kc, const bf16* A, i64 a_ks, const float* gi, i64 gi_ks, const float* hp, i64 hp_ks, const float* g, i64 g_ks,
+                 int nk, const bf16* W, CellArgs ca, cudaStream_t s) {
+  using C = cellk::CellCfg<HAS_G>;
+  if (nk <= 0) return true;
+  if (!ensure_driver()) return false;
+  static bool attr_set = false;
+  auto kern = umma_cell_kernel<LIN, HAS_G>;
+  if (!attr_set) {
+    if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, C::kSmemBytes) != cudaSuccess) return false;
+    attr_set = true;
+  }
+  const int B = ca.B, H = ca.H, kt = 128 / B;
+  ca.kt = kt; ca.M = nk * B;
+  CUtensorMap ta, tb, tgi, thp, tg;
+  if (!make_map3(&ta, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, A, H, B, nk, H, a_ks, BK, kt, CU_TENSOR_MAP_SWIZZLE_128B)) return false;
+  if (!make_map(&tb, W, (uint64_t)H, (uint64_t)3 * H, (uint64_t)H, cellk::UN)) return false;
+  if (!make_map3(&tgi, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 4, gi, 3 * H, B, nk, 3 * H, gi_ks, cellk::CH, kt, CU_TENSOR_MAP_SWIZZLE_64B)) return false;
+  if (!make_map3(&thp, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 4, hp, H, B, nk, H, hp_ks, cellk::CH, kt, CU_TENSOR_MAP_SWIZZLE_64B)) return false;
+  if (HAS_G) {
+    if (!make_map3(&tg, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 4, g, H, B, nk, H, g_ks, cellk::CH, kt, CU_TENSOR_MAP_SWIZZLE_64B)) return false;
+  } else {
+    tg = thp;
+  }
+  int tiles = ((ca.M + BM - 1) / BM) * (H / cellk::UN);
+  int grid = tiles < kSMs ? tiles : kSMs;
+  prof_begin(kc, 2.0 * ca.M * 3.0 * H * H, s);
+  kern<<<grid, cellk::kThreads, C::kSmemBytes, s>>>(ta, tb, tgi, thp, tg, ca, g_status_ptr);
   prof_end(s);
   count_launch();
   return true;
@@ -431,6 +483,8 @@ void umma_plan_adj(const mgrit_gru_cfg* c, const int* N, int L, char* base, size
   o->hprevT = take<bf16>(base, off, H * TB);
   o->xT = take<bf16>(base, off, I * TB);
   o->dbpart = nullptr;
+  o->hb0 = take<bf16>(base, off, (size_t)c->B * H);
+  o->hb = take<bf16>(base, off, TB * H);
 }
 
 int umma_prepare_fwd(const mgrit_gru_cfg* c, const gru_params* p, const float* x, float* gi, UmmaFwdWs* w, cudaStream_t s) {
@@ -445,15 +499,28 @@ int umma_prepare_fwd(const mgrit_gru_cfg* c, const gru_params* p, const float* x
   return MGRIT_OK;
 }
 
-int umma_prepare_adj(const mgrit_gru_cfg* c, const gru_params* p, UmmaAdjWs* w, cudaStream_t s) {
+int umma_prepare_adj(const mgrit_gru_cfg* c, const gru_params* p, const float* h0, const float* h, UmmaAdjWs* w, cudaStream_t s) {
   const int H = c->H, I = c->I;
   convert(p->W_hh, w->W_hh, (i64)3 * H * H, s);
+  convert(h0, w->hb0, (i64)c->B * H, s);
+  convert(h, w->hb, (i64)c->T * c->B * H, s);
   transpose(p->W_hh, 3 * H, H, w->W_hhT, 3 * H, 0, s);   // [H, 3H]
   transpose(p->W_ih, 3 * H, I, w->W_ihT, 3 * H, 0, s);   // [I, 3H]
   return ensure_driver() ? MGRIT_OK : MGRIT_CUDA_ERROR;
 }
 
 void umma_fwd_step(const FwdStepArgs& a, UmmaFwdWs* w, cudaStream_t s) {
+  if (a.hin_b && 128 % a.B == 0) {
+    // operands through strided tensor maps, bf16 copy of the new state written by the epilogue
+    CellArgs ca{};
+    ca.B = a.B; ca.H = a.H; ca.hout = a.hout; ca.hout_ks = a.hout_ks; ca.hout_b = a.hout_b;
+    ca.b_hh = a.b_hh; ca.gamma = a.gamma; ca.cell = a.cell; ca.mode = a.mode;
+    const int nk = a.M / a.B;
+    if (a.mode == 1) launch_cell<false, true>(KC_FWD_STEP, a.hin_b, a.hin_ks, a.gi, a.gi_ks, a.hin, a.hin_ks, a.hout, a.hout_ks, nk, w->W_hh, ca, s);
+    else if (a.gadd) launch_cell<false, true>(KC_FWD_STEP, a.hin_b, a.hin_ks, a.gi, a.gi_ks, a.hin, a.hin_ks, a.gadd, a.gadd_ks, nk, w->W_hh, ca, s);
+    else launch_cell<false, false>(KC_FWD_STEP, a.hin_b, a.hin_ks, a.gi, a.gi_ks, a.hin, a.hin_ks, nullptr, 0, nk, w->W_hh, ca, s);
+    return;
+  }
   pack_rows_kernel<<<pgrid((i64)a.M * (a.H / 4)), kPT, 0, s>>>(a.hin, a.hin_ks, a.B, a.H / 4, a.M, reinterpret_cast<uint2*>(w->Apack));
   count_launch();
   launch_gemm<192, true>(KC_FWD_STEP, w->Apack, a.H, w->W_hh, a.H, a.M, a.H, a.H, a.H, 3 * a.H, EpiFwd{a}, s);
@@ -462,6 +529,21 @@ void umma_fwd_step(const FwdStepArgs& a, UmmaFwdWs* w, cudaStream_t s) {
 void umma_linearise(const LinArgs& a, UmmaAdjWs* w, cudaStream_t s) {
   // rows (j-1, b): state entering forward step j of the level = h_{stride*(j-1)}
   const i64 BH = (i64)a.B * a.H;
+  const int N = a.M / a.B;
+  if (128 % a.B == 0) {
+    CellArgs ca{};
+    ca.B = a.B; ca.H = a.H; ca.b_hh = a.b_hh; ca.gamma = a.gamma; ca.cell = a.cell;
+    const float* gi0 = a.gi + (a.stride_t - 1) * BH * 3;
+    // step 1 starts from h_0 (its own array); steps 2..N from h[stride*(j-1) - 1]
+    ca.a = a.a; ca.cr = a.cr; ca.cz = a.cz; ca.cn = a.cn; ca.cnp = a.cnp;
+    launch_cell<true, false>(KC_LINEARISE, w->hb0, 0, gi0, 0, a.h0, 0, nullptr, 0, 1, w->W_hh, ca, s);
+    if (N > 1) {
+      ca.a = a.a + BH; ca.cr = a.cr + BH; ca.cz = a.cz + BH; ca.cn = a.cn + BH; ca.cnp = a.cnp ? a.cnp + BH : nullptr;
+      launch_cell<true, false>(KC_LINEARISE, w->hb + (a.stride_t - 1) * BH, a.stride_t * BH, gi0 + a.stride_t * BH * 3, a.stride_t * BH * 3,
+                               a.h + (a.stride_t - 1) * BH, a.stride_t * BH, nullptr, 0, N - 1, w->W_hh, ca, s);
+    }
+    return;
+  }
   pack_rows_kernel<<<pgrid((i64)a.B * (a.H / 4)), kPT, 0, s>>>(a.h0, 0, a.B, a.H / 4, a.B, reinterpret_cast<uint2*>(w->Apack));
   count_launch();
   if (a.M > a.B) {
@@ -503,6 +585,8 @@ int umma_gradients(const mgrit_gru_cfg* c, const gru_params* p, const float* x, 
   if (dx) ok = ok && launch_gemm<256, false>(KC_WGRAD, w->dAi, 3 * H, w->W_ihT, 3 * H, (int)M, I, 3 * H, 0, I, EpiStore{dx, I, (int)M, I}, s);
   return ok ? MGRIT_OK : MGRIT_CUDA_ERROR;
 }
+
+void umma_convert(const float* src, __nv_bfloat16* dst, i64 n, cudaStream_t s) { convert(src, dst, n, s); }
 
 int umma_device_status() {
   if (!g_status_ptr) return 0;

@@ -23,6 +23,8 @@ struct UmmaAdjWs {
   __nv_bfloat16* hprevT;  // [H,T*B]
   __nv_bfloat16* xT;      // [I,T*B]
   float* dbpart;          // partial column sums
+  __nv_bfloat16* hb0;     // [B,H]    bf16 copy of h_0
+  __nv_bfloat16* hb;      // [T*B,H]  bf16 copy of the given states
   size_t maxM;
 };
 
@@ -30,7 +32,8 @@ int umma_supported(const mgrit_gru_cfg* c);
 void umma_plan_fwd(const mgrit_gru_cfg* c, const int* N, int L, char* base, size_t* off, UmmaFwdWs* o);
 void umma_plan_adj(const mgrit_gru_cfg* c, const int* N, int L, char* base, size_t* off, UmmaAdjWs* o);
 int umma_prepare_fwd(const mgrit_gru_cfg* c, const gru_params* p, const float* x, float* gi, UmmaFwdWs* w, cudaStream_t s);
-int umma_prepare_adj(const mgrit_gru_cfg* c, const gru_params* p, UmmaAdjWs* w, cudaStream_t s);
+int umma_prepare_adj(const mgrit_gru_cfg* c, const gru_params* p, const float* h0, const float* h, UmmaAdjWs* w, cudaStream_t s);
+void umma_convert(const float* src, __nv_bfloat16* dst, i64 n, cudaStream_t s);
 void umma_fwd_step(const FwdStepArgs& a, UmmaFwdWs* w, cudaStream_t s);
 void umma_linearise(const LinArgs& a, UmmaAdjWs* w, cudaStream_t s);
 void umma_adj_step(const AdjStepArgs& a, UmmaAdjWs* w, cudaStream_t s);

@@ -164,3 +164,26 @@ def test_prefix_exactness_and_convergence_at_full_size(B):
     assert e8 < e3 and e8 < 2e-2
     h_dup, _, _ = B.mgrit_gru_forward(_cfg(B, w, 3, T=1024, flags=B.FLAG_SKIP_DUPLICATE_FRELAX), p, x, h0)
     assert torch.equal(h, h_dup)
+
+
+def test_run_to_run_bit_identical_and_workspace_content_irrelevant(B):
+    # The result must not depend on scheduling (many tiles per CTA, three levels, additive terms on the inner
+    # level) nor on what the caller's workspace held before the call.
+    w = Workload("det", T=1024, B=32, I=64, H=512, cf=4, levels=3, iters_fwd=2, iters_adj=2, relax_fine=0, relax_coarse=1,
+                 operands=2, classes=8, relu=True, seed=7)
+    d = make_inputs(w)
+    p, x, h0 = upload(d)
+    cfg = _cfg(B, w, 2)
+    nf, na = B.workspace_bytes(cfg)
+    outs = []
+    for fill in (0x00, 0x7F, 0x00, 0xFF):
+        ws = torch.full((nf,), fill, dtype=torch.uint8, device="cuda")
+        h, gi, _ = B.mgrit_gru_forward(cfg, p, x, h0, ws=ws)
+        wa = torch.full((na,), fill, dtype=torch.uint8, device="cuda")
+        r = B.mgrit_gru_adjoint(cfg, p, x, h0, gi, h, dhT=h[-1].contiguous(), ws=wa)
+        outs.append((h.clone(), r.dh.clone(), r.dW_hh.clone()))
+    for o in outs[1:]:
+        assert torch.equal(o[0], outs[0][0])
+        assert torch.equal(o[1], outs[0][1])
+        assert torch.allclose(o[2], outs[0][2], rtol=1e-4, atol=1e-6)   # bias/weight sums use float atomics
+    assert B.last_device_status() == 0
