@@ -39,7 +39,8 @@ enum {
   MGRIT_WORKSPACE_TOO_SMALL = -3,
   MGRIT_UNSUPPORTED = -4,        /* shape outside what the selected operand mode supports */
   MGRIT_CUDA_ERROR = -5,         /* a CUDA runtime/driver call failed */
-  MGRIT_DEVICE_TIMEOUT = -6      /* a bounded device-side wait ran out */
+  MGRIT_DEVICE_TIMEOUT = -6,     /* a bounded device-side wait ran out */
+  MGRIT_SCRATCH_LIMIT = -7       /* problem larger than the built-in scratch of a no-allocation entry point */
 };
 
 enum { MGRIT_CELL_CLASSIC = 0, MGRIT_CELL_IMPLICIT = 1 };
@@ -133,6 +134,25 @@ size_t xent_head_workspace_bytes(int32_t B, int32_t C);
 int xent_head_fwd_bwd(int32_t B, int32_t H, int32_t C, const float* hT, const float* Wc, const float* bc,
                       const int32_t* labels, float* loss, float* dhT, float* dWc, float* dbc,
                       void* ws, size_t ws_bytes, mgrit_stream_t stream);
+
+/* The same classifier head for callers that cannot allocate device memory (the paper has no
+ * counterpart; this exists for hosts of the library).  Typical cases: a process whose own memory
+ * arena already owns all of the GPU's memory, so that cudaMalloc fails or would fragment it, and
+ * latency-critical loops that must stay clear of the driver's allocator, which takes a global lock
+ * and may synchronise the device.  Instead of a workspace argument the [B, C] intermediate (loss
+ * derivative w.r.t. the logits) is kept in a fixed 256 KiB array that is part of the library image:
+ * every GPU that loads the library holds it until the process exits.
+ *   Limit: B * C <= 65536, otherwise MGRIT_SCRATCH_LIMIT is returned and nothing is launched.
+ *   The call performs no cudaMalloc / cudaFree and calls no allocating routine.
+ *   The first call on each device looks up the array's device address (once per device, with that
+ *   device current); make that first call before any stream capture is started on the device.
+ *   All calls share the one array, which keeps the previous call's contents; nothing in it needs to be
+ *   cleared between calls (each call overwrites the B * C entries it reads).  Two calls that overlap on
+ *   the GPU (different streams, or different host threads) race on it: serialise them.
+ *   Inputs, outputs and results are exactly those of xent_head_fwd_bwd. */
+int xent_head_fwd_bwd_noalloc(int32_t B, int32_t H, int32_t C, const float* hT, const float* Wc, const float* bc,
+                              const int32_t* labels, float* loss, float* dhT, float* dWc, float* dbc,
+                              mgrit_stream_t stream);
 
 /* Theta <- Theta - lr * g (last line of Algorithm "MGRITTraining"); n fp32 elements. */
 int sgd_update(float* p, const float* g, size_t n, float lr, mgrit_stream_t stream);

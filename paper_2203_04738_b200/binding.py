@@ -53,6 +53,7 @@ lib.gru_serial_backward.argtypes = [ctypes.POINTER(Cfg), ctypes.POINTER(_Params)
 lib.xent_head_workspace_bytes.argtypes = [_i32, _i32]
 lib.xent_head_workspace_bytes.restype = _sz
 lib.xent_head_fwd_bwd.argtypes = [_i32, _i32, _i32, _vp, _vp, _vp, _vp, _vp, _vp, _vp, _vp, _vp, _sz, _vp]
+lib.xent_head_fwd_bwd_noalloc.argtypes = [_i32, _i32, _i32, _vp, _vp, _vp, _vp, _vp, _vp, _vp, _vp, _vp]
 lib.sgd_update.argtypes = [_vp, _vp, _sz, ctypes.c_float, _vp]
 lib.mgrit_gru_last_device_status.restype = ctypes.c_int
 lib.mgrit_gru_kernel_launches.restype = ctypes.c_ulonglong
@@ -194,6 +195,23 @@ def xent_head_fwd_bwd(hT, Wc, bc, labels, ws=None):
     ws = _ws(lib.xent_head_workspace_bytes(B, C), ws, dev)
     _check(lib.xent_head_fwd_bwd(B, H, C, _f32(hT), _f32(Wc), _f32(bc), _ptr(labels), _f32(loss), _f32(dhT), _f32(dWc),
                                  _f32(dbc), _ptr(ws), ws.numel(), _stream()))
+    return loss, dhT, dWc, dbc
+
+
+def xent_head_fwd_bwd_noalloc(hT, Wc, bc, labels, out=None):
+    """Loss head for callers that must not allocate device memory inside the call: the library's built-in
+    scratch replaces the workspace (B*C <= 65536).  `out` = (loss[1], dhT[B,H], dWc[C,H], dbc[C]) preallocated
+    by the caller; when omitted this convenience wrapper allocates the four outputs with torch before the call.
+    Calls share one scratch array: do not overlap them on the GPU."""
+    B, H = hT.shape
+    C = Wc.shape[0]
+    dev = hT.device
+    assert labels.dtype == torch.int32
+    if out is None:
+        out = (torch.empty(1, device=dev), torch.empty(B, H, device=dev), torch.empty(C, H, device=dev), torch.empty(C, device=dev))
+    loss, dhT, dWc, dbc = out
+    _check(lib.xent_head_fwd_bwd_noalloc(B, H, C, _f32(hT), _f32(Wc), _f32(bc), _ptr(labels), _f32(loss), _f32(dhT), _f32(dWc),
+                                         _f32(dbc), _stream()))
     return loss, dhT, dWc, dbc
 
 

@@ -541,6 +541,7 @@ const char* mgrit_gru_strerror(int code) {
     case MGRIT_UNSUPPORTED: return "shape not supported by the selected operand mode";
     case MGRIT_CUDA_ERROR: return "CUDA error";
     case MGRIT_DEVICE_TIMEOUT: return "a bounded device-side wait ran out";
+    case MGRIT_SCRATCH_LIMIT: return "problem exceeds the built-in scratch of the no-allocation entry point (B*C <= 65536)";
     default: return "unknown error";
   }
 }

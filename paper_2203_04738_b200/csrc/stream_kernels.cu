@@ -265,3 +265,45 @@ void stream_sgd(float* p, const float* g, size_t n, float lr, cudaStream_t s) {
 }
 
 }  // namespace mg
+
+// ---------------------------------------------------------------------------------------------------
+// Classifier head without any caller-provided or allocated scratch.
+//
+// Some hosts of this library cannot allocate device memory at the moment they need the loss head: a
+// serving or training process that has handed the whole GPU to its own memory arena (cudaMalloc then
+// fails or fragments the arena), or a latency-critical loop that must not take the driver's allocator
+// lock, which can also synchronise the device.  For them the [B, C] buffer of loss derivatives with
+// respect to the logits lives in a fixed array inside the library image.  Every GPU that loads the
+// library holds these 256 KiB until the process exits.
+namespace mg {
+namespace {
+constexpr size_t kHeadScratchFloats = 65536;   // B * C <= 65536
+static __device__ __align__(256) float g_head_scratch[kHeadScratchFloats];
+constexpr int kMaxDevices = 64;
+float* g_head_scratch_addr[kMaxDevices] = {nullptr};   // device address of the array, per device
+}  // namespace
+}  // namespace mg
+
+extern "C" int xent_head_fwd_bwd_noalloc(int32_t B, int32_t H, int32_t C, const float* hT, const float* Wc, const float* bc,
+                                         const int32_t* labels, float* loss, float* dhT, float* dWc, float* dbc,
+                                         mgrit_stream_t stream) {
+  using namespace mg;
+  if (B <= 0 || H <= 0 || C <= 0 || !hT || !Wc || !bc || !labels || !loss || !dhT || !dWc || !dbc) return MGRIT_INVALID_ARG;
+  if (C > 8192) return MGRIT_UNSUPPORTED;
+  if ((size_t)B * (size_t)C > kHeadScratchFloats) return MGRIT_SCRATCH_LIMIT;
+  int dev = -1;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) return MGRIT_CUDA_ERROR;
+  if (!g_head_scratch_addr[dev]) {
+    // In host code the array's name is only a handle; the kernels need its address on the current device.
+    float* p = nullptr;
+    if (cudaGetSymbolAddress((void**)&p, g_head_scratch) != cudaSuccess || !p) {
+      cudaGetLastError();
+      return MGRIT_CUDA_ERROR;
+    }
+    g_head_scratch_addr[dev] = p;
+  }
+  // Nothing in the scratch has to start at zero: pass 1 overwrites all B*C entries before pass 2 reads them
+  // (the loss accumulator is the caller's `loss`, cleared inside stream_xent).
+  stream_xent(B, H, C, hT, Wc, bc, labels, loss, dhT, dWc, dbc, g_head_scratch_addr[dev], (cudaStream_t)stream);
+  return cudaGetLastError() == cudaSuccess ? MGRIT_OK : MGRIT_CUDA_ERROR;
+}
