@@ -112,7 +112,7 @@ void plan_fwd(const mgrit_gru_cfg* c, const Hier& hr, Ws& w, FwdWs* o) {
     umma_plan_fwd(c, hr.N, hr.L, w.base, &w.off, &o->um);
     for (int l = 0; l < hr.L; ++l) o->Ub[l] = w.take<__nv_bfloat16>((size_t)(hr.N[l] + 1) * BH);
     o->chain_ub = w.take<__nv_bfloat16>(2 * BH);
-    o->chain_bar = w.take<unsigned>(64 + (size_t)c->B / 16);
+    o->chain_bar = w.take<unsigned>(((size_t)c->B / 16 + 1) * ((size_t)c->H / 8) + 64);
   }
 }
 
@@ -132,7 +132,7 @@ void plan_adj(const mgrit_gru_cfg* c, const Hier& hr, Ws& w, AdjWs* o) {
     o->dA_h = o->dA_i = nullptr;
     umma_plan_adj(c, hr.N, hr.L, w.base, &w.off, &o->um);
     o->chain_dAb = w.take<__nv_bfloat16>(6 * BH);
-    o->chain_bar = w.take<unsigned>(64 + (size_t)c->B / 16);
+    o->chain_bar = w.take<unsigned>(((size_t)c->B / 16 + 1) * ((size_t)c->H / 8) + 64);
   } else {
     o->chain_dAb = nullptr; o->chain_bar = nullptr;
     o->dA_h = w.take<float>((size_t)c->T * BH * 3);
