@@ -174,6 +174,7 @@ def main():
     import torch
     import torch.distributed as dist
     from paper_2203_04738_b200 import binding as B
+    from paper_2203_04738_b200.replicas import job_throughput, max_over_ranks
     from paper_2203_04738_b200.train_step import alloc_buffers, training_step
 
     torch.cuda.set_device(local_rank)
@@ -217,12 +218,9 @@ def main():
     ms = e0.elapsed_time(e1)
     launches = B.kernel_launches() - l0
     clocks = sampler.stop() if sampler else None
-    if world > 1:
-        t = torch.tensor([ms], device=dev)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        ms = float(t.item())
+    ms = max_over_ranks(ms, dev)
     ms_step = ms / args.steps
-    value = world * T * w.B / (ms_step * 1e-3)
+    value = job_throughput(T * w.B, ms_step, world)
 
     # end to end: inputs start in pinned host memory, the loss is read back, every step
     e2e = None
@@ -237,11 +235,8 @@ def main():
         e1.record()
         barrier()
         ms2 = e0.elapsed_time(e1)
-        if world > 1:
-            t = torch.tensor([ms2], device=dev)
-            dist.all_reduce(t, op=dist.ReduceOp.MAX)
-            ms2 = float(t.item())
-        e2e = {"value": world * T * w.B / (ms2 / args.steps * 1e-3), "unit": UNIT,
+        ms2 = max_over_ranks(ms2, dev)
+        e2e = {"value": job_throughput(T * w.B, ms2 / args.steps, world), "unit": UNIT,
                "h2d_bytes_per_step": x_host.numel() * 4, "d2h_bytes_per_step": 4}
 
     # per-kernel timing pass (CUDA events around every GEMM-shaped launch; outside the timed region so

@@ -1,0 +1,49 @@
+"""The C-ABI library loads without a GPU and exports every function that include/mgrit_gru.h declares;
+host-side argument checks answer without touching a device."""
+import ctypes
+import os
+import re
+
+import pytest
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+HEADER = os.path.join(ROOT, "include", "mgrit_gru.h")
+
+
+@pytest.fixture(scope="module")
+def lib():
+    from paper_2203_04738_b200.build import build
+    return ctypes.CDLL(build())
+
+
+def declared_functions():
+    src = open(HEADER).read()
+    src = re.sub(r"/\*.*?\*/", "", src, flags=re.S)
+    names = re.findall(r"\b([a-z_0-9]+)\s*\(", src)
+    return sorted({n for n in names if n not in ("defined",)})
+
+
+def test_every_declared_symbol_is_exported(lib):
+    names = declared_functions()
+    assert "mgrit_gru_forward" in names and "mgrit_gru_adjoint" in names and "gru_serial_backward" in names
+    assert "xent_head_fwd_bwd_noalloc" in names and len(names) >= 14
+    for n in names:
+        assert hasattr(lib, n), n
+
+
+def test_host_side_validation_without_a_device(lib):
+    from paper_2203_04738_b200.binding import Cfg, make_cfg
+    f, a = ctypes.c_size_t(0), ctypes.c_size_t(0)
+    fn = lib.mgrit_gru_workspace_bytes
+    fn.argtypes = [ctypes.POINTER(Cfg), ctypes.POINTER(ctypes.c_size_t), ctypes.POINTER(ctypes.c_size_t)]
+    assert fn(ctypes.byref(make_cfg(128, 4, 16, 32, cf=4, levels=3)), ctypes.byref(f), ctypes.byref(a)) == 0
+    assert f.value > 0 and a.value > f.value
+    assert fn(ctypes.byref(make_cfg(100, 4, 16, 32, cf=8, levels=3)), ctypes.byref(f), ctypes.byref(a)) == -2   # not divisible
+    assert fn(ctypes.byref(make_cfg(128, 4, 16, 32, cf=1, levels=2)), ctypes.byref(f), ctypes.byref(a)) == -1   # cf < 2
+    assert fn(ctypes.byref(make_cfg(128, 4, 16, 36, cf=4, levels=2)), ctypes.byref(f), ctypes.byref(a)) == -4   # H % 8
+    assert fn(ctypes.byref(make_cfg(128, 4, 16, 32, cf=4, levels=2, operands=2)), ctypes.byref(f), ctypes.byref(a)) == -4  # bf16 needs H % 64
+    assert fn(None, ctypes.byref(f), ctypes.byref(a)) == -1
+    lib.mgrit_gru_strerror.restype = ctypes.c_char_p
+    assert b"divisible" in lib.mgrit_gru_strerror(-2)
+    lib.xent_head_workspace_bytes.restype = ctypes.c_size_t
+    assert lib.xent_head_workspace_bytes(32, 51) >= 32 * 51 * 4

@@ -213,3 +213,19 @@ def test_toy_ode_two_level_convergence_shape():
     assert all(b_ < a_ for a_, b_ in zip(errs, errs[1:]) if a_ > 1e-13)
     # residual and error of similar size, as in the printed run (ratio ~0.7)
     assert 0.05 < paper_res[0] / paper_err[0] < 2
+
+
+def test_finite_cycle_iterates_match_the_stored_fixture():
+    # regression fixture written by tests/golden/make_golden.py (oracle only); the iterates after 1-4 cycles
+    # have no closed form and the paper prints none
+    import importlib.util
+    spec = importlib.util.spec_from_file_location("make_golden", os.path.join(GOLDEN, "make_golden.py"))
+    mod = importlib.util.module_from_spec(spec)
+    spec.loader.exec_module(mod)
+    want = [l.split() for l in open(os.path.join(GOLDEN, "tiny_cycles.txt")) if not l.startswith("#")]
+    got = mod.rows()
+    assert len(want) == len(got) == 8
+    for w_, g_ in zip(want, got):
+        assert int(w_[0]) == g_[0] and int(w_[1]) == g_[1]
+        assert abs(float(w_[2]) - g_[2]) <= 1e-9 * float(w_[2])
+        assert abs(float(w_[3]) - g_[3]) <= 1e-9 * float(w_[3])
