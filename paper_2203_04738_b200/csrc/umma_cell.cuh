@@ -89,6 +89,7 @@ umma_cell_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
   auto eempty_bar = [&](int e) { return bars + 8u * (2 * C::kStages + 6 + e); };
   __shared__ uint32_t tmem_base_smem;
   __shared__ int abort_flag;
+  __shared__ uint32_t lds_sink[cellk::kThreads];   // see the operand-buffer release in the epilogue
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int H = p.H;
@@ -214,7 +215,18 @@ umma_cell_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
         tmem_ld8(taddr + UN + cu, az);
         tmem_ld8(taddr + 2 * UN + cu, an);
         tmem_ld_wait8x3(ar, az, an);
-        const int eb_done = eb;
+        // Release the operand buffer as soon as its values are in registers.  An mbarrier.arrive issued right
+        // after the ld.shared instructions is NOT ordered behind loads whose results are still in flight (the
+        // refilling TMA then overwrote rows that had not been read yet).  So one word that depends on every
+        // load's result is stored first: the store cannot issue before the loads have delivered, and the
+        // arrive issues after the store.
+        {
+          uint32_t dep = __float_as_uint(gr[0]) ^ __float_as_uint(gr[4]) ^ __float_as_uint(gz[0]) ^ __float_as_uint(gz[4]) ^
+                         __float_as_uint(gn[0]) ^ __float_as_uint(gn[4]) ^ __float_as_uint(hp[0]) ^ __float_as_uint(hp[4]);
+          if (HAS_G) dep ^= __float_as_uint(gg[0]) ^ __float_as_uint(gg[4]);
+          asm volatile("st.shared.b32 [%0], %1;" ::"r"(smem_u32(&lds_sink[threadIdx.x])), "r"(dep) : "memory");
+        }
+        mbar_arrive(eempty_bar(eb));
         if (++eb == 2) { eb = 0; ephase ^= 1u; }
         if (valid) {
           const int u = nt * UN + cu;
@@ -266,10 +278,6 @@ umma_cell_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
             }
           }
         }
-        // Release the operand buffer only here, after the values read from it have been used: an
-        // mbarrier.arrive issued right after the ld.shared instructions is not ordered behind loads whose
-        // results are still in flight, and the refilling TMA then overwrote rows that had not been read.
-        mbar_arrive(eempty_bar(eb_done));
       }
       if (!ok) break;
       tc_fence_before();
