@@ -79,6 +79,33 @@ bool launch_gemm(int kc, const bf16* A, i64 lda, const bf16* Bm, i64 ldb, int M,
   return true;
 }
 
+// D[m, n] = sum_k A[k, m] * B[k, n]: both operands stored with the reduction index as the ROW index
+// (A: [K, Mdim], B: [K, Ndim], row-major), consumed as MN-major tensor-core operands -- the shape of the
+// weight-gradient reductions dW = dA^T h, which therefore need no transposed copies.
+template <class Epi>
+bool launch_gemm_mn(int kc, const bf16* A, i64 lda, int Mdim, const bf16* Bm, i64 ldb, int Ndim, int K, Epi epi, cudaStream_t s) {
+  using C = Cfg<256, false>;
+  if (Mdim <= 0 || Ndim <= 0) return true;
+  if (!ensure_driver()) return false;
+  static bool attr_set = false;
+  auto kern = umma_gemm_kernel<256, false, Epi, true>;
+  if (!attr_set) {
+    if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, C::kSmemBytes) != cudaSuccess) return false;
+    attr_set = true;
+  }
+  CUtensorMap ta, tb;
+  if (!make_map(&ta, A, (uint64_t)Mdim, (uint64_t)K, (uint64_t)lda, 64)) return false;
+  if (!make_map(&tb, Bm, (uint64_t)Ndim, (uint64_t)K, (uint64_t)ldb, 64)) return false;
+  GemmShape sh{Mdim, Ndim, K, 0};
+  int tiles = ((Mdim + BM - 1) / BM) * ((Ndim + 255) / 256);
+  int grid = tiles < kSMs ? tiles : kSMs;
+  prof_begin(kc, 2.0 * Mdim * (double)Ndim * K, s);
+  kern<<<grid, kThreads, C::kSmemBytes, s>>>(ta, tb, sh, epi, g_status_ptr);
+  prof_end(s);
+  count_launch();
+  return true;
+}
+
 // 3-D map {column, batch row, k}: rows (k, b) at base + k*ks + b*ld, `inner` columns
 bool make_map3(CUtensorMap* m, CUtensorMapDataType dt, size_t esize, const void* base, uint64_t inner, uint64_t B, uint64_t nk,
                uint64_t ld, i64 ks, uint32_t box_inner, uint32_t box_k, CUtensorMapSwizzle sw) {
@@ -374,57 +401,53 @@ __global__ void __launch_bounds__(1024) transpose_kernel(const float* __restrict
   if (rr < R && cc < C) dst[(i64)cc * dst_ld + col0 + rr] = __float2bfloat16(tile[threadIdx.x][threadIdx.y]);
 }
 
-// Gradient-pass operands from the final sensitivities: dA_h = [cr|cz|cn]*lam, dA_i = [cr|cz|cnp]*lam.
-// Writes dA_h^T, dA_i^T ([3H, M] bf16), optionally dA_i ([M, 3H] bf16), and adds the fp32 column sums
-// (bias gradients) of 32-row x 32-unit tiles into db_hh / db_ih.
-__global__ void __launch_bounds__(1024) form_dA_T_kernel(const float* __restrict__ lam, const float* __restrict__ cr,
-                                                         const float* __restrict__ cz, const float* __restrict__ cn,
-                                                         const float* __restrict__ cnp, i64 M, int H, bf16* __restrict__ dAhT,
-                                                         bf16* __restrict__ dAiT, bf16* __restrict__ dAi,
-                                                         float* __restrict__ db_hh, float* __restrict__ db_ih, int row_tiles) {
-  __shared__ float t[4][32][33];
-  const int tx = threadIdx.x, ty = threadIdx.y;
-  const int i = blockIdx.y * 32 + tx;
-  float s[4] = {0.f, 0.f, 0.f, 0.f};
-  for (int rt = 0; rt < row_tiles; ++rt) {
-    i64 m0 = ((i64)blockIdx.x * row_tiles + rt) * 32;
-    if (m0 >= M) break;
-    i64 m = m0 + ty;
-    float v[4] = {0.f, 0.f, 0.f, 0.f};
-    if (m < M && i < H) {
-      i64 e = m * H + i;
-      float l = lam[e];
-      v[0] = cr[e] * l; v[1] = cz[e] * l; v[2] = cn[e] * l; v[3] = cnp[e] * l;
-      if (dAi) {
-        i64 o = m * 3 * H + i;
-        dAi[o] = __float2bfloat16(v[0]); dAi[o + H] = __float2bfloat16(v[1]); dAi[o + 2 * H] = __float2bfloat16(v[3]);
-      }
-    }
+// Gradient-pass operands, row-major: dA_h = [cr|cz|cn]*lam and dA_i = [cr|cz|cnp]*lam as bf16 [M, 3H], plus the
+// fp32 column sums (bias gradients) added into db_hh / db_ih.  Block = 32 float4 columns (128 units) x 8 rows.
+__global__ void __launch_bounds__(256) form_dA_rows_kernel(const float* __restrict__ lam, const float* __restrict__ cr,
+                                                           const float* __restrict__ cz, const float* __restrict__ cn,
+                                                           const float* __restrict__ cnp, i64 M, int H, uint2* __restrict__ dAh,
+                                                           uint2* __restrict__ dAi, float* __restrict__ db_hh,
+                                                           float* __restrict__ db_ih, int rows_per_block) {
+  __shared__ float red[4][8][128];
+  const int tx = threadIdx.x & 31, ty = threadIdx.x >> 5;
+  const int H4 = H / 4, c4 = blockIdx.y * 32 + tx;
+  const i64 m0 = (i64)blockIdx.x * rows_per_block;
+  float4 s[4];
 #pragma unroll
-    for (int g = 0; g < 4; ++g) { t[g][ty][tx] = v[g]; s[g] += v[g]; }
-    __syncthreads();
-    i64 mm = m0 + tx; int ii = blockIdx.y * 32 + ty;
-    if (mm < M && ii < H) {
-      bf16 r_ = __float2bfloat16(t[0][tx][ty]), z_ = __float2bfloat16(t[1][tx][ty]);
-      dAhT[(i64)ii * M + mm] = r_;            dAiT[(i64)ii * M + mm] = r_;
-      dAhT[((i64)H + ii) * M + mm] = z_;      dAiT[((i64)H + ii) * M + mm] = z_;
-      dAhT[((i64)2 * H + ii) * M + mm] = __float2bfloat16(t[2][tx][ty]);
-      dAiT[((i64)2 * H + ii) * M + mm] = __float2bfloat16(t[3][tx][ty]);
+  for (int g = 0; g < 4; ++g) s[g] = make_float4(0.f, 0.f, 0.f, 0.f);
+  if (c4 < H4) {
+    for (i64 m = m0 + ty; m < m0 + rows_per_block && m < M; m += 8) {
+      i64 e = m * H4 + c4;
+      float4 l = reinterpret_cast<const float4*>(lam)[e];
+      float4 r = reinterpret_cast<const float4*>(cr)[e], z = reinterpret_cast<const float4*>(cz)[e];
+      float4 n = reinterpret_cast<const float4*>(cn)[e], q = reinterpret_cast<const float4*>(cnp)[e];
+      float4 v[4] = {make_float4(r.x * l.x, r.y * l.y, r.z * l.z, r.w * l.w), make_float4(z.x * l.x, z.y * l.y, z.z * l.z, z.w * l.w),
+                     make_float4(n.x * l.x, n.y * l.y, n.z * l.z, n.w * l.w), make_float4(q.x * l.x, q.y * l.y, q.z * l.z, q.w * l.w)};
+      i64 o = m * 3 * H4 + c4;
+      uint2 pr = pack4(v[0]), pz = pack4(v[1]);
+      dAh[o] = pr; dAi[o] = pr;
+      dAh[o + H4] = pz; dAi[o + H4] = pz;
+      dAh[o + 2 * H4] = pack4(v[2]);
+      dAi[o + 2 * H4] = pack4(v[3]);
+#pragma unroll
+      for (int g = 0; g < 4; ++g) { s[g].x += v[g].x; s[g].y += v[g].y; s[g].z += v[g].z; s[g].w += v[g].w; }
     }
-    __syncthreads();
   }
-  // column sums over this block's rows
 #pragma unroll
-  for (int g = 0; g < 4; ++g) t[g][ty][tx] = s[g];
+  for (int g = 0; g < 4; ++g) {
+    red[g][ty][tx * 4] = s[g].x; red[g][ty][tx * 4 + 1] = s[g].y; red[g][ty][tx * 4 + 2] = s[g].z; red[g][ty][tx * 4 + 3] = s[g].w;
+  }
   __syncthreads();
-  if (ty < 4 && i < H) {
+  for (int e = threadIdx.x; e < 4 * 128; e += 256) {
+    int g = e / 128, u = e % 128, col = blockIdx.y * 128 + u;
+    if (col >= H) continue;
     float acc = 0.f;
 #pragma unroll
-    for (int r = 0; r < 32; ++r) acc += t[ty][r][tx];
-    if (ty == 0) { atomicAdd(db_hh + i, acc); atomicAdd(db_ih + i, acc); }
-    else if (ty == 1) { atomicAdd(db_hh + H + i, acc); atomicAdd(db_ih + H + i, acc); }
-    else if (ty == 2) atomicAdd(db_hh + 2 * H + i, acc);
-    else atomicAdd(db_ih + 2 * H + i, acc);
+    for (int r = 0; r < 8; ++r) acc += red[g][r][u];
+    if (g == 0) { atomicAdd(db_hh + col, acc); atomicAdd(db_ih + col, acc); }
+    else if (g == 1) { atomicAdd(db_hh + H + col, acc); atomicAdd(db_ih + H + col, acc); }
+    else if (g == 2) atomicAdd(db_hh + 2 * H + col, acc);
+    else atomicAdd(db_ih + 2 * H + col, acc);
   }
 }
 
@@ -477,14 +500,11 @@ void umma_plan_adj(const mgrit_gru_cfg* c, const int* N, int L, char* base, size
   size_t apack = o->maxM * 3 * H;
   if (TB * H > apack) apack = TB * H;     // the linearisation packs all T*B rows of a level at once
   o->Apack = take<bf16>(base, off, apack);
-  o->dAhT = take<bf16>(base, off, 3 * H * TB);
-  o->dAiT = take<bf16>(base, off, 3 * H * TB);
+  o->dAh = take<bf16>(base, off, 3 * H * TB);
   o->dAi = take<bf16>(base, off, 3 * H * TB);
-  o->hprevT = take<bf16>(base, off, H * TB);
-  o->xT = take<bf16>(base, off, I * TB);
-  o->dbpart = nullptr;
-  o->hb0 = take<bf16>(base, off, (size_t)c->B * H);
-  o->hb = take<bf16>(base, off, TB * H);
+  o->xb = take<bf16>(base, off, I * TB);
+  o->hb0 = take<bf16>(base, off, (size_t)c->B * H + TB * H);   // [h_0; h] contiguous: rows (t, b) of h_{t-1} start at hb0
+  o->hb = o->hb0 ? o->hb0 + (size_t)c->B * H : nullptr;
 }
 
 int umma_prepare_fwd(const mgrit_gru_cfg* c, const gru_params* p, const float* x, float* gi, UmmaFwdWs* w, cudaStream_t s) {
@@ -568,21 +588,20 @@ int umma_gradients(const mgrit_gru_cfg* c, const gru_params* p, const float* x, 
   const i64 M = (i64)c->T * B;
   cudaMemsetAsync(g->db_hh, 0, sizeof(float) * 3 * H, s);
   cudaMemsetAsync(g->db_ih, 0, sizeof(float) * 3 * H, s);
-  const int row_tiles = 16;
-  dim3 grid((unsigned)((M + 32 * row_tiles - 1) / (32 * row_tiles)), (H + 31) / 32);
-  form_dA_T_kernel<<<grid, dim3(32, 32), 0, s>>>(lam, cr, cz, cn, cnp, M, H, w->dAhT, w->dAiT, dx ? w->dAi : nullptr, g->db_hh,
-                                                 g->db_ih, row_tiles);
+  // operands of the three gradient GEMMs, all row-major (the reduction index t,b is the row index)
+  bf16* dAh = w->dAh; bf16* dAi = w->dAi;        // [M, 3H] each
+  const int rows_per_block = 256;
+  dim3 grid((unsigned)((M + rows_per_block - 1) / rows_per_block), (H / 4 + 31) / 32);
+  form_dA_rows_kernel<<<grid, 256, 0, s>>>(lam, cr, cz, cn, cnp, M, H, reinterpret_cast<uint2*>(dAh), reinterpret_cast<uint2*>(dAi),
+                                           g->db_hh, g->db_ih, rows_per_block);
   count_launch();
-  // h_{t-1} for t = 1..T, transposed: columns (t, b)
-  transpose(h0, B, H, w->hprevT, M, 0, s);
-  transpose(h, M - B, H, w->hprevT, M, B, s);
-  transpose(x, M, I, w->xT, M, 0, s);
+  convert(x, w->xb, M * I, s);                   // x as bf16 [M, I]; h_{t-1} as bf16 = [h_0; h] without its last slot (w->hb0)
   bool ok = true;
-  // dW_hh[3H, H] = dA_h^T h_prev ;  dW_ih[3H, I] = dA_i^T x    (K = T*B)
-  ok = ok && launch_gemm<256, false>(KC_WGRAD, w->dAhT, M, w->hprevT, M, 3 * H, H, (int)M, 0, H, EpiStore{g->dW_hh, H, 3 * H, H}, s);
-  ok = ok && launch_gemm<256, false>(KC_WGRAD, w->dAiT, M, w->xT, M, 3 * H, I, (int)M, 0, I, EpiStore{g->dW_ih, I, 3 * H, I}, s);
-  // dx[T*B, I] = dA_i W_ih   (K = 3H)
-  if (dx) ok = ok && launch_gemm<256, false>(KC_WGRAD, w->dAi, 3 * H, w->W_ihT, 3 * H, (int)M, I, 3 * H, 0, I, EpiStore{dx, I, (int)M, I}, s);
+  // dW_hh[3H, H] = dA_h^T h_prev ;  dW_ih[3H, I] = dA_i^T x    (K = T*B, MN-major operands)
+  ok = ok && launch_gemm_mn(KC_WGRAD, dAh, 3 * H, 3 * H, w->hb0, H, H, (int)M, EpiStore{g->dW_hh, H, 3 * H, H}, s);
+  ok = ok && launch_gemm_mn(KC_WGRAD, dAi, 3 * H, 3 * H, w->xb, I, I, (int)M, EpiStore{g->dW_ih, I, 3 * H, I}, s);
+  // dx[T*B, I] = dA_i W_ih   (K = 3H, K-major operands)
+  if (dx) ok = ok && launch_gemm<256, false>(KC_WGRAD, dAi, 3 * H, w->W_ihT, 3 * H, (int)M, I, 3 * H, 0, I, EpiStore{dx, I, (int)M, I}, s);
   return ok ? MGRIT_OK : MGRIT_CUDA_ERROR;
 }
 

@@ -17,14 +17,11 @@ struct UmmaAdjWs {
   __nv_bfloat16* W_hhT;   // [H,3H]   (adjoint step: B operand, K = 3H contiguous)
   __nv_bfloat16* W_ihT;   // [I,3H]   (dx = dA_i W_ih)
   __nv_bfloat16* Apack;   // [maxM,3H]
-  __nv_bfloat16* dAhT;    // [3H,T*B]
-  __nv_bfloat16* dAiT;    // [3H,T*B]
-  __nv_bfloat16* dAi;     // [T*B,3H]
-  __nv_bfloat16* hprevT;  // [H,T*B]
-  __nv_bfloat16* xT;      // [I,T*B]
-  float* dbpart;          // partial column sums
-  __nv_bfloat16* hb0;     // [B,H]    bf16 copy of h_0
-  __nv_bfloat16* hb;      // [T*B,H]  bf16 copy of the given states
+  __nv_bfloat16* dAh;     // [T*B,3H]  gradient-pass operand [cr|cz|cn]*lambda
+  __nv_bfloat16* dAi;     // [T*B,3H]  gradient-pass operand [cr|cz|cn']*lambda
+  __nv_bfloat16* xb;      // [T*B,I]   bf16 copy of the layer input
+  __nv_bfloat16* hb0;     // [(T+1)*B,H] bf16 copy of [h_0; h]: row (t,b) is h_{t-1} of step t
+  __nv_bfloat16* hb;      // = hb0 + B*H: the given states
   size_t maxM;
 };
 

@@ -88,10 +88,26 @@ __device__ __forceinline__ uint64_t smem_desc_sw128(uint32_t addr) {
   return d;
 }
 
+// Same for an MN-major operand (the matrix is stored [K rows][MN columns]): the stage holds one
+// [64 k][64 mn] box (8 KiB, 128-byte rows) per 64 MN elements; leading byte offset = distance between
+// those boxes, stride byte offset = distance between groups of 8 k rows.
+__device__ __forceinline__ uint64_t smem_desc_mn_sw128(uint32_t addr) {
+  uint64_t d = 0;
+  d |= (uint64_t)((addr & 0x3FFFFu) >> 4);
+  d |= (uint64_t)(8192 >> 4) << 16;
+  d |= (uint64_t)(1024 >> 4) << 32;
+  d |= (uint64_t)1 << 46;
+  d |= (uint64_t)2 << 61;
+  return d;
+}
+
 // Instruction descriptor: D fp32, A and B bf16, both K-major, M = 128, N = n.
 __host__ __device__ constexpr uint32_t instr_desc_bf16(int n) {
   return (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(n >> 3) << 17) | ((uint32_t)(BM >> 4) << 24);
 }
+
+// ... both MN-major (bits 15 and 16)
+__host__ __device__ constexpr uint32_t instr_desc_bf16_mn(int n) { return instr_desc_bf16(n) | (1u << 15) | (1u << 16); }
 
 __device__ __forceinline__ void mma_bf16(uint32_t d_tmem, uint64_t adesc, uint64_t bdesc, uint32_t idesc, uint32_t accumulate) {
   asm volatile(
@@ -141,7 +157,8 @@ struct Cfg {
 //   row: global output row of this thread (may be >= M: then only the tcgen05.ld's are executed)
 //   n0 : first output column (GATES: first hidden unit) of the tile
 //   half: 0 or 1, the half of the tile's output columns this warp is responsible for
-template <int BN, bool GATES, class Epi>
+// MNMAJ: D[m, n] = sum_k A[k, m] * B[k, n] with A stored [K, M] and B stored [K, N] (both row-major)
+template <int BN, bool GATES, class Epi, bool MNMAJ = false>
 __global__ void __launch_bounds__(kThreads, 1)
 umma_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB, GemmShape sh, Epi epi,
                  int* status) {
@@ -194,6 +211,12 @@ umma_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
           const uint32_t a_dst = tiles_base + stage * C::kStageBytes;
           const uint32_t b_dst = a_dst + C::kABytes;
           mbar_expect_tx(full_bar(stage), C::kStageBytes);
+          if (MNMAJ) {
+#pragma unroll
+            for (int i = 0; i < BM / 64; ++i) tma_load_2d(a_dst + i * 8192, &tmA, full_bar(stage), mt * BM + i * 64, kb * BK);
+#pragma unroll
+            for (int i = 0; i < BN / 64; ++i) tma_load_2d(b_dst + i * 8192, &tmB, full_bar(stage), nt * BN + i * 64, kb * BK);
+          } else {
           tma_load_2d(a_dst, &tmA, full_bar(stage), kb * BK, mt * BM);
           if (GATES) {
 #pragma unroll
@@ -202,6 +225,7 @@ umma_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
           } else {
             tma_load_2d(b_dst, &tmB, full_bar(stage), kb * BK, nt * BN);
           }
+          }
           if (++stage == C::kStages) { stage = 0; phase ^= 1u; }
         }
       }
@@ -209,7 +233,7 @@ umma_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
   } else if (warp == 1) {
     // ------------------------------------------------------------ MMA issuer
     if (lane == 0) {
-      constexpr uint32_t idesc = instr_desc_bf16(BN);
+      constexpr uint32_t idesc = MNMAJ ? instr_desc_bf16_mn(BN) : instr_desc_bf16(BN);
       int stage = 0; uint32_t phase = 0;
       int it = 0;
       bool ok = true;
@@ -223,11 +247,13 @@ umma_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
           if (!mbar_wait(full_bar(stage), phase, abortp, status, 3)) { ok = false; break; }
           tc_fence_after();
           const uint32_t a_src = tiles_base + stage * C::kStageBytes;
-          const uint64_t adesc = smem_desc_sw128(a_src);
-          const uint64_t bdesc = smem_desc_sw128(a_src + C::kABytes);
+          const uint64_t adesc = MNMAJ ? smem_desc_mn_sw128(a_src) : smem_desc_sw128(a_src);
+          const uint64_t bdesc = MNMAJ ? smem_desc_mn_sw128(a_src + C::kABytes) : smem_desc_sw128(a_src + C::kABytes);
+          // one MMA consumes 16 k: 32 bytes along a K-major row, 16 rows of 128 bytes (2048 bytes) when MN-major
+          constexpr uint64_t kstep = MNMAJ ? (2048 >> 4) : (32 >> 4);
 #pragma unroll
           for (int k = 0; k < BK / 16; ++k)
-            mma_bf16(d_tmem, adesc + (uint64_t)(k * 2), bdesc + (uint64_t)(k * 2), idesc, (kb | k) != 0 ? 1u : 0u);
+            mma_bf16(d_tmem, adesc + kstep * k, bdesc + kstep * k, idesc, (kb | k) != 0 ? 1u : 0u);
           mma_commit(empty_bar(stage));   // frees the stage when the MMAs have read it
           if (++stage == C::kStages) { stage = 0; phase ^= 1u; }
         }
