@@ -23,9 +23,10 @@ sys.path.insert(0, ROOT)
 
 METRIC = "MGRIT-GRU fwd+adjoint timesteps*batch/sec"
 UNIT = "timesteps*batch/s"
-# DRAM bytes (read + write) per launch of the forward relaxation-step GEMM, from the ncu capture
-# summarised in profiles/ (per workload); None where no capture exists.
-NCU_TRAFFIC_BYTES_PER_LAUNCH = {}
+# DRAM bytes (read + write) of the fused forward-step kernel per (row x hidden unit), from the ncu capture
+# summarised in profiles/fused_cell_kernel_medium.md (81.7 MB for 8192 rows x 512 units).  Traffic grows in
+# proportion to rows x hidden units, so a workload's per-launch traffic is this figure x its average rows x H.
+NCU_DRAM_BYTES_PER_ROW_UNIT = {"forward_step": 19.5}
 
 
 def measured_peaks():
@@ -273,7 +274,11 @@ def main():
                 peak = 148 * 128 * 2 * float(peaks.get("sm_max_mhz", 1965.0)) * 1e6 / 1e12
                 bound, note = "alu", "fp32 FFMA: 148 SMs x 128 lanes x 2 flop x max SM clock"
             roofline = {"kernel": name, "bound": bound, "achieved": achieved, "peak": peak, "unit": "TFLOP/s",
-                        "frac": achieved / peak, "traffic": NCU_TRAFFIC_BYTES_PER_LAUNCH.get(w.name),
+                        "frac": achieved / peak,
+                        "traffic": (NCU_DRAM_BYTES_PER_ROW_UNIT[name] * (fl / n) / (6.0 * w.H)
+                                    if name in NCU_DRAM_BYTES_PER_ROW_UNIT else None),
+                        "traffic_note": "DRAM bytes per launch, scaled from the ncu capture of a smaller case by rows x hidden units",
+                        "algorithmic_bytes": 24.0 * (fl / n) / (6.0 * w.H) if name == "forward_step" else None,
                         "avg_launch_us": tms / n * 1e3, "launches_per_step": n // nprof,
                         "share_of_gemm_time": tms / max(sum(v[0] for v in prof.values()), 1e-9), "peak_source": note}
 
