@@ -41,8 +41,8 @@ __device__ __forceinline__ int ld_relaxed(const int* p) {
 __device__ __forceinline__ bool grid_barrier(unsigned* ctr, unsigned target, int* status, int* ok_smem) {
   __syncthreads();
   if (threadIdx.x == 0) {
-    __threadfence();
-    atomicAdd(ctr, 1u);
+    // release: the CTA's stores (ordered before this thread by the barrier above) become visible before the count
+    asm volatile("red.release.gpu.global.add.u32 [%0], 1;" ::"l"(ctr) : "memory");
     int ok = 1;
     unsigned spins = 0;
     uint64_t t0 = 0;
@@ -53,8 +53,7 @@ __device__ __forceinline__ bool grid_barrier(unsigned* ctr, unsigned target, int
         if (global_ns() - t0 > kWaitLimitNs) { atomicCAS(status, 0, 5); ok = 0; break; }
       }
     }
-    __threadfence();
-    *ok_smem = ok;
+    *ok_smem = ok;      // the acquire load above orders the reloads that follow the barrier below
   }
   __syncthreads();
   return *ok_smem != 0;
