@@ -157,6 +157,14 @@ int xent_head_fwd_bwd_noalloc(int32_t B, int32_t H, int32_t C, const float* hT, 
 /* Theta <- Theta - lr * g (last line of Algorithm "MGRITTraining"); n fp32 elements. */
 int sgd_update(float* p, const float* g, size_t n, float lr, mgrit_stream_t stream);
 
+/* Adam step with bias correction, the optimiser of the paper's experiments (Section "Training with MGRIT";
+ * tables of training parameters: Adam, learning rate 0.001).  Same update as the usual Adam without weight
+ * decay:  m <- b1 m + (1-b1) g;  v <- b2 v + (1-b2) g^2;  p <- p - lr/(1-b1^t) * m / (sqrt(v)/sqrt(1-b2^t) + eps).
+ * p, g, m, v: n fp32 elements each (device; m and v are the caller-owned moment buffers, zero before step 1);
+ * step = t >= 1. */
+int adam_update(float* p, const float* g, float* m, float* v, size_t n, float lr, float beta1, float beta2, float eps,
+                int32_t step, mgrit_stream_t stream);
+
 /* Status word written by bounded device-side waits since the library was loaded (0 = none ran out).
  * Synchronises the device. */
 int mgrit_gru_last_device_status(void);

@@ -18,6 +18,7 @@ What pins each function (see tests/test_oracle_*.py):
                                                 propagator for the linear adjoint problem,
                                                 hierarchy sizes quoted in the paper
   * loss head ................................. torch.nn.functional.cross_entropy float64
+  * Adam ...................................... torch.optim.Adam float64
   * values after a FEW cycles (2-3) ........... parity unpinned by the paper (an iteration's
                                                 intermediate iterates have no closed form);
                                                 they are covered only indirectly by the pins
@@ -328,3 +329,12 @@ def xent_head(hT, W_c, b_c, labels):
 def sgd_update(p, g, lr):
     """Theta <- Theta - l_r g (last line of Algorithm "MGRITTraining")."""
     return p - lr * g
+
+
+def adam_update(p, g, m, v, lr, step, beta1=0.9, beta2=0.999, eps=1e-8):
+    """Adam step with bias correction (the optimiser of the paper's experiments); returns new (p, m, v)."""
+    m = beta1 * m + (1.0 - beta1) * g
+    v = beta2 * v + (1.0 - beta2) * g * g
+    mhat = m / (1.0 - beta1 ** step)
+    vhat = v / (1.0 - beta2 ** step)
+    return p - lr * mhat / (np.sqrt(vhat) + eps), m, v

@@ -55,6 +55,7 @@ lib.xent_head_workspace_bytes.restype = _sz
 lib.xent_head_fwd_bwd.argtypes = [_i32, _i32, _i32, _vp, _vp, _vp, _vp, _vp, _vp, _vp, _vp, _vp, _sz, _vp]
 lib.xent_head_fwd_bwd_noalloc.argtypes = [_i32, _i32, _i32, _vp, _vp, _vp, _vp, _vp, _vp, _vp, _vp, _vp]
 lib.sgd_update.argtypes = [_vp, _vp, _sz, ctypes.c_float, _vp]
+lib.adam_update.argtypes = [_vp, _vp, _vp, _vp, _sz, ctypes.c_float, ctypes.c_float, ctypes.c_float, ctypes.c_float, _i32, _vp]
 lib.mgrit_gru_last_device_status.restype = ctypes.c_int
 lib.mgrit_gru_kernel_launches.restype = ctypes.c_ulonglong
 lib.mgrit_gru_profile_enable.argtypes = [ctypes.c_int]
@@ -217,6 +218,12 @@ def xent_head_fwd_bwd_noalloc(hT, Wc, bc, labels, out=None):
 
 def sgd_update(p, g, lr):
     _check(lib.sgd_update(_f32(p), _f32(g), p.numel(), ctypes.c_float(lr), _stream()))
+    return p
+
+
+def adam_update(p, g, m, v, lr, step, beta1=0.9, beta2=0.999, eps=1e-8):
+    _check(lib.adam_update(_f32(p), _f32(g), _f32(m), _f32(v), p.numel(), ctypes.c_float(lr), ctypes.c_float(beta1),
+                           ctypes.c_float(beta2), ctypes.c_float(eps), int(step), _stream()))
     return p
 
 

@@ -488,6 +488,15 @@ int sgd_update(float* p, const float* g, size_t n, float lr, mgrit_stream_t stre
   return finish((cudaStream_t)stream, false);
 }
 
+int adam_update(float* p, const float* g, float* m, float* v, size_t n, float lr, float beta1, float beta2, float eps, int32_t step,
+                mgrit_stream_t stream) {
+  if (!p || !g || !m || !v || step < 1 || !(beta1 >= 0.f && beta1 < 1.f) || !(beta2 >= 0.f && beta2 < 1.f) || !(eps > 0.f))
+    return MGRIT_INVALID_ARG;
+  if (n == 0) return MGRIT_OK;
+  stream_adam(p, g, m, v, n, lr, beta1, beta2, eps, step, (cudaStream_t)stream);
+  return finish((cudaStream_t)stream, false);
+}
+
 int mgrit_gru_last_device_status(void) {
   if (cudaDeviceSynchronize() != cudaSuccess) return MGRIT_CUDA_ERROR;
   return (umma_device_status() != 0 || serial_device_status() != 0) ? MGRIT_DEVICE_TIMEOUT : MGRIT_OK;

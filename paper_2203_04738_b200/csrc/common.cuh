@@ -89,5 +89,7 @@ void stream_sqrt_to_float(const double* acc, float* out, int n, cudaStream_t s);
 void stream_xent(int B, int H, int C, const float* hT, const float* Wc, const float* bc, const int32_t* labels,
                  float* loss, float* dhT, float* dWc, float* dbc, float* dlogits, cudaStream_t s);
 void stream_sgd(float* p, const float* g, size_t n, float lr, cudaStream_t s);
+void stream_adam(float* p, const float* g, float* m, float* v, size_t n, float lr, float b1, float b2, float eps, int step,
+                 cudaStream_t s);
 
 }  // namespace mg

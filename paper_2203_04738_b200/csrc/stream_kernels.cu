@@ -1,6 +1,8 @@
 // Streaming (HBM-bound) kernels: grid transfers of the multigrid cycle, operand forming for the
 // gradient pass, column sums, the classifier head and the SGD update.  float4 accesses,
 // coalesced along the hidden dimension; grids sized in multiples of the SM count.
+#include <math.h>
+
 #include "common.cuh"
 
 namespace mg {
@@ -201,7 +203,29 @@ __global__ void __launch_bounds__(kThreads) sgd_kernel(float* __restrict__ p, co
   for (size_t e = n4 * 4 + t; e < n; e += stride) p[e] -= lr * g[e];
 }
 
+// Adam with bias correction (the optimiser of the paper's experiments; same update as torch.optim.Adam without
+// weight decay): m <- b1 m + (1-b1) g, v <- b2 v + (1-b2) g^2, p <- p - lr/(1-b1^t) * m / (sqrt(v)/sqrt(1-b2^t) + eps).
+__global__ void __launch_bounds__(kThreads) adam_kernel(float* __restrict__ p, const float* __restrict__ g, float* __restrict__ m,
+                                                        float* __restrict__ v, size_t n, float step_size, float inv_sqrt_bc2,
+                                                        float b1, float b2, float eps) {
+  size_t stride = (size_t)gridDim.x * blockDim.x;
+  for (size_t e = (size_t)blockIdx.x * blockDim.x + threadIdx.x; e < n; e += stride) {
+    float gg = g[e];
+    float mm = b1 * m[e] + (1.f - b1) * gg;
+    float vv = b2 * v[e] + (1.f - b2) * gg * gg;
+    m[e] = mm; v[e] = vv;
+    p[e] -= step_size * mm / (sqrtf(vv) * inv_sqrt_bc2 + eps);
+  }
+}
+
 }  // namespace
+
+void stream_adam(float* p, const float* g, float* m, float* v, size_t n, float lr, float b1, float b2, float eps, int step,
+                 cudaStream_t s) {
+  double bc1 = 1.0 - pow((double)b1, (double)step), bc2 = 1.0 - pow((double)b2, (double)step);
+  adam_kernel<<<stream_grid((i64)n), kThreads, 0, s>>>(p, g, m, v, n, (float)(lr / bc1), (float)(1.0 / sqrt(bc2)), b1, b2, eps);
+  count_launch();
+}
 
 void stream_restrict_residual(const float* uf, int cf, const float* v, float* uc, __nv_bfloat16* ucb, int nc, i64 rowlen, double* acc,
                               cudaStream_t s) {

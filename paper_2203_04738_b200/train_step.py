@@ -50,9 +50,26 @@ def alloc_buffers(w: Workload, T: int, Bsz: int, device, serial: bool = False, f
                        [mk(T, Bsz, 3 * w.H) for _ in fw], [mk(T, Bsz, w.H) for _ in fw], adj, serial)
 
 
-def training_step(w: Workload, layers, W_c, b_c, x, h0, labels, buf: StepBuffers, lr: float = 1e-3, update: bool = True):
-    """Forward (all layers) -> loss head -> adjoint (top layer first) -> weight gradients -> SGD.
-    layers: list of dicts W_ih, W_hh, b_ih, b_hh (device fp32).  Returns the loss tensor (device)."""
+class AdamState:
+    """Moment buffers of the Adam optimiser (the optimiser of the paper's experiments), one pair per parameter."""
+
+    def __init__(self, params):
+        self.m = [torch.zeros_like(p) for p in params]
+        self.v = [torch.zeros_like(p) for p in params]
+        self.step = 0
+
+
+def all_params(layers, W_c, b_c):
+    out = []
+    for p in layers:
+        out += [p["W_ih"], p["W_hh"], p["b_ih"], p["b_hh"]]
+    return out + [W_c, b_c]
+
+
+def training_step(w: Workload, layers, W_c, b_c, x, h0, labels, buf: StepBuffers, lr: float = 1e-3, update: bool = True,
+                  adam: AdamState | None = None):
+    """Forward (all layers) -> loss head -> adjoint (top layer first) -> weight gradients -> SGD (or Adam when an
+    AdamState is given).  layers: list of dicts W_ih, W_hh, b_ih, b_hh (device fp32).  Returns the loss (device)."""
     inp = x
     for l, p in enumerate(layers):
         if buf.serial:
@@ -68,7 +85,16 @@ def training_step(w: Workload, layers, W_c, b_c, x, h0, labels, buf: StepBuffers
         fn(buf.cfgs_adj[l], layers[l], inp, h0, buf.gi[l], buf.h[l], dh_seed=seed, dhT=dhT if seed is None else None,
            want_dx=l > 0, ws=buf.ws_adj, out=buf.adj[l])
         seed = buf.adj[l].dx
-    if update:
+    if update and adam is not None:
+        grads = []
+        for l in range(len(layers)):
+            a = buf.adj[l]
+            grads += [a.dW_ih, a.dW_hh, a.db_ih, a.db_hh]
+        grads += [dWc, dbc]
+        adam.step += 1
+        for p_, g_, m_, v_ in zip(all_params(layers, W_c, b_c), grads, adam.m, adam.v):
+            B.adam_update(p_, g_, m_, v_, lr, adam.step)
+    elif update:
         for l, p in enumerate(layers):
             a = buf.adj[l]
             for name, g in (("W_ih", a.dW_ih), ("W_hh", a.dW_hh), ("b_ih", a.db_ih), ("b_hh", a.db_hh)):

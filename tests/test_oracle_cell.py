@@ -198,3 +198,17 @@ def test_xent_head_equals_library():
     assert np.max(np.abs(Wt.grad.numpy() - dW)) < 1e-13
     assert np.max(np.abs(bt.grad.numpy() - db)) < 1e-13
     assert np.allclose(O.sgd_update(Wc, dW, 0.5), Wc - 0.5 * dW)
+
+
+def test_adam_equals_library():
+    rng = np.random.default_rng(6)
+    p0 = rng.standard_normal(17)
+    pt = torch.from_numpy(p0.copy()).requires_grad_(True)
+    opt = torch.optim.Adam([pt], lr=1e-2)
+    p, m, v = p0.copy(), np.zeros(17), np.zeros(17)
+    for step in range(1, 6):
+        g = rng.standard_normal(17)
+        pt.grad = torch.from_numpy(g.copy())
+        opt.step()
+        p, m, v = O.adam_update(p, g, m, v, 1e-2, step)
+        assert np.max(np.abs(p - pt.detach().numpy())) < 1e-12
