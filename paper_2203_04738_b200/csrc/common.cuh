@@ -15,6 +15,27 @@ typedef long long i64;
 extern unsigned long long g_kernel_launches;
 inline void count_launch(int n = 1) { g_kernel_launches += (unsigned long long)n; }
 
+// Programmatic dependent launch: a kernel launched through launch_pdl() may become resident (and run its
+// prologue: barrier set-up, TMEM allocation, descriptor prefetch) while its predecessor in the stream is
+// still running.  Such a kernel calls pdl_wait() in EVERY thread before its first access to global memory
+// (the wait returns once the predecessor has completed and its writes are visible), then pdl_trigger() to
+// let its own successor start the same way.  At most two kernels overlap, and never their memory traffic.
+#ifdef __CUDACC__
+__device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+__device__ __forceinline__ void pdl_trigger() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+
+template <class... KArgs, class... Args>
+inline cudaError_t launch_pdl(void (*kern)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t s, Args&&... args) {
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = grid; cfg.blockDim = block; cfg.dynamicSmemBytes = smem; cfg.stream = s;
+  cudaLaunchAttribute at[1];
+  at[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  at[0].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = at; cfg.numAttrs = 1;
+  return cudaLaunchKernelEx(&cfg, kern, KArgs(args)...);
+}
+#endif
+
 // Optional per-launch timing of the GEMM-shaped kernels (CUDA events on the launching stream).
 enum KernelClass { KC_PROJ = 0, KC_FWD_STEP, KC_LINEARISE, KC_ADJ_STEP, KC_WGRAD, KC_FWD_SERIAL, KC_ADJ_SERIAL, KC_COUNT };
 extern bool g_prof_on;

@@ -115,6 +115,8 @@ umma_cell_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
   tc_fence_after();
   const uint32_t tmem_base = tmem_base_smem;
   volatile int* abortp = &abort_flag;
+  pdl_wait();     // everything above touched only shared memory and TMEM
+  pdl_trigger();
 
   if (warp == 0) {
     // ------------------------------------------------------------ A/B producer

@@ -73,7 +73,7 @@ bool launch_gemm(int kc, const bf16* A, i64 lda, const bf16* Bm, i64 ldb, int M,
   int tiles = m_tiles * n_tiles;
   int grid = tiles < kSMs ? tiles : kSMs;
   prof_begin(kc, 2.0 * M * (GATES ? 3.0 * N : (double)N) * K, s);
-  kern<<<grid, kThreads, C::kSmemBytes, s>>>(ta, tb, sh, epi, g_status_ptr);
+  if (launch_pdl(kern, dim3(grid), dim3(kThreads), C::kSmemBytes, s, ta, tb, sh, epi, g_status_ptr) != cudaSuccess) return false;
   prof_end(s);
   count_launch();
   return true;
@@ -100,7 +100,7 @@ bool launch_gemm_mn(int kc, const bf16* A, i64 lda, int Mdim, const bf16* Bm, i6
   int tiles = ((Mdim + BM - 1) / BM) * ((Ndim + 255) / 256);
   int grid = tiles < kSMs ? tiles : kSMs;
   prof_begin(kc, 2.0 * Mdim * (double)Ndim * K, s);
-  kern<<<grid, kThreads, C::kSmemBytes, s>>>(ta, tb, sh, epi, g_status_ptr);
+  if (launch_pdl(kern, dim3(grid), dim3(kThreads), C::kSmemBytes, s, ta, tb, sh, epi, g_status_ptr) != cudaSuccess) return false;
   prof_end(s);
   count_launch();
   return true;
@@ -150,7 +150,7 @@ bool launch_cell(int kc, const bf16* A, i64 a_ks, const float* gi, i64 gi_ks, co
   int tiles = ((ca.M + BM - 1) / BM) * (H / cellk::UN);
   int grid = tiles < kSMs ? tiles : kSMs;
   prof_begin(kc, 2.0 * ca.M * 3.0 * H * H, s);
-  kern<<<grid, cellk::kThreads, C::kSmemBytes, s>>>(ta, tb, tgi, thp, tg, ca, g_status_ptr);
+  if (launch_pdl(kern, dim3(grid), dim3(cellk::kThreads), C::kSmemBytes, s, ta, tb, tgi, thp, tg, ca, g_status_ptr) != cudaSuccess) return false;
   prof_end(s);
   count_launch();
   return true;
@@ -304,7 +304,8 @@ struct EpiLin {  // adjoint coefficients of every step of a level
   }
 };
 
-struct EpiAdj {  // lambda_prev = a*lambda + acc (+ source)
+template <int BN>
+struct EpiAdj {  // lambda_prev = a*lambda + acc (+ source); each epilogue warp half owns BN / 2 columns
   AdjStepArgs a;
   __device__ void operator()(uint32_t taddr, int row, int n0, int half) const {
     const bool valid = row < a.M;
@@ -313,9 +314,9 @@ struct EpiAdj {  // lambda_prev = a*lambda + acc (+ source)
     const float* __restrict__ ca = a.a + (i64)k * a.coef_ks + (i64)b * a.H + n0;
     float* __restrict__ lo = a.lout + (i64)k * a.lout_ks + (i64)b * a.H + n0;
     const float* __restrict__ ga = a.mode == 1 ? lo : (a.gadd ? a.gadd + (i64)k * a.gadd_ks + (i64)b * a.H + n0 : nullptr);
-    const int cbeg = half * 128;
+    const int cbeg = half * (BN / 2);
 #pragma unroll 2
-    for (int c0 = cbeg; c0 < cbeg + 128 && n0 + c0 < a.H; c0 += 16) {
+    for (int c0 = cbeg; c0 < cbeg + BN / 2 && n0 + c0 < a.H; c0 += 16) {
       float4 l4[4], a4[4], g4[4];
       if (valid) {
 #pragma unroll
@@ -361,6 +362,8 @@ __global__ void __launch_bounds__(kPT) convert_kernel(const float4* __restrict__
 // dst[m, :] = bf16(src row (k, b)),  m = k*B + b
 __global__ void __launch_bounds__(kPT) pack_rows_kernel(const float* __restrict__ src, i64 ks, int B, int H4, i64 M,
                                                         uint2* __restrict__ dst) {
+  pdl_wait();
+  pdl_trigger();
   i64 total = M * H4;
   for (i64 e = (i64)blockIdx.x * blockDim.x + threadIdx.x; e < total; e += (i64)gridDim.x * blockDim.x) {
     i64 m = e / H4; int c = (int)(e % H4);
@@ -373,6 +376,8 @@ __global__ void __launch_bounds__(kPT) pack_rows_kernel(const float* __restrict_
 __global__ void __launch_bounds__(kPT) pack_adj_kernel(const float* __restrict__ lin, i64 lin_ks, const float* __restrict__ cr,
                                                        const float* __restrict__ cz, const float* __restrict__ cn, i64 coef_ks,
                                                        int B, int H4, i64 M, uint2* __restrict__ dst) {
+  pdl_wait();
+  pdl_trigger();
   i64 total = M * H4;
   for (i64 e = (i64)blockIdx.x * blockDim.x + threadIdx.x; e < total; e += (i64)gridDim.x * blockDim.x) {
     i64 m = e / H4; int c = (int)(e % H4);
@@ -541,7 +546,7 @@ void umma_fwd_step(const FwdStepArgs& a, UmmaFwdWs* w, cudaStream_t s) {
     else launch_cell<false, false>(KC_FWD_STEP, a.hin_b, a.hin_ks, a.gi, a.gi_ks, a.hin, a.hin_ks, nullptr, 0, nk, w->W_hh, ca, s);
     return;
   }
-  pack_rows_kernel<<<pgrid((i64)a.M * (a.H / 4)), kPT, 0, s>>>(a.hin, a.hin_ks, a.B, a.H / 4, a.M, reinterpret_cast<uint2*>(w->Apack));
+  launch_pdl(pack_rows_kernel, dim3(pgrid((i64)a.M * (a.H / 4))), dim3(kPT), 0, s, a.hin, a.hin_ks, a.B, a.H / 4, (i64)a.M, reinterpret_cast<uint2*>(w->Apack));
   count_launch();
   launch_gemm<192, true>(KC_FWD_STEP, w->Apack, a.H, w->W_hh, a.H, a.M, a.H, a.H, a.H, 3 * a.H, EpiFwd{a}, s);
 }
@@ -564,21 +569,27 @@ void umma_linearise(const LinArgs& a, UmmaAdjWs* w, cudaStream_t s) {
     }
     return;
   }
-  pack_rows_kernel<<<pgrid((i64)a.B * (a.H / 4)), kPT, 0, s>>>(a.h0, 0, a.B, a.H / 4, a.B, reinterpret_cast<uint2*>(w->Apack));
+  launch_pdl(pack_rows_kernel, dim3(pgrid((i64)a.B * (a.H / 4))), dim3(kPT), 0, s, a.h0, (i64)0, a.B, a.H / 4, (i64)a.B, reinterpret_cast<uint2*>(w->Apack));
   count_launch();
   if (a.M > a.B) {
-    pack_rows_kernel<<<pgrid((i64)(a.M - a.B) * (a.H / 4)), kPT, 0, s>>>(a.h + (a.stride_t - 1) * BH, a.stride_t * BH, a.B, a.H / 4,
-                                                                         a.M - a.B, reinterpret_cast<uint2*>(w->Apack + BH));
+    launch_pdl(pack_rows_kernel, dim3(pgrid((i64)(a.M - a.B) * (a.H / 4))), dim3(kPT), 0, s, a.h + (a.stride_t - 1) * BH,
+               (i64)(a.stride_t * BH), a.B, a.H / 4, (i64)(a.M - a.B), reinterpret_cast<uint2*>(w->Apack + BH));
     count_launch();
   }
   launch_gemm<192, true>(KC_LINEARISE, w->Apack, a.H, w->W_hh, a.H, a.M, a.H, a.H, a.H, 3 * a.H, EpiLin{a}, s);
 }
 
 void umma_adj_step(const AdjStepArgs& a, UmmaAdjWs* w, cudaStream_t s) {
-  pack_adj_kernel<<<pgrid((i64)a.M * (a.H / 4)), kPT, 0, s>>>(a.lin, a.lin_ks, a.cr, a.cz, a.cn, a.coef_ks, a.B, a.H / 4, a.M,
-                                                              reinterpret_cast<uint2*>(w->Apack));
+  launch_pdl(pack_adj_kernel, dim3(pgrid((i64)a.M * (a.H / 4))), dim3(kPT), 0, s, a.lin, a.lin_ks, a.cr, a.cz, a.cn, a.coef_ks, a.B,
+             a.H / 4, (i64)a.M, reinterpret_cast<uint2*>(w->Apack));
   count_launch();
-  launch_gemm<256, false>(KC_ADJ_STEP, w->Apack, 3 * a.H, w->W_hhT, 3 * a.H, a.M, a.H, 3 * a.H, 0, a.H, EpiAdj{a}, s);
+  // Few-row launches (coarse levels, short prefixes) cannot fill the SMs with 256-column tiles and are
+  // bound by one CTA streaming all of K; 64-column tiles spread that stream over four times the CTAs.
+  const int tiles256 = ((a.M + BM - 1) / BM) * ((a.H + 255) / 256);
+  if (tiles256 * 2 <= kSMs)
+    launch_gemm<64, false>(KC_ADJ_STEP, w->Apack, 3 * a.H, w->W_hhT, 3 * a.H, a.M, a.H, 3 * a.H, 0, a.H, EpiAdj<64>{a}, s);
+  else
+    launch_gemm<256, false>(KC_ADJ_STEP, w->Apack, 3 * a.H, w->W_hhT, 3 * a.H, a.M, a.H, 3 * a.H, 0, a.H, EpiAdj<256>{a}, s);
 }
 
 int umma_gradients(const mgrit_gru_cfg* c, const gru_params* p, const float* x, const float* h0, const float* h, const float* lam,

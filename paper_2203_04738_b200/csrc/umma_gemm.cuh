@@ -143,7 +143,7 @@ struct GemmShape {
 
 template <int BN, bool GATES>
 struct Cfg {
-  static constexpr int kStages = GATES ? 5 : 4;
+  static constexpr int kStages = GATES ? 5 : (BN <= 64 ? 8 : 4);
   static constexpr int kABytes = BM * BK * 2;
   static constexpr int kBBytes = BN * BK * 2;
   static constexpr int kStageBytes = kABytes + kBBytes;
@@ -198,6 +198,8 @@ umma_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
   tc_fence_after();
   const uint32_t tmem_base = tmem_base_smem;
   volatile int* abortp = &abort_flag;
+  pdl_wait();     // everything above touched only shared memory and TMEM
+  pdl_trigger();
 
   if (warp == 0) {
     // ------------------------------------------------------------ TMA producer
