@@ -176,7 +176,7 @@ def main():
     import torch.distributed as dist
     from paper_2203_04738_b200 import binding as B
     from paper_2203_04738_b200.replicas import job_throughput, max_over_ranks
-    from paper_2203_04738_b200.train_step import alloc_buffers, training_step
+    from paper_2203_04738_b200.train_step import HostInputPipeline, alloc_buffers, training_step
 
     torch.cuda.set_device(local_rank)
     dev = torch.device("cuda", local_rank)
@@ -226,11 +226,18 @@ def main():
     # end to end: inputs start in pinned host memory, the loss is read back, every step
     e2e = None
     if not args.no_e2e:
+        # Every step's input is copied from pinned host memory inside the timed region; the copy of step k+1
+        # runs on a side stream while step k computes (two device buffers), and the loss is read back every step.
+        pipe = HostInputPipeline(x.shape, x.dtype, dev)
         barrier()
         e0.record()
-        for _ in range(args.steps):
-            x.copy_(x_host, non_blocking=True)
-            loss = step()
+        pipe.submit(x_host)
+        for k in range(args.steps):
+            xk = pipe.acquire()
+            if k + 1 < args.steps:
+                pipe.submit(x_host)
+            loss = training_step(w, layers, W_c, b_c, xk, h0, labels, buf)
+            pipe.release()
             loss_host.copy_(loss, non_blocking=True)
             torch.cuda.current_stream().synchronize()
         e1.record()
@@ -238,7 +245,8 @@ def main():
         ms2 = e0.elapsed_time(e1)
         ms2 = max_over_ranks(ms2, dev)
         e2e = {"value": job_throughput(T * w.B, ms2 / args.steps, world), "unit": UNIT,
-               "h2d_bytes_per_step": x_host.numel() * 4, "d2h_bytes_per_step": 4}
+               "h2d_bytes_per_step": x_host.numel() * 4, "d2h_bytes_per_step": 4,
+               "overlap": "input copy of step k+1 on a side stream during step k (all copies inside the timed region)"}
 
     # per-kernel timing pass (CUDA events around every GEMM-shaped launch; outside the timed region so
     # that the event records do not perturb it)

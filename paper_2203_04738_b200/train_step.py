@@ -50,6 +50,46 @@ def alloc_buffers(w: Workload, T: int, Bsz: int, device, serial: bool = False, f
                        [mk(T, Bsz, 3 * w.H) for _ in fw], [mk(T, Bsz, w.H) for _ in fw], adj, serial)
 
 
+class HostInputPipeline:
+    """Double-buffered staging of each step's input from pinned host memory.
+
+    The copy of step k+1's input runs on a side stream while step k computes, so an end-to-end step costs
+    max(copy, compute) instead of their sum.  Usage per step: ``x = acquire()`` (the compute stream waits
+    for that buffer's copy), optionally ``submit(next_host_input)``, run the step on ``x``, ``release()``.
+    No arithmetic here: two device buffers, one stream, four events."""
+
+    def __init__(self, shape, dtype, device):
+        self.bufs = [torch.empty(shape, dtype=dtype, device=device) for _ in range(2)]
+        self.stream = torch.cuda.Stream(device=device)
+        self.ready = [torch.cuda.Event() for _ in range(2)]
+        self.free = [None, None]
+        self.n_sub = 0
+        self.n_acq = 0
+
+    def submit(self, x_host: torch.Tensor) -> None:
+        i = self.n_sub % 2
+        self.n_sub += 1
+        if self.free[i] is not None:
+            self.stream.wait_event(self.free[i])      # the step that read this buffer has finished
+        with torch.cuda.stream(self.stream):
+            self.bufs[i].copy_(x_host, non_blocking=True)
+            self.ready[i].record(self.stream)
+
+    def acquire(self) -> torch.Tensor:
+        if self.n_acq >= self.n_sub:
+            raise RuntimeError("HostInputPipeline.acquire() without a submitted input")
+        i = self.n_acq % 2
+        torch.cuda.current_stream().wait_event(self.ready[i])
+        return self.bufs[i]
+
+    def release(self) -> None:
+        i = self.n_acq % 2
+        self.n_acq += 1
+        ev = torch.cuda.Event()
+        ev.record(torch.cuda.current_stream())
+        self.free[i] = ev
+
+
 class AdamState:
     """Moment buffers of the Adam optimiser (the optimiser of the paper's experiments), one pair per parameter."""
 
