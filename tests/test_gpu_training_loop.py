@@ -118,3 +118,31 @@ def test_training_with_mgrit_learns_like_serial_and_inference_agrees():
     assert agree >= 0.9 * total, (agree, total)
     assert correct >= 0.5 * total, (correct, total)       # chance is 0.25
     assert B.last_device_status() == 0
+
+
+def test_host_input_pipeline_feeds_the_right_inputs():
+    """Three steps with three DIFFERENT host inputs through the double-buffered pipeline give the same losses
+    as the same steps run on plainly copied inputs (no update, so the steps are independent)."""
+    from paper_2203_04738_b200.train_step import HostInputPipeline, alloc_buffers, training_step
+    w = Workload("hp", T=64, B=4, I=16, H=32, cf=4, levels=3, iters_fwd=2, iters_adj=1, relax_fine=0, relax_coarse=1,
+                 operands=0, classes=8, relu=False, seed=5)
+    d = make_inputs(w)
+    layers = [{n: to_dev(d["layers"][0][n]) for n in NAMES}]
+    W_c, b_c, h0, labels = to_dev(d["W_c"]), to_dev(d["b_c"]), to_dev(d["h0"]), to_dev(d["labels"])
+    buf = alloc_buffers(w, w.T, w.B, torch.device("cuda"))
+    rng = np.random.default_rng(9)
+    hosts = [torch.from_numpy(rng.standard_normal(d["x"].shape).astype(np.float32)).pin_memory() for _ in range(3)]
+    want = [float(training_step(w, layers, W_c, b_c, xh.cuda(), h0, labels, buf, update=False)) for xh in hosts]
+    pipe = HostInputPipeline(hosts[0].shape, hosts[0].dtype, torch.device("cuda"))
+    got = []
+    pipe.submit(hosts[0])
+    for k in range(3):
+        xk = pipe.acquire()
+        if k + 1 < 3:
+            pipe.submit(hosts[k + 1])
+        loss = training_step(w, layers, W_c, b_c, xk, h0, labels, buf, update=False)
+        pipe.release()
+        got.append(float(loss))
+    # the loss is a sum over batch rows accumulated with atomics, so equal inputs agree to rounding, not bitwise
+    assert np.max(np.abs(np.array(got) - np.array(want))) < 1e-5
+    assert min(abs(want[0] - want[1]), abs(want[1] - want[2]), abs(want[0] - want[2])) > 5e-5
