@@ -23,10 +23,12 @@ sys.path.insert(0, ROOT)
 
 METRIC = "MGRIT-GRU fwd+adjoint timesteps*batch/sec"
 UNIT = "timesteps*batch/s"
-# DRAM bytes (read + write) of the fused forward-step kernel per (row x hidden unit), from the ncu capture
-# summarised in profiles/fused_cell_kernel_medium.md (81.7 MB for 8192 rows x 512 units).  Traffic grows in
-# proportion to rows x hidden units, so a workload's per-launch traffic is this figure x its average rows x H.
-NCU_DRAM_BYTES_PER_ROW_UNIT = {"forward_step": 19.5}
+# DRAM bytes (read + write) of the fused forward-step kernel per (row x hidden unit), from ncu captures of that
+# kernel: 23.2 B on the default workload's own 16384-row launches (389 MB per launch, H = 1024;
+# profiles/fused_cell_kernel_train.md) and 19.5 B on the smaller `medium` case (81.7 MB for 8192 rows x 512 units,
+# where more of the previous step's output is still in L2; profiles/fused_cell_kernel_medium.md).  Traffic grows
+# in proportion to rows x hidden units, so a workload's per-launch traffic is its figure x its average rows x H.
+NCU_DRAM_BYTES_PER_ROW_UNIT = {"forward_step": {1024: 23.2, 512: 19.5}}
 
 
 def measured_peaks():
@@ -283,9 +285,9 @@ def main():
                 bound, note = "alu", "fp32 FFMA: 148 SMs x 128 lanes x 2 flop x max SM clock"
             roofline = {"kernel": name, "bound": bound, "achieved": achieved, "peak": peak, "unit": "TFLOP/s",
                         "frac": achieved / peak,
-                        "traffic": (NCU_DRAM_BYTES_PER_ROW_UNIT[name] * (fl / n) / (6.0 * w.H)
-                                    if name in NCU_DRAM_BYTES_PER_ROW_UNIT else None),
-                        "traffic_note": "DRAM bytes per launch, scaled from the ncu capture of a smaller case by rows x hidden units",
+                        "traffic": (NCU_DRAM_BYTES_PER_ROW_UNIT[name][w.H] * (fl / n) / (6.0 * w.H)
+                                    if w.H in NCU_DRAM_BYTES_PER_ROW_UNIT.get(name, {}) else None),
+                        "traffic_note": "DRAM bytes per average launch: ncu figure per (row x hidden unit) of this kernel at this H x the launch's rows x H",
                         "algorithmic_bytes": 24.0 * (fl / n) / (6.0 * w.H) if name == "forward_step" else None,
                         "avg_launch_us": tms / n * 1e3, "launches_per_step": n // nprof,
                         "share_of_gemm_time": tms / max(sum(v[0] for v in prof.values()), 1e-9), "peak_source": note}
