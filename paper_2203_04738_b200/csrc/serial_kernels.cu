@@ -59,6 +59,15 @@ __device__ __forceinline__ bool grid_barrier(unsigned* ctr, unsigned target, int
   return *ok_smem != 0;
 }
 
+// 16-byte asynchronous copy global (through L2, not L1) -> shared: no register staging, so a thread keeps all
+// of its copies of a reload in flight at once instead of a few dependent load/store pairs.
+__device__ __forceinline__ void cp_async16(void* smem_dst, const void* gsrc) {
+  asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"((uint32_t)__cvta_generic_to_shared(smem_dst)), "l"(gsrc) : "memory");
+}
+__device__ __forceinline__ void cp_async_wait_all() {
+  asm volatile("cp.async.commit_group;\n\tcp.async.wait_group 0;" ::: "memory");
+}
+
 __device__ __forceinline__ void mma16816(float* c, const uint32_t* a, uint32_t b0, uint32_t b1) {
   asm volatile(
       "mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
@@ -194,8 +203,9 @@ __global__ void __launch_bounds__(kThreads, 1) serial_fwd_kernel(SerialFwdArgs a
     // the full new state of this row group, as the bf16 A operand
     for (int e = tid; e < nrows * (H / 8); e += kThreads) {
       int r = e / (H / 8), c = e % (H / 8);
-      *reinterpret_cast<uint4*>(As + r * ldk + c * 8) = __ldcg(reinterpret_cast<const uint4*>(ub + (i64)(row0 + r) * H + c * 8));
+      cp_async16(As + r * ldk + c * 8, ub + (i64)(row0 + r) * H + c * 8);
     }
+    cp_async_wait_all();
     __syncthreads();
   }
 }
@@ -291,8 +301,9 @@ __global__ void __launch_bounds__(kThreads, 1) serial_adj_kernel(SerialAdjArgs a
     if (!grid_barrier(a.bar + rg, (unsigned)s * ncta_rg, status, &ok_smem)) return;
     for (int e = tid; e < nrows * (K / 8); e += kThreads) {
       int r = e / (K / 8), c = e % (K / 8);
-      *reinterpret_cast<uint4*>(As + r * ldk + c * 8) = __ldcg(reinterpret_cast<const uint4*>(dAb + (i64)(row0 + r) * K + c * 8));
+      cp_async16(As + r * ldk + c * 8, dAb + (i64)(row0 + r) * K + c * 8);
     }
+    cp_async_wait_all();
     __syncthreads();
   }
 }
