@@ -43,6 +43,13 @@ __device__ __forceinline__ void tmem_ld_wait8x3(float* a, float* b, float* c) {
                :
                : "memory");
 }
+// One 32-byte store per thread: a warp's lanes write 32 different rows, and two 16-byte stores per row would
+// reach L2 as two half-filled sector writes each.
+__device__ __forceinline__ void stg8(float* p, const float* v) {
+  asm volatile("st.global.v8.f32 [%0], {%1,%2,%3,%4,%5,%6,%7,%8};" ::"l"(p), "f"(v[0]), "f"(v[1]), "f"(v[2]), "f"(v[3]), "f"(v[4]),
+               "f"(v[5]), "f"(v[6]), "f"(v[7])
+               : "memory");
+}
 __device__ __forceinline__ float4 lds4(uint32_t addr) {
   float4 v;
   asm volatile("ld.shared.v4.f32 {%0,%1,%2,%3}, [%4];" : "=f"(v.x), "=f"(v.y), "=f"(v.z), "=f"(v.w) : "r"(addr));
@@ -247,9 +254,7 @@ umma_cell_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
               o[e] = HAS_G ? (p.mode == 1 ? gg[e] - phi : phi + gg[e]) : phi;
             }
             const i64 idx = (i64)k * p.hout_ks + (i64)b * H + u;
-            float* ho = p.hout + idx;
-            *reinterpret_cast<float4*>(ho) = make_float4(o[0], o[1], o[2], o[3]);
-            *reinterpret_cast<float4*>(ho + 4) = make_float4(o[4], o[5], o[6], o[7]);
+            stg8(p.hout + idx, o);
             if (p.hout_b) {
               __nv_bfloat162 p0 = __floats2bfloat162_rn(o[0], o[1]), p1 = __floats2bfloat162_rn(o[2], o[3]);
               __nv_bfloat162 p2 = __floats2bfloat162_rn(o[4], o[5]), p3 = __floats2bfloat162_rn(o[6], o[7]);
@@ -266,18 +271,11 @@ umma_cell_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
               oa[e] = L.a; ocr[e] = L.cr; ocz[e] = L.cz; ocn[e] = L.cn; ocp[e] = L.cnp;
             }
             const i64 idx = (i64)row * H + u;
-            *reinterpret_cast<float4*>(p.a + idx) = make_float4(oa[0], oa[1], oa[2], oa[3]);
-            *reinterpret_cast<float4*>(p.a + idx + 4) = make_float4(oa[4], oa[5], oa[6], oa[7]);
-            *reinterpret_cast<float4*>(p.cr + idx) = make_float4(ocr[0], ocr[1], ocr[2], ocr[3]);
-            *reinterpret_cast<float4*>(p.cr + idx + 4) = make_float4(ocr[4], ocr[5], ocr[6], ocr[7]);
-            *reinterpret_cast<float4*>(p.cz + idx) = make_float4(ocz[0], ocz[1], ocz[2], ocz[3]);
-            *reinterpret_cast<float4*>(p.cz + idx + 4) = make_float4(ocz[4], ocz[5], ocz[6], ocz[7]);
-            *reinterpret_cast<float4*>(p.cn + idx) = make_float4(ocn[0], ocn[1], ocn[2], ocn[3]);
-            *reinterpret_cast<float4*>(p.cn + idx + 4) = make_float4(ocn[4], ocn[5], ocn[6], ocn[7]);
-            if (p.cnp) {
-              *reinterpret_cast<float4*>(p.cnp + idx) = make_float4(ocp[0], ocp[1], ocp[2], ocp[3]);
-              *reinterpret_cast<float4*>(p.cnp + idx + 4) = make_float4(ocp[4], ocp[5], ocp[6], ocp[7]);
-            }
+            stg8(p.a + idx, oa);
+            stg8(p.cr + idx, ocr);
+            stg8(p.cz + idx, ocz);
+            stg8(p.cn + idx, ocn);
+            if (p.cnp) stg8(p.cnp + idx, ocp);
           }
         }
       }

@@ -161,6 +161,18 @@ bool launch_cell(int kc, const bf16* A, i64 a_ks, const float* gi, i64 gi_ks, co
 // Per 16-column chunk the global loads are issued first, then the accumulator is read, so that the
 // memory latency of a chunk overlaps its tcgen05.ld and the other warps' work.
 __device__ __forceinline__ float4 ld4(const float* p) { return *reinterpret_cast<const float4*>(p); }
+// 32-byte accesses: in these epilogues the lanes of a warp touch 32 different rows, so a 16-byte access uses half
+// of each 32-byte sector it moves; one 32-byte access per lane moves whole sectors.
+__device__ __forceinline__ void ld8(const float* p, float* v) {
+  asm volatile("ld.global.v8.f32 {%0,%1,%2,%3,%4,%5,%6,%7}, [%8];"
+               : "=f"(v[0]), "=f"(v[1]), "=f"(v[2]), "=f"(v[3]), "=f"(v[4]), "=f"(v[5]), "=f"(v[6]), "=f"(v[7])
+               : "l"(p));
+}
+__device__ __forceinline__ void st8(float* p, const float* v) {
+  asm volatile("st.global.v8.f32 [%0], {%1,%2,%3,%4,%5,%6,%7,%8};" ::"l"(p), "f"(v[0]), "f"(v[1]), "f"(v[2]), "f"(v[3]), "f"(v[4]),
+               "f"(v[5]), "f"(v[6]), "f"(v[7])
+               : "memory");
+}
 __device__ __forceinline__ float4 ldg4(const float* p) { return __ldg(reinterpret_cast<const float4*>(p)); }
 __device__ __forceinline__ void st4(float* p, float a, float b, float c, float d) {
   *reinterpret_cast<float4*>(p) = make_float4(a, b, c, d);
@@ -181,8 +193,10 @@ struct EpiBias {  // out[m, n] = acc + bias[n]      (input projection)
 #pragma unroll
         for (int i = 0; i < 16; i += 4) {
           float4 b = ldg4(bias + n0 + c0 + i);
-          st4(o + c0 + i, v[i] + b.x, v[i + 1] + b.y, v[i + 2] + b.z, v[i + 3] + b.w);
+          v[i] += b.x; v[i + 1] += b.y; v[i + 2] += b.z; v[i + 3] += b.w;
         }
+        st8(o + c0, v);
+        st8(o + c0 + 8, v + 8);
       }
     }
   }
@@ -199,8 +213,8 @@ struct EpiStore {  // out[m, n] = acc            (weight / input gradients)
       tmem_ld16(taddr + c0, v);
       tmem_ld_wait();
       if (valid) {
-#pragma unroll
-        for (int i = 0; i < 16; i += 4) st4(o + c0 + i, v[i], v[i + 1], v[i + 2], v[i + 3]);
+        st8(o + c0, v);
+        st8(o + c0 + 8, v + 8);
       }
     }
   }
@@ -317,12 +331,15 @@ struct EpiAdj {  // lambda_prev = a*lambda + acc (+ source); each epilogue warp 
     const int cbeg = half * (BN / 2);
 #pragma unroll 2
     for (int c0 = cbeg; c0 < cbeg + BN / 2 && n0 + c0 < a.H; c0 += 16) {
-      float4 l4[4], a4[4], g4[4];
+      float l[16], ac[16], g[16];
       if (valid) {
+        ld8(li + c0, l); ld8(li + c0 + 8, l + 8);
+        ld8(ca + c0, ac); ld8(ca + c0 + 8, ac + 8);
+        if (ga) {
+          ld8(ga + c0, g); ld8(ga + c0 + 8, g + 8);
+        } else {
 #pragma unroll
-        for (int i = 0; i < 4; ++i) {
-          l4[i] = ld4(li + c0 + 4 * i); a4[i] = ld4(ca + c0 + 4 * i);
-          g4[i] = ga ? ld4(ga + c0 + 4 * i) : make_float4(0.f, 0.f, 0.f, 0.f);
+          for (int i = 0; i < 16; ++i) g[i] = 0.f;
         }
       }
       float v[16];
@@ -330,12 +347,12 @@ struct EpiAdj {  // lambda_prev = a*lambda + acc (+ source); each epilogue warp 
       tmem_ld_wait();
       if (valid) {
 #pragma unroll
-        for (int i = 0; i < 4; ++i) {
-          float o0 = a4[i].x * l4[i].x + v[4 * i], o1 = a4[i].y * l4[i].y + v[4 * i + 1];
-          float o2 = a4[i].z * l4[i].z + v[4 * i + 2], o3 = a4[i].w * l4[i].w + v[4 * i + 3];
-          if (a.mode == 1) st4(lo + c0 + 4 * i, g4[i].x - o0, g4[i].y - o1, g4[i].z - o2, g4[i].w - o3);
-          else st4(lo + c0 + 4 * i, o0 + g4[i].x, o1 + g4[i].y, o2 + g4[i].z, o3 + g4[i].w);
+        for (int i = 0; i < 16; ++i) {
+          float o = ac[i] * l[i] + v[i];
+          v[i] = a.mode == 1 ? g[i] - o : o + g[i];
         }
+        st8(lo + c0, v);
+        st8(lo + c0 + 8, v + 8);
       }
     }
   }
