@@ -328,11 +328,12 @@ struct EpiAdj {  // lambda_prev = a*lambda + acc (+ source); each epilogue warp 
     const float* __restrict__ ca = a.a + (i64)k * a.coef_ks + (i64)b * a.H + n0;
     float* __restrict__ lo = a.lout + (i64)k * a.lout_ks + (i64)b * a.H + n0;
     const float* __restrict__ ga = a.mode == 1 ? lo : (a.gadd ? a.gadd + (i64)k * a.gadd_ks + (i64)b * a.H + n0 : nullptr);
-    const int cbeg = half * (BN / 2);
-#pragma unroll 2
-    for (int c0 = cbeg; c0 < cbeg + BN / 2 && n0 + c0 < a.H; c0 += 16) {
-      float l[16], ac[16], g[16];
-      if (valid) {
+    const int cbeg = half * (BN / 2), cend = cbeg + BN / 2;
+    // The operands of 16 columns come straight from global memory (each lane its own row) and the wait for the
+    // accumulator load is a compiler barrier, so the loads of the NEXT 16 columns are issued by hand before the
+    // current ones are consumed: two register sets, two column groups per trip.
+    auto load = [&](int c0, float* l, float* ac, float* g) {
+      if (valid && c0 < cend && n0 + c0 < a.H) {
         ld8(li + c0, l); ld8(li + c0 + 8, l + 8);
         ld8(ca + c0, ac); ld8(ca + c0 + 8, ac + 8);
         if (ga) {
@@ -342,6 +343,9 @@ struct EpiAdj {  // lambda_prev = a*lambda + acc (+ source); each epilogue warp 
           for (int i = 0; i < 16; ++i) g[i] = 0.f;
         }
       }
+    };
+    auto finish = [&](int c0, const float* l, const float* ac, const float* g) {
+      if (n0 + c0 >= a.H) return;          // warp-uniform: the accumulator load is collective
       float v[16];
       tmem_ld16(taddr + c0, v);
       tmem_ld_wait();
@@ -354,6 +358,15 @@ struct EpiAdj {  // lambda_prev = a*lambda + acc (+ source); each epilogue warp 
         st8(lo + c0, v);
         st8(lo + c0 + 8, v + 8);
       }
+    };
+    float l0[16], a0[16], g0[16], l1[16], a1[16], g1[16];
+    load(cbeg, l0, a0, g0);
+#pragma unroll 1
+    for (int c0 = cbeg; c0 < cend; c0 += 32) {
+      load(c0 + 16, l1, a1, g1);
+      finish(c0, l0, a0, g0);
+      load(c0 + 32, l0, a0, g0);
+      finish(c0 + 16, l1, a1, g1);
     }
   }
 };
