@@ -7,7 +7,8 @@
  * gradients, a classifier/loss head, the SGD update, and the exact serial sweep it converges to.
  *
  * Conventions
- *  - Every data pointer is a DEVICE pointer owned by the caller, 16-byte aligned, fp32, row-major,
+ *  - Every data pointer is a DEVICE pointer owned by the caller, 32-byte aligned (the kernels move whole
+ *    32-byte sectors per thread; a misaligned pointer is rejected with MGRIT_INVALID_ARG), fp32, row-major,
  *    time-major: x[T,B,I], gi[T,B,3H], h[T,B,H]; h[k] is the paper's h_{k+1}, h_0 is passed
  *    separately.  Gate order along 3H is r | z | n (Eq. "gru").
  *  - cfg, resnorm and the size outputs are HOST pointers.

@@ -58,6 +58,14 @@ struct Hier {
   int L; int N[kMaxLevels]; i64 stride_t[kMaxLevels]; float gamma[kMaxLevels];
 };
 
+// every data pointer must be 32-byte aligned (nullptr passes: optional arguments are checked for presence elsewhere)
+template <class... P>
+bool aligned32(P... ptrs) {
+  uintptr_t m = 0;
+  ((m |= (uintptr_t)(const void*)ptrs), ...);
+  return (m & 31u) == 0;
+}
+
 int check_cfg(const mgrit_gru_cfg* c, Hier* hr) {
   if (!c) return MGRIT_INVALID_ARG;
   if (c->T <= 0 || c->B <= 0 || c->I <= 0 || c->H <= 0 || c->levels < 1 || c->levels > kMaxLevels) return MGRIT_INVALID_ARG;
@@ -278,6 +286,7 @@ int fetch_resnorm(const double* acc, float* resnorm, int iters, cudaStream_t s) 
 int forward_impl(const mgrit_gru_cfg* cfg_in, bool serial, const gru_params* p, const float* x, const float* h0, float* gi,
                  float* h, float* resnorm, void* ws, size_t ws_bytes, cudaStream_t s) {
   if (!cfg_in || !p || !x || !h0 || !gi || !h || !ws || !p->W_ih || !p->W_hh || !p->b_ih || !p->b_hh) return MGRIT_INVALID_ARG;
+  if (!aligned32(x, h0, gi, h, ws, p->W_ih, p->W_hh, p->b_ih, p->b_hh)) return MGRIT_INVALID_ARG;
   mgrit_gru_cfg c = *cfg_in;
   if (serial) { c.levels = 1; c.iters = 1; c.cf = 2; }
   Hier hr;
@@ -323,6 +332,8 @@ int adjoint_impl(const mgrit_gru_cfg* cfg_in, bool serial, const gru_params* p, 
   if (!cfg_in || !p || !x || !h0 || !gi || !h || !dh || !dh0 || !g || !ws) return MGRIT_INVALID_ARG;
   if (!dh_seed && !dhT) return MGRIT_INVALID_ARG;
   if (!p->W_ih || !p->W_hh || !p->b_ih || !p->b_hh || !g->dW_ih || !g->dW_hh || !g->db_ih || !g->db_hh) return MGRIT_INVALID_ARG;
+  if (!aligned32(x, h0, gi, h, dh_seed, dhT, dh, dh0, dx, ws, p->W_ih, p->W_hh, p->b_ih, p->b_hh, g->dW_ih, g->dW_hh, g->db_ih, g->db_hh))
+    return MGRIT_INVALID_ARG;
   mgrit_gru_cfg c = *cfg_in;
   if (serial) { c.levels = 1; c.iters = 1; c.cf = 2; }
   Hier hr;
@@ -426,6 +437,7 @@ int mgrit_gru_workspace_bytes(const mgrit_gru_cfg* cfg, size_t* fwd_bytes, size_
 int gru_input_projection(const mgrit_gru_cfg* cfg, const gru_params* p, const float* x, float* gi, void* ws, size_t ws_bytes,
                          mgrit_stream_t stream) {
   if (!cfg || !p || !x || !gi || !p->W_ih || !p->b_ih) return MGRIT_INVALID_ARG;
+  if (!aligned32(x, gi, ws, p->W_ih, p->b_ih)) return MGRIT_INVALID_ARG;
   Hier hr;
   int rc = check_cfg(cfg, &hr);
   if (rc) return rc;

@@ -200,3 +200,21 @@ def test_error_codes(B):
                                  small.data_ptr(), 256, None)
     assert rc == -1
     assert B.last_device_status() == 0
+
+
+def test_misaligned_pointer_is_rejected(B):
+    """Data pointers must be 32-byte aligned (the kernels move whole 32-byte sectors per thread)."""
+    import ctypes
+    w = WORKLOADS["tiny"]
+    d = make_inputs(w)
+    p, x, h0 = upload(d)
+    cfg = _cfg(B, w, 2)
+    nb = B.workspace_bytes(cfg)[0]
+    ws = torch.empty(nb, dtype=torch.uint8, device="cuda")
+    gi = torch.empty(w.T * w.B * 3 * w.H + 8, device="cuda")
+    h = torch.empty(w.T, w.B, w.H, device="cuda")
+    args = lambda gi_ptr: (ctypes.byref(cfg), ctypes.byref(B._params(p)), x.data_ptr(), h0.data_ptr(), gi_ptr, h.data_ptr(),
+                           None, ws.data_ptr(), nb, None)
+    assert B.lib.mgrit_gru_forward(*args(gi.data_ptr())) == 0
+    assert B.lib.mgrit_gru_forward(*args(gi.data_ptr() + 16)) == -1      # 16-byte aligned only
+    torch.cuda.synchronize()
