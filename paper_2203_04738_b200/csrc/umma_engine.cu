@@ -7,6 +7,7 @@
 #include "umma_engine.cuh"
 #include "umma_cell.cuh"
 #include "umma_gemm.cuh"
+#include "umma_gemm_pair.cuh"
 
 namespace mg {
 
@@ -74,6 +75,38 @@ bool launch_gemm(int kc, const bf16* A, i64 lda, const bf16* Bm, i64 ldb, int M,
   int grid = tiles < kSMs ? tiles : kSMs;
   prof_begin(kc, 2.0 * M * (GATES ? 3.0 * N : (double)N) * K, s);
   if (launch_pdl(kern, dim3(grid), dim3(kThreads), C::kSmemBytes, s, ta, tb, sh, epi, g_status_ptr) != cudaSuccess) return false;
+  prof_end(s);
+  count_launch();
+  return true;
+}
+
+// The same product on CTA pairs (256 x 256 tiles); K-major operands, N columns in tiles of 256.
+// Used when the product has more 128 x 256 tiles than SMs (below that every CTA has at most one tile and the
+// single-CTA kernel is as fast).  MGRIT_GRU_GEMM_PAIR=0 in the environment keeps every product on single CTAs.
+static bool gemm_pair_enabled(int M, int N) {
+  static int v = -1;
+  if (v < 0) { const char* e = getenv("MGRIT_GRU_GEMM_PAIR"); v = (e && e[0] == '0') ? 0 : 1; }
+  return v == 1 && (i64)((M + BM - 1) / BM) * ((N + 255) / 256) > kSMs;
+}
+template <class Epi>
+bool launch_gemm_pair(int kc, const bf16* A, i64 lda, const bf16* Bm, i64 ldb, int M, int N, int K, int b_rows, Epi epi, cudaStream_t s) {
+  if (M <= 0 || N <= 0) return true;
+  if (!ensure_driver()) return false;
+  static bool attr_set = false;
+  auto kern = umma_gemm_pair_kernel<Epi>;
+  if (!attr_set) {
+    if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, pairk::kSmemBytes) != cudaSuccess) return false;
+    attr_set = true;
+  }
+  CUtensorMap ta, tb;
+  if (!make_map(&ta, A, (uint64_t)K, (uint64_t)M, (uint64_t)lda, BM)) return false;
+  if (!make_map(&tb, Bm, (uint64_t)K, (uint64_t)b_rows, (uint64_t)ldb, pairk::BN / 2)) return false;
+  GemmShape sh{M, N, K, 0};
+  int tiles = ((M + 2 * BM - 1) / (2 * BM)) * ((N + pairk::BN - 1) / pairk::BN);
+  int grid = 2 * (tiles < kSMs / 2 ? tiles : kSMs / 2);
+  prof_begin(kc, 2.0 * M * (double)N * K, s);
+  if (launch_pdl_cluster(kern, 2, dim3(grid), dim3(kThreads), pairk::kSmemBytes, s, ta, tb, sh, epi, g_status_ptr) != cudaSuccess)
+    return false;
   prof_end(s);
   count_launch();
   return true;
@@ -549,7 +582,9 @@ int umma_prepare_fwd(const mgrit_gru_cfg* c, const gru_params* p, const float* x
   convert(p->W_ih, w->W_ih, (i64)3 * H * I, s);
   convert(x, w->xb, TB * I, s);
   // gi = x W_ih^T + b_ih :  M = T*B, N = 3H, K = I
-  if (!launch_gemm<256, false>(KC_PROJ, w->xb, I, w->W_ih, I, (int)TB, 3 * H, I, 0, 3 * H, EpiBias{gi, 3 * H, p->b_ih, (int)TB, 3 * H}, s))
+  if (gemm_pair_enabled((int)TB, 3 * H)
+          ? !launch_gemm_pair(KC_PROJ, w->xb, I, w->W_ih, I, (int)TB, 3 * H, I, 3 * H, EpiBias{gi, 3 * H, p->b_ih, (int)TB, 3 * H}, s)
+          : !launch_gemm<256, false>(KC_PROJ, w->xb, I, w->W_ih, I, (int)TB, 3 * H, I, 0, 3 * H, EpiBias{gi, 3 * H, p->b_ih, (int)TB, 3 * H}, s))
     return MGRIT_CUDA_ERROR;
   return MGRIT_OK;
 }
@@ -618,6 +653,8 @@ void umma_adj_step(const AdjStepArgs& a, UmmaAdjWs* w, cudaStream_t s) {
   const int tiles256 = ((a.M + BM - 1) / BM) * ((a.H + 255) / 256);
   if (tiles256 * 2 <= kSMs)
     launch_gemm<64, false>(KC_ADJ_STEP, w->Apack, 3 * a.H, w->W_hhT, 3 * a.H, a.M, a.H, 3 * a.H, 0, a.H, EpiAdj<64>{a}, s);
+  else if (gemm_pair_enabled(a.M, a.H))
+    launch_gemm_pair(KC_ADJ_STEP, w->Apack, 3 * a.H, w->W_hhT, 3 * a.H, a.M, a.H, 3 * a.H, a.H, EpiAdj<256>{a}, s);
   else
     launch_gemm<256, false>(KC_ADJ_STEP, w->Apack, 3 * a.H, w->W_hhT, 3 * a.H, a.M, a.H, 3 * a.H, 0, a.H, EpiAdj<256>{a}, s);
 }
@@ -642,7 +679,10 @@ int umma_gradients(const mgrit_gru_cfg* c, const gru_params* p, const float* x, 
   ok = ok && launch_gemm_mn(KC_WGRAD, dAh, 3 * H, 3 * H, w->hb0, H, H, (int)M, EpiStore{g->dW_hh, H, 3 * H, H}, s);
   ok = ok && launch_gemm_mn(KC_WGRAD, dAi, 3 * H, 3 * H, w->xb, I, I, (int)M, EpiStore{g->dW_ih, I, 3 * H, I}, s);
   // dx[T*B, I] = dA_i W_ih   (K = 3H, K-major operands)
-  if (dx) ok = ok && launch_gemm<256, false>(KC_WGRAD, dAi, 3 * H, w->W_ihT, 3 * H, (int)M, I, 3 * H, 0, I, EpiStore{dx, I, (int)M, I}, s);
+  if (dx)
+    ok = ok && (gemm_pair_enabled((int)M, I)
+                    ? launch_gemm_pair(KC_WGRAD, dAi, 3 * H, w->W_ihT, 3 * H, (int)M, I, 3 * H, I, EpiStore{dx, I, (int)M, I}, s)
+                    : launch_gemm<256, false>(KC_WGRAD, dAi, 3 * H, w->W_ihT, 3 * H, (int)M, I, 3 * H, 0, I, EpiStore{dx, I, (int)M, I}, s));
   return ok ? MGRIT_OK : MGRIT_CUDA_ERROR;
 }
 
