@@ -116,7 +116,8 @@ bool launch_gemm_pair(int kc, const bf16* A, i64 lda, const bf16* Bm, i64 ldb, i
 // (A: [K, Mdim], B: [K, Ndim], row-major), consumed as MN-major tensor-core operands -- the shape of the
 // weight-gradient reductions dW = dA^T h, which therefore need no transposed copies.
 template <class Epi>
-bool launch_gemm_mn(int kc, const bf16* A, i64 lda, int Mdim, const bf16* Bm, i64 ldb, int Ndim, int K, Epi epi, cudaStream_t s) {
+bool launch_gemm_mn(int kc, const bf16* A, i64 lda, int Mdim, const bf16* Bm, i64 ldb, int Ndim, int K, int splits, Epi epi,
+                    cudaStream_t s) {
   using C = Cfg<256, false>;
   if (Mdim <= 0 || Ndim <= 0) return true;
   if (!ensure_driver()) return false;
@@ -129,8 +130,10 @@ bool launch_gemm_mn(int kc, const bf16* A, i64 lda, int Mdim, const bf16* Bm, i6
   CUtensorMap ta, tb;
   if (!make_map(&ta, A, (uint64_t)Mdim, (uint64_t)K, (uint64_t)lda, 64)) return false;
   if (!make_map(&tb, Bm, (uint64_t)Ndim, (uint64_t)K, (uint64_t)ldb, 64)) return false;
-  GemmShape sh{Mdim, Ndim, K, 0};
-  int tiles = ((Mdim + BM - 1) / BM) * ((Ndim + 255) / 256);
+  const int k_blocks = (K + BK - 1) / BK;
+  if (splits < 1) splits = 1;
+  GemmShape sh{Mdim, Ndim, K, 0, splits, (k_blocks + splits - 1) / splits};
+  int tiles = ((Mdim + BM - 1) / BM) * ((Ndim + 255) / 256) * splits;
   int grid = tiles < kSMs ? tiles : kSMs;
   prof_begin(kc, 2.0 * Mdim * (double)Ndim * K, s);
   if (launch_pdl(kern, dim3(grid), dim3(kThreads), C::kSmemBytes, s, ta, tb, sh, epi, g_status_ptr) != cudaSuccess) return false;
@@ -237,6 +240,12 @@ struct EpiBias {  // out[m, n] = acc + bias[n]      (input projection)
 
 struct EpiStore {  // out[m, n] = acc            (weight / input gradients)
   float* out; i64 ld; int M, N;
+  i64 split_stride;   // split products: range `sp` of the reduction goes to out + sp*split_stride (summed afterwards)
+  __device__ void operator()(uint32_t taddr, int row, int n0, int half, int sp) const {
+    EpiStore e = *this;
+    e.out += (i64)sp * split_stride;
+    e(taddr, row, n0, half);
+  }
   __device__ void operator()(uint32_t taddr, int row, int n0, int half) const {
     const bool valid = row < M;
     float* o = out + (i64)row * ld + n0;
@@ -568,6 +577,7 @@ void umma_plan_adj(const mgrit_gru_cfg* c, const int* N, int L, char* base, size
   size_t apack = o->maxM * 3 * H;
   if (TB * H > apack) apack = TB * H;     // the linearisation packs all T*B rows of a level at once
   o->Apack = take<bf16>(base, off, apack);
+  o->apack_elems = apack;
   o->dAh = take<bf16>(base, off, 3 * H * TB);
   o->dAi = take<bf16>(base, off, 3 * H * TB);
   o->xb = take<bf16>(base, off, I * TB);
@@ -659,6 +669,45 @@ void umma_adj_step(const AdjStepArgs& a, UmmaAdjWs* w, cudaStream_t s) {
     launch_gemm<256, false>(KC_ADJ_STEP, w->Apack, 3 * a.H, w->W_hhT, 3 * a.H, a.M, a.H, 3 * a.H, 0, a.H, EpiAdj<256>{a}, s);
 }
 
+// dst[e] = sum over the `splits` partial products (float4 stream)
+__global__ void __launch_bounds__(kPT) sum_splits_kernel(const float4* __restrict__ part, i64 n4, int splits, float4* __restrict__ dst) {
+  for (i64 e = (i64)blockIdx.x * blockDim.x + threadIdx.x; e < n4; e += (i64)gridDim.x * blockDim.x) {
+    float4 a = part[e];
+    for (int sp = 1; sp < splits; ++sp) {
+      float4 b = part[(i64)sp * n4 + e];
+      a.x += b.x; a.y += b.y; a.z += b.z; a.w += b.w;
+    }
+    dst[e] = a;
+  }
+}
+
+// A weight-gradient product has few output tiles (3H/128 x cols/256) and a very long reduction (T*B): with fewer
+// tiles than SMs, or a ragged last wave, the reduction is cut into up to four ranges so that the (tile, range)
+// items fill the SMs; the partial products go to `scratch` (scratch_bytes available) and are summed afterwards.
+static int pick_splits(int Mdim, int Ndim, int K, size_t scratch_bytes) {
+  const int tiles = ((Mdim + BM - 1) / BM) * ((Ndim + 255) / 256), k_blocks = (K + BK - 1) / BK;
+  int best = 1; double best_eff = 0.0;
+  for (int sp = 1; sp <= 4; ++sp) {
+    if (sp > 1 && ((size_t)sp * Mdim * Ndim * sizeof(float) > scratch_bytes || k_blocks / sp < 32)) break;
+    const int items = tiles * sp, waves = (items + kSMs - 1) / kSMs;
+    const double eff = (double)items / ((double)waves * kSMs);
+    if (eff > best_eff + 0.05) { best_eff = eff; best = sp; }
+  }
+  return best;
+}
+
+template <class OutT>
+static bool wgrad_gemm(const bf16* dA, int H3, const bf16* R, int cols, int K, OutT* out, float* scratch, size_t scratch_bytes,
+                       cudaStream_t s) {
+  const int splits = (((i64)H3 * cols) % 4 == 0) ? pick_splits(H3, cols, K, scratch_bytes) : 1;
+  if (splits == 1) return launch_gemm_mn(KC_WGRAD, dA, H3, H3, R, cols, cols, K, 1, EpiStore{out, cols, H3, cols, 0}, s);
+  const i64 n = (i64)H3 * cols;
+  if (!launch_gemm_mn(KC_WGRAD, dA, H3, H3, R, cols, cols, K, splits, EpiStore{scratch, cols, H3, cols, n}, s)) return false;
+  sum_splits_kernel<<<pgrid(n / 4), kPT, 0, s>>>(reinterpret_cast<const float4*>(scratch), n / 4, splits, reinterpret_cast<float4*>(out));
+  count_launch();
+  return true;
+}
+
 int umma_gradients(const mgrit_gru_cfg* c, const gru_params* p, const float* x, const float* h0, const float* h, const float* lam,
                    const float* cr, const float* cz, const float* cn, const float* cnp, float* dx, const gru_grads* g,
                    UmmaAdjWs* w, cudaStream_t s) {
@@ -676,13 +725,16 @@ int umma_gradients(const mgrit_gru_cfg* c, const gru_params* p, const float* x, 
   convert(x, w->xb, M * I, s);                   // x as bf16 [M, I]; h_{t-1} as bf16 = [h_0; h] without its last slot (w->hb0)
   bool ok = true;
   // dW_hh[3H, H] = dA_h^T h_prev ;  dW_ih[3H, I] = dA_i^T x    (K = T*B, MN-major operands)
-  ok = ok && launch_gemm_mn(KC_WGRAD, dAh, 3 * H, 3 * H, w->hb0, H, H, (int)M, EpiStore{g->dW_hh, H, 3 * H, H}, s);
-  ok = ok && launch_gemm_mn(KC_WGRAD, dAi, 3 * H, 3 * H, w->xb, I, I, (int)M, EpiStore{g->dW_ih, I, 3 * H, I}, s);
+  // (the step operand buffer is free during the gradient pass: scratch for the split partial products)
+  float* scratch = reinterpret_cast<float*>(w->Apack);
+  const size_t scratch_bytes = w->apack_elems * sizeof(bf16);
+  ok = ok && wgrad_gemm(dAh, 3 * H, w->hb0, H, (int)M, g->dW_hh, scratch, scratch_bytes, s);
+  ok = ok && wgrad_gemm(dAi, 3 * H, w->xb, I, (int)M, g->dW_ih, scratch, scratch_bytes, s);
   // dx[T*B, I] = dA_i W_ih   (K = 3H, K-major operands)
   if (dx)
     ok = ok && (gemm_pair_enabled((int)M, I)
-                    ? launch_gemm_pair(KC_WGRAD, dAi, 3 * H, w->W_ihT, 3 * H, (int)M, I, 3 * H, I, EpiStore{dx, I, (int)M, I}, s)
-                    : launch_gemm<256, false>(KC_WGRAD, dAi, 3 * H, w->W_ihT, 3 * H, (int)M, I, 3 * H, 0, I, EpiStore{dx, I, (int)M, I}, s));
+                    ? launch_gemm_pair(KC_WGRAD, dAi, 3 * H, w->W_ihT, 3 * H, (int)M, I, 3 * H, I, EpiStore{dx, I, (int)M, I, 0}, s)
+                    : launch_gemm<256, false>(KC_WGRAD, dAi, 3 * H, w->W_ihT, 3 * H, (int)M, I, 3 * H, 0, I, EpiStore{dx, I, (int)M, I, 0}, s));
   return ok ? MGRIT_OK : MGRIT_CUDA_ERROR;
 }
 

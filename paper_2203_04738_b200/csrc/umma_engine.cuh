@@ -17,6 +17,7 @@ struct UmmaAdjWs {
   __nv_bfloat16* W_hhT;   // [H,3H]   (adjoint step: B operand, K = 3H contiguous)
   __nv_bfloat16* W_ihT;   // [I,3H]   (dx = dA_i W_ih)
   __nv_bfloat16* Apack;   // [maxM,3H]
+  size_t apack_elems;     // its size in elements
   __nv_bfloat16* dAh;     // [T*B,3H]  gradient-pass operand [cr|cz|cn]*lambda
   __nv_bfloat16* dAi;     // [T*B,3H]  gradient-pass operand [cr|cz|cn']*lambda
   __nv_bfloat16* xb;      // [T*B,I]   bf16 copy of the layer input

@@ -139,6 +139,8 @@ __device__ __forceinline__ void tmem_ld_wait() { asm volatile("tcgen05.wait::ld.
 struct GemmShape {
   int M, N, K;          // K a multiple of 8 (TMA stride rule); any M, N
   int gate_rows;        // GATES: row distance between the r, z, n blocks of B (= H); else 0
+  int splits;           // MN-major products only: the reduction is cut into `splits` ranges of kb_per_split k-blocks,
+  int kb_per_split;     // each (tile, range) is one work item and the epilogue is told which range it finishes
 };
 
 template <int BN, bool GATES>
@@ -178,8 +180,17 @@ umma_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int m_tiles = (sh.M + BM - 1) / BM;
   const int n_tiles = (sh.N + C::kNPerTile - 1) / C::kNPerTile;
-  const int tiles = m_tiles * n_tiles;
-  const int k_blocks = (sh.K + BK - 1) / BK;
+  const int k_blocks_all = (sh.K + BK - 1) / BK;
+  const int splits = MNMAJ ? sh.splits : 1;
+  const int mn_tiles = m_tiles * n_tiles;
+  const int tiles = mn_tiles * splits;                   // work items
+  // k-block range of item t (the whole reduction unless split)
+  auto kb_begin = [&](int t) { return MNMAJ ? (t / mn_tiles) * sh.kb_per_split : 0; };
+  auto kb_end = [&](int t) {
+    if (!MNMAJ) return k_blocks_all;
+    int e = (t / mn_tiles + 1) * sh.kb_per_split;
+    return e < k_blocks_all ? e : k_blocks_all;
+  };
 
   if (threadIdx.x == 0) {
     abort_flag = 0;
@@ -207,8 +218,8 @@ umma_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
       int stage = 0; uint32_t phase = 0;
       bool ok = true;
       for (int t = blockIdx.x; t < tiles && ok; t += gridDim.x) {
-        const int mt = t / n_tiles, nt = t % n_tiles;
-        for (int kb = 0; kb < k_blocks; ++kb) {
+        const int mt = (t % mn_tiles) / n_tiles, nt = t % n_tiles;
+        for (int kb = kb_begin(t), kbe = kb_end(t); kb < kbe; ++kb) {
           if (!mbar_wait(empty_bar(stage), phase ^ 1u, abortp, status, 1)) { ok = false; break; }
           const uint32_t a_dst = tiles_base + stage * C::kStageBytes;
           const uint32_t b_dst = a_dst + C::kABytes;
@@ -245,7 +256,8 @@ umma_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
         if (!mbar_wait(tempty_bar(as), aphase ^ 1u, abortp, status, 2)) { ok = false; break; }
         tc_fence_after();
         const uint32_t d_tmem = tmem_base + (uint32_t)(as * BN);
-        for (int kb = 0; kb < k_blocks; ++kb) {
+        const int kb0 = kb_begin(t);
+        for (int kb = kb0, kbe = kb_end(t); kb < kbe; ++kb) {
           if (!mbar_wait(full_bar(stage), phase, abortp, status, 3)) { ok = false; break; }
           tc_fence_after();
           const uint32_t a_src = tiles_base + stage * C::kStageBytes;
@@ -255,7 +267,7 @@ umma_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
           constexpr uint64_t kstep = MNMAJ ? (2048 >> 4) : (32 >> 4);
 #pragma unroll
           for (int k = 0; k < BK / 16; ++k)
-            mma_bf16(d_tmem, adesc + kstep * k, bdesc + kstep * k, idesc, (kb | k) != 0 ? 1u : 0u);
+            mma_bf16(d_tmem, adesc + kstep * k, bdesc + kstep * k, idesc, ((kb - kb0) | k) != 0 ? 1u : 0u);
           mma_commit(empty_bar(stage));   // frees the stage when the MMAs have read it
           if (++stage == C::kStages) { stage = 0; phase ^= 1u; }
         }
@@ -268,13 +280,14 @@ umma_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
     const int half = (warp - 2) >> 2;   // which half of the tile's columns this warp handles
     int it = 0;
     for (int t = blockIdx.x; t < tiles; t += gridDim.x, ++it) {
-      const int mt = t / n_tiles, nt = t % n_tiles;
+      const int mt = (t % mn_tiles) / n_tiles, nt = t % n_tiles;
       const int as = it & 1;
       const uint32_t aphase = (uint32_t)(it >> 1) & 1u;
       if (!mbar_wait(tfull_bar(as), aphase, abortp, status, 4)) break;
       tc_fence_after();
       const uint32_t taddr = tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(as * BN);
-      epi(taddr, mt * BM + q * 32 + lane, nt * C::kNPerTile, half);
+      if constexpr (MNMAJ) epi(taddr, mt * BM + q * 32 + lane, nt * C::kNPerTile, half, t / mn_tiles);
+      else epi(taddr, mt * BM + q * 32 + lane, nt * C::kNPerTile, half);
       tc_fence_before();
       mbar_arrive(tempty_bar(as));
     }
