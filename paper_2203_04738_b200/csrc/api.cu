@@ -102,7 +102,8 @@ struct FwdWs {
 };
 struct AdjWs {
   float* U[kMaxLevels]; float* G[kMaxLevels];
-  float *a[kMaxLevels], *cr[kMaxLevels], *cz[kMaxLevels], *cn[kMaxLevels], *cnp;
+  float *a[kMaxLevels], *cr[kMaxLevels], *cz[kMaxLevels], *cn[kMaxLevels], *cnp;   // gate coefficients: fp32 engine
+  __nv_bfloat16 *crb[kMaxLevels], *czb[kMaxLevels], *cnb[kMaxLevels], *cnpb;       // ... tensor-core engine (bf16)
   float *dA_h, *dA_i; double* res_acc; UmmaAdjWs um;
   __nv_bfloat16* chain_dAb; unsigned* chain_bar;
 };
@@ -130,11 +131,20 @@ void plan_adj(const mgrit_gru_cfg* c, const Hier& hr, Ws& w, AdjWs* o) {
     o->U[l] = w.take<float>((size_t)(hr.N[l] + 1) * BH);
     o->G[l] = w.take<float>((size_t)(hr.N[l] + 1) * BH);
     o->a[l] = w.take<float>((size_t)hr.N[l] * BH);
-    o->cr[l] = w.take<float>((size_t)hr.N[l] * BH);
-    o->cz[l] = w.take<float>((size_t)hr.N[l] * BH);
-    o->cn[l] = w.take<float>((size_t)hr.N[l] * BH);
+    if (c->operands == MGRIT_OPERANDS_BF16) {
+      o->cr[l] = o->cz[l] = o->cn[l] = nullptr;
+      o->crb[l] = w.take<__nv_bfloat16>((size_t)hr.N[l] * BH);
+      o->czb[l] = w.take<__nv_bfloat16>((size_t)hr.N[l] * BH);
+      o->cnb[l] = w.take<__nv_bfloat16>((size_t)hr.N[l] * BH);
+    } else {
+      o->crb[l] = o->czb[l] = o->cnb[l] = nullptr;
+      o->cr[l] = w.take<float>((size_t)hr.N[l] * BH);
+      o->cz[l] = w.take<float>((size_t)hr.N[l] * BH);
+      o->cn[l] = w.take<float>((size_t)hr.N[l] * BH);
+    }
   }
-  o->cnp = w.take<float>((size_t)hr.N[0] * BH);
+  if (c->operands == MGRIT_OPERANDS_BF16) { o->cnp = nullptr; o->cnpb = w.take<__nv_bfloat16>((size_t)hr.N[0] * BH); }
+  else { o->cnpb = nullptr; o->cnp = w.take<float>((size_t)hr.N[0] * BH); }
   o->res_acc = w.take<double>((size_t)(c->iters > 0 ? c->iters : 1));
   if (c->operands == MGRIT_OPERANDS_BF16) {
     o->dA_h = o->dA_i = nullptr;
@@ -244,7 +254,7 @@ struct AdjCycle : Cycle {
     a.B = c->B; a.H = c->H; a.nsteps = hr.N[l];
     a.mu = U[l]; a.dAb = w->chain_dAb;
     i64 row0 = (i64)(hr.N[l] - 1) * BH;        // step s = 1 applies forward step N_l, stored at row N_l - 1
-    a.a = w->a[l] + row0; a.cr = w->cr[l] + row0; a.cz = w->cz[l] + row0; a.cn = w->cn[l] + row0;
+    a.a = w->a[l] + row0; a.cr = w->crb[l] + row0; a.cz = w->czb[l] + row0; a.cn = w->cnb[l] + row0;
     a.coef_step = -(i64)BH;
     a.g = G[l]; a.WT = w->um.W_hhT; a.bar = w->chain_bar;
     return serial_adj_solve(a, s);
@@ -257,7 +267,14 @@ struct AdjCycle : Cycle {
     a.gadd = d.gadd ? d.gadd + (size_t)d.gadd_slot * BH : nullptr; a.gadd_ks = (i64)d.gadd_stride * BH;
     // the step arriving at reversed point s applies forward step j = N_l - s + 1, stored at row N_l - s
     i64 row0 = (i64)(hr.N[d.l] - d.tgt_slot) * BH;
-    a.a = w->a[d.l] + row0; a.cr = w->cr[d.l] + row0; a.cz = w->cz[d.l] + row0; a.cn = w->cn[d.l] + row0;
+    a.a = w->a[d.l] + row0;
+    if (c->operands == MGRIT_OPERANDS_BF16) {
+      a.cr = a.cz = a.cn = nullptr;
+      a.crb = w->crb[d.l] + row0; a.czb = w->czb[d.l] + row0; a.cnb = w->cnb[d.l] + row0;
+    } else {
+      a.crb = a.czb = a.cnb = nullptr;
+      a.cr = w->cr[d.l] + row0; a.cz = w->cz[d.l] + row0; a.cn = w->cn[d.l] + row0;
+    }
     a.coef_ks = -(i64)d.tgt_stride * BH;
     a.W_hh = p->W_hh; a.mode = d.mode;
     if (c->operands == MGRIT_OPERANDS_BF16) umma_adj_step(a, &w->um, s); else simt_adj_step(a, s);
@@ -357,6 +374,7 @@ int adjoint_impl(const mgrit_gru_cfg* cfg_in, bool serial, const gru_params* p, 
     a.M = hr.N[l] * c.B; a.B = c.B; a.H = c.H; a.h0 = h0; a.h = h; a.stride_t = hr.stride_t[l]; a.gi = gi;
     a.W_hh = p->W_hh; a.b_hh = p->b_hh; a.gamma = hr.gamma[l]; a.cell = c.cell;
     a.a = aw.a[l]; a.cr = aw.cr[l]; a.cz = aw.cz[l]; a.cn = aw.cn[l]; a.cnp = l == 0 ? aw.cnp : nullptr;
+    a.crb = aw.crb[l]; a.czb = aw.czb[l]; a.cnb = aw.cnb[l]; a.cnpb = l == 0 ? aw.cnpb : nullptr;
     if (bf16) umma_linearise(a, &aw.um, s); else simt_linearise(a, s);
   }
   // mu_0 = lambda_T; zero initial guess elsewhere; fine-level source = reversed dh_seed
@@ -386,7 +404,7 @@ int adjoint_impl(const mgrit_gru_cfg* cfg_in, bool serial, const gru_params* p, 
 
   // gradient pass g = w * dh/dTheta over all fine steps at once
   if (bf16) {
-    rc = umma_gradients(&c, p, x, h0, h, dh, aw.cr[0], aw.cz[0], aw.cn[0], aw.cnp, dx, g, &aw.um, s);
+    rc = umma_gradients(&c, p, x, h0, h, dh, aw.crb[0], aw.czb[0], aw.cnb[0], aw.cnpb, dx, g, &aw.um, s);
     if (rc) return rc;
   } else {
     i64 M = (i64)T * c.B;

@@ -81,6 +81,9 @@ struct LinArgs {
   const float* W_hh; const float* b_hh;
   float gamma; int cell;
   float *a, *cr, *cz, *cn, *cnp;    // cnp may be nullptr (only level 0 needs it)
+  // The tensor-core engine keeps the four gate coefficients in bf16 (they only ever enter bf16 operands;
+  // `a`, which multiplies the carried sensitivity in fp32, stays fp32): it writes these and ignores the fp32 ones.
+  __nv_bfloat16 *crb, *czb, *cnb, *cnpb;
 };
 
 // ---- one adjoint step for M = nk*B rows:  out = a*lam + [cr*lam | cz*lam | cn*lam] W_hh (+ gadd) ----
@@ -90,6 +93,7 @@ struct AdjStepArgs {
   float* lout;       i64 lout_ks;
   const float* gadd; i64 gadd_ks;   // optional source / FAS term, same shape as lout
   const float *a, *cr, *cz, *cn; i64 coef_ks;   // coefficient rows (+k*coef_ks + b*H), already offset to k = 0
+  const __nv_bfloat16 *crb, *czb, *cnb;         // the same rows in bf16 (tensor-core engine; same indexing)
   const float* W_hh;                // [3H,H] fp32
   int mode;                         // as FwdStepArgs
 };

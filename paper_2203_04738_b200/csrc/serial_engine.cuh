@@ -22,7 +22,8 @@ struct SerialAdjArgs {
   int B, H, nsteps;
   float* mu;                     // [nsteps+1][B][H], slot 0 given
   __nv_bfloat16* dAb;            // [2][B][3H] scratch
-  const float *a, *cr, *cz, *cn; // coefficient rows of step 1; step s at + (s-1)*coef_step
+  const float* a;                // coefficient rows of step 1; step s at + (s-1)*coef_step
+  const __nv_bfloat16 *cr, *cz, *cn;
   i64 coef_step;
   const float* g;                // [nsteps+1][B][H] or nullptr
   const __nv_bfloat16* WT;       // [H][3H] = W_hh^T

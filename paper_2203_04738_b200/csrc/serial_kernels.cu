@@ -239,11 +239,12 @@ __global__ void __launch_bounds__(kThreads, 1) serial_adj_kernel(SerialAdjArgs a
     int r = e / H, i = e % H;
     i64 off = (i64)(row0 + r) * H + i;
     float m = __ldcg(a.mu + off);
-    As[r * ldk + i] = __float2bfloat16(a.cr[off] * m);
-    As[r * ldk + H + i] = __float2bfloat16(a.cz[off] * m);
-    As[r * ldk + 2 * H + i] = __float2bfloat16(a.cn[off] * m);
+    As[r * ldk + i] = __float2bfloat16(__bfloat162float(a.cr[off]) * m);
+    As[r * ldk + H + i] = __float2bfloat16(__bfloat162float(a.cz[off]) * m);
+    As[r * ldk + 2 * H + i] = __float2bfloat16(__bfloat162float(a.cn[off]) * m);
   }
-  float mp[OPT], pa[OPT], pg[OPT], ncr[OPT], ncz[OPT], ncn[OPT];
+  float mp[OPT], pa[OPT], pg[OPT];
+  bf16 ncr[OPT], ncz[OPT], ncn[OPT];   // kept raw: converting at the load would wait for it before the barrier
 #pragma unroll
   for (int o = 0; o < OPT; ++o) {
     int idx = tid + o * kThreads, r = idx / UNC, i = idx % UNC;
@@ -253,9 +254,10 @@ __global__ void __launch_bounds__(kThreads, 1) serial_adj_kernel(SerialAdjArgs a
     pa[o] = v ? a.a[off] : 0.f;
     pg[o] = (v && a.g) ? a.g[BH + off] : 0.f;
     bool more = v && a.nsteps > 1;
-    ncr[o] = more ? a.cr[a.coef_step + off] : 0.f;
-    ncz[o] = more ? a.cz[a.coef_step + off] : 0.f;
-    ncn[o] = more ? a.cn[a.coef_step + off] : 0.f;
+    const bf16 zero = __float2bfloat16(0.f);
+    ncr[o] = more ? a.cr[a.coef_step + off] : zero;
+    ncz[o] = more ? a.cz[a.coef_step + off] : zero;
+    ncn[o] = more ? a.cn[a.coef_step + off] : zero;
   }
   __syncthreads();
 
@@ -278,9 +280,9 @@ __global__ void __launch_bounds__(kThreads, 1) serial_adj_kernel(SerialAdjArgs a
         a.mu[(i64)s * BH + off] = val;
         if (s < a.nsteps) {
           bf16* d = dAb + (i64)(row0 + r) * K + u0 + i;
-          d[0] = __float2bfloat16(ncr[o] * val);
-          d[H] = __float2bfloat16(ncz[o] * val);
-          d[2 * H] = __float2bfloat16(ncn[o] * val);
+          d[0] = __float2bfloat16(__bfloat162float(ncr[o]) * val);
+          d[H] = __float2bfloat16(__bfloat162float(ncz[o]) * val);
+          d[2 * H] = __float2bfloat16(__bfloat162float(ncn[o]) * val);
         }
       }
     }

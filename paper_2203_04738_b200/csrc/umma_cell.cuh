@@ -50,6 +50,15 @@ __device__ __forceinline__ void stg8(float* p, const float* v) {
                "f"(v[5]), "f"(v[6]), "f"(v[7])
                : "memory");
 }
+// eight values as bf16: one 16-byte store
+__device__ __forceinline__ void stg_bf8(__nv_bfloat16* p, const float* v) {
+  __nv_bfloat162 p0 = __floats2bfloat162_rn(v[0], v[1]), p1 = __floats2bfloat162_rn(v[2], v[3]);
+  __nv_bfloat162 p2 = __floats2bfloat162_rn(v[4], v[5]), p3 = __floats2bfloat162_rn(v[6], v[7]);
+  uint4 pk;
+  pk.x = *reinterpret_cast<uint32_t*>(&p0); pk.y = *reinterpret_cast<uint32_t*>(&p1);
+  pk.z = *reinterpret_cast<uint32_t*>(&p2); pk.w = *reinterpret_cast<uint32_t*>(&p3);
+  *reinterpret_cast<uint4*>(p) = pk;
+}
 __device__ __forceinline__ float4 lds4(uint32_t addr) {
   float4 v;
   asm volatile("ld.shared.v4.f32 {%0,%1,%2,%3}, [%4];" : "=f"(v.x), "=f"(v.y), "=f"(v.z), "=f"(v.w) : "r"(addr));
@@ -59,7 +68,8 @@ __device__ __forceinline__ float4 lds4(uint32_t addr) {
 struct CellArgs {
   int M, B, H, kt;                                    // kt = 128 / B
   float* hout; i64 hout_ks; __nv_bfloat16* hout_b;    // forward: fp32 rows (k, b) and their bf16 copy (or nullptr)
-  float *a, *cr, *cz, *cn, *cnp;                      // linearise: row-major [M, H] (cnp may be nullptr)
+  float* a;                                           // linearise: row-major [M, H]; a in fp32,
+  __nv_bfloat16 *cr, *cz, *cn, *cnp;                  // the gate coefficients in bf16 (cnp may be nullptr)
   const float* b_hh; float gamma; int cell; int mode;
 };
 
@@ -272,10 +282,10 @@ umma_cell_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
             }
             const i64 idx = (i64)row * H + u;
             stg8(p.a + idx, oa);
-            stg8(p.cr + idx, ocr);
-            stg8(p.cz + idx, ocz);
-            stg8(p.cn + idx, ocn);
-            if (p.cnp) stg8(p.cnp + idx, ocp);
+            stg_bf8(p.cr + idx, ocr);
+            stg_bf8(p.cz + idx, ocz);
+            stg_bf8(p.cn + idx, ocn);
+            if (p.cnp) stg_bf8(p.cnp + idx, ocp);
           }
         }
       }

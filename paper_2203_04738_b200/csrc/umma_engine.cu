@@ -196,6 +196,19 @@ bool launch_cell(int kc, const bf16* A, i64 a_ks, const float* gi, i64 gi_ks, co
 // Each epilogue warp handles 32 rows (its TMEM lane quarter) and one half of the tile's columns.
 // Per 16-column chunk the global loads are issued first, then the accumulator is read, so that the
 // memory latency of a chunk overlaps its tcgen05.ld and the other warps' work.
+__device__ __forceinline__ uint2 pack4(float4 v) {
+  __nv_bfloat162 lo = __floats2bfloat162_rn(v.x, v.y), hi = __floats2bfloat162_rn(v.z, v.w);
+  uint2 o;
+  o.x = *reinterpret_cast<uint32_t*>(&lo);
+  o.y = *reinterpret_cast<uint32_t*>(&hi);
+  return o;
+}
+__device__ __forceinline__ float4 unpack4(uint2 v) {
+  __nv_bfloat162 lo = *reinterpret_cast<__nv_bfloat162*>(&v.x), hi = *reinterpret_cast<__nv_bfloat162*>(&v.y);
+  float2 a = __bfloat1622float2(lo), b = __bfloat1622float2(hi);
+  return make_float4(a.x, a.y, b.x, b.y);
+}
+
 __device__ __forceinline__ float4 ld4(const float* p) { return *reinterpret_cast<const float4*>(p); }
 // 32-byte accesses: in these epilogues the lanes of a warp touch 32 different rows, so a 16-byte access uses half
 // of each 32-byte sector it moves; one 32-byte access per lane moves whole sectors.
@@ -350,10 +363,10 @@ struct EpiLin {  // adjoint coefficients of every step of a level
             oa[e] = L.a; ocr[e] = L.cr; ocz[e] = L.cz; ocn[e] = L.cn; ocp[e] = L.cnp;
           }
           st4(a.a + o + c, oa[0], oa[1], oa[2], oa[3]);
-          st4(a.cr + o + c, ocr[0], ocr[1], ocr[2], ocr[3]);
-          st4(a.cz + o + c, ocz[0], ocz[1], ocz[2], ocz[3]);
-          st4(a.cn + o + c, ocn[0], ocn[1], ocn[2], ocn[3]);
-          if (a.cnp) st4(a.cnp + o + c, ocp[0], ocp[1], ocp[2], ocp[3]);
+          *reinterpret_cast<uint2*>(a.crb + o + c) = pack4(make_float4(ocr[0], ocr[1], ocr[2], ocr[3]));
+          *reinterpret_cast<uint2*>(a.czb + o + c) = pack4(make_float4(ocz[0], ocz[1], ocz[2], ocz[3]));
+          *reinterpret_cast<uint2*>(a.cnb + o + c) = pack4(make_float4(ocn[0], ocn[1], ocn[2], ocn[3]));
+          if (a.cnpb) *reinterpret_cast<uint2*>(a.cnpb + o + c) = pack4(make_float4(ocp[0], ocp[1], ocp[2], ocp[3]));
         }
       }
     }
@@ -419,13 +432,6 @@ inline int pgrid(i64 items) {
   i64 b = (items + kPT - 1) / kPT, cap = (i64)kSMs * 8;
   return (int)(b < 1 ? 1 : (b > cap ? cap : b));
 }
-__device__ __forceinline__ uint2 pack4(float4 v) {
-  __nv_bfloat162 lo = __floats2bfloat162_rn(v.x, v.y), hi = __floats2bfloat162_rn(v.z, v.w);
-  uint2 o;
-  o.x = *reinterpret_cast<uint32_t*>(&lo);
-  o.y = *reinterpret_cast<uint32_t*>(&hi);
-  return o;
-}
 
 __global__ void __launch_bounds__(kPT) convert_kernel(const float4* __restrict__ src, uint2* __restrict__ dst, i64 n4) {
   for (i64 e = (i64)blockIdx.x * blockDim.x + threadIdx.x; e < n4; e += (i64)gridDim.x * blockDim.x) dst[e] = pack4(src[e]);
@@ -445,8 +451,8 @@ __global__ void __launch_bounds__(kPT) pack_rows_kernel(const float* __restrict_
 }
 
 // dst[m, g*H + i] = bf16(c_g[m, i] * lam[m, i])
-__global__ void __launch_bounds__(kPT) pack_adj_kernel(const float* __restrict__ lin, i64 lin_ks, const float* __restrict__ cr,
-                                                       const float* __restrict__ cz, const float* __restrict__ cn, i64 coef_ks,
+__global__ void __launch_bounds__(kPT) pack_adj_kernel(const float* __restrict__ lin, i64 lin_ks, const bf16* __restrict__ cr,
+                                                       const bf16* __restrict__ cz, const bf16* __restrict__ cn, i64 coef_ks,
                                                        int B, int H4, i64 M, uint2* __restrict__ dst) {
   pdl_wait();
   pdl_trigger();
@@ -456,9 +462,9 @@ __global__ void __launch_bounds__(kPT) pack_adj_kernel(const float* __restrict__
     i64 k = m / B; int b = (int)(m % B);
     i64 ro = ((i64)b * H4 + c) * 4;
     float4 l = *reinterpret_cast<const float4*>(lin + k * lin_ks + ro);
-    float4 r = *reinterpret_cast<const float4*>(cr + k * coef_ks + ro);
-    float4 z = *reinterpret_cast<const float4*>(cz + k * coef_ks + ro);
-    float4 n = *reinterpret_cast<const float4*>(cn + k * coef_ks + ro);
+    float4 r = unpack4(*reinterpret_cast<const uint2*>(cr + k * coef_ks + ro));
+    float4 z = unpack4(*reinterpret_cast<const uint2*>(cz + k * coef_ks + ro));
+    float4 n = unpack4(*reinterpret_cast<const uint2*>(cn + k * coef_ks + ro));
     i64 o = m * 3 * H4 + c;
     dst[o] = pack4(make_float4(r.x * l.x, r.y * l.y, r.z * l.z, r.w * l.w));
     dst[o + H4] = pack4(make_float4(z.x * l.x, z.y * l.y, z.z * l.z, z.w * l.w));
@@ -480,9 +486,9 @@ __global__ void __launch_bounds__(1024) transpose_kernel(const float* __restrict
 
 // Gradient-pass operands, row-major: dA_h = [cr|cz|cn]*lam and dA_i = [cr|cz|cnp]*lam as bf16 [M, 3H], plus the
 // fp32 column sums (bias gradients) added into db_hh / db_ih.  Block = 32 float4 columns (128 units) x 8 rows.
-__global__ void __launch_bounds__(256) form_dA_rows_kernel(const float* __restrict__ lam, const float* __restrict__ cr,
-                                                           const float* __restrict__ cz, const float* __restrict__ cn,
-                                                           const float* __restrict__ cnp, i64 M, int H, uint2* __restrict__ dAh,
+__global__ void __launch_bounds__(256) form_dA_rows_kernel(const float* __restrict__ lam, const bf16* __restrict__ cr,
+                                                           const bf16* __restrict__ cz, const bf16* __restrict__ cn,
+                                                           const bf16* __restrict__ cnp, i64 M, int H, uint2* __restrict__ dAh,
                                                            uint2* __restrict__ dAi, float* __restrict__ db_hh,
                                                            float* __restrict__ db_ih, int rows_per_block) {
   __shared__ float red[4][8][128];
@@ -496,8 +502,8 @@ __global__ void __launch_bounds__(256) form_dA_rows_kernel(const float* __restri
     for (i64 m = m0 + ty; m < m0 + rows_per_block && m < M; m += 8) {
       i64 e = m * H4 + c4;
       float4 l = reinterpret_cast<const float4*>(lam)[e];
-      float4 r = reinterpret_cast<const float4*>(cr)[e], z = reinterpret_cast<const float4*>(cz)[e];
-      float4 n = reinterpret_cast<const float4*>(cn)[e], q = reinterpret_cast<const float4*>(cnp)[e];
+      float4 r = unpack4(reinterpret_cast<const uint2*>(cr)[e]), z = unpack4(reinterpret_cast<const uint2*>(cz)[e]);
+      float4 n = unpack4(reinterpret_cast<const uint2*>(cn)[e]), q = unpack4(reinterpret_cast<const uint2*>(cnp)[e]);
       float4 v[4] = {make_float4(r.x * l.x, r.y * l.y, r.z * l.z, r.w * l.w), make_float4(z.x * l.x, z.y * l.y, z.z * l.z, z.w * l.w),
                      make_float4(n.x * l.x, n.y * l.y, n.z * l.z, n.w * l.w), make_float4(q.x * l.x, q.y * l.y, q.z * l.z, q.w * l.w)};
       i64 o = m * 3 * H4 + c4;
@@ -635,10 +641,10 @@ void umma_linearise(const LinArgs& a, UmmaAdjWs* w, cudaStream_t s) {
     ca.B = a.B; ca.H = a.H; ca.b_hh = a.b_hh; ca.gamma = a.gamma; ca.cell = a.cell;
     const float* gi0 = a.gi + (a.stride_t - 1) * BH * 3;
     // step 1 starts from h_0 (its own array); steps 2..N from h[stride*(j-1) - 1]
-    ca.a = a.a; ca.cr = a.cr; ca.cz = a.cz; ca.cn = a.cn; ca.cnp = a.cnp;
+    ca.a = a.a; ca.cr = a.crb; ca.cz = a.czb; ca.cn = a.cnb; ca.cnp = a.cnpb;
     launch_cell<true, false>(KC_LINEARISE, w->hb0, 0, gi0, 0, a.h0, 0, nullptr, 0, 1, w->W_hh, ca, s);
     if (N > 1) {
-      ca.a = a.a + BH; ca.cr = a.cr + BH; ca.cz = a.cz + BH; ca.cn = a.cn + BH; ca.cnp = a.cnp ? a.cnp + BH : nullptr;
+      ca.a = a.a + BH; ca.cr = a.crb + BH; ca.cz = a.czb + BH; ca.cn = a.cnb + BH; ca.cnp = a.cnpb ? a.cnpb + BH : nullptr;
       launch_cell<true, false>(KC_LINEARISE, w->hb + (a.stride_t - 1) * BH, a.stride_t * BH, gi0 + a.stride_t * BH * 3, a.stride_t * BH * 3,
                                a.h + (a.stride_t - 1) * BH, a.stride_t * BH, nullptr, 0, N - 1, w->W_hh, ca, s);
     }
@@ -655,7 +661,7 @@ void umma_linearise(const LinArgs& a, UmmaAdjWs* w, cudaStream_t s) {
 }
 
 void umma_adj_step(const AdjStepArgs& a, UmmaAdjWs* w, cudaStream_t s) {
-  launch_pdl(pack_adj_kernel, dim3(pgrid((i64)a.M * (a.H / 4))), dim3(kPT), 0, s, a.lin, a.lin_ks, a.cr, a.cz, a.cn, a.coef_ks, a.B,
+  launch_pdl(pack_adj_kernel, dim3(pgrid((i64)a.M * (a.H / 4))), dim3(kPT), 0, s, a.lin, a.lin_ks, a.crb, a.czb, a.cnb, a.coef_ks, a.B,
              a.H / 4, (i64)a.M, reinterpret_cast<uint2*>(w->Apack));
   count_launch();
   // Few-row launches (coarse levels, short prefixes) cannot fill the SMs with 256-column tiles and are
@@ -709,7 +715,7 @@ static bool wgrad_gemm(const bf16* dA, int H3, const bf16* R, int cols, int K, O
 }
 
 int umma_gradients(const mgrit_gru_cfg* c, const gru_params* p, const float* x, const float* h0, const float* h, const float* lam,
-                   const float* cr, const float* cz, const float* cn, const float* cnp, float* dx, const gru_grads* g,
+                   const bf16* cr, const bf16* cz, const bf16* cn, const bf16* cnp, float* dx, const gru_grads* g,
                    UmmaAdjWs* w, cudaStream_t s) {
   const int H = c->H, I = c->I, B = c->B;
   const i64 M = (i64)c->T * B;

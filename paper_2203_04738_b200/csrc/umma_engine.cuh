@@ -36,7 +36,8 @@ void umma_fwd_step(const FwdStepArgs& a, UmmaFwdWs* w, cudaStream_t s);
 void umma_linearise(const LinArgs& a, UmmaAdjWs* w, cudaStream_t s);
 void umma_adj_step(const AdjStepArgs& a, UmmaAdjWs* w, cudaStream_t s);
 int umma_gradients(const mgrit_gru_cfg* c, const gru_params* p, const float* x, const float* h0, const float* h,
-                   const float* lam, const float* cr, const float* cz, const float* cn, const float* cnp, float* dx,
+                   const float* lam, const __nv_bfloat16* cr, const __nv_bfloat16* cz, const __nv_bfloat16* cn,
+                   const __nv_bfloat16* cnp, float* dx,
                    const gru_grads* g, UmmaAdjWs* w, cudaStream_t s);
 int umma_device_status();
 
