@@ -68,7 +68,8 @@ def test_tiny_forward_two_level(B, iters, relax_fine):
         assert max_abs(h.cpu().numpy(), O.serial_forward(*P, xr, h0r)) < TOL_H
 
 
-@pytest.mark.parametrize("levels,cf,T,rf,rc", [(3, 4, 64, 0, 1), (3, 2, 64, 1, 1), (4, 2, 48, 0, 0), (2, 8, 64, 0, 1), (3, 4, 80, 1, 0)])
+@pytest.mark.parametrize("levels,cf,T,rf,rc", [(3, 4, 64, 0, 1), (3, 2, 64, 1, 1), (4, 2, 48, 0, 0), (2, 8, 64, 0, 1), (3, 4, 80, 1, 0),
+                                                 (3, 4, 16, 0, 1), (4, 2, 8, 1, 1)])   # the last two: one-point coarsest level
 def test_tiny_forward_multilevel_and_ragged(B, levels, cf, T, rf, rc):
     w = WORKLOADS["tiny"]
     d = make_inputs(w, T=T, B=3)

@@ -229,3 +229,32 @@ def test_finite_cycle_iterates_match_the_stored_fixture():
         assert int(w_[0]) == g_[0] and int(w_[1]) == g_[1]
         assert abs(float(w_[2]) - g_[2]) <= 1e-9 * float(w_[2])
         assert abs(float(w_[3]) - g_[3]) <= 1e-9 * float(w_[3])
+
+
+@pytest.mark.parametrize("rf,rc", [(O.RELAX_F, O.RELAX_F), (O.RELAX_F, O.RELAX_FCF), (O.RELAX_FCF, O.RELAX_FCF)])
+def test_extra_level_with_a_single_point_changes_nothing(rf, rc):
+    # A level whose coarse grid has ONE point is solved exactly by one cycle: F-relaxation propagates exactly from
+    # the fixed end through the only interval, and the FAS coarse equation U_1 = Phi(U_0) + (v - Phi(U_0)) returns
+    # v, the exact C-point value.  So a hierarchy L+1 deep whose last level has one point must reproduce the
+    # hierarchy L deep (whose last level is then swept serially) to rounding, forward and adjoint, at any cycle
+    # count: this pins the recursion -- FAS right-hand side of an intermediate level, coarse initial guess,
+    # correction, level strides of inputs and coefficients -- to the two- and three-level results pinned above.
+    for cf, deep, T in ((4, 3, 16), (2, 4, 8), (2, 5, 16)):      # level sizes 16/4/1, 8/4/2/1, 16/8/4/2/1
+        assert O.level_sizes(T, cf, deep)[-1] == 1
+        w = tiny_workload(T=T, B=2, I=3, H=5)
+        P, x, h0, _ = f64_inputs(w)
+        hs = O.serial_forward(*P, x, h0)
+        for iters in (1, 2):
+            ha, ra = O.mgrit_forward(*P, x, h0, cf=cf, levels=deep, iters=iters, relax_fine=rf, relax_coarse=rc)
+            hb, rb = O.mgrit_forward(*P, x, h0, cf=cf, levels=deep - 1, iters=iters, relax_fine=rf, relax_coarse=rc)
+            assert np.max(np.abs(ha - hb)) < 1e-13
+            assert np.max(np.abs(np.array(ra) - np.array(rb))) < 1e-13
+            if iters == 1:
+                assert np.max(np.abs(ha - hs)) > 1e-6      # not vacuous: one cycle is not converged
+        rng = np.random.default_rng(4)
+        seed = rng.standard_normal(hs.shape)
+        la, l0a, ga, _ = O.mgrit_adjoint(*P, x, h0, hs, seed, cf=cf, levels=deep, iters=2, relax_fine=rf, relax_coarse=rc)
+        lb, l0b, gb, _ = O.mgrit_adjoint(*P, x, h0, hs, seed, cf=cf, levels=deep - 1, iters=2, relax_fine=rf, relax_coarse=rc)
+        assert np.max(np.abs(la - lb)) < 1e-12 and np.max(np.abs(l0a - l0b)) < 1e-12
+        for k in ga:
+            assert np.max(np.abs(ga[k] - gb[k])) < 1e-11, k
