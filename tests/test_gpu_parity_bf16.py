@@ -87,6 +87,12 @@ def test_small_single_level_and_tiny_batch(B):
                            operands=2, classes=8, relu=False, seed=9))
 
 
+def test_small_four_level_one_point_coarsest(B):
+    # level sizes 64/16/4/1: the persistent chain of the coarsest level has a single step
+    _full_case(B, Workload("s4", T=64, B=8, I=64, H=128, cf=4, levels=4, iters_fwd=2, iters_adj=2, relax_fine=0, relax_coarse=1,
+                           operands=2, classes=8, relu=True, seed=10))
+
+
 def test_medium_full(B):
     # third configuration, everything compared: I=1024 H=512 B=32 T=1024, cf=4, 3 levels, 2 + 2 cycles
     _full_case(B, WORKLOADS["medium"])
