@@ -5,7 +5,7 @@
 // Protocol (every wait bounded as in the single-CTA kernel):
 //  * both CTAs' TMA loads complete on the LEADER's (rank 0) full barrier, which expects the bytes of both;
 //  * the leader's MMA thread issues for the pair and commits each stage to both CTAs' empty barriers and each
-//    accumulator to both CTAs' tfull barriers (one commit per destination; no multicast loads anywhere);
+//    accumulator to both CTAs' tfull barriers (one commit per destination; every TMA load has a single destination CTA);
 //  * both CTAs' epilogue warps arrive on the leader's tempty barrier (remote arrive for rank 1);
 //  * tensor memory is allocated and freed by the same warp of both CTAs, behind cluster barriers.
 #pragma once
