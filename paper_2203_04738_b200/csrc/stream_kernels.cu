@@ -40,6 +40,8 @@ __global__ void __launch_bounds__(kThreads) restrict_residual_kernel(const float
                                                                      const float4* __restrict__ v,
                                                                      float4* __restrict__ uc, uint2* __restrict__ ucb,
                                                                      int nc, i64 row4, double* acc) {
+  pdl_wait();      // launched with programmatic stream serialisation: nothing is read before the predecessor is done
+  pdl_trigger();
   i64 total = (i64)nc * row4;
   float s = 0.f;
   for (i64 e = (i64)blockIdx.x * blockDim.x + threadIdx.x; e < total; e += (i64)gridDim.x * blockDim.x) {
@@ -65,6 +67,8 @@ __global__ void __launch_bounds__(kThreads) restrict_residual_kernel(const float
 // Correction h'' = h' + P(h_c* - h'_c): only C-points are read afterwards, so u_{cf k} <- U_k.
 __global__ void __launch_bounds__(kThreads) correct_kernel(float4* __restrict__ uf, uint2* __restrict__ ufb, int cf,
                                                            const float4* __restrict__ uc, int nc, i64 row4) {
+  pdl_wait();
+  pdl_trigger();
   i64 total = (i64)nc * row4;
   for (i64 e = (i64)blockIdx.x * blockDim.x + threadIdx.x; e < total; e += (i64)gridDim.x * blockDim.x) {
     i64 k = e / row4 + 1, c = e % row4;
@@ -230,16 +234,15 @@ void stream_adam(float* p, const float* g, float* m, float* v, size_t n, float l
 void stream_restrict_residual(const float* uf, int cf, const float* v, float* uc, __nv_bfloat16* ucb, int nc, i64 rowlen, double* acc,
                               cudaStream_t s) {
   i64 row4 = rowlen / 4;
-  restrict_residual_kernel<<<stream_grid((i64)nc * row4), kThreads, 0, s>>>(
-      reinterpret_cast<const float4*>(uf), cf, reinterpret_cast<const float4*>(v), reinterpret_cast<float4*>(uc),
-      reinterpret_cast<uint2*>(ucb), nc, row4, acc);
+  launch_pdl(restrict_residual_kernel, dim3(stream_grid((i64)nc * row4)), dim3(kThreads), 0, s, reinterpret_cast<const float4*>(uf), cf,
+             reinterpret_cast<const float4*>(v), reinterpret_cast<float4*>(uc), reinterpret_cast<uint2*>(ucb), nc, row4, acc);
   count_launch();
 }
 
 void stream_correct(float* uf, __nv_bfloat16* ufb, int cf, const float* uc, int nc, i64 rowlen, cudaStream_t s) {
   i64 row4 = rowlen / 4;
-  correct_kernel<<<stream_grid((i64)nc * row4), kThreads, 0, s>>>(reinterpret_cast<float4*>(uf), reinterpret_cast<uint2*>(ufb), cf,
-                                                                  reinterpret_cast<const float4*>(uc), nc, row4);
+  launch_pdl(correct_kernel, dim3(stream_grid((i64)nc * row4)), dim3(kThreads), 0, s, reinterpret_cast<float4*>(uf),
+             reinterpret_cast<uint2*>(ufb), cf, reinterpret_cast<const float4*>(uc), nc, row4);
   count_launch();
 }
 
