@@ -157,6 +157,7 @@ def main():
     ap.add_argument("--serial", action="store_true", help="time the GPU serial sweep + exact BPTT instead of MGRIT")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
+    ap.add_argument("--no-graph", action="store_true", help="launch every kernel from the host instead of replaying a CUDA graph")
     ap.add_argument("--no-kernel-timing", action="store_true", help="skip the per-kernel CUDA-event pass")
     args = ap.parse_args()
 
@@ -188,7 +189,7 @@ def main():
     import torch.distributed as dist
     from paper_2203_04738_b200 import binding as B
     from paper_2203_04738_b200.replicas import job_throughput, max_over_ranks
-    from paper_2203_04738_b200.train_step import HostInputPipeline, alloc_buffers, training_step
+    from paper_2203_04738_b200.train_step import GraphedTrainingStep, HostInputPipeline, alloc_buffers, training_step
 
     torch.cuda.set_device(local_rank)
     dev = torch.device("cuda", local_rank)
@@ -205,8 +206,19 @@ def main():
     buf = alloc_buffers(w, T, w.B, dev, serial=args.serial, flags=B.FLAG_SKIP_DUPLICATE_FRELAX)
     loss_host = torch.empty(1).pin_memory()
 
-    def step():
+    def eager_step():
         return training_step(w, layers, W_c, b_c, x, h0, labels, buf)
+
+    # The step is captured once into a CUDA graph and replayed (same kernels, same order, same buffers).
+    graphed = None
+    if not args.no_graph:
+        try:
+            graphed = GraphedTrainingStep(w, layers, W_c, b_c, x, h0, labels, buf)
+        except Exception as e:      # capture unavailable here: launch from the host
+            sys.stderr.write(f"bench: CUDA graph capture failed ({e!r}); launching from the host\n")
+            graphed = None
+    step = graphed if graphed is not None else eager_step
+    config["launch"] = "one CUDA graph replay per step" if graphed is not None else "host launches"
 
     def barrier():
         torch.cuda.synchronize()
@@ -232,7 +244,7 @@ def main():
     barrier()
     wall1 = datetime.datetime.now()
     ms = e0.elapsed_time(e1)
-    launches = B.kernel_launches() - l0
+    launches = graphed.launches * args.steps if graphed is not None else B.kernel_launches() - l0
     clocks = sampler.stop(wall0, wall1) if sampler else None
     ms = max_over_ranks(ms, dev)
     ms_step = ms / args.steps
@@ -244,6 +256,12 @@ def main():
         # Every step's input is copied from pinned host memory inside the timed region; the copy of step k+1
         # runs on a side stream while step k computes (two device buffers), and the loss is read back every step.
         pipe = HostInputPipeline(x.shape, x.dtype, dev)
+        e2e_graphs = None
+        if graphed is not None:     # one captured step per input buffer of the pipeline
+            try:
+                e2e_graphs = [GraphedTrainingStep(w, layers, W_c, b_c, xb_, h0, labels, buf) for xb_ in pipe.bufs]
+            except Exception as e:
+                sys.stderr.write(f"bench: CUDA graph capture failed ({e!r}); launching from the host\n")
         barrier()
         e0.record()
         pipe.submit(x_host)
@@ -251,7 +269,7 @@ def main():
             xk = pipe.acquire()
             if k + 1 < args.steps:
                 pipe.submit(x_host)
-            loss = training_step(w, layers, W_c, b_c, xk, h0, labels, buf)
+            loss = e2e_graphs[k % 2]() if e2e_graphs else training_step(w, layers, W_c, b_c, xk, h0, labels, buf)
             pipe.release()
             loss_host.copy_(loss, non_blocking=True)
             torch.cuda.current_stream().synchronize()
@@ -271,7 +289,7 @@ def main():
         nprof = 2
         B.profile_enable(True)
         for _ in range(nprof):
-            step()
+            eager_step()
         prof = B.profile_read()
         by_size = {}
         for name, tms_, fl_ in B.profile_records():

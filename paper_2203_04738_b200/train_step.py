@@ -142,3 +142,31 @@ def training_step(w: Workload, layers, W_c, b_c, x, h0, labels, buf: StepBuffers
         B.sgd_update(W_c, dWc, lr)
         B.sgd_update(b_c, dbc, lr)
     return loss
+
+
+class GraphedTrainingStep:
+    """One training step captured once into a CUDA graph and replayed: the step is a fixed sequence of a few hundred
+    dependent launches (cooperative chain launches and programmatic dependent launches included), so replaying it
+    removes the per-launch CPU work and shortens the gaps between launches.  All pointers are baked in: the
+    tensors passed here must stay alive and keep their addresses; new data is copied INTO them.  ``launches`` is
+    the number of library kernels one replay runs."""
+
+    def __init__(self, w: Workload, layers, W_c, b_c, x, h0, labels, buf: StepBuffers, **kw):
+        args = (w, layers, W_c, b_c, x, h0, labels, buf)
+        side = torch.cuda.Stream()
+        side.wait_stream(torch.cuda.current_stream())
+        with torch.cuda.stream(side):               # first use of every kernel outside the capture (attribute set-up)
+            training_step(*args, **kw)
+        torch.cuda.current_stream().wait_stream(side)
+        torch.cuda.synchronize()
+        n0 = B.kernel_launches()
+        self.graph = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(self.graph):
+            self.loss = training_step(*args, **kw)
+        self.launches = B.kernel_launches() - n0
+        self._keep = args
+
+    def __call__(self):
+        self.graph.replay()
+        return self.loss
+

@@ -146,3 +146,29 @@ def test_host_input_pipeline_feeds_the_right_inputs():
     # the loss is a sum over batch rows accumulated with atomics, so equal inputs agree to rounding, not bitwise
     assert np.max(np.abs(np.array(got) - np.array(want))) < 1e-5
     assert min(abs(want[0] - want[1]), abs(want[1] - want[2]), abs(want[0] - want[2])) > 5e-5
+
+
+def test_graph_replay_equals_host_launches():
+    """The captured step replays the same kernels on the same buffers: with the update switched off two replays and
+    a host-launched step give the same loss (to the rounding of the loss's atomic batch sum) and the same gradients."""
+    from paper_2203_04738_b200.train_step import GraphedTrainingStep, alloc_buffers, training_step
+    w = Workload("gr", T=64, B=8, I=128, H=128, cf=4, levels=3, iters_fwd=2, iters_adj=2, relax_fine=0, relax_coarse=1,
+                 operands=2, classes=8, relu=True, seed=21)
+    d = make_inputs(w)
+    layers = [{n: to_dev(d["layers"][0][n]) for n in NAMES}]
+    W_c, b_c, h0, labels, x = to_dev(d["W_c"]), to_dev(d["b_c"]), to_dev(d["h0"]), to_dev(d["labels"]), to_dev(d["x"])
+    buf = alloc_buffers(w, w.T, w.B, torch.device("cuda"))
+    want = float(training_step(w, layers, W_c, b_c, x, h0, labels, buf, update=False))
+    g_want = buf.adj[0].dW_hh.clone()
+    g = GraphedTrainingStep(w, layers, W_c, b_c, x, h0, labels, buf, update=False)
+    assert g.launches > 50
+    for _ in range(2):
+        buf.adj[0].dW_hh.zero_()
+        got = float(g())
+        assert abs(got - want) < 1e-5
+        assert torch.equal(buf.adj[0].dW_hh, g_want)
+    # new data goes INTO the captured input tensor
+    x.mul_(0.5)
+    got = float(g())
+    ref = float(training_step(w, layers, W_c, b_c, x, h0, labels, buf, update=False))
+    assert abs(got - ref) < 1e-5 and abs(got - want) > 1e-4
