@@ -60,7 +60,9 @@ typedef struct {
   int32_t relax_fine;   /* relaxation on level 0: MGRIT_RELAX_F or MGRIT_RELAX_FCF (Eq. "fcf-relax") */
   int32_t relax_coarse; /* relaxation on levels 1 .. levels-2 */
   int32_t operands;     /* MGRIT_OPERANDS_FP32: FFMA everywhere; MGRIT_OPERANDS_BF16: bf16 tensor-core
-                           operands with fp32 accumulation; states, gates and gradients stay fp32 */
+                           operands with fp32 accumulation; states, gates and gradients stay fp32 (the
+                           adjoint's gate coefficients, which only ever enter such operands, are kept
+                           in bf16 inside the workspace) */
   int32_t flags;        /* MGRIT_FLAG_SKIP_DUPLICATE_FRELAX: a cycle after the first starts from C-points
                            whose F-points the previous cycle's final F-relaxation already filled; skip
                            re-doing it (results are identical) */
