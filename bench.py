@@ -167,11 +167,15 @@ def main():
     world = int(os.environ.get("WORLD_SIZE", "1"))
     local_rank = int(os.environ.get("LOCAL_RANK", "0"))
     T = args.T or w.T
+    # bytes one step streams: x, gi and the states of every layer (fp32)
+    stream_mb = 4.0 * T * w.B * (w.I + w.layers * 4 * w.H) / 1e6
+    l2_note = (f"inputs larger than L2 (x, gi and states, {stream_mb:.0f} MB, are re-streamed from HBM every step)" if stream_mb > 126.0
+               else f"working set {stream_mb:.1f} MB fits the 126 MB L2 and no flush is done: an L2-resident side case, not the headline configuration")
     config = {"workload": f"{w.name}: {w.layers}-layer GRU I={w.I} H={w.H} B={w.B} T={T}, cf={w.cf}, levels={w.levels}, "
                           f"iters fwd/adj={w.iters_fwd}/{w.iters_adj}, relax fine/coarse={'FCF' if w.relax_fine else 'F'}/"
                           f"{'FCF' if w.relax_coarse else 'F'}, implicit cell, {w.classes}-class xent on h_T, SGD",
               "solver": "serial sweep + BPTT" if args.serial else "MGRIT",
-              "l2": "inputs larger than L2 (x, gi and states are re-streamed from HBM every step)",
+              "l2": l2_note,
               "parallelism": f"replicas x{args.gpus} (no sharding, no collective)"}
 
     if args.impl == "reference":
