@@ -50,14 +50,17 @@ __device__ __forceinline__ void stg8(float* p, const float* v) {
                "f"(v[5]), "f"(v[6]), "f"(v[7])
                : "memory");
 }
-// eight values as bf16: one 16-byte store
-__device__ __forceinline__ void stg_bf8(__nv_bfloat16* p, const float* v) {
+__device__ __forceinline__ void tma_store_2d(const CUtensorMap* map, uint32_t src, int c0, int c1) {
+  asm volatile("cp.async.bulk.tensor.2d.global.shared::cta.tile.bulk_group [%0, {%2, %3}], [%1];" ::"l"(map), "r"(src), "r"(c0), "r"(c1)
+               : "memory");
+}
+// eight values as bf16 into shared memory: one 16-byte store
+__device__ __forceinline__ void sts_bf8(uint32_t addr, const float* v) {
   __nv_bfloat162 p0 = __floats2bfloat162_rn(v[0], v[1]), p1 = __floats2bfloat162_rn(v[2], v[3]);
   __nv_bfloat162 p2 = __floats2bfloat162_rn(v[4], v[5]), p3 = __floats2bfloat162_rn(v[6], v[7]);
-  uint4 pk;
-  pk.x = *reinterpret_cast<uint32_t*>(&p0); pk.y = *reinterpret_cast<uint32_t*>(&p1);
-  pk.z = *reinterpret_cast<uint32_t*>(&p2); pk.w = *reinterpret_cast<uint32_t*>(&p3);
-  *reinterpret_cast<uint4*>(p) = pk;
+  asm volatile("st.shared.v4.b32 [%0], {%1,%2,%3,%4};" ::"r"(addr), "r"(*reinterpret_cast<uint32_t*>(&p0)),
+               "r"(*reinterpret_cast<uint32_t*>(&p1)), "r"(*reinterpret_cast<uint32_t*>(&p2)), "r"(*reinterpret_cast<uint32_t*>(&p3))
+               : "memory");
 }
 __device__ __forceinline__ float4 lds4(uint32_t addr) {
   float4 v;
@@ -78,11 +81,16 @@ constexpr int BN = 192, UN = 64, CH = 16, NCH = UN / CH;
 constexpr int kThreads = 352;
 constexpr int kABytes = BM * BK * 2, kBBytes = BN * BK * 2, kStageBytes = kABytes + kBBytes;
 constexpr int kOpBytes = BM * CH * 4;   // one epilogue operand chunk: 128 rows x 16 floats
-template <bool HAS_G> struct CellCfg {
-  static constexpr int kStages = HAS_G ? 3 : 4;
+// The linearisation's four bf16 coefficient arrays leave through shared memory: per chunk four [128 x 16] bf16
+// tiles (32-byte swizzle), two buffers, written to global memory by TMA stores.  (Four 16-byte st.global per thread
+// and chunk, each touching 32 different rows, cost a third of that kernel's time.)
+constexpr int kCoefBytes = BM * CH * 2;   // one coefficient chunk: 128 rows x 16 bf16
+template <bool HAS_G, bool LIN = false> struct CellCfg {
+  static constexpr int kStages = (HAS_G || LIN) ? 3 : 4;
   static constexpr int kOps = HAS_G ? 5 : 4;
   static constexpr int kEpiBytes = kOps * kOpBytes;
-  static constexpr int kSmemBytes = kStages * kStageBytes + 2 * kEpiBytes + 1024 + 256;
+  static constexpr int kOutBytes = LIN ? 4 * kCoefBytes : 0;      // per buffer
+  static constexpr int kSmemBytes = kStages * kStageBytes + 2 * kEpiBytes + 2 * kOutBytes + 1024 + 256;
 };
 }  // namespace cellk
 
@@ -90,14 +98,17 @@ template <bool LIN, bool HAS_G>
 __global__ void __launch_bounds__(cellk::kThreads, 1)
 umma_cell_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB,
                  const __grid_constant__ CUtensorMap tmGI, const __grid_constant__ CUtensorMap tmHP,
-                 const __grid_constant__ CUtensorMap tmG, CellArgs p, int* status) {
+                 const __grid_constant__ CUtensorMap tmG, const __grid_constant__ CUtensorMap tmCR,
+                 const __grid_constant__ CUtensorMap tmCZ, const __grid_constant__ CUtensorMap tmCN,
+                 const __grid_constant__ CUtensorMap tmCP, CellArgs p, int* status) {
   using namespace cellk;
-  using C = CellCfg<HAS_G>;
+  using C = CellCfg<HAS_G, LIN>;
   extern __shared__ uint8_t smem_raw[];
   const uint32_t raw = smem_u32(smem_raw);
   const uint32_t tiles_base = (raw + 1023u) & ~1023u;
   const uint32_t epi_base = tiles_base + C::kStages * kStageBytes;
-  const uint32_t bars = epi_base + 2 * C::kEpiBytes;
+  const uint32_t out_base = epi_base + 2 * C::kEpiBytes;
+  const uint32_t bars = out_base + 2 * C::kOutBytes;
   auto full_bar = [&](int s) { return bars + 8u * s; };
   auto empty_bar = [&](int s) { return bars + 8u * (C::kStages + s); };
   auto tfull_bar = [&](int a) { return bars + 8u * (2 * C::kStages + a); };
@@ -205,20 +216,26 @@ umma_cell_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
     const uint32_t sw = (uint32_t)((r >> 1) & 3);
     const uint32_t off0 = (uint32_t)r * 64u + ((((uint32_t)half * 2u) ^ sw) << 4);
     const uint32_t off1 = (uint32_t)r * 64u + ((((uint32_t)half * 2u + 1u) ^ sw) << 4);
-    int it = 0, eb = 0; uint32_t ephase = 0;
+    // bf16 coefficient tiles, 32-byte swizzle: rows of 32 bytes, 16-byte piece index XOR ((row >> 2) & 1)
+    const uint32_t offb = (uint32_t)r * 32u + ((((uint32_t)half) ^ ((uint32_t)(r >> 2) & 1u)) << 4);
+    const bool storer = threadIdx.x == 96;   // the epilogue thread that issues the TMA stores
+    int it = 0, eb = 0, ob = 0; uint32_t ephase = 0;
+    // A thread whose wait ran out (ok = false) keeps walking the loops without touching data, so that the named
+    // barrier of the linearisation's store hand-over still sees all 256 epilogue threads.
     bool ok = true;
-    for (int t = blockIdx.x; t < tiles && ok; t += gridDim.x, ++it) {
+    for (int t = blockIdx.x; t < tiles; t += gridDim.x, ++it) {
       const int mt = t / n_tiles, nt = t % n_tiles;
       const int as = it & 1;
       const uint32_t aphase = (uint32_t)(it >> 1) & 1u;
       const int row = mt * BM + r;
       const bool valid = row < p.M;
       const int k = valid ? row / p.B : 0, b = valid ? row % p.B : 0;
-      if (!mbar_wait(tfull_bar(as), aphase, abortp, status, 15)) break;
+      if (ok && !mbar_wait(tfull_bar(as), aphase, abortp, status, 15)) ok = false;
       tc_fence_after();
       const uint32_t taddr = tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(as * BN);
       for (int c = 0; c < NCH; ++c) {
-        if (!mbar_wait(efull_bar(eb), ephase, abortp, status, 16)) { ok = false; break; }
+        if (ok && !mbar_wait(efull_bar(eb), ephase, abortp, status, 16)) ok = false;
+        if (ok) {
         const uint32_t src = epi_base + eb * C::kEpiBytes;
         float gr[8], gz[8], gn[8], hp[8], gg[8];
         *reinterpret_cast<float4*>(gr) = lds4(src + off0);                 *reinterpret_cast<float4*>(gr + 4) = lds4(src + off1);
@@ -282,17 +299,39 @@ umma_cell_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
             }
             const i64 idx = (i64)row * H + u;
             stg8(p.a + idx, oa);
-            stg_bf8(p.cr + idx, ocr);
-            stg_bf8(p.cz + idx, ocz);
-            stg_bf8(p.cn + idx, ocn);
-            if (p.cnp) stg_bf8(p.cnp + idx, ocp);
+            const uint32_t dst = out_base + ob * C::kOutBytes + offb;
+            sts_bf8(dst, ocr);
+            sts_bf8(dst + kCoefBytes, ocz);
+            sts_bf8(dst + 2 * kCoefBytes, ocn);
+            if (p.cnp) sts_bf8(dst + 3 * kCoefBytes, ocp);
           }
         }
+        }  // ok
+        if (LIN) {
+          // Chunk c's coefficients sit in output buffer ob.  Make them visible to the async proxy; the storing
+          // thread first waits until the stores issued one chunk ago have finished READING the other buffer (they
+          // had a whole chunk of time), so that after the barrier everybody may overwrite it with chunk c + 1.
+          asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+          if (storer) asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory");
+          asm volatile("bar.sync 1, 256;" ::: "memory");
+          if (storer && ok) {
+            const uint32_t srcb = out_base + ob * C::kOutBytes;
+            const int u = nt * UN + c * CH, row0 = mt * BM;
+            tma_store_2d(&tmCR, srcb, u, row0);
+            tma_store_2d(&tmCZ, srcb + kCoefBytes, u, row0);
+            tma_store_2d(&tmCN, srcb + 2 * kCoefBytes, u, row0);
+            if (p.cnp) tma_store_2d(&tmCP, srcb + 3 * kCoefBytes, u, row0);
+            asm volatile("cp.async.bulk.commit_group;" ::: "memory");
+          }
+          ob ^= 1;
+        }
       }
-      if (!ok) break;
-      tc_fence_before();
-      mbar_arrive(tempty_bar(as));
+      if (ok) {
+        tc_fence_before();
+        mbar_arrive(tempty_bar(as));
+      }
     }
+    if (LIN && storer) asm volatile("cp.async.bulk.wait_group 0;" ::: "memory");   // coefficients are in global memory before exit
   }
 
   // ------------------------------------------------------------ teardown

@@ -156,13 +156,26 @@ bool make_map3(CUtensorMap* m, CUtensorMapDataType dt, size_t esize, const void*
   return r == CUDA_SUCCESS;
 }
 
+// 2-D map of a row-major [rows, inner] array (row pitch ld elements), box {box_inner, box_rows}
+bool make_map2(CUtensorMap* m, CUtensorMapDataType dt, size_t esize, const void* base, uint64_t inner, uint64_t rows, uint64_t ld,
+               uint32_t box_inner, uint32_t box_rows, CUtensorMapSwizzle sw) {
+  cuuint64_t dims[2] = {inner, rows};
+  cuuint64_t strides[1] = {ld * esize};
+  cuuint32_t box[2] = {box_inner, box_rows};
+  cuuint32_t estr[2] = {1, 1};
+  CUresult r = g_encode(m, dt, 2, (void*)base, dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE, sw,
+                        CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  if (r != CUDA_SUCCESS) fprintf(stderr, "mgrit_gru: cuTensorMapEncodeTiled (2-D) failed (%d)\n", (int)r);
+  return r == CUDA_SUCCESS;
+}
+
 // Fused recurrent GEMM + cell (forward step or linearisation) with TMA-staged epilogue operands.
 // Rows (k, b), k = 0..nk-1: A rows at A + k*a_ks + b*H (bf16), gi rows at gi + k*gi_ks + b*3H,
 // previous state at hp + k*hp_ks + b*H, optional additive term at g + k*g_ks + b*H.
 template <bool LIN, bool HAS_G>
 bool launch_cell(int kc, const bf16* A, i64 a_ks, const float* gi, i64 gi_ks, const float* hp, i64 hp_ks, const float* g, i64 g_ks,
                  int nk, const bf16* W, CellArgs ca, cudaStream_t s) {
-  using C = cellk::CellCfg<HAS_G>;
+  using C = cellk::CellCfg<HAS_G, LIN>;
   if (nk <= 0) return true;
   if (!ensure_driver()) return false;
   static bool attr_set = false;
@@ -183,10 +196,18 @@ bool launch_cell(int kc, const bf16* A, i64 a_ks, const float* gi, i64 gi_ks, co
   } else {
     tg = thp;
   }
+  // linearisation: the four bf16 coefficient arrays [M, H] are written by TMA stores of [128 x 16] tiles
+  CUtensorMap tcr = thp, tcz = thp, tcn = thp, tcp = thp;
+  if (LIN) {
+    auto cmap = [&](CUtensorMap* m, const bf16* base) {
+      return make_map2(m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, base, H, (uint64_t)ca.M, H, cellk::CH, BM, CU_TENSOR_MAP_SWIZZLE_32B);
+    };
+    if (!cmap(&tcr, ca.cr) || !cmap(&tcz, ca.cz) || !cmap(&tcn, ca.cn) || (ca.cnp && !cmap(&tcp, ca.cnp))) return false;
+  }
   int tiles = ((ca.M + BM - 1) / BM) * (H / cellk::UN);
   int grid = tiles < kSMs ? tiles : kSMs;
   prof_begin(kc, 2.0 * ca.M * 3.0 * H * H, s);
-  if (launch_pdl(kern, dim3(grid), dim3(cellk::kThreads), C::kSmemBytes, s, ta, tb, tgi, thp, tg, ca, g_status_ptr) != cudaSuccess) return false;
+  if (launch_pdl(kern, dim3(grid), dim3(cellk::kThreads), C::kSmemBytes, s, ta, tb, tgi, thp, tg, tcr, tcz, tcn, tcp, ca, g_status_ptr) != cudaSuccess) return false;
   prof_end(s);
   count_launch();
   return true;
