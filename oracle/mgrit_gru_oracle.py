@@ -17,6 +17,10 @@ What pins each function (see tests/test_oracle_*.py):
                                                 brute force on T=8, dense two-level error
                                                 propagator for the linear adjoint problem,
                                                 hierarchy sizes quoted in the paper
+  * multilevel recursion (time step c_f^l, input
+    row c_f^l j - 1, FAS term of inner levels) .. three-level cycles written out level by level
+                                                with each level's own propagator, forward and
+                                                adjoint, c_f = 2, 3, 4 (tests/test_oracle_three_level.py)
   * loss head ................................. torch.nn.functional.cross_entropy float64
   * Adam ...................................... torch.optim.Adam float64
   * values after a FEW cycles (2-3) ........... parity unpinned by the paper (an iteration's
