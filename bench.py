@@ -23,12 +23,14 @@ sys.path.insert(0, ROOT)
 
 METRIC = "MGRIT-GRU fwd+adjoint timesteps*batch/sec"
 UNIT = "timesteps*batch/s"
-# DRAM bytes (read + write) of the fused forward-step kernel per (row x hidden unit), from ncu captures of that
-# kernel: 23.2 B on the default workload's own 16384-row launches (389 MB per launch, H = 1024;
-# profiles/fused_cell_kernel_train.md) and 19.5 B on the smaller `medium` case (81.7 MB for 8192 rows x 512 units,
-# where more of the previous step's output is still in L2; profiles/fused_cell_kernel_medium.md).  Traffic grows
-# in proportion to rows x hidden units, so a workload's per-launch traffic is its figure x its average rows x H.
+# DRAM bytes (dram__bytes_read.sum + dram__bytes_write.sum) of the fused forward-step kernel per (row x hidden
+# unit).  These are constants taken from `ncu --set full --clock-control none` captures of two launches of that
+# kernel, NOT measured in a bench run: 23.2 B on the default workload's own 16384-row launches (389 MB per launch,
+# H = 1024) and 19.5 B on the smaller `medium` case (81.7 MB for 8192 rows x 512 units, where more of the previous
+# step's output is still in L2).  Traffic grows in proportion to rows x hidden units, so a workload's per-launch
+# traffic is its figure x its average rows x H.
 NCU_DRAM_BYTES_PER_ROW_UNIT = {"forward_step": {1024: 23.2, 512: 19.5}}
+NOMINAL_BF16_TFLOPS = 2250.0       # dense bf16, vendor figure (context only)
 
 
 def measured_peaks():
@@ -122,17 +124,25 @@ class ClockSampler:
         except Exception:
             self.p.kill()
             out = ""
+        self.p = None
         names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
-        rows = []
+        self.rows = []
         for line in out.strip().splitlines():
             f = [s.strip() for s in line.split(",")]
             if len(f) < 8:
                 continue
             try:
                 ts = datetime.datetime.strptime(f[0], "%Y/%m/%d %H:%M:%S.%f")
-                rows.append((ts, float(f[1]), float(f[2]), [n for n, v in zip(names, f[4:8]) if v.lower().startswith("active")]))
+                self.rows.append((ts, float(f[1]), float(f[2]), [n for n, v in zip(names, f[4:8]) if v.lower().startswith("active")]))
             except ValueError:
                 continue
+        return self.window(t0, t1)
+
+    def window(self, t0, t1):
+        """Clock summary of the samples inside [t0, t1] (host wall clock); valid after stop()."""
+        rows = getattr(self, "rows", [])
+        if not rows:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": [], "samples": 0}
         inside = [r for r in rows if t0 is not None and t0 <= r[0] <= t1]
         scope = "timed region"
         if not inside:        # region shorter than the polling period: take the samples nearest to it
@@ -143,6 +153,46 @@ class ClockSampler:
         reasons = sorted({n for r in inside for n in r[3]})
         return {"sm_mhz": statistics.median(sm) if sm else None, "sm_max_mhz": max(r[2] for r in inside) if inside else None,
                 "reasons": reasons, "samples": len(sm), "scope": scope}
+
+
+# ------------------------------------------------------------------------------------------ GPU helpers
+def describe(w, T, Bsz):
+    return (f"{w.name}: {w.layers}-layer GRU I={w.I} H={w.H} B={Bsz} T={T}, cf={w.cf}, levels={w.levels}, "
+            f"iters fwd/adj={w.iters_fwd}/{w.iters_adj}, relax fine/coarse={'FCF' if w.relax_fine else 'F'}/"
+            f"{'FCF' if w.relax_coarse else 'F'}, implicit cell, {w.classes}-class xent on h_T, SGD")
+
+
+def time_gpu_step(w, T, serial, steps, warmup, dev, use_graph=True):
+    """Device-resident inputs; returns (ms per step, wall-clock window of the timed region).  The same step as the
+    headline (all layers forward, head, adjoint, gradients, SGD) with MGRIT or with the serial sweep + exact BPTT."""
+    import datetime
+    import torch
+    from paper_2203_04738_b200 import binding as B
+    from paper_2203_04738_b200.synthetic import make_inputs
+    from paper_2203_04738_b200.train_step import GraphedTrainingStep, alloc_buffers, training_step
+    d = make_inputs(w, T=T)
+    up = lambda a: torch.from_numpy(a).to(dev)
+    layers = [{n: up(l[n]) for n in ("W_ih", "W_hh", "b_ih", "b_hh")} for l in d["layers"]]
+    W_c, b_c, labels, h0, x = up(d["W_c"]), up(d["b_c"]), up(d["labels"]), up(d["h0"]), up(d["x"])
+    buf = alloc_buffers(w, T, w.B, dev, serial=serial, flags=B.FLAG_SKIP_DUPLICATE_FRELAX)
+    step = lambda: training_step(w, layers, W_c, b_c, x, h0, labels, buf)
+    if use_graph:
+        try:
+            step = GraphedTrainingStep(w, layers, W_c, b_c, x, h0, labels, buf)
+        except Exception as e:
+            sys.stderr.write(f"bench: CUDA graph capture failed ({e!r}); launching from the host\n")
+    for _ in range(max(warmup, 3)):
+        step()
+    torch.cuda.synchronize()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    t0 = datetime.datetime.now()
+    e0.record()
+    for _ in range(steps):
+        step()
+    e1.record()
+    torch.cuda.synchronize()
+    t1 = datetime.datetime.now()
+    return e0.elapsed_time(e1) / steps, (t0, t1)
 
 
 # ------------------------------------------------------------------------------------------ main
@@ -159,6 +209,8 @@ def main():
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-graph", action="store_true", help="launch every kernel from the host instead of replaying a CUDA graph")
     ap.add_argument("--no-kernel-timing", action="store_true", help="skip the per-kernel CUDA-event pass")
+    ap.add_argument("--no-serial", action="store_true", help="skip the GPU serial-sweep leg (gpu_serial)")
+    ap.add_argument("--no-sweep", action="store_true", help="skip the sequence-length sweep (t_sweep)")
     args = ap.parse_args()
 
     from paper_2203_04738_b200.synthetic import WORKLOADS, make_inputs
@@ -171,9 +223,7 @@ def main():
     stream_mb = 4.0 * T * w.B * (w.I + w.layers * 4 * w.H) / 1e6
     l2_note = (f"inputs larger than L2 (x, gi and states, {stream_mb:.0f} MB, are re-streamed from HBM every step)" if stream_mb > 126.0
                else f"working set {stream_mb:.1f} MB fits the 126 MB L2 and no flush is done: an L2-resident side case, not the headline configuration")
-    config = {"workload": f"{w.name}: {w.layers}-layer GRU I={w.I} H={w.H} B={w.B} T={T}, cf={w.cf}, levels={w.levels}, "
-                          f"iters fwd/adj={w.iters_fwd}/{w.iters_adj}, relax fine/coarse={'FCF' if w.relax_fine else 'F'}/"
-                          f"{'FCF' if w.relax_coarse else 'F'}, implicit cell, {w.classes}-class xent on h_T, SGD",
+    config = {"workload": describe(w, T, w.B),
               "solver": "serial sweep + BPTT" if args.serial else "MGRIT",
               "l2": l2_note,
               "parallelism": f"replicas x{args.gpus} (no sharding, no collective)"}
@@ -182,6 +232,12 @@ def main():
         if rank != 0:
             return
         cb, sec = time_oracle(w, steps=args.steps, warmup=min(args.warmup, 1))
+        # this arm times a bounded sample of the workload (same widths, levels and cycle counts): say so
+        Ts, Bs = cpu_sample_shape(w)
+        config = {"workload": describe(w, Ts, Bs) + f" -- a bounded sample of '{w.name}' (T={w.T}, B={w.B}), which the fp64 "
+                              "oracle cannot finish within minutes",
+                  "solver": "MGRIT (fp64 NumPy oracle on the host cores)", "l2": "n/a (CPU)",
+                  "parallelism": "host threads of the BLAS library"}
         print(json.dumps({"metric": METRIC, "value": cb["value"], "unit": UNIT, "n_gpus": args.gpus, "steps": args.steps,
                           "warmup": args.warmup, "ms_per_step": sec * 1e3, "higher_is_better": True, "scaling": "weak",
                           "vs_baseline": None, "dtype": "f64", "data": "synthetic", "config": config, "impl": "reference",
@@ -249,7 +305,7 @@ def main():
     wall1 = datetime.datetime.now()
     ms = e0.elapsed_time(e1)
     launches = graphed.launches * args.steps if graphed is not None else B.kernel_launches() - l0
-    clocks = sampler.stop(wall0, wall1) if sampler else None
+    windows = {"headline": (wall0, wall1)}      # the clock sampler keeps running through the later legs
     ms = max_over_ranks(ms, dev)
     ms_step = ms / args.steps
     value = job_throughput(T * w.B, ms_step, world)
@@ -287,7 +343,7 @@ def main():
 
     # per-kernel timing pass (CUDA events around every GEMM-shaped launch; outside the timed region so
     # that the event records do not perturb it)
-    roofline, breakdown, by_size = None, None, None
+    roofline, breakdown, by_size, roofline_by_class = None, None, None, None
     if rank == 0 and not args.no_kernel_timing:
         torch.cuda.synchronize()
         nprof = 2
@@ -307,25 +363,78 @@ def main():
         bf16 = w.operands == 2
         breakdown = {k: {"ms_per_step": v[0] / nprof, "launches_per_step": v[1] // nprof,
                          "tflops": (v[2] / (v[0] * 1e-3) / 1e12) if v[0] > 0 else None} for k, v in prof.items()}
-        dom = max(prof.items(), key=lambda kv: kv[1][0])
-        name, (tms, n, fl) = dom
+        # The dominant KERNEL: classes that time one kernel per record (the adjoint-step class times its operand
+        # packing kernel together with the product, the gradient class a whole pass of several kernels).
+        single = {k: v for k, v in prof.items() if k not in ("adjoint_step", "gradient_gemms")}
+        name, (tms, n, fl) = max(single.items(), key=lambda kv: kv[1][0])
+        if bf16:
+            peak = float(peaks.get("bf16_tflops_sustained", peaks["bf16_tflops"]))
+            burst = float(peaks["bf16_tflops"])
+            bound, note = "tensor", (f"bf16 dense cuBLAS figures ({pk}): `peak`/`frac` use the sustained one (the kernel is timed inside "
+                                     "whole steps), `frac_burst` the burst one, `frac_nominal` the vendor's 2250 TFLOP/s")
+        else:
+            # fp32 FFMA: 148 SMs x 128 lanes x 2 flop x max SM clock
+            peak = burst = 148 * 128 * 2 * float(peaks.get("sm_max_mhz", 1965.0)) * 1e6 / 1e12
+            bound, note = "alu", "fp32 FFMA: 148 SMs x 128 lanes x 2 flop x max SM clock"
         if tms > 0 and n > 0:
             achieved = fl / (tms * 1e-3) / 1e12
-            if bf16:
-                peak = float(peaks.get("bf16_tflops_sustained", peaks["bf16_tflops"]))
-                bound, note = "tensor", f"bf16 dense, sustained cuBLAS figure ({pk})"
-            else:
-                # fp32 FFMA: 148 SMs x 128 lanes x 2 flop x max SM clock
-                peak = 148 * 128 * 2 * float(peaks.get("sm_max_mhz", 1965.0)) * 1e6 / 1e12
-                bound, note = "alu", "fp32 FFMA: 148 SMs x 128 lanes x 2 flop x max SM clock"
+            units = (fl / n) / (6.0 * w.H)          # (row x hidden unit) pairs of an average launch
             roofline = {"kernel": name, "bound": bound, "achieved": achieved, "peak": peak, "unit": "TFLOP/s",
-                        "frac": achieved / peak,
-                        "traffic": (NCU_DRAM_BYTES_PER_ROW_UNIT[name][w.H] * (fl / n) / (6.0 * w.H)
+                        "frac": achieved / peak, "frac_sustained": achieved / peak, "frac_burst": achieved / burst,
+                        "frac_nominal": achieved / NOMINAL_BF16_TFLOPS if bf16 else None, "peak_burst": burst,
+                        "traffic": (NCU_DRAM_BYTES_PER_ROW_UNIT[name][w.H] * units
                                     if w.H in NCU_DRAM_BYTES_PER_ROW_UNIT.get(name, {}) else None),
-                        "traffic_note": "DRAM bytes per average launch: ncu figure per (row x hidden unit) of this kernel at this H x the launch's rows x H",
-                        "algorithmic_bytes": 24.0 * (fl / n) / (6.0 * w.H) if name == "forward_step" else None,
+                        "traffic_note": "DRAM bytes per average launch = a constant from an ncu capture of this kernel (bytes per "
+                                        "row x hidden unit at this H) x the launch's rows x H; not measured in this run",
+                        # per cell evaluation the method moves 3H of gi + H written + H/(cf-1) read of state, fp32:
+                        # 16H + 4H/(cf-1) bytes; this implementation also writes and reads a bf16 copy of the state
+                        # and re-reads the fp32 state every step: 24H bytes
+                        "algorithmic_bytes": (16.0 + 4.0 / (w.cf - 1)) * units if name == "forward_step" else None,
+                        "implementation_bytes": 24.0 * units if name == "forward_step" else None,
                         "avg_launch_us": tms / n * 1e3, "launches_per_step": n // nprof,
                         "share_of_gemm_time": tms / max(sum(v[0] for v in prof.values()), 1e-9), "peak_source": note}
+        roofline_by_class = {k: {"tflops": v[2] / (v[0] * 1e-3) / 1e12, "frac_sustained": v[2] / (v[0] * 1e-3) / 1e12 / peak,
+                                 "frac_burst": v[2] / (v[0] * 1e-3) / 1e12 / burst, "ms_per_step": v[0] / nprof}
+                             for k, v in prof.items() if v[0] > 0 and k not in ("forward_serial_chain", "adjoint_serial_chain")}
+        for k in ("forward_serial_chain", "adjoint_serial_chain"):     # latency-bound: time per dependent step
+            if prof[k][0] > 0:
+                nsteps = prof[k][2] / (2.0 * w.B * 3.0 * w.H * w.H)
+                roofline_by_class[k] = {"us_per_dependent_step": prof[k][0] * 1e3 / nsteps, "ms_per_step": prof[k][0] / nprof}
+
+    # ---- the same GPU's serial sweep + exact BPTT on the same workload, and the speed-up over it as T grows
+    gpu_serial, t_sweep = None, None
+    if rank == 0 and world == 1 and not args.serial:
+        from paper_2203_04738_b200.synthetic import WORKLOADS as _W
+        if not args.no_serial:
+            ms_s, win = time_gpu_step(w, T, True, 5, 3, dev, use_graph=not args.no_graph)
+            windows["gpu_serial"] = win
+            gpu_serial = {"ms_per_step": ms_s, "value": T * w.B / (ms_s * 1e-3), "unit": UNIT, "steps": 5,
+                          "speedup_mgrit_over_serial": ms_s / ms_step,
+                          "what": "same step with gru_serial_forward / gru_serial_backward (exact sweep + BPTT) instead of MGRIT"}
+        if not args.no_sweep:
+            wl = _W["long"]
+            t_sweep = {"workload": describe(wl, "{512,1024,2048,4096}", wl.B), "points": []}
+            for Ts in (512, 1024, 2048, 4096):
+                ms_m, win_m = time_gpu_step(wl, Ts, False, 5, 3, dev, use_graph=not args.no_graph)
+                ms_r, win_r = time_gpu_step(wl, Ts, True, 3, 3, dev, use_graph=not args.no_graph)
+                windows[f"sweep_T{Ts}_mgrit"] = win_m
+                windows[f"sweep_T{Ts}_serial"] = win_r
+                t_sweep["points"].append({"T": Ts, "mgrit_ms": ms_m, "serial_ms": ms_r, "speedup": ms_r / ms_m})
+                torch.cuda.empty_cache()
+    clocks = None
+    if sampler:
+        clocks = sampler.stop(*windows["headline"])
+        for k, win in windows.items():
+            if k == "headline":
+                continue
+            c = sampler.window(*win)
+            if k == "gpu_serial" and gpu_serial:
+                gpu_serial["clocks"] = c
+            elif t_sweep:
+                Ts, leg = k.split("_")[1][1:], k.split("_")[2]
+                for pt in t_sweep["points"]:
+                    if str(pt["T"]) == Ts:
+                        pt[f"clocks_{leg}"] = {"sm_mhz": c["sm_mhz"], "reasons": c["reasons"], "samples": c["samples"]}
 
     if rank != 0:
         if world > 1:
@@ -339,6 +448,9 @@ def main():
            "ms_per_step": ms_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
            "dtype": "bf16" if w.operands == 2 else "f32", "data": "synthetic", "config": config, "clocks": clocks,
            "e2e": e2e, "gpu_launches": int(launches), "roofline": roofline, "cpu_baseline": cpu,
+           "gpu_serial": gpu_serial, "t_sweep": t_sweep, "roofline_by_class": roofline_by_class,
+           "paper_context": "the paper reports up to 6.5x over serial training on 288 Xeon cores (32 MPI ranks x 9 threads) for T=128; "
+                            "another machine and workload: context, not a target",
            "host_enqueue_ms_per_step": host_ms, "kernel_breakdown": breakdown, "kernel_by_size": by_size, "loss": float(loss.item()), "device_status": status}
     print(json.dumps(out))
     if world > 1:

@@ -19,7 +19,12 @@
  *  - Return value: MGRIT_OK (0) or a negative error code; outputs are undefined after an error.
  *    Nothing aborts the process.  Device-side waits are bounded: a wait that runs out makes the
  *    next synchronising call (or mgrit_gru_last_device_status) report MGRIT_DEVICE_TIMEOUT.
- *  - One GPU, the current device.  Calls that share a workspace must not overlap on the GPU.
+ *  - A call works on the device that is current when it is made (no sharding, no collectives); a process may use
+ *    the library on several devices, each with its own workspaces.  Calls that share a workspace must not overlap
+ *    on the GPU.  The library is NOT thread-safe: calls made from several host threads must be serialised by the
+ *    caller (the launch counter is atomic; the profiling records and the first-use set-up of a device are not).
+ *  - Sizes: (T + 1) * B must stay below 2^31 - 1024 (row counts are 32-bit inside the kernels; element offsets
+ *    are 64-bit); larger problems are rejected with MGRIT_UNSUPPORTED.
  */
 #ifndef MGRIT_GRU_H_
 #define MGRIT_GRU_H_
@@ -38,8 +43,9 @@ enum {
   MGRIT_INVALID_ARG = -1,        /* NULL pointer, non-positive size, unknown enum value */
   MGRIT_NOT_DIVISIBLE = -2,      /* T is not a multiple of cf^(levels-1) */
   MGRIT_WORKSPACE_TOO_SMALL = -3,
-  MGRIT_UNSUPPORTED = -4,        /* shape outside what the selected operand mode supports */
-  MGRIT_CUDA_ERROR = -5,         /* a CUDA runtime/driver call failed */
+  MGRIT_UNSUPPORTED = -4,        /* shape outside what the selected operand mode supports, or beyond 32-bit row counts */
+  MGRIT_CUDA_ERROR = -5,         /* a CUDA runtime/driver call failed: a launch, or the preparation of one (tensor-map
+                                    encoding); nothing further is enqueued by that call and its outputs are undefined */
   MGRIT_DEVICE_TIMEOUT = -6,     /* a bounded device-side wait ran out */
   MGRIT_SCRATCH_LIMIT = -7       /* problem larger than the built-in scratch of a no-allocation entry point */
 };
@@ -111,7 +117,8 @@ int mgrit_gru_forward(const mgrit_gru_cfg* cfg, const gru_params* p, const float
  * pass g_i = w_i dh_i/dTheta.
  *   dh_seed[T,B,H] or NULL: direct loss derivative w.r.t. every h_t (stacked layers);
  *   dhT[B,H] or NULL: direct loss derivative w.r.t. h_T, added to dh_seed[T-1]; one of the two
- *   must be given.  Outputs: dh[T,B,H] total dL/dh_t, dh0[B,H], dx[T,B,I] or NULL, grads.
+ *   must be given.  Outputs: dh[T,B,H] total dL/dh_t or NULL (a training step only needs dx and the gradients),
+ *   dh0[B,H], dx[T,B,I] or NULL, grads.
  *   gi is the projection written by the forward call for the same x and parameters. */
 int mgrit_gru_adjoint(const mgrit_gru_cfg* cfg, const gru_params* p, const float* x, const float* h0,
                       const float* gi, const float* h, const float* dh_seed, const float* dhT,
@@ -132,7 +139,9 @@ int gru_serial_backward(const mgrit_gru_cfg* cfg, const gru_params* p, const flo
 /* Classifier head on h_T with mean softmax cross-entropy (the loss whose gradient seeds the
  * backward block: w_T = grad_{h_T} L).  hT[B,H], Wc[C,H], bc[C], labels[B] (int32, device)
  * -> loss[1] (device), dhT[B,H], dWc[C,H], dbc[C].  ws: device scratch of at least
- * xent_head_workspace_bytes(B, C) bytes. */
+ * xent_head_workspace_bytes(B, C) bytes.  C <= 8192 (the logits of a row are kept in shared memory), otherwise
+ * MGRIT_UNSUPPORTED.  A label outside [0, C) marks a row without a target: it contributes nothing to the loss and
+ * has no one-hot term (the mean still divides by B).  All sums run in a fixed order: results repeat bit for bit. */
 size_t xent_head_workspace_bytes(int32_t B, int32_t C);
 int xent_head_fwd_bwd(int32_t B, int32_t H, int32_t C, const float* hT, const float* Wc, const float* bc,
                       const int32_t* labels, float* loss, float* dhT, float* dWc, float* dbc,
@@ -145,12 +154,13 @@ int xent_head_fwd_bwd(int32_t B, int32_t H, int32_t C, const float* hT, const fl
  * and may synchronise the device.  Instead of a workspace argument the [B, C] intermediate (loss
  * derivative w.r.t. the logits) is kept in a fixed 256 KiB array that is part of the library image:
  * every GPU that loads the library holds it until the process exits.
- *   Limit: B * C <= 65536, otherwise MGRIT_SCRATCH_LIMIT is returned and nothing is launched.
+ *   Limit: B * (C + 1) <= 65536 (the derivatives and one loss term per row), otherwise MGRIT_SCRATCH_LIMIT is
+ *   returned and nothing is launched; C <= 8192 as for xent_head_fwd_bwd (MGRIT_UNSUPPORTED).
  *   The call performs no cudaMalloc / cudaFree and calls no allocating routine.
  *   The first call on each device looks up the array's device address (once per device, with that
  *   device current); make that first call before any stream capture is started on the device.
  *   All calls share the one array, which keeps the previous call's contents; nothing in it needs to be
- *   cleared between calls (each call overwrites the B * C entries it reads).  Two calls that overlap on
+ *   cleared between calls (each call overwrites the B * (C + 1) entries it reads).  Two calls that overlap on
  *   the GPU (different streams, or different host threads) race on it: serialise them.
  *   Inputs, outputs and results are exactly those of xent_head_fwd_bwd. */
 int xent_head_fwd_bwd_noalloc(int32_t B, int32_t H, int32_t C, const float* hT, const float* Wc, const float* bc,
@@ -168,9 +178,15 @@ int sgd_update(float* p, const float* g, size_t n, float lr, mgrit_stream_t stre
 int adam_update(float* p, const float* g, float* m, float* v, size_t n, float lr, float beta1, float beta2, float eps,
                 int32_t step, mgrit_stream_t stream);
 
-/* Status word written by bounded device-side waits since the library was loaded (0 = none ran out).
- * Synchronises the device. */
+/* Status of the bounded device-side waits on the current device since the library was loaded or the status was
+ * last cleared: MGRIT_OK, or MGRIT_DEVICE_TIMEOUT when one ran out.  Synchronises the device.
+ * The status words are sticky: once a wait has run out, every later persistent kernel on that device sees the
+ * non-zero word and leaves early (its results are then incomplete), until mgrit_gru_clear_device_status() is
+ * called.  Asynchronous calls cannot report the condition themselves; after MGRIT_DEVICE_TIMEOUT discard the
+ * results computed since the last MGRIT_OK status, clear the status and repeat the work. */
 int mgrit_gru_last_device_status(void);
+/* Synchronises the current device and resets its status words to zero. */
+int mgrit_gru_clear_device_status(void);
 
 /* Number of kernels this library has launched since it was loaded (all streams). */
 unsigned long long mgrit_gru_kernel_launches(void);

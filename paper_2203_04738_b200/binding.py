@@ -57,6 +57,7 @@ lib.xent_head_fwd_bwd_noalloc.argtypes = [_i32, _i32, _i32, _vp, _vp, _vp, _vp, 
 lib.sgd_update.argtypes = [_vp, _vp, _sz, ctypes.c_float, _vp]
 lib.adam_update.argtypes = [_vp, _vp, _vp, _vp, _sz, ctypes.c_float, ctypes.c_float, ctypes.c_float, ctypes.c_float, _i32, _vp]
 lib.mgrit_gru_last_device_status.restype = ctypes.c_int
+lib.mgrit_gru_clear_device_status.restype = ctypes.c_int
 lib.mgrit_gru_kernel_launches.restype = ctypes.c_ulonglong
 lib.mgrit_gru_profile_enable.argtypes = [ctypes.c_int]
 lib.mgrit_gru_profile_read.argtypes = [ctypes.c_int, ctypes.POINTER(ctypes.c_double), ctypes.POINTER(ctypes.c_ulonglong),
@@ -146,7 +147,7 @@ def gru_serial_forward(cfg, p, x, h0, gi=None, h=None, ws=None):
 
 @dataclass
 class AdjointResult:
-    dh: torch.Tensor
+    dh: torch.Tensor | None
     dh0: torch.Tensor
     dx: torch.Tensor | None
     dW_ih: torch.Tensor
@@ -156,10 +157,10 @@ class AdjointResult:
     resnorm: list | None = None
 
 
-def _adjoint(fn, serial, cfg, p, x, h0, gi, h, dh_seed, dhT, want_dx, want_resnorm, ws, out):
+def _adjoint(fn, serial, cfg, p, x, h0, gi, h, dh_seed, dhT, want_dx, want_resnorm, ws, out, want_dh=True):
     dev = x.device
     o = out or AdjointResult(
-        dh=torch.empty(cfg.T, cfg.B, cfg.H, device=dev), dh0=torch.empty(cfg.B, cfg.H, device=dev),
+        dh=torch.empty(cfg.T, cfg.B, cfg.H, device=dev) if want_dh else None, dh0=torch.empty(cfg.B, cfg.H, device=dev),
         dx=torch.empty(cfg.T, cfg.B, cfg.I, device=dev) if want_dx else None,
         dW_ih=torch.empty(3 * cfg.H, cfg.I, device=dev), dW_hh=torch.empty(3 * cfg.H, cfg.H, device=dev),
         db_ih=torch.empty(3 * cfg.H, device=dev), db_hh=torch.empty(3 * cfg.H, device=dev))
@@ -177,12 +178,13 @@ def _adjoint(fn, serial, cfg, p, x, h0, gi, h, dh_seed, dhT, want_dx, want_resno
     return o
 
 
-def mgrit_gru_adjoint(cfg, p, x, h0, gi, h, dh_seed=None, dhT=None, want_dx=True, want_resnorm=False, ws=None, out=None):
-    return _adjoint(lib.mgrit_gru_adjoint, False, cfg, p, x, h0, gi, h, dh_seed, dhT, want_dx, want_resnorm, ws, out)
+def mgrit_gru_adjoint(cfg, p, x, h0, gi, h, dh_seed=None, dhT=None, want_dx=True, want_resnorm=False, ws=None, out=None,
+                      want_dh=True):
+    return _adjoint(lib.mgrit_gru_adjoint, False, cfg, p, x, h0, gi, h, dh_seed, dhT, want_dx, want_resnorm, ws, out, want_dh)
 
 
-def gru_serial_backward(cfg, p, x, h0, gi, h, dh_seed=None, dhT=None, want_dx=True, ws=None, out=None):
-    return _adjoint(lib.gru_serial_backward, True, cfg, p, x, h0, gi, h, dh_seed, dhT, want_dx, False, ws, out)
+def gru_serial_backward(cfg, p, x, h0, gi, h, dh_seed=None, dhT=None, want_dx=True, ws=None, out=None, want_dh=True):
+    return _adjoint(lib.gru_serial_backward, True, cfg, p, x, h0, gi, h, dh_seed, dhT, want_dx, False, ws, out, want_dh)
 
 
 def xent_head_fwd_bwd(hT, Wc, bc, labels, ws=None):
@@ -229,6 +231,10 @@ def adam_update(p, g, m, v, lr, step, beta1=0.9, beta2=0.999, eps=1e-8):
 
 def last_device_status() -> int:
     return lib.mgrit_gru_last_device_status()
+
+
+def clear_device_status() -> None:
+    _check(lib.mgrit_gru_clear_device_status())
 
 
 def kernel_launches() -> int:

@@ -1,6 +1,7 @@
 // C ABI, argument validation, workspace layout and the host side of the multigrid cycle.
 // The cycle logic is written once over an abstract "step" and instantiated for the forward
 // recurrence and for its adjoint; every step, transfer and reduction is a kernel launch.
+#include <limits.h>
 #include <math.h>
 #include <stdio.h>
 #include <string.h>
@@ -13,7 +14,7 @@
 
 namespace mg {
 
-unsigned long long g_kernel_launches = 0;
+std::atomic<unsigned long long> g_kernel_launches{0};
 bool g_prof_on = false;
 
 namespace {
@@ -28,14 +29,17 @@ cudaEvent_t prof_event() {
 }
 }  // namespace
 
+static int g_prof_depth = 0;
 void prof_begin(int kc, double flops, cudaStream_t s) {
   if (!g_prof_on) return;
+  if (g_prof_depth++ > 0) return;     // inside an open record
   ProfRec r{kc, flops, prof_event(), prof_event()};
   cudaEventRecord(r.e0, s);
   g_prof_recs.push_back(r);
 }
 void prof_end(cudaStream_t s) {
-  if (!g_prof_on || g_prof_recs.empty()) return;
+  if (!g_prof_on || g_prof_depth == 0) return;
+  if (--g_prof_depth > 0 || g_prof_recs.empty()) return;
   cudaEventRecord(g_prof_recs.back().e1, s);
 }
 
@@ -76,6 +80,8 @@ int check_cfg(const mgrit_gru_cfg* c, Hier* hr) {
   if (c->operands != MGRIT_OPERANDS_FP32 && c->operands != MGRIT_OPERANDS_BF16) return MGRIT_INVALID_ARG;
   if (!(c->dt > 0.f)) return MGRIT_INVALID_ARG;
   if (c->H % 8 != 0 || c->I % 8 != 0) return MGRIT_UNSUPPORTED;
+  // row counts (T+1)*B, widths and grid sizes are 32-bit inside the kernels; element offsets are 64-bit
+  if (((i64)c->T + 1) * c->B > (i64)INT_MAX - 1024 || (i64)3 * c->H > INT_MAX / 4 || c->I > INT_MAX / 4) return MGRIT_UNSUPPORTED;
   i64 m = 1;
   hr->L = c->levels;
   for (int l = 0; l < c->levels; ++l) {
@@ -104,7 +110,7 @@ struct AdjWs {
   float* U[kMaxLevels]; float* G[kMaxLevels];
   float *a[kMaxLevels], *cr[kMaxLevels], *cz[kMaxLevels], *cn[kMaxLevels], *cnp;   // gate coefficients: fp32 engine
   __nv_bfloat16 *crb[kMaxLevels], *czb[kMaxLevels], *cnb[kMaxLevels], *cnpb;       // ... tensor-core engine (bf16)
-  float *dA_h, *dA_i; double* res_acc; UmmaAdjWs um;
+  float *dA_h, *dA_i, *lam_tmp; double* res_acc; UmmaAdjWs um;
   __nv_bfloat16* chain_dAb; unsigned* chain_bar;
 };
 
@@ -147,7 +153,7 @@ void plan_adj(const mgrit_gru_cfg* c, const Hier& hr, Ws& w, AdjWs* o) {
   else { o->cnpb = nullptr; o->cnp = w.take<float>((size_t)hr.N[0] * BH); }
   o->res_acc = w.take<double>((size_t)(c->iters > 0 ? c->iters : 1));
   if (c->operands == MGRIT_OPERANDS_BF16) {
-    o->dA_h = o->dA_i = nullptr;
+    o->dA_h = o->dA_i = o->lam_tmp = nullptr;
     umma_plan_adj(c, hr.N, hr.L, w.base, &w.off, &o->um);
     o->chain_dAb = w.take<__nv_bfloat16>(6 * BH);
     o->chain_bar = w.take<unsigned>(((size_t)c->B / 16 + 1) * ((size_t)c->H / 8) + 64);
@@ -155,6 +161,7 @@ void plan_adj(const mgrit_gru_cfg* c, const Hier& hr, Ws& w, AdjWs* o) {
     o->chain_dAb = nullptr; o->chain_bar = nullptr;
     o->dA_h = w.take<float>((size_t)c->T * BH * 3);
     o->dA_i = w.take<float>((size_t)c->T * BH * 3);
+    o->lam_tmp = w.take<float>((size_t)c->T * BH);     // lambda in forward order when the caller wants no dh
   }
 }
 
@@ -175,7 +182,12 @@ struct Cycle {
   float** U; float** G; double* res_acc; int cycle_idx = 0;
   __nv_bfloat16** Ub = nullptr;   // optional bf16 copies of U (kept in step with every writer)
   size_t BH;
-  virtual void step(const StepDesc& d) = 0;
+  int rc = MGRIT_OK;              // first failure of a launch (a step that cannot be prepared or launched)
+  virtual int launch_step(const StepDesc& d) = 0;
+  void step(const StepDesc& d) {
+    if (rc != MGRIT_OK) return;   // after a failure nothing more is enqueued: outputs are undefined
+    rc = launch_step(d);
+  }
   // all N_l dependent steps of level l in one persistent launch; false = not available here
   virtual bool chain(int l) { (void)l; return false; }
   virtual ~Cycle() {}
@@ -212,10 +224,11 @@ struct Cycle {
     stream_correct(U[l], Ub ? Ub[l] : nullptr, cf, U[l + 1], nc, (i64)BH, s);
     frelax(l);
   }
-  void solve() {
-    if (hr.L == 1) { vcycle(0); return; }
+  int solve() {
+    if (hr.L == 1) { vcycle(0); return rc; }
     cudaMemsetAsync(res_acc, 0, sizeof(double) * (size_t)(c->iters > 0 ? c->iters : 1), s);
-    for (cycle_idx = 0; cycle_idx < c->iters; ++cycle_idx) vcycle(0);
+    for (cycle_idx = 0; cycle_idx < c->iters && rc == MGRIT_OK; ++cycle_idx) vcycle(0);
+    return rc;
   }
 };
 
@@ -231,7 +244,7 @@ struct FwdCycle : Cycle {
     a.g = G[l]; a.W = um->W_hh; a.b_hh = p->b_hh; a.gamma = hr.gamma[l]; a.cell = c->cell; a.bar = fw->chain_bar;
     return serial_fwd_solve(a, s);
   }
-  void step(const StepDesc& d) override {
+  int launch_step(const StepDesc& d) override {
     FwdStepArgs a;
     a.M = d.nk * c->B; a.B = c->B; a.H = c->H;
     a.hin = U[d.l] + (size_t)d.in_slot * BH; a.hin_ks = (i64)d.in_stride * BH;
@@ -242,7 +255,9 @@ struct FwdCycle : Cycle {
     a.gi = gi + ((i64)st * d.tgt_slot - 1) * (i64)BH * 3; a.gi_ks = st * d.tgt_stride * (i64)BH * 3;
     a.gadd = d.gadd ? d.gadd + (size_t)d.gadd_slot * BH : nullptr; a.gadd_ks = (i64)d.gadd_stride * BH;
     a.W_hh = p->W_hh; a.b_hh = p->b_hh; a.gamma = hr.gamma[d.l]; a.cell = c->cell; a.mode = d.mode;
-    if (c->operands == MGRIT_OPERANDS_BF16) umma_fwd_step(a, um, s); else simt_fwd_step(a, s);
+    if (c->operands == MGRIT_OPERANDS_BF16) return umma_fwd_step(a, um, s);
+    simt_fwd_step(a, s);
+    return MGRIT_OK;
   }
 };
 
@@ -259,7 +274,7 @@ struct AdjCycle : Cycle {
     a.g = G[l]; a.WT = w->um.W_hhT; a.bar = w->chain_bar;
     return serial_adj_solve(a, s);
   }
-  void step(const StepDesc& d) override {
+  int launch_step(const StepDesc& d) override {
     AdjStepArgs a;
     a.M = d.nk * c->B; a.B = c->B; a.H = c->H;
     a.lin = U[d.l] + (size_t)d.in_slot * BH; a.lin_ks = (i64)d.in_stride * BH;
@@ -277,7 +292,9 @@ struct AdjCycle : Cycle {
     }
     a.coef_ks = -(i64)d.tgt_stride * BH;
     a.W_hh = p->W_hh; a.mode = d.mode;
-    if (c->operands == MGRIT_OPERANDS_BF16) umma_adj_step(a, &w->um, s); else simt_adj_step(a, s);
+    if (c->operands == MGRIT_OPERANDS_BF16) return umma_adj_step(a, &w->um, s);
+    simt_adj_step(a, s);
+    return MGRIT_OK;
   }
 };
 
@@ -333,7 +350,8 @@ int forward_impl(const mgrit_gru_cfg* cfg_in, bool serial, const gru_params* p, 
   cy.c = &c; cy.hr = hr; cy.s = s; cy.U = fw.U; cy.G = fw.G; cy.res_acc = fw.res_acc; cy.BH = BH;
   cy.p = p; cy.gi = gi; cy.um = &fw.um; cy.fw = &fw;
   cy.Ub = shadows ? fw.Ub : nullptr;
-  cy.solve();
+  rc = cy.solve();
+  if (rc) return rc;
   cudaMemcpyAsync(h, fw.U[0] + BH, sizeof(float) * (size_t)c.T * BH, cudaMemcpyDeviceToDevice, s);
   if (resnorm && hr.L > 1 && c.iters > 0) {
     rc = fetch_resnorm(fw.res_acc, resnorm, c.iters, s);
@@ -346,7 +364,7 @@ int forward_impl(const mgrit_gru_cfg* cfg_in, bool serial, const gru_params* p, 
 int adjoint_impl(const mgrit_gru_cfg* cfg_in, bool serial, const gru_params* p, const float* x, const float* h0,
                  const float* gi, const float* h, const float* dh_seed, const float* dhT, float* dh, float* dh0, float* dx,
                  const gru_grads* g, float* resnorm, void* ws, size_t ws_bytes, cudaStream_t s) {
-  if (!cfg_in || !p || !x || !h0 || !gi || !h || !dh || !dh0 || !g || !ws) return MGRIT_INVALID_ARG;
+  if (!cfg_in || !p || !x || !h0 || !gi || !h || !dh0 || !g || !ws) return MGRIT_INVALID_ARG;
   if (!dh_seed && !dhT) return MGRIT_INVALID_ARG;
   if (!p->W_ih || !p->W_hh || !p->b_ih || !p->b_hh || !g->dW_ih || !g->dW_hh || !g->db_ih || !g->db_hh) return MGRIT_INVALID_ARG;
   if (!aligned32(x, h0, gi, h, dh_seed, dhT, dh, dh0, dx, ws, p->W_ih, p->W_hh, p->b_ih, p->b_hh, g->dW_ih, g->dW_hh, g->db_ih, g->db_hh))
@@ -375,7 +393,12 @@ int adjoint_impl(const mgrit_gru_cfg* cfg_in, bool serial, const gru_params* p, 
     a.W_hh = p->W_hh; a.b_hh = p->b_hh; a.gamma = hr.gamma[l]; a.cell = c.cell;
     a.a = aw.a[l]; a.cr = aw.cr[l]; a.cz = aw.cz[l]; a.cn = aw.cn[l]; a.cnp = l == 0 ? aw.cnp : nullptr;
     a.crb = aw.crb[l]; a.czb = aw.czb[l]; a.cnb = aw.cnb[l]; a.cnpb = l == 0 ? aw.cnpb : nullptr;
-    if (bf16) umma_linearise(a, &aw.um, s); else simt_linearise(a, s);
+    if (bf16) {
+      rc = umma_linearise(a, &aw.um, s);
+      if (rc) return rc;
+    } else {
+      simt_linearise(a, s);
+    }
   }
   // mu_0 = lambda_T; zero initial guess elsewhere; fine-level source = reversed dh_seed
   cudaMemsetAsync(aw.U[0], 0, sizeof(float) * (size_t)(T + 1) * BH, s);
@@ -396,19 +419,27 @@ int adjoint_impl(const mgrit_gru_cfg* cfg_in, bool serial, const gru_params* p, 
   AdjCycle cy;
   cy.c = &c; cy.hr = hr; cy.s = s; cy.U = aw.U; cy.G = Gl; cy.res_acc = aw.res_acc; cy.BH = BH;
   cy.p = p; cy.w = &aw;
-  cy.solve();
+  rc = cy.solve();
+  if (rc) return rc;
 
-  // dh[k] = lambda_{k+1} = mu_{T-1-k};  dh0 = lambda_0 = mu_T
-  stream_gather_rows(dh, (i64)BH, aw.U[0] + (size_t)(T - 1) * BH, -(i64)BH, T, (i64)BH, s);
+  // dh[k] = lambda_{k+1} = mu_{T-1-k} (optional output);  dh0 = lambda_0 = mu_T
+  if (dh) stream_gather_rows(dh, (i64)BH, aw.U[0] + (size_t)(T - 1) * BH, -(i64)BH, T, (i64)BH, s);
   cudaMemcpyAsync(dh0, aw.U[0] + (size_t)T * BH, sizeof(float) * BH, cudaMemcpyDeviceToDevice, s);
 
   // gradient pass g = w * dh/dTheta over all fine steps at once
   if (bf16) {
-    rc = umma_gradients(&c, p, x, h0, h, dh, aw.crb[0], aw.czb[0], aw.cnb[0], aw.cnpb, dx, g, &aw.um, s);
+    // lambda_{t+1} for t = 0..T-1 is read in place from the reversed unknowns (row stride -B*H)
+    rc = umma_gradients(&c, p, x, h0, h, aw.U[0] + (size_t)(T - 1) * BH, -(i64)BH, aw.crb[0], aw.czb[0], aw.cnb[0], aw.cnpb, dx, g,
+                        &aw.um, s);
     if (rc) return rc;
   } else {
     i64 M = (i64)T * c.B;
-    stream_form_dA(dh, aw.cr[0], aw.cz[0], aw.cn[0], aw.cnp, aw.dA_h, aw.dA_i, M, c.H, s);
+    const float* lam = dh;
+    if (!lam) {   // no dh output requested: gather lambda in forward order into workspace scratch
+      lam = aw.lam_tmp;
+      stream_gather_rows(aw.lam_tmp, (i64)BH, aw.U[0] + (size_t)(T - 1) * BH, -(i64)BH, T, (i64)BH, s);
+    }
+    stream_form_dA(lam, aw.cr[0], aw.cz[0], aw.cn[0], aw.cnp, aw.dA_h, aw.dA_i, M, c.H, s);
     simt_wgrad(aw.dA_h, (int)M, 3 * c.H, h0, c.B, h, c.H, g->dW_hh, s);
     simt_wgrad(aw.dA_i, (int)M, 3 * c.H, nullptr, 0, x, c.I, g->dW_ih, s);
     stream_colsum(aw.dA_h, M, 3 * c.H, g->db_hh, s);
@@ -498,7 +529,7 @@ int gru_serial_backward(const mgrit_gru_cfg* cfg, const gru_params* p, const flo
 
 size_t xent_head_workspace_bytes(int32_t B, int32_t C) {
   if (B <= 0 || C <= 0) return 0;
-  return (((size_t)B * C * sizeof(float)) + 255) & ~(size_t)255;
+  return ((((size_t)B * C + (size_t)B) * sizeof(float)) + 255) & ~(size_t)255;     // dlogits [B, C] + per-row loss terms [B]
 }
 
 int xent_head_fwd_bwd(int32_t B, int32_t H, int32_t C, const float* hT, const float* Wc, const float* bc, const int32_t* labels,
@@ -532,11 +563,17 @@ int mgrit_gru_last_device_status(void) {
   return (umma_device_status() != 0 || serial_device_status() != 0) ? MGRIT_DEVICE_TIMEOUT : MGRIT_OK;
 }
 
-unsigned long long mgrit_gru_kernel_launches(void) { return g_kernel_launches; }
+int mgrit_gru_clear_device_status(void) {
+  if (cudaDeviceSynchronize() != cudaSuccess) return MGRIT_CUDA_ERROR;
+  return (umma_clear_device_status() == 0 && serial_clear_device_status() == 0) ? MGRIT_OK : MGRIT_CUDA_ERROR;
+}
+
+unsigned long long mgrit_gru_kernel_launches(void) { return g_kernel_launches.load(std::memory_order_relaxed); }
 
 int mgrit_gru_profile_enable(int on) {
   for (auto& r : g_prof_recs) { g_prof_pool.push_back(r.e0); g_prof_pool.push_back(r.e1); }
   g_prof_recs.clear();
+  g_prof_depth = 0;
   g_prof_on = on != 0;
   return MGRIT_OK;
 }
@@ -577,10 +614,10 @@ const char* mgrit_gru_strerror(int code) {
     case MGRIT_INVALID_ARG: return "invalid argument";
     case MGRIT_NOT_DIVISIBLE: return "T is not divisible by cf^(levels-1)";
     case MGRIT_WORKSPACE_TOO_SMALL: return "workspace too small";
-    case MGRIT_UNSUPPORTED: return "shape not supported by the selected operand mode";
+    case MGRIT_UNSUPPORTED: return "shape not supported (operand mode limits, C > 8192 in the loss head, or sizes beyond 32-bit row counts)";
     case MGRIT_CUDA_ERROR: return "CUDA error";
     case MGRIT_DEVICE_TIMEOUT: return "a bounded device-side wait ran out";
-    case MGRIT_SCRATCH_LIMIT: return "problem exceeds the built-in scratch of the no-allocation entry point (B*C <= 65536)";
+    case MGRIT_SCRATCH_LIMIT: return "problem exceeds the built-in scratch of the no-allocation entry point (B*(C+1) <= 65536)";
     default: return "unknown error";
   }
 }

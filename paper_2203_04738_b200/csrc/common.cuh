@@ -2,6 +2,8 @@
 #pragma once
 #include <cuda_runtime.h>
 #include <cuda_bf16.h>
+
+#include <atomic>
 #include <stdint.h>
 #include <stddef.h>
 
@@ -12,8 +14,29 @@ namespace mg {
 typedef long long i64;
 
 // Every launch goes through this counter (reported by mgrit_gru_kernel_launches()).
-extern unsigned long long g_kernel_launches;
-inline void count_launch(int n = 1) { g_kernel_launches += (unsigned long long)n; }
+extern std::atomic<unsigned long long> g_kernel_launches;
+inline void count_launch(int n = 1) { g_kernel_launches.fetch_add((unsigned long long)n, std::memory_order_relaxed); }
+
+// Host-side caches that depend on the device (addresses of __device__ variables, function attributes, SM
+// count) are kept per device ordinal and filled on the first call made with that device current.
+constexpr int kMaxDevices = 64;
+// ordinal of the current device, or -1 (no device / more than kMaxDevices)
+inline int current_device_slot() {
+  int dev = -1;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) return -1;
+  return dev;
+}
+// cudaFuncSetAttribute(MaxDynamicSharedMemorySize) once per (kernel instantiation, device); `done` is the
+// instantiation's own per-device flag array
+template <class K>
+inline bool set_smem_once(K kern, int bytes, bool (&done)[kMaxDevices]) {
+  const int dev = current_device_slot();
+  if (dev < 0) return false;
+  if (done[dev]) return true;
+  if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes) != cudaSuccess) return false;
+  done[dev] = true;
+  return true;
+}
 
 // Programmatic dependent launch: a kernel launched through launch_pdl() may become resident (and run its
 // prologue: barrier set-up, TMEM allocation, descriptor prefetch) while its predecessor in the stream is
@@ -50,8 +73,16 @@ inline cudaError_t launch_pdl(void (*kern)(KArgs...), dim3 grid, dim3 block, siz
 // Optional per-launch timing of the GEMM-shaped kernels (CUDA events on the launching stream).
 enum KernelClass { KC_PROJ = 0, KC_FWD_STEP, KC_LINEARISE, KC_ADJ_STEP, KC_WGRAD, KC_FWD_SERIAL, KC_ADJ_SERIAL, KC_COUNT };
 extern bool g_prof_on;
+// prof_begin/prof_end bracket one record; records do not nest: a begin issued while a record is open (a GEMM
+// launcher called from a function that times itself together with its operand-forming kernels) is ignored
+// together with its matching end.
 void prof_begin(int kc, double flops, cudaStream_t s);
 void prof_end(cudaStream_t s);
+struct ProfScope {
+  cudaStream_t s;
+  ProfScope(int kc, double flops, cudaStream_t st) : s(st) { prof_begin(kc, flops, st); }
+  ~ProfScope() { prof_end(s); }
+};
 
 // ---- one forward cell evaluation for M = nk*B rows (Eq. "gru" + Eq. "gru-classic"/"gru-imap") ----
 // Row m = (k, b): k = m / B, b = m % B.  All *_ks are strides per k in ELEMENTS (may be negative).

@@ -36,5 +36,6 @@ bool serial_adj_supported(int B, int H);
 bool serial_fwd_solve(const SerialFwdArgs& a, cudaStream_t s);
 bool serial_adj_solve(const SerialAdjArgs& a, cudaStream_t s);
 int serial_device_status();
+int serial_clear_device_status();
 
 }  // namespace mg

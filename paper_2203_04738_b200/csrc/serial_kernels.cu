@@ -19,7 +19,7 @@ constexpr int kThreads = 256, kWarps = 8, kRows = 16;
 constexpr uint64_t kWaitLimitNs = 2000000000ull;
 
 __device__ int g_serial_status = 0;
-int* g_serial_status_ptr = nullptr;
+int* g_serial_status_ptrs[kMaxDevices] = {nullptr};   // its address on each device
 
 __device__ __forceinline__ uint64_t global_ns() {
   uint64_t t;
@@ -310,20 +310,29 @@ __global__ void __launch_bounds__(kThreads, 1) serial_adj_kernel(SerialAdjArgs a
   }
 }
 
-bool ensure_status() {
-  if (g_serial_status_ptr) return true;
-  return cudaGetSymbolAddress((void**)&g_serial_status_ptr, g_serial_status) == cudaSuccess;
+int* status_ptr() {     // status word of the current device, nullptr on failure
+  const int dev = current_device_slot();
+  if (dev < 0) return nullptr;
+  if (!g_serial_status_ptrs[dev]) {
+    int* p = nullptr;
+    if (cudaGetSymbolAddress((void**)&p, g_serial_status) != cudaSuccess) { cudaGetLastError(); return nullptr; }
+    g_serial_status_ptrs[dev] = p;
+  }
+  return g_serial_status_ptrs[dev];
 }
 
 constexpr size_t kSmemLimit = 227 * 1024 - 64;
-int g_sm_count = 0;
+int g_sm_count[kMaxDevices] = {0};
 int sm_count() {
-  if (g_sm_count == 0) {
-    int dev = 0;
-    cudaGetDevice(&dev);
-    if (cudaDeviceGetAttribute(&g_sm_count, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || g_sm_count <= 0) g_sm_count = 148;
+  const int dev = current_device_slot();
+  if (dev < 0) return 148;
+  if (g_sm_count[dev] == 0) {
+    if (cudaDeviceGetAttribute(&g_sm_count[dev], cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || g_sm_count[dev] <= 0) {
+      cudaGetLastError();
+      g_sm_count[dev] = 148;
+    }
   }
-  return g_sm_count;
+  return g_sm_count[dev];
 }
 
 size_t fwd_smem(int unc, int H) { return (size_t)(3 * unc + kRows) * (H + 8) * 2 + (size_t)kWarps * kRows * 3 * unc * 4; }
@@ -350,7 +359,8 @@ bool launch_coop(Kern kern, const Args& a, int unc, size_t smem, cudaStream_t s)
   int rgs = (a.B + kRows - 1) / kRows;
   if (cudaMemsetAsync(a.bar, 0, sizeof(unsigned) * rgs, s) != cudaSuccess) return false;
   Args args = a;
-  int* st = g_serial_status_ptr;
+  int* st = status_ptr();
+  if (!st) return false;
   void* params[2] = {(void*)&args, (void*)&st};
   dim3 grid(a.H / unc, rgs);
   if (cudaLaunchCooperativeKernel((const void*)kern, grid, dim3(kThreads), params, smem, s) != cudaSuccess) {
@@ -368,7 +378,7 @@ bool serial_adj_supported(int B, int H) { return pick_unc(B, H, true) != 0; }
 
 bool serial_fwd_solve(const SerialFwdArgs& a, cudaStream_t s) {
   int unc = pick_unc(a.B, a.H, false);
-  if (unc == 0 || a.nsteps <= 0 || !ensure_status()) return false;
+  if (unc == 0 || a.nsteps <= 0 || !status_ptr()) return false;
   size_t smem = fwd_smem(unc, a.H);
   prof_begin(KC_FWD_SERIAL, 2.0 * a.B * 3.0 * a.H * a.H * a.nsteps, s);
   bool ok = unc == 8 ? launch_coop(serial_fwd_kernel<8>, a, unc, smem, s)
@@ -380,7 +390,7 @@ bool serial_fwd_solve(const SerialFwdArgs& a, cudaStream_t s) {
 
 bool serial_adj_solve(const SerialAdjArgs& a, cudaStream_t s) {
   int unc = pick_unc(a.B, a.H, true);
-  if (unc == 0 || a.nsteps <= 0 || !ensure_status()) return false;
+  if (unc == 0 || a.nsteps <= 0 || !status_ptr()) return false;
   size_t smem = adj_smem(unc, a.H);
   prof_begin(KC_ADJ_SERIAL, 2.0 * a.B * 3.0 * a.H * a.H * a.nsteps, s);
   bool ok = unc == 8 ? launch_coop(serial_adj_kernel<8>, a, unc, smem, s)
@@ -391,10 +401,19 @@ bool serial_adj_solve(const SerialAdjArgs& a, cudaStream_t s) {
 }
 
 int serial_device_status() {
-  if (!g_serial_status_ptr) return 0;
+  const int dev = current_device_slot();
+  if (dev < 0) return -1;
+  if (!g_serial_status_ptrs[dev]) return 0;     // no chain kernel has run on this device
   int v = 0;
-  if (cudaMemcpy(&v, g_serial_status_ptr, sizeof(int), cudaMemcpyDeviceToHost) != cudaSuccess) return -1;
+  if (cudaMemcpy(&v, g_serial_status_ptrs[dev], sizeof(int), cudaMemcpyDeviceToHost) != cudaSuccess) return -1;
   return v;
+}
+
+int serial_clear_device_status() {
+  const int dev = current_device_slot();
+  if (dev < 0) return -1;
+  if (!g_serial_status_ptrs[dev]) return 0;
+  return cudaMemset(g_serial_status_ptrs[dev], 0, sizeof(int)) == cudaSuccess ? 0 : -1;
 }
 
 }  // namespace mg

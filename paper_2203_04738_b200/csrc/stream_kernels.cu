@@ -135,10 +135,11 @@ __global__ void sqrt_to_float_kernel(const double* acc, float* out, int n) {
   if (i < n) out[i] = (float)sqrt(acc[i]);
 }
 
-// Classifier head, pass 1: one block per batch row: logits, softmax, loss term, dlogits = (p - onehot)/B.
+// Classifier head, pass 1: one block per batch row: logits, softmax, the row's loss term, dlogits = (p - onehot)/B.
+// A label outside [0, C) marks a row without a target: it adds nothing to the loss and its one-hot term is absent.
 __global__ void __launch_bounds__(kThreads) xent_rows_kernel(int B, int H, int C, const float* __restrict__ hT,
                                                              const float* __restrict__ Wc, const float* __restrict__ bc,
-                                                             const int32_t* __restrict__ labels, float* loss,
+                                                             const int32_t* __restrict__ labels, float* __restrict__ rowloss,
                                                              float* __restrict__ dlogits) {
   extern __shared__ float logit[];  // C floats
   int b = blockIdx.x;
@@ -158,23 +159,32 @@ __global__ void __launch_bounds__(kThreads) xent_rows_kernel(int B, int H, int C
     float se = 0.f;
     for (int c = lane; c < C; c += 32) se += __expf(logit[c] - mx);
     se = warp_sum(se);
-    int lab = labels[b];
+    const int lab = labels[b];
+    const bool has_label = lab >= 0 && lab < C;
     float invB = 1.0f / (float)B;
     for (int c = lane; c < C; c += 32) {
       float p = __expf(logit[c] - mx) / se;
       dlogits[(i64)b * C + c] = (p - (c == lab ? 1.f : 0.f)) * invB;
     }
-    if (lane == 0) atomicAdd(loss, -((logit[lab] - mx) - logf(se)) * invB);
+    if (lane == 0) rowloss[b] = has_label ? -((logit[lab] - mx) - logf(se)) * invB : 0.f;
   }
 }
 
-// pass 2: dhT = dlogits Wc ; dWc = dlogits^T hT ; dbc = column sums of dlogits.
+// pass 2: dhT = dlogits Wc ; dWc = dlogits^T hT ; dbc = column sums of dlogits ; loss = sum of the row terms in
+// row order (fixed order: the same bits on every run).
 __global__ void __launch_bounds__(kThreads) xent_grads_kernel(int B, int H, int C, const float* __restrict__ hT,
                                                               const float* __restrict__ Wc,
-                                                              const float* __restrict__ dlogits, float* __restrict__ dhT,
+                                                              const float* __restrict__ dlogits, const float* __restrict__ rowloss,
+                                                              float* __restrict__ loss, float* __restrict__ dhT,
                                                               float* __restrict__ dWc, float* __restrict__ dbc) {
   i64 nBH = (i64)B * H, nCH = (i64)C * H;
-  for (i64 e = (i64)blockIdx.x * blockDim.x + threadIdx.x; e < nBH + nCH + C; e += (i64)gridDim.x * blockDim.x) {
+  for (i64 e = (i64)blockIdx.x * blockDim.x + threadIdx.x; e < nBH + nCH + C + 1; e += (i64)gridDim.x * blockDim.x) {
+    if (e == nBH + nCH + C) {
+      float s = 0.f;
+      for (int b = 0; b < B; ++b) s += rowloss[b];
+      *loss = s;
+      continue;
+    }
     if (e < nBH) {
       int b = e / H, i = e % H;
       float s = 0.f;
@@ -280,9 +290,10 @@ void stream_sqrt_to_float(const double* acc, float* out, int n, cudaStream_t s) 
 
 void stream_xent(int B, int H, int C, const float* hT, const float* Wc, const float* bc, const int32_t* labels, float* loss,
                  float* dhT, float* dWc, float* dbc, float* dlogits, cudaStream_t s) {
-  cudaMemsetAsync(loss, 0, sizeof(float), s);
-  xent_rows_kernel<<<B, kThreads, (size_t)C * sizeof(float), s>>>(B, H, C, hT, Wc, bc, labels, loss, dlogits);
-  xent_grads_kernel<<<stream_grid((i64)B * H + (i64)C * H + C), kThreads, 0, s>>>(B, H, C, hT, Wc, dlogits, dhT, dWc, dbc);
+  float* rowloss = dlogits + (size_t)B * C;      // the scratch holds [B, C] derivatives followed by B row terms
+  xent_rows_kernel<<<B, kThreads, (size_t)C * sizeof(float), s>>>(B, H, C, hT, Wc, bc, labels, rowloss, dlogits);
+  xent_grads_kernel<<<stream_grid((i64)B * H + (i64)C * H + C + 1), kThreads, 0, s>>>(B, H, C, hT, Wc, dlogits, rowloss, loss, dhT, dWc,
+                                                                                     dbc);
   count_launch(2);
 }
 
@@ -300,13 +311,12 @@ void stream_sgd(float* p, const float* g, size_t n, float lr, cudaStream_t s) {
 // serving or training process that has handed the whole GPU to its own memory arena (cudaMalloc then
 // fails or fragments the arena), or a latency-critical loop that must not take the driver's allocator
 // lock, which can also synchronise the device.  For them the [B, C] buffer of loss derivatives with
-// respect to the logits lives in a fixed array inside the library image.  Every GPU that loads the
+// respect to the logits (and the B per-row loss terms) lives in a fixed array inside the library image.  Every GPU that loads the
 // library holds these 256 KiB until the process exits.
 namespace mg {
 namespace {
-constexpr size_t kHeadScratchFloats = 65536;   // B * C <= 65536
+constexpr size_t kHeadScratchFloats = 65536;   // B * (C + 1) <= 65536: [B, C] derivatives + B row loss terms
 static __device__ __align__(256) float g_head_scratch[kHeadScratchFloats];
-constexpr int kMaxDevices = 64;
 float* g_head_scratch_addr[kMaxDevices] = {nullptr};   // device address of the array, per device
 }  // namespace
 }  // namespace mg
@@ -317,9 +327,9 @@ extern "C" int xent_head_fwd_bwd_noalloc(int32_t B, int32_t H, int32_t C, const 
   using namespace mg;
   if (B <= 0 || H <= 0 || C <= 0 || !hT || !Wc || !bc || !labels || !loss || !dhT || !dWc || !dbc) return MGRIT_INVALID_ARG;
   if (C > 8192) return MGRIT_UNSUPPORTED;
-  if ((size_t)B * (size_t)C > kHeadScratchFloats) return MGRIT_SCRATCH_LIMIT;
-  int dev = -1;
-  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) return MGRIT_CUDA_ERROR;
+  if ((size_t)B * ((size_t)C + 1) > kHeadScratchFloats) return MGRIT_SCRATCH_LIMIT;
+  const int dev = current_device_slot();
+  if (dev < 0) return MGRIT_CUDA_ERROR;
   if (!g_head_scratch_addr[dev]) {
     // In host code the array's name is only a handle; the kernels need its address on the current device.
     float* p = nullptr;
@@ -329,8 +339,7 @@ extern "C" int xent_head_fwd_bwd_noalloc(int32_t B, int32_t H, int32_t C, const 
     }
     g_head_scratch_addr[dev] = p;
   }
-  // Nothing in the scratch has to start at zero: pass 1 overwrites all B*C entries before pass 2 reads them
-  // (the loss accumulator is the caller's `loss`, cleared inside stream_xent).
+  // Nothing in the scratch has to start at zero: pass 1 overwrites all B*C + B entries before pass 2 reads them.
   stream_xent(B, H, C, hT, Wc, bc, labels, loss, dhT, dWc, dbc, g_head_scratch_addr[dev], (cudaStream_t)stream);
   return cudaGetLastError() == cudaSuccess ? MGRIT_OK : MGRIT_CUDA_ERROR;
 }

@@ -17,7 +17,7 @@ using namespace umma;
 typedef __nv_bfloat16 bf16;
 
 __device__ int g_umma_status = 0;   // first error code of a bounded wait that ran out (0 = none)
-int* g_status_ptr = nullptr;
+int* g_status_ptrs[kMaxDevices] = {nullptr};   // its address on each device
 
 constexpr int kSMs = 148;
 
@@ -27,18 +27,27 @@ typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t,
                                   CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
 EncodeTiledFn g_encode = nullptr;
 
-bool ensure_driver() {
-  if (g_encode && g_status_ptr) return true;
+// Status word of the current device (nullptr on failure); also resolves the tensor-map encoder.
+// MGRIT_GRU_TEST_FAIL_ENCODE=1 in the environment makes this fail, so that the error path of a launch that
+// cannot be prepared can be exercised from the host without launching anything.
+int* status_ptr() {
+  static int fail = -1;
+  if (fail < 0) { const char* e = getenv("MGRIT_GRU_TEST_FAIL_ENCODE"); fail = (e && e[0] == '1') ? 1 : 0; }
+  if (fail) return nullptr;
   if (!g_encode) {
     void* fn = nullptr;
     cudaDriverEntryPointQueryResult q;
-    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &fn, cudaEnableDefault, &q) != cudaSuccess || !fn) return false;
+    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &fn, cudaEnableDefault, &q) != cudaSuccess || !fn) return nullptr;
     g_encode = (EncodeTiledFn)fn;
   }
-  if (!g_status_ptr) {
-    if (cudaGetSymbolAddress((void**)&g_status_ptr, g_umma_status) != cudaSuccess) return false;
+  const int dev = current_device_slot();
+  if (dev < 0) return nullptr;
+  if (!g_status_ptrs[dev]) {
+    int* p = nullptr;
+    if (cudaGetSymbolAddress((void**)&p, g_umma_status) != cudaSuccess) { cudaGetLastError(); return nullptr; }
+    g_status_ptrs[dev] = p;
   }
-  return true;
+  return g_status_ptrs[dev];
 }
 
 // bf16 matrix [rows, inner] with row pitch `pitch` elements; box = 64 x box_rows, 128-byte swizzle
@@ -59,13 +68,11 @@ bool launch_gemm(int kc, const bf16* A, i64 lda, const bf16* Bm, i64 ldb, int M,
                  cudaStream_t s) {
   using C = Cfg<BN, GATES>;
   if (M <= 0 || N <= 0) return true;
-  if (!ensure_driver()) return false;
-  static bool attr_set = false;
+  int* const status = status_ptr();
+  if (!status) return false;
+  static bool attr_set[kMaxDevices] = {false};
   auto kern = umma_gemm_kernel<BN, GATES, Epi>;
-  if (!attr_set) {
-    if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, C::kSmemBytes) != cudaSuccess) return false;
-    attr_set = true;
-  }
+  if (!set_smem_once(kern, C::kSmemBytes, attr_set)) return false;
   CUtensorMap ta, tb;
   if (!make_map(&ta, A, (uint64_t)K, (uint64_t)M, (uint64_t)lda, BM)) return false;
   if (!make_map(&tb, Bm, (uint64_t)K, (uint64_t)b_rows, (uint64_t)ldb, GATES ? BN / 3 : BN)) return false;
@@ -73,9 +80,8 @@ bool launch_gemm(int kc, const bf16* A, i64 lda, const bf16* Bm, i64 ldb, int M,
   int m_tiles = (M + BM - 1) / BM, n_tiles = (N + C::kNPerTile - 1) / C::kNPerTile;
   int tiles = m_tiles * n_tiles;
   int grid = tiles < kSMs ? tiles : kSMs;
-  prof_begin(kc, 2.0 * M * (GATES ? 3.0 * N : (double)N) * K, s);
-  if (launch_pdl(kern, dim3(grid), dim3(kThreads), C::kSmemBytes, s, ta, tb, sh, epi, g_status_ptr) != cudaSuccess) return false;
-  prof_end(s);
+  ProfScope prof_(kc, 2.0 * M * (GATES ? 3.0 * N : (double)N) * K, s);
+  if (launch_pdl(kern, dim3(grid), dim3(kThreads), C::kSmemBytes, s, ta, tb, sh, epi, status) != cudaSuccess) return false;
   count_launch();
   return true;
 }
@@ -91,23 +97,20 @@ static bool gemm_pair_enabled(int M, int N) {
 template <class Epi>
 bool launch_gemm_pair(int kc, const bf16* A, i64 lda, const bf16* Bm, i64 ldb, int M, int N, int K, int b_rows, Epi epi, cudaStream_t s) {
   if (M <= 0 || N <= 0) return true;
-  if (!ensure_driver()) return false;
-  static bool attr_set = false;
+  int* const status = status_ptr();
+  if (!status) return false;
+  static bool attr_set[kMaxDevices] = {false};
   auto kern = umma_gemm_pair_kernel<Epi>;
-  if (!attr_set) {
-    if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, pairk::kSmemBytes) != cudaSuccess) return false;
-    attr_set = true;
-  }
+  if (!set_smem_once(kern, pairk::kSmemBytes, attr_set)) return false;
   CUtensorMap ta, tb;
   if (!make_map(&ta, A, (uint64_t)K, (uint64_t)M, (uint64_t)lda, BM)) return false;
   if (!make_map(&tb, Bm, (uint64_t)K, (uint64_t)b_rows, (uint64_t)ldb, pairk::BN / 2)) return false;
   GemmShape sh{M, N, K, 0};
   int tiles = ((M + 2 * BM - 1) / (2 * BM)) * ((N + pairk::BN - 1) / pairk::BN);
   int grid = 2 * (tiles < kSMs / 2 ? tiles : kSMs / 2);
-  prof_begin(kc, 2.0 * M * (double)N * K, s);
-  if (launch_pdl_cluster(kern, 2, dim3(grid), dim3(kThreads), pairk::kSmemBytes, s, ta, tb, sh, epi, g_status_ptr) != cudaSuccess)
+  ProfScope prof_(kc, 2.0 * M * (double)N * K, s);
+  if (launch_pdl_cluster(kern, 2, dim3(grid), dim3(kThreads), pairk::kSmemBytes, s, ta, tb, sh, epi, status) != cudaSuccess)
     return false;
-  prof_end(s);
   count_launch();
   return true;
 }
@@ -120,13 +123,11 @@ bool launch_gemm_mn(int kc, const bf16* A, i64 lda, int Mdim, const bf16* Bm, i6
                     cudaStream_t s) {
   using C = Cfg<256, false>;
   if (Mdim <= 0 || Ndim <= 0) return true;
-  if (!ensure_driver()) return false;
-  static bool attr_set = false;
+  int* const status = status_ptr();
+  if (!status) return false;
+  static bool attr_set[kMaxDevices] = {false};
   auto kern = umma_gemm_kernel<256, false, Epi, true>;
-  if (!attr_set) {
-    if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, C::kSmemBytes) != cudaSuccess) return false;
-    attr_set = true;
-  }
+  if (!set_smem_once(kern, C::kSmemBytes, attr_set)) return false;
   CUtensorMap ta, tb;
   if (!make_map(&ta, A, (uint64_t)Mdim, (uint64_t)K, (uint64_t)lda, 64)) return false;
   if (!make_map(&tb, Bm, (uint64_t)Ndim, (uint64_t)K, (uint64_t)ldb, 64)) return false;
@@ -135,9 +136,8 @@ bool launch_gemm_mn(int kc, const bf16* A, i64 lda, int Mdim, const bf16* Bm, i6
   GemmShape sh{Mdim, Ndim, K, 0, splits, (k_blocks + splits - 1) / splits};
   int tiles = ((Mdim + BM - 1) / BM) * ((Ndim + 255) / 256) * splits;
   int grid = tiles < kSMs ? tiles : kSMs;
-  prof_begin(kc, 2.0 * Mdim * (double)Ndim * K, s);
-  if (launch_pdl(kern, dim3(grid), dim3(kThreads), C::kSmemBytes, s, ta, tb, sh, epi, g_status_ptr) != cudaSuccess) return false;
-  prof_end(s);
+  ProfScope prof_(kc, 2.0 * Mdim * (double)Ndim * K, s);
+  if (launch_pdl(kern, dim3(grid), dim3(kThreads), C::kSmemBytes, s, ta, tb, sh, epi, status) != cudaSuccess) return false;
   count_launch();
   return true;
 }
@@ -177,13 +177,11 @@ bool launch_cell(int kc, const bf16* A, i64 a_ks, const float* gi, i64 gi_ks, co
                  int nk, const bf16* W, CellArgs ca, cudaStream_t s) {
   using C = cellk::CellCfg<HAS_G, LIN>;
   if (nk <= 0) return true;
-  if (!ensure_driver()) return false;
-  static bool attr_set = false;
+  int* const status = status_ptr();
+  if (!status) return false;
+  static bool attr_set[kMaxDevices] = {false};
   auto kern = umma_cell_kernel<LIN, HAS_G>;
-  if (!attr_set) {
-    if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, C::kSmemBytes) != cudaSuccess) return false;
-    attr_set = true;
-  }
+  if (!set_smem_once(kern, C::kSmemBytes, attr_set)) return false;
   const int B = ca.B, H = ca.H, kt = 128 / B;
   ca.kt = kt; ca.M = nk * B;
   CUtensorMap ta, tb, tgi, thp, tg;
@@ -206,9 +204,8 @@ bool launch_cell(int kc, const bf16* A, i64 a_ks, const float* gi, i64 gi_ks, co
   }
   int tiles = ((ca.M + BM - 1) / BM) * (H / cellk::UN);
   int grid = tiles < kSMs ? tiles : kSMs;
-  prof_begin(kc, 2.0 * ca.M * 3.0 * H * H, s);
-  if (launch_pdl(kern, dim3(grid), dim3(cellk::kThreads), C::kSmemBytes, s, ta, tb, tgi, thp, tg, tcr, tcz, tcn, tcp, ca, g_status_ptr) != cudaSuccess) return false;
-  prof_end(s);
+  ProfScope prof_(kc, 2.0 * ca.M * 3.0 * H * H, s);
+  if (launch_pdl(kern, dim3(grid), dim3(cellk::kThreads), C::kSmemBytes, s, ta, tb, tgi, thp, tg, tcr, tcz, tcn, tcp, ca, status) != cudaSuccess) return false;
   count_launch();
   return true;
 }
@@ -505,13 +502,14 @@ __global__ void __launch_bounds__(1024) transpose_kernel(const float* __restrict
   if (rr < R && cc < C) dst[(i64)cc * dst_ld + col0 + rr] = __float2bfloat16(tile[threadIdx.x][threadIdx.y]);
 }
 
-// Gradient-pass operands, row-major: dA_h = [cr|cz|cn]*lam and dA_i = [cr|cz|cnp]*lam as bf16 [M, 3H], plus the
-// fp32 column sums (bias gradients) added into db_hh / db_ih.  Block = 32 float4 columns (128 units) x 8 rows.
-__global__ void __launch_bounds__(256) form_dA_rows_kernel(const float* __restrict__ lam, const bf16* __restrict__ cr,
+// Gradient-pass operands, row-major: dA_h = [cr|cz|cn]*lam and dA_i = [cr|cz|cnp]*lam as bf16 [M, 3H], plus this
+// block's fp32 column sums of the four products (bias-gradient partials) to part[blockIdx.x][4][H].
+// Row m = (t, b): lam row at lam + t*lam_ts + b*H (lam_ts may be negative: the adjoint keeps its unknowns in
+// reversed time order).  Block = 32 float4 columns (128 units) x 8 rows at a time.
+__global__ void __launch_bounds__(256) form_dA_rows_kernel(const float* __restrict__ lam, i64 lam_ts, int B, const bf16* __restrict__ cr,
                                                            const bf16* __restrict__ cz, const bf16* __restrict__ cn,
                                                            const bf16* __restrict__ cnp, i64 M, int H, uint2* __restrict__ dAh,
-                                                           uint2* __restrict__ dAi, float* __restrict__ db_hh,
-                                                           float* __restrict__ db_ih, int rows_per_block) {
+                                                           uint2* __restrict__ dAi, float* __restrict__ part, int rows_per_block) {
   __shared__ float red[4][8][128];
   const int tx = threadIdx.x & 31, ty = threadIdx.x >> 5;
   const int H4 = H / 4, c4 = blockIdx.y * 32 + tx;
@@ -522,7 +520,8 @@ __global__ void __launch_bounds__(256) form_dA_rows_kernel(const float* __restri
   if (c4 < H4) {
     for (i64 m = m0 + ty; m < m0 + rows_per_block && m < M; m += 8) {
       i64 e = m * H4 + c4;
-      float4 l = reinterpret_cast<const float4*>(lam)[e];
+      const i64 t = m / B; const int bb = (int)(m % B);
+      float4 l = *reinterpret_cast<const float4*>(lam + t * lam_ts + ((i64)bb * H4 + c4) * 4);
       float4 r = unpack4(reinterpret_cast<const uint2*>(cr)[e]), z = unpack4(reinterpret_cast<const uint2*>(cz)[e]);
       float4 n = unpack4(reinterpret_cast<const uint2*>(cn)[e]), q = unpack4(reinterpret_cast<const uint2*>(cnp)[e]);
       float4 v[4] = {make_float4(r.x * l.x, r.y * l.y, r.z * l.z, r.w * l.w), make_float4(z.x * l.x, z.y * l.y, z.z * l.z, z.w * l.w),
@@ -548,10 +547,22 @@ __global__ void __launch_bounds__(256) form_dA_rows_kernel(const float* __restri
     float acc = 0.f;
 #pragma unroll
     for (int r = 0; r < 8; ++r) acc += red[g][r][u];
-    if (g == 0) { atomicAdd(db_hh + col, acc); atomicAdd(db_ih + col, acc); }
-    else if (g == 1) { atomicAdd(db_hh + H + col, acc); atomicAdd(db_ih + H + col, acc); }
-    else if (g == 2) atomicAdd(db_hh + 2 * H + col, acc);
-    else atomicAdd(db_ih + 2 * H + col, acc);
+    part[((i64)blockIdx.x * 4 + g) * H + col] = acc;
+  }
+}
+
+// Bias gradients from the per-block partials, summed in block order (the same bits on every run):
+// db_hh = [sum cr*lam | sum cz*lam | sum cn*lam],  db_ih = [sum cr*lam | sum cz*lam | sum cnp*lam].
+__global__ void __launch_bounds__(kPT) sum_db_kernel(const float* __restrict__ part, int nblk, int H, float* __restrict__ db_hh,
+                                                     float* __restrict__ db_ih) {
+  for (int e = blockIdx.x * blockDim.x + threadIdx.x; e < 4 * H; e += gridDim.x * blockDim.x) {
+    const int g = e / H, col = e % H;
+    float acc = 0.f;
+    for (int k = 0; k < nblk; ++k) acc += part[((i64)k * 4 + g) * H + col];
+    if (g == 0) { db_hh[col] = acc; db_ih[col] = acc; }
+    else if (g == 1) { db_hh[H + col] = acc; db_ih[H + col] = acc; }
+    else if (g == 2) db_hh[2 * H + col] = acc;
+    else db_ih[2 * H + col] = acc;
   }
 }
 
@@ -633,27 +644,31 @@ int umma_prepare_adj(const mgrit_gru_cfg* c, const gru_params* p, const float* h
   convert(h, w->hb, (i64)c->T * c->B * H, s);
   transpose(p->W_hh, 3 * H, H, w->W_hhT, 3 * H, 0, s);   // [H, 3H]
   transpose(p->W_ih, 3 * H, I, w->W_ihT, 3 * H, 0, s);   // [I, 3H]
-  return ensure_driver() ? MGRIT_OK : MGRIT_CUDA_ERROR;
+  return status_ptr() ? MGRIT_OK : MGRIT_CUDA_ERROR;
 }
 
-void umma_fwd_step(const FwdStepArgs& a, UmmaFwdWs* w, cudaStream_t s) {
+int umma_fwd_step(const FwdStepArgs& a, UmmaFwdWs* w, cudaStream_t s) {
+  bool ok;
   if (a.hin_b && 128 % a.B == 0) {
     // operands through strided tensor maps, bf16 copy of the new state written by the epilogue
     CellArgs ca{};
     ca.B = a.B; ca.H = a.H; ca.hout = a.hout; ca.hout_ks = a.hout_ks; ca.hout_b = a.hout_b;
     ca.b_hh = a.b_hh; ca.gamma = a.gamma; ca.cell = a.cell; ca.mode = a.mode;
     const int nk = a.M / a.B;
-    if (a.mode == 1) launch_cell<false, true>(KC_FWD_STEP, a.hin_b, a.hin_ks, a.gi, a.gi_ks, a.hin, a.hin_ks, a.hout, a.hout_ks, nk, w->W_hh, ca, s);
-    else if (a.gadd) launch_cell<false, true>(KC_FWD_STEP, a.hin_b, a.hin_ks, a.gi, a.gi_ks, a.hin, a.hin_ks, a.gadd, a.gadd_ks, nk, w->W_hh, ca, s);
-    else launch_cell<false, false>(KC_FWD_STEP, a.hin_b, a.hin_ks, a.gi, a.gi_ks, a.hin, a.hin_ks, nullptr, 0, nk, w->W_hh, ca, s);
-    return;
+    if (a.mode == 1) ok = launch_cell<false, true>(KC_FWD_STEP, a.hin_b, a.hin_ks, a.gi, a.gi_ks, a.hin, a.hin_ks, a.hout, a.hout_ks, nk, w->W_hh, ca, s);
+    else if (a.gadd) ok = launch_cell<false, true>(KC_FWD_STEP, a.hin_b, a.hin_ks, a.gi, a.gi_ks, a.hin, a.hin_ks, a.gadd, a.gadd_ks, nk, w->W_hh, ca, s);
+    else ok = launch_cell<false, false>(KC_FWD_STEP, a.hin_b, a.hin_ks, a.gi, a.gi_ks, a.hin, a.hin_ks, nullptr, 0, nk, w->W_hh, ca, s);
+    return ok ? MGRIT_OK : MGRIT_CUDA_ERROR;
   }
-  launch_pdl(pack_rows_kernel, dim3(pgrid((i64)a.M * (a.H / 4))), dim3(kPT), 0, s, a.hin, a.hin_ks, a.B, a.H / 4, (i64)a.M, reinterpret_cast<uint2*>(w->Apack));
+  if (launch_pdl(pack_rows_kernel, dim3(pgrid((i64)a.M * (a.H / 4))), dim3(kPT), 0, s, a.hin, a.hin_ks, a.B, a.H / 4, (i64)a.M,
+                 reinterpret_cast<uint2*>(w->Apack)) != cudaSuccess)
+    return MGRIT_CUDA_ERROR;
   count_launch();
-  launch_gemm<192, true>(KC_FWD_STEP, w->Apack, a.H, w->W_hh, a.H, a.M, a.H, a.H, a.H, 3 * a.H, EpiFwd{a}, s);
+  ok = launch_gemm<192, true>(KC_FWD_STEP, w->Apack, a.H, w->W_hh, a.H, a.M, a.H, a.H, a.H, 3 * a.H, EpiFwd{a}, s);
+  return ok ? MGRIT_OK : MGRIT_CUDA_ERROR;
 }
 
-void umma_linearise(const LinArgs& a, UmmaAdjWs* w, cudaStream_t s) {
+int umma_linearise(const LinArgs& a, UmmaAdjWs* w, cudaStream_t s) {
   // rows (j-1, b): state entering forward step j of the level = h_{stride*(j-1)}
   const i64 BH = (i64)a.B * a.H;
   const int N = a.M / a.B;
@@ -663,37 +678,46 @@ void umma_linearise(const LinArgs& a, UmmaAdjWs* w, cudaStream_t s) {
     const float* gi0 = a.gi + (a.stride_t - 1) * BH * 3;
     // step 1 starts from h_0 (its own array); steps 2..N from h[stride*(j-1) - 1]
     ca.a = a.a; ca.cr = a.crb; ca.cz = a.czb; ca.cn = a.cnb; ca.cnp = a.cnpb;
-    launch_cell<true, false>(KC_LINEARISE, w->hb0, 0, gi0, 0, a.h0, 0, nullptr, 0, 1, w->W_hh, ca, s);
+    if (!launch_cell<true, false>(KC_LINEARISE, w->hb0, 0, gi0, 0, a.h0, 0, nullptr, 0, 1, w->W_hh, ca, s)) return MGRIT_CUDA_ERROR;
     if (N > 1) {
       ca.a = a.a + BH; ca.cr = a.crb + BH; ca.cz = a.czb + BH; ca.cn = a.cnb + BH; ca.cnp = a.cnpb ? a.cnpb + BH : nullptr;
-      launch_cell<true, false>(KC_LINEARISE, w->hb + (a.stride_t - 1) * BH, a.stride_t * BH, gi0 + a.stride_t * BH * 3, a.stride_t * BH * 3,
-                               a.h + (a.stride_t - 1) * BH, a.stride_t * BH, nullptr, 0, N - 1, w->W_hh, ca, s);
+      if (!launch_cell<true, false>(KC_LINEARISE, w->hb + (a.stride_t - 1) * BH, a.stride_t * BH, gi0 + a.stride_t * BH * 3,
+                                    a.stride_t * BH * 3, a.h + (a.stride_t - 1) * BH, a.stride_t * BH, nullptr, 0, N - 1, w->W_hh, ca, s))
+        return MGRIT_CUDA_ERROR;
     }
-    return;
+    return MGRIT_OK;
   }
-  launch_pdl(pack_rows_kernel, dim3(pgrid((i64)a.B * (a.H / 4))), dim3(kPT), 0, s, a.h0, (i64)0, a.B, a.H / 4, (i64)a.B, reinterpret_cast<uint2*>(w->Apack));
+  if (launch_pdl(pack_rows_kernel, dim3(pgrid((i64)a.B * (a.H / 4))), dim3(kPT), 0, s, a.h0, (i64)0, a.B, a.H / 4, (i64)a.B,
+                 reinterpret_cast<uint2*>(w->Apack)) != cudaSuccess)
+    return MGRIT_CUDA_ERROR;
   count_launch();
   if (a.M > a.B) {
-    launch_pdl(pack_rows_kernel, dim3(pgrid((i64)(a.M - a.B) * (a.H / 4))), dim3(kPT), 0, s, a.h + (a.stride_t - 1) * BH,
-               (i64)(a.stride_t * BH), a.B, a.H / 4, (i64)(a.M - a.B), reinterpret_cast<uint2*>(w->Apack + BH));
+    if (launch_pdl(pack_rows_kernel, dim3(pgrid((i64)(a.M - a.B) * (a.H / 4))), dim3(kPT), 0, s, a.h + (a.stride_t - 1) * BH,
+                   (i64)(a.stride_t * BH), a.B, a.H / 4, (i64)(a.M - a.B), reinterpret_cast<uint2*>(w->Apack + BH)) != cudaSuccess)
+      return MGRIT_CUDA_ERROR;
     count_launch();
   }
-  launch_gemm<192, true>(KC_LINEARISE, w->Apack, a.H, w->W_hh, a.H, a.M, a.H, a.H, a.H, 3 * a.H, EpiLin{a}, s);
+  return launch_gemm<192, true>(KC_LINEARISE, w->Apack, a.H, w->W_hh, a.H, a.M, a.H, a.H, a.H, 3 * a.H, EpiLin{a}, s) ? MGRIT_OK
+                                                                                                                      : MGRIT_CUDA_ERROR;
 }
 
-void umma_adj_step(const AdjStepArgs& a, UmmaAdjWs* w, cudaStream_t s) {
-  launch_pdl(pack_adj_kernel, dim3(pgrid((i64)a.M * (a.H / 4))), dim3(kPT), 0, s, a.lin, a.lin_ks, a.crb, a.czb, a.cnb, a.coef_ks, a.B,
-             a.H / 4, (i64)a.M, reinterpret_cast<uint2*>(w->Apack));
+int umma_adj_step(const AdjStepArgs& a, UmmaAdjWs* w, cudaStream_t s) {
+  ProfScope prof(KC_ADJ_STEP, 2.0 * a.M * 3.0 * a.H * a.H, s);     // operand packing + product, timed together
+  if (launch_pdl(pack_adj_kernel, dim3(pgrid((i64)a.M * (a.H / 4))), dim3(kPT), 0, s, a.lin, a.lin_ks, a.crb, a.czb, a.cnb, a.coef_ks,
+                 a.B, a.H / 4, (i64)a.M, reinterpret_cast<uint2*>(w->Apack)) != cudaSuccess)
+    return MGRIT_CUDA_ERROR;
   count_launch();
   // Few-row launches (coarse levels, short prefixes) cannot fill the SMs with 256-column tiles and are
   // bound by one CTA streaming all of K; 64-column tiles spread that stream over four times the CTAs.
   const int tiles256 = ((a.M + BM - 1) / BM) * ((a.H + 255) / 256);
+  bool ok;
   if (tiles256 * 2 <= kSMs)
-    launch_gemm<64, false>(KC_ADJ_STEP, w->Apack, 3 * a.H, w->W_hhT, 3 * a.H, a.M, a.H, 3 * a.H, 0, a.H, EpiAdj<64>{a}, s);
+    ok = launch_gemm<64, false>(KC_ADJ_STEP, w->Apack, 3 * a.H, w->W_hhT, 3 * a.H, a.M, a.H, 3 * a.H, 0, a.H, EpiAdj<64>{a}, s);
   else if (gemm_pair_enabled(a.M, a.H))
-    launch_gemm_pair(KC_ADJ_STEP, w->Apack, 3 * a.H, w->W_hhT, 3 * a.H, a.M, a.H, 3 * a.H, a.H, EpiAdj<256>{a}, s);
+    ok = launch_gemm_pair(KC_ADJ_STEP, w->Apack, 3 * a.H, w->W_hhT, 3 * a.H, a.M, a.H, 3 * a.H, a.H, EpiAdj<256>{a}, s);
   else
-    launch_gemm<256, false>(KC_ADJ_STEP, w->Apack, 3 * a.H, w->W_hhT, 3 * a.H, a.M, a.H, 3 * a.H, 0, a.H, EpiAdj<256>{a}, s);
+    ok = launch_gemm<256, false>(KC_ADJ_STEP, w->Apack, 3 * a.H, w->W_hhT, 3 * a.H, a.M, a.H, 3 * a.H, 0, a.H, EpiAdj<256>{a}, s);
+  return ok ? MGRIT_OK : MGRIT_CUDA_ERROR;
 }
 
 // dst[e] = sum over the `splits` partial products (float4 stream)
@@ -736,25 +760,29 @@ static bool wgrad_gemm(const bf16* dA, int H3, const bf16* R, int cols, int K, O
 }
 
 int umma_gradients(const mgrit_gru_cfg* c, const gru_params* p, const float* x, const float* h0, const float* h, const float* lam,
-                   const bf16* cr, const bf16* cz, const bf16* cn, const bf16* cnp, float* dx, const gru_grads* g,
+                   i64 lam_ts, const bf16* cr, const bf16* cz, const bf16* cn, const bf16* cnp, float* dx, const gru_grads* g,
                    UmmaAdjWs* w, cudaStream_t s) {
+  (void)h0; (void)h;
   const int H = c->H, I = c->I, B = c->B;
   const i64 M = (i64)c->T * B;
-  cudaMemsetAsync(g->db_hh, 0, sizeof(float) * 3 * H, s);
-  cudaMemsetAsync(g->db_ih, 0, sizeof(float) * 3 * H, s);
+  // one timing record for the whole pass: operand forming, bias sums, the three products and their split sums
+  ProfScope prof(KC_WGRAD, 2.0 * M * 3.0 * H * ((double)H + I + (dx ? I : 0)), s);
   // operands of the three gradient GEMMs, all row-major (the reduction index t,b is the row index)
   bf16* dAh = w->dAh; bf16* dAi = w->dAi;        // [M, 3H] each
   const int rows_per_block = 256;
+  // (the step operand buffer is free during the gradient pass: scratch for the bias partials, then for the split
+  // partial products of the weight-gradient GEMMs; M >= 8 makes nblk*16H <= 2MH bytes)
+  float* scratch = reinterpret_cast<float*>(w->Apack);
+  const size_t scratch_bytes = w->apack_elems * sizeof(bf16);
   dim3 grid((unsigned)((M + rows_per_block - 1) / rows_per_block), (H / 4 + 31) / 32);
-  form_dA_rows_kernel<<<grid, 256, 0, s>>>(lam, cr, cz, cn, cnp, M, H, reinterpret_cast<uint2*>(dAh), reinterpret_cast<uint2*>(dAi),
-                                           g->db_hh, g->db_ih, rows_per_block);
-  count_launch();
+  if ((size_t)grid.x * 4 * H * sizeof(float) > scratch_bytes) return MGRIT_UNSUPPORTED;
+  form_dA_rows_kernel<<<grid, 256, 0, s>>>(lam, lam_ts, B, cr, cz, cn, cnp, M, H, reinterpret_cast<uint2*>(dAh),
+                                           reinterpret_cast<uint2*>(dAi), scratch, rows_per_block);
+  sum_db_kernel<<<pgrid(4 * H), kPT, 0, s>>>(scratch, (int)grid.x, H, g->db_hh, g->db_ih);
+  count_launch(2);
   convert(x, w->xb, M * I, s);                   // x as bf16 [M, I]; h_{t-1} as bf16 = [h_0; h] without its last slot (w->hb0)
   bool ok = true;
   // dW_hh[3H, H] = dA_h^T h_prev ;  dW_ih[3H, I] = dA_i^T x    (K = T*B, MN-major operands)
-  // (the step operand buffer is free during the gradient pass: scratch for the split partial products)
-  float* scratch = reinterpret_cast<float*>(w->Apack);
-  const size_t scratch_bytes = w->apack_elems * sizeof(bf16);
   ok = ok && wgrad_gemm(dAh, 3 * H, w->hb0, H, (int)M, g->dW_hh, scratch, scratch_bytes, s);
   ok = ok && wgrad_gemm(dAi, 3 * H, w->xb, I, (int)M, g->dW_ih, scratch, scratch_bytes, s);
   // dx[T*B, I] = dA_i W_ih   (K = 3H, K-major operands)
@@ -768,10 +796,19 @@ int umma_gradients(const mgrit_gru_cfg* c, const gru_params* p, const float* x, 
 void umma_convert(const float* src, __nv_bfloat16* dst, i64 n, cudaStream_t s) { convert(src, dst, n, s); }
 
 int umma_device_status() {
-  if (!g_status_ptr) return 0;
+  const int dev = current_device_slot();
+  if (dev < 0) return -1;
+  if (!g_status_ptrs[dev]) return 0;     // no tensor-core kernel has run on this device
   int v = 0;
-  if (cudaMemcpy(&v, g_status_ptr, sizeof(int), cudaMemcpyDeviceToHost) != cudaSuccess) return -1;
+  if (cudaMemcpy(&v, g_status_ptrs[dev], sizeof(int), cudaMemcpyDeviceToHost) != cudaSuccess) return -1;
   return v;
+}
+
+int umma_clear_device_status() {
+  const int dev = current_device_slot();
+  if (dev < 0) return -1;
+  if (!g_status_ptrs[dev]) return 0;
+  return cudaMemset(g_status_ptrs[dev], 0, sizeof(int)) == cudaSuccess ? 0 : -1;
 }
 
 }  // namespace mg

@@ -36,14 +36,15 @@ def make_cfgs(w: Workload, T: int, Bsz: int, serial: bool = False, flags: int = 
     return fw, ad
 
 
-def alloc_buffers(w: Workload, T: int, Bsz: int, device, serial: bool = False, flags: int = 0) -> StepBuffers:
+def alloc_buffers(w: Workload, T: int, Bsz: int, device, serial: bool = False, flags: int = 0, want_dh: bool = False) -> StepBuffers:
     fw, ad = make_cfgs(w, T, Bsz, serial, flags)
     nf = max(B.workspace_bytes(c)[0] for c in fw)
     na = max(B.workspace_bytes(c)[1] for c in ad)
     mk = lambda *s: torch.empty(*s, device=device)
     adj = []
     for l, c in enumerate(ad):
-        adj.append(B.AdjointResult(dh=mk(T, Bsz, w.H), dh0=mk(Bsz, w.H), dx=mk(T, Bsz, c.I) if l > 0 else None,
+        # dh (dL/dh_t for every t) is not an input of anything in a training step: only written when asked for
+        adj.append(B.AdjointResult(dh=mk(T, Bsz, w.H) if want_dh else None, dh0=mk(Bsz, w.H), dx=mk(T, Bsz, c.I) if l > 0 else None,
                                    dW_ih=mk(3 * w.H, c.I), dW_hh=mk(3 * w.H, w.H), db_ih=mk(3 * w.H), db_hh=mk(3 * w.H)))
     return StepBuffers(fw, ad, torch.empty(nf, dtype=torch.uint8, device=device), torch.empty(na, dtype=torch.uint8, device=device),
                        torch.empty(B.lib.xent_head_workspace_bytes(Bsz, w.classes), dtype=torch.uint8, device=device),

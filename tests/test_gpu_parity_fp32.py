@@ -154,6 +154,37 @@ def test_tiny_adjoint_three_level_fcf(B):
     _adjoint_case(B, w, d, _cfg(B, w, 2, levels=3, cf=2, relax_fine=1), 2, seed_all=True, cf=2, levels=3, rf=1)
 
 
+def test_whole_chain_against_the_oracles_own_forward(B):
+    # Forward, loss head, adjoint and gradients on the GPU against the same chain run by the oracle alone (its
+    # adjoint linearised at its OWN forward states): nothing of the GPU's output enters the reference.
+    w = WORKLOADS["tiny"]
+    d = make_inputs(w)
+    p, x, h0 = upload(d)
+    P = oracle_params(d)
+    xr, h0r = d["x"].astype(np.float64), d["h0"].astype(np.float64)
+    for levels, cf, rf in ((2, 4, 0), (3, 2, 1)):
+        cfg = _cfg(B, w, 2, levels=levels, cf=cf, relax_fine=rf)
+        kw = dict(cf=cf, levels=levels, relax_fine=rf, relax_coarse=w.relax_coarse, iters=2)
+        h, gi, _ = B.mgrit_gru_forward(cfg, p, x, h0)
+        loss, dhT, dWc, dbc = B.xent_head_fwd_bwd(h[-1].contiguous(), to_dev(d["W_c"]), to_dev(d["b_c"]), to_dev(d["labels"]))
+        r = B.mgrit_gru_adjoint(cfg, p, x, h0, gi, h, dhT=dhT)
+        href, _ = O.mgrit_forward(*P, xr, h0r, **kw)
+        loss_r, dhT_r, dWc_r, dbc_r = O.xent_head(href[-1], d["W_c"].astype(np.float64), d["b_c"].astype(np.float64), d["labels"])
+        seed = np.zeros_like(href)
+        seed[-1] = dhT_r
+        lam, lam0, g, _ = O.mgrit_adjoint(*P, xr, h0r, href, seed, **kw)
+        assert abs(loss.item() - loss_r) < 1e-5
+        assert rel_inf(dWc.cpu().numpy(), dWc_r) < TOL_G and rel_inf(dbc.cpu().numpy(), dbc_r) < TOL_G
+        assert rel_inf(r.dh.cpu().numpy(), lam) < TOL_G
+        for k in ("dx", "dW_ih", "dW_hh", "db_ih", "db_hh"):
+            assert rel_inf(getattr(r, k).cpu().numpy(), g[k]) < TOL_G, (k, levels)
+        # dh is an optional output: without it everything else is unchanged, bit for bit
+        r2 = B.mgrit_gru_adjoint(cfg, p, x, h0, gi, h, dhT=dhT, want_dh=False)
+        assert r2.dh is None
+        for k in ("dh0", "dx", "dW_ih", "dW_hh", "db_ih", "db_hh"):
+            assert torch.equal(getattr(r, k), getattr(r2, k)), k
+
+
 def test_tiny_serial_backward(B):
     w = WORKLOADS["tiny"]
     d = make_inputs(w)

@@ -47,3 +47,25 @@ def test_host_side_validation_without_a_device(lib):
     assert b"divisible" in lib.mgrit_gru_strerror(-2)
     lib.xent_head_workspace_bytes.restype = ctypes.c_size_t
     assert lib.xent_head_workspace_bytes(32, 51) >= 32 * 51 * 4
+
+
+def test_sizes_beyond_32_bit_row_counts_are_rejected(lib):
+    from paper_2203_04738_b200.binding import Cfg, make_cfg
+    f = ctypes.c_size_t(0)
+    fn = lib.mgrit_gru_workspace_bytes
+    fn.argtypes = [ctypes.POINTER(Cfg), ctypes.POINTER(ctypes.c_size_t), ctypes.POINTER(ctypes.c_size_t)]
+    # (T + 1) * B just above 2^31: row counts are 32-bit inside the kernels
+    assert fn(ctypes.byref(make_cfg(1 << 26, 32, 16, 64, cf=4, levels=2)), ctypes.byref(f), None) == -4
+    assert fn(ctypes.byref(make_cfg(1 << 25, 32, 16, 64, cf=4, levels=2)), ctypes.byref(f), None) == 0
+    assert f.value > (1 << 25) * 32 * 64 * 4          # the size itself is computed in 64 bits
+
+
+def test_status_calls_answer_without_a_device(lib):
+    # no device: nothing to wait for and nothing recorded -- the calls must return an error code, never crash
+    lib.mgrit_gru_last_device_status.restype = ctypes.c_int
+    lib.mgrit_gru_clear_device_status.restype = ctypes.c_int
+    import torch
+    if torch.cuda.is_available():
+        assert lib.mgrit_gru_clear_device_status() == 0 and lib.mgrit_gru_last_device_status() == 0
+    else:
+        assert lib.mgrit_gru_last_device_status() == -5 and lib.mgrit_gru_clear_device_status() == -5
