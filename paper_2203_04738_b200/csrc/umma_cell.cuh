@@ -1,11 +1,27 @@
-// Fused "recurrent GEMM + GRU cell" kernel for sm_100a, second form: every operand of the epilogue
-// is staged through shared memory by TMA, so that the only latency-exposed global accesses of the
-// epilogue are its stores.
+// Fused "recurrent GEMM + GRU cell" kernel for sm_100a: every operand of the epilogue is staged through
+// shared memory by TMA, so that the only latency-exposed global accesses of the epilogue are its stores.
 //
-//   rows m = (k, b)      k = interval / coarse point, b = batch row, 128 rows per tile = kt k's x B
+//   rows m = (k, b)      k = interval / coarse point, b = batch row, 128 rows per CTA tile = kt k's x B
 //   D[m, gate, u] = sum_j hb[m, j] * W_hh[gate*H + u, j]          (tcgen05, bf16 x bf16 -> fp32 in TMEM)
 //   forward : out[m, u] = Phi_gamma(gi[m, :, u], D + b_hh, h[m, u]) (+ g[m, u])   or   g - Phi   (mode 1)
 //   linearise: a, c_r, c_z, c_n, c_n'[m, u] = transposed-Jacobian coefficients of that step
+//
+// Two geometries of the same kernel:
+//   PAIR = false  one CTA per 128 x (3 x 64) tile, tcgen05.mma.cta_group::1 with N = 192.
+//   PAIR = true   clusters of two CTAs (the two SMs of a TPC) share one 256 x (3 x 80) tile:
+//                 tcgen05.mma.cta_group::2 with N = 240.  Each CTA stages its own 128 rows of A and HALF of the
+//                 weight tile (120 of the 240 gate rows: 31 KiB per k-block instead of 40), so the operand bytes an
+//                 SM takes in per flop drop by 40 %.  The width is 80 units because the duration of a pair MMA does
+//                 not depend on N (measured on a bare main loop: 256 x N x 16 takes the same 164 cycles for every
+//                 N from 128 to 256), so a tile should be as close to 256 columns as three equal gates allow; 240
+//                 columns twice fit the 512 columns of tensor memory.  The last unit tile of a row is ragged
+//                 (H = 1024: twelve tiles of 80 units and one of 64); its surplus columns are computed on
+//                 whatever weight rows follow and never stored.
+//   Pair protocol: both CTAs' operand loads complete on the LEADER's (rank 0) full barrier, which expects the
+//   bytes of both; the leader's MMA thread issues for the pair and commits each stage to both CTAs' empty barriers
+//   and each accumulator to both CTAs' tfull barriers (one commit per destination, no multicast load anywhere);
+//   one elected lane per epilogue warp of both CTAs releases the leader's accumulator barrier (remote arrive
+//   for rank 1); tensor memory is allocated and freed by the same warp of both CTAs behind cluster barriers.
 //
 // Warp roles (352 threads): 0 = TMA producer of the A/B ring, 1 = MMA issuer and TMEM owner,
 // 2 = TMA producer of the epilogue operands (gi r|z|n, h, g in chunks of 16 hidden units, two
@@ -14,9 +30,11 @@
 // maps {column, batch row, k} whose k-stride is the slot stride of the relaxation, so no gather
 // kernel is needed; the epilogue also writes the bf16 copy of the new state for the next step.
 // Epilogue tiles use the 64-byte swizzle: rows of 16 floats, 16-byte chunk index XOR ((row >> 1) & 3).
+// Every wait on an mbarrier is bounded (2 s): a wait that runs out records a code in the status word and the
+// CTA stops issuing work, so both CTAs of a pair reach the closing cluster barrier.
 #pragma once
 #include "cell.cuh"
-#include "umma_gemm.cuh"
+#include "umma_gemm_pair.cuh"
 
 namespace mg {
 namespace umma {
@@ -24,6 +42,13 @@ namespace umma {
 __device__ __forceinline__ void tma_load_3d(uint32_t dst, const CUtensorMap* map, uint32_t bar, int c0, int c1, int c2) {
   asm volatile(
       "cp.async.bulk.tensor.3d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, %5}], [%2];"
+      ::"r"(dst), "l"(map), "r"(bar), "r"(c0), "r"(c1), "r"(c2)
+      : "memory");
+}
+// ... whose completion barrier may live in the other CTA of the pair (bar is a shared::cluster address)
+__device__ __forceinline__ void tma_load_3d_pair(uint32_t dst, const CUtensorMap* map, uint32_t bar, int c0, int c1, int c2) {
+  asm volatile(
+      "cp.async.bulk.tensor.3d.cta_group::2.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, %5}], [%2];"
       ::"r"(dst), "l"(map), "r"(bar), "r"(c0), "r"(c1), "r"(c2)
       : "memory");
 }
@@ -77,24 +102,44 @@ struct CellArgs {
 };
 
 namespace cellk {
-constexpr int BN = 192, UN = 64, CH = 16, NCH = UN / CH;
+constexpr int CH = 16;                  // hidden units per epilogue chunk
 constexpr int kThreads = 352;
-constexpr int kABytes = BM * BK * 2, kBBytes = BN * BK * 2, kStageBytes = kABytes + kBBytes;
+constexpr int kABytes = BM * BK * 2;
 constexpr int kOpBytes = BM * CH * 4;   // one epilogue operand chunk: 128 rows x 16 floats
 // The linearisation's four bf16 coefficient arrays leave through shared memory: per chunk four [128 x 16] bf16
 // tiles (32-byte swizzle), two buffers, written to global memory by TMA stores.  (Four 16-byte st.global per thread
-// and chunk, each touching 32 different rows, cost a third of that kernel's time.)
+// and chunk, each touching 32 different rows, cost a third of that kernel's time.)  The forward step's two stores
+// per thread and chunk (32 bytes of state, 16 bytes of its bf16 copy) stay direct: staged the same way they cost
+// the same 20 us of a 118 us step and one stage of the operand ring; what a store costs here is the number of
+// row pieces that reach L2, not the path they take (rows of 128 bytes instead of 64 halve it).
 constexpr int kCoefBytes = BM * CH * 2;   // one coefficient chunk: 128 rows x 16 bf16
-template <bool HAS_G, bool LIN = false> struct CellCfg {
-  static constexpr int kStages = (HAS_G || LIN) ? 3 : 4;
+template <bool PAIR> struct Geo {
+  static constexpr int UN = PAIR ? 80 : 64;         // hidden units per tile
+  static constexpr int BN = 3 * UN;                 // accumulator columns: r | z | n
+  static constexpr int NCH = UN / CH;
+  static constexpr int kBox = PAIR ? 40 : 64;       // weight rows per TMA box
+  static constexpr int kBBytes = (PAIR ? BN / 2 : BN) * BK * 2;   // weight bytes staged per CTA and k-block
+  static constexpr int kStageBytes = kABytes + kBBytes;           // 31 KiB / 40 KiB (multiples of 1 KiB)
+};
+template <bool HAS_G, bool LIN = false, bool PAIR = false> struct CellCfg {
+  using G = Geo<PAIR>;
+#ifndef CELL_PAIR_STAGES
+#define CELL_PAIR_STAGES ((HAS_G || LIN) ? 4 : 5)
+#endif
+#ifndef CELL_PAIR_EBUFS
+#define CELL_PAIR_EBUFS 2
+#endif
+  static constexpr int kStages = PAIR ? CELL_PAIR_STAGES : ((HAS_G || LIN) ? 3 : 4);
+  static constexpr int kEpiBufs = PAIR ? CELL_PAIR_EBUFS : 2;     // epilogue-operand chunks in flight
   static constexpr int kOps = HAS_G ? 5 : 4;
   static constexpr int kEpiBytes = kOps * kOpBytes;
   static constexpr int kOutBytes = LIN ? 4 * kCoefBytes : 0;      // per buffer
-  static constexpr int kSmemBytes = kStages * kStageBytes + 2 * kEpiBytes + 2 * kOutBytes + 1024 + 256;
+  static constexpr int kSmemBytes = kStages * G::kStageBytes + kEpiBufs * kEpiBytes + 2 * kOutBytes + 1024 + 256;
+  static_assert(kSmemBytes + 1536 <= 232448, "shared memory budget (dynamic + static <= 227 KiB)");
 };
 }  // namespace cellk
 
-template <bool LIN, bool HAS_G>
+template <bool LIN, bool HAS_G, bool PAIR>
 __global__ void __launch_bounds__(cellk::kThreads, 1)
 umma_cell_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB,
                  const __grid_constant__ CUtensorMap tmGI, const __grid_constant__ CUtensorMap tmHP,
@@ -102,44 +147,59 @@ umma_cell_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
                  const __grid_constant__ CUtensorMap tmCZ, const __grid_constant__ CUtensorMap tmCN,
                  const __grid_constant__ CUtensorMap tmCP, CellArgs p, int* status) {
   using namespace cellk;
-  using C = CellCfg<HAS_G, LIN>;
+  using C = CellCfg<HAS_G, LIN, PAIR>;
+  using G = Geo<PAIR>;
+  constexpr int UN = G::UN, BN = G::BN, NCH = G::NCH, kStageBytes = G::kStageBytes;
   extern __shared__ uint8_t smem_raw[];
   const uint32_t raw = smem_u32(smem_raw);
   const uint32_t tiles_base = (raw + 1023u) & ~1023u;
   const uint32_t epi_base = tiles_base + C::kStages * kStageBytes;
-  const uint32_t out_base = epi_base + 2 * C::kEpiBytes;
+  const uint32_t out_base = epi_base + C::kEpiBufs * C::kEpiBytes;
   const uint32_t bars = out_base + 2 * C::kOutBytes;
   auto full_bar = [&](int s) { return bars + 8u * s; };
   auto empty_bar = [&](int s) { return bars + 8u * (C::kStages + s); };
   auto tfull_bar = [&](int a) { return bars + 8u * (2 * C::kStages + a); };
   auto tempty_bar = [&](int a) { return bars + 8u * (2 * C::kStages + 2 + a); };
   auto efull_bar = [&](int e) { return bars + 8u * (2 * C::kStages + 4 + e); };
-  auto eempty_bar = [&](int e) { return bars + 8u * (2 * C::kStages + 6 + e); };
+  auto eempty_bar = [&](int e) { return bars + 8u * (2 * C::kStages + 4 + C::kEpiBufs + e); };
   __shared__ uint32_t tmem_base_smem;
   __shared__ int abort_flag;
   __shared__ uint32_t lds_sink[cellk::kThreads];   // see the operand-buffer release in the epilogue
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int H = p.H;
-  const int m_tiles = (p.M + BM - 1) / BM, n_tiles = H / UN, tiles = m_tiles * n_tiles;
+  // PAIR: a tile is 256 rows; CTA `rank` of the pair owns its rows [128 rank, 128 rank + 128).
+  const uint32_t rank = PAIR ? cluster_ctarank() : 0u;
+  const int cta = PAIR ? (int)(blockIdx.x >> 1) : (int)blockIdx.x, ncta = PAIR ? (int)(gridDim.x >> 1) : (int)gridDim.x;
+  constexpr int kTileRows = PAIR ? 2 * BM : BM;
+  const int m_tiles = (p.M + kTileRows - 1) / kTileRows, n_tiles = (H + UN - 1) / UN, tiles = m_tiles * n_tiles;
   const int k_blocks = (H + BK - 1) / BK;
+  auto row_tile = [&](int t) { return PAIR ? 2 * (t / n_tiles) + (int)rank : t / n_tiles; };
 
   if (threadIdx.x == 0) {
     abort_flag = 0;
     for (int s = 0; s < C::kStages; ++s) { mbar_init(full_bar(s), 1); mbar_init(empty_bar(s), 1); }
     for (int a = 0; a < 2; ++a) {
-      mbar_init(tfull_bar(a), 1); mbar_init(tempty_bar(a), 256);
-      mbar_init(efull_bar(a), 1); mbar_init(eempty_bar(a), 256);
+      mbar_init(tfull_bar(a), 1);
+      mbar_init(tempty_bar(a), PAIR ? 16 : 8);      // one elected lane per epilogue warp (of both CTAs)
     }
+    for (int e = 0; e < C::kEpiBufs; ++e) { mbar_init(efull_bar(e), 1); mbar_init(eempty_bar(e), 256); }
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
   if (warp == 1) {
-    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&tmem_base_smem)), "r"(512u)
-                 : "memory");
-    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+    if (PAIR) {   // the same warp of both CTAs allocates the same columns in both tensor memories
+      asm volatile("tcgen05.alloc.cta_group::2.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&tmem_base_smem)), "r"(512u)
+                   : "memory");
+      asm volatile("tcgen05.relinquish_alloc_permit.cta_group::2.sync.aligned;" ::: "memory");
+    } else {
+      asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&tmem_base_smem)), "r"(512u)
+                   : "memory");
+      asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+    }
   }
   tc_fence_before();
   __syncthreads();
+  if (PAIR) cluster_sync_all();   // the peer's barriers are initialised before anything signals them
   tc_fence_after();
   const uint32_t tmem_base = tmem_base_smem;
   volatile int* abortp = &abort_flag;
@@ -150,25 +210,38 @@ umma_cell_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
     // ------------------------------------------------------------ A/B producer
     if (lane == 0) {
       int stage = 0; uint32_t phase = 0; bool ok = true;
-      for (int t = blockIdx.x; t < tiles && ok; t += gridDim.x) {
-        const int mt = t / n_tiles, nt = t % n_tiles;
+      for (int t = cta; t < tiles && ok; t += ncta) {
+        const int mt = row_tile(t), nt = t % n_tiles;
         for (int kb = 0; kb < k_blocks; ++kb) {
           if (!mbar_wait(empty_bar(stage), phase ^ 1u, abortp, status, 11)) { ok = false; break; }
           const uint32_t a_dst = tiles_base + stage * kStageBytes, b_dst = a_dst + kABytes;
-          mbar_expect_tx(full_bar(stage), kStageBytes);
-          tma_load_3d(a_dst, &tmA, full_bar(stage), kb * BK, 0, mt * p.kt);
+          if (PAIR) {
+            // The accumulator columns r | z | n (80 each) split into two halves of 120: CTA 0 stages the weight rows
+            // of r and of the first 40 units of z, CTA 1 the rest -- six 40-row boxes, three per CTA.
+            const uint32_t fullL = mapa_shared(full_bar(stage), 0);
+            if (rank == 0) mbar_expect_tx(full_bar(stage), 2 * kStageBytes);
+            tma_load_3d_pair(a_dst, &tmA, fullL, kb * BK, 0, mt * p.kt);
 #pragma unroll
-          for (int g = 0; g < 3; ++g) tma_load_2d(b_dst + g * (kBBytes / 3), &tmB, full_bar(stage), kb * BK, g * H + nt * UN);
+            for (int j = 0; j < 3; ++j) {
+              const int piece = 3 * (int)rank + j;
+              tma_load_2d_pair(b_dst + j * (G::kBox * BK * 2), &tmB, fullL, kb * BK, (piece >> 1) * H + nt * UN + (piece & 1) * G::kBox);
+            }
+          } else {
+            mbar_expect_tx(full_bar(stage), kStageBytes);
+            tma_load_3d(a_dst, &tmA, full_bar(stage), kb * BK, 0, mt * p.kt);
+#pragma unroll
+            for (int g = 0; g < 3; ++g) tma_load_2d(b_dst + g * (G::kBBytes / 3), &tmB, full_bar(stage), kb * BK, g * H + nt * UN);
+          }
           if (++stage == C::kStages) { stage = 0; phase ^= 1u; }
         }
       }
     }
   } else if (warp == 1) {
-    // ------------------------------------------------------------ MMA issuer
-    if (lane == 0) {
-      constexpr uint32_t idesc = instr_desc_bf16(BN);
+    // ------------------------------------------------------------ MMA issuer (PAIR: the leader issues for both CTAs)
+    if (lane == 0 && rank == 0) {
+      constexpr uint32_t idesc = PAIR ? instr_desc_bf16_pair(BN) : instr_desc_bf16(BN);
       int stage = 0; uint32_t phase = 0; int it = 0; bool ok = true;
-      for (int t = blockIdx.x; t < tiles && ok; t += gridDim.x, ++it) {
+      for (int t = cta; t < tiles && ok; t += ncta, ++it) {
         const int as = it & 1;
         const uint32_t aphase = (uint32_t)(it >> 1) & 1u;
         if (!mbar_wait(tempty_bar(as), aphase ^ 1u, abortp, status, 12)) { ok = false; break; }
@@ -180,31 +253,46 @@ umma_cell_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
           const uint32_t a_src = tiles_base + stage * kStageBytes;
           const uint64_t adesc = smem_desc_sw128(a_src), bdesc = smem_desc_sw128(a_src + kABytes);
 #pragma unroll
-          for (int k = 0; k < BK / 16; ++k)
-            mma_bf16(d_tmem, adesc + (uint64_t)(k * 2), bdesc + (uint64_t)(k * 2), idesc, (kb | k) != 0 ? 1u : 0u);
-          mma_commit(empty_bar(stage));
+          for (int k = 0; k < BK / 16; ++k) {
+            if (PAIR) mma_bf16_pair(d_tmem, adesc + (uint64_t)(k * 2), bdesc + (uint64_t)(k * 2), idesc, (kb | k) != 0 ? 1u : 0u);
+            else mma_bf16(d_tmem, adesc + (uint64_t)(k * 2), bdesc + (uint64_t)(k * 2), idesc, (kb | k) != 0 ? 1u : 0u);
+          }
+          if (PAIR) {   // the stage is free again in both CTAs
+            mma_commit_pair(mapa_shared(empty_bar(stage), 0));
+            mma_commit_pair(mapa_shared(empty_bar(stage), 1));
+          } else {
+            mma_commit(empty_bar(stage));
+          }
           if (++stage == C::kStages) { stage = 0; phase ^= 1u; }
         }
-        if (ok) mma_commit(tfull_bar(as));
+        if (ok) {
+          if (PAIR) {
+            mma_commit_pair(mapa_shared(tfull_bar(as), 0));
+            mma_commit_pair(mapa_shared(tfull_bar(as), 1));
+          } else {
+            mma_commit(tfull_bar(as));
+          }
+        }
       }
     }
   } else if (warp == 2) {
     // ------------------------------------------------------------ epilogue-operand producer
     if (lane == 0) {
       int eb = 0; uint32_t ephase = 0; bool ok = true;
-      for (int t = blockIdx.x; t < tiles && ok; t += gridDim.x) {
-        const int mt = t / n_tiles, nt = t % n_tiles;
+      for (int t = cta; t < tiles && ok; t += ncta) {
+        const int mt = row_tile(t), nt = t % n_tiles;
         for (int c = 0; c < NCH; ++c) {
+          const int u = nt * UN + c * CH, k0 = mt * p.kt;
+          if (u >= H) break;                       // ragged last unit tile: these columns are never stored
           if (!mbar_wait(eempty_bar(eb), ephase ^ 1u, abortp, status, 14)) { ok = false; break; }
           const uint32_t dst = epi_base + eb * C::kEpiBytes;
-          const int u = nt * UN + c * CH, k0 = mt * p.kt;
           mbar_expect_tx(efull_bar(eb), C::kEpiBytes);
           tma_load_3d(dst, &tmGI, efull_bar(eb), u, 0, k0);
           tma_load_3d(dst + kOpBytes, &tmGI, efull_bar(eb), H + u, 0, k0);
           tma_load_3d(dst + 2 * kOpBytes, &tmGI, efull_bar(eb), 2 * H + u, 0, k0);
           tma_load_3d(dst + 3 * kOpBytes, &tmHP, efull_bar(eb), u, 0, k0);
           if (HAS_G) tma_load_3d(dst + 4 * kOpBytes, &tmG, efull_bar(eb), u, 0, k0);
-          if (++eb == 2) { eb = 0; ephase ^= 1u; }
+          if (++eb == C::kEpiBufs) { eb = 0; ephase ^= 1u; }
         }
       }
     }
@@ -212,7 +300,7 @@ umma_cell_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
     // ------------------------------------------------------------ epilogue (warps 3..10)
     const int q = warp & 3;              // TMEM lane quarter of this warp
     const int half = (warp - 3) >> 2;    // which 8 of a chunk's 16 hidden units
-    const int r = q * 32 + lane;         // row inside the tile
+    const int r = q * 32 + lane;         // row inside the CTA's 128 rows
     const uint32_t sw = (uint32_t)((r >> 1) & 3);
     const uint32_t off0 = (uint32_t)r * 64u + ((((uint32_t)half * 2u) ^ sw) << 4);
     const uint32_t off1 = (uint32_t)r * 64u + ((((uint32_t)half * 2u + 1u) ^ sw) << 4);
@@ -223,18 +311,21 @@ umma_cell_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
     // A thread whose wait ran out (ok = false) keeps walking the loops without touching data, so that the named
     // barrier of the linearisation's store hand-over still sees all 256 epilogue threads.
     bool ok = true;
-    for (int t = blockIdx.x; t < tiles; t += gridDim.x, ++it) {
-      const int mt = t / n_tiles, nt = t % n_tiles;
+    for (int t = cta; t < tiles; t += ncta, ++it) {
+      const int mt = row_tile(t), nt = t % n_tiles;
       const int as = it & 1;
       const uint32_t aphase = (uint32_t)(it >> 1) & 1u;
       const int row = mt * BM + r;
       const bool valid = row < p.M;
       const int k = valid ? row / p.B : 0, b = valid ? row % p.B : 0;
       if (ok && !mbar_wait(tfull_bar(as), aphase, abortp, status, 15)) ok = false;
+      ok = __all_sync(0xffffffffu, ok);      // warp-uniform: the accumulator loads below are warp-collective
       tc_fence_after();
       const uint32_t taddr = tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(as * BN);
       for (int c = 0; c < NCH; ++c) {
+        if (nt * UN + c * CH >= H) break;          // ragged last unit tile (uniform over the CTA)
         if (ok && !mbar_wait(efull_bar(eb), ephase, abortp, status, 16)) ok = false;
+        ok = __all_sync(0xffffffffu, ok);
         if (ok) {
         const uint32_t src = epi_base + eb * C::kEpiBytes;
         float gr[8], gz[8], gn[8], hp[8], gg[8];
@@ -263,7 +354,7 @@ umma_cell_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
           asm volatile("st.shared.b32 [%0], %1;" ::"r"(smem_u32(&lds_sink[threadIdx.x])), "r"(dep) : "memory");
         }
         mbar_arrive(eempty_bar(eb));
-        if (++eb == 2) { eb = 0; ephase ^= 1u; }
+        if (++eb == C::kEpiBufs) { eb = 0; ephase ^= 1u; }
         if (valid) {
           const int u = nt * UN + cu;
           float br[8], bz[8], bn[8];
@@ -314,7 +405,7 @@ umma_cell_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
           asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
           if (storer) asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory");
           asm volatile("bar.sync 1, 256;" ::: "memory");
-          if (storer && ok) {
+          if (storer && ok && mt * BM < p.M) {
             const uint32_t srcb = out_base + ob * C::kOutBytes;
             const int u = nt * UN + c * CH, row0 = mt * BM;
             tma_store_2d(&tmCR, srcb, u, row0);
@@ -327,8 +418,13 @@ umma_cell_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
         }
       }
       if (ok) {
+        // every lane's accumulator loads have completed (tcgen05.wait::ld above); one lane releases for the warp
         tc_fence_before();
-        mbar_arrive(tempty_bar(as));
+        __syncwarp();
+        if (lane == 0) {
+          if (PAIR) mbar_arrive_cluster(mapa_shared(tempty_bar(as), 0));
+          else mbar_arrive(tempty_bar(as));
+        }
       }
     }
     if (LIN && storer) asm volatile("cp.async.bulk.wait_group 0;" ::: "memory");   // coefficients are in global memory before exit
@@ -337,10 +433,12 @@ umma_cell_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
   // ------------------------------------------------------------ teardown
   tc_fence_before();
   __syncthreads();
+  if (PAIR) cluster_sync_all();   // neither CTA leaves (or frees tensor memory) while the other may still signal it
   tc_fence_after();
   if (warp == 1) {
     __syncwarp();
-    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(512u) : "memory");
+    if (PAIR) asm volatile("tcgen05.dealloc.cta_group::2.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(512u) : "memory");
+    else asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(512u) : "memory");
   }
 }
 

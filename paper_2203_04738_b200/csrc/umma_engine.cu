@@ -169,24 +169,33 @@ bool make_map2(CUtensorMap* m, CUtensorMapDataType dt, size_t esize, const void*
   return r == CUDA_SUCCESS;
 }
 
+// The fused kernel on CTA pairs (256 x 240 tiles) is used when the step has at least one full wave of such tiles;
+// smaller steps stay on single CTAs (128 x 192 tiles).  MGRIT_GRU_CELL_PAIR=0 keeps every step on single CTAs.
+static bool cell_pair_enabled(int M, int H) {
+  static int v = -1;
+  if (v < 0) { const char* e = getenv("MGRIT_GRU_CELL_PAIR"); v = (e && e[0] == '0') ? 0 : 1; }
+  return v == 1 && (i64)(M / (2 * BM)) * ((H + 79) / 80) >= kSMs / 2;
+}
+
 // Fused recurrent GEMM + cell (forward step or linearisation) with TMA-staged epilogue operands.
 // Rows (k, b), k = 0..nk-1: A rows at A + k*a_ks + b*H (bf16), gi rows at gi + k*gi_ks + b*3H,
 // previous state at hp + k*hp_ks + b*H, optional additive term at g + k*g_ks + b*H.
-template <bool LIN, bool HAS_G>
-bool launch_cell(int kc, const bf16* A, i64 a_ks, const float* gi, i64 gi_ks, const float* hp, i64 hp_ks, const float* g, i64 g_ks,
-                 int nk, const bf16* W, CellArgs ca, cudaStream_t s) {
-  using C = cellk::CellCfg<HAS_G, LIN>;
+template <bool LIN, bool HAS_G, bool PAIR>
+bool launch_cell_geo(int kc, const bf16* A, i64 a_ks, const float* gi, i64 gi_ks, const float* hp, i64 hp_ks, const float* g, i64 g_ks,
+                     int nk, const bf16* W, CellArgs ca, cudaStream_t s) {
+  using C = cellk::CellCfg<HAS_G, LIN, PAIR>;
+  using G = cellk::Geo<PAIR>;
   if (nk <= 0) return true;
   int* const status = status_ptr();
   if (!status) return false;
   static bool attr_set[kMaxDevices] = {false};
-  auto kern = umma_cell_kernel<LIN, HAS_G>;
+  auto kern = umma_cell_kernel<LIN, HAS_G, PAIR>;
   if (!set_smem_once(kern, C::kSmemBytes, attr_set)) return false;
   const int B = ca.B, H = ca.H, kt = 128 / B;
   ca.kt = kt; ca.M = nk * B;
   CUtensorMap ta, tb, tgi, thp, tg;
   if (!make_map3(&ta, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, A, H, B, nk, H, a_ks, BK, kt, CU_TENSOR_MAP_SWIZZLE_128B)) return false;
-  if (!make_map(&tb, W, (uint64_t)H, (uint64_t)3 * H, (uint64_t)H, cellk::UN)) return false;
+  if (!make_map(&tb, W, (uint64_t)H, (uint64_t)3 * H, (uint64_t)H, G::kBox)) return false;
   if (!make_map3(&tgi, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 4, gi, 3 * H, B, nk, 3 * H, gi_ks, cellk::CH, kt, CU_TENSOR_MAP_SWIZZLE_64B)) return false;
   if (!make_map3(&thp, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 4, hp, H, B, nk, H, hp_ks, cellk::CH, kt, CU_TENSOR_MAP_SWIZZLE_64B)) return false;
   if (HAS_G) {
@@ -202,12 +211,27 @@ bool launch_cell(int kc, const bf16* A, i64 a_ks, const float* gi, i64 gi_ks, co
     };
     if (!cmap(&tcr, ca.cr) || !cmap(&tcz, ca.cz) || !cmap(&tcn, ca.cn) || (ca.cnp && !cmap(&tcp, ca.cnp))) return false;
   }
-  int tiles = ((ca.M + BM - 1) / BM) * (H / cellk::UN);
-  int grid = tiles < kSMs ? tiles : kSMs;
+  constexpr int kTileRows = PAIR ? 2 * BM : BM;
+  const int tiles = ((ca.M + kTileRows - 1) / kTileRows) * ((H + G::UN - 1) / G::UN);
   ProfScope prof_(kc, 2.0 * ca.M * 3.0 * H * H, s);
-  if (launch_pdl(kern, dim3(grid), dim3(cellk::kThreads), C::kSmemBytes, s, ta, tb, tgi, thp, tg, tcr, tcz, tcn, tcp, ca, status) != cudaSuccess) return false;
+  cudaError_t e;
+  if (PAIR) {
+    const int grid = 2 * (tiles < kSMs / 2 ? tiles : kSMs / 2);
+    e = launch_pdl_cluster(kern, 2, dim3(grid), dim3(cellk::kThreads), C::kSmemBytes, s, ta, tb, tgi, thp, tg, tcr, tcz, tcn, tcp, ca, status);
+  } else {
+    const int grid = tiles < kSMs ? tiles : kSMs;
+    e = launch_pdl(kern, dim3(grid), dim3(cellk::kThreads), C::kSmemBytes, s, ta, tb, tgi, thp, tg, tcr, tcz, tcn, tcp, ca, status);
+  }
+  if (e != cudaSuccess) return false;
   count_launch();
   return true;
+}
+template <bool LIN, bool HAS_G>
+bool launch_cell(int kc, const bf16* A, i64 a_ks, const float* gi, i64 gi_ks, const float* hp, i64 hp_ks, const float* g, i64 g_ks,
+                 int nk, const bf16* W, CellArgs ca, cudaStream_t s) {
+  if (cell_pair_enabled(nk * ca.B, ca.H))
+    return launch_cell_geo<LIN, HAS_G, true>(kc, A, a_ks, gi, gi_ks, hp, hp_ks, g, g_ks, nk, W, ca, s);
+  return launch_cell_geo<LIN, HAS_G, false>(kc, A, a_ks, gi, gi_ks, hp, hp_ks, g, g_ks, nk, W, ca, s);
 }
 
 // ---------------------------------------------------------------- epilogues (one output row per thread)

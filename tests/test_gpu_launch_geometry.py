@@ -1,5 +1,6 @@
-"""The same solve on two launch geometries: the plain tensor-core products on CTA pairs (256 x 256 tiles, two CTAs
-per MMA) and on single CTAs (128 x 256 tiles).  Each output element is accumulated over the same k-blocks in the
+"""The same solve on two launch geometries: the tensor-core products on CTA pairs (plain products: 256 x 256 tiles;
+fused recurrent product + cell: 256 x 240 tiles of 80 hidden units; two CTAs per MMA) and on single CTAs (128 x 256
+and 128 x 192 tiles).  Each output element is accumulated over the same k-blocks in the
 same order either way, so the results may differ by rounding of the accumulation inside the tensor core at most:
 every output must agree to 1e-5 of its largest magnitude (bf16-operand noise is 100 times that).  The shape makes
 the projection (40960 x 1536), the level-0 adjoint steps (10240 x 512) and the input gradient (40960 x 256) multi-wave
@@ -40,7 +41,7 @@ def test_pair_and_single_cta_products_agree(tmp_path):
     outs = []
     for flag in ("1", "0"):
         out = str(tmp_path / f"geo{flag}.npz")
-        env = dict(os.environ, MGRIT_GRU_GEMM_PAIR=flag, PYTHONPATH=root)
+        env = dict(os.environ, MGRIT_GRU_GEMM_PAIR=flag, MGRIT_GRU_CELL_PAIR=flag, PYTHONPATH=root)
         subprocess.run([sys.executable, "-c", CHILD, out], check=True, env=env, cwd=root, timeout=600)
         outs.append(np.load(out))
     a, b = outs

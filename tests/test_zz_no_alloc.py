@@ -10,6 +10,7 @@ in the shared array); no device memory is allocated by a call; and a clear error
 limit.  Passes alone in a fresh process and after the other tests.
 """
 import ctypes
+import gc
 
 import numpy as np
 import pytest
@@ -44,12 +45,18 @@ def test_noalloc_head_matches_workspace_head_twice_in_a_row():
             assert float(np.max(np.abs(a.cpu().numpy() - b))) <= 1e-3 * float(np.max(np.abs(b))) + 1e-7, call
         # The set-up call above resolved the built-in array's address.  From here on a call must leave the
         # device's memory as it found it: nothing allocated through torch, nothing taken from the driver.
-        torch.cuda.synchronize()
-        free0, alloc0, reserved0 = torch.cuda.mem_get_info()[0], torch.cuda.memory_allocated(), torch.cuda.memory_reserved()
-        B.xent_head_fwd_bwd_noalloc(hT, Wc, bc, lab, out=out)
-        torch.cuda.synchronize()
-        assert torch.cuda.mem_get_info()[0] == free0 and torch.cuda.memory_allocated() == alloc0
-        assert torch.cuda.memory_reserved() == reserved0
+        # (Python's cycle collector is held off meanwhile: it may free tensors of earlier tests at any moment.)
+        gc.collect()
+        gc.disable()
+        try:
+            torch.cuda.synchronize()
+            free0, alloc0, reserved0 = torch.cuda.mem_get_info()[0], torch.cuda.memory_allocated(), torch.cuda.memory_reserved()
+            B.xent_head_fwd_bwd_noalloc(hT, Wc, bc, lab, out=out)
+            torch.cuda.synchronize()
+            assert torch.cuda.mem_get_info()[0] == free0 and torch.cuda.memory_allocated() == alloc0
+            assert torch.cuda.memory_reserved() == reserved0
+        finally:
+            gc.enable()
     assert B.last_device_status() == 0
 
 
