@@ -103,7 +103,7 @@ int check_cfg(const mgrit_gru_cfg* c, Hier* hr) {
 
 struct FwdWs {
   float* U[kMaxLevels]; float* G[kMaxLevels]; double* res_acc; UmmaFwdWs um;
-  __nv_bfloat16* chain_ub; unsigned* chain_bar;   // scratch of the persistent serial-chain kernel
+  __nv_bfloat16* chain_ub; unsigned* chain_bar; uint4* chain_xw; size_t chain_xw_bytes;   // scratch of the persistent serial-chain kernel
   __nv_bfloat16* Ub[kMaxLevels];                  // bf16 copies of the level states (tensor-core A operands)
 };
 struct AdjWs {
@@ -111,7 +111,7 @@ struct AdjWs {
   float *a[kMaxLevels], *cr[kMaxLevels], *cz[kMaxLevels], *cn[kMaxLevels], *cnp;   // gate coefficients: fp32 engine
   __nv_bfloat16 *crb[kMaxLevels], *czb[kMaxLevels], *cnb[kMaxLevels], *cnpb;       // ... tensor-core engine (bf16)
   float *dA_h, *dA_i, *lam_tmp; double* res_acc; UmmaAdjWs um;
-  __nv_bfloat16* chain_dAb; unsigned* chain_bar;
+  __nv_bfloat16* chain_dAb; unsigned* chain_bar; uint4* chain_xw; size_t chain_xw_bytes;
 };
 
 void plan_fwd(const mgrit_gru_cfg* c, const Hier& hr, Ws& w, FwdWs* o) {
@@ -121,13 +121,15 @@ void plan_fwd(const mgrit_gru_cfg* c, const Hier& hr, Ws& w, FwdWs* o) {
     o->G[l] = l == 0 ? nullptr : w.take<float>((size_t)(hr.N[l] + 1) * BH);
   }
   o->res_acc = w.take<double>((size_t)(c->iters > 0 ? c->iters : 1));
-  o->chain_ub = nullptr; o->chain_bar = nullptr;
+  o->chain_ub = nullptr; o->chain_bar = nullptr; o->chain_xw = nullptr; o->chain_xw_bytes = 0;
   for (int l = 0; l < kMaxLevels; ++l) o->Ub[l] = nullptr;
   if (c->operands == MGRIT_OPERANDS_BF16) {
     umma_plan_fwd(c, hr.N, hr.L, w.base, &w.off, &o->um);
     for (int l = 0; l < hr.L; ++l) o->Ub[l] = w.take<__nv_bfloat16>((size_t)(hr.N[l] + 1) * BH);
     o->chain_ub = w.take<__nv_bfloat16>(2 * BH);
     o->chain_bar = w.take<unsigned>(((size_t)c->B / 16 + 1) * ((size_t)c->H / 8) + 64);
+    o->chain_xw_bytes = serial_xw_bytes(c->B, c->H, 1);
+    o->chain_xw = reinterpret_cast<uint4*>(w.take<char>(o->chain_xw_bytes));
   }
 }
 
@@ -157,8 +159,10 @@ void plan_adj(const mgrit_gru_cfg* c, const Hier& hr, Ws& w, AdjWs* o) {
     umma_plan_adj(c, hr.N, hr.L, w.base, &w.off, &o->um);
     o->chain_dAb = w.take<__nv_bfloat16>(6 * BH);
     o->chain_bar = w.take<unsigned>(((size_t)c->B / 16 + 1) * ((size_t)c->H / 8) + 64);
+    o->chain_xw_bytes = serial_xw_bytes(c->B, c->H, 3);
+    o->chain_xw = reinterpret_cast<uint4*>(w.take<char>(o->chain_xw_bytes));
   } else {
-    o->chain_dAb = nullptr; o->chain_bar = nullptr;
+    o->chain_dAb = nullptr; o->chain_bar = nullptr; o->chain_xw = nullptr; o->chain_xw_bytes = 0;
     o->dA_h = w.take<float>((size_t)c->T * BH * 3);
     o->dA_i = w.take<float>((size_t)c->T * BH * 3);
     o->lam_tmp = w.take<float>((size_t)c->T * BH);     // lambda in forward order when the caller wants no dh
@@ -242,6 +246,7 @@ struct FwdCycle : Cycle {
     i64 st = hr.stride_t[l];
     a.gi = gi + (st - 1) * (i64)BH * 3; a.gi_step = st * (i64)BH * 3;
     a.g = G[l]; a.W = um->W_hh; a.b_hh = p->b_hh; a.gamma = hr.gamma[l]; a.cell = c->cell; a.bar = fw->chain_bar;
+    a.xw = fw->chain_xw; a.xw_bytes = fw->chain_xw_bytes;
     return serial_fwd_solve(a, s);
   }
   int launch_step(const StepDesc& d) override {
@@ -272,6 +277,7 @@ struct AdjCycle : Cycle {
     a.a = w->a[l] + row0; a.cr = w->crb[l] + row0; a.cz = w->czb[l] + row0; a.cn = w->cnb[l] + row0;
     a.coef_step = -(i64)BH;
     a.g = G[l]; a.WT = w->um.W_hhT; a.bar = w->chain_bar;
+    a.xw = w->chain_xw; a.xw_bytes = w->chain_xw_bytes;
     return serial_adj_solve(a, s);
   }
   int launch_step(const StepDesc& d) override {

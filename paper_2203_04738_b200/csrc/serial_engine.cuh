@@ -15,6 +15,7 @@ struct SerialFwdArgs {
   const float* b_hh;
   float gamma; int cell;
   unsigned* bar;                 // [ceil(B/16)] barrier counters (scratch)
+  uint4* xw; size_t xw_bytes;    // exchange words of the flag-in-data hand-over (scratch, serial_xw_bytes()), or nullptr
 };
 
 // mu_s = a_s*mu_{s-1} + ([cr_s|cz_s|cn_s]*mu_{s-1}) W_hh + g_s,  s = 1..nsteps
@@ -28,7 +29,11 @@ struct SerialAdjArgs {
   const float* g;                // [nsteps+1][B][H] or nullptr
   const __nv_bfloat16* WT;       // [H][3H] = W_hh^T
   unsigned* bar;
+  uint4* xw; size_t xw_bytes;    // as in SerialFwdArgs (three gate blocks per producer)
 };
+
+// bytes of exchange words for a chain over B rows of H units carrying `gates` values per (row, unit)
+size_t serial_xw_bytes(int B, int H, int gates);
 
 bool serial_fwd_supported(int B, int H);
 bool serial_adj_supported(int B, int H);

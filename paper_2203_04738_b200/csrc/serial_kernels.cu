@@ -7,6 +7,8 @@
 //
 // A wait that runs out writes a non-zero code to the status word; every CTA that sees a non-zero
 // status leaves at its next barrier, so the launch always terminates.
+#include <stdlib.h>
+
 #include "cell.cuh"
 #include "serial_engine.cuh"
 
@@ -68,6 +70,82 @@ __device__ __forceinline__ void cp_async_wait_all() {
   asm volatile("cp.async.commit_group;\n\tcp.async.wait_group 0;" ::: "memory");
 }
 
+// ---- exchange of the new state between CTAs with the "ready" flag inside the data --------------------------------
+// A 16-byte word carries six bf16 values and the number of the step that produced them; it is written by ONE
+// 16-byte store of one thread (a single transaction inside one 32-byte sector), so a reader that sees the step
+// number sees the six values too.  Readers poll the words they need directly: one trip to L2 once the data is
+// there, instead of an arrival counter, a poll of that counter and a reload.  Two buffers alternate by step
+// parity: a CTA writes step j + 2 only after it has read all of step j + 1, which nobody could produce before
+// reading all of step j.  The host clears the words before every launch (step numbers start at 1).
+constexpr int kValsPerWord = 6;
+__device__ __forceinline__ uint4 ld_word(const uint4* p) {
+  uint4 v;
+  asm volatile("ld.volatile.global.v4.u32 {%0,%1,%2,%3}, [%4];" : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "l"(p) : "memory");
+  return v;
+}
+__device__ __forceinline__ void st_word(uint4* p, uint4 v) {
+  asm volatile("st.volatile.global.v4.u32 [%0], {%1,%2,%3,%4};" ::"l"(p), "r"(v.x), "r"(v.y), "r"(v.z), "r"(v.w) : "memory");
+}
+// Words of one producer block of `nvals` bf16 values (a multiple of 2) staged in shared memory -> global, tagged `step`.
+__device__ __forceinline__ void publish_block(const bf16* stage, int nvals, uint4* dst, unsigned step) {
+  const int nwords = (nvals + kValsPerWord - 1) / kValsPerWord;
+  for (int w = threadIdx.x; w < nwords; w += kThreads) {
+    const uint32_t* s32 = reinterpret_cast<const uint32_t*>(stage) + 3 * w;      // values 6w .. 6w+5 as three pairs
+    uint4 v;
+    v.x = 6 * w < nvals ? s32[0] : 0u;
+    v.y = 6 * w + 2 < nvals ? s32[1] : 0u;
+    v.z = 6 * w + 4 < nvals ? s32[2] : 0u;
+    v.w = step;
+    st_word(dst + w, v);
+  }
+}
+// All producers' blocks of step `step` -> the CTA's operand rows in shared memory.  A block holds GATES x 16 x UNC
+// values in the order [gate][row][unit]; value (g, r, i) of producer x goes to As[r][g*H + x*UNC + i].
+// Every round a thread issues the loads of all its words that are still missing together and then looks at what
+// came back, so a round costs one trip to L2 however many words are outstanding.
+template <int UNC, int GATES>
+__device__ __forceinline__ bool gather_blocks(const uint4* src, int nprod, unsigned step, bf16* As, int ldk, int H, int* status) {
+  constexpr int kBlockVals = GATES * kRows * UNC, kBlockWords = (kBlockVals + kValsPerWord - 1) / kValsPerWord;
+  constexpr int kBatch = GATES == 1 ? 12 : 16;
+  const int total = nprod * kBlockWords;
+  for (int base = threadIdx.x; base < total; base += kThreads * kBatch) {
+    unsigned pending = 0;
+#pragma unroll
+    for (int q = 0; q < kBatch; ++q)
+      if (base + q * kThreads < total) pending |= 1u << q;
+    unsigned rounds = 0;
+    uint64_t t0 = 0;
+    while (pending) {
+      uint4 v[kBatch];
+#pragma unroll
+      for (int q = 0; q < kBatch; ++q)
+        if (pending & (1u << q)) v[q] = ld_word(src + base + q * kThreads);
+#pragma unroll
+      for (int q = 0; q < kBatch; ++q) {
+        if ((pending & (1u << q)) && v[q].w == step) {
+          pending &= ~(1u << q);
+          const int e = base + q * kThreads, x = e / kBlockWords, w = e % kBlockWords;
+          const uint32_t d[3] = {v[q].x, v[q].y, v[q].z};
+#pragma unroll
+          for (int t = 0; t < 3; ++t) {
+            const int vv = kValsPerWord * w + 2 * t;
+            if (vv < kBlockVals) {
+              const int g = vv / (kRows * UNC), r = (vv / UNC) % kRows, i = vv % UNC;
+              *reinterpret_cast<uint32_t*>(As + r * ldk + g * H + x * UNC + i) = d[t];
+            }
+          }
+        }
+      }
+      if (pending && (++rounds & 31u) == 0) {      // bounded: give up once the status word is set or after the limit
+        if (t0 == 0) t0 = global_ns();
+        if (ld_relaxed(status) != 0) return false;
+        if (global_ns() - t0 > kWaitLimitNs) { atomicCAS(status, 0, 6); return false; }
+      }
+    }
+  }
+  return true;
+}
+
 __device__ __forceinline__ void mma16816(float* c, const uint32_t* a, uint32_t b0, uint32_t b1) {
   asm volatile(
       "mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
@@ -117,9 +195,11 @@ __device__ __forceinline__ float sum_partials(const float* red, int row, int col
 
 // ------------------------------------------------------------------------------------------------
 // forward chain:  u_j = Phi_gamma(gi_j, u_{j-1}) + g_j ,  j = 1..nsteps
-template <int UNC>
+template <int UNC, bool LL>
 __global__ void __launch_bounds__(kThreads, 1) serial_fwd_kernel(SerialFwdArgs a, int* status) {
   constexpr int NW = 3 * UNC, NT = NW / 8, OPT = (kRows * UNC + kThreads - 1) / kThreads;
+  constexpr int kBlockVals = kRows * UNC, kBlockWords = (kBlockVals + kValsPerWord - 1) / kValsPerWord;
+  __shared__ __align__(16) bf16 xstage[kRows * 32];
   extern __shared__ __align__(16) uint8_t smem[];
   const int H = a.H, ldk = H + 8;
   bf16* Ws = reinterpret_cast<bf16*>(smem);                 // [NW][ldk]
@@ -141,6 +221,7 @@ __global__ void __launch_bounds__(kThreads, 1) serial_fwd_kernel(SerialFwdArgs a
   }
   // rows beyond the batch stay zero
   for (int e = tid; e < kRows * ldk / 2; e += kThreads) reinterpret_cast<uint32_t*>(As)[e] = 0u;
+  if (tid == 0) ok_smem = 1;
   __syncthreads();
   // step 1 reads the fp32 initial state
   for (int e = tid; e < nrows * (H / 4); e += kThreads) {
@@ -177,18 +258,24 @@ __global__ void __launch_bounds__(kThreads, 1) serial_fwd_kernel(SerialFwdArgs a
 #pragma unroll
     for (int o = 0; o < OPT; ++o) {
       int idx = tid + o * kThreads, r = idx / UNC, i = idx % UNC;
+      float val = 0.f;
       if (idx < kRows * UNC && r < nrows) {
         float ghr = sum_partials<NW>(red, r, i) + br[o];
         float ghz = sum_partials<NW>(red, r, UNC + i) + bz[o];
         float ghn = sum_partials<NW>(red, r, 2 * UNC + i) + bn[o];
-        float val = cell_forward<true>(pgr[o], pgz[o], pgn[o], ghr, ghz, ghn, hp[o], a.gamma, a.cell) + pg[o];
+        val = cell_forward<true>(pgr[o], pgz[o], pgn[o], ghr, ghz, ghn, hp[o], a.gamma, a.cell) + pg[o];
         hp[o] = val;
         i64 off = (i64)(row0 + r) * H + u0 + i;
         a.u[(i64)j * BH + off] = val;
-        ub[off] = __float2bfloat16(val);
+        if (!LL) ub[off] = __float2bfloat16(val);
       }
+      if (LL && idx < kRows * UNC) xstage[idx] = __float2bfloat16(val);      // rows beyond the batch travel as zeros
     }
     if (j == a.nsteps) break;
+    if (LL) {
+      __syncthreads();
+      publish_block(xstage, kBlockVals, a.xw + ((i64)(rg * 2 + (j & 1)) * gridDim.x + blockIdx.x) * kBlockWords, (unsigned)j);
+    }
     // operands of the next step that do not depend on other CTAs
 #pragma unroll
     for (int o = 0; o < OPT; ++o) {
@@ -199,23 +286,34 @@ __global__ void __launch_bounds__(kThreads, 1) serial_fwd_kernel(SerialFwdArgs a
         if (a.g) pg[o] = a.g[(i64)(j + 1) * BH + (i64)(row0 + r) * H + u0 + i];
       }
     }
-    if (!grid_barrier(a.bar + rg, (unsigned)j * ncta_rg, status, &ok_smem)) return;
-    // the full new state of this row group, as the bf16 A operand
-    for (int e = tid; e < nrows * (H / 8); e += kThreads) {
-      int r = e / (H / 8), c = e % (H / 8);
-      cp_async16(As + r * ldk + c * 8, ub + (i64)(row0 + r) * H + c * 8);
+    if (LL) {
+      // the full new state of this row group, as the bf16 A operand: every producer's words, polled in place
+      const bool ok = gather_blocks<UNC, 1>(a.xw + (i64)(rg * 2 + (j & 1)) * gridDim.x * kBlockWords, (int)gridDim.x, (unsigned)j, As, ldk,
+                                            H, status);
+      if (!ok) ok_smem = 0;
+      __syncthreads();
+      if (ok_smem == 0) return;
+    } else {
+      if (!grid_barrier(a.bar + rg, (unsigned)j * ncta_rg, status, &ok_smem)) return;
+      // the full new state of this row group, as the bf16 A operand
+      for (int e = tid; e < nrows * (H / 8); e += kThreads) {
+        int r = e / (H / 8), c = e % (H / 8);
+        cp_async16(As + r * ldk + c * 8, ub + (i64)(row0 + r) * H + c * 8);
+      }
+      cp_async_wait_all();
+      __syncthreads();
     }
-    cp_async_wait_all();
-    __syncthreads();
   }
 }
 
 // ------------------------------------------------------------------------------------------------
 // adjoint chain:  mu_s = a_s * mu_{s-1} + [cr_s|cz_s|cn_s]*mu_{s-1} W_hh + g_s ,  s = 1..nsteps
 // The bf16 operand copy carries dA_{s+1} = [cr|cz|cn]_{s+1} * mu_s, formed by the CTA that produced mu_s.
-template <int UNC>
+template <int UNC, bool LL>
 __global__ void __launch_bounds__(kThreads, 1) serial_adj_kernel(SerialAdjArgs a, int* status) {
   constexpr int NT = UNC / 8, OPT = (kRows * UNC + kThreads - 1) / kThreads;
+  constexpr int kBlockVals = 3 * kRows * UNC, kBlockWords = (kBlockVals + kValsPerWord - 1) / kValsPerWord;
+  __shared__ __align__(16) bf16 xstage[3 * kRows * 32];
   extern __shared__ __align__(16) uint8_t smem[];
   const int H = a.H, K = 3 * H, ldk = K + 8;
   bf16* Ws = reinterpret_cast<bf16*>(smem);                 // [UNC][ldk]   rows of W_hh^T
@@ -233,6 +331,7 @@ __global__ void __launch_bounds__(kThreads, 1) serial_adj_kernel(SerialAdjArgs a
     *reinterpret_cast<uint4*>(Ws + r * ldk + c * 8) = __ldg(reinterpret_cast<const uint4*>(a.WT + (i64)(u0 + r) * K + c * 8));
   }
   for (int e = tid; e < kRows * ldk / 2; e += kThreads) reinterpret_cast<uint32_t*>(As)[e] = 0u;
+  if (tid == 0) ok_smem = 1;
   __syncthreads();
   // step 1: dA_1 = c_1 * mu_0 for all 3H columns of this row group
   for (int e = tid; e < nrows * H; e += kThreads) {
@@ -273,20 +372,31 @@ __global__ void __launch_bounds__(kThreads, 1) serial_adj_kernel(SerialAdjArgs a
 #pragma unroll
     for (int o = 0; o < OPT; ++o) {
       int idx = tid + o * kThreads, r = idx / UNC, i = idx % UNC;
-      if (idx < kRows * UNC && r < nrows) {
-        float val = pa[o] * mp[o] + sum_partials<UNC>(red, r, i) + pg[o];
+      float val = 0.f;
+      const bool live = idx < kRows * UNC && r < nrows;
+      if (live) {
+        val = pa[o] * mp[o] + sum_partials<UNC>(red, r, i) + pg[o];
         mp[o] = val;
         i64 off = (i64)(row0 + r) * H + u0 + i;
         a.mu[(i64)s * BH + off] = val;
-        if (s < a.nsteps) {
+        if (!LL && s < a.nsteps) {
           bf16* d = dAb + (i64)(row0 + r) * K + u0 + i;
           d[0] = __float2bfloat16(__bfloat162float(ncr[o]) * val);
           d[H] = __float2bfloat16(__bfloat162float(ncz[o]) * val);
           d[2 * H] = __float2bfloat16(__bfloat162float(ncn[o]) * val);
         }
       }
+      if (LL && idx < kRows * UNC) {     // block order [gate][row][unit]; rows beyond the batch travel as zeros
+        xstage[idx] = __float2bfloat16(live ? __bfloat162float(ncr[o]) * val : 0.f);
+        xstage[kRows * UNC + idx] = __float2bfloat16(live ? __bfloat162float(ncz[o]) * val : 0.f);
+        xstage[2 * kRows * UNC + idx] = __float2bfloat16(live ? __bfloat162float(ncn[o]) * val : 0.f);
+      }
     }
     if (s == a.nsteps) break;
+    if (LL) {
+      __syncthreads();
+      publish_block(xstage, kBlockVals, a.xw + ((i64)(rg * 2 + (s & 1)) * gridDim.x + blockIdx.x) * kBlockWords, (unsigned)s);
+    }
 #pragma unroll
     for (int o = 0; o < OPT; ++o) {
       int idx = tid + o * kThreads, r = idx / UNC, i = idx % UNC;
@@ -300,13 +410,21 @@ __global__ void __launch_bounds__(kThreads, 1) serial_adj_kernel(SerialAdjArgs a
         }
       }
     }
-    if (!grid_barrier(a.bar + rg, (unsigned)s * ncta_rg, status, &ok_smem)) return;
-    for (int e = tid; e < nrows * (K / 8); e += kThreads) {
-      int r = e / (K / 8), c = e % (K / 8);
-      cp_async16(As + r * ldk + c * 8, dAb + (i64)(row0 + r) * K + c * 8);
+    if (LL) {
+      const bool ok = gather_blocks<UNC, 3>(a.xw + (i64)(rg * 2 + (s & 1)) * gridDim.x * kBlockWords, (int)gridDim.x, (unsigned)s, As, ldk,
+                                            H, status);
+      if (!ok) ok_smem = 0;
+      __syncthreads();
+      if (ok_smem == 0) return;
+    } else {
+      if (!grid_barrier(a.bar + rg, (unsigned)s * ncta_rg, status, &ok_smem)) return;
+      for (int e = tid; e < nrows * (K / 8); e += kThreads) {
+        int r = e / (K / 8), c = e % (K / 8);
+        cp_async16(As + r * ldk + c * 8, dAb + (i64)(row0 + r) * K + c * 8);
+      }
+      cp_async_wait_all();
+      __syncthreads();
     }
-    cp_async_wait_all();
-    __syncthreads();
   }
 }
 
@@ -321,7 +439,7 @@ int* status_ptr() {     // status word of the current device, nullptr on failure
   return g_serial_status_ptrs[dev];
 }
 
-constexpr size_t kSmemLimit = 227 * 1024 - 64;
+constexpr size_t kSmemLimit = 227 * 1024 - 4096;   // dynamic part: the kernels also hold up to 3 KiB of static shared memory
 int g_sm_count[kMaxDevices] = {0};
 int sm_count() {
   const int dev = current_device_slot();
@@ -353,11 +471,23 @@ int pick_unc(int B, int H, bool adj) {
   return 0;
 }
 
+// MGRIT_GRU_CHAIN_LL=0 in the environment selects the counter barrier + reload instead of the flag-in-data exchange.
+bool chain_ll_enabled() {
+  static int v = -1;
+  if (v < 0) { const char* e = getenv("MGRIT_GRU_CHAIN_LL"); v = (e && e[0] == '0') ? 0 : 1; }
+  return v == 1;
+}
+
 template <class Args, class Kern>
-bool launch_coop(Kern kern, const Args& a, int unc, size_t smem, cudaStream_t s) {
+bool launch_coop(Kern kern, const Args& a, int unc, size_t smem, bool ll, int gates, cudaStream_t s) {
   if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess) return false;
   int rgs = (a.B + kRows - 1) / kRows;
   if (cudaMemsetAsync(a.bar, 0, sizeof(unsigned) * rgs, s) != cudaSuccess) return false;
+  if (ll) {   // no word may carry a step number of an earlier launch
+    const size_t words = (size_t)rgs * 2 * (a.H / unc) * ((size_t)(gates * kRows * unc + kValsPerWord - 1) / kValsPerWord);
+    if (words * sizeof(uint4) > a.xw_bytes) return false;
+    if (cudaMemsetAsync(a.xw, 0, words * sizeof(uint4), s) != cudaSuccess) return false;
+  }
   Args args = a;
   int* st = status_ptr();
   if (!st) return false;
@@ -373,6 +503,12 @@ bool launch_coop(Kern kern, const Args& a, int unc, size_t smem, cudaStream_t s)
 
 }  // namespace
 
+size_t serial_xw_bytes(int B, int H, int gates) {
+  // the smallest unit slice (8) has the most words: 2 parities x row groups x (H / 8) producers x ceil(gates*16*8 / 6)
+  const size_t rgs = (size_t)(B + kRows - 1) / kRows;
+  return rgs * 2 * (size_t)(H / 8) * (size_t)((gates * kRows * 8 + kValsPerWord - 1) / kValsPerWord) * sizeof(uint4) + 256;
+}
+
 bool serial_fwd_supported(int B, int H) { return pick_unc(B, H, false) != 0; }
 bool serial_adj_supported(int B, int H) { return pick_unc(B, H, true) != 0; }
 
@@ -381,9 +517,13 @@ bool serial_fwd_solve(const SerialFwdArgs& a, cudaStream_t s) {
   if (unc == 0 || a.nsteps <= 0 || !status_ptr()) return false;
   size_t smem = fwd_smem(unc, a.H);
   prof_begin(KC_FWD_SERIAL, 2.0 * a.B * 3.0 * a.H * a.H * a.nsteps, s);
-  bool ok = unc == 8 ? launch_coop(serial_fwd_kernel<8>, a, unc, smem, s)
-          : unc == 16 ? launch_coop(serial_fwd_kernel<16>, a, unc, smem, s)
-                      : launch_coop(serial_fwd_kernel<32>, a, unc, smem, s);
+  const bool ll = chain_ll_enabled() && a.xw != nullptr;
+  bool ok = ll ? (unc == 8 ? launch_coop(serial_fwd_kernel<8, true>, a, unc, smem, true, 1, s)
+                  : unc == 16 ? launch_coop(serial_fwd_kernel<16, true>, a, unc, smem, true, 1, s)
+                              : launch_coop(serial_fwd_kernel<32, true>, a, unc, smem, true, 1, s))
+               : (unc == 8 ? launch_coop(serial_fwd_kernel<8, false>, a, unc, smem, false, 1, s)
+                  : unc == 16 ? launch_coop(serial_fwd_kernel<16, false>, a, unc, smem, false, 1, s)
+                              : launch_coop(serial_fwd_kernel<32, false>, a, unc, smem, false, 1, s));
   prof_end(s);
   return ok;
 }
@@ -393,9 +533,13 @@ bool serial_adj_solve(const SerialAdjArgs& a, cudaStream_t s) {
   if (unc == 0 || a.nsteps <= 0 || !status_ptr()) return false;
   size_t smem = adj_smem(unc, a.H);
   prof_begin(KC_ADJ_SERIAL, 2.0 * a.B * 3.0 * a.H * a.H * a.nsteps, s);
-  bool ok = unc == 8 ? launch_coop(serial_adj_kernel<8>, a, unc, smem, s)
-          : unc == 16 ? launch_coop(serial_adj_kernel<16>, a, unc, smem, s)
-                      : launch_coop(serial_adj_kernel<32>, a, unc, smem, s);
+  const bool ll = chain_ll_enabled() && a.xw != nullptr;
+  bool ok = ll ? (unc == 8 ? launch_coop(serial_adj_kernel<8, true>, a, unc, smem, true, 3, s)
+                  : unc == 16 ? launch_coop(serial_adj_kernel<16, true>, a, unc, smem, true, 3, s)
+                              : launch_coop(serial_adj_kernel<32, true>, a, unc, smem, true, 3, s))
+               : (unc == 8 ? launch_coop(serial_adj_kernel<8, false>, a, unc, smem, false, 3, s)
+                  : unc == 16 ? launch_coop(serial_adj_kernel<16, false>, a, unc, smem, false, 3, s)
+                              : launch_coop(serial_adj_kernel<32, false>, a, unc, smem, false, 3, s));
   prof_end(s);
   return ok;
 }
