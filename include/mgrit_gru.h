@@ -51,27 +51,39 @@ enum {
 };
 
 enum { MGRIT_CELL_CLASSIC = 0, MGRIT_CELL_IMPLICIT = 1 };
-enum { MGRIT_RELAX_F = 0, MGRIT_RELAX_FCF = 1 };
+/* relaxation = n means F (CF)^n: F-relaxation followed by n C- and F-sweeps (Eq. "fcf-relax" is n = 1) */
+enum { MGRIT_RELAX_F = 0, MGRIT_RELAX_FCF = 1, MGRIT_RELAX_FCFCF = 2, MGRIT_RELAX_MAX = 8 };
 enum { MGRIT_OPERANDS_FP32 = 0, MGRIT_OPERANDS_BF16 = 2 };
-enum { MGRIT_FLAG_SKIP_DUPLICATE_FRELAX = 1 };
+enum {
+  MGRIT_FLAG_SKIP_DUPLICATE_FRELAX = 1,
+  /* F-cycles instead of V-cycles: when the correction of a level has been spread by its final F-relaxation, one
+   * more V-cycle is run from that level down (on the last two levels: two V-cycles).  The paper's Algorithm
+   * "MGProp" with the recursion of remark "Beyond Two-Level" is the V-cycle; the F-cycle is the usual multigrid
+   * variant of it.  resnorm keeps one entry per cycle: the level-0 residual of the cycle's first visit. */
+  MGRIT_FLAG_F_CYCLE = 2,
+  /* Accept any T >= cf^(levels-1): the C-points of a level are its points 0, cf, 2 cf, ...; what follows the last
+   * one is a shorter last interval of F-points, so N_{l+1} = floor(N_l / cf).  The forward grids are anchored at
+   * t = 0, the adjoint's reversed grids at t = T (the paper always uses T = 128 = a multiple of cf^(levels-1)). */
+  MGRIT_FLAG_RAGGED_T = 4
+};
 
 /* Problem and cycle description (Algorithm "MGProp", remark "Beyond Two-Level", Section
  * "Coarse Grid Propagators").  Level l has N_l = T / cf^l points and time step cf^l * dt. */
 typedef struct {
   int32_t T, B, I, H;   /* sequence length, batch, input width, hidden width; H % 8 == 0, I % 8 == 0 */
   int32_t cf;           /* coarsening factor c_f >= 2 */
-  int32_t levels;       /* >= 1; 1 = plain serial sweep; needs T % cf^(levels-1) == 0 */
+  int32_t levels;       /* >= 1; 1 = plain serial sweep; needs T % cf^(levels-1) == 0 unless MGRIT_FLAG_RAGGED_T */
   int32_t iters;        /* number of MGRIT cycles (ForwardIters / BackwardIters of Algorithm "MGRITTraining") */
   int32_t cell;         /* MGRIT_CELL_CLASSIC: Eq. "gru-classic"; MGRIT_CELL_IMPLICIT: Eq. "gru-imap"; same on all levels */
-  int32_t relax_fine;   /* relaxation on level 0: MGRIT_RELAX_F or MGRIT_RELAX_FCF (Eq. "fcf-relax") */
+  int32_t relax_fine;   /* relaxation on level 0: MGRIT_RELAX_F, MGRIT_RELAX_FCF (Eq. "fcf-relax"), MGRIT_RELAX_FCFCF, ... */
   int32_t relax_coarse; /* relaxation on levels 1 .. levels-2 */
   int32_t operands;     /* MGRIT_OPERANDS_FP32: FFMA everywhere; MGRIT_OPERANDS_BF16: bf16 tensor-core
                            operands with fp32 accumulation; states, gates and gradients stay fp32 (the
                            adjoint's gate coefficients, which only ever enter such operands, are kept
                            in bf16 inside the workspace) */
-  int32_t flags;        /* MGRIT_FLAG_SKIP_DUPLICATE_FRELAX: a cycle after the first starts from C-points
-                           whose F-points the previous cycle's final F-relaxation already filled; skip
-                           re-doing it (results are identical) */
+  int32_t flags;        /* OR of MGRIT_FLAG_*.  MGRIT_FLAG_SKIP_DUPLICATE_FRELAX: a cycle after the first starts
+                           from C-points whose F-points the previous cycle's final F-relaxation already filled;
+                           skip re-doing it (results are identical) */
   float dt;             /* fine time step (1.0 in every experiment of the paper) */
 } mgrit_gru_cfg;
 

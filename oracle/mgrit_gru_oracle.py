@@ -37,8 +37,11 @@ import numpy as np
 
 CELL_CLASSIC = 0   # explicit Euler propagator, Eq. "gru-classic"
 CELL_IMPLICIT = 1  # Implicit GRU propagator, Eq. "gru-imap"
-RELAX_F = 0
-RELAX_FCF = 1
+RELAX_F = 0        # F-relaxation
+RELAX_FCF = 1      # F, then C, then F (Eq. "fcf-relax")
+RELAX_FCFCF = 2    # ... and C, F once more; in general relax = n means F (CF)^n
+CYCLE_V = 0        # Algorithm "MGProp" with one recursive coarse solve per level (remark "Beyond Two-Level")
+CYCLE_F = 1        # F-cycle: after the correction of a level, one more V-cycle from that level down
 
 
 # --------------------------------------------------------------------------- cell
@@ -163,16 +166,26 @@ def serial_backward(W_ih, W_hh, b_ih, b_hh, x, h0, h, dh_seed, cell=CELL_IMPLICI
 
 
 # --------------------------------------------------------------------------- MGRIT cycle
-def level_sizes(T, cf, levels):
-    """N_l = T / c_f^l (e.g. 128/32/8 for c_f = 4 and three levels)."""
+def level_sizes(T, cf, levels, ragged=False):
+    """N_l = T / c_f^l (e.g. 128/32/8 for c_f = 4 and three levels).
+
+    ragged=True admits any T: the C-points of a level are its points 0, c_f, 2 c_f, ...; what follows the last of
+    them is a shorter last interval of F-points only, so N_{l+1} = floor(N_l / c_f) (at least one point per level)."""
     if cf < 2 or levels < 1:
         raise ValueError("cf >= 2 and levels >= 1 required")
-    if T % (cf ** (levels - 1)) != 0:
-        raise ValueError("T must be divisible by cf^(levels-1)")
-    return [T // cf ** l for l in range(levels)]
+    if not ragged:
+        if T % (cf ** (levels - 1)) != 0:
+            raise ValueError("T must be divisible by cf^(levels-1)")
+        return [T // cf ** l for l in range(levels)]
+    N = [T]
+    for _ in range(levels - 1):
+        N.append(N[-1] // cf)
+    if N[-1] < 1:
+        raise ValueError("too many levels for this T")
+    return N
 
 
-def fas_vcycle(step, N, cf, relax, u, g, l=0, resnorm=None):
+def fas_vcycle(step, N, cf, relax, u, g, l=0, resnorm=None, cycle=CYCLE_V):
     """One multigrid cycle on level l (Algorithm "MGProp" with the recursive coarse solve of
     the remark "Beyond Two-Level"), for the level-l system
 
@@ -180,7 +193,10 @@ def fas_vcycle(step, N, cf, relax, u, g, l=0, resnorm=None):
 
     step(l, j, u_prev): j is an integer array of target points, u_prev their predecessors'
     states; all entries are independent (the "ParallelFor" of Algorithm "F-relaxation").
-    u[l], g[l]: arrays [N_l+1, ...].  relax[l] in {RELAX_F, RELAX_FCF}.  Modifies u in place.
+    u[l], g[l]: arrays [N_l+1, ...].  relax[l] = n means F (CF)^n.  Modifies u in place.
+    N_l need not be a multiple of c_f: points after the last C-point form a shorter last interval of F-points.
+    cycle = CYCLE_F: when the correction has been spread (the cycle below is complete) one more V-cycle is run
+    from this level down, as in the F-cycle of multigrid; on the last two levels that is simply two V-cycles.
     """
     Nl = N[l]
     ul, gl = u[l], g[l]
@@ -190,26 +206,28 @@ def fas_vcycle(step, N, cf, relax, u, g, l=0, resnorm=None):
         for j in range(1, Nl + 1):
             ul[j] = step(l, np.array([j]), ul[j - 1:j])[0] + gl[j]
         return
+    Nc = N[l + 1]                                 # number of C-points after point 0 (= floor(N_l / c_f))
 
     def f_relax():
-        # from every C-point fill the F-points up to the next C-point, exclusive
+        # from every C-point fill the F-points up to the next C-point, exclusive (or to the end of the level)
         for s in range(1, cf):
-            j = np.arange(0, Nl, cf) + s
+            j = np.arange(0, Nl + 1, cf) + s
+            j = j[j <= Nl]
             ul[j] = step(l, j, ul[j - 1]) + gl[j]
 
     def c_relax():
         # one more step from the last F-point of each interval onto the next C-point
-        j = np.arange(cf, Nl + 1, cf)
+        j = cf * np.arange(1, Nc + 1)
         ul[j] = step(l, j, ul[j - 1]) + gl[j]
 
     # relax the current guess
     f_relax()
-    if relax[l] == RELAX_FCF:
+    for _ in range(relax[l]):
         c_relax()
         f_relax()
 
     # residual at the C-points, restricted by injection:  r_c = R(f(h')),  h'_c = R(h')
-    jc = np.arange(cf, Nl + 1, cf)
+    jc = cf * np.arange(1, Nc + 1)
     v = step(l, jc, ul[jc - 1]) + gl[jc]
     r_c = ul[jc] - v
     if resnorm is not None and l == 0:
@@ -218,17 +236,20 @@ def fas_vcycle(step, N, cf, relax, u, g, l=0, resnorm=None):
 
     # coarse equation f_c(h_c*) = f_c(h'_c) - r_c, i.e.  U_k = step(l+1,k,U_{k-1}) + G_k  with
     # G_k = U'_k - step(l+1,k,U'_{k-1}) - r_k = v_k - step(l+1,k,U'_{k-1})
-    k = np.arange(1, N[l + 1] + 1)
+    k = np.arange(1, Nc + 1)
     G = np.zeros_like(Uc)
     G[k] = v - step(l + 1, k, Uc[k - 1])
     u[l + 1] = Uc.copy()                                       # initial guess = restricted state
     g[l + 1] = G
-    fas_vcycle(step, N, cf, relax, u, g, l + 1, resnorm)
+    fas_vcycle(step, N, cf, relax, u, g, l + 1, resnorm, cycle)
 
     # h'' = h' + P(h_c* - h'_c): only the C-point values are read afterwards
     ul[jc] = u[l + 1][1:]
     # final F-relaxation spreads the correction over the F-points
     f_relax()
+    if cycle == CYCLE_F:
+        # F-cycle: one V-cycle from this level down on the corrected state (its level-0 residual is not recorded again)
+        fas_vcycle(step, N, cf, relax, u, g, l, None, CYCLE_V)
 
 
 def _relax_list(levels, relax_fine, relax_coarse):
@@ -236,7 +257,7 @@ def _relax_list(levels, relax_fine, relax_coarse):
 
 
 def mgrit_forward(W_ih, W_hh, b_ih, b_hh, x, h0, cf, levels, iters, cell=CELL_IMPLICIT,
-                  relax_fine=RELAX_F, relax_coarse=RELAX_FCF, dt=1.0, h_init=None):
+                  relax_fine=RELAX_F, relax_coarse=RELAX_FCF, dt=1.0, h_init=None, cycle=CYCLE_V, ragged=False):
     """Forward propagation by `iters` MGRIT cycles from the zero initial guess
     (Algorithm "MGRITTraining", forward block).  Level l uses the same cell with time step
     gamma = c_f^l * dt and, for its point j, the input of fine step c_f^l * j.
@@ -244,7 +265,7 @@ def mgrit_forward(W_ih, W_hh, b_ih, b_hh, x, h0, cf, levels, iters, cell=CELL_IM
     Returns h[T,B,H] and the list of level-0 C-point residual 2-norms, one per cycle, each
     measured after that cycle's pre-relaxation."""
     T = x.shape[0]
-    N = level_sizes(T, cf, levels)
+    N = level_sizes(T, cf, levels, ragged)
     gi = input_projection(W_ih, b_ih, x)
 
     def step(l, j, u_prev):
@@ -264,32 +285,34 @@ def mgrit_forward(W_ih, W_hh, b_ih, b_hh, x, h0, cf, levels, iters, cell=CELL_IM
         fas_vcycle(step, N, cf, relax, u, g, 0, None)
         return u[0][1:].copy(), resnorm
     for _ in range(iters):
-        fas_vcycle(step, N, cf, relax, u, g, 0, resnorm)
+        fas_vcycle(step, N, cf, relax, u, g, 0, resnorm, cycle)
     return u[0][1:].copy(), resnorm
 
 
 def mgrit_adjoint(W_ih, W_hh, b_ih, b_hh, x, h0, h, dh_seed, cf, levels, iters, cell=CELL_IMPLICIT,
-                  relax_fine=RELAX_F, relax_coarse=RELAX_FCF, dt=1.0, want_dx=True):
+                  relax_fine=RELAX_F, relax_coarse=RELAX_FCF, dt=1.0, want_dx=True, cycle=CYCLE_V, ragged=False):
     """Backward propagation by MGRIT on the adjoint recurrence, time reversed
     (Algorithm "MGRITTraining", backward block; Appendix "Training With MGRIT").
 
-    Reversed index s = N_l - j: the level-l unknown mu_s approximates lambda at forward
-    point N_l - s.  mu_0 = lambda_T is fixed; the step arriving at s applies the transposed
-    Jacobian of forward step j = N_l - s + 1 of level l, linearised at the GIVEN states h
-    (restricted by injection) with gamma = c_f^l dt.  The fine-level source is the direct
-    loss derivative dh_seed at that time.  Zero initial guess.
+    Reversed index: the level-l unknown mu_s approximates lambda at fine time T - c_f^l s.
+    mu_0 = lambda_T is fixed; the step arriving at s applies the transposed Jacobian of the
+    level-l forward step (gamma = c_f^l dt) that ARRIVES at fine time T - c_f^l (s-1), i.e. with
+    that time's input and linearised at the GIVEN state c_f^l fine steps earlier (restriction by
+    injection).  For T divisible by c_f^(levels-1) this is forward step j = N_l - s + 1 of the
+    level; otherwise the reversed coarse grids are anchored at T, not at 0.  The fine-level
+    source is the direct loss derivative dh_seed at that time.  Zero initial guess.
 
     Returns lam[T,B,H] (lam[k] = dL/dh_{k+1}), lam0, gradients (one time-parallel pass with
     the final lam and h) and the residual norms."""
     T = x.shape[0]
-    N = level_sizes(T, cf, levels)
+    N = level_sizes(T, cf, levels, ragged)
     gi = input_projection(W_ih, b_ih, x)
     hfull = np.concatenate([h0[None], h], axis=0)                 # h_0 .. h_T
 
     def step(l, s, mu_prev):
         m = cf ** l
-        j = N[l] - s + 1
-        a, c_r, c_z, c_n, _ = adjoint_coefficients(W_hh, b_hh, gi[m * j - 1], hfull[m * (j - 1)],
+        t_arrive = T - m * (s - 1)                                # fine time the transposed forward step arrives at
+        a, c_r, c_z, c_n, _ = adjoint_coefficients(W_hh, b_hh, gi[t_arrive - 1], hfull[t_arrive - m],
                                                    m * dt, cell)
         return a * mu_prev + np.concatenate([c_r * mu_prev, c_z * mu_prev, c_n * mu_prev], axis=-1) @ W_hh
 
@@ -306,7 +329,7 @@ def mgrit_adjoint(W_ih, W_hh, b_ih, b_hh, x, h0, h, dh_seed, cf, levels, iters, 
         fas_vcycle(step, N, cf, relax, u, g, 0, None)
     else:
         for _ in range(iters):
-            fas_vcycle(step, N, cf, relax, u, g, 0, resnorm)
+            fas_vcycle(step, N, cf, relax, u, g, 0, resnorm, cycle)
     lam = np.ascontiguousarray(u[0][0:T][::-1])                    # lam[k] = mu_{T-1-k}
     lam0 = u[0][T].copy()
     grads = weight_gradients(W_ih, W_hh, b_ih, b_hh, x, h0, h, lam, cell, dt, want_dx)

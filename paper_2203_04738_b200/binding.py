@@ -21,9 +21,9 @@ lib = ctypes.CDLL(LIB_PATH)
 
 OK = 0
 CELL_CLASSIC, CELL_IMPLICIT = 0, 1
-RELAX_F, RELAX_FCF = 0, 1
+RELAX_F, RELAX_FCF, RELAX_FCFCF = 0, 1, 2
 OPERANDS_FP32, OPERANDS_BF16 = 0, 2
-FLAG_SKIP_DUPLICATE_FRELAX = 1
+FLAG_SKIP_DUPLICATE_FRELAX, FLAG_F_CYCLE, FLAG_RAGGED_T = 1, 2, 4
 
 
 class Cfg(ctypes.Structure):

@@ -60,6 +60,7 @@ struct Ws {  // bump allocator over the caller's workspace; base == nullptr only
 
 struct Hier {
   int L; int N[kMaxLevels]; i64 stride_t[kMaxLevels]; float gamma[kMaxLevels];
+  i64 rem[kMaxLevels];   // T - stride_t * N: fine steps before the first reversed (adjoint) point of the level; 0 unless T is ragged
 };
 
 // every data pointer must be 32-byte aligned (nullptr passes: optional arguments are checked for presence elsewhere)
@@ -75,8 +76,8 @@ int check_cfg(const mgrit_gru_cfg* c, Hier* hr) {
   if (c->T <= 0 || c->B <= 0 || c->I <= 0 || c->H <= 0 || c->levels < 1 || c->levels > kMaxLevels) return MGRIT_INVALID_ARG;
   if (c->levels > 1 && (c->cf < 2 || c->iters < 0)) return MGRIT_INVALID_ARG;
   if (c->cell != MGRIT_CELL_CLASSIC && c->cell != MGRIT_CELL_IMPLICIT) return MGRIT_INVALID_ARG;
-  if (c->relax_fine != MGRIT_RELAX_F && c->relax_fine != MGRIT_RELAX_FCF) return MGRIT_INVALID_ARG;
-  if (c->relax_coarse != MGRIT_RELAX_F && c->relax_coarse != MGRIT_RELAX_FCF) return MGRIT_INVALID_ARG;
+  if (c->relax_fine < MGRIT_RELAX_F || c->relax_fine > MGRIT_RELAX_MAX) return MGRIT_INVALID_ARG;
+  if (c->relax_coarse < MGRIT_RELAX_F || c->relax_coarse > MGRIT_RELAX_MAX) return MGRIT_INVALID_ARG;
   if (c->operands != MGRIT_OPERANDS_FP32 && c->operands != MGRIT_OPERANDS_BF16) return MGRIT_INVALID_ARG;
   if (!(c->dt > 0.f)) return MGRIT_INVALID_ARG;
   if (c->H % 8 != 0 || c->I % 8 != 0) return MGRIT_UNSUPPORTED;
@@ -84,11 +85,14 @@ int check_cfg(const mgrit_gru_cfg* c, Hier* hr) {
   if (((i64)c->T + 1) * c->B > (i64)INT_MAX - 1024 || (i64)3 * c->H > INT_MAX / 4 || c->I > INT_MAX / 4) return MGRIT_UNSUPPORTED;
   i64 m = 1;
   hr->L = c->levels;
+  const bool ragged = (c->flags & MGRIT_FLAG_RAGGED_T) != 0;
   for (int l = 0; l < c->levels; ++l) {
-    if (c->T % m != 0) return MGRIT_NOT_DIVISIBLE;
+    // ragged: the C-points of a level are its points 0, cf, 2 cf, ...; N_{l+1} = floor(N_l / cf) = floor(T / cf^(l+1))
+    if (!ragged && c->T % m != 0) return MGRIT_NOT_DIVISIBLE;
     hr->N[l] = (int)(c->T / m);
     hr->stride_t[l] = m;
     hr->gamma[l] = (float)m * c->dt;
+    hr->rem[l] = c->T - m * hr->N[l];
     if (l + 1 < c->levels) {
       m *= c->cf;
       if (m > c->T) return MGRIT_NOT_DIVISIBLE;
@@ -196,42 +200,58 @@ struct Cycle {
   virtual bool chain(int l) { (void)l; return false; }
   virtual ~Cycle() {}
 
+  // F-relaxation: from every C-point the cf - 1 F-points of its interval, one dependent step per launch over all
+  // intervals; a ragged level has one more, shorter interval of N % cf F-points behind its last C-point.
   void frelax(int l) {
-    int cf = c->cf, nki = hr.N[l] / cf;
+    int cf = c->cf, nki = hr.N[l] / cf, tail = hr.N[l] % cf;
     for (int sI = 1; sI < cf; ++sI)
-      step(StepDesc{l, nki, sI - 1, cf, U[l], sI, cf, G[l], sI, cf, sI, cf, 0});
+      step(StepDesc{l, nki + (sI <= tail ? 1 : 0), sI - 1, cf, U[l], sI, cf, G[l], sI, cf, sI, cf, 0});
   }
   void crelax(int l) {
     int cf = c->cf, nki = hr.N[l] / cf;
     step(StepDesc{l, nki, cf - 1, cf, U[l], cf, cf, G[l], cf, cf, cf, cf, 0});
   }
-  void vcycle(int l) {
+  // One cycle from level l down.  skip_first_f: the state of level l was F-relaxed last and no C-point has changed
+  // since, so the opening F-relaxation would reproduce it bit for bit.  record: store the level-0 residual norm.
+  void cycle(int l, bool skip_first_f, bool record) {
     int cf = c->cf, N = hr.N[l];
     if (l == hr.L - 1) {  // coarsest level: serial propagation
       if (chain(l)) return;
       for (int j = 1; j <= N; ++j) step(StepDesc{l, 1, j - 1, 1, U[l], j, 1, G[l], j, 1, j, 1, 0});
       return;
     }
-    int relax = l == 0 ? c->relax_fine : c->relax_coarse;
-    bool dup = l == 0 && cycle_idx > 0 && (c->flags & MGRIT_FLAG_SKIP_DUPLICATE_FRELAX);
-    if (!dup) frelax(l);
-    if (relax == MGRIT_RELAX_FCF) { crelax(l); frelax(l); }
-    int nc = N / cf;
+    int relax = l == 0 ? c->relax_fine : c->relax_coarse;       // n: F (CF)^n
+    if (!skip_first_f) frelax(l);
+    for (int n = 0; n < relax; ++n) { crelax(l); frelax(l); }
+    int nc = hr.N[l + 1];
     // v_k = step_l(u_{cf k - 1}) + g_{cf k}  ->  G[l+1][k]
     step(StepDesc{l, nc, cf - 1, cf, G[l + 1], 1, 1, G[l], cf, cf, cf, cf, 0});
     // r_k = u_{cf k} - v_k ; U'_k = u_{cf k}
     stream_restrict_residual(U[l], cf, G[l + 1], U[l + 1], Ub ? Ub[l + 1] : nullptr, nc, (i64)BH,
-                             l == 0 ? res_acc + cycle_idx : nullptr, s);
+                             (l == 0 && record) ? res_acc + cycle_idx : nullptr, s);
     // G_k = v_k - step_{l+1}(U'_{k-1})
     step(StepDesc{l + 1, nc, 0, 1, G[l + 1], 1, 1, nullptr, 0, 0, 1, 1, 1});
-    vcycle(l + 1);
+    cycle(l + 1, false, false);
     stream_correct(U[l], Ub ? Ub[l] : nullptr, cf, U[l + 1], nc, (i64)BH, s);
     frelax(l);
+    // F-cycle: one more V-cycle from this level down on the corrected state (on the last two levels: a second
+    // V-cycle).  Its opening F-relaxation would repeat the one just done.
+    if ((c->flags & MGRIT_FLAG_F_CYCLE) && fcycle_leg) {
+      const bool saved = fcycle_leg;
+      fcycle_leg = false;
+      cycle(l, true, false);
+      fcycle_leg = saved;
+    }
   }
+  bool fcycle_leg = true;     // false while a trailing V-cycle of an F-cycle runs (it does not spawn further ones)
   int solve() {
-    if (hr.L == 1) { vcycle(0); return rc; }
+    if (hr.L == 1) { cycle(0, false, false); return rc; }
     cudaMemsetAsync(res_acc, 0, sizeof(double) * (size_t)(c->iters > 0 ? c->iters : 1), s);
-    for (cycle_idx = 0; cycle_idx < c->iters && rc == MGRIT_OK; ++cycle_idx) vcycle(0);
+    for (cycle_idx = 0; cycle_idx < c->iters && rc == MGRIT_OK; ++cycle_idx) {
+      // the previous cycle ended with an F-relaxation of level 0: the caller may ask not to repeat it
+      const bool dup = cycle_idx > 0 && (c->flags & MGRIT_FLAG_SKIP_DUPLICATE_FRELAX);
+      cycle(0, dup, true);
+    }
     return rc;
   }
 };
@@ -396,6 +416,7 @@ int adjoint_impl(const mgrit_gru_cfg* cfg_in, bool serial, const gru_params* p, 
   for (int l = 0; l < hr.L; ++l) {
     LinArgs a;
     a.M = hr.N[l] * c.B; a.B = c.B; a.H = c.H; a.h0 = h0; a.h = h; a.stride_t = hr.stride_t[l]; a.gi = gi;
+    a.t0 = hr.rem[l];     // the level's reversed grid is anchored at T: its forward steps arrive at t0 + stride * j
     a.W_hh = p->W_hh; a.b_hh = p->b_hh; a.gamma = hr.gamma[l]; a.cell = c.cell;
     a.a = aw.a[l]; a.cr = aw.cr[l]; a.cz = aw.cz[l]; a.cn = aw.cn[l]; a.cnp = l == 0 ? aw.cnp : nullptr;
     a.crb = aw.crb[l]; a.czb = aw.czb[l]; a.cnb = aw.cnb[l]; a.cnpb = l == 0 ? aw.cnpb : nullptr;

@@ -102,12 +102,14 @@ struct FwdStepArgs {
 };
 
 // ---- adjoint coefficients of every step of one level (discrete adjoint of the cell) ----
-// Row m = (j-1, b) for forward steps j = 1..N_l.  Outputs are [N_l*B, H] each.
+// Row m = (j-1, b) for the level's forward steps j = 1..N_l; step j leaves fine time t0 + stride_t*(j-1) and arrives
+// at t0 + stride_t*j with that time's input.  Outputs are [N_l*B, H] each.
 struct LinArgs {
   int M, B, H;
-  const float* h0;                  // [B,H]   state at level point 0
+  const float* h0;                  // [B,H]   state at fine time 0
   const float* h;                   // [T,B,H] fine states (h[k] = h_{k+1})
   i64 stride_t;                     // fine steps per level step: cf^l
+  i64 t0;                           // fine time the level's first step leaves from (0 unless T is ragged)
   const float* gi;                  // [T,B,3H]
   const float* W_hh; const float* b_hh;
   float gamma; int cell;

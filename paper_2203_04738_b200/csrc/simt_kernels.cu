@@ -110,11 +110,12 @@ struct FirstRestBT {  // B(0, n, k=m): m < nfirst ? first[m*C + n] : rest[(m - n
     return k < nfirst ? first[(i64)k * C + n] : rest[(i64)(k - nfirst) * C + n];
   }
 };
-struct LinA {  // state entering forward step j = m/B + 1 of a level: h_{stride*(j-1)}
-  const float* h0; const float* h; i64 stride_t; int B, H;
+struct LinA {  // state entering forward step j = m/B + 1 of a level: h at fine time t0 + stride*(j-1)
+  const float* h0; const float* h; i64 stride_t, t0; int B, H;
   __device__ float operator()(int m, int k) const {
     int j1 = m / B, b = m % B;
-    return j1 == 0 ? h0[(i64)b * H + k] : h[((i64)j1 * stride_t - 1) * B * H + (i64)b * H + k];
+    const i64 t = t0 + (i64)j1 * stride_t;
+    return t == 0 ? h0[(i64)b * H + k] : h[(t - 1) * B * H + (i64)b * H + k];
   }
 };
 struct AdjA {  // A[m, g*H + i] = c_g[m, i] * lam[m, i]
@@ -156,8 +157,9 @@ struct LinEpi {
   LinArgs a;
   __device__ void operator()(int m, int n, const float* v) const {
     int j1 = m / a.B, b = m % a.B;
-    const float* gi = a.gi + (((i64)(j1 + 1) * a.stride_t - 1) * a.B + b) * 3 * a.H;
-    float hp = j1 == 0 ? a.h0[(i64)b * a.H + n] : a.h[(((i64)j1 * a.stride_t - 1) * a.B + b) * a.H + n];
+    const i64 t = a.t0 + (i64)j1 * a.stride_t;        // fine time the step leaves from
+    const float* gi = a.gi + ((t + a.stride_t - 1) * a.B + b) * 3 * a.H;
+    float hp = t == 0 ? a.h0[(i64)b * a.H + n] : a.h[((t - 1) * a.B + b) * a.H + n];
     CellLin c = cell_linearise(gi[n], gi[a.H + n], gi[2 * a.H + n], v[0] + a.b_hh[n], v[1] + a.b_hh[a.H + n],
                                v[2] + a.b_hh[2 * a.H + n], hp, a.gamma, a.cell);
     i64 o = (i64)m * a.H + n;
@@ -192,7 +194,7 @@ void simt_fwd_step(const FwdStepArgs& a, cudaStream_t s) {
 }
 
 void simt_linearise(const LinArgs& a, cudaStream_t s) {
-  launch<3, true, true>(KC_LINEARISE, a.M, a.H, a.H, LinA{a.h0, a.h, a.stride_t, a.B, a.H}, GateW{a.W_hh, a.H, a.H}, LinEpi{a}, s);
+  launch<3, true, true>(KC_LINEARISE, a.M, a.H, a.H, LinA{a.h0, a.h, a.stride_t, a.t0, a.B, a.H}, GateW{a.W_hh, a.H, a.H}, LinEpi{a}, s);
 }
 
 void simt_adj_step(const AdjStepArgs& a, cudaStream_t s) {

@@ -372,8 +372,9 @@ struct EpiLin {  // adjoint coefficients of every step of a level
     const bool valid = row < a.M;
     const int j1 = valid ? row / a.B : 0, b = valid ? row % a.B : 0;
     const int H = a.H;
-    const float* __restrict__ gi = a.gi + (((i64)(j1 + 1) * a.stride_t - 1) * a.B + b) * 3 * H + u0;
-    const float* __restrict__ hp = (j1 == 0 ? a.h0 + (i64)b * H : a.h + (((i64)j1 * a.stride_t - 1) * a.B + b) * H) + u0;
+    const i64 t = a.t0 + (i64)j1 * a.stride_t;      // fine time the step leaves from
+    const float* __restrict__ gi = a.gi + ((t + a.stride_t - 1) * a.B + b) * 3 * H + u0;
+    const float* __restrict__ hp = (t == 0 ? a.h0 + (i64)b * H : a.h + ((t - 1) * a.B + b) * H) + u0;
     const i64 o = (i64)row * H + u0;
     const float* __restrict__ bh = a.b_hh + u0;
 #pragma unroll
@@ -609,7 +610,7 @@ template <class T> T* take(char* base, size_t* off, size_t n) {
 size_t max_step_rows(const mgrit_gru_cfg* c, const int* N, int L) {
   size_t m = (size_t)c->B;
   for (int l = 0; l + 1 < L; ++l) {
-    size_t r = (size_t)(N[l] / c->cf) * c->B;   // relaxation / residual / FAS right-hand side rows
+    size_t r = (size_t)((N[l] + c->cf - 1) / c->cf) * c->B;   // relaxation (a ragged level has one more interval) / residual / FAS rows
     if (r > m) m = r;
   }
   return m;
@@ -693,31 +694,42 @@ int umma_fwd_step(const FwdStepArgs& a, UmmaFwdWs* w, cudaStream_t s) {
 }
 
 int umma_linearise(const LinArgs& a, UmmaAdjWs* w, cudaStream_t s) {
-  // rows (j-1, b): state entering forward step j of the level = h_{stride*(j-1)}
+  // rows (j-1, b): state entering forward step j of the level = h at fine time t0 + stride*(j-1); w->hb0 holds the
+  // bf16 copy of [h_0; h], so fine time t is its slot t, and in fp32 time t >= 1 is slot t - 1 of h
   const i64 BH = (i64)a.B * a.H;
   const int N = a.M / a.B;
+  const float* gi0 = a.gi + (a.t0 + a.stride_t - 1) * BH * 3;       // input of the fine step that arrives with step 1
   if (128 % a.B == 0) {
     CellArgs ca{};
     ca.B = a.B; ca.H = a.H; ca.b_hh = a.b_hh; ca.gamma = a.gamma; ca.cell = a.cell;
-    const float* gi0 = a.gi + (a.stride_t - 1) * BH * 3;
-    // step 1 starts from h_0 (its own array); steps 2..N from h[stride*(j-1) - 1]
     ca.a = a.a; ca.cr = a.crb; ca.cz = a.czb; ca.cn = a.cnb; ca.cnp = a.cnpb;
-    if (!launch_cell<true, false>(KC_LINEARISE, w->hb0, 0, gi0, 0, a.h0, 0, nullptr, 0, 1, w->W_hh, ca, s)) return MGRIT_CUDA_ERROR;
-    if (N > 1) {
-      ca.a = a.a + BH; ca.cr = a.crb + BH; ca.cz = a.czb + BH; ca.cn = a.cnb + BH; ca.cnp = a.cnpb ? a.cnpb + BH : nullptr;
-      if (!launch_cell<true, false>(KC_LINEARISE, w->hb + (a.stride_t - 1) * BH, a.stride_t * BH, gi0 + a.stride_t * BH * 3,
-                                    a.stride_t * BH * 3, a.h + (a.stride_t - 1) * BH, a.stride_t * BH, nullptr, 0, N - 1, w->W_hh, ca, s))
+    int done = 0;
+    if (a.t0 == 0) {   // step 1 starts from h_0 (its own array)
+      if (!launch_cell<true, false>(KC_LINEARISE, w->hb0, 0, gi0, 0, a.h0, 0, nullptr, 0, 1, w->W_hh, ca, s)) return MGRIT_CUDA_ERROR;
+      done = 1;
+    }
+    if (N > done) {
+      const i64 off = (i64)done * BH;
+      ca.a = a.a + off; ca.cr = a.crb + off; ca.cz = a.czb + off; ca.cn = a.cnb + off; ca.cnp = a.cnpb ? a.cnpb + off : nullptr;
+      const i64 t1 = a.t0 + (i64)done * a.stride_t;                  // fine time the first of these steps leaves from (>= 1)
+      if (!launch_cell<true, false>(KC_LINEARISE, w->hb0 + t1 * BH, a.stride_t * BH, gi0 + (i64)done * a.stride_t * BH * 3,
+                                    a.stride_t * BH * 3, a.h + (t1 - 1) * BH, a.stride_t * BH, nullptr, 0, N - done, w->W_hh, ca, s))
         return MGRIT_CUDA_ERROR;
     }
     return MGRIT_OK;
   }
-  if (launch_pdl(pack_rows_kernel, dim3(pgrid((i64)a.B * (a.H / 4))), dim3(kPT), 0, s, a.h0, (i64)0, a.B, a.H / 4, (i64)a.B,
-                 reinterpret_cast<uint2*>(w->Apack)) != cudaSuccess)
-    return MGRIT_CUDA_ERROR;
-  count_launch();
-  if (a.M > a.B) {
-    if (launch_pdl(pack_rows_kernel, dim3(pgrid((i64)(a.M - a.B) * (a.H / 4))), dim3(kPT), 0, s, a.h + (a.stride_t - 1) * BH,
-                   (i64)(a.stride_t * BH), a.B, a.H / 4, (i64)(a.M - a.B), reinterpret_cast<uint2*>(w->Apack + BH)) != cudaSuccess)
+  int done = 0;
+  if (a.t0 == 0) {
+    if (launch_pdl(pack_rows_kernel, dim3(pgrid((i64)a.B * (a.H / 4))), dim3(kPT), 0, s, a.h0, (i64)0, a.B, a.H / 4, (i64)a.B,
+                   reinterpret_cast<uint2*>(w->Apack)) != cudaSuccess)
+      return MGRIT_CUDA_ERROR;
+    count_launch();
+    done = 1;
+  }
+  if (N > done) {
+    const i64 t1 = a.t0 + (i64)done * a.stride_t;
+    if (launch_pdl(pack_rows_kernel, dim3(pgrid((i64)(N - done) * a.B * (a.H / 4))), dim3(kPT), 0, s, a.h + (t1 - 1) * BH,
+                   (i64)(a.stride_t * BH), a.B, a.H / 4, (i64)(N - done) * a.B, reinterpret_cast<uint2*>(w->Apack + (i64)done * BH)) != cudaSuccess)
       return MGRIT_CUDA_ERROR;
     count_launch();
   }

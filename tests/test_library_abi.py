@@ -69,3 +69,16 @@ def test_status_calls_answer_without_a_device(lib):
         assert lib.mgrit_gru_clear_device_status() == 0 and lib.mgrit_gru_last_device_status() == 0
     else:
         assert lib.mgrit_gru_last_device_status() == -5 and lib.mgrit_gru_clear_device_status() == -5
+
+
+def test_cycle_variant_flags_are_validated_on_the_host(lib):
+    from paper_2203_04738_b200.binding import Cfg, FLAG_F_CYCLE, FLAG_RAGGED_T, make_cfg
+    f, a = ctypes.c_size_t(0), ctypes.c_size_t(0)
+    fn = lib.mgrit_gru_workspace_bytes
+    fn.argtypes = [ctypes.POINTER(Cfg), ctypes.POINTER(ctypes.c_size_t), ctypes.POINTER(ctypes.c_size_t)]
+    assert fn(ctypes.byref(make_cfg(23, 2, 16, 32, cf=4, levels=2)), ctypes.byref(f), ctypes.byref(a)) == -2
+    assert fn(ctypes.byref(make_cfg(23, 2, 16, 32, cf=4, levels=2, flags=FLAG_RAGGED_T)), ctypes.byref(f), ctypes.byref(a)) == 0
+    assert fn(ctypes.byref(make_cfg(7, 2, 16, 32, cf=4, levels=3, flags=FLAG_RAGGED_T)), ctypes.byref(f), ctypes.byref(a)) == -2
+    assert fn(ctypes.byref(make_cfg(64, 2, 16, 32, cf=4, levels=3, relax_fine=2, relax_coarse=3, flags=FLAG_F_CYCLE)),
+              ctypes.byref(f), ctypes.byref(a)) == 0
+    assert fn(ctypes.byref(make_cfg(64, 2, 16, 32, cf=4, levels=3, relax_fine=9)), ctypes.byref(f), ctypes.byref(a)) == -1
