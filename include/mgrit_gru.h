@@ -148,6 +148,27 @@ int gru_serial_backward(const mgrit_gru_cfg* cfg, const gru_params* p, const flo
                         float* dh, float* dh0, float* dx, const gru_grads* grads,
                         void* ws, size_t ws_bytes, mgrit_stream_t stream);
 
+/* Stacked layers in ONE state (tables of training parameters: "Num. Layers 2"): the state of a time point is the
+ * stack of all layers' hidden states, layer k's input at a step is layer k-1's new state of the same step (layer 0
+ * reads x), and one MGRIT cycle (Algorithm "MGProp") advances the whole stack; on level l every layer uses the cell
+ * with time step cf^l.  With levels == 1 this is the serial sweep of the stacked network (the usual multi-layer GRU
+ * for the classic cell and dt = 1).  The alternative -- one MGRIT solve per layer, the layer below solved first --
+ * is composed from mgrit_gru_forward / mgrit_gru_adjoint by the caller.
+ *   cfg->I is the input width of layer 0; layers >= 1 have input width H.  n_layers <= 8.
+ *   layers: HOST array of n_layers gru_params (device pointers inside).  h0[n_layers,B,H]; h[T,n_layers,B,H];
+ *   gi0[T,B,3H]: projection of x for layer 0 (written by the forward call, read by the adjoint call).
+ *   Adjoint: linearised at the GIVEN states; on coarse levels the input of layer k >= 1 is the layer below's given
+ *   state at the step's arrival time (restriction by injection for inputs as for states).
+ *   dh_seed[T,n_layers,B,H] or NULL; dhT[B,H] or NULL: loss derivative w.r.t. the TOP layer's last state; dh (optional)
+ *   and dh0 have the shapes of h and h0: the sensitivities of the states as step outputs; dx[T,B,I] or NULL;
+ *   grads: HOST array of n_layers gru_grads.  The coarsest level is advanced step by step (no persistent chain). */
+int mgrit_gru_stack_workspace_bytes(const mgrit_gru_cfg* cfg, int32_t n_layers, size_t* fwd_bytes, size_t* adj_bytes);
+int mgrit_gru_stack_forward(const mgrit_gru_cfg* cfg, int32_t n_layers, const gru_params* layers, const float* x, const float* h0,
+                            float* gi0, float* h, float* resnorm, void* ws, size_t ws_bytes, mgrit_stream_t stream);
+int mgrit_gru_stack_adjoint(const mgrit_gru_cfg* cfg, int32_t n_layers, const gru_params* layers, const float* x, const float* h0,
+                            const float* gi0, const float* h, const float* dh_seed, const float* dhT, float* dh, float* dh0,
+                            float* dx, const gru_grads* grads, float* resnorm, void* ws, size_t ws_bytes, mgrit_stream_t stream);
+
 /* Classifier head on h_T with mean softmax cross-entropy (the loss whose gradient seeds the
  * backward block: w_T = grad_{h_T} L).  hT[B,H], Wc[C,H], bc[C], labels[B] (int32, device)
  * -> loss[1] (device), dhT[B,H], dWc[C,H], dbc[C].  ws: device scratch of at least

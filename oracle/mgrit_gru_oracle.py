@@ -365,3 +365,159 @@ def adam_update(p, g, m, v, lr, step, beta1=0.9, beta2=0.999, eps=1e-8):
     mhat = m / (1.0 - beta1 ** step)
     vhat = v / (1.0 - beta2 ** step)
     return p - lr * mhat / (np.sqrt(vhat) + eps), m, v
+
+
+# --------------------------------------------------------------------------- stacked layers in one state
+# A multi-layer GRU advanced one TIME step at a time: the state of a time point is the stack of all layers' hidden
+# states, and layer k's input at a step is layer k-1's NEW state of the same step (layer 0 reads x).  MGRIT then
+# runs ONE cycle for the whole stack (the paper's experiments use two layers); on level l every layer uses the same
+# cell with time step c_f^l and layer 0 the input of fine step c_f^l j.
+# layers: list of (W_ih, W_hh, b_ih, b_hh); states are arrays [..., n_layers, B, H].
+
+def stacked_phi(layers, gi0, u_prev, gamma, cell):
+    """One step of the stack.  gi0 = W_i x + b_i of layer 0 for this step; u_prev[..., k, :, :] the layers' states."""
+    out = []
+    gik = gi0
+    for k, (W_ih, W_hh, b_ih, b_hh) in enumerate(layers):
+        if k > 0:
+            gik = out[-1] @ W_ih.T + b_ih          # input projection of the layer below's new state
+        out.append(phi(W_hh, b_hh, gik, u_prev[..., k, :, :], gamma, cell))
+    return np.stack(out, axis=-3)
+
+
+def stacked_serial_forward(layers, x, h0, cell=CELL_IMPLICIT, dt=1.0):
+    """h0: [n_layers, B, H] -> h[T, n_layers, B, H]; with the classic cell and dt = 1 this is the usual stacked GRU."""
+    T = x.shape[0]
+    gi0 = input_projection(layers[0][0], layers[0][2], x)
+    h = np.empty((T,) + h0.shape)
+    prev = h0
+    for t in range(T):
+        prev = stacked_phi(layers, gi0[t], prev, dt, cell)
+        h[t] = prev
+    return h
+
+
+def stacked_mgrit_forward(layers, x, h0, cf, levels, iters, cell=CELL_IMPLICIT, relax_fine=RELAX_F, relax_coarse=RELAX_FCF,
+                          dt=1.0, cycle=CYCLE_V, ragged=False, h_init=None):
+    """`iters` MGRIT cycles on the stacked state from the zero initial guess; returns h[T, n_layers, B, H] and the
+    level-0 C-point residual norms (over all layers)."""
+    T = x.shape[0]
+    N = level_sizes(T, cf, levels, ragged)
+    gi0 = input_projection(layers[0][0], layers[0][2], x)
+
+    def step(l, j, u_prev):
+        m = cf ** l
+        return stacked_phi(layers, gi0[m * j - 1], u_prev, m * dt, cell)
+
+    u = [None] * levels
+    g = [None] * levels
+    u[0] = np.zeros((T + 1,) + h0.shape)
+    u[0][0] = h0
+    if h_init is not None:
+        u[0][1:] = h_init
+    g[0] = np.zeros_like(u[0])
+    relax = _relax_list(levels, relax_fine, relax_coarse)
+    resnorm = []
+    if levels == 1:
+        fas_vcycle(step, N, cf, relax, u, g, 0, None)
+    else:
+        for _ in range(iters):
+            fas_vcycle(step, N, cf, relax, u, g, 0, resnorm, cycle)
+    return u[0][1:].copy(), resnorm
+
+
+def stacked_adjoint_step(layers, coefs, lam_out):
+    """Transposed Jacobian of one step of the stack applied to lam_out[..., k, :, :] (sensitivities of the step's
+    outputs).  coefs[k] = (a, c_r, c_z, c_n, c_np) of layer k at the step's linearisation point.  Works from the top
+    layer down: what layer k+1 sends to its input joins layer k's own output sensitivity.
+    Returns (sensitivities of the step's input states, the per-layer TOTAL output sensitivities used on the way --
+    the ones the parameter gradients of that step need)."""
+    nl = len(layers)
+    lam_in = [None] * nl
+    lam_tot = [None] * nl
+    from_above = 0.0
+    for k in range(nl - 1, -1, -1):
+        W_ih, W_hh, _, _ = layers[k]
+        a, c_r, c_z, c_n, c_np = coefs[k]
+        lt = lam_out[..., k, :, :] + from_above
+        lam_tot[k] = lt
+        lam_in[k] = a * lt + np.concatenate([c_r * lt, c_z * lt, c_n * lt], axis=-1) @ W_hh
+        from_above = np.concatenate([c_r * lt, c_z * lt, c_np * lt], axis=-1) @ W_ih if k > 0 else 0.0
+    return np.stack(lam_in, axis=-3), np.stack(lam_tot, axis=-3)
+
+
+def _stacked_inputs(layers, x, h):
+    """Layer k's input sequence given the states h[T, nl, B, H]: x for layer 0, the layer below's states otherwise."""
+    return [x if k == 0 else h[:, k - 1] for k in range(len(layers))]
+
+
+def stacked_serial_backward(layers, x, h0, h, dh_seed, cell=CELL_IMPLICIT, dt=1.0):
+    """Exact back-propagation through time of the stacked sweep.  dh_seed[T, nl, B, H]: direct loss derivatives.
+    Returns lam[T, nl, B, H] (sensitivity of every state as a step OUTPUT, before the within-step coupling),
+    lam0[nl, B, H] and per-layer gradient dicts."""
+    T = x.shape[0]
+    nl = len(layers)
+    hfull = np.concatenate([h0[None], h], axis=0)
+    inps = _stacked_inputs(layers, x, h)
+    gis = [input_projection(layers[k][0], layers[k][2], inps[k]) for k in range(nl)]
+    lam = np.empty_like(h)
+    lam_tot = np.empty_like(h)
+    cur = dh_seed[T - 1].copy()
+    for t in range(T, 0, -1):
+        lam[t - 1] = cur
+        coefs = [adjoint_coefficients(layers[k][1], layers[k][3], gis[k][t - 1], hfull[t - 1, k], dt, cell) for k in range(nl)]
+        back, tot = stacked_adjoint_step(layers, coefs, cur)
+        lam_tot[t - 1] = tot
+        cur = back + (dh_seed[t - 2] if t >= 2 else 0.0)
+    grads = [weight_gradients(*layers[k], inps[k], h0[k], h[:, k], lam_tot[:, k], cell, dt, want_dx=(k == 0)) for k in range(nl)]
+    return lam, cur, grads
+
+
+def stacked_mgrit_adjoint(layers, x, h0, h, dh_seed, cf, levels, iters, cell=CELL_IMPLICIT, relax_fine=RELAX_F,
+                          relax_coarse=RELAX_FCF, dt=1.0, cycle=CYCLE_V, ragged=False):
+    """MGRIT on the adjoint of the stacked recurrence, time reversed, linearised at the GIVEN states h[T, nl, B, H].
+    The level-l step arriving at reversed point s transposes the level's forward step (time step c_f^l) that arrives
+    at fine time t = T - c_f^l (s-1): every layer is linearised at its given state c_f^l fine steps earlier, with the
+    input that the given states provide at time t (x_t for layer 0, the layer below's given state at t otherwise:
+    restriction by injection for the inputs as for the states).  Gradients: one time-parallel pass with the final
+    sensitivities, top layer first (its input gradient joins the layer below's sensitivity)."""
+    T = x.shape[0]
+    nl = len(layers)
+    N = level_sizes(T, cf, levels, ragged)
+    hfull = np.concatenate([h0[None], h], axis=0)
+    inps = _stacked_inputs(layers, x, h)
+    gis = [input_projection(layers[k][0], layers[k][2], inps[k]) for k in range(nl)]
+
+    def coefs_at(t_arrive, m):
+        return [adjoint_coefficients(layers[k][1], layers[k][3], gis[k][t_arrive - 1], hfull[t_arrive - m][..., k, :, :], m * dt, cell)
+                for k in range(nl)]
+
+    def step(l, s, mu_prev):
+        m = cf ** l
+        out = np.empty_like(mu_prev)
+        for q, sq in enumerate(np.atleast_1d(s)):
+            out[q], _ = stacked_adjoint_step(layers, coefs_at(T - m * (int(sq) - 1), m), mu_prev[q])
+        return out
+
+    u = [None] * levels
+    g = [None] * levels
+    u[0] = np.zeros((T + 1,) + h0.shape)
+    u[0][0] = dh_seed[T - 1]
+    g[0] = np.zeros_like(u[0])
+    for s in range(1, T):
+        g[0][s] = dh_seed[T - s - 1]
+    relax = _relax_list(levels, relax_fine, relax_coarse)
+    resnorm = []
+    if levels == 1:
+        fas_vcycle(step, N, cf, relax, u, g, 0, None)
+    else:
+        for _ in range(iters):
+            fas_vcycle(step, N, cf, relax, u, g, 0, resnorm, cycle)
+    lam = np.ascontiguousarray(u[0][0:T][::-1])
+    lam0 = u[0][T].copy()
+    # total output sensitivities of every fine step (the within-step coupling added), then the gradient pass
+    lam_tot = np.empty_like(lam)
+    for t in range(1, T + 1):
+        _, lam_tot[t - 1] = stacked_adjoint_step(layers, coefs_at(t, 1), lam[t - 1])
+    grads = [weight_gradients(*layers[k], inps[k], h0[k], h[:, k], lam_tot[:, k], cell, dt, want_dx=(k == 0)) for k in range(nl)]
+    return lam, lam0, grads, resnorm

@@ -50,6 +50,11 @@ lib.mgrit_gru_adjoint.argtypes = [ctypes.POINTER(Cfg), ctypes.POINTER(_Params), 
                                   ctypes.POINTER(_Grads), ctypes.POINTER(ctypes.c_float), _vp, _sz, _vp]
 lib.gru_serial_backward.argtypes = [ctypes.POINTER(Cfg), ctypes.POINTER(_Params), _vp, _vp, _vp, _vp, _vp, _vp, _vp, _vp, _vp,
                                     ctypes.POINTER(_Grads), _vp, _sz, _vp]
+lib.mgrit_gru_stack_workspace_bytes.argtypes = [ctypes.POINTER(Cfg), _i32, ctypes.POINTER(_sz), ctypes.POINTER(_sz)]
+lib.mgrit_gru_stack_forward.argtypes = [ctypes.POINTER(Cfg), _i32, ctypes.POINTER(_Params), _vp, _vp, _vp, _vp,
+                                        ctypes.POINTER(ctypes.c_float), _vp, _sz, _vp]
+lib.mgrit_gru_stack_adjoint.argtypes = [ctypes.POINTER(Cfg), _i32, ctypes.POINTER(_Params), _vp, _vp, _vp, _vp, _vp, _vp, _vp, _vp, _vp,
+                                        ctypes.POINTER(_Grads), ctypes.POINTER(ctypes.c_float), _vp, _sz, _vp]
 lib.xent_head_workspace_bytes.argtypes = [_i32, _i32]
 lib.xent_head_workspace_bytes.restype = _sz
 lib.xent_head_fwd_bwd.argtypes = [_i32, _i32, _i32, _vp, _vp, _vp, _vp, _vp, _vp, _vp, _vp, _vp, _sz, _vp]
@@ -185,6 +190,52 @@ def mgrit_gru_adjoint(cfg, p, x, h0, gi, h, dh_seed=None, dhT=None, want_dx=True
 
 def gru_serial_backward(cfg, p, x, h0, gi, h, dh_seed=None, dhT=None, want_dx=True, ws=None, out=None, want_dh=True):
     return _adjoint(lib.gru_serial_backward, True, cfg, p, x, h0, gi, h, dh_seed, dhT, want_dx, False, ws, out, want_dh)
+
+
+def stack_workspace_bytes(cfg: Cfg, n_layers: int):
+    f, a = _sz(0), _sz(0)
+    _check(lib.mgrit_gru_stack_workspace_bytes(ctypes.byref(cfg), n_layers, ctypes.byref(f), ctypes.byref(a)))
+    return f.value, a.value
+
+
+def _param_array(layers):
+    arr = (_Params * len(layers))()
+    for k, p in enumerate(layers):
+        arr[k] = _params(p)
+    return arr
+
+
+def mgrit_gru_stack_forward(cfg, layers, x, h0, want_resnorm=False, ws=None):
+    """All layers in one state, one MGRIT cycle for the stack.  layers: list of parameter dicts; h0[n_layers,B,H].
+    -> (h[T,n_layers,B,H], gi0[T,B,3H], resnorm list or None)"""
+    dev, nl = x.device, len(layers)
+    gi0 = torch.empty(cfg.T, cfg.B, 3 * cfg.H, device=dev)
+    h = torch.empty(cfg.T, nl, cfg.B, cfg.H, device=dev)
+    ws = _ws(stack_workspace_bytes(cfg, nl)[0], ws, dev)
+    rn = (ctypes.c_float * max(cfg.iters, 1))() if want_resnorm else None
+    _check(lib.mgrit_gru_stack_forward(ctypes.byref(cfg), nl, _param_array(layers), _f32(x), _f32(h0), _f32(gi0), _f32(h), rn,
+                                       _ptr(ws), ws.numel(), _stream()))
+    return h, gi0, (list(rn)[:cfg.iters] if want_resnorm else None)
+
+
+def mgrit_gru_stack_adjoint(cfg, layers, x, h0, gi0, h, dh_seed=None, dhT=None, want_dx=True, want_dh=True, want_resnorm=False, ws=None):
+    """-> (dh[T,n_layers,B,H] or None, dh0[n_layers,B,H], dx or None, list of per-layer AdjointResult (gradients only), resnorm)"""
+    dev, nl = x.device, len(layers)
+    dh = torch.empty(cfg.T, nl, cfg.B, cfg.H, device=dev) if want_dh else None
+    dh0 = torch.empty(nl, cfg.B, cfg.H, device=dev)
+    dx = torch.empty(cfg.T, cfg.B, cfg.I, device=dev) if want_dx else None
+    outs, garr = [], (_Grads * nl)()
+    for k in range(nl):
+        Ik = cfg.I if k == 0 else cfg.H
+        o = AdjointResult(dh=None, dh0=None, dx=None, dW_ih=torch.empty(3 * cfg.H, Ik, device=dev), dW_hh=torch.empty(3 * cfg.H, cfg.H, device=dev),
+                          db_ih=torch.empty(3 * cfg.H, device=dev), db_hh=torch.empty(3 * cfg.H, device=dev))
+        garr[k] = _Grads(o.dW_ih.data_ptr(), o.dW_hh.data_ptr(), o.db_ih.data_ptr(), o.db_hh.data_ptr())
+        outs.append(o)
+    ws = _ws(stack_workspace_bytes(cfg, nl)[1], ws, dev)
+    rn = (ctypes.c_float * max(cfg.iters, 1))() if want_resnorm else None
+    _check(lib.mgrit_gru_stack_adjoint(ctypes.byref(cfg), nl, _param_array(layers), _f32(x), _f32(h0), _f32(gi0), _f32(h), _f32(dh_seed),
+                                       _f32(dhT), _f32(dh), _f32(dh0), _f32(dx), garr, rn, _ptr(ws), ws.numel(), _stream()))
+    return dh, dh0, dx, outs, (list(rn)[:cfg.iters] if want_resnorm else None)
 
 
 def xent_head_fwd_bwd(hT, Wc, bc, labels, ws=None):

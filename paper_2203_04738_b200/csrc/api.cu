@@ -481,6 +481,321 @@ int adjoint_impl(const mgrit_gru_cfg* cfg_in, bool serial, const gru_params* p, 
   return finish(s, false);
 }
 
+
+// ======================================================================================================
+// Stacked layers in one state: the state of a time point is the stack of all layers' hidden states, layer k's input
+// at a step is layer k-1's NEW state of the same step, and ONE multigrid cycle advances the whole stack.  Level
+// arrays are [N_l + 1][n_layers][B][H]; the cycle logic (Cycle) is the same, a "step" becomes a short sequence of
+// launches per layer: cell step on the raw result, FAS combination, input projection for the layer above.
+constexpr int kMaxStack = 8;
+
+size_t stack_max_rows(const mgrit_gru_cfg* c, const Hier& hr) {
+  size_t m = (size_t)c->B;
+  for (int l = 0; l + 1 < hr.L; ++l) {
+    size_t r = (size_t)((hr.N[l] + c->cf - 1) / c->cf) * c->B;
+    if (r > m) m = r;
+  }
+  return m;
+}
+
+struct StackFwdWs {
+  float* U[kMaxLevels]; float* G[kMaxLevels]; double* res_acc;
+  float* tmpPhi; float* gi_tmp; size_t maxM;
+  UmmaFwdWs um[kMaxStack];
+};
+
+mgrit_gru_cfg layer_cfg(const mgrit_gru_cfg& c, int k) {
+  mgrit_gru_cfg ck = c;
+  if (k > 0) ck.I = c.H;
+  return ck;
+}
+
+void plan_stack_fwd(const mgrit_gru_cfg* c, int nl, const Hier& hr, Ws& w, StackFwdWs* o) {
+  const size_t slot = (size_t)nl * c->B * c->H;
+  for (int l = 0; l < hr.L; ++l) {
+    o->U[l] = w.take<float>((size_t)(hr.N[l] + 1) * slot);
+    o->G[l] = l == 0 ? nullptr : w.take<float>((size_t)(hr.N[l] + 1) * slot);
+  }
+  o->res_acc = w.take<double>((size_t)(c->iters > 0 ? c->iters : 1));
+  o->maxM = stack_max_rows(c, hr);
+  o->tmpPhi = w.take<float>(o->maxM * c->H);
+  o->gi_tmp = w.take<float>(o->maxM * 3 * c->H);
+  if (c->operands == MGRIT_OPERANDS_BF16)
+    for (int k = 0; k < nl; ++k) {
+      mgrit_gru_cfg ck = layer_cfg(*c, k);
+      umma_plan_fwd(&ck, hr.N, hr.L, w.base, &w.off, &o->um[k]);
+    }
+}
+
+struct StackFwdCycle : Cycle {
+  int nl; const gru_params* p; const float* gi0; StackFwdWs* fw;
+  int launch_step(const StepDesc& d) override {
+    const size_t bh = (size_t)c->B * c->H, slot = (size_t)nl * bh;
+    const int M = d.nk * c->B;
+    const bool bf16 = c->operands == MGRIT_OPERANDS_BF16;
+    const i64 st = hr.stride_t[d.l];
+    for (int k = 0; k < nl; ++k) {
+      FwdStepArgs a;
+      a.M = M; a.B = c->B; a.H = c->H;
+      a.hin = U[d.l] + ((size_t)d.in_slot * nl + k) * bh; a.hin_ks = (i64)d.in_stride * slot;
+      a.hout = fw->tmpPhi; a.hout_ks = (i64)bh;            // the raw step result, rows (k, b) contiguous
+      a.hin_b = nullptr; a.hout_b = nullptr;
+      if (k == 0) { a.gi = gi0 + ((i64)st * d.tgt_slot - 1) * (i64)bh * 3; a.gi_ks = st * d.tgt_stride * (i64)bh * 3; }
+      else { a.gi = fw->gi_tmp; a.gi_ks = (i64)bh * 3; }
+      a.gadd = nullptr; a.gadd_ks = 0;
+      a.W_hh = p[k].W_hh; a.b_hh = p[k].b_hh; a.gamma = hr.gamma[d.l]; a.cell = c->cell; a.mode = 0;
+      if (bf16) { int r = umma_fwd_step(a, &fw->um[k], s); if (r) return r; }
+      else simt_fwd_step(a, s);
+      // level unknown = raw result + FAS term (mode 0), or right-hand side -= raw result (mode 1)
+      const float* g = d.gadd ? d.gadd + ((size_t)d.gadd_slot * nl + k) * bh : nullptr;
+      stream_combine_rows(fw->tmpPhi, g, (i64)d.gadd_stride * slot, d.out + ((size_t)d.out_slot * nl + k) * bh, (i64)d.out_stride * slot,
+                          c->B, c->H, (i64)M, d.mode, s);
+      if (k + 1 < nl) {   // input projection of the layer above: its input is this layer's raw new state
+        if (bf16) {
+          int r = umma_project_rows(fw->tmpPhi, fw->um[k + 1].xb, fw->um[k + 1].W_ih, p[k + 1].b_ih, fw->gi_tmp, M, c->H, 3 * c->H, s);
+          if (r) return r;
+        } else {
+          simt_project(fw->tmpPhi, p[k + 1].W_ih, p[k + 1].b_ih, fw->gi_tmp, M, c->H, 3 * c->H, s);
+        }
+      }
+    }
+    return MGRIT_OK;
+  }
+};
+
+bool stack_args_ok(const mgrit_gru_cfg* c, int nl, const gru_params* p) {
+  if (!c || !p || nl < 1 || nl > kMaxStack) return false;
+  for (int k = 0; k < nl; ++k)
+    if (!p[k].W_ih || !p[k].W_hh || !p[k].b_ih || !p[k].b_hh || !aligned32(p[k].W_ih, p[k].W_hh, p[k].b_ih, p[k].b_hh)) return false;
+  return true;
+}
+
+int stack_forward_impl(const mgrit_gru_cfg* cfg, int nl, const gru_params* p, const float* x, const float* h0, float* gi0, float* h,
+                       float* resnorm, void* ws, size_t ws_bytes, cudaStream_t s) {
+  if (!stack_args_ok(cfg, nl, p) || !x || !h0 || !gi0 || !h || !ws) return MGRIT_INVALID_ARG;
+  if (!aligned32(x, h0, gi0, h, ws)) return MGRIT_INVALID_ARG;
+  mgrit_gru_cfg c = *cfg;
+  Hier hr;
+  int rc = check_cfg(&c, &hr);
+  if (rc) return rc;
+  if (nl > 1) { mgrit_gru_cfg c1 = layer_cfg(c, 1); Hier h1; rc = check_cfg(&c1, &h1); if (rc) return rc; }
+  Ws w{(char*)ws, ws_bytes, 0};
+  StackFwdWs fw;
+  plan_stack_fwd(&c, nl, hr, w, &fw);
+  if (!w.fits()) return MGRIT_WORKSPACE_TOO_SMALL;
+  const size_t bh = (size_t)c.B * c.H, slot = (size_t)nl * bh;
+  if (c.operands == MGRIT_OPERANDS_BF16) {
+    rc = umma_prepare_fwd(&c, &p[0], x, gi0, &fw.um[0], s);
+    if (rc) return rc;
+    for (int k = 1; k < nl; ++k) {
+      umma_convert(p[k].W_hh, fw.um[k].W_hh, (i64)3 * c.H * c.H, s);
+      umma_convert(p[k].W_ih, fw.um[k].W_ih, (i64)3 * c.H * c.H, s);
+    }
+  } else {
+    simt_project(x, p[0].W_ih, p[0].b_ih, gi0, c.T * c.B, c.I, 3 * c.H, s);
+  }
+  cudaMemsetAsync(fw.U[0] + slot, 0, sizeof(float) * (size_t)c.T * slot, s);
+  for (int l = 0; l < hr.L; ++l) cudaMemcpyAsync(fw.U[l], h0, sizeof(float) * slot, cudaMemcpyDeviceToDevice, s);
+  StackFwdCycle cy;
+  cy.c = &c; cy.hr = hr; cy.s = s; cy.U = fw.U; cy.G = fw.G; cy.res_acc = fw.res_acc; cy.BH = slot;
+  cy.nl = nl; cy.p = p; cy.gi0 = gi0; cy.fw = &fw;
+  rc = cy.solve();
+  if (rc) return rc;
+  cudaMemcpyAsync(h, fw.U[0] + slot, sizeof(float) * (size_t)c.T * slot, cudaMemcpyDeviceToDevice, s);
+  if (resnorm && hr.L > 1 && c.iters > 0) {
+    rc = fetch_resnorm(fw.res_acc, resnorm, c.iters, s);
+    if (rc) return rc;
+    return finish(s, true);
+  }
+  return finish(s, false);
+}
+
+struct StackLayerAdj {
+  float *a[kMaxLevels], *cr[kMaxLevels], *cz[kMaxLevels], *cn[kMaxLevels], *cnp[kMaxLevels];                 // fp32 engine
+  __nv_bfloat16 *crb[kMaxLevels], *czb[kMaxLevels], *cnb[kMaxLevels], *cnpb[kMaxLevels];                     // tensor-core engine
+  float* hk;                 // this layer's given states [T, B, H], contiguous
+  float* gik;                // layers >= 1: input projection of the layer below's given states [T, B, 3H]
+  __nv_bfloat16* Wihb;       // layers >= 1, tensor-core engine: W_ih as bf16 [3H, H]
+  UmmaAdjWs um;
+};
+struct StackAdjWs {
+  float* U[kMaxLevels]; float* G[kMaxLevels]; double* res_acc;
+  float *tmpLin, *tmpDx, *lamk, *dxk, *dA_h, *dA_i; size_t maxM;
+  StackLayerAdj L[kMaxStack];
+};
+
+void plan_stack_adj(const mgrit_gru_cfg* c, int nl, const Hier& hr, Ws& w, StackAdjWs* o) {
+  const size_t bh = (size_t)c->B * c->H, slot = (size_t)nl * bh, TB = (size_t)c->T * c->B;
+  const bool bf16 = c->operands == MGRIT_OPERANDS_BF16;
+  for (int l = 0; l < hr.L; ++l) {
+    o->U[l] = w.take<float>((size_t)(hr.N[l] + 1) * slot);
+    o->G[l] = w.take<float>((size_t)(hr.N[l] + 1) * slot);
+  }
+  o->res_acc = w.take<double>((size_t)(c->iters > 0 ? c->iters : 1));
+  o->maxM = stack_max_rows(c, hr);
+  o->tmpLin = w.take<float>(o->maxM * c->H);
+  o->tmpDx = w.take<float>(o->maxM * c->H);
+  o->lamk = w.take<float>(TB * c->H);
+  o->dxk = w.take<float>(TB * c->H);
+  if (bf16) { o->dA_h = o->dA_i = nullptr; }
+  else { o->dA_h = w.take<float>(TB * 3 * c->H); o->dA_i = w.take<float>(TB * 3 * c->H); }
+  for (int k = 0; k < nl; ++k) {
+    StackLayerAdj& L = o->L[k];
+    for (int l = 0; l < hr.L; ++l) {
+      const size_t n = (size_t)hr.N[l] * bh;
+      L.a[l] = w.take<float>(n);
+      if (bf16) {
+        L.cr[l] = L.cz[l] = L.cn[l] = L.cnp[l] = nullptr;
+        L.crb[l] = w.take<__nv_bfloat16>(n); L.czb[l] = w.take<__nv_bfloat16>(n);
+        L.cnb[l] = w.take<__nv_bfloat16>(n); L.cnpb[l] = w.take<__nv_bfloat16>(n);
+      } else {
+        L.crb[l] = L.czb[l] = L.cnb[l] = L.cnpb[l] = nullptr;
+        L.cr[l] = w.take<float>(n); L.cz[l] = w.take<float>(n); L.cn[l] = w.take<float>(n); L.cnp[l] = w.take<float>(n);
+      }
+    }
+    L.hk = w.take<float>(TB * c->H);
+    L.gik = k > 0 ? w.take<float>(TB * 3 * c->H) : nullptr;
+    L.Wihb = (bf16 && k > 0) ? w.take<__nv_bfloat16>((size_t)3 * c->H * c->H) : nullptr;
+    if (bf16) { mgrit_gru_cfg ck = layer_cfg(*c, k); umma_plan_adj(&ck, hr.N, hr.L, w.base, &w.off, &L.um); }
+  }
+}
+
+struct StackAdjCycle : Cycle {
+  int nl; const gru_params* p; StackAdjWs* w;
+  int launch_step(const StepDesc& d) override {
+    const size_t bh = (size_t)c->B * c->H, slot = (size_t)nl * bh;
+    const int M = d.nk * c->B;
+    const bool bf16 = c->operands == MGRIT_OPERANDS_BF16;
+    // the step arriving at reversed point s applies the level's forward step stored at coefficient row N_l - s
+    const i64 row0 = (i64)(hr.N[d.l] - d.tgt_slot) * (i64)bh, coef_ks = -(i64)d.tgt_stride * (i64)bh;
+    for (int k = nl - 1; k >= 0; --k) {       // top layer first: what it sends to its input joins the layer below
+      StackLayerAdj& L = w->L[k];
+      AdjStepArgs a;
+      a.M = M; a.B = c->B; a.H = c->H;
+      if (k == nl - 1) { a.lin = U[d.l] + ((size_t)d.in_slot * nl + k) * bh; a.lin_ks = (i64)d.in_stride * slot; }
+      else { a.lin = w->tmpLin; a.lin_ks = (i64)bh; }
+      a.lout = d.out + ((size_t)d.out_slot * nl + k) * bh; a.lout_ks = (i64)d.out_stride * slot;
+      a.gadd = d.gadd ? d.gadd + ((size_t)d.gadd_slot * nl + k) * bh : nullptr; a.gadd_ks = (i64)d.gadd_stride * slot;
+      a.a = L.a[d.l] + row0; a.coef_ks = coef_ks; a.W_hh = p[k].W_hh; a.mode = d.mode;
+      if (bf16) { a.cr = a.cz = a.cn = nullptr; a.crb = L.crb[d.l] + row0; a.czb = L.czb[d.l] + row0; a.cnb = L.cnb[d.l] + row0; }
+      else { a.crb = a.czb = a.cnb = nullptr; a.cr = L.cr[d.l] + row0; a.cz = L.cz[d.l] + row0; a.cn = L.cn[d.l] + row0; }
+      if (bf16) { int r = umma_adj_step(a, &L.um, s); if (r) return r; }
+      else simt_adj_step(a, s);
+      if (k > 0) {
+        // total output sensitivity of the layer below = its own entry of the incoming unknown + [c_r|c_z|c_n'] * lin W_ih
+        AdjStepArgs b = a;
+        if (bf16) { b.cnb = L.cnpb[d.l] + row0; int r = umma_adj_dx(b, L.um.W_ihT, c->H, w->tmpDx, &L.um, s); if (r) return r; }
+        else { b.cn = L.cnp[d.l] + row0; simt_adj_dx(b, p[k].W_ih, c->H, w->tmpDx, s); }
+        stream_gather_rows(w->tmpLin, (i64)bh, U[d.l] + ((size_t)d.in_slot * nl + (k - 1)) * bh, (i64)d.in_stride * slot, d.nk, (i64)bh, s);
+        stream_add_rows(w->tmpLin, w->tmpDx, (i64)M * c->H, s);
+      }
+    }
+    return MGRIT_OK;
+  }
+};
+
+// time-parallel gradient pass of one layer given its total output sensitivities lam[T, B, H] (forward order, contiguous)
+int stack_layer_gradients(const mgrit_gru_cfg& ck, const gru_params* pk, const float* xk, const float* h0k, StackLayerAdj& L,
+                          StackAdjWs& w, float* dx, const gru_grads* g, cudaStream_t s) {
+  const i64 bh = (i64)ck.B * ck.H, M = (i64)ck.T * ck.B;
+  if (ck.operands == MGRIT_OPERANDS_BF16)
+    return umma_gradients(&ck, pk, xk, h0k, L.hk, w.lamk, bh, L.crb[0], L.czb[0], L.cnb[0], L.cnpb[0], dx, g, &L.um, s);
+  stream_form_dA(w.lamk, L.cr[0], L.cz[0], L.cn[0], L.cnp[0], w.dA_h, w.dA_i, M, ck.H, s);
+  simt_wgrad(w.dA_h, (int)M, 3 * ck.H, h0k, ck.B, L.hk, ck.H, g->dW_hh, s);
+  simt_wgrad(w.dA_i, (int)M, 3 * ck.H, nullptr, 0, xk, ck.I, g->dW_ih, s);
+  stream_colsum(w.dA_h, M, 3 * ck.H, g->db_hh, s);
+  stream_colsum(w.dA_i, M, 3 * ck.H, g->db_ih, s);
+  if (dx) simt_dgrad(w.dA_i, (int)M, 3 * ck.H, pk->W_ih, ck.I, dx, s);
+  return MGRIT_OK;
+}
+
+int stack_adjoint_impl(const mgrit_gru_cfg* cfg, int nl, const gru_params* p, const float* x, const float* h0, const float* gi0,
+                       const float* h, const float* dh_seed, const float* dhT, float* dh, float* dh0, float* dx, const gru_grads* g,
+                       float* resnorm, void* ws, size_t ws_bytes, cudaStream_t s) {
+  if (!stack_args_ok(cfg, nl, p) || !x || !h0 || !gi0 || !h || !dh0 || !g || !ws) return MGRIT_INVALID_ARG;
+  if (!dh_seed && !dhT) return MGRIT_INVALID_ARG;
+  if (!aligned32(x, h0, gi0, h, dh_seed, dhT, dh, dh0, dx, ws)) return MGRIT_INVALID_ARG;
+  for (int k = 0; k < nl; ++k)
+    if (!g[k].dW_ih || !g[k].dW_hh || !g[k].db_ih || !g[k].db_hh || !aligned32(g[k].dW_ih, g[k].dW_hh, g[k].db_ih, g[k].db_hh))
+      return MGRIT_INVALID_ARG;
+  mgrit_gru_cfg c = *cfg;
+  Hier hr;
+  int rc = check_cfg(&c, &hr);
+  if (rc) return rc;
+  if (nl > 1) { mgrit_gru_cfg c1 = layer_cfg(c, 1); Hier h1; rc = check_cfg(&c1, &h1); if (rc) return rc; }
+  Ws w{(char*)ws, ws_bytes, 0};
+  StackAdjWs aw;
+  plan_stack_adj(&c, nl, hr, w, &aw);
+  if (!w.fits()) return MGRIT_WORKSPACE_TOO_SMALL;
+  const size_t bh = (size_t)c.B * c.H, slot = (size_t)nl * bh;
+  const int T = c.T;
+  const bool bf16 = c.operands == MGRIT_OPERANDS_BF16;
+
+  // every layer's given states as their own [T, B, H] array; input projections of the layers above the first
+  for (int k = 0; k < nl; ++k) stream_gather_rows(aw.L[k].hk, (i64)bh, h + (size_t)k * bh, (i64)slot, T, (i64)bh, s);
+  for (int k = 0; k < nl; ++k) {
+    StackLayerAdj& L = aw.L[k];
+    mgrit_gru_cfg ck = layer_cfg(c, k);
+    if (bf16) {
+      rc = umma_prepare_adj(&ck, &p[k], h0 + (size_t)k * bh, L.hk, &L.um, s);
+      if (rc) return rc;
+    }
+    if (k > 0) {
+      if (bf16) {
+        umma_convert(p[k].W_ih, L.Wihb, (i64)3 * c.H * c.H, s);
+        rc = umma_project_rows(aw.L[k - 1].hk, L.um.xb, L.Wihb, p[k].b_ih, L.gik, T * c.B, c.H, 3 * c.H, s);
+        if (rc) return rc;
+      } else {
+        simt_project(aw.L[k - 1].hk, p[k].W_ih, p[k].b_ih, L.gik, T * c.B, c.H, 3 * c.H, s);
+      }
+    }
+    for (int l = 0; l < hr.L; ++l) {
+      LinArgs a;
+      a.M = hr.N[l] * c.B; a.B = c.B; a.H = c.H; a.h0 = h0 + (size_t)k * bh; a.h = L.hk; a.stride_t = hr.stride_t[l];
+      a.t0 = hr.rem[l]; a.gi = k == 0 ? gi0 : L.gik;
+      a.W_hh = p[k].W_hh; a.b_hh = p[k].b_hh; a.gamma = hr.gamma[l]; a.cell = c.cell;
+      a.a = L.a[l]; a.cr = L.cr[l]; a.cz = L.cz[l]; a.cn = L.cn[l]; a.cnp = L.cnp[l];
+      a.crb = L.crb[l]; a.czb = L.czb[l]; a.cnb = L.cnb[l]; a.cnpb = L.cnpb[l];
+      if (bf16) { rc = umma_linearise(a, &L.um, s); if (rc) return rc; }
+      else simt_linearise(a, s);
+    }
+  }
+  // mu_0 = lambda_T (all layers); zero initial guess elsewhere; fine-level source = reversed dh_seed
+  cudaMemsetAsync(aw.U[0], 0, sizeof(float) * (size_t)(T + 1) * slot, s);
+  cudaMemsetAsync(aw.G[0], 0, sizeof(float) * (size_t)(T + 1) * slot, s);
+  if (dh_seed) {
+    cudaMemcpyAsync(aw.U[0], dh_seed + (size_t)(T - 1) * slot, sizeof(float) * slot, cudaMemcpyDeviceToDevice, s);
+    if (T > 1) stream_gather_rows(aw.G[0] + slot, (i64)slot, dh_seed + (size_t)(T - 2) * slot, -(i64)slot, T - 1, (i64)slot, s);
+  }
+  if (dhT) stream_add_rows(aw.U[0] + (size_t)(nl - 1) * bh, dhT, (i64)bh, s);       // loss on the top layer's last state
+  for (int l = 1; l < hr.L; ++l) cudaMemcpyAsync(aw.U[l], aw.U[0], sizeof(float) * slot, cudaMemcpyDeviceToDevice, s);
+
+  StackAdjCycle cy;
+  cy.c = &c; cy.hr = hr; cy.s = s; cy.U = aw.U; cy.G = aw.G; cy.res_acc = aw.res_acc; cy.BH = slot;
+  cy.nl = nl; cy.p = p; cy.w = &aw;
+  rc = cy.solve();
+  if (rc) return rc;
+
+  if (dh) stream_gather_rows(dh, (i64)slot, aw.U[0] + (size_t)(T - 1) * slot, -(i64)slot, T, (i64)slot, s);
+  cudaMemcpyAsync(dh0, aw.U[0] + (size_t)T * slot, sizeof(float) * slot, cudaMemcpyDeviceToDevice, s);
+
+  // gradient pass, top layer first: a layer's total output sensitivity is its entry of the unknown plus what the layer
+  // above sends to its input (that layer's input gradient)
+  for (int k = nl - 1; k >= 0; --k) {
+    stream_gather_rows(aw.lamk, (i64)bh, aw.U[0] + (size_t)(T - 1) * slot + (size_t)k * bh, -(i64)slot, T, (i64)bh, s);
+    if (k < nl - 1) stream_add_rows(aw.lamk, aw.dxk, (i64)T * (i64)bh, s);
+    mgrit_gru_cfg ck = layer_cfg(c, k);
+    rc = stack_layer_gradients(ck, &p[k], k == 0 ? x : aw.L[k - 1].hk, h0 + (size_t)k * bh, aw.L[k], aw, k > 0 ? aw.dxk : dx, &g[k], s);
+    if (rc) return rc;
+  }
+  if (resnorm && hr.L > 1 && c.iters > 0) {
+    rc = fetch_resnorm(aw.res_acc, resnorm, c.iters, s);
+    if (rc) return rc;
+    return finish(s, true);
+  }
+  return finish(s, false);
+}
+
 }  // namespace
 }  // namespace mg
 
@@ -552,6 +867,29 @@ int gru_serial_backward(const mgrit_gru_cfg* cfg, const gru_params* p, const flo
                         const float* h, const float* dh_seed, const float* dhT, float* dh, float* dh0, float* dx,
                         const gru_grads* grads, void* ws, size_t ws_bytes, mgrit_stream_t stream) {
   return adjoint_impl(cfg, true, p, x, h0, gi, h, dh_seed, dhT, dh, dh0, dx, grads, nullptr, ws, ws_bytes, (cudaStream_t)stream);
+}
+
+int mgrit_gru_stack_workspace_bytes(const mgrit_gru_cfg* cfg, int32_t n_layers, size_t* fwd_bytes, size_t* adj_bytes) {
+  Hier hr;
+  int rc = check_cfg(cfg, &hr);
+  if (rc) return rc;
+  if (n_layers < 1 || n_layers > kMaxStack) return MGRIT_INVALID_ARG;
+  if (n_layers > 1) { mgrit_gru_cfg c1 = layer_cfg(*cfg, 1); Hier h1; rc = check_cfg(&c1, &h1); if (rc) return rc; }
+  if (fwd_bytes) { Ws w{nullptr, 0, 0}; StackFwdWs f; plan_stack_fwd(cfg, n_layers, hr, w, &f); *fwd_bytes = w.off + 256; }
+  if (adj_bytes) { Ws w{nullptr, 0, 0}; StackAdjWs a; plan_stack_adj(cfg, n_layers, hr, w, &a); *adj_bytes = w.off + 256; }
+  return MGRIT_OK;
+}
+
+int mgrit_gru_stack_forward(const mgrit_gru_cfg* cfg, int32_t n_layers, const gru_params* layers, const float* x, const float* h0,
+                            float* gi0, float* h, float* resnorm, void* ws, size_t ws_bytes, mgrit_stream_t stream) {
+  return stack_forward_impl(cfg, n_layers, layers, x, h0, gi0, h, resnorm, ws, ws_bytes, (cudaStream_t)stream);
+}
+
+int mgrit_gru_stack_adjoint(const mgrit_gru_cfg* cfg, int32_t n_layers, const gru_params* layers, const float* x, const float* h0,
+                            const float* gi0, const float* h, const float* dh_seed, const float* dhT, float* dh, float* dh0, float* dx,
+                            const gru_grads* grads, float* resnorm, void* ws, size_t ws_bytes, mgrit_stream_t stream) {
+  return stack_adjoint_impl(cfg, n_layers, layers, x, h0, gi0, h, dh_seed, dhT, dh, dh0, dx, grads, resnorm, ws, ws_bytes,
+                            (cudaStream_t)stream);
 }
 
 size_t xent_head_workspace_bytes(int32_t B, int32_t C) {

@@ -140,6 +140,9 @@ void simt_adj_step(const AdjStepArgs& a, cudaStream_t s);
 void simt_wgrad(const float* dA, int M, int H3, const float* first, int Bfirst, const float* rest, int C, float* dW, cudaStream_t s);
 // dx[m, c] = sum_n3 dA[m, n3] * W[n3, c]
 void simt_dgrad(const float* dA, int M, int H3, const float* W, int C, float* dx, cudaStream_t s);
+// out[m, c] = sum_{g,i} (c_g * lam)[m, i] W_ih[g*H + i, c]: what the step described by `a` (its cn slot holding c_n') sends to
+// the input of its cell, contiguous rows [M, C]
+void simt_adj_dx(const AdjStepArgs& a, const float* W_ih, int C, float* out, cudaStream_t s);
 
 // streaming kernels
 // r = uC - v at the C-points, sum of squares into *acc (double, device), copy of the C-point state
@@ -150,6 +153,9 @@ void stream_correct(float* uf, __nv_bfloat16* ufb, int cf, const float* uc, int 
 // dst[k] = src[k*src_ks], k = 0..nk-1, rows of rowlen floats (src_ks in elements, may be negative)
 void stream_gather_rows(float* dst, i64 dst_ks, const float* src, i64 src_ks, int nk, i64 rowlen, cudaStream_t s);
 void stream_add_rows(float* dst, const float* src, i64 n, cudaStream_t s);
+// tmp[M, H] contiguous (rows (k, b)) -> dst rows at dst + k*dst_ks + b*H: mode 0 dst = tmp (+ g rows, same indexing with g_ks),
+// mode 1 dst = dst - tmp
+void stream_combine_rows(const float* tmp, const float* g, i64 g_ks, float* dst, i64 dst_ks, int B, int H, i64 M, int mode, cudaStream_t s);
 // dA_h = [cr*lam | cz*lam | cn*lam], dA_i = [cr*lam | cz*lam | cnp*lam]  for M rows of H
 void stream_form_dA(const float* lam, const float* cr, const float* cz, const float* cn, const float* cnp,
                     float* dA_h, float* dA_i, i64 M, int H, cudaStream_t s);

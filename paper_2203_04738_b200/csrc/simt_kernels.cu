@@ -207,6 +207,11 @@ void simt_wgrad(const float* dA, int M, int H3, const float* first, int Bfirst, 
   launch<1, false, false>(KC_WGRAD, H3, C, M, DenseAT{dA, H3}, FirstRestBT{first, Bfirst, rest, C}, StoreEpi{dW, C}, s);
 }
 
+void simt_adj_dx(const AdjStepArgs& a, const float* W_ih, int C, float* out, cudaStream_t s) {
+  launch<1, true, false>(KC_ADJ_STEP, a.M, C, 3 * a.H, AdjA{a.lin, a.lin_ks, a.cr, a.cz, a.cn, a.coef_ks, a.B, a.H}, DenseBT{W_ih, C},
+                         StoreEpi{out, C}, s);
+}
+
 void simt_dgrad(const float* dA, int M, int H3, const float* W, int C, float* dx, cudaStream_t s) {
   launch<1, true, false>(KC_WGRAD, M, C, H3, DenseA{dA, H3}, DenseBT{W, C}, StoreEpi{dx, C}, s);
 }

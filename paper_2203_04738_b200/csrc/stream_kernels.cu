@@ -88,6 +88,29 @@ __global__ void __launch_bounds__(kThreads) gather_rows_kernel(float4* __restric
   }
 }
 
+// Stacked layers: raw step result tmp[m, :] (rows m = (k, b), contiguous) -> level unknown rows (k, b) at dst + k*dst_ks + b*H:
+// mode 0: dst = tmp + g (g optional, same indexing with g_ks);  mode 1: dst = dst - tmp  (FAS right-hand side).
+__global__ void __launch_bounds__(kThreads) combine_rows_kernel(const float4* __restrict__ tmp, const float4* __restrict__ g, i64 g_ks4,
+                                                                float4* __restrict__ dst, i64 dst_ks4, int B, int H4, i64 M, int mode) {
+  i64 total = M * H4;
+  for (i64 e = (i64)blockIdx.x * blockDim.x + threadIdx.x; e < total; e += (i64)gridDim.x * blockDim.x) {
+    i64 m = e / H4; int c = (int)(e % H4);
+    i64 k = m / B; int b = (int)(m % B);
+    float4 t = tmp[e];
+    float4* d = dst + k * dst_ks4 + (i64)b * H4 + c;
+    if (mode == 1) {
+      float4 o = *d;
+      *d = make_float4(o.x - t.x, o.y - t.y, o.z - t.z, o.w - t.w);
+    } else {
+      if (g) {
+        float4 a = g[k * g_ks4 + (i64)b * H4 + c];
+        t = make_float4(t.x + a.x, t.y + a.y, t.z + a.z, t.w + a.w);
+      }
+      *d = t;
+    }
+  }
+}
+
 __global__ void __launch_bounds__(kThreads) add_rows_kernel(float4* __restrict__ dst, const float4* __restrict__ src, i64 n4) {
   for (i64 e = (i64)blockIdx.x * blockDim.x + threadIdx.x; e < n4; e += (i64)gridDim.x * blockDim.x) {
     float4 a = dst[e], b = src[e];
@@ -261,6 +284,12 @@ void stream_gather_rows(float* dst, i64 dst_ks, const float* src, i64 src_ks, in
   i64 row4 = rowlen / 4;
   gather_rows_kernel<<<stream_grid((i64)nk * row4), kThreads, 0, s>>>(reinterpret_cast<float4*>(dst), dst_ks / 4,
                                                                       reinterpret_cast<const float4*>(src), src_ks / 4, nk, row4);
+  count_launch();
+}
+
+void stream_combine_rows(const float* tmp, const float* g, i64 g_ks, float* dst, i64 dst_ks, int B, int H, i64 M, int mode, cudaStream_t s) {
+  combine_rows_kernel<<<stream_grid(M * (H / 4)), kThreads, 0, s>>>(reinterpret_cast<const float4*>(tmp), reinterpret_cast<const float4*>(g),
+                                                                   g_ks / 4, reinterpret_cast<float4*>(dst), dst_ks / 4, B, H / 4, M, mode);
   count_launch();
 }
 

@@ -831,6 +831,22 @@ int umma_gradients(const mgrit_gru_cfg* c, const gru_params* p, const float* x, 
 
 void umma_convert(const float* src, __nv_bfloat16* dst, i64 n, cudaStream_t s) { convert(src, dst, n, s); }
 
+// out[M, 3H] = X[M, K] W^T + bias with X fp32 contiguous (converted into xb first) and W already bf16 [3H, K]
+int umma_project_rows(const float* X, bf16* xb, const bf16* Wb, const float* bias, float* out, int M, int K, int H3, cudaStream_t s) {
+  convert(X, xb, (i64)M * K, s);
+  return launch_gemm<256, false>(KC_PROJ, xb, K, Wb, K, M, H3, K, 0, H3, EpiBias{out, H3, bias, M, H3}, s) ? MGRIT_OK : MGRIT_CUDA_ERROR;
+}
+
+// out[M, C] = ([cr|cz|cn]*lam of the step `a`) W_ihT^T: the sensitivity a cell sends to its input (a.cnb holding c_n')
+int umma_adj_dx(const AdjStepArgs& a, const bf16* W_ihT, int C, float* out, UmmaAdjWs* w, cudaStream_t s) {
+  if (launch_pdl(pack_adj_kernel, dim3(pgrid((i64)a.M * (a.H / 4))), dim3(kPT), 0, s, a.lin, a.lin_ks, a.crb, a.czb, a.cnb, a.coef_ks,
+                 a.B, a.H / 4, (i64)a.M, reinterpret_cast<uint2*>(w->Apack)) != cudaSuccess)
+    return MGRIT_CUDA_ERROR;
+  count_launch();
+  return launch_gemm<256, false>(KC_ADJ_STEP, w->Apack, 3 * a.H, W_ihT, 3 * a.H, a.M, C, 3 * a.H, 0, C, EpiStore{out, C, a.M, C, 0}, s)
+             ? MGRIT_OK : MGRIT_CUDA_ERROR;
+}
+
 int umma_device_status() {
   const int dev = current_device_slot();
   if (dev < 0) return -1;

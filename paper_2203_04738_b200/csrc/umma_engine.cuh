@@ -32,6 +32,9 @@ void umma_plan_adj(const mgrit_gru_cfg* c, const int* N, int L, char* base, size
 int umma_prepare_fwd(const mgrit_gru_cfg* c, const gru_params* p, const float* x, float* gi, UmmaFwdWs* w, cudaStream_t s);
 int umma_prepare_adj(const mgrit_gru_cfg* c, const gru_params* p, const float* h0, const float* h, UmmaAdjWs* w, cudaStream_t s);
 void umma_convert(const float* src, __nv_bfloat16* dst, i64 n, cudaStream_t s);
+int umma_project_rows(const float* X, __nv_bfloat16* xb, const __nv_bfloat16* Wb, const float* bias, float* out, int M, int K, int H3,
+                      cudaStream_t s);
+int umma_adj_dx(const AdjStepArgs& a, const __nv_bfloat16* W_ihT, int C, float* out, UmmaAdjWs* w, cudaStream_t s);
 int umma_fwd_step(const FwdStepArgs& a, UmmaFwdWs* w, cudaStream_t s);
 int umma_linearise(const LinArgs& a, UmmaAdjWs* w, cudaStream_t s);
 int umma_adj_step(const AdjStepArgs& a, UmmaAdjWs* w, cudaStream_t s);
