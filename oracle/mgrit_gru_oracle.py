@@ -521,3 +521,167 @@ def stacked_mgrit_adjoint(layers, x, h0, h, dh_seed, cf, levels, iters, cell=CEL
         _, lam_tot[t - 1] = stacked_adjoint_step(layers, coefs_at(t, 1), lam[t - 1])
     grads = [weight_gradients(*layers[k], inps[k], h0[k], h[:, k], lam_tot[:, k], cell, dt, want_dx=(k == 0)) for k in range(nl)]
     return lam, lam0, grads, resnorm
+
+
+# --------------------------------------------------------------------------- Implicit LSTM
+# The paper's conclusion names the LSTM as a cell the same treatment applies to.  Reading taken here: the LSTM cell
+# state obeys  c_t = f c_{t-1} + i g = c_{t-1} + [ -(1-f) c_{t-1} + i g ], a unit-step forward-Euler update of
+# c' = -(1-f) c + i g, exactly as Eq. "gru-classic" reads the GRU; the stiff decay term -(1-f) c is taken implicitly
+# as in Eq. "gru-implicit":  (1 + gamma (1-f)) c_t = c_{t-1} + gamma i g.  The hidden state h_t = o tanh(c_t) has no
+# dynamics of its own and is re-evaluated from the new cell state.  gamma = 1 explicit is the textbook LSTM.
+# Gate order along 4H is i | f | g | o (the usual library order); the state of a time point is (c, h), stored as
+# [..., 2, B, H] with part 0 = c and part 1 = h.
+
+def lstm_gates(W_hh, b_hh, gi, h_prev):
+    H = h_prev.shape[-1]
+    pre = gi + h_prev @ W_hh.T + b_hh
+    return sigmoid(pre[..., 0:H]), sigmoid(pre[..., H:2 * H]), np.tanh(pre[..., 2 * H:3 * H]), sigmoid(pre[..., 3 * H:4 * H])
+
+
+def lstm_phi(W_hh, b_hh, gi, u_prev, gamma, cell):
+    """One LSTM step on the state u_prev[..., 0] = c, u_prev[..., 1] = h with the pre-computed input part gi."""
+    c_prev, h_prev = u_prev[..., 0, :, :], u_prev[..., 1, :, :]
+    i, f, g, o = lstm_gates(W_hh, b_hh, gi, h_prev)
+    q = gamma * (1.0 - f)
+    if cell == CELL_CLASSIC:
+        c = c_prev - q * c_prev + gamma * i * g
+    elif cell == CELL_IMPLICIT:
+        c = (c_prev + gamma * i * g) / (1.0 + q)
+    else:
+        raise ValueError("cell")
+    return np.stack([c, o * np.tanh(c)], axis=-3)
+
+
+def lstm_adjoint_coefficients(W_hh, b_hh, gi, u_prev, gamma, cell):
+    """Entries of the transposed Jacobian of one LSTM step.  With (L_c, L_h) the sensitivities of the step's outputs:
+
+        dc      = L_c + p * L_h                       total sensitivity of the new cell state
+        dA      = [ c_i*dc | c_f*dc | c_g*dc | c_o*L_h ]      = d(pre-activations) = d(gi)
+        L_c_in  = a * dc ,   L_h_in = dA W_hh
+
+    Returns a, p, c_i, c_f, c_g, c_o."""
+    c_prev, h_prev = u_prev[..., 0, :, :], u_prev[..., 1, :, :]
+    i, f, g, o = lstm_gates(W_hh, b_hh, gi, h_prev)
+    q = gamma * (1.0 - f)
+    if cell == CELL_IMPLICIT:
+        D = 1.0 + q
+        c = (c_prev + gamma * i * g) / D
+        a, dci, dcg, dcf = 1.0 / D, gamma * g / D, gamma * i / D, gamma * c / D
+    elif cell == CELL_CLASSIC:
+        c = c_prev - q * c_prev + gamma * i * g
+        a, dci, dcg, dcf = 1.0 - q, gamma * g, gamma * i, gamma * c_prev
+    else:
+        raise ValueError("cell")
+    th = np.tanh(c)
+    return a, o * (1.0 - th * th), dci * i * (1.0 - i), dcf * f * (1.0 - f), dcg * (1.0 - g * g), th * o * (1.0 - o)
+
+
+def lstm_adjoint_step(W_hh, coefs, lam_out):
+    """Applies the transposed Jacobian: lam_out[..., 0] = L_c, lam_out[..., 1] = L_h -> (input sensitivities, dA)."""
+    a, p, c_i, c_f, c_g, c_o = coefs
+    Lc, Lh = lam_out[..., 0, :, :], lam_out[..., 1, :, :]
+    dc = Lc + p * Lh
+    dA = np.concatenate([c_i * dc, c_f * dc, c_g * dc, c_o * Lh], axis=-1)
+    return np.stack([a * dc, dA @ W_hh], axis=-3), dA
+
+
+def lstm_serial_forward(W_ih, W_hh, b_ih, b_hh, x, u0, cell=CELL_IMPLICIT, dt=1.0):
+    """u0[2, B, H] = (c_0, h_0) -> u[T, 2, B, H]."""
+    T = x.shape[0]
+    gi = input_projection(W_ih, b_ih, x)
+    u = np.empty((T,) + u0.shape)
+    prev = u0
+    for t in range(T):
+        prev = lstm_phi(W_hh, b_hh, gi[t], prev, dt, cell)
+        u[t] = prev
+    return u
+
+
+def lstm_weight_gradients(W_ih, W_hh, b_ih, b_hh, x, u0, u, lam, cell=CELL_IMPLICIT, dt=1.0, want_dx=True):
+    """Time-parallel gradient pass: dA_t from the step-output sensitivities lam[T, 2, B, H] and the given states."""
+    gi = input_projection(W_ih, b_ih, x)
+    uprev = np.concatenate([u0[None], u[:-1]], axis=0)
+    coefs = lstm_adjoint_coefficients(W_hh, b_hh, gi, uprev, dt, cell)
+    _, dA = lstm_adjoint_step(W_hh, coefs, lam)
+    G4 = dA.shape[-1]
+    hprev = uprev[:, 1]
+    out = {"dW_hh": dA.reshape(-1, G4).T @ hprev.reshape(-1, hprev.shape[-1]), "dW_ih": dA.reshape(-1, G4).T @ x.reshape(-1, x.shape[-1]),
+           "db_hh": dA.reshape(-1, G4).sum(axis=0), "db_ih": dA.reshape(-1, G4).sum(axis=0)}
+    if want_dx:
+        out["dx"] = dA @ W_ih
+    return out
+
+
+def lstm_serial_backward(W_ih, W_hh, b_ih, b_hh, x, u0, u, du_seed, cell=CELL_IMPLICIT, dt=1.0):
+    """Exact BPTT.  du_seed[T, 2, B, H]: direct loss derivatives w.r.t. (c_t, h_t).  Returns lam, lam0, gradients."""
+    T = x.shape[0]
+    gi = input_projection(W_ih, b_ih, x)
+    ufull = np.concatenate([u0[None], u], axis=0)
+    lam = np.empty_like(u)
+    cur = du_seed[T - 1].copy()
+    for t in range(T, 0, -1):
+        lam[t - 1] = cur
+        back, _ = lstm_adjoint_step(W_hh, lstm_adjoint_coefficients(W_hh, b_hh, gi[t - 1], ufull[t - 1], dt, cell), cur)
+        cur = back + (du_seed[t - 2] if t >= 2 else 0.0)
+    return lam, cur, lstm_weight_gradients(W_ih, W_hh, b_ih, b_hh, x, u0, u, lam, cell, dt)
+
+
+def lstm_mgrit_forward(W_ih, W_hh, b_ih, b_hh, x, u0, cf, levels, iters, cell=CELL_IMPLICIT, relax_fine=RELAX_F,
+                       relax_coarse=RELAX_FCF, dt=1.0, cycle=CYCLE_V, ragged=False, u_init=None):
+    """MGRIT on the LSTM recurrence of the state (c, h); level l uses time step c_f^l and the input of fine step c_f^l j."""
+    T = x.shape[0]
+    N = level_sizes(T, cf, levels, ragged)
+    gi = input_projection(W_ih, b_ih, x)
+
+    def step(l, j, u_prev):
+        m = cf ** l
+        return lstm_phi(W_hh, b_hh, gi[m * j - 1], u_prev, m * dt, cell)
+
+    u = [None] * levels
+    g = [None] * levels
+    u[0] = np.zeros((T + 1,) + u0.shape)
+    u[0][0] = u0
+    if u_init is not None:
+        u[0][1:] = u_init
+    g[0] = np.zeros_like(u[0])
+    relax = _relax_list(levels, relax_fine, relax_coarse)
+    resnorm = []
+    if levels == 1:
+        fas_vcycle(step, N, cf, relax, u, g, 0, None)
+    else:
+        for _ in range(iters):
+            fas_vcycle(step, N, cf, relax, u, g, 0, resnorm, cycle)
+    return u[0][1:].copy(), resnorm
+
+
+def lstm_mgrit_adjoint(W_ih, W_hh, b_ih, b_hh, x, u0, u, du_seed, cf, levels, iters, cell=CELL_IMPLICIT, relax_fine=RELAX_F,
+                       relax_coarse=RELAX_FCF, dt=1.0, cycle=CYCLE_V, ragged=False, want_dx=True):
+    """MGRIT on the adjoint LSTM recurrence, time reversed, linearised at the GIVEN states (as mgrit_adjoint)."""
+    T = x.shape[0]
+    N = level_sizes(T, cf, levels, ragged)
+    gi = input_projection(W_ih, b_ih, x)
+    ufull = np.concatenate([u0[None], u], axis=0)
+
+    def step(l, s, mu_prev):
+        m = cf ** l
+        t_arrive = T - m * (s - 1)
+        back, _ = lstm_adjoint_step(W_hh, lstm_adjoint_coefficients(W_hh, b_hh, gi[t_arrive - 1], ufull[t_arrive - m], m * dt, cell), mu_prev)
+        return back
+
+    v = [None] * levels
+    g = [None] * levels
+    v[0] = np.zeros((T + 1,) + u0.shape)
+    v[0][0] = du_seed[T - 1]
+    g[0] = np.zeros_like(v[0])
+    for s in range(1, T):
+        g[0][s] = du_seed[T - s - 1]
+    relax = _relax_list(levels, relax_fine, relax_coarse)
+    resnorm = []
+    if levels == 1:
+        fas_vcycle(step, N, cf, relax, v, g, 0, None)
+    else:
+        for _ in range(iters):
+            fas_vcycle(step, N, cf, relax, v, g, 0, resnorm, cycle)
+    lam = np.ascontiguousarray(v[0][0:T][::-1])
+    lam0 = v[0][T].copy()
+    return lam, lam0, lstm_weight_gradients(W_ih, W_hh, b_ih, b_hh, x, u0, u, lam, cell, dt, want_dx), resnorm
