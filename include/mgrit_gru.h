@@ -169,6 +169,23 @@ int mgrit_gru_stack_adjoint(const mgrit_gru_cfg* cfg, int32_t n_layers, const gr
                             const float* gi0, const float* h, const float* dh_seed, const float* dhT, float* dh, float* dh0,
                             float* dx, const gru_grads* grads, float* resnorm, void* ws, size_t ws_bytes, mgrit_stream_t stream);
 
+/* Implicit LSTM (the paper's conclusion names the LSTM as a cell the same implicit treatment applies to).  Reading:
+ * the cell state is a unit-step forward-Euler update of c' = -(1-f) c + i g, as Eq. "gru-classic" reads the GRU, and
+ * the stiff decay term is taken implicitly as in Eq. "gru-implicit": (1 + gamma (1-f)) c_t = c_{t-1} + gamma i g;
+ * h_t = o tanh(c_t) is re-evaluated from the new cell state.  cfg->cell selects this (MGRIT_CELL_IMPLICIT) or the
+ * explicit update (MGRIT_CELL_CLASSIC: with dt = 1 the textbook LSTM); level l uses gamma = cf^l dt.
+ *   Parameters: gru_params with W_ih[4H,I], W_hh[4H,H], b_ih[4H], b_hh[4H], gate order i | f | g | o.
+ *   The state of a time point is (c, h): u0[2,B,H], u[T,2,B,H], du_seed / du likewise; gi[T,B,4H].
+ *   dhT[B,H]: loss derivative w.r.t. the last HIDDEN state.  grads: one gru_grads with the 4H-row shapes.
+ *   Everything else (cycles, relaxation, flags, resnorm, levels == 1 = serial sweep / exact BPTT) as for the GRU calls.
+ *   Operand mode MGRIT_OPERANDS_FP32 only (others: MGRIT_UNSUPPORTED). */
+int mgrit_lstm_workspace_bytes(const mgrit_gru_cfg* cfg, size_t* fwd_bytes, size_t* adj_bytes);
+int mgrit_lstm_forward(const mgrit_gru_cfg* cfg, const gru_params* p, const float* x, const float* u0, float* gi, float* u,
+                       float* resnorm, void* ws, size_t ws_bytes, mgrit_stream_t stream);
+int mgrit_lstm_adjoint(const mgrit_gru_cfg* cfg, const gru_params* p, const float* x, const float* u0, const float* gi,
+                       const float* u, const float* du_seed, const float* dhT, float* du, float* du0, float* dx,
+                       const gru_grads* grads, float* resnorm, void* ws, size_t ws_bytes, mgrit_stream_t stream);
+
 /* Classifier head on h_T with mean softmax cross-entropy (the loss whose gradient seeds the
  * backward block: w_T = grad_{h_T} L).  hT[B,H], Wc[C,H], bc[C], labels[B] (int32, device)
  * -> loss[1] (device), dhT[B,H], dWc[C,H], dbc[C].  ws: device scratch of at least

@@ -55,6 +55,10 @@ lib.mgrit_gru_stack_forward.argtypes = [ctypes.POINTER(Cfg), _i32, ctypes.POINTE
                                         ctypes.POINTER(ctypes.c_float), _vp, _sz, _vp]
 lib.mgrit_gru_stack_adjoint.argtypes = [ctypes.POINTER(Cfg), _i32, ctypes.POINTER(_Params), _vp, _vp, _vp, _vp, _vp, _vp, _vp, _vp, _vp,
                                         ctypes.POINTER(_Grads), ctypes.POINTER(ctypes.c_float), _vp, _sz, _vp]
+lib.mgrit_lstm_workspace_bytes.argtypes = [ctypes.POINTER(Cfg), ctypes.POINTER(_sz), ctypes.POINTER(_sz)]
+lib.mgrit_lstm_forward.argtypes = [ctypes.POINTER(Cfg), ctypes.POINTER(_Params), _vp, _vp, _vp, _vp, ctypes.POINTER(ctypes.c_float), _vp, _sz, _vp]
+lib.mgrit_lstm_adjoint.argtypes = [ctypes.POINTER(Cfg), ctypes.POINTER(_Params), _vp, _vp, _vp, _vp, _vp, _vp, _vp, _vp, _vp,
+                                   ctypes.POINTER(_Grads), ctypes.POINTER(ctypes.c_float), _vp, _sz, _vp]
 lib.xent_head_workspace_bytes.argtypes = [_i32, _i32]
 lib.xent_head_workspace_bytes.restype = _sz
 lib.xent_head_fwd_bwd.argtypes = [_i32, _i32, _i32, _vp, _vp, _vp, _vp, _vp, _vp, _vp, _vp, _vp, _sz, _vp]
@@ -236,6 +240,41 @@ def mgrit_gru_stack_adjoint(cfg, layers, x, h0, gi0, h, dh_seed=None, dhT=None, 
     _check(lib.mgrit_gru_stack_adjoint(ctypes.byref(cfg), nl, _param_array(layers), _f32(x), _f32(h0), _f32(gi0), _f32(h), _f32(dh_seed),
                                        _f32(dhT), _f32(dh), _f32(dh0), _f32(dx), garr, rn, _ptr(ws), ws.numel(), _stream()))
     return dh, dh0, dx, outs, (list(rn)[:cfg.iters] if want_resnorm else None)
+
+
+def lstm_workspace_bytes(cfg: Cfg):
+    f, a = _sz(0), _sz(0)
+    _check(lib.mgrit_lstm_workspace_bytes(ctypes.byref(cfg), ctypes.byref(f), ctypes.byref(a)))
+    return f.value, a.value
+
+
+def mgrit_lstm_forward(cfg, p, x, u0, want_resnorm=False, ws=None):
+    """Implicit LSTM by MGRIT.  p: dict W_ih[4H,I], W_hh[4H,H], b_ih, b_hh; u0[2,B,H] = (c_0, h_0).
+    -> (u[T,2,B,H], gi[T,B,4H], resnorm list or None)"""
+    dev = x.device
+    gi = torch.empty(cfg.T, cfg.B, 4 * cfg.H, device=dev)
+    u = torch.empty(cfg.T, 2, cfg.B, cfg.H, device=dev)
+    ws = _ws(lstm_workspace_bytes(cfg)[0], ws, dev)
+    rn = (ctypes.c_float * max(cfg.iters, 1))() if want_resnorm else None
+    _check(lib.mgrit_lstm_forward(ctypes.byref(cfg), ctypes.byref(_params(p)), _f32(x), _f32(u0), _f32(gi), _f32(u), rn, _ptr(ws),
+                                  ws.numel(), _stream()))
+    return u, gi, (list(rn)[:cfg.iters] if want_resnorm else None)
+
+
+def mgrit_lstm_adjoint(cfg, p, x, u0, gi, u, du_seed=None, dhT=None, want_dx=True, want_du=True, want_resnorm=False, ws=None):
+    """-> (du[T,2,B,H] or None, du0[2,B,H], AdjointResult with dx and the 4H-row gradients, resnorm)"""
+    dev = x.device
+    du = torch.empty(cfg.T, 2, cfg.B, cfg.H, device=dev) if want_du else None
+    du0 = torch.empty(2, cfg.B, cfg.H, device=dev)
+    o = AdjointResult(dh=None, dh0=None, dx=torch.empty(cfg.T, cfg.B, cfg.I, device=dev) if want_dx else None,
+                      dW_ih=torch.empty(4 * cfg.H, cfg.I, device=dev), dW_hh=torch.empty(4 * cfg.H, cfg.H, device=dev),
+                      db_ih=torch.empty(4 * cfg.H, device=dev), db_hh=torch.empty(4 * cfg.H, device=dev))
+    g = _Grads(o.dW_ih.data_ptr(), o.dW_hh.data_ptr(), o.db_ih.data_ptr(), o.db_hh.data_ptr())
+    ws = _ws(lstm_workspace_bytes(cfg)[1], ws, dev)
+    rn = (ctypes.c_float * max(cfg.iters, 1))() if want_resnorm else None
+    _check(lib.mgrit_lstm_adjoint(ctypes.byref(cfg), ctypes.byref(_params(p)), _f32(x), _f32(u0), _f32(gi), _f32(u), _f32(du_seed),
+                                  _f32(dhT), _f32(du), _f32(du0), _f32(o.dx), ctypes.byref(g), rn, _ptr(ws), ws.numel(), _stream()))
+    return du, du0, o, (list(rn)[:cfg.iters] if want_resnorm else None)
 
 
 def xent_head_fwd_bwd(hT, Wc, bc, labels, ws=None):

@@ -796,6 +796,183 @@ int stack_adjoint_impl(const mgrit_gru_cfg* cfg, int nl, const gru_params* p, co
   return finish(s, false);
 }
 
+
+// ======================================================================================================
+// Implicit LSTM: the state of a time point is (c, h); level arrays are [N_l + 1][2][B][H] (part 0 = c, part 1 = h) and
+// the same Cycle drives them.  fp32 engine only (four-gate FFMA products).
+struct LstmFwdWs { float* U[kMaxLevels]; float* G[kMaxLevels]; double* res_acc; float *tmpC, *tmpH; size_t maxM; };
+struct LstmAdjWs {
+  float* U[kMaxLevels]; float* G[kMaxLevels]; double* res_acc;
+  float *a[kMaxLevels], *p[kMaxLevels], *ci[kMaxLevels], *cf[kMaxLevels], *cg[kMaxLevels], *co[kMaxLevels];
+  float *tmpC, *tmpH, *hk, *dA; size_t maxM;
+};
+
+void plan_lstm_fwd(const mgrit_gru_cfg* c, const Hier& hr, Ws& w, LstmFwdWs* o) {
+  const size_t slot = (size_t)2 * c->B * c->H;
+  for (int l = 0; l < hr.L; ++l) {
+    o->U[l] = w.take<float>((size_t)(hr.N[l] + 1) * slot);
+    o->G[l] = l == 0 ? nullptr : w.take<float>((size_t)(hr.N[l] + 1) * slot);
+  }
+  o->res_acc = w.take<double>((size_t)(c->iters > 0 ? c->iters : 1));
+  o->maxM = stack_max_rows(c, hr);
+  o->tmpC = w.take<float>(o->maxM * c->H);
+  o->tmpH = w.take<float>(o->maxM * c->H);
+}
+
+void plan_lstm_adj(const mgrit_gru_cfg* c, const Hier& hr, Ws& w, LstmAdjWs* o) {
+  const size_t bh = (size_t)c->B * c->H, slot = 2 * bh, TB = (size_t)c->T * c->B;
+  for (int l = 0; l < hr.L; ++l) {
+    o->U[l] = w.take<float>((size_t)(hr.N[l] + 1) * slot);
+    o->G[l] = w.take<float>((size_t)(hr.N[l] + 1) * slot);
+    const size_t n = (size_t)hr.N[l] * bh;
+    o->a[l] = w.take<float>(n); o->p[l] = w.take<float>(n); o->ci[l] = w.take<float>(n);
+    o->cf[l] = w.take<float>(n); o->cg[l] = w.take<float>(n); o->co[l] = w.take<float>(n);
+  }
+  o->res_acc = w.take<double>((size_t)(c->iters > 0 ? c->iters : 1));
+  o->maxM = stack_max_rows(c, hr);
+  o->tmpC = w.take<float>(o->maxM * c->H);
+  o->tmpH = w.take<float>(o->maxM * c->H);
+  o->hk = w.take<float>(TB * c->H);
+  o->dA = w.take<float>(TB * 4 * c->H);
+}
+
+struct LstmFwdCycle : Cycle {
+  const gru_params* p; const float* gi; LstmFwdWs* fw;
+  int launch_step(const StepDesc& d) override {
+    const size_t bh = (size_t)c->B * c->H, slot = 2 * bh;
+    const i64 st = hr.stride_t[d.l];
+    LstmFwdArgs a;
+    a.M = d.nk * c->B; a.B = c->B; a.H = c->H;
+    a.cin = U[d.l] + (size_t)d.in_slot * slot; a.hin = a.cin + bh; a.in_ks = (i64)d.in_stride * slot;
+    a.cout = fw->tmpC; a.hout = fw->tmpH;
+    a.gi = gi + ((i64)st * d.tgt_slot - 1) * (i64)bh * 4; a.gi_ks = st * d.tgt_stride * (i64)bh * 4;
+    a.W_hh = p->W_hh; a.b_hh = p->b_hh; a.gamma = hr.gamma[d.l]; a.cell = c->cell;
+    simt_lstm_fwd_step(a, s);
+    for (int part = 0; part < 2; ++part) {
+      const float* g = d.gadd ? d.gadd + (size_t)d.gadd_slot * slot + part * bh : nullptr;
+      stream_combine_rows(part == 0 ? fw->tmpC : fw->tmpH, g, (i64)d.gadd_stride * slot, d.out + (size_t)d.out_slot * slot + part * bh,
+                          (i64)d.out_stride * slot, c->B, c->H, (i64)a.M, d.mode, s);
+    }
+    return MGRIT_OK;
+  }
+};
+
+struct LstmAdjCycle : Cycle {
+  const gru_params* p; LstmAdjWs* w;
+  int launch_step(const StepDesc& d) override {
+    const size_t bh = (size_t)c->B * c->H, slot = 2 * bh;
+    const i64 row0 = (i64)(hr.N[d.l] - d.tgt_slot) * (i64)bh;
+    LstmAdjArgs a;
+    a.M = d.nk * c->B; a.B = c->B; a.H = c->H;
+    a.lc = U[d.l] + (size_t)d.in_slot * slot; a.lh = a.lc + bh; a.in_ks = (i64)d.in_stride * slot;
+    a.lc_out = w->tmpC; a.lh_out = w->tmpH;
+    a.a = w->a[d.l] + row0; a.p = w->p[d.l] + row0; a.ci = w->ci[d.l] + row0; a.cf = w->cf[d.l] + row0;
+    a.cg = w->cg[d.l] + row0; a.co = w->co[d.l] + row0; a.coef_ks = -(i64)d.tgt_stride * (i64)bh;
+    a.W_hh = p->W_hh;
+    simt_lstm_adj_step(a, s);
+    for (int part = 0; part < 2; ++part) {
+      const float* g = d.gadd ? d.gadd + (size_t)d.gadd_slot * slot + part * bh : nullptr;
+      stream_combine_rows(part == 0 ? w->tmpC : w->tmpH, g, (i64)d.gadd_stride * slot, d.out + (size_t)d.out_slot * slot + part * bh,
+                          (i64)d.out_stride * slot, c->B, c->H, (i64)a.M, d.mode, s);
+    }
+    return MGRIT_OK;
+  }
+};
+
+int lstm_check(const mgrit_gru_cfg* cfg, Hier* hr) {
+  if (!cfg) return MGRIT_INVALID_ARG;
+  if (cfg->operands != MGRIT_OPERANDS_FP32) return MGRIT_UNSUPPORTED;      // four-gate products run on the fp32 engine only
+  return check_cfg(cfg, hr);
+}
+
+int lstm_forward_impl(const mgrit_gru_cfg* cfg, const gru_params* p, const float* x, const float* u0, float* gi, float* u,
+                      float* resnorm, void* ws, size_t ws_bytes, cudaStream_t s) {
+  if (!cfg || !p || !x || !u0 || !gi || !u || !ws || !p->W_ih || !p->W_hh || !p->b_ih || !p->b_hh) return MGRIT_INVALID_ARG;
+  if (!aligned32(x, u0, gi, u, ws, p->W_ih, p->W_hh, p->b_ih, p->b_hh)) return MGRIT_INVALID_ARG;
+  mgrit_gru_cfg c = *cfg;
+  Hier hr;
+  int rc = lstm_check(&c, &hr);
+  if (rc) return rc;
+  Ws w{(char*)ws, ws_bytes, 0};
+  LstmFwdWs fw;
+  plan_lstm_fwd(&c, hr, w, &fw);
+  if (!w.fits()) return MGRIT_WORKSPACE_TOO_SMALL;
+  const size_t slot = (size_t)2 * c.B * c.H;
+  simt_project(x, p->W_ih, p->b_ih, gi, c.T * c.B, c.I, 4 * c.H, s);
+  cudaMemsetAsync(fw.U[0] + slot, 0, sizeof(float) * (size_t)c.T * slot, s);
+  for (int l = 0; l < hr.L; ++l) cudaMemcpyAsync(fw.U[l], u0, sizeof(float) * slot, cudaMemcpyDeviceToDevice, s);
+  LstmFwdCycle cy;
+  cy.c = &c; cy.hr = hr; cy.s = s; cy.U = fw.U; cy.G = fw.G; cy.res_acc = fw.res_acc; cy.BH = slot;
+  cy.p = p; cy.gi = gi; cy.fw = &fw;
+  rc = cy.solve();
+  if (rc) return rc;
+  cudaMemcpyAsync(u, fw.U[0] + slot, sizeof(float) * (size_t)c.T * slot, cudaMemcpyDeviceToDevice, s);
+  if (resnorm && hr.L > 1 && c.iters > 0) {
+    rc = fetch_resnorm(fw.res_acc, resnorm, c.iters, s);
+    if (rc) return rc;
+    return finish(s, true);
+  }
+  return finish(s, false);
+}
+
+int lstm_adjoint_impl(const mgrit_gru_cfg* cfg, const gru_params* p, const float* x, const float* u0, const float* gi, const float* u,
+                      const float* du_seed, const float* dhT, float* du, float* du0, float* dx, const gru_grads* g, float* resnorm,
+                      void* ws, size_t ws_bytes, cudaStream_t s) {
+  if (!cfg || !p || !x || !u0 || !gi || !u || !du0 || !g || !ws) return MGRIT_INVALID_ARG;
+  if (!du_seed && !dhT) return MGRIT_INVALID_ARG;
+  if (!p->W_ih || !p->W_hh || !p->b_ih || !p->b_hh || !g->dW_ih || !g->dW_hh || !g->db_ih || !g->db_hh) return MGRIT_INVALID_ARG;
+  if (!aligned32(x, u0, gi, u, du_seed, dhT, du, du0, dx, ws, p->W_ih, p->W_hh, p->b_ih, p->b_hh, g->dW_ih, g->dW_hh, g->db_ih, g->db_hh))
+    return MGRIT_INVALID_ARG;
+  mgrit_gru_cfg c = *cfg;
+  Hier hr;
+  int rc = lstm_check(&c, &hr);
+  if (rc) return rc;
+  Ws w{(char*)ws, ws_bytes, 0};
+  LstmAdjWs aw;
+  plan_lstm_adj(&c, hr, w, &aw);
+  if (!w.fits()) return MGRIT_WORKSPACE_TOO_SMALL;
+  const size_t bh = (size_t)c.B * c.H, slot = 2 * bh;
+  const int T = c.T;
+  for (int l = 0; l < hr.L; ++l) {
+    LstmLinArgs a;
+    a.M = hr.N[l] * c.B; a.B = c.B; a.H = c.H; a.c0 = u0; a.h0 = u0 + bh; a.c = u; a.h = u + bh; a.ts = (i64)slot;
+    a.stride_t = hr.stride_t[l]; a.t0 = hr.rem[l]; a.gi = gi; a.W_hh = p->W_hh; a.b_hh = p->b_hh; a.gamma = hr.gamma[l]; a.cell = c.cell;
+    a.a = aw.a[l]; a.p = aw.p[l]; a.ci = aw.ci[l]; a.cf = aw.cf[l]; a.cg = aw.cg[l]; a.co = aw.co[l];
+    simt_lstm_linearise(a, s);
+  }
+  cudaMemsetAsync(aw.U[0], 0, sizeof(float) * (size_t)(T + 1) * slot, s);
+  cudaMemsetAsync(aw.G[0], 0, sizeof(float) * (size_t)(T + 1) * slot, s);
+  if (du_seed) {
+    cudaMemcpyAsync(aw.U[0], du_seed + (size_t)(T - 1) * slot, sizeof(float) * slot, cudaMemcpyDeviceToDevice, s);
+    if (T > 1) stream_gather_rows(aw.G[0] + slot, (i64)slot, du_seed + (size_t)(T - 2) * slot, -(i64)slot, T - 1, (i64)slot, s);
+  }
+  if (dhT) stream_add_rows(aw.U[0] + bh, dhT, (i64)bh, s);      // loss on the last hidden state
+  for (int l = 1; l < hr.L; ++l) cudaMemcpyAsync(aw.U[l], aw.U[0], sizeof(float) * slot, cudaMemcpyDeviceToDevice, s);
+  LstmAdjCycle cy;
+  cy.c = &c; cy.hr = hr; cy.s = s; cy.U = aw.U; cy.G = aw.G; cy.res_acc = aw.res_acc; cy.BH = slot;
+  cy.p = p; cy.w = &aw;
+  rc = cy.solve();
+  if (rc) return rc;
+  if (du) stream_gather_rows(du, (i64)slot, aw.U[0] + (size_t)(T - 1) * slot, -(i64)slot, T, (i64)slot, s);
+  cudaMemcpyAsync(du0, aw.U[0] + (size_t)T * slot, sizeof(float) * slot, cudaMemcpyDeviceToDevice, s);
+  // gradient pass over all fine steps at once: dA_t from the step-output sensitivities (read in place, reversed in time)
+  const i64 M = (i64)T * c.B;
+  const float* lam_c = aw.U[0] + (size_t)(T - 1) * slot;
+  simt_lstm_form_dA(lam_c, lam_c + bh, -(i64)slot, c.B, aw.p[0], aw.ci[0], aw.cf[0], aw.cg[0], aw.co[0], aw.dA, M, c.H, s);
+  stream_gather_rows(aw.hk, (i64)bh, u + bh, (i64)slot, T, (i64)bh, s);        // hidden states as their own [T, B, H] array
+  simt_wgrad(aw.dA, (int)M, 4 * c.H, u0 + bh, c.B, aw.hk, c.H, g->dW_hh, s);
+  simt_wgrad(aw.dA, (int)M, 4 * c.H, nullptr, 0, x, c.I, g->dW_ih, s);
+  stream_colsum(aw.dA, M, 4 * c.H, g->db_hh, s);
+  cudaMemcpyAsync(g->db_ih, g->db_hh, sizeof(float) * 4 * c.H, cudaMemcpyDeviceToDevice, s);
+  if (dx) simt_dgrad(aw.dA, (int)M, 4 * c.H, p->W_ih, c.I, dx, s);
+  if (resnorm && hr.L > 1 && c.iters > 0) {
+    rc = fetch_resnorm(aw.res_acc, resnorm, c.iters, s);
+    if (rc) return rc;
+    return finish(s, true);
+  }
+  return finish(s, false);
+}
+
 }  // namespace
 }  // namespace mg
 
@@ -890,6 +1067,26 @@ int mgrit_gru_stack_adjoint(const mgrit_gru_cfg* cfg, int32_t n_layers, const gr
                             const gru_grads* grads, float* resnorm, void* ws, size_t ws_bytes, mgrit_stream_t stream) {
   return stack_adjoint_impl(cfg, n_layers, layers, x, h0, gi0, h, dh_seed, dhT, dh, dh0, dx, grads, resnorm, ws, ws_bytes,
                             (cudaStream_t)stream);
+}
+
+int mgrit_lstm_workspace_bytes(const mgrit_gru_cfg* cfg, size_t* fwd_bytes, size_t* adj_bytes) {
+  Hier hr;
+  int rc = lstm_check(cfg, &hr);
+  if (rc) return rc;
+  if (fwd_bytes) { Ws w{nullptr, 0, 0}; LstmFwdWs f; plan_lstm_fwd(cfg, hr, w, &f); *fwd_bytes = w.off + 256; }
+  if (adj_bytes) { Ws w{nullptr, 0, 0}; LstmAdjWs a; plan_lstm_adj(cfg, hr, w, &a); *adj_bytes = w.off + 256; }
+  return MGRIT_OK;
+}
+
+int mgrit_lstm_forward(const mgrit_gru_cfg* cfg, const gru_params* p, const float* x, const float* u0, float* gi, float* u,
+                       float* resnorm, void* ws, size_t ws_bytes, mgrit_stream_t stream) {
+  return lstm_forward_impl(cfg, p, x, u0, gi, u, resnorm, ws, ws_bytes, (cudaStream_t)stream);
+}
+
+int mgrit_lstm_adjoint(const mgrit_gru_cfg* cfg, const gru_params* p, const float* x, const float* u0, const float* gi,
+                       const float* u, const float* du_seed, const float* dhT, float* du, float* du0, float* dx,
+                       const gru_grads* grads, float* resnorm, void* ws, size_t ws_bytes, mgrit_stream_t stream) {
+  return lstm_adjoint_impl(cfg, p, x, u0, gi, u, du_seed, dhT, du, du0, dx, grads, resnorm, ws, ws_bytes, (cudaStream_t)stream);
 }
 
 size_t xent_head_workspace_bytes(int32_t B, int32_t C) {

@@ -68,4 +68,43 @@ __device__ __forceinline__ CellLin cell_linearise(float gir, float giz, float gi
   return o;
 }
 
+// ---- Implicit LSTM: the cell state is an Euler step of c' = -(1-f) c + i g with step gamma, decay term implicit
+// (implicit) or explicit (classic; gamma = 1 is the textbook LSTM); h = o tanh(c) is re-evaluated from the new c.
+// Pre-activations: gi_* = W_i* x + b_i*, gh_* = W_h* h + b_h*, gate order i | f | g | o.
+struct LstmOut { float c, h; };
+template <bool FAST = false>
+__device__ __forceinline__ LstmOut lstm_forward(float gii, float gif, float gig, float gio, float ghi, float ghf, float ghg, float gho,
+                                                float cp, float gamma, int cell) {
+  float i = sigmoid_t<FAST>(gii + ghi), f = sigmoid_t<FAST>(gif + ghf), g = tanh_t<FAST>(gig + ghg), o = sigmoid_t<FAST>(gio + gho);
+  float q = gamma * (1.0f - f);
+  LstmOut r;
+  r.c = cell == MGRIT_CELL_IMPLICIT ? fmaf(gamma * i, g, cp) * inv_t<FAST>(1.0f + q) : fmaf(gamma * i, g, cp - q * cp);
+  r.h = o * tanh_t<FAST>(r.c);
+  return r;
+}
+
+// Transposed Jacobian of one LSTM step: with (L_c, L_h) the sensitivities of the outputs,
+//   dc = L_c + p*L_h;  d(pre-activations) = [ci*dc | cf*dc | cg*dc | co*L_h];  L_c_in = a*dc;  L_h_in = d(pre) W_hh
+struct LstmLin { float a, p, ci, cf, cg, co; };
+template <bool FAST = false>
+__device__ __forceinline__ LstmLin lstm_linearise(float gii, float gif, float gig, float gio, float ghi, float ghf, float ghg, float gho,
+                                                  float cp, float gamma, int cell) {
+  float i = sigmoid_t<FAST>(gii + ghi), f = sigmoid_t<FAST>(gif + ghf), g = tanh_t<FAST>(gig + ghg), o = sigmoid_t<FAST>(gio + gho);
+  float q = gamma * (1.0f - f);
+  float c, a, dci, dcg, dcf;
+  if (cell == MGRIT_CELL_IMPLICIT) {
+    float inv = inv_t<FAST>(1.0f + q);
+    c = fmaf(gamma * i, g, cp) * inv;
+    a = inv; dci = gamma * g * inv; dcg = gamma * i * inv; dcf = gamma * c * inv;
+  } else {
+    c = fmaf(gamma * i, g, cp - q * cp);
+    a = 1.0f - q; dci = gamma * g; dcg = gamma * i; dcf = gamma * cp;
+  }
+  float th = tanh_t<FAST>(c);
+  LstmLin r;
+  r.a = a; r.p = o * (1.0f - th * th);
+  r.ci = dci * i * (1.0f - i); r.cf = dcf * f * (1.0f - f); r.cg = dcg * (1.0f - g * g); r.co = th * o * (1.0f - o);
+  return r;
+}
+
 }  // namespace mg

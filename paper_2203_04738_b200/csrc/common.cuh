@@ -131,6 +131,40 @@ struct AdjStepArgs {
   int mode;                         // as FwdStepArgs
 };
 
+// ---- Implicit LSTM steps (state of a point = (c, h), 4H gate rows i | f | g | o); rows m = (k, b) as above ----
+struct LstmFwdArgs {
+  int M, B, H;
+  const float* cin; const float* hin; i64 in_ks;    // previous cell / hidden state rows (+ k*in_ks + b*H)
+  float* cout; float* hout;                         // raw new states, contiguous [M, H] each
+  const float* gi; i64 gi_ks;                       // input projection rows (+ k*gi_ks + b*4H)
+  const float* W_hh; const float* b_hh;             // [4H, H], [4H]
+  float gamma; int cell;
+};
+// coefficients of every step of one level: step j = 1..N leaves fine time t0 + stride_t*(j-1); the given states are
+// c/h[t] at c + (t-1)*ts / h + (t-1)*ts for t >= 1 and c0/h0 for t = 0; outputs [N*B, H] each
+struct LstmLinArgs {
+  int M, B, H;
+  const float *c0, *h0, *c, *h; i64 ts;
+  i64 stride_t, t0;
+  const float* gi;                                  // [T, B, 4H]
+  const float* W_hh; const float* b_hh; float gamma; int cell;
+  float *a, *p, *ci, *cf, *cg, *co;
+};
+// one adjoint step: dc = Lc + p*Lh; lc_out = a*dc; lh_out = [ci*dc | cf*dc | cg*dc | co*Lh] W_hh   (raw, contiguous [M, H] each)
+struct LstmAdjArgs {
+  int M, B, H;
+  const float* lc; const float* lh; i64 in_ks;      // incoming sensitivities rows
+  float* lc_out; float* lh_out;
+  const float *a, *p, *ci, *cf, *cg, *co; i64 coef_ks;
+  const float* W_hh;
+};
+void simt_lstm_fwd_step(const LstmFwdArgs& a, cudaStream_t s);
+void simt_lstm_linearise(const LstmLinArgs& a, cudaStream_t s);
+void simt_lstm_adj_step(const LstmAdjArgs& a, cudaStream_t s);
+// dA[m, :] = [ci*dc | cf*dc | cg*dc | co*Lh] for M contiguous rows (gradient pass); lam rows (c, h) at lc/lh + m-row stride lam_ks per time
+void simt_lstm_form_dA(const float* lc, const float* lh, i64 lam_ts, int B, const float* p, const float* ci, const float* cf,
+                       const float* cg, const float* co, float* dA, i64 M, int H, cudaStream_t s);
+
 // SIMT (fp32 FFMA) engine
 void simt_project(const float* x, const float* W_ih, const float* b_ih, float* gi, int M, int I, int H3, cudaStream_t s);
 void simt_fwd_step(const FwdStepArgs& a, cudaStream_t s);

@@ -183,7 +183,98 @@ struct AdjEpi {
   }
 };
 
+// ---------------------------------------------------------------- Implicit LSTM (four gates)
+struct LstmFwdEpi {
+  LstmFwdArgs a;
+  __device__ void operator()(int m, int n, const float* v) const {
+    int k = m / a.B, b = m % a.B;
+    const float* gi = a.gi + (i64)k * a.gi_ks + (i64)b * 4 * a.H;
+    float cp = a.cin[(i64)k * a.in_ks + (i64)b * a.H + n];
+    LstmOut o = lstm_forward(gi[n], gi[a.H + n], gi[2 * a.H + n], gi[3 * a.H + n], v[0] + a.b_hh[n], v[1] + a.b_hh[a.H + n],
+                             v[2] + a.b_hh[2 * a.H + n], v[3] + a.b_hh[3 * a.H + n], cp, a.gamma, a.cell);
+    a.cout[(i64)m * a.H + n] = o.c;
+    a.hout[(i64)m * a.H + n] = o.h;
+  }
+};
+struct LstmLinA {   // hidden state entering step j = m/B + 1: h at fine time t0 + stride*(j-1)
+  const float* h0; const float* h; i64 ts, stride_t, t0; int B, H;
+  __device__ float operator()(int m, int k) const {
+    int j1 = m / B, b = m % B;
+    const i64 t = t0 + (i64)j1 * stride_t;
+    return t == 0 ? h0[(i64)b * H + k] : h[(t - 1) * ts + (i64)b * H + k];
+  }
+};
+struct LstmLinEpi {
+  LstmLinArgs a;
+  __device__ void operator()(int m, int n, const float* v) const {
+    int j1 = m / a.B, b = m % a.B;
+    const i64 t = a.t0 + (i64)j1 * a.stride_t;
+    const float* gi = a.gi + ((t + a.stride_t - 1) * a.B + b) * 4 * a.H;
+    float cp = t == 0 ? a.c0[(i64)b * a.H + n] : a.c[(t - 1) * a.ts + (i64)b * a.H + n];
+    LstmLin L = lstm_linearise(gi[n], gi[a.H + n], gi[2 * a.H + n], gi[3 * a.H + n], v[0] + a.b_hh[n], v[1] + a.b_hh[a.H + n],
+                               v[2] + a.b_hh[2 * a.H + n], v[3] + a.b_hh[3 * a.H + n], cp, a.gamma, a.cell);
+    i64 o = (i64)m * a.H + n;
+    a.a[o] = L.a; a.p[o] = L.p; a.ci[o] = L.ci; a.cf[o] = L.cf; a.cg[o] = L.cg; a.co[o] = L.co;
+  }
+};
+struct LstmAdjA {   // A[m, g*H + i] = coefficient_g * (g < 3 ? Lc + p*Lh : Lh)
+  LstmAdjArgs a;
+  __device__ float operator()(int m, int k) const {
+    int kk = m / a.B, b = m % a.B, g = k / a.H, i = k - g * a.H;
+    i64 ci = (i64)kk * a.coef_ks + (i64)b * a.H + i, li = (i64)kk * a.in_ks + (i64)b * a.H + i;
+    float lh = a.lh[li];
+    if (g == 3) return a.co[ci] * lh;
+    float dc = a.lc[li] + a.p[ci] * lh;
+    return (g == 0 ? a.ci[ci] : (g == 1 ? a.cf[ci] : a.cg[ci])) * dc;
+  }
+};
+__global__ void __launch_bounds__(256) lstm_adj_c_kernel(LstmAdjArgs a) {
+  i64 total = (i64)a.M * a.H;
+  for (i64 e = (i64)blockIdx.x * blockDim.x + threadIdx.x; e < total; e += (i64)gridDim.x * blockDim.x) {
+    i64 m = e / a.H; int i = (int)(e % a.H);
+    i64 kk = m / a.B; int b = (int)(m % a.B);
+    i64 ci = kk * a.coef_ks + (i64)b * a.H + i, li = kk * a.in_ks + (i64)b * a.H + i;
+    a.lc_out[e] = a.a[ci] * (a.lc[li] + a.p[ci] * a.lh[li]);
+  }
+}
+__global__ void __launch_bounds__(256) lstm_form_dA_kernel(const float* __restrict__ lc, const float* __restrict__ lh, i64 lam_ts, int B,
+                                                           const float* __restrict__ p, const float* __restrict__ ci,
+                                                           const float* __restrict__ cf, const float* __restrict__ cg,
+                                                           const float* __restrict__ co, float* __restrict__ dA, i64 M, int H) {
+  i64 total = M * H;
+  for (i64 e = (i64)blockIdx.x * blockDim.x + threadIdx.x; e < total; e += (i64)gridDim.x * blockDim.x) {
+    i64 m = e / H; int i = (int)(e % H);
+    i64 t = m / B; int b = (int)(m % B);
+    i64 li = t * lam_ts + (i64)b * H + i;
+    float h = lh[li], dc = lc[li] + p[e] * h;
+    float* d = dA + m * 4 * H + i;
+    d[0] = ci[e] * dc; d[H] = cf[e] * dc; d[2 * H] = cg[e] * dc; d[3 * H] = co[e] * h;
+  }
+}
+
 }  // namespace
+
+void simt_lstm_fwd_step(const LstmFwdArgs& a, cudaStream_t s) {
+  launch<4, true, true>(KC_FWD_STEP, a.M, a.H, a.H, StridedRowsA{a.hin, a.in_ks, a.B, a.H}, GateW{a.W_hh, a.H, a.H}, LstmFwdEpi{a}, s);
+}
+void simt_lstm_linearise(const LstmLinArgs& a, cudaStream_t s) {
+  launch<4, true, true>(KC_LINEARISE, a.M, a.H, a.H, LstmLinA{a.h0, a.h, a.ts, a.stride_t, a.t0, a.B, a.H}, GateW{a.W_hh, a.H, a.H},
+                        LstmLinEpi{a}, s);
+}
+void simt_lstm_adj_step(const LstmAdjArgs& a, cudaStream_t s) {
+  i64 items = (i64)a.M * a.H;
+  int grid = (int)((items + 255) / 256 < 1184 ? (items + 255) / 256 : 1184);
+  lstm_adj_c_kernel<<<grid < 1 ? 1 : grid, 256, 0, s>>>(a);
+  count_launch();
+  launch<1, true, false>(KC_ADJ_STEP, a.M, a.H, 4 * a.H, LstmAdjA{a}, DenseBT{a.W_hh, a.H}, StoreEpi{a.lh_out, a.H}, s);
+}
+void simt_lstm_form_dA(const float* lc, const float* lh, i64 lam_ts, int B, const float* p, const float* ci, const float* cf,
+                       const float* cg, const float* co, float* dA, i64 M, int H, cudaStream_t s) {
+  i64 items = M * H;
+  int grid = (int)((items + 255) / 256 < 1184 ? (items + 255) / 256 : 1184);
+  lstm_form_dA_kernel<<<grid < 1 ? 1 : grid, 256, 0, s>>>(lc, lh, lam_ts, B, p, ci, cf, cg, co, dA, M, H);
+  count_launch();
+}
 
 void simt_project(const float* x, const float* W_ih, const float* b_ih, float* gi, int M, int I, int H3, cudaStream_t s) {
   launch<1, true, true>(KC_PROJ, M, H3, I, DenseA{x, I}, DenseB{W_ih, I}, BiasEpi{gi, H3, b_ih}, s);

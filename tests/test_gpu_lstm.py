@@ -1,0 +1,68 @@
+"""GPU parity of the Implicit LSTM solved by MGRIT (fp32 engine) against the fp64 oracle at the same cycle count:
+states (c, h), adjoint sensitivities, all gradients; cycle variants; the serial sweep and exact BPTT (levels = 1)."""
+import numpy as np
+import pytest
+import torch
+
+from oracle import mgrit_gru_oracle as O
+from tests.gpu_util import max_abs, rel_inf, to_dev
+
+pytestmark = pytest.mark.gpu
+
+CASES = [
+    dict(T=64, B=2, I=16, H=32, cf=4, levels=2, rf=0, rc=1, flags=0, cell=1),
+    dict(T=64, B=3, I=24, H=40, cf=2, levels=4, rf=1, rc=1, flags=0, cell=1),
+    dict(T=50, B=2, I=16, H=32, cf=3, levels=3, rf=0, rc=2, flags=2 | 4, cell=1),     # F-cycle, ragged T, FCFCF inside
+    dict(T=32, B=2, I=16, H=32, cf=2, levels=2, rf=0, rc=1, flags=0, cell=0),         # explicit (classic) cell, gamma <= 2
+    dict(T=40, B=4, I=16, H=32, cf=4, levels=1, rf=0, rc=0, flags=0, cell=1),         # serial sweep + exact BPTT
+]
+
+
+@pytest.mark.parametrize("c", CASES, ids=lambda c: "T{T}B{B}H{H}cf{cf}L{levels}r{rf}{rc}f{flags}c{cell}".format(**c))
+def test_lstm_solve(c):
+    from paper_2203_04738_b200 import binding as B
+    rng = np.random.default_rng(700 + c["T"])
+    T, Bn, I, H = c["T"], c["B"], c["I"], c["H"]
+    k = 1.0 / np.sqrt(H)
+    P32 = [rng.uniform(-k, k, s).astype(np.float32) for s in ((4 * H, I), (4 * H, H), (4 * H,), (4 * H,))]
+    x32 = np.maximum(rng.standard_normal((T, Bn, I)), 0).astype(np.float32)
+    u032 = (rng.standard_normal((2, Bn, H)) * 0.3).astype(np.float32)
+    P = [a.astype(np.float64) for a in P32]
+    p = dict(zip(("W_ih", "W_hh", "b_ih", "b_hh"), [to_dev(a) for a in P32]))
+    cfg = B.make_cfg(T, Bn, I, H, cf=c["cf"], levels=c["levels"], iters=2, cell=c["cell"], relax_fine=c["rf"], relax_coarse=c["rc"],
+                     operands=B.OPERANDS_FP32, flags=c["flags"])
+    kw = dict(cf=c["cf"], levels=c["levels"], iters=2, cell=c["cell"], relax_fine=c["rf"], relax_coarse=c["rc"],
+              cycle=O.CYCLE_F if c["flags"] & 2 else O.CYCLE_V, ragged=bool(c["flags"] & 4))
+    multi = c["levels"] > 1
+    u, gi, rn = B.mgrit_lstm_forward(cfg, p, to_dev(x32), to_dev(u032), want_resnorm=multi)
+    uref, rref = O.lstm_mgrit_forward(*P, x32.astype(np.float64), u032.astype(np.float64), **kw)
+    assert max_abs(u.cpu().numpy(), uref) < 1e-4
+    if multi:
+        for a, b in zip(rn, rref):
+            assert abs(a - b) <= 1e-3 * b + 1e-5
+    else:
+        assert max_abs(u.cpu().numpy(), O.lstm_serial_forward(*P, x32.astype(np.float64), u032.astype(np.float64), cell=c["cell"])) < 1e-4
+    un = u.cpu().numpy().astype(np.float64)
+    seed = (rng.standard_normal(un.shape) * 0.05).astype(np.float32)
+    dhT = rng.standard_normal((Bn, H)).astype(np.float32)
+    du, du0, r, rna = B.mgrit_lstm_adjoint(cfg, p, to_dev(x32), to_dev(u032), gi, u, du_seed=to_dev(seed), dhT=to_dev(dhT), want_resnorm=multi)
+    seed64 = seed.astype(np.float64)
+    seed64[-1, 1] += dhT
+    if multi:
+        lam, lam0, g, rref = O.lstm_mgrit_adjoint(*P, x32.astype(np.float64), u032.astype(np.float64), un, seed64, **kw)
+        for a, b in zip(rna, rref):
+            assert abs(a - b) <= 1e-3 * b + 1e-7
+    else:
+        lam, lam0, g = O.lstm_serial_backward(*P, x32.astype(np.float64), u032.astype(np.float64), un, seed64, cell=c["cell"])
+    assert rel_inf(du.cpu().numpy(), lam) < 1e-3
+    assert max_abs(du0.cpu().numpy(), lam0) / np.max(np.abs(lam)) < 1e-3
+    for key in ("dx", "dW_ih", "dW_hh", "db_ih", "db_hh"):
+        assert rel_inf(getattr(r, key).cpu().numpy(), g[key]) < 1e-3, key
+    assert B.last_device_status() == 0
+
+
+def test_lstm_rejects_other_operand_modes():
+    from paper_2203_04738_b200 import binding as B
+    with pytest.raises(B.MgritError) as e:
+        B.lstm_workspace_bytes(B.make_cfg(64, 8, 64, 128, cf=4, levels=2, operands=B.OPERANDS_BF16))
+    assert e.value.code == -4
