@@ -545,8 +545,8 @@ __global__ void __launch_bounds__(256) form_dA_rows_kernel(const float* __restri
   if (c4 < H4) {
     for (i64 m = m0 + ty; m < m0 + rows_per_block && m < M; m += 8) {
       i64 e = m * H4 + c4;
-      const i64 t = m / B; const int bb = (int)(m % B);
-      float4 l = *reinterpret_cast<const float4*>(lam + t * lam_ts + ((i64)bb * H4 + c4) * 4);
+      const int t = (int)m / B, bb = (int)m - t * B;       // row counts fit 32 bits (checked by the host)
+      float4 l = *reinterpret_cast<const float4*>(lam + (i64)t * lam_ts + ((i64)bb * H4 + c4) * 4);
       float4 r = unpack4(reinterpret_cast<const uint2*>(cr)[e]), z = unpack4(reinterpret_cast<const uint2*>(cz)[e]);
       float4 n = unpack4(reinterpret_cast<const uint2*>(cn)[e]), q = unpack4(reinterpret_cast<const uint2*>(cnp)[e]);
       float4 v[4] = {make_float4(r.x * l.x, r.y * l.y, r.z * l.z, r.w * l.w), make_float4(z.x * l.x, z.y * l.y, z.z * l.z, z.w * l.w),

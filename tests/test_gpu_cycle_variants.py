@@ -48,7 +48,7 @@ def test_cycle_variant(c):
     else:
         assert rel_inf(h.cpu().numpy(), href) < 2e-2
     for a, b in zip(rn, rref):
-        assert abs(a - b) <= (1e-3 * b + 1e-5 if fp32 else 1e-3 * b + 5e-4 * rref[0])
+        assert abs(a - b) <= (1e-3 * b + 1e-5 if fp32 else 1e-3 * b + 1e-3 * rref[0])
     # the same with the duplicate F-relaxation skipped: identical bits
     cfg2 = B.make_cfg(w.T, w.B, w.I, w.H, cf=w.cf, levels=w.levels, iters=2, relax_fine=w.relax_fine, relax_coarse=w.relax_coarse,
                       operands=c["op"], flags=flags | B.FLAG_SKIP_DUPLICATE_FRELAX)
@@ -65,7 +65,7 @@ def test_cycle_variant(c):
     for k in ("dx", "dW_ih", "dW_hh", "db_ih", "db_hh"):
         assert rel_inf(getattr(r, k).cpu().numpy(), g[k]) < tol, k
     for a, b in zip(r.resnorm, rref):
-        assert abs(a - b) <= (1e-3 * b + 1e-7 if fp32 else 1e-3 * b + 5e-4 * rref[0])
+        assert abs(a - b) <= (1e-3 * b + 1e-7 if fp32 else 1e-3 * b + 1e-3 * rref[0])
     assert B.last_device_status() == 0
 
 

@@ -1,9 +1,10 @@
 """GPU parity, bf16 tensor-core operand mode (tcgen05 GEMMs, fp32 accumulation, fp32 state), against the
 fp64 oracle at the same cycle count.  Tolerance: 2e-2 norm-relative (||a-b||_inf / ||b||_inf) on h, on
-every gradient and on dh; residual norms within 1e-3 of their own size plus 5e-4 of the first cycle's residual.
+every gradient and on dh; residual norms within 1e-3 of their own size plus 1e-3 of the first cycle's residual.
 (A late residual is a difference of nearly equal bf16-perturbed states, so its error has a floor that scales with the
 state error, i.e. with the first residual r_0.  Measured over these workloads at up to five cycles: the mismatch is
-at most 7e-4 of the residual while the residual is above 1e-2 r_0, and never above 3.1e-4 r_0.)
+at most 7e-4 of the residual while the residual is above 1e-2 r_0, and never above 3.1e-4 r_0; the fastest-converging
+variant case, F-cycles with FCFCF relaxation, reaches its floor in the second cycle with a mismatch of 6.6e-4 r_0.)
 
 Small shapes are compared element by element over everything.  The full-size configurations are compared
 on sampled batch rows (rows of a batch never interact in the forward or adjoint recurrences, so the oracle
@@ -46,7 +47,7 @@ def _full_case(B, w, check_grads=True):
     assert rel_inf(gi.cpu().numpy(), O.input_projection(P[0], P[2], xr)) < TOL
     assert rel_inf(h.cpu().numpy(), href) < TOL
     for a, b in zip(rn, rref):
-        assert abs(a - b) <= 1e-3 * b + 5e-4 * rref[0]   # floor: bf16 noise of the states, a fraction of the first residual
+        assert abs(a - b) <= 1e-3 * b + 1e-3 * rref[0]   # floor: bf16 noise of the states, a fraction of the first residual
     hs, _ = B.gru_serial_forward(cfg, p, x, h0)
     assert rel_inf(hs.cpu().numpy(), O.serial_forward(*P, xr, h0r)) < TOL
     if not check_grads:
@@ -62,7 +63,7 @@ def _full_case(B, w, check_grads=True):
     gi64 = None
     lam, lam0, g, rref = O.mgrit_adjoint(*P, xr, h0r, hn, seed64, iters=w.iters_adj, **kw)
     for a, b in zip(r.resnorm, rref):
-        assert abs(a - b) <= 1e-3 * b + 5e-4 * rref[0]   # floor: bf16 noise of the states, a fraction of the first residual
+        assert abs(a - b) <= 1e-3 * b + 1e-3 * rref[0]   # floor: bf16 noise of the states, a fraction of the first residual
     assert rel_inf(r.dh.cpu().numpy(), lam) < TOL
     assert max_abs(r.dh0.cpu().numpy(), lam0) / np.max(np.abs(lam)) < TOL
     for k in ("dx", "dW_ih", "dW_hh", "db_ih", "db_hh"):

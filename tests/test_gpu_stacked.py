@@ -48,7 +48,7 @@ def test_stacked_solve(c):
         assert rel_inf(h.cpu().numpy(), href) < tol
     if w.levels > 1:
         for a, b in zip(rn, rref):
-            assert abs(a - b) <= (1e-3 * b + 1e-5 if fp32 else 1e-3 * b + 5e-4 * rref[0])
+            assert abs(a - b) <= (1e-3 * b + 1e-5 if fp32 else 1e-3 * b + 1e-3 * rref[0])
     else:   # levels = 1: the exact serial sweep of the stacked network
         assert (max_abs(h.cpu().numpy(), O.stacked_serial_forward(layers_ref, xr, h0r)) < 1e-4 if fp32 else True)
     # adjoint at the GPU's states: loss derivative on the top layer's last state plus small seeds everywhere
@@ -62,7 +62,7 @@ def test_stacked_solve(c):
     if w.levels > 1:
         lam, lam0, g, rref = O.stacked_mgrit_adjoint(layers_ref, xr, h0r, hn, seed64, **kw)
         for a, b in zip(rna, rref):
-            assert abs(a - b) <= (1e-3 * b + 1e-7 if fp32 else 1e-3 * b + 5e-4 * rref[0])
+            assert abs(a - b) <= (1e-3 * b + 1e-7 if fp32 else 1e-3 * b + 1e-3 * rref[0])
     else:
         lam, lam0, g = O.stacked_serial_backward(layers_ref, xr, h0r, hn, seed64)
     assert rel_inf(dh.cpu().numpy(), lam) < tol
