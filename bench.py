@@ -211,6 +211,7 @@ def main():
     ap.add_argument("--no-kernel-timing", action="store_true", help="skip the per-kernel CUDA-event pass")
     ap.add_argument("--no-serial", action="store_true", help="skip the GPU serial-sweep leg (gpu_serial)")
     ap.add_argument("--no-sweep", action="store_true", help="skip the sequence-length sweep (t_sweep)")
+    ap.add_argument("--stacked", action="store_true", help="also time the step with all layers in one state (one MGRIT cycle for the stack)")
     args = ap.parse_args()
 
     from paper_2203_04738_b200.synthetic import WORKLOADS, make_inputs
@@ -421,6 +422,28 @@ def main():
                 windows[f"sweep_T{Ts}_serial"] = win_r
                 t_sweep["points"].append({"T": Ts, "mgrit_ms": ms_m, "serial_ms": ms_r, "speedup": ms_r / ms_m})
                 torch.cuda.empty_cache()
+    stacked = None
+    if rank == 0 and world == 1 and args.stacked and w.layers > 1:
+        from paper_2203_04738_b200.train_step import stacked_training_step
+        cfg_s = B.make_cfg(T, w.B, w.I, w.H, cf=w.cf, levels=w.levels, iters=w.iters_fwd, relax_fine=w.relax_fine,
+                           relax_coarse=w.relax_coarse, operands=w.operands)
+        nf, na = B.stack_workspace_bytes(cfg_s, w.layers)
+        wsf, wsa = torch.empty(nf, dtype=torch.uint8, device=dev), torch.empty(na, dtype=torch.uint8, device=dev)
+        h0s = torch.zeros(w.layers, w.B, w.H, device=dev)
+        sstep = lambda: stacked_training_step(w, layers, W_c, b_c, x, h0s, labels, ws_fwd=wsf, ws_adj=wsa, ws_head=buf.ws_head)
+        for _ in range(2):
+            sstep()
+        torch.cuda.synchronize()
+        s0, s1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        s0.record()
+        for _ in range(3):
+            sstep()
+        s1.record()
+        torch.cuda.synchronize()
+        ms_st = s0.elapsed_time(s1) / 3
+        stacked = {"ms_per_step": ms_st, "value": T * w.B / (ms_st * 1e-3), "unit": UNIT, "steps": 3, "launch": "host launches",
+                   "what": "all layers in one time-step state, one MGRIT cycle for the stack (generic step kernels: not tuned)"}
+        del wsf, wsa
     clocks = None
     if sampler:
         clocks = sampler.stop(*windows["headline"])
@@ -448,7 +471,7 @@ def main():
            "ms_per_step": ms_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
            "dtype": "bf16" if w.operands == 2 else "f32", "data": "synthetic", "config": config, "clocks": clocks,
            "e2e": e2e, "gpu_launches": int(launches), "roofline": roofline, "cpu_baseline": cpu,
-           "gpu_serial": gpu_serial, "t_sweep": t_sweep, "roofline_by_class": roofline_by_class,
+           "gpu_serial": gpu_serial, "t_sweep": t_sweep, "stacked_state": stacked, "roofline_by_class": roofline_by_class,
            "paper_context": "the paper reports up to 6.5x over serial training on 288 Xeon cores (32 MPI ranks x 9 threads) for T=128; "
                             "another machine and workload: context, not a target",
            "host_enqueue_ms_per_step": host_ms, "kernel_breakdown": breakdown, "kernel_by_size": by_size, "loss": float(loss.item()), "device_status": status}

@@ -64,7 +64,13 @@ enum {
   /* Accept any T >= cf^(levels-1): the C-points of a level are its points 0, cf, 2 cf, ...; what follows the last
    * one is a shorter last interval of F-points, so N_{l+1} = floor(N_l / cf).  The forward grids are anchored at
    * t = 0, the adjoint's reversed grids at t = T (the paper always uses T = 128 = a multiple of cf^(levels-1)). */
-  MGRIT_FLAG_RAGGED_T = 4
+  MGRIT_FLAG_RAGGED_T = 4,
+  /* The gi buffer of mgrit_gru_forward / mgrit_gru_adjoint has mgrit_gru_gi_bytes(cfg) bytes: the projection
+   * gi[T,B,3H] followed by room for the bf16 copies of x and of [h_0; h] that the forward call makes anyway in the
+   * bf16 operand mode; the adjoint call, given the same buffer (and the h that forward call returned), reads them
+   * instead of converting x and h again.  Set it in the cfg of BOTH calls.  Ignored (and harmless) where no such
+   * copies exist: fp32 operands, B not dividing 128, levels == 1, the serial entry points. */
+  MGRIT_FLAG_GI_CARRIES_COPIES = 8
 };
 
 /* Problem and cycle description (Algorithm "MGProp", remark "Beyond Two-Level", Section
@@ -107,6 +113,9 @@ typedef struct {
  * mgrit_gru_forward and gru_serial_forward; adj_bytes serves mgrit_gru_adjoint and
  * gru_serial_backward.  Either output may be NULL. */
 int mgrit_gru_workspace_bytes(const mgrit_gru_cfg* cfg, size_t* fwd_bytes, size_t* adj_bytes);
+
+/* Size in bytes of the gi buffer for this cfg: T*B*3H floats, more with MGRIT_FLAG_GI_CARRIES_COPIES (0 for a bad cfg). */
+size_t mgrit_gru_gi_bytes(const mgrit_gru_cfg* cfg);
 
 /* gi[t] = W_ih x_t + b_ih for all t (input half of Eq. "gru"); computed once on the fine grid
  * and reused by every level and by the adjoint.  x[T,B,I] -> gi[T,B,3H]. */

@@ -23,7 +23,7 @@ OK = 0
 CELL_CLASSIC, CELL_IMPLICIT = 0, 1
 RELAX_F, RELAX_FCF, RELAX_FCFCF = 0, 1, 2
 OPERANDS_FP32, OPERANDS_BF16 = 0, 2
-FLAG_SKIP_DUPLICATE_FRELAX, FLAG_F_CYCLE, FLAG_RAGGED_T = 1, 2, 4
+FLAG_SKIP_DUPLICATE_FRELAX, FLAG_F_CYCLE, FLAG_RAGGED_T, FLAG_GI_CARRIES_COPIES = 1, 2, 4, 8
 
 
 class Cfg(ctypes.Structure):
@@ -42,6 +42,8 @@ class _Grads(ctypes.Structure):
 
 _vp, _sz, _i32 = ctypes.c_void_p, ctypes.c_size_t, ctypes.c_int32
 lib.mgrit_gru_workspace_bytes.argtypes = [ctypes.POINTER(Cfg), ctypes.POINTER(_sz), ctypes.POINTER(_sz)]
+lib.mgrit_gru_gi_bytes.argtypes = [ctypes.POINTER(Cfg)]
+lib.mgrit_gru_gi_bytes.restype = _sz
 lib.gru_input_projection.argtypes = [ctypes.POINTER(Cfg), ctypes.POINTER(_Params), _vp, _vp, _vp, _sz, _vp]
 lib.mgrit_gru_forward.argtypes = [ctypes.POINTER(Cfg), ctypes.POINTER(_Params), _vp, _vp, _vp, _vp,
                                   ctypes.POINTER(ctypes.c_float), _vp, _sz, _vp]
@@ -119,6 +121,19 @@ def workspace_bytes(cfg: Cfg):
     return f.value, a.value
 
 
+def alloc_gi(cfg: Cfg, device) -> torch.Tensor:
+    """The gi buffer for cfg as a flat fp32 tensor: gi[T,B,3H] first, then (with FLAG_GI_CARRIES_COPIES) room for the
+    bf16 copies that travel from the forward call to the adjoint call.  `gi_view(cfg, buf)` is the projection itself."""
+    nbytes = lib.mgrit_gru_gi_bytes(ctypes.byref(cfg))
+    if nbytes == 0:
+        raise MgritError(-1)
+    return torch.empty((nbytes + 3) // 4, dtype=torch.float32, device=device)
+
+
+def gi_view(cfg: Cfg, buf: torch.Tensor) -> torch.Tensor:
+    return buf[: cfg.T * cfg.B * 3 * cfg.H].view(cfg.T, cfg.B, 3 * cfg.H)
+
+
 def _ws(nbytes, ws, dev):
     if ws is None or ws.numel() < nbytes:
         ws = torch.empty(nbytes, dtype=torch.uint8, device=dev)
@@ -135,7 +150,9 @@ def gru_input_projection(cfg, p, x, gi=None, ws=None):
 def mgrit_gru_forward(cfg, p, x, h0, want_resnorm=False, gi=None, h=None, ws=None):
     """-> (h[T,B,H], gi[T,B,3H], resnorm list or None)"""
     dev = x.device
-    gi = torch.empty(cfg.T, cfg.B, 3 * cfg.H, device=dev) if gi is None else gi
+    gi = alloc_gi(cfg, dev) if gi is None else gi       # (a flat buffer when the copies flag is set, else viewed as [T,B,3H])
+    if gi.dim() == 1 and not (cfg.flags & FLAG_GI_CARRIES_COPIES):
+        gi = gi_view(cfg, gi)
     h = torch.empty(cfg.T, cfg.B, cfg.H, device=dev) if h is None else h
     ws = _ws(workspace_bytes(cfg)[0], ws, dev)
     rn = (ctypes.c_float * max(cfg.iters, 1))() if want_resnorm else None

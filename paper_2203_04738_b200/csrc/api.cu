@@ -105,6 +105,25 @@ int check_cfg(const mgrit_gru_cfg* c, Hier* hr) {
   return MGRIT_OK;
 }
 
+// With MGRIT_FLAG_GI_CARRIES_COPIES the caller's gi buffer is followed by the bf16 copies that the forward call makes
+// anyway and the adjoint call needs again: x as [T*B, I] and the level-0 state [h_0; h] as [(T+1)*B, H].
+struct GiTail { __nv_bfloat16* xb; __nv_bfloat16* hb0; size_t total_bytes; };
+GiTail gi_tail(const mgrit_gru_cfg* c, float* gi) {
+  const size_t TB = (size_t)c->T * c->B;
+  size_t off = (TB * 3 * c->H * sizeof(float) + 255) & ~(size_t)255;
+  GiTail t;
+  t.xb = gi ? reinterpret_cast<__nv_bfloat16*>(reinterpret_cast<char*>(gi) + off) : nullptr;
+  off += (TB * c->I * sizeof(__nv_bfloat16) + 255) & ~(size_t)255;
+  t.hb0 = gi ? reinterpret_cast<__nv_bfloat16*>(reinterpret_cast<char*>(gi) + off) : nullptr;
+  off += ((TB + c->B) * c->H * sizeof(__nv_bfloat16) + 255) & ~(size_t)255;
+  t.total_bytes = off;
+  return t;
+}
+// the copies exist when the tensor-core engine keeps bf16 shadows of the level states (B divides 128) in an MGRIT solve
+bool carries_copies(const mgrit_gru_cfg* c, bool serial) {
+  return !serial && (c->flags & MGRIT_FLAG_GI_CARRIES_COPIES) && c->operands == MGRIT_OPERANDS_BF16 && 128 % c->B == 0 && c->levels > 1;
+}
+
 struct FwdWs {
   float* U[kMaxLevels]; float* G[kMaxLevels]; double* res_acc; UmmaFwdWs um;
   __nv_bfloat16* chain_ub; unsigned* chain_bar; uint4* chain_xw; size_t chain_xw_bytes;   // scratch of the persistent serial-chain kernel
@@ -357,6 +376,11 @@ int forward_impl(const mgrit_gru_cfg* cfg_in, bool serial, const gru_params* p, 
   plan_fwd(&c, hr, w, &fw);
   if (!w.fits()) return MGRIT_WORKSPACE_TOO_SMALL;
   size_t BH = (size_t)c.B * c.H;
+  if (carries_copies(&c, serial)) {      // make the copies where the adjoint call will look for them
+    GiTail t = gi_tail(&c, gi);
+    fw.um.xb = t.xb;
+    fw.Ub[0] = t.hb0;
+  }
 
   if (c.operands == MGRIT_OPERANDS_BF16) {
     rc = umma_prepare_fwd(&c, p, x, gi, &fw.um, s);
@@ -408,8 +432,15 @@ int adjoint_impl(const mgrit_gru_cfg* cfg_in, bool serial, const gru_params* p, 
   const int T = c.T;
   const bool bf16 = c.operands == MGRIT_OPERANDS_BF16;
 
+  const bool copies = carries_copies(&c, serial);
+  if (copies) {                           // bf16 x and [h_0; h] were left behind the projection by the forward call
+    GiTail t = gi_tail(&c, const_cast<float*>(gi));
+    aw.um.xb = t.xb;
+    aw.um.hb0 = t.hb0;
+    aw.um.hb = t.hb0 + BH;
+  }
   if (bf16) {
-    rc = umma_prepare_adj(&c, p, h0, h, &aw.um, s);
+    rc = umma_prepare_adj(&c, p, h0, h, &aw.um, copies, s);
     if (rc) return rc;
   }
   // adjoint coefficients of every level's steps at the given states (restricted by injection)
@@ -457,7 +488,7 @@ int adjoint_impl(const mgrit_gru_cfg* cfg_in, bool serial, const gru_params* p, 
   if (bf16) {
     // lambda_{t+1} for t = 0..T-1 is read in place from the reversed unknowns (row stride -B*H)
     rc = umma_gradients(&c, p, x, h0, h, aw.U[0] + (size_t)(T - 1) * BH, -(i64)BH, aw.crb[0], aw.czb[0], aw.cnb[0], aw.cnpb, dx, g,
-                        &aw.um, s);
+                        &aw.um, copies, s);
     if (rc) return rc;
   } else {
     i64 M = (i64)T * c.B;
@@ -699,7 +730,7 @@ int stack_layer_gradients(const mgrit_gru_cfg& ck, const gru_params* pk, const f
                           StackAdjWs& w, float* dx, const gru_grads* g, cudaStream_t s) {
   const i64 bh = (i64)ck.B * ck.H, M = (i64)ck.T * ck.B;
   if (ck.operands == MGRIT_OPERANDS_BF16)
-    return umma_gradients(&ck, pk, xk, h0k, L.hk, w.lamk, bh, L.crb[0], L.czb[0], L.cnb[0], L.cnpb[0], dx, g, &L.um, s);
+    return umma_gradients(&ck, pk, xk, h0k, L.hk, w.lamk, bh, L.crb[0], L.czb[0], L.cnb[0], L.cnpb[0], dx, g, &L.um, false, s);
   stream_form_dA(w.lamk, L.cr[0], L.cz[0], L.cn[0], L.cnp[0], w.dA_h, w.dA_i, M, ck.H, s);
   simt_wgrad(w.dA_h, (int)M, 3 * ck.H, h0k, ck.B, L.hk, ck.H, g->dW_hh, s);
   simt_wgrad(w.dA_i, (int)M, 3 * ck.H, nullptr, 0, xk, ck.I, g->dW_ih, s);
@@ -737,7 +768,7 @@ int stack_adjoint_impl(const mgrit_gru_cfg* cfg, int nl, const gru_params* p, co
     StackLayerAdj& L = aw.L[k];
     mgrit_gru_cfg ck = layer_cfg(c, k);
     if (bf16) {
-      rc = umma_prepare_adj(&ck, &p[k], h0 + (size_t)k * bh, L.hk, &L.um, s);
+      rc = umma_prepare_adj(&ck, &p[k], h0 + (size_t)k * bh, L.hk, &L.um, false, s);
       if (rc) return rc;
     }
     if (k > 0) {
@@ -1000,6 +1031,13 @@ int mgrit_gru_workspace_bytes(const mgrit_gru_cfg* cfg, size_t* fwd_bytes, size_
     *adj_bytes = (w.off > w1.off ? w.off : w1.off) + 256;
   }
   return MGRIT_OK;
+}
+
+size_t mgrit_gru_gi_bytes(const mgrit_gru_cfg* cfg) {
+  Hier hr;
+  if (check_cfg(cfg, &hr) != MGRIT_OK) return 0;
+  const size_t plain = (size_t)cfg->T * cfg->B * 3 * cfg->H * sizeof(float);
+  return (cfg->flags & MGRIT_FLAG_GI_CARRIES_COPIES) ? gi_tail(cfg, nullptr).total_bytes : plain;
 }
 
 int gru_input_projection(const mgrit_gru_cfg* cfg, const gru_params* p, const float* x, float* gi, void* ws, size_t ws_bytes,

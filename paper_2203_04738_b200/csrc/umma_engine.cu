@@ -662,11 +662,14 @@ int umma_prepare_fwd(const mgrit_gru_cfg* c, const gru_params* p, const float* x
   return MGRIT_OK;
 }
 
-int umma_prepare_adj(const mgrit_gru_cfg* c, const gru_params* p, const float* h0, const float* h, UmmaAdjWs* w, cudaStream_t s) {
+int umma_prepare_adj(const mgrit_gru_cfg* c, const gru_params* p, const float* h0, const float* h, UmmaAdjWs* w, bool have_hb,
+                     cudaStream_t s) {
   const int H = c->H, I = c->I;
   convert(p->W_hh, w->W_hh, (i64)3 * H * H, s);
-  convert(h0, w->hb0, (i64)c->B * H, s);
-  convert(h, w->hb, (i64)c->T * c->B * H, s);
+  if (!have_hb) {      // otherwise w->hb0 already points at the forward call's bf16 copy of [h_0; h]
+    convert(h0, w->hb0, (i64)c->B * H, s);
+    convert(h, w->hb, (i64)c->T * c->B * H, s);
+  }
   transpose(p->W_hh, 3 * H, H, w->W_hhT, 3 * H, 0, s);   // [H, 3H]
   transpose(p->W_ih, 3 * H, I, w->W_ihT, 3 * H, 0, s);   // [I, 3H]
   return status_ptr() ? MGRIT_OK : MGRIT_CUDA_ERROR;
@@ -797,7 +800,7 @@ static bool wgrad_gemm(const bf16* dA, int H3, const bf16* R, int cols, int K, O
 
 int umma_gradients(const mgrit_gru_cfg* c, const gru_params* p, const float* x, const float* h0, const float* h, const float* lam,
                    i64 lam_ts, const bf16* cr, const bf16* cz, const bf16* cn, const bf16* cnp, float* dx, const gru_grads* g,
-                   UmmaAdjWs* w, cudaStream_t s) {
+                   UmmaAdjWs* w, bool have_xb, cudaStream_t s) {
   (void)h0; (void)h;
   const int H = c->H, I = c->I, B = c->B;
   const i64 M = (i64)c->T * B;
@@ -816,7 +819,7 @@ int umma_gradients(const mgrit_gru_cfg* c, const gru_params* p, const float* x, 
                                            reinterpret_cast<uint2*>(dAi), scratch, rows_per_block);
   sum_db_kernel<<<pgrid(4 * H), kPT, 0, s>>>(scratch, (int)grid.x, H, g->db_hh, g->db_ih);
   count_launch(2);
-  convert(x, w->xb, M * I, s);                   // x as bf16 [M, I]; h_{t-1} as bf16 = [h_0; h] without its last slot (w->hb0)
+  if (!have_xb) convert(x, w->xb, M * I, s);     // x as bf16 [M, I]; h_{t-1} as bf16 = [h_0; h] without its last slot (w->hb0)
   bool ok = true;
   // dW_hh[3H, H] = dA_h^T h_prev ;  dW_ih[3H, I] = dA_i^T x    (K = T*B, MN-major operands)
   ok = ok && wgrad_gemm(dAh, 3 * H, w->hb0, H, (int)M, g->dW_hh, scratch, scratch_bytes, s);

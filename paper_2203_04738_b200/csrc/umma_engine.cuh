@@ -30,7 +30,8 @@ int umma_supported(const mgrit_gru_cfg* c);
 void umma_plan_fwd(const mgrit_gru_cfg* c, const int* N, int L, char* base, size_t* off, UmmaFwdWs* o);
 void umma_plan_adj(const mgrit_gru_cfg* c, const int* N, int L, char* base, size_t* off, UmmaAdjWs* o);
 int umma_prepare_fwd(const mgrit_gru_cfg* c, const gru_params* p, const float* x, float* gi, UmmaFwdWs* w, cudaStream_t s);
-int umma_prepare_adj(const mgrit_gru_cfg* c, const gru_params* p, const float* h0, const float* h, UmmaAdjWs* w, cudaStream_t s);
+int umma_prepare_adj(const mgrit_gru_cfg* c, const gru_params* p, const float* h0, const float* h, UmmaAdjWs* w, bool have_hb,
+                     cudaStream_t s);
 void umma_convert(const float* src, __nv_bfloat16* dst, i64 n, cudaStream_t s);
 int umma_project_rows(const float* X, __nv_bfloat16* xb, const __nv_bfloat16* Wb, const float* bias, float* out, int M, int K, int H3,
                       cudaStream_t s);
@@ -41,7 +42,7 @@ int umma_adj_step(const AdjStepArgs& a, UmmaAdjWs* w, cudaStream_t s);
 int umma_gradients(const mgrit_gru_cfg* c, const gru_params* p, const float* x, const float* h0, const float* h,
                    const float* lam, i64 lam_ts, const __nv_bfloat16* cr, const __nv_bfloat16* cz, const __nv_bfloat16* cn,
                    const __nv_bfloat16* cnp, float* dx,
-                   const gru_grads* g, UmmaAdjWs* w, cudaStream_t s);
+                   const gru_grads* g, UmmaAdjWs* w, bool have_xb, cudaStream_t s);
 // the three step functions return MGRIT_OK or MGRIT_CUDA_ERROR (a tensor map could not be encoded, a launch failed)
 int umma_device_status();
 int umma_clear_device_status();

@@ -30,7 +30,7 @@ def make_cfgs(w: Workload, T: int, Bsz: int, serial: bool = False, flags: int = 
     for l in range(w.layers):
         I = w.I if l == 0 else w.H
         kw = dict(cf=w.cf, levels=1 if serial else w.levels, cell=w.cell, relax_fine=w.relax_fine,
-                  relax_coarse=w.relax_coarse, operands=w.operands, flags=flags)
+                  relax_coarse=w.relax_coarse, operands=w.operands, flags=flags | B.FLAG_GI_CARRIES_COPIES)
         fw.append(B.make_cfg(T, Bsz, I, w.H, iters=w.iters_fwd, **kw))
         ad.append(B.make_cfg(T, Bsz, I, w.H, iters=w.iters_adj, **kw))
     return fw, ad
@@ -48,7 +48,7 @@ def alloc_buffers(w: Workload, T: int, Bsz: int, device, serial: bool = False, f
                                    dW_ih=mk(3 * w.H, c.I), dW_hh=mk(3 * w.H, w.H), db_ih=mk(3 * w.H), db_hh=mk(3 * w.H)))
     return StepBuffers(fw, ad, torch.empty(nf, dtype=torch.uint8, device=device), torch.empty(na, dtype=torch.uint8, device=device),
                        torch.empty(B.lib.xent_head_workspace_bytes(Bsz, w.classes), dtype=torch.uint8, device=device),
-                       [mk(T, Bsz, 3 * w.H) for _ in fw], [mk(T, Bsz, w.H) for _ in fw], adj, serial)
+                       [B.alloc_gi(c, device) for c in fw], [mk(T, Bsz, w.H) for _ in fw], adj, serial)
 
 
 class HostInputPipeline:
@@ -171,3 +171,24 @@ class GraphedTrainingStep:
         self.graph.replay()
         return self.loss
 
+
+
+def stacked_training_step(w: Workload, layers, W_c, b_c, x, h0s, labels, ws_fwd=None, ws_adj=None, ws_head=None, lr: float = 1e-3,
+                          update: bool = True, flags: int = 0):
+    """The same training step with ALL layers in one time-step state and ONE MGRIT cycle for the stack
+    (mgrit_gru_stack_forward / mgrit_gru_stack_adjoint): forward -> loss head on the top layer's last state -> adjoint ->
+    per-layer gradients -> SGD.  h0s[n_layers,B,H].  Returns (loss, forward residual norms or None)."""
+    T, Bsz = x.shape[0], x.shape[1]
+    kw = dict(cf=w.cf, levels=w.levels, cell=w.cell, relax_fine=w.relax_fine, relax_coarse=w.relax_coarse, operands=w.operands, flags=flags)
+    cf_ = B.make_cfg(T, Bsz, w.I, w.H, iters=w.iters_fwd, **kw)
+    ca_ = B.make_cfg(T, Bsz, w.I, w.H, iters=w.iters_adj, **kw)
+    h, gi0, _ = B.mgrit_gru_stack_forward(cf_, layers, x, h0s, ws=ws_fwd)
+    loss, dhT, dWc, dbc = B.xent_head_fwd_bwd(h[-1, -1], W_c, b_c, labels, ws=ws_head)
+    _, _, _, grads, _ = B.mgrit_gru_stack_adjoint(ca_, layers, x, h0s, gi0, h, dhT=dhT, want_dx=False, want_dh=False, ws=ws_adj)
+    if update:
+        for p, g in zip(layers, grads):
+            for name, gg in (("W_ih", g.dW_ih), ("W_hh", g.dW_hh), ("b_ih", g.db_ih), ("b_hh", g.db_hh)):
+                B.sgd_update(p[name], gg, lr)
+        B.sgd_update(W_c, dWc, lr)
+        B.sgd_update(b_c, dbc, lr)
+    return loss

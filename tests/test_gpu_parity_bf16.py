@@ -235,3 +235,25 @@ def test_run_to_run_bit_identical_and_workspace_content_irrelevant(B):
         for a, b in zip(o, outs[0]):
             assert torch.equal(a, b)      # every reduction (split GEMMs, bias sums, loss) runs in a fixed order
     assert B.last_device_status() == 0
+
+
+def test_copies_carried_behind_gi_give_the_same_bits(B):
+    # FLAG_GI_CARRIES_COPIES only moves where the bf16 copies of x and [h_0; h] live: every output must keep its bits,
+    # also with the larger buffer poisoned beforehand; a case without shadows (B does not divide 128) ignores the flag.
+    for Bsz in (32, 24):
+        w = Workload("carry", T=256, B=Bsz, I=64, H=256, cf=4, levels=3, iters_fwd=2, iters_adj=2, relax_fine=0, relax_coarse=1,
+                     operands=2, classes=8, relu=True, seed=11)
+        d = make_inputs(w)
+        p, x, h0 = upload(d)
+        plain, carry = _cfg(B, w, 2), _cfg(B, w, 2, flags=B.FLAG_GI_CARRIES_COPIES)
+        h, gi, _ = B.mgrit_gru_forward(plain, p, x, h0)
+        r = B.mgrit_gru_adjoint(plain, p, x, h0, gi, h, dhT=h[-1].contiguous())
+        buf = B.alloc_gi(carry, x.device)
+        assert buf.numel() * 4 == B.lib.mgrit_gru_gi_bytes(carry) > gi.numel() * 4 + 2 * (x.numel() + h.numel())
+        buf.fill_(float("nan"))
+        h2, gi2, _ = B.mgrit_gru_forward(carry, p, x, h0, gi=buf)
+        assert gi2 is buf and torch.equal(B.gi_view(carry, buf), gi) and torch.equal(h2, h)
+        r2 = B.mgrit_gru_adjoint(carry, p, x, h0, buf, h2, dhT=h2[-1].contiguous())
+        for k in ("dh", "dh0", "dx", "dW_ih", "dW_hh", "db_ih", "db_hh"):
+            assert torch.equal(getattr(r, k), getattr(r2, k)), k
+    assert B.last_device_status() == 0

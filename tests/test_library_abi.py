@@ -82,3 +82,15 @@ def test_cycle_variant_flags_are_validated_on_the_host(lib):
     assert fn(ctypes.byref(make_cfg(64, 2, 16, 32, cf=4, levels=3, relax_fine=2, relax_coarse=3, flags=FLAG_F_CYCLE)),
               ctypes.byref(f), ctypes.byref(a)) == 0
     assert fn(ctypes.byref(make_cfg(64, 2, 16, 32, cf=4, levels=3, relax_fine=9)), ctypes.byref(f), ctypes.byref(a)) == -1
+
+
+def test_gi_buffer_size_with_and_without_carried_copies(lib):
+    from paper_2203_04738_b200.binding import Cfg, FLAG_GI_CARRIES_COPIES, make_cfg
+    fn = lib.mgrit_gru_gi_bytes
+    fn.argtypes, fn.restype = [ctypes.POINTER(Cfg)], ctypes.c_size_t
+    T, Bz, I, H = 128, 4, 16, 64
+    assert fn(ctypes.byref(make_cfg(T, Bz, I, H, cf=4, levels=3))) == T * Bz * 3 * H * 4
+    n = fn(ctypes.byref(make_cfg(T, Bz, I, H, cf=4, levels=3, flags=FLAG_GI_CARRIES_COPIES)))
+    need = T * Bz * 3 * H * 4 + T * Bz * I * 2 + (T + 1) * Bz * H * 2
+    assert need <= n <= need + 3 * 256 and n % 256 == 0
+    assert fn(ctypes.byref(make_cfg(100, Bz, I, H, cf=8, levels=3))) == 0       # a bad cfg has no size
