@@ -156,10 +156,15 @@ class ClockSampler:
 
 
 # ------------------------------------------------------------------------------------------ GPU helpers
+OPERAND_NAMES = {0: "fp32 (FFMA)", 1: "tf32 tensor cores, three-term split", 2: "bf16 tensor cores", 3: "tf32 tensor cores, single pass"}
+OPERAND_DTYPES = {0: "f32", 1: "tf32x3", 2: "bf16", 3: "tf32"}
+
+
 def describe(w, T, Bsz):
     return (f"{w.name}: {w.layers}-layer GRU I={w.I} H={w.H} B={Bsz} T={T}, cf={w.cf}, levels={w.levels}, "
             f"iters fwd/adj={w.iters_fwd}/{w.iters_adj}, relax fine/coarse={'FCF' if w.relax_fine else 'F'}/"
-            f"{'FCF' if w.relax_coarse else 'F'}, implicit cell, {w.classes}-class xent on h_T, SGD")
+            f"{'FCF' if w.relax_coarse else 'F'}, implicit cell, {w.classes}-class xent on h_T, SGD, "
+            f"operands {OPERAND_NAMES[w.operands]}")
 
 
 def time_gpu_step(w, T, serial, steps, warmup, dev, use_graph=True):
@@ -211,11 +216,16 @@ def main():
     ap.add_argument("--no-kernel-timing", action="store_true", help="skip the per-kernel CUDA-event pass")
     ap.add_argument("--no-serial", action="store_true", help="skip the GPU serial-sweep leg (gpu_serial)")
     ap.add_argument("--no-sweep", action="store_true", help="skip the sequence-length sweep (t_sweep)")
+    ap.add_argument("--operands", default=None, choices=["fp32", "tf32", "bf16", "tf32_1pass"],
+                    help="override the workload's operand mode (tf32: three-term split on the tensor cores, fp32-level accuracy)")
     ap.add_argument("--stacked", action="store_true", help="also time the step with all layers in one state (one MGRIT cycle for the stack)")
     args = ap.parse_args()
 
     from paper_2203_04738_b200.synthetic import WORKLOADS, make_inputs
     w = WORKLOADS[args.workload]
+    if args.operands:
+        import dataclasses
+        w = dataclasses.replace(w, operands={"fp32": 0, "tf32": 1, "bf16": 2, "tf32_1pass": 3}[args.operands])
     rank = int(os.environ.get("RANK", "0"))
     world = int(os.environ.get("WORLD_SIZE", "1"))
     local_rank = int(os.environ.get("LOCAL_RANK", "0"))
@@ -373,6 +383,13 @@ def main():
             burst = float(peaks["bf16_tflops"])
             bound, note = "tensor", (f"bf16 dense cuBLAS figures ({pk}): `peak`/`frac` use the sustained one (the kernel is timed inside "
                                      "whole steps), `frac_burst` the burst one, `frac_nominal` the vendor's 2250 TFLOP/s")
+        elif w.operands in (1, 3):
+            # tf32 products: the measured bf16 figures scaled by the nominal tf32 : bf16 ratio (1.1 : 2.25 PFLOP/s dense);
+            # the recorded flops are those the tensor cores execute (three products per element in the split mode)
+            ratio = 1.1 / 2.25
+            peak = float(peaks.get("bf16_tflops_sustained", peaks["bf16_tflops"])) * ratio
+            burst = float(peaks["bf16_tflops"]) * ratio
+            bound, note = "tensor", f"tf32: bf16 dense cuBLAS figures ({pk}) x the nominal tf32:bf16 ratio 1.1/2.25"
         else:
             # fp32 FFMA: 148 SMs x 128 lanes x 2 flop x max SM clock
             peak = burst = 148 * 128 * 2 * float(peaks.get("sm_max_mhz", 1965.0)) * 1e6 / 1e12
@@ -469,7 +486,7 @@ def main():
     status = B.last_device_status()
     out = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": max(args.warmup, 3),
            "ms_per_step": ms_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
-           "dtype": "bf16" if w.operands == 2 else "f32", "data": "synthetic", "config": config, "clocks": clocks,
+           "dtype": OPERAND_DTYPES[w.operands], "data": "synthetic", "config": config, "clocks": clocks,
            "e2e": e2e, "gpu_launches": int(launches), "roofline": roofline, "cpu_baseline": cpu,
            "gpu_serial": gpu_serial, "t_sweep": t_sweep, "stacked_state": stacked, "roofline_by_class": roofline_by_class,
            "paper_context": "the paper reports up to 6.5x over serial training on 288 Xeon cores (32 MPI ranks x 9 threads) for T=128; "

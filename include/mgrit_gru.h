@@ -53,7 +53,7 @@ enum {
 enum { MGRIT_CELL_CLASSIC = 0, MGRIT_CELL_IMPLICIT = 1 };
 /* relaxation = n means F (CF)^n: F-relaxation followed by n C- and F-sweeps (Eq. "fcf-relax" is n = 1) */
 enum { MGRIT_RELAX_F = 0, MGRIT_RELAX_FCF = 1, MGRIT_RELAX_FCFCF = 2, MGRIT_RELAX_MAX = 8 };
-enum { MGRIT_OPERANDS_FP32 = 0, MGRIT_OPERANDS_BF16 = 2 };
+enum { MGRIT_OPERANDS_FP32 = 0, MGRIT_OPERANDS_TF32 = 1, MGRIT_OPERANDS_BF16 = 2, MGRIT_OPERANDS_TF32_1PASS = 3 };
 enum {
   MGRIT_FLAG_SKIP_DUPLICATE_FRELAX = 1,
   /* F-cycles instead of V-cycles: when the correction of a level has been spread by its final F-relaxation, one
@@ -86,7 +86,12 @@ typedef struct {
   int32_t operands;     /* MGRIT_OPERANDS_FP32: FFMA everywhere; MGRIT_OPERANDS_BF16: bf16 tensor-core
                            operands with fp32 accumulation; states, gates and gradients stay fp32 (the
                            adjoint's gate coefficients, which only ever enter such operands, are kept
-                           in bf16 inside the workspace) */
+                           in bf16 inside the workspace); MGRIT_OPERANDS_TF32: every product on the tensor
+                           cores as a three-term split of tf32 operands (x_hi w_hi + x_lo w_hi + x_hi w_lo),
+                           fp32 accumulation and fp32 everything else: meets the fp32 tolerances;
+                           MGRIT_OPERANDS_TF32_1PASS: operands rounded to tf32 once (10 mantissa bits).
+                           The tf32 modes need H % 64 == 0, I % 16 == 0, (T*B) % 4 == 0 and serve the
+                           mgrit_gru_* / gru_serial_* / gru_input_projection calls of one layer. */
   int32_t flags;        /* OR of MGRIT_FLAG_*.  MGRIT_FLAG_SKIP_DUPLICATE_FRELAX: a cycle after the first starts
                            from C-points whose F-points the previous cycle's final F-relaxation already filled;
                            skip re-doing it (results are identical) */

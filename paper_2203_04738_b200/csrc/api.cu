@@ -71,6 +71,8 @@ bool aligned32(P... ptrs) {
   return (m & 31u) == 0;
 }
 
+inline bool is_tf32(const mgrit_gru_cfg* c) { return c->operands == MGRIT_OPERANDS_TF32 || c->operands == MGRIT_OPERANDS_TF32_1PASS; }
+
 int check_cfg(const mgrit_gru_cfg* c, Hier* hr) {
   if (!c) return MGRIT_INVALID_ARG;
   if (c->T <= 0 || c->B <= 0 || c->I <= 0 || c->H <= 0 || c->levels < 1 || c->levels > kMaxLevels) return MGRIT_INVALID_ARG;
@@ -78,7 +80,7 @@ int check_cfg(const mgrit_gru_cfg* c, Hier* hr) {
   if (c->cell != MGRIT_CELL_CLASSIC && c->cell != MGRIT_CELL_IMPLICIT) return MGRIT_INVALID_ARG;
   if (c->relax_fine < MGRIT_RELAX_F || c->relax_fine > MGRIT_RELAX_MAX) return MGRIT_INVALID_ARG;
   if (c->relax_coarse < MGRIT_RELAX_F || c->relax_coarse > MGRIT_RELAX_MAX) return MGRIT_INVALID_ARG;
-  if (c->operands != MGRIT_OPERANDS_FP32 && c->operands != MGRIT_OPERANDS_BF16) return MGRIT_INVALID_ARG;
+  if (c->operands < MGRIT_OPERANDS_FP32 || c->operands > MGRIT_OPERANDS_TF32_1PASS) return MGRIT_INVALID_ARG;
   if (!(c->dt > 0.f)) return MGRIT_INVALID_ARG;
   if (c->H % 8 != 0 || c->I % 8 != 0) return MGRIT_UNSUPPORTED;
   // row counts (T+1)*B, widths and grid sizes are 32-bit inside the kernels; element offsets are 64-bit
@@ -100,6 +102,10 @@ int check_cfg(const mgrit_gru_cfg* c, Hier* hr) {
   }
   if (c->operands == MGRIT_OPERANDS_BF16) {
     int rc = umma_supported(c);
+    if (rc != MGRIT_OK) return rc;
+  }
+  if (is_tf32(c)) {
+    int rc = tf32_supported(c);
     if (rc != MGRIT_OK) return rc;
   }
   return MGRIT_OK;
@@ -125,7 +131,7 @@ bool carries_copies(const mgrit_gru_cfg* c, bool serial) {
 }
 
 struct FwdWs {
-  float* U[kMaxLevels]; float* G[kMaxLevels]; double* res_acc; UmmaFwdWs um;
+  float* U[kMaxLevels]; float* G[kMaxLevels]; double* res_acc; UmmaFwdWs um; Tf32Ws tf;
   __nv_bfloat16* chain_ub; unsigned* chain_bar; uint4* chain_xw; size_t chain_xw_bytes;   // scratch of the persistent serial-chain kernel
   __nv_bfloat16* Ub[kMaxLevels];                  // bf16 copies of the level states (tensor-core A operands)
 };
@@ -133,7 +139,7 @@ struct AdjWs {
   float* U[kMaxLevels]; float* G[kMaxLevels];
   float *a[kMaxLevels], *cr[kMaxLevels], *cz[kMaxLevels], *cn[kMaxLevels], *cnp;   // gate coefficients: fp32 engine
   __nv_bfloat16 *crb[kMaxLevels], *czb[kMaxLevels], *cnb[kMaxLevels], *cnpb;       // ... tensor-core engine (bf16)
-  float *dA_h, *dA_i, *lam_tmp; double* res_acc; UmmaAdjWs um;
+  float *dA_h, *dA_i, *lam_tmp; double* res_acc; UmmaAdjWs um; Tf32Ws tf;
   __nv_bfloat16* chain_dAb; unsigned* chain_bar; uint4* chain_xw; size_t chain_xw_bytes;
 };
 
@@ -154,6 +160,7 @@ void plan_fwd(const mgrit_gru_cfg* c, const Hier& hr, Ws& w, FwdWs* o) {
     o->chain_xw_bytes = serial_xw_bytes(c->B, c->H, 1);
     o->chain_xw = reinterpret_cast<uint4*>(w.take<char>(o->chain_xw_bytes));
   }
+  if (is_tf32(c)) tf32_plan_fwd(c, hr.N, hr.L, w.base, &w.off, &o->tf);
 }
 
 void plan_adj(const mgrit_gru_cfg* c, const Hier& hr, Ws& w, AdjWs* o) {
@@ -190,6 +197,7 @@ void plan_adj(const mgrit_gru_cfg* c, const Hier& hr, Ws& w, AdjWs* o) {
     o->dA_i = w.take<float>((size_t)c->T * BH * 3);
     o->lam_tmp = w.take<float>((size_t)c->T * BH);     // lambda in forward order when the caller wants no dh
   }
+  if (is_tf32(c)) tf32_plan_adj(c, hr.N, hr.L, w.base, &w.off, &o->tf);
 }
 
 // One launch of "advance nk*B rows by one step of level l".
@@ -300,6 +308,7 @@ struct FwdCycle : Cycle {
     a.gadd = d.gadd ? d.gadd + (size_t)d.gadd_slot * BH : nullptr; a.gadd_ks = (i64)d.gadd_stride * BH;
     a.W_hh = p->W_hh; a.b_hh = p->b_hh; a.gamma = hr.gamma[d.l]; a.cell = c->cell; a.mode = d.mode;
     if (c->operands == MGRIT_OPERANDS_BF16) return umma_fwd_step(a, um, s);
+    if (is_tf32(c)) return tf32_fwd_step(a, &fw->tf, s);
     simt_fwd_step(a, s);
     return MGRIT_OK;
   }
@@ -338,6 +347,7 @@ struct AdjCycle : Cycle {
     a.coef_ks = -(i64)d.tgt_stride * BH;
     a.W_hh = p->W_hh; a.mode = d.mode;
     if (c->operands == MGRIT_OPERANDS_BF16) return umma_adj_step(a, &w->um, s);
+    if (is_tf32(c)) return tf32_adj_step(a, &w->tf, s);
     simt_adj_step(a, s);
     return MGRIT_OK;
   }
@@ -384,6 +394,9 @@ int forward_impl(const mgrit_gru_cfg* cfg_in, bool serial, const gru_params* p, 
 
   if (c.operands == MGRIT_OPERANDS_BF16) {
     rc = umma_prepare_fwd(&c, p, x, gi, &fw.um, s);
+    if (rc) return rc;
+  } else if (is_tf32(&c)) {
+    rc = tf32_prepare_fwd(&c, p, x, gi, &fw.tf, s);
     if (rc) return rc;
   } else {
     simt_project(x, p->W_ih, p->b_ih, gi, c.T * c.B, c.I, 3 * c.H, s);
@@ -443,6 +456,11 @@ int adjoint_impl(const mgrit_gru_cfg* cfg_in, bool serial, const gru_params* p, 
     rc = umma_prepare_adj(&c, p, h0, h, &aw.um, copies, s);
     if (rc) return rc;
   }
+  const bool tf32 = is_tf32(&c);
+  if (tf32) {
+    rc = tf32_prepare_adj(&c, p, &aw.tf, s);
+    if (rc) return rc;
+  }
   // adjoint coefficients of every level's steps at the given states (restricted by injection)
   for (int l = 0; l < hr.L; ++l) {
     LinArgs a;
@@ -453,6 +471,9 @@ int adjoint_impl(const mgrit_gru_cfg* cfg_in, bool serial, const gru_params* p, 
     a.crb = aw.crb[l]; a.czb = aw.czb[l]; a.cnb = aw.cnb[l]; a.cnpb = l == 0 ? aw.cnpb : nullptr;
     if (bf16) {
       rc = umma_linearise(a, &aw.um, s);
+      if (rc) return rc;
+    } else if (tf32) {
+      rc = tf32_linearise(a, &aw.tf, s);
       if (rc) return rc;
     } else {
       simt_linearise(a, s);
@@ -498,11 +519,20 @@ int adjoint_impl(const mgrit_gru_cfg* cfg_in, bool serial, const gru_params* p, 
       stream_gather_rows(aw.lam_tmp, (i64)BH, aw.U[0] + (size_t)(T - 1) * BH, -(i64)BH, T, (i64)BH, s);
     }
     stream_form_dA(lam, aw.cr[0], aw.cz[0], aw.cn[0], aw.cnp, aw.dA_h, aw.dA_i, M, c.H, s);
-    simt_wgrad(aw.dA_h, (int)M, 3 * c.H, h0, c.B, h, c.H, g->dW_hh, s);
-    simt_wgrad(aw.dA_i, (int)M, 3 * c.H, nullptr, 0, x, c.I, g->dW_ih, s);
+    if (tf32) {
+      rc = tf32_wgrad(aw.dA_h, (int)M, 3 * c.H, h0, c.B, h, c.H, g->dW_hh, &aw.tf, s);
+      if (!rc) rc = tf32_wgrad(aw.dA_i, (int)M, 3 * c.H, nullptr, 0, x, c.I, g->dW_ih, &aw.tf, s);
+      if (rc) return rc;
+    } else {
+      simt_wgrad(aw.dA_h, (int)M, 3 * c.H, h0, c.B, h, c.H, g->dW_hh, s);
+      simt_wgrad(aw.dA_i, (int)M, 3 * c.H, nullptr, 0, x, c.I, g->dW_ih, s);
+    }
     stream_colsum(aw.dA_h, M, 3 * c.H, g->db_hh, s);
     stream_colsum(aw.dA_i, M, 3 * c.H, g->db_ih, s);
-    if (dx) simt_dgrad(aw.dA_i, (int)M, 3 * c.H, p->W_ih, c.I, dx, s);
+    if (dx) {
+      if (tf32) { rc = tf32_dgrad(aw.dA_i, (int)M, 3 * c.H, c.I, dx, &aw.tf, s); if (rc) return rc; }
+      else simt_dgrad(aw.dA_i, (int)M, 3 * c.H, p->W_ih, c.I, dx, s);
+    }
   }
   if (resnorm && hr.L > 1 && c.iters > 0) {
     rc = fetch_resnorm(aw.res_acc, resnorm, c.iters, s);
@@ -609,6 +639,7 @@ int stack_forward_impl(const mgrit_gru_cfg* cfg, int nl, const gru_params* p, co
   Hier hr;
   int rc = check_cfg(&c, &hr);
   if (rc) return rc;
+  if (is_tf32(&c)) return MGRIT_UNSUPPORTED;      // the stacked solve runs on the fp32 or the bf16 engine
   if (nl > 1) { mgrit_gru_cfg c1 = layer_cfg(c, 1); Hier h1; rc = check_cfg(&c1, &h1); if (rc) return rc; }
   Ws w{(char*)ws, ws_bytes, 0};
   StackFwdWs fw;
@@ -753,6 +784,7 @@ int stack_adjoint_impl(const mgrit_gru_cfg* cfg, int nl, const gru_params* p, co
   Hier hr;
   int rc = check_cfg(&c, &hr);
   if (rc) return rc;
+  if (is_tf32(&c)) return MGRIT_UNSUPPORTED;      // the stacked solve runs on the fp32 or the bf16 engine
   if (nl > 1) { mgrit_gru_cfg c1 = layer_cfg(c, 1); Hier h1; rc = check_cfg(&c1, &h1); if (rc) return rc; }
   Ws w{(char*)ws, ws_bytes, 0};
   StackAdjWs aw;
@@ -1056,6 +1088,14 @@ int gru_input_projection(const mgrit_gru_cfg* cfg, const gru_params* p, const fl
     if (!w.fits()) return MGRIT_WORKSPACE_TOO_SMALL;
     rc = umma_prepare_fwd(cfg, p, x, gi, &fw.um, s);
     if (rc) return rc;
+  } else if (is_tf32(cfg)) {
+    if (!ws) return MGRIT_INVALID_ARG;
+    Ws w{(char*)ws, ws_bytes, 0};
+    FwdWs fw;
+    plan_fwd(cfg, hr, w, &fw);
+    if (!w.fits()) return MGRIT_WORKSPACE_TOO_SMALL;
+    rc = tf32_prepare_fwd(cfg, p, x, gi, &fw.tf, s);
+    if (rc) return rc;
   } else {
     simt_project(x, p->W_ih, p->b_ih, gi, cfg->T * cfg->B, cfg->I, 3 * cfg->H, s);
   }
@@ -1089,6 +1129,7 @@ int mgrit_gru_stack_workspace_bytes(const mgrit_gru_cfg* cfg, int32_t n_layers, 
   int rc = check_cfg(cfg, &hr);
   if (rc) return rc;
   if (n_layers < 1 || n_layers > kMaxStack) return MGRIT_INVALID_ARG;
+  if (is_tf32(cfg)) return MGRIT_UNSUPPORTED;
   if (n_layers > 1) { mgrit_gru_cfg c1 = layer_cfg(*cfg, 1); Hier h1; rc = check_cfg(&c1, &h1); if (rc) return rc; }
   if (fwd_bytes) { Ws w{nullptr, 0, 0}; StackFwdWs f; plan_stack_fwd(cfg, n_layers, hr, w, &f); *fwd_bytes = w.off + 256; }
   if (adj_bytes) { Ws w{nullptr, 0, 0}; StackAdjWs a; plan_stack_adj(cfg, n_layers, hr, w, &a); *adj_bytes = w.off + 256; }

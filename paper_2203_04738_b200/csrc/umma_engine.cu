@@ -63,22 +63,39 @@ bool make_map(CUtensorMap* m, const bf16* base, uint64_t inner, uint64_t rows, u
   return r == CUDA_SUCCESS;
 }
 
-template <int BN, bool GATES, class Epi>
-bool launch_gemm(int kc, const bf16* A, i64 lda, const bf16* Bm, i64 ldb, int M, int N, int K, int gate_rows, int b_rows, Epi epi,
-                 cudaStream_t s) {
+// fp32 words holding tf32 values: box = 32 x box_rows (again 128-byte rows)
+bool make_map(CUtensorMap* m, const float* base, uint64_t inner, uint64_t rows, uint64_t pitch, uint32_t box_rows) {
+  cuuint64_t dims[2] = {inner, rows};
+  cuuint64_t strides[1] = {pitch * sizeof(float)};
+  cuuint32_t box[2] = {(cuuint32_t)(BK / 2), box_rows};
+  cuuint32_t estr[2] = {1, 1};
+  CUresult r = g_encode(m, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 2, (void*)base, dims, strides, box, estr,
+                        CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                        CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  if (r != CUDA_SUCCESS) fprintf(stderr, "mgrit_gru: cuTensorMapEncodeTiled (fp32) failed (%d)\n", (int)r);
+  return r == CUDA_SUCCESS;
+}
+
+// ET = bf16, or float for operands that hold tf32 values.  splits > 1 (split-aware epilogues only) cuts the reduction.
+template <int BN, bool GATES, class Epi, class ET>
+bool launch_gemm(int kc, const ET* A, i64 lda, const ET* Bm, i64 ldb, int M, int N, int K, int gate_rows, int b_rows, Epi epi,
+                 cudaStream_t s, int splits = 1) {
   using C = Cfg<BN, GATES>;
+  constexpr bool TF32 = sizeof(ET) == 4;
   if (M <= 0 || N <= 0) return true;
   int* const status = status_ptr();
   if (!status) return false;
   static bool attr_set[kMaxDevices] = {false};
-  auto kern = umma_gemm_kernel<BN, GATES, Epi>;
+  auto kern = umma_gemm_kernel<BN, GATES, Epi, false, TF32>;
   if (!set_smem_once(kern, C::kSmemBytes, attr_set)) return false;
   CUtensorMap ta, tb;
   if (!make_map(&ta, A, (uint64_t)K, (uint64_t)M, (uint64_t)lda, BM)) return false;
   if (!make_map(&tb, Bm, (uint64_t)K, (uint64_t)b_rows, (uint64_t)ldb, GATES ? BN / 3 : BN)) return false;
-  GemmShape sh{M, N, K, gate_rows};
+  const int k_blocks = (K + (TF32 ? BK / 2 : BK) - 1) / (TF32 ? BK / 2 : BK);
+  if (splits < 1 || !EpiSplitAware<Epi>::value) splits = 1;
+  GemmShape sh{M, N, K, gate_rows, splits, (k_blocks + splits - 1) / splits};
   int m_tiles = (M + BM - 1) / BM, n_tiles = (N + C::kNPerTile - 1) / C::kNPerTile;
-  int tiles = m_tiles * n_tiles;
+  int tiles = m_tiles * n_tiles * splits;
   int grid = tiles < kSMs ? tiles : kSMs;
   ProfScope prof_(kc, 2.0 * M * (GATES ? 3.0 * N : (double)N) * K, s);
   if (launch_pdl(kern, dim3(grid), dim3(kThreads), C::kSmemBytes, s, ta, tb, sh, epi, status) != cudaSuccess) return false;
@@ -294,6 +311,7 @@ struct EpiBias {  // out[m, n] = acc + bias[n]      (input projection)
 };
 
 struct EpiStore {  // out[m, n] = acc            (weight / input gradients)
+  static constexpr bool kSplitAware = true;
   float* out; i64 ld; int M, N;
   i64 split_stride;   // split products: range `sp` of the reduction goes to out + sp*split_stride (summed afterwards)
   __device__ void operator()(uint32_t taddr, int row, int n0, int half, int sp) const {
@@ -366,7 +384,8 @@ struct EpiFwd {  // GRU cell on the r|z|n accumulator columns of 64 hidden units
   }
 };
 
-struct EpiLin {  // adjoint coefficients of every step of a level
+template <bool BF16C = true>
+struct EpiLin {  // adjoint coefficients of every step of a level (gate coefficients stored in bf16, or in fp32)
   LinArgs a;
   __device__ void operator()(uint32_t taddr, int row, int u0, int half) const {
     const bool valid = row < a.M;
@@ -406,10 +425,17 @@ struct EpiLin {  // adjoint coefficients of every step of a level
             oa[e] = L.a; ocr[e] = L.cr; ocz[e] = L.cz; ocn[e] = L.cn; ocp[e] = L.cnp;
           }
           st4(a.a + o + c, oa[0], oa[1], oa[2], oa[3]);
-          *reinterpret_cast<uint2*>(a.crb + o + c) = pack4(make_float4(ocr[0], ocr[1], ocr[2], ocr[3]));
-          *reinterpret_cast<uint2*>(a.czb + o + c) = pack4(make_float4(ocz[0], ocz[1], ocz[2], ocz[3]));
-          *reinterpret_cast<uint2*>(a.cnb + o + c) = pack4(make_float4(ocn[0], ocn[1], ocn[2], ocn[3]));
-          if (a.cnpb) *reinterpret_cast<uint2*>(a.cnpb + o + c) = pack4(make_float4(ocp[0], ocp[1], ocp[2], ocp[3]));
+          if constexpr (BF16C) {
+            *reinterpret_cast<uint2*>(a.crb + o + c) = pack4(make_float4(ocr[0], ocr[1], ocr[2], ocr[3]));
+            *reinterpret_cast<uint2*>(a.czb + o + c) = pack4(make_float4(ocz[0], ocz[1], ocz[2], ocz[3]));
+            *reinterpret_cast<uint2*>(a.cnb + o + c) = pack4(make_float4(ocn[0], ocn[1], ocn[2], ocn[3]));
+            if (a.cnpb) *reinterpret_cast<uint2*>(a.cnpb + o + c) = pack4(make_float4(ocp[0], ocp[1], ocp[2], ocp[3]));
+          } else {
+            st4(a.cr + o + c, ocr[0], ocr[1], ocr[2], ocr[3]);
+            st4(a.cz + o + c, ocz[0], ocz[1], ocz[2], ocz[3]);
+            st4(a.cn + o + c, ocn[0], ocn[1], ocn[2], ocn[3]);
+            if (a.cnp) st4(a.cnp + o + c, ocp[0], ocp[1], ocp[2], ocp[3]);
+          }
         }
       }
     }
@@ -736,7 +762,7 @@ int umma_linearise(const LinArgs& a, UmmaAdjWs* w, cudaStream_t s) {
       return MGRIT_CUDA_ERROR;
     count_launch();
   }
-  return launch_gemm<192, true>(KC_LINEARISE, w->Apack, a.H, w->W_hh, a.H, a.M, a.H, a.H, a.H, 3 * a.H, EpiLin{a}, s) ? MGRIT_OK
+  return launch_gemm<192, true>(KC_LINEARISE, w->Apack, a.H, w->W_hh, a.H, a.M, a.H, a.H, a.H, 3 * a.H, EpiLin<true>{a}, s) ? MGRIT_OK
                                                                                                                       : MGRIT_CUDA_ERROR;
 }
 
@@ -847,6 +873,216 @@ int umma_adj_dx(const AdjStepArgs& a, const bf16* W_ihT, int C, float* out, Umma
     return MGRIT_CUDA_ERROR;
   count_launch();
   return launch_gemm<256, false>(KC_ADJ_STEP, w->Apack, 3 * a.H, W_ihT, 3 * a.H, a.M, C, 3 * a.H, 0, C, EpiStore{out, C, a.M, C, 0}, s)
+             ? MGRIT_OK : MGRIT_CUDA_ERROR;
+}
+
+// ======================================================================================================
+// TF32 operand modes: the same persistent tcgen05 GEMM with `.kind::tf32`, fp32 state, fp32 coefficients, the
+// row-per-thread epilogues above.  A tf32 value keeps 10 mantissa bits, so one product x*w is good to about 1e-3
+// relative.  MGRIT_OPERANDS_TF32 therefore runs every product as the three-term split
+//     x w  ~=  x_hi w_hi + x_lo w_hi + x_hi w_lo,     x_hi = tf32(x), x_lo = tf32(x - x_hi)   (the dropped term is 2^-22),
+// laid out as ONE product over a three times longer reduction: the operand-forming kernels write A' = [hi | lo | hi] and
+// B' = [hi | hi | lo] along K, and the GEMM kernel does not know.  MGRIT_OPERANDS_TF32_1PASS writes only tf32(x).
+namespace {
+
+__device__ __forceinline__ float tf32_rna(float x) {
+  uint32_t r;
+  asm("cvt.rna.tf32.f32 %0, %1;" : "=r"(r) : "f"(x));
+  return __uint_as_float(r);
+}
+// segment `seg` (0..S-1) of the split of x for an A-side (roleB = false: hi, lo, hi) or B-side (hi, hi, lo) operand
+__device__ __forceinline__ float split_part(float x, int seg, bool roleB) {
+  const float hi = tf32_rna(x);
+  const bool want_lo = roleB ? (seg == 2) : (seg == 1);
+  return want_lo ? tf32_rna(x - hi) : hi;
+}
+
+// dst[m, seg*K + c] = split(src row (k, b))[c],  m = k*B + b, rows of K floats
+__global__ void __launch_bounds__(kPT) split_rows_kernel(const float* __restrict__ src, i64 ks, int B, int K, i64 M, int S, int roleB,
+                                                         float* __restrict__ dst) {
+  pdl_wait();
+  pdl_trigger();
+  const i64 total = M * K;
+  for (i64 e = (i64)blockIdx.x * blockDim.x + threadIdx.x; e < total; e += (i64)gridDim.x * blockDim.x) {
+    const i64 m = e / K; const int c = (int)(e % K);
+    const i64 k = m / B; const int b = (int)(m % B);
+    const float x = src[k * ks + (i64)b * K + c];
+    for (int seg = 0; seg < S; ++seg) dst[m * S * K + (i64)seg * K + c] = split_part(x, seg, roleB != 0);
+  }
+}
+
+// dst[m, seg*3H + g*H + i] = split(c_g[m, i] * lam[m, i])   (A side)
+__global__ void __launch_bounds__(kPT) split_adj_kernel(const float* __restrict__ lin, i64 lin_ks, const float* __restrict__ cr,
+                                                        const float* __restrict__ cz, const float* __restrict__ cn, i64 coef_ks, int B,
+                                                        int H, i64 M, int S, float* __restrict__ dst) {
+  pdl_wait();
+  pdl_trigger();
+  const i64 total = M * H;
+  for (i64 e = (i64)blockIdx.x * blockDim.x + threadIdx.x; e < total; e += (i64)gridDim.x * blockDim.x) {
+    const i64 m = e / H; const int i = (int)(e % H);
+    const i64 k = m / B; const int b = (int)(m % B);
+    const i64 ro = (i64)b * H + i;
+    const float l = lin[k * lin_ks + ro];
+    const float v[3] = {cr[k * coef_ks + ro] * l, cz[k * coef_ks + ro] * l, cn[k * coef_ks + ro] * l};
+    for (int seg = 0; seg < S; ++seg)
+#pragma unroll
+      for (int g = 0; g < 3; ++g) dst[m * S * 3 * H + (i64)seg * 3 * H + g * H + i] = split_part(v[g], seg, false);
+  }
+}
+
+// dst[c, seg*R + r] = split(src row r)[c]; src rows: r < Rfirst ? first + r*C : rest + (r - Rfirst)*C   ([R, C] -> [C, S*R])
+__global__ void __launch_bounds__(1024) transpose_split_kernel(const float* __restrict__ first, i64 Rfirst, const float* __restrict__ rest,
+                                                               i64 R, int C, int S, int roleB, float* __restrict__ dst) {
+  __shared__ float tile[32][33];
+  const i64 r0 = (i64)blockIdx.x * 32; const int c0 = blockIdx.y * 32;
+  const i64 r = r0 + threadIdx.y; const int c = c0 + threadIdx.x;
+  float v = 0.f;
+  if (r < R && c < C) v = r < Rfirst ? first[r * C + c] : rest[(r - Rfirst) * C + c];
+  tile[threadIdx.y][threadIdx.x] = v;
+  __syncthreads();
+  const i64 rr = r0 + threadIdx.x; const int cc = c0 + threadIdx.y;
+  if (rr < R && cc < C) {
+    const float x = tile[threadIdx.x][threadIdx.y];
+    for (int seg = 0; seg < S; ++seg) dst[(i64)cc * S * R + (i64)seg * R + rr] = split_part(x, seg, roleB != 0);
+  }
+}
+
+bool split_rows(const float* src, i64 ks, int B, int K, i64 M, int S, bool roleB, float* dst, cudaStream_t s) {
+  if (M <= 0) return true;
+  if (launch_pdl(split_rows_kernel, dim3(pgrid(M * K)), dim3(kPT), 0, s, src, ks, B, K, M, S, (int)roleB, dst) != cudaSuccess) return false;
+  count_launch();
+  return true;
+}
+void transpose_split(const float* first, i64 Rfirst, const float* rest, i64 R, int C, int S, bool roleB, float* dst, cudaStream_t s) {
+  if (R <= 0) return;
+  transpose_split_kernel<<<dim3((unsigned)((R + 31) / 32), (C + 31) / 32), dim3(32, 32), 0, s>>>(first, Rfirst, rest, R, C, S, (int)roleB, dst);
+  count_launch();
+}
+
+}  // namespace
+
+int tf32_supported(const mgrit_gru_cfg* c) {
+  // 64 hidden units per gate tile, 16-column epilogue chunks, 16-byte row pitches of the [., S*T*B] gradient operands
+  if (c->H % 64 != 0 || c->I % 16 != 0 || ((i64)c->T * c->B) % 4 != 0) return MGRIT_UNSUPPORTED;
+  return MGRIT_OK;
+}
+
+void tf32_plan_fwd(const mgrit_gru_cfg* c, const int* N, int L, char* base, size_t* off, Tf32Ws* o) {
+  const size_t S = c->operands == MGRIT_OPERANDS_TF32 ? 3 : 1, H = c->H, I = c->I, TB = (size_t)c->T * c->B;
+  o->S = (int)S;
+  o->W_hh = take<float>(base, off, 3 * H * S * H);
+  o->W_ih = take<float>(base, off, 3 * H * S * I);
+  o->W_hhT = o->W_ihT = o->dAT = o->RT = nullptr;
+  size_t ap = max_step_rows(c, N, L) * S * H;
+  if (TB * S * I > ap) ap = TB * S * I;
+  o->apack_elems = ap;
+  o->Apack = take<float>(base, off, ap);
+}
+
+void tf32_plan_adj(const mgrit_gru_cfg* c, const int* N, int L, char* base, size_t* off, Tf32Ws* o) {
+  const size_t S = c->operands == MGRIT_OPERANDS_TF32 ? 3 : 1, H = c->H, I = c->I, TB = (size_t)c->T * c->B;
+  o->S = (int)S;
+  o->W_hh = take<float>(base, off, 3 * H * S * H);
+  o->W_ih = nullptr;
+  o->W_hhT = take<float>(base, off, H * S * 3 * H);
+  o->W_ihT = take<float>(base, off, I * S * 3 * H);
+  o->apack_elems = TB * S * 3 * H;       // the input-gradient product packs all T*B rows of dA; every step needs less
+  o->Apack = take<float>(base, off, o->apack_elems);
+  o->dAT = take<float>(base, off, 3 * H * S * TB);
+  o->RT = take<float>(base, off, (H > I ? H : I) * S * TB);
+  o->split_scratch = take<float>(base, off, 4 * 3 * H * (H > I ? H : I));
+}
+
+int tf32_prepare_fwd(const mgrit_gru_cfg* c, const gru_params* p, const float* x, float* gi, Tf32Ws* w, cudaStream_t s) {
+  const int H = c->H, I = c->I, S = w->S;
+  const int TB = c->T * c->B;
+  if (!status_ptr()) return MGRIT_CUDA_ERROR;
+  bool ok = split_rows(p->W_hh, 0, 3 * H, H, 3 * H, S, true, w->W_hh, s) && split_rows(p->W_ih, 0, 3 * H, I, 3 * H, S, true, w->W_ih, s) &&
+            split_rows(x, 0, TB, I, TB, S, false, w->Apack, s);
+  // gi = x W_ih^T + b_ih :  M = T*B, N = 3H, K = S*I
+  ok = ok && launch_gemm<256, false>(KC_PROJ, (const float*)w->Apack, (i64)S * I, (const float*)w->W_ih, (i64)S * I, TB, 3 * H, S * I, 0, 3 * H,
+                                     EpiBias{gi, 3 * H, p->b_ih, TB, 3 * H}, s);
+  return ok ? MGRIT_OK : MGRIT_CUDA_ERROR;
+}
+
+int tf32_fwd_step(const FwdStepArgs& a, Tf32Ws* w, cudaStream_t s) {
+  const int S = w->S;
+  if (!split_rows(a.hin, a.hin_ks, a.B, a.H, a.M, S, false, w->Apack, s)) return MGRIT_CUDA_ERROR;
+  return launch_gemm<192, true>(KC_FWD_STEP, (const float*)w->Apack, (i64)S * a.H, (const float*)w->W_hh, (i64)S * a.H, a.M, a.H, S * a.H, a.H,
+                                3 * a.H, EpiFwd{a}, s) ? MGRIT_OK : MGRIT_CUDA_ERROR;
+}
+
+int tf32_prepare_adj(const mgrit_gru_cfg* c, const gru_params* p, Tf32Ws* w, cudaStream_t s) {
+  const int H = c->H, I = c->I, S = w->S;
+  if (!status_ptr()) return MGRIT_CUDA_ERROR;
+  if (!split_rows(p->W_hh, 0, 3 * H, H, 3 * H, S, true, w->W_hh, s)) return MGRIT_CUDA_ERROR;
+  transpose_split(nullptr, 0, p->W_hh, 3 * H, H, S, true, w->W_hhT, s);   // [H, S*3H]
+  transpose_split(nullptr, 0, p->W_ih, 3 * H, I, S, true, w->W_ihT, s);   // [I, S*3H]
+  return MGRIT_OK;
+}
+
+int tf32_linearise(const LinArgs& a, Tf32Ws* w, cudaStream_t s) {
+  // rows (j-1, b): state entering forward step j of the level = h at fine time t0 + stride*(j-1) (h_0 for time 0)
+  const i64 BH = (i64)a.B * a.H;
+  const int N = a.M / a.B, S = w->S;
+  int done = 0;
+  if (a.t0 == 0) {
+    if (!split_rows(a.h0, 0, a.B, a.H, a.B, S, false, w->Apack, s)) return MGRIT_CUDA_ERROR;
+    done = 1;
+  }
+  if (N > done) {
+    const i64 t1 = a.t0 + (i64)done * a.stride_t;
+    if (!split_rows(a.h + (t1 - 1) * BH, a.stride_t * BH, a.B, a.H, (i64)(N - done) * a.B, S, false, w->Apack + (i64)done * BH * S, s))
+      return MGRIT_CUDA_ERROR;
+  }
+  return launch_gemm<192, true>(KC_LINEARISE, (const float*)w->Apack, (i64)S * a.H, (const float*)w->W_hh, (i64)S * a.H, a.M, a.H, S * a.H, a.H,
+                                3 * a.H, EpiLin<false>{a}, s) ? MGRIT_OK : MGRIT_CUDA_ERROR;
+}
+
+int tf32_adj_step(const AdjStepArgs& a, Tf32Ws* w, cudaStream_t s) {
+  const int S = w->S, K = S * 3 * a.H;
+  ProfScope prof(KC_ADJ_STEP, 2.0 * a.M * (double)K * a.H, s);
+  if (launch_pdl(split_adj_kernel, dim3(pgrid((i64)a.M * a.H)), dim3(kPT), 0, s, a.lin, a.lin_ks, a.cr, a.cz, a.cn, a.coef_ks, a.B, a.H,
+                 (i64)a.M, S, w->Apack) != cudaSuccess)
+    return MGRIT_CUDA_ERROR;
+  count_launch();
+  const int tiles256 = ((a.M + BM - 1) / BM) * ((a.H + 255) / 256);
+  bool ok;
+  if (tiles256 * 2 <= kSMs)
+    ok = launch_gemm<64, false>(KC_ADJ_STEP, (const float*)w->Apack, (i64)K, (const float*)w->W_hhT, (i64)K, a.M, a.H, K, 0, a.H, EpiAdj<64>{a}, s);
+  else
+    ok = launch_gemm<256, false>(KC_ADJ_STEP, (const float*)w->Apack, (i64)K, (const float*)w->W_hhT, (i64)K, a.M, a.H, K, 0, a.H, EpiAdj<256>{a}, s);
+  return ok ? MGRIT_OK : MGRIT_CUDA_ERROR;
+}
+
+// dW[n3, c] = sum_m dA[m, n3] * R[m, c],  R rows: m < Bfirst ? first[m] : rest[m - Bfirst]: both operands transposed (and
+// split) so that the reduction index m runs along K-major rows; the long reduction is cut into up to four ranges.
+int tf32_wgrad(const float* dA, int M, int H3, const float* first, int Bfirst, const float* rest, int C, float* dW, Tf32Ws* w,
+               cudaStream_t s) {
+  const int S = w->S, K = S * M;
+  ProfScope prof(KC_WGRAD, 2.0 * H3 * (double)C * K, s);
+  transpose_split(nullptr, 0, dA, M, H3, S, false, w->dAT, s);          // [3H, S*M]
+  transpose_split(first, Bfirst, rest, M, C, S, true, w->RT, s);        // [C,  S*M]
+  const size_t scratch_bytes = (size_t)4 * H3 * C * sizeof(float);
+  const int splits = (((i64)H3 * C) % 4 == 0) ? pick_splits(H3, C, K, scratch_bytes) : 1;
+  if (splits == 1)
+    return launch_gemm<256, false>(KC_WGRAD, (const float*)w->dAT, (i64)K, (const float*)w->RT, (i64)K, H3, C, K, 0, C, EpiStore{dW, C, H3, C, 0}, s)
+               ? MGRIT_OK : MGRIT_CUDA_ERROR;
+  const i64 n = (i64)H3 * C;
+  if (!launch_gemm<256, false>(KC_WGRAD, (const float*)w->dAT, (i64)K, (const float*)w->RT, (i64)K, H3, C, K, 0, C,
+                               EpiStore{w->split_scratch, C, H3, C, n}, s, splits))
+    return MGRIT_CUDA_ERROR;
+  sum_splits_kernel<<<pgrid(n / 4), kPT, 0, s>>>(reinterpret_cast<const float4*>(w->split_scratch), n / 4, splits, reinterpret_cast<float4*>(dW));
+  count_launch();
+  return MGRIT_OK;
+}
+
+// dx[m, c] = sum_n3 dA[m, n3] * W_ih[n3, c]
+int tf32_dgrad(const float* dA, int M, int H3, int C, float* dx, Tf32Ws* w, cudaStream_t s) {
+  const int S = w->S, K = S * H3;
+  if ((size_t)M * K > w->apack_elems) return MGRIT_UNSUPPORTED;
+  if (!split_rows(dA, 0, M, H3, M, S, false, w->Apack, s)) return MGRIT_CUDA_ERROR;
+  return launch_gemm<256, false>(KC_WGRAD, (const float*)w->Apack, (i64)K, (const float*)w->W_ihT, (i64)K, M, C, K, 0, C, EpiStore{dx, C, M, C, 0}, s)
              ? MGRIT_OK : MGRIT_CUDA_ERROR;
 }
 

@@ -26,6 +26,32 @@ struct UmmaAdjWs {
   size_t maxM;
 };
 
+// TF32 operand modes (same GEMM kernel, `.kind::tf32`): operands are fp32 arrays of tf32 values, split in S = 3 parts
+// along the reduction (MGRIT_OPERANDS_TF32) or rounded once (S = 1, MGRIT_OPERANDS_TF32_1PASS)
+struct Tf32Ws {
+  int S;
+  float* W_hh;    // [3H, S*H]   B side of the forward product
+  float* W_ih;    // [3H, S*I]   forward call only
+  float* W_hhT;   // [H, S*3H]   adjoint call: B side of the adjoint step
+  float* W_ihT;   // [I, S*3H]   adjoint call: B side of dx = dA_i W_ih
+  float* Apack;   // A side of the current product
+  size_t apack_elems;
+  float* dAT;     // [3H, S*T*B] gradient pass: dA^T
+  float* RT;      // [max(H,I), S*T*B]: h_prev^T or x^T
+  float* split_scratch;   // partial products of a split reduction
+};
+int tf32_supported(const mgrit_gru_cfg* c);
+void tf32_plan_fwd(const mgrit_gru_cfg* c, const int* N, int L, char* base, size_t* off, Tf32Ws* o);
+void tf32_plan_adj(const mgrit_gru_cfg* c, const int* N, int L, char* base, size_t* off, Tf32Ws* o);
+int tf32_prepare_fwd(const mgrit_gru_cfg* c, const gru_params* p, const float* x, float* gi, Tf32Ws* w, cudaStream_t s);
+int tf32_prepare_adj(const mgrit_gru_cfg* c, const gru_params* p, Tf32Ws* w, cudaStream_t s);
+int tf32_fwd_step(const FwdStepArgs& a, Tf32Ws* w, cudaStream_t s);
+int tf32_linearise(const LinArgs& a, Tf32Ws* w, cudaStream_t s);
+int tf32_adj_step(const AdjStepArgs& a, Tf32Ws* w, cudaStream_t s);
+int tf32_wgrad(const float* dA, int M, int H3, const float* first, int Bfirst, const float* rest, int C, float* dW, Tf32Ws* w,
+               cudaStream_t s);
+int tf32_dgrad(const float* dA, int M, int H3, int C, float* dx, Tf32Ws* w, cudaStream_t s);
+
 int umma_supported(const mgrit_gru_cfg* c);
 void umma_plan_fwd(const mgrit_gru_cfg* c, const int* N, int L, char* base, size_t* off, UmmaFwdWs* o);
 void umma_plan_adj(const mgrit_gru_cfg* c, const int* N, int L, char* base, size_t* off, UmmaAdjWs* o);

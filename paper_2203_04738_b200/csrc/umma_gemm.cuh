@@ -109,11 +109,25 @@ __host__ __device__ constexpr uint32_t instr_desc_bf16(int n) {
 // ... both MN-major (bits 15 and 16)
 __host__ __device__ constexpr uint32_t instr_desc_bf16_mn(int n) { return instr_desc_bf16(n) | (1u << 15) | (1u << 16); }
 
+// D fp32, A and B tf32 (fp32 words whose low 13 mantissa bits the producer has already rounded away), both K-major
+__host__ __device__ constexpr uint32_t instr_desc_tf32(int n) {
+  return (1u << 4) | (2u << 7) | (2u << 10) | ((uint32_t)(n >> 3) << 17) | ((uint32_t)(BM >> 4) << 24);
+}
+
 __device__ __forceinline__ void mma_bf16(uint32_t d_tmem, uint64_t adesc, uint64_t bdesc, uint32_t idesc, uint32_t accumulate) {
   asm volatile(
       "{\n\t.reg .pred p;\n\t"
       "setp.ne.b32 p, %4, 0;\n\t"
       "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
+      ::"r"(d_tmem), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate)
+      : "memory");
+}
+// one MMA of .kind::tf32 consumes 8 k (again 32 bytes of a K-major row)
+__device__ __forceinline__ void mma_tf32(uint32_t d_tmem, uint64_t adesc, uint64_t bdesc, uint32_t idesc, uint32_t accumulate) {
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "setp.ne.b32 p, %4, 0;\n\t"
+      "tcgen05.mma.cta_group::1.kind::tf32 [%0], %1, %2, %3, p;\n\t}"
       ::"r"(d_tmem), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate)
       : "memory");
 }
@@ -137,11 +151,17 @@ __device__ __forceinline__ void tmem_ld16(uint32_t taddr, float* v) {
 __device__ __forceinline__ void tmem_ld_wait() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
 
 struct GemmShape {
-  int M, N, K;          // K a multiple of 8 (TMA stride rule); any M, N
+  int M, N, K;          // row pitches must be multiples of 16 bytes (TMA stride rule); any M, N
   int gate_rows;        // GATES: row distance between the r, z, n blocks of B (= H); else 0
-  int splits;           // MN-major products only: the reduction is cut into `splits` ranges of kb_per_split k-blocks,
-  int kb_per_split;     // each (tile, range) is one work item and the epilogue is told which range it finishes
+  int splits;           // split products (MN-major, or an epilogue with kSplitAware): the reduction is cut into `splits`
+  int kb_per_split;     // ranges of kb_per_split k-blocks, each (tile, range) is one work item and the epilogue is told
+                        // which range it finishes; 0 or 1 = the whole reduction in one item
 };
+
+// An epilogue that can finish one range of a split reduction declares `static constexpr bool kSplitAware = true`
+// and takes the range index as a fifth argument.
+template <class E, class = void> struct EpiSplitAware { static constexpr bool value = false; };
+template <class E> struct EpiSplitAware<E, decltype((void)E::kSplitAware)> { static constexpr bool value = E::kSplitAware; };
 
 template <int BN, bool GATES>
 struct Cfg {
@@ -160,7 +180,8 @@ struct Cfg {
 //   n0 : first output column (GATES: first hidden unit) of the tile
 //   half: 0 or 1, the half of the tile's output columns this warp is responsible for
 // MNMAJ: D[m, n] = sum_k A[k, m] * B[k, n] with A stored [K, M] and B stored [K, N] (both row-major)
-template <int BN, bool GATES, class Epi, bool MNMAJ = false>
+// TF32: the operands are fp32 words holding tf32 values (K-major only); a k-block is 32 of them, again 128 bytes a row
+template <int BN, bool GATES, class Epi, bool MNMAJ = false, bool TF32 = false>
 __global__ void __launch_bounds__(kThreads, 1)
 umma_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB, GemmShape sh, Epi epi,
                  int* status) {
@@ -180,14 +201,17 @@ umma_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int m_tiles = (sh.M + BM - 1) / BM;
   const int n_tiles = (sh.N + C::kNPerTile - 1) / C::kNPerTile;
-  const int k_blocks_all = (sh.K + BK - 1) / BK;
-  const int splits = MNMAJ ? sh.splits : 1;
+  static_assert(!(MNMAJ && TF32), "tf32 operands are K-major here");
+  constexpr int kBK = TF32 ? BK / 2 : BK;                // elements of one 128-byte k-block row
+  constexpr bool SPLITK = MNMAJ || EpiSplitAware<Epi>::value;
+  const int k_blocks_all = (sh.K + kBK - 1) / kBK;
+  const int splits = (SPLITK && sh.splits > 1) ? sh.splits : 1;
   const int mn_tiles = m_tiles * n_tiles;
   const int tiles = mn_tiles * splits;                   // work items
   // k-block range of item t (the whole reduction unless split)
-  auto kb_begin = [&](int t) { return MNMAJ ? (t / mn_tiles) * sh.kb_per_split : 0; };
+  auto kb_begin = [&](int t) { return splits > 1 ? (t / mn_tiles) * sh.kb_per_split : 0; };
   auto kb_end = [&](int t) {
-    if (!MNMAJ) return k_blocks_all;
+    if (splits == 1) return k_blocks_all;
     int e = (t / mn_tiles + 1) * sh.kb_per_split;
     return e < k_blocks_all ? e : k_blocks_all;
   };
@@ -230,13 +254,13 @@ umma_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
 #pragma unroll
             for (int i = 0; i < BN / 64; ++i) tma_load_2d(b_dst + i * 8192, &tmB, full_bar(stage), nt * BN + i * 64, kb * BK);
           } else {
-          tma_load_2d(a_dst, &tmA, full_bar(stage), kb * BK, mt * BM);
+          tma_load_2d(a_dst, &tmA, full_bar(stage), kb * kBK, mt * BM);
           if (GATES) {
 #pragma unroll
             for (int g = 0; g < 3; ++g)
-              tma_load_2d(b_dst + g * (C::kBBytes / 3), &tmB, full_bar(stage), kb * BK, g * sh.gate_rows + nt * C::kNPerTile);
+              tma_load_2d(b_dst + g * (C::kBBytes / 3), &tmB, full_bar(stage), kb * kBK, g * sh.gate_rows + nt * C::kNPerTile);
           } else {
-            tma_load_2d(b_dst, &tmB, full_bar(stage), kb * BK, nt * BN);
+            tma_load_2d(b_dst, &tmB, full_bar(stage), kb * kBK, nt * BN);
           }
           }
           if (++stage == C::kStages) { stage = 0; phase ^= 1u; }
@@ -246,7 +270,7 @@ umma_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
   } else if (warp == 1) {
     // ------------------------------------------------------------ MMA issuer
     if (lane == 0) {
-      constexpr uint32_t idesc = MNMAJ ? instr_desc_bf16_mn(BN) : instr_desc_bf16(BN);
+      constexpr uint32_t idesc = TF32 ? instr_desc_tf32(BN) : (MNMAJ ? instr_desc_bf16_mn(BN) : instr_desc_bf16(BN));
       int stage = 0; uint32_t phase = 0;
       int it = 0;
       bool ok = true;
@@ -263,11 +287,13 @@ umma_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
           const uint32_t a_src = tiles_base + stage * C::kStageBytes;
           const uint64_t adesc = MNMAJ ? smem_desc_mn_sw128(a_src) : smem_desc_sw128(a_src);
           const uint64_t bdesc = MNMAJ ? smem_desc_mn_sw128(a_src + C::kABytes) : smem_desc_sw128(a_src + C::kABytes);
-          // one MMA consumes 16 k: 32 bytes along a K-major row, 16 rows of 128 bytes (2048 bytes) when MN-major
+          // one MMA consumes 16 bf16 (8 tf32) k: 32 bytes along a K-major row, 16 rows of 128 bytes (2048 bytes) when MN-major
           constexpr uint64_t kstep = MNMAJ ? (2048 >> 4) : (32 >> 4);
 #pragma unroll
-          for (int k = 0; k < BK / 16; ++k)
-            mma_bf16(d_tmem, adesc + kstep * k, bdesc + kstep * k, idesc, ((kb - kb0) | k) != 0 ? 1u : 0u);
+          for (int k = 0; k < 4; ++k) {
+            if constexpr (TF32) mma_tf32(d_tmem, adesc + kstep * k, bdesc + kstep * k, idesc, ((kb - kb0) | k) != 0 ? 1u : 0u);
+            else mma_bf16(d_tmem, adesc + kstep * k, bdesc + kstep * k, idesc, ((kb - kb0) | k) != 0 ? 1u : 0u);
+          }
           mma_commit(empty_bar(stage));   // frees the stage when the MMAs have read it
           if (++stage == C::kStages) { stage = 0; phase ^= 1u; }
         }
@@ -286,7 +312,7 @@ umma_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
       if (!mbar_wait(tfull_bar(as), aphase, abortp, status, 4)) break;
       tc_fence_after();
       const uint32_t taddr = tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(as * BN);
-      if constexpr (MNMAJ) epi(taddr, mt * BM + q * 32 + lane, nt * C::kNPerTile, half, t / mn_tiles);
+      if constexpr (SPLITK) epi(taddr, mt * BM + q * 32 + lane, nt * C::kNPerTile, half, t / mn_tiles);
       else epi(taddr, mt * BM + q * 32 + lane, nt * C::kNPerTile, half);
       tc_fence_before();
       mbar_arrive(tempty_bar(as));
