@@ -134,6 +134,7 @@ struct FwdWs {
   float* U[kMaxLevels]; float* G[kMaxLevels]; double* res_acc; UmmaFwdWs um; Tf32Ws tf;
   __nv_bfloat16* chain_ub; unsigned* chain_bar; uint4* chain_xw; size_t chain_xw_bytes;   // scratch of the persistent serial-chain kernel
   __nv_bfloat16* Ub[kMaxLevels];                  // bf16 copies of the level states (tensor-core A operands)
+  int* sweep_ctr; size_t sweep_ctr_n, sweep_ctr_used;   // progress counters of the multi-step relaxation launches (zeroed per call)
 };
 struct AdjWs {
   float* U[kMaxLevels]; float* G[kMaxLevels];
@@ -151,6 +152,7 @@ void plan_fwd(const mgrit_gru_cfg* c, const Hier& hr, Ws& w, FwdWs* o) {
   }
   o->res_acc = w.take<double>((size_t)(c->iters > 0 ? c->iters : 1));
   o->chain_ub = nullptr; o->chain_bar = nullptr; o->chain_xw = nullptr; o->chain_xw_bytes = 0;
+  o->sweep_ctr = nullptr; o->sweep_ctr_n = o->sweep_ctr_used = 0;
   for (int l = 0; l < kMaxLevels; ++l) o->Ub[l] = nullptr;
   if (c->operands == MGRIT_OPERANDS_BF16) {
     umma_plan_fwd(c, hr.N, hr.L, w.base, &w.off, &o->um);
@@ -159,6 +161,8 @@ void plan_fwd(const mgrit_gru_cfg* c, const Hier& hr, Ws& w, FwdWs* o) {
     o->chain_bar = w.take<unsigned>(((size_t)c->B / 16 + 1) * ((size_t)c->H / 8) + 64);
     o->chain_xw_bytes = serial_xw_bytes(c->B, c->H, 1);
     o->chain_xw = reinterpret_cast<uint4*>(w.take<char>(o->chain_xw_bytes));
+    o->sweep_ctr_n = 1 << 16;
+    o->sweep_ctr = w.take<int>(o->sweep_ctr_n);
   }
   if (is_tf32(c)) tf32_plan_fwd(c, hr.N, hr.L, w.base, &w.off, &o->tf);
 }
@@ -225,6 +229,21 @@ struct Cycle {
   }
   // all N_l dependent steps of level l in one persistent launch; false = not available here
   virtual bool chain(int l) { (void)l; return false; }
+  // A relaxation sweep of level l in one launch: kinds[i] = s in 1..cf-1: F-step to slot s of every interval;
+  // cf: C-step; cf + 1: the step that evaluates v at the C-points into G[l+1].  false = not available here.
+  virtual bool launch_sweep(int l, const int* kinds, int n) { (void)l; (void)kinds; (void)n; return false; }
+  // F (CF)^relax (the opening F optional), optionally followed by the evaluation of v at the C-points
+  bool relax_sweep(int l, bool first_f, int relax, bool with_v) {
+    if (rc != MGRIT_OK) return true;
+    int kinds[64], n = 0;
+    const int cf = c->cf;
+    if ((cf - 1) * (relax + 1) + relax + 1 > 64) return false;
+    if (first_f) for (int sI = 1; sI < cf; ++sI) kinds[n++] = sI;
+    for (int r = 0; r < relax; ++r) { kinds[n++] = cf; for (int sI = 1; sI < cf; ++sI) kinds[n++] = sI; }
+    if (with_v) kinds[n++] = cf + 1;
+    if (n < 2) return false;
+    return launch_sweep(l, kinds, n);
+  }
   virtual ~Cycle() {}
 
   // F-relaxation: from every C-point the cf - 1 F-points of its interval, one dependent step per launch over all
@@ -248,11 +267,13 @@ struct Cycle {
       return;
     }
     int relax = l == 0 ? c->relax_fine : c->relax_coarse;       // n: F (CF)^n
-    if (!skip_first_f) frelax(l);
-    for (int n = 0; n < relax; ++n) { crelax(l); frelax(l); }
     int nc = hr.N[l + 1];
-    // v_k = step_l(u_{cf k - 1}) + g_{cf k}  ->  G[l+1][k]
-    step(StepDesc{l, nc, cf - 1, cf, G[l + 1], 1, 1, G[l], cf, cf, cf, cf, 0});
+    if (!relax_sweep(l, !skip_first_f, relax, true)) {
+      if (!skip_first_f) frelax(l);
+      for (int n = 0; n < relax; ++n) { crelax(l); frelax(l); }
+      // v_k = step_l(u_{cf k - 1}) + g_{cf k}  ->  G[l+1][k]
+      step(StepDesc{l, nc, cf - 1, cf, G[l + 1], 1, 1, G[l], cf, cf, cf, cf, 0});
+    }
     // r_k = u_{cf k} - v_k ; U'_k = u_{cf k}
     stream_restrict_residual(U[l], cf, G[l + 1], U[l + 1], Ub ? Ub[l + 1] : nullptr, nc, (i64)BH,
                              (l == 0 && record) ? res_acc + cycle_idx : nullptr, s);
@@ -260,7 +281,7 @@ struct Cycle {
     step(StepDesc{l + 1, nc, 0, 1, G[l + 1], 1, 1, nullptr, 0, 0, 1, 1, 1});
     cycle(l + 1, false, false);
     stream_correct(U[l], Ub ? Ub[l] : nullptr, cf, U[l + 1], nc, (i64)BH, s);
-    frelax(l);
+    if (!relax_sweep(l, true, 0, false)) frelax(l);
     // F-cycle: one more V-cycle from this level down on the corrected state (on the last two levels: a second
     // V-cycle).  Its opening F-relaxation would repeat the one just done.
     if ((c->flags & MGRIT_FLAG_F_CYCLE) && fcycle_leg) {
@@ -295,6 +316,42 @@ struct FwdCycle : Cycle {
     a.g = G[l]; a.W = um->W_hh; a.b_hh = p->b_hh; a.gamma = hr.gamma[l]; a.cell = c->cell; a.bar = fw->chain_bar;
     a.xw = fw->chain_xw; a.xw_bytes = fw->chain_xw_bytes;
     return serial_fwd_solve(a, s);
+  }
+  bool launch_sweep(int l, const int* kinds, int n) override {
+    const int cf = c->cf;
+    if (c->operands != MGRIT_OPERANDS_BF16 || !Ub || hr.N[l] % cf != 0 || n > kMaxFwdSweepSteps) return false;
+    FwdSweepArgs a;
+    a.B = c->B; a.H = c->H; a.nk = hr.N[l] / cf; a.cf = cf; a.n = n;
+    const size_t need = (size_t)n * (((size_t)a.nk * c->B + 127) / 128);
+    if (!fw->sweep_ctr || fw->sweep_ctr_used + need > fw->sweep_ctr_n) return false;
+    a.U = U[l]; a.Ub = Ub[l];
+    const i64 st = hr.stride_t[l];
+    a.gi = gi + (st - 1) * (i64)BH * 3; a.gi_ss = st * (i64)BH * 3; a.gi_ks = st * cf * (i64)BH * 3;
+    a.g = G[l] ? G[l] + BH : nullptr;
+    a.b_hh = p->b_hh; a.gamma = hr.gamma[l]; a.cell = c->cell;
+    a.ctr = fw->sweep_ctr + fw->sweep_ctr_used;
+    for (int i = 0; i < n; ++i) {
+      FwdSweepStep& q = a.st[i];
+      const int kd = kinds[i], prev = i ? kinds[i - 1] : 0;
+      if (kd < cf) {             // F-step to slot kd
+        q.in_s = kd - 1; q.tgt_s = kd - 1;
+        q.out = U[l] + (size_t)kd * BH; q.out_ks = (i64)cf * BH; q.out_b = Ub[l] + (size_t)kd * BH;
+        q.dep = prev == cf ? 2 : 1;
+      } else if (kd == cf) {     // C-step: slot cf of interval k = slot 0 of interval k + 1
+        q.in_s = cf - 1; q.tgt_s = cf - 1;
+        q.out = U[l] + (size_t)cf * BH; q.out_ks = (i64)cf * BH; q.out_b = Ub[l] + (size_t)cf * BH;
+        q.dep = 3;
+      } else {                   // v at the C-points, into the coarse level's G
+        q.in_s = cf - 1; q.tgt_s = cf - 1;
+        q.out = G[l + 1] + BH; q.out_ks = (i64)BH; q.out_b = nullptr;
+        q.dep = 1;
+      }
+    }
+    const int r = umma_fwd_sweep(a, um, s);
+    if (r == MGRIT_UNSUPPORTED) return false;
+    fw->sweep_ctr_used += need;
+    if (r != MGRIT_OK) rc = r;
+    return true;
   }
   int launch_step(const StepDesc& d) override {
     FwdStepArgs a;
@@ -404,6 +461,7 @@ int forward_impl(const mgrit_gru_cfg* cfg_in, bool serial, const gru_params* p, 
   cudaMemsetAsync(fw.U[0] + BH, 0, sizeof(float) * (size_t)c.T * BH, s);
   for (int l = 0; l < hr.L; ++l) cudaMemcpyAsync(fw.U[l], h0, sizeof(float) * BH, cudaMemcpyDeviceToDevice, s);
   const bool shadows = c.operands == MGRIT_OPERANDS_BF16 && 128 % c.B == 0;
+  if (shadows && fw.sweep_ctr) cudaMemsetAsync(fw.sweep_ctr, 0, sizeof(int) * fw.sweep_ctr_n, s);
   if (shadows) {
     cudaMemsetAsync(fw.Ub[0] + BH, 0, sizeof(__nv_bfloat16) * (size_t)c.T * BH, s);
     for (int l = 0; l < hr.L; ++l) umma_convert(h0, fw.Ub[l], (i64)BH, s);

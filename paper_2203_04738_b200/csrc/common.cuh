@@ -101,6 +101,27 @@ struct FwdStepArgs {
   int mode;                         // 0: hout = Phi + gadd ; 1: hout = hout - Phi   (FAS right-hand side)
 };
 
+// ---- a relaxation sweep: n dependent forward steps of one level over the same nk intervals, in ONE launch ----
+// Slots of the level: point j = k*cf + s (interval k, slot s).  A step starts from slot coordinate in_s of every
+// interval and arrives at target coordinate tgt_s, counted from slot 1 (tgt_s = cf - 1 is the C-point that closes
+// the interval); its result goes to rows out + k*out_ks + b*H (and their bf16 copy).
+struct FwdSweepStep {
+  int in_s, tgt_s;
+  float* out; i64 out_ks; __nv_bfloat16* out_b;
+  int dep;       // 0: first step; 1: follows a step on the same intervals; 2: follows a step that advanced the C-points
+                 // (reads what the neighbouring interval wrote); 3: advances the C-points (must not overtake their readers)
+};
+constexpr int kMaxFwdSweepSteps = 20;
+struct FwdSweepArgs {
+  int B, H, nk, cf, n;
+  const float* U; const __nv_bfloat16* Ub;   // level state and its bf16 copy, from slot 0
+  const float* gi; i64 gi_ss, gi_ks;         // input projection of target coordinate 0 of interval 0; element strides per slot / interval
+  const float* g;                            // FAS term of target coordinate 0 of interval 0 (slots like U), or nullptr
+  const float* b_hh; float gamma; int cell;
+  int* ctr;                                  // n * ceil(nk*B / 128) zeroed ints
+  FwdSweepStep st[kMaxFwdSweepSteps];
+};
+
 // ---- adjoint coefficients of every step of one level (discrete adjoint of the cell) ----
 // Row m = (j-1, b) for the level's forward steps j = 1..N_l; step j leaves fine time t0 + stride_t*(j-1) and arrives
 // at t0 + stride_t*j with that time's input.  Outputs are [N_l*B, H] each.

@@ -52,6 +52,21 @@ __device__ __forceinline__ void tma_load_3d_pair(uint32_t dst, const CUtensorMap
       ::"r"(dst), "l"(map), "r"(bar), "r"(c0), "r"(c1), "r"(c2)
       : "memory");
 }
+// 4-D maps {column, batch row, slot inside the interval, interval}: the forward kernel addresses the level state, the
+// input projection and the additive term by (slot, first interval of the tile), so that ONE launch can run several
+// dependent relaxation steps (a sweep) that differ only in the slot coordinate.
+__device__ __forceinline__ void tma_load_4d(uint32_t dst, const CUtensorMap* map, uint32_t bar, int c0, int c1, int c2, int c3) {
+  asm volatile(
+      "cp.async.bulk.tensor.4d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, %5, %6}], [%2];"
+      ::"r"(dst), "l"(map), "r"(bar), "r"(c0), "r"(c1), "r"(c2), "r"(c3)
+      : "memory");
+}
+__device__ __forceinline__ void tma_load_4d_pair(uint32_t dst, const CUtensorMap* map, uint32_t bar, int c0, int c1, int c2, int c3) {
+  asm volatile(
+      "cp.async.bulk.tensor.4d.cta_group::2.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, %5, %6}], [%2];"
+      ::"r"(dst), "l"(map), "r"(bar), "r"(c0), "r"(c1), "r"(c2), "r"(c3)
+      : "memory");
+}
 // tcgen05.ld is asynchronous: its destination registers are only valid after tcgen05.wait::ld.  The
 // results are therefore produced directly in their final registers (no copies that the compiler could
 // schedule before the wait), and tmem_ld_wait8 makes every later use depend on the wait.
@@ -101,6 +116,48 @@ struct CellArgs {
   const float* b_hh; float gamma; int cell; int mode;
 };
 
+// A sweep: up to kMaxSweepSteps dependent forward steps over the same rows (k, b) in one launch.  Work items are
+// (step, tile) in step-major order, CTA c takes items c, c + #CTAs, ...; an item of step s > 0 first waits until the
+// row tiles of step s - 1 that it reads (and whose earlier readers it must not overtake) are complete: the epilogue
+// warps count finished items per (step, row tile) in global memory.  Every dependency points to an earlier item and
+// all CTAs of the launch are resident (at most one per SM), so the earliest unfinished item can always proceed;
+// the wait is bounded like every other wait here.
+constexpr int kMaxSweepSteps = 20;
+struct SweepStep {
+  float* hout; i64 hout_ks; __nv_bfloat16* hout_b;   // destination rows (k, b): fp32 state and its bf16 copy (or nullptr)
+  int in_s;     // slot coordinate of the state the step starts from (maps A and HP)
+  int tgt_s;    // slot coordinate of the point it arrives at (maps GI and G)
+  int dep;      // row tiles of the previous step that must be complete: 0 none, 1 {mt}, 2 {mt - 1, mt}, 3 {mt, mt + 1}
+};
+struct SweepArgs {
+  int n_steps;
+  int* ctr;     // [n_steps][row tiles] zeroed counters (nullptr for a single step)
+  SweepStep st[kMaxSweepSteps];
+};
+
+// Bounded wait until *ctr >= target (acquire), then order the async proxy (TMA reads) behind what was acquired.
+__device__ __forceinline__ bool sweep_wait(const int* ctr, int target, volatile int* abort_flag, int* status, int code) {
+  uint64_t t0 = 0;
+  uint32_t spins = 0;
+  while (true) {
+    int v;
+    asm volatile("ld.acquire.gpu.global.s32 %0, [%1];" : "=r"(v) : "l"(ctr) : "memory");
+    if (v >= target) break;
+    if ((++spins & 63u) == 0) {
+      if (*abort_flag) return false;
+      const uint64_t now = global_ns();
+      if (t0 == 0) t0 = now;
+      if (now - t0 > kWaitLimitNs) {
+        *abort_flag = 1;
+        atomicCAS(status, 0, code);
+        return false;
+      }
+    }
+  }
+  asm volatile("fence.proxy.async;" ::: "memory");
+  return true;
+}
+
 namespace cellk {
 constexpr int CH = 16;                  // hidden units per epilogue chunk
 constexpr int kThreads = 352;
@@ -145,7 +202,7 @@ umma_cell_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
                  const __grid_constant__ CUtensorMap tmGI, const __grid_constant__ CUtensorMap tmHP,
                  const __grid_constant__ CUtensorMap tmG, const __grid_constant__ CUtensorMap tmCR,
                  const __grid_constant__ CUtensorMap tmCZ, const __grid_constant__ CUtensorMap tmCN,
-                 const __grid_constant__ CUtensorMap tmCP, CellArgs p, int* status) {
+                 const __grid_constant__ CUtensorMap tmCP, CellArgs p, const __grid_constant__ SweepArgs swp, int* status) {
   using namespace cellk;
   using C = CellCfg<HAS_G, LIN, PAIR>;
   using G = Geo<PAIR>;
@@ -175,6 +232,20 @@ umma_cell_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
   const int m_tiles = (p.M + kTileRows - 1) / kTileRows, n_tiles = (H + UN - 1) / UN, tiles = m_tiles * n_tiles;
   const int k_blocks = (H + BK - 1) / BK;
   auto row_tile = [&](int t) { return PAIR ? 2 * (t / n_tiles) + (int)rank : t / n_tiles; };
+  // forward: items (step, tile); the linearisation is a single step
+  const int n_items = LIN ? tiles : tiles * swp.n_steps;
+  constexpr int kCtrTarget = PAIR ? 16 : 8;       // epilogue warps that finish one item (both CTAs of a pair)
+  // the row tiles of step sg - 1 that item (sg, row tile mtile) depends on are complete (true also when there are none)
+  auto deps_ready = [&](int sg, int mtile, int code) {
+    if (LIN || sg == 0 || swp.st[sg].dep == 0) return true;
+    const int dep = swp.st[sg].dep;
+    const int lo = dep == 2 ? mtile - 1 : mtile, hi = dep == 3 ? mtile + 1 : mtile;
+    for (int m = lo; m <= hi; ++m) {
+      if (m < 0 || m >= m_tiles) continue;
+      if (!sweep_wait(swp.ctr + (sg - 1) * m_tiles + m, n_tiles * kCtrTarget, (volatile int*)&abort_flag, status, code)) return false;
+    }
+    return true;
+  };
 
   if (threadIdx.x == 0) {
     abort_flag = 0;
@@ -210,8 +281,11 @@ umma_cell_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
     // ------------------------------------------------------------ A/B producer
     if (lane == 0) {
       int stage = 0; uint32_t phase = 0; bool ok = true;
-      for (int t = cta; t < tiles && ok; t += ncta) {
+      for (int w = cta; w < n_items && ok; w += ncta) {
+        const int sg = LIN ? 0 : w / tiles, t = w - sg * tiles;
         const int mt = row_tile(t), nt = t % n_tiles;
+        const int in_s = LIN ? 0 : swp.st[sg].in_s;
+        if (!deps_ready(sg, t / n_tiles, 17)) { ok = false; break; }
         for (int kb = 0; kb < k_blocks; ++kb) {
           if (!mbar_wait(empty_bar(stage), phase ^ 1u, abortp, status, 11)) { ok = false; break; }
           const uint32_t a_dst = tiles_base + stage * kStageBytes, b_dst = a_dst + kABytes;
@@ -220,7 +294,8 @@ umma_cell_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
             // of r and of the first 40 units of z, CTA 1 the rest -- six 40-row boxes, three per CTA.
             const uint32_t fullL = mapa_shared(full_bar(stage), 0);
             if (rank == 0) mbar_expect_tx(full_bar(stage), 2 * kStageBytes);
-            tma_load_3d_pair(a_dst, &tmA, fullL, kb * BK, 0, mt * p.kt);
+            if (LIN) tma_load_3d_pair(a_dst, &tmA, fullL, kb * BK, 0, mt * p.kt);
+            else tma_load_4d_pair(a_dst, &tmA, fullL, kb * BK, 0, in_s, mt * p.kt);
 #pragma unroll
             for (int j = 0; j < 3; ++j) {
               const int piece = 3 * (int)rank + j;
@@ -228,7 +303,8 @@ umma_cell_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
             }
           } else {
             mbar_expect_tx(full_bar(stage), kStageBytes);
-            tma_load_3d(a_dst, &tmA, full_bar(stage), kb * BK, 0, mt * p.kt);
+            if (LIN) tma_load_3d(a_dst, &tmA, full_bar(stage), kb * BK, 0, mt * p.kt);
+            else tma_load_4d(a_dst, &tmA, full_bar(stage), kb * BK, 0, in_s, mt * p.kt);
 #pragma unroll
             for (int g = 0; g < 3; ++g) tma_load_2d(b_dst + g * (G::kBBytes / 3), &tmB, full_bar(stage), kb * BK, g * H + nt * UN);
           }
@@ -241,7 +317,7 @@ umma_cell_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
     if (lane == 0 && rank == 0) {
       constexpr uint32_t idesc = PAIR ? instr_desc_bf16_pair(BN) : instr_desc_bf16(BN);
       int stage = 0; uint32_t phase = 0; int it = 0; bool ok = true;
-      for (int t = cta; t < tiles && ok; t += ncta, ++it) {
+      for (int w = cta; w < n_items && ok; w += ncta, ++it) {
         const int as = it & 1;
         const uint32_t aphase = (uint32_t)(it >> 1) & 1u;
         if (!mbar_wait(tempty_bar(as), aphase ^ 1u, abortp, status, 12)) { ok = false; break; }
@@ -279,19 +355,29 @@ umma_cell_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
     // ------------------------------------------------------------ epilogue-operand producer
     if (lane == 0) {
       int eb = 0; uint32_t ephase = 0; bool ok = true;
-      for (int t = cta; t < tiles && ok; t += ncta) {
+      for (int w = cta; w < n_items && ok; w += ncta) {
+        const int sg = LIN ? 0 : w / tiles, t = w - sg * tiles;
         const int mt = row_tile(t), nt = t % n_tiles;
+        const int in_s = LIN ? 0 : swp.st[sg].in_s, tgt_s = LIN ? 0 : swp.st[sg].tgt_s;
+        if (!deps_ready(sg, t / n_tiles, 18)) { ok = false; break; }
         for (int c = 0; c < NCH; ++c) {
           const int u = nt * UN + c * CH, k0 = mt * p.kt;
           if (u >= H) break;                       // ragged last unit tile: these columns are never stored
           if (!mbar_wait(eempty_bar(eb), ephase ^ 1u, abortp, status, 14)) { ok = false; break; }
           const uint32_t dst = epi_base + eb * C::kEpiBytes;
           mbar_expect_tx(efull_bar(eb), C::kEpiBytes);
-          tma_load_3d(dst, &tmGI, efull_bar(eb), u, 0, k0);
-          tma_load_3d(dst + kOpBytes, &tmGI, efull_bar(eb), H + u, 0, k0);
-          tma_load_3d(dst + 2 * kOpBytes, &tmGI, efull_bar(eb), 2 * H + u, 0, k0);
-          tma_load_3d(dst + 3 * kOpBytes, &tmHP, efull_bar(eb), u, 0, k0);
-          if (HAS_G) tma_load_3d(dst + 4 * kOpBytes, &tmG, efull_bar(eb), u, 0, k0);
+          if (LIN) {
+            tma_load_3d(dst, &tmGI, efull_bar(eb), u, 0, k0);
+            tma_load_3d(dst + kOpBytes, &tmGI, efull_bar(eb), H + u, 0, k0);
+            tma_load_3d(dst + 2 * kOpBytes, &tmGI, efull_bar(eb), 2 * H + u, 0, k0);
+            tma_load_3d(dst + 3 * kOpBytes, &tmHP, efull_bar(eb), u, 0, k0);
+          } else {
+            tma_load_4d(dst, &tmGI, efull_bar(eb), u, 0, tgt_s, k0);
+            tma_load_4d(dst + kOpBytes, &tmGI, efull_bar(eb), H + u, 0, tgt_s, k0);
+            tma_load_4d(dst + 2 * kOpBytes, &tmGI, efull_bar(eb), 2 * H + u, 0, tgt_s, k0);
+            tma_load_4d(dst + 3 * kOpBytes, &tmHP, efull_bar(eb), u, 0, in_s, k0);
+            if (HAS_G) tma_load_4d(dst + 4 * kOpBytes, &tmG, efull_bar(eb), u, 0, tgt_s, k0);
+          }
           if (++eb == C::kEpiBufs) { eb = 0; ephase ^= 1u; }
         }
       }
@@ -311,7 +397,8 @@ umma_cell_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
     // A thread whose wait ran out (ok = false) keeps walking the loops without touching data, so that the named
     // barrier of the linearisation's store hand-over still sees all 256 epilogue threads.
     bool ok = true;
-    for (int t = cta; t < tiles; t += ncta, ++it) {
+    for (int w = cta; w < n_items; w += ncta, ++it) {
+      const int sg = LIN ? 0 : w / tiles, t = w - sg * tiles;
       const int mt = row_tile(t), nt = t % n_tiles;
       const int as = it & 1;
       const uint32_t aphase = (uint32_t)(it >> 1) & 1u;
@@ -371,15 +458,15 @@ umma_cell_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
               float phi = cell_forward<true>(gr[e], gz[e], gn[e], ar[e] + br[e], az[e] + bz[e], an[e] + bn[e], hp[e], p.gamma, p.cell);
               o[e] = HAS_G ? (p.mode == 1 ? gg[e] - phi : phi + gg[e]) : phi;
             }
-            const i64 idx = (i64)k * p.hout_ks + (i64)b * H + u;
-            stg8(p.hout + idx, o);
-            if (p.hout_b) {
+            const i64 idx = (i64)k * swp.st[sg].hout_ks + (i64)b * H + u;
+            stg8(swp.st[sg].hout + idx, o);
+            if (swp.st[sg].hout_b) {
               __nv_bfloat162 p0 = __floats2bfloat162_rn(o[0], o[1]), p1 = __floats2bfloat162_rn(o[2], o[3]);
               __nv_bfloat162 p2 = __floats2bfloat162_rn(o[4], o[5]), p3 = __floats2bfloat162_rn(o[6], o[7]);
               uint4 pk;
               pk.x = *reinterpret_cast<uint32_t*>(&p0); pk.y = *reinterpret_cast<uint32_t*>(&p1);
               pk.z = *reinterpret_cast<uint32_t*>(&p2); pk.w = *reinterpret_cast<uint32_t*>(&p3);
-              *reinterpret_cast<uint4*>(p.hout_b + idx) = pk;
+              *reinterpret_cast<uint4*>(swp.st[sg].hout_b + idx) = pk;
             }
           } else {
             float oa[8], ocr[8], ocz[8], ocn[8], ocp[8];
@@ -424,6 +511,12 @@ umma_cell_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
         if (lane == 0) {
           if (PAIR) mbar_arrive_cluster(mapa_shared(tempty_bar(as), 0));
           else mbar_arrive(tempty_bar(as));
+          // sweep: this warp's rows of the item are written (the warp barrier above ordered every lane's stores before
+          // this lane; the fence makes them visible before the count)
+          if (!LIN && swp.ctr) {
+            __threadfence();
+            asm volatile("red.release.gpu.global.add.s32 [%0], 1;" ::"l"(swp.ctr + sg * m_tiles + t / n_tiles) : "memory");
+          }
         }
       }
     }

@@ -194,61 +194,121 @@ static bool cell_pair_enabled(int M, int H) {
   return v == 1 && (i64)(M / (2 * BM)) * ((H + 79) / 80) >= kSMs / 2;
 }
 
-// Fused recurrent GEMM + cell (forward step or linearisation) with TMA-staged epilogue operands.
+// 4-D map {column, batch row, slot, interval}: element (c, b, sl, k) at base + k*ks + sl*ss + b*ld + c
+bool make_map4(CUtensorMap* m, CUtensorMapDataType dt, size_t esize, const void* base, uint64_t inner, uint64_t B, uint64_t nslots,
+               uint64_t nk, uint64_t ld, i64 ss, i64 ks, uint32_t box_inner, uint32_t box_k, CUtensorMapSwizzle sw) {
+  if (ks <= 0) ks = (i64)(ld * B);       // a single interval: any legal stride
+  if (ss <= 0) ss = (i64)(ld * B);       // a single slot
+  cuuint64_t dims[4] = {inner, B, nslots, nk};
+  cuuint64_t strides[3] = {ld * esize, (cuuint64_t)ss * esize, (cuuint64_t)ks * esize};
+  cuuint32_t box[4] = {box_inner, (cuuint32_t)B, 1, box_k};
+  cuuint32_t estr[4] = {1, 1, 1, 1};
+  CUresult r = g_encode(m, dt, 4, (void*)base, dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE, sw,
+                        CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  if (r != CUDA_SUCCESS) fprintf(stderr, "mgrit_gru: cuTensorMapEncodeTiled (4-D) failed (%d)\n", (int)r);
+  return r == CUDA_SUCCESS;
+}
+
+// Adjoint linearisation on the fused kernel, TMA-staged epilogue operands.
 // Rows (k, b), k = 0..nk-1: A rows at A + k*a_ks + b*H (bf16), gi rows at gi + k*gi_ks + b*3H,
-// previous state at hp + k*hp_ks + b*H, optional additive term at g + k*g_ks + b*H.
-template <bool LIN, bool HAS_G, bool PAIR>
-bool launch_cell_geo(int kc, const bf16* A, i64 a_ks, const float* gi, i64 gi_ks, const float* hp, i64 hp_ks, const float* g, i64 g_ks,
-                     int nk, const bf16* W, CellArgs ca, cudaStream_t s) {
-  using C = cellk::CellCfg<HAS_G, LIN, PAIR>;
+// previous state at hp + k*hp_ks + b*H.
+template <bool PAIR>
+bool launch_lin_geo(int kc, const bf16* A, i64 a_ks, const float* gi, i64 gi_ks, const float* hp, i64 hp_ks, int nk, const bf16* W,
+                    CellArgs ca, cudaStream_t s) {
+  using C = cellk::CellCfg<false, true, PAIR>;
   using G = cellk::Geo<PAIR>;
   if (nk <= 0) return true;
   int* const status = status_ptr();
   if (!status) return false;
   static bool attr_set[kMaxDevices] = {false};
-  auto kern = umma_cell_kernel<LIN, HAS_G, PAIR>;
+  auto kern = umma_cell_kernel<true, false, PAIR>;
   if (!set_smem_once(kern, C::kSmemBytes, attr_set)) return false;
   const int B = ca.B, H = ca.H, kt = 128 / B;
   ca.kt = kt; ca.M = nk * B;
-  CUtensorMap ta, tb, tgi, thp, tg;
+  CUtensorMap ta, tb, tgi, thp;
   if (!make_map3(&ta, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, A, H, B, nk, H, a_ks, BK, kt, CU_TENSOR_MAP_SWIZZLE_128B)) return false;
   if (!make_map(&tb, W, (uint64_t)H, (uint64_t)3 * H, (uint64_t)H, G::kBox)) return false;
   if (!make_map3(&tgi, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 4, gi, 3 * H, B, nk, 3 * H, gi_ks, cellk::CH, kt, CU_TENSOR_MAP_SWIZZLE_64B)) return false;
   if (!make_map3(&thp, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 4, hp, H, B, nk, H, hp_ks, cellk::CH, kt, CU_TENSOR_MAP_SWIZZLE_64B)) return false;
-  if (HAS_G) {
-    if (!make_map3(&tg, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 4, g, H, B, nk, H, g_ks, cellk::CH, kt, CU_TENSOR_MAP_SWIZZLE_64B)) return false;
-  } else {
-    tg = thp;
-  }
-  // linearisation: the four bf16 coefficient arrays [M, H] are written by TMA stores of [128 x 16] tiles
+  // the four bf16 coefficient arrays [M, H] are written by TMA stores of [128 x 16] tiles
   CUtensorMap tcr = thp, tcz = thp, tcn = thp, tcp = thp;
-  if (LIN) {
-    auto cmap = [&](CUtensorMap* m, const bf16* base) {
-      return make_map2(m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, base, H, (uint64_t)ca.M, H, cellk::CH, BM, CU_TENSOR_MAP_SWIZZLE_32B);
-    };
-    if (!cmap(&tcr, ca.cr) || !cmap(&tcz, ca.cz) || !cmap(&tcn, ca.cn) || (ca.cnp && !cmap(&tcp, ca.cnp))) return false;
-  }
+  auto cmap = [&](CUtensorMap* m, const bf16* base) {
+    return make_map2(m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, base, H, (uint64_t)ca.M, H, cellk::CH, BM, CU_TENSOR_MAP_SWIZZLE_32B);
+  };
+  if (!cmap(&tcr, ca.cr) || !cmap(&tcz, ca.cz) || !cmap(&tcn, ca.cn) || (ca.cnp && !cmap(&tcp, ca.cnp))) return false;
   constexpr int kTileRows = PAIR ? 2 * BM : BM;
   const int tiles = ((ca.M + kTileRows - 1) / kTileRows) * ((H + G::UN - 1) / G::UN);
+  SweepArgs sw{};
+  sw.n_steps = 1;
   ProfScope prof_(kc, 2.0 * ca.M * 3.0 * H * H, s);
   cudaError_t e;
   if (PAIR) {
     const int grid = 2 * (tiles < kSMs / 2 ? tiles : kSMs / 2);
-    e = launch_pdl_cluster(kern, 2, dim3(grid), dim3(cellk::kThreads), C::kSmemBytes, s, ta, tb, tgi, thp, tg, tcr, tcz, tcn, tcp, ca, status);
+    e = launch_pdl_cluster(kern, 2, dim3(grid), dim3(cellk::kThreads), C::kSmemBytes, s, ta, tb, tgi, thp, thp, tcr, tcz, tcn, tcp, ca, sw, status);
   } else {
     const int grid = tiles < kSMs ? tiles : kSMs;
-    e = launch_pdl(kern, dim3(grid), dim3(cellk::kThreads), C::kSmemBytes, s, ta, tb, tgi, thp, tg, tcr, tcz, tcn, tcp, ca, status);
+    e = launch_pdl(kern, dim3(grid), dim3(cellk::kThreads), C::kSmemBytes, s, ta, tb, tgi, thp, thp, tcr, tcz, tcn, tcp, ca, sw, status);
   }
   if (e != cudaSuccess) return false;
   count_launch();
   return true;
 }
-template <bool LIN, bool HAS_G>
-bool launch_cell(int kc, const bf16* A, i64 a_ks, const float* gi, i64 gi_ks, const float* hp, i64 hp_ks, const float* g, i64 g_ks,
-                 int nk, const bf16* W, CellArgs ca, cudaStream_t s) {
-  if (cell_pair_enabled(nk * ca.B, ca.H))
-    return launch_cell_geo<LIN, HAS_G, true>(kc, A, a_ks, gi, gi_ks, hp, hp_ks, g, g_ks, nk, W, ca, s);
-  return launch_cell_geo<LIN, HAS_G, false>(kc, A, a_ks, gi, gi_ks, hp, hp_ks, g, g_ks, nk, W, ca, s);
+bool launch_lin(int kc, const bf16* A, i64 a_ks, const float* gi, i64 gi_ks, const float* hp, i64 hp_ks, int nk, const bf16* W, CellArgs ca,
+                cudaStream_t s) {
+  if (cell_pair_enabled(nk * ca.B, ca.H)) return launch_lin_geo<true>(kc, A, a_ks, gi, gi_ks, hp, hp_ks, nk, W, ca, s);
+  return launch_lin_geo<false>(kc, A, a_ks, gi, gi_ks, hp, hp_ks, nk, W, ca, s);
+}
+
+// Forward steps on the fused kernel: one launch runs sw.n_steps dependent steps over the same rows (k, b), k = 0..nk-1.
+// The state (A: bf16 copy, hp: fp32), the input projection and the additive term are addressed as
+// base + k*ks + slot*ss + b*ld with the slot coordinate taken from each step (nslots = 1: a single step, coordinate 0).
+struct CellFwdOperands {
+  const bf16* A; const float* hp; i64 in_ss, in_ks; int in_slots;
+  const float* gi; i64 gi_ss, gi_ks; const float* g; i64 g_ss, g_ks; int tgt_slots;
+};
+template <bool HAS_G, bool PAIR>
+bool launch_fwd_geo(int kc, const CellFwdOperands& o, int nk, const bf16* W, CellArgs ca, const SweepArgs& sw, cudaStream_t s) {
+  using C = cellk::CellCfg<HAS_G, false, PAIR>;
+  using G = cellk::Geo<PAIR>;
+  if (nk <= 0) return true;
+  int* const status = status_ptr();
+  if (!status) return false;
+  static bool attr_set[kMaxDevices] = {false};
+  auto kern = umma_cell_kernel<false, HAS_G, PAIR>;
+  if (!set_smem_once(kern, C::kSmemBytes, attr_set)) return false;
+  const int B = ca.B, H = ca.H, kt = 128 / B;
+  ca.kt = kt; ca.M = nk * B;
+  CUtensorMap ta, tb, tgi, thp, tg;
+  const auto f32 = CU_TENSOR_MAP_DATA_TYPE_FLOAT32;
+  if (!make_map4(&ta, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, o.A, H, B, o.in_slots, nk, H, o.in_ss, o.in_ks, BK, kt, CU_TENSOR_MAP_SWIZZLE_128B)) return false;
+  if (!make_map(&tb, W, (uint64_t)H, (uint64_t)3 * H, (uint64_t)H, G::kBox)) return false;
+  if (!make_map4(&tgi, f32, 4, o.gi, 3 * H, B, o.tgt_slots, nk, 3 * H, o.gi_ss, o.gi_ks, cellk::CH, kt, CU_TENSOR_MAP_SWIZZLE_64B)) return false;
+  if (!make_map4(&thp, f32, 4, o.hp, H, B, o.in_slots, nk, H, o.in_ss, o.in_ks, cellk::CH, kt, CU_TENSOR_MAP_SWIZZLE_64B)) return false;
+  if (HAS_G) {
+    if (!make_map4(&tg, f32, 4, o.g, H, B, o.tgt_slots, nk, H, o.g_ss, o.g_ks, cellk::CH, kt, CU_TENSOR_MAP_SWIZZLE_64B)) return false;
+  } else {
+    tg = thp;
+  }
+  constexpr int kTileRows = PAIR ? 2 * BM : BM;
+  const int tiles = ((ca.M + kTileRows - 1) / kTileRows) * ((H + G::UN - 1) / G::UN);
+  const i64 items = (i64)tiles * sw.n_steps;
+  ProfScope prof_(kc, 2.0 * ca.M * 3.0 * H * H * sw.n_steps, s);
+  cudaError_t e;
+  if (PAIR) {
+    const int grid = 2 * (int)(items < kSMs / 2 ? items : kSMs / 2);
+    e = launch_pdl_cluster(kern, 2, dim3(grid), dim3(cellk::kThreads), C::kSmemBytes, s, ta, tb, tgi, thp, tg, thp, thp, thp, thp, ca, sw, status);
+  } else {
+    const int grid = (int)(items < kSMs ? items : kSMs);
+    e = launch_pdl(kern, dim3(grid), dim3(cellk::kThreads), C::kSmemBytes, s, ta, tb, tgi, thp, tg, thp, thp, thp, thp, ca, sw, status);
+  }
+  if (e != cudaSuccess) return false;
+  count_launch();
+  return true;
+}
+template <bool HAS_G>
+bool launch_fwd(int kc, const CellFwdOperands& o, int nk, const bf16* W, const CellArgs& ca, const SweepArgs& sw, cudaStream_t s) {
+  if (cell_pair_enabled(nk * ca.B, ca.H)) return launch_fwd_geo<HAS_G, true>(kc, o, nk, W, ca, sw, s);
+  return launch_fwd_geo<HAS_G, false>(kc, o, nk, W, ca, sw, s);
 }
 
 // ---------------------------------------------------------------- epilogues (one output row per thread)
@@ -706,12 +766,18 @@ int umma_fwd_step(const FwdStepArgs& a, UmmaFwdWs* w, cudaStream_t s) {
   if (a.hin_b && 128 % a.B == 0) {
     // operands through strided tensor maps, bf16 copy of the new state written by the epilogue
     CellArgs ca{};
-    ca.B = a.B; ca.H = a.H; ca.hout = a.hout; ca.hout_ks = a.hout_ks; ca.hout_b = a.hout_b;
-    ca.b_hh = a.b_hh; ca.gamma = a.gamma; ca.cell = a.cell; ca.mode = a.mode;
+    ca.B = a.B; ca.H = a.H; ca.b_hh = a.b_hh; ca.gamma = a.gamma; ca.cell = a.cell; ca.mode = a.mode;
     const int nk = a.M / a.B;
-    if (a.mode == 1) ok = launch_cell<false, true>(KC_FWD_STEP, a.hin_b, a.hin_ks, a.gi, a.gi_ks, a.hin, a.hin_ks, a.hout, a.hout_ks, nk, w->W_hh, ca, s);
-    else if (a.gadd) ok = launch_cell<false, true>(KC_FWD_STEP, a.hin_b, a.hin_ks, a.gi, a.gi_ks, a.hin, a.hin_ks, a.gadd, a.gadd_ks, nk, w->W_hh, ca, s);
-    else ok = launch_cell<false, false>(KC_FWD_STEP, a.hin_b, a.hin_ks, a.gi, a.gi_ks, a.hin, a.hin_ks, nullptr, 0, nk, w->W_hh, ca, s);
+    SweepArgs sw{};
+    sw.n_steps = 1;
+    sw.st[0].hout = a.hout; sw.st[0].hout_ks = a.hout_ks; sw.st[0].hout_b = a.hout_b;
+    CellFwdOperands o{};
+    o.A = a.hin_b; o.hp = a.hin; o.in_ks = a.hin_ks; o.in_slots = 1;
+    o.gi = a.gi; o.gi_ks = a.gi_ks; o.tgt_slots = 1;
+    // in mode 1 the previous content of the destination plays the role of the additive term
+    if (a.mode == 1) { o.g = a.hout; o.g_ks = a.hout_ks; }
+    else { o.g = a.gadd; o.g_ks = a.gadd_ks; }
+    ok = o.g ? launch_fwd<true>(KC_FWD_STEP, o, nk, w->W_hh, ca, sw, s) : launch_fwd<false>(KC_FWD_STEP, o, nk, w->W_hh, ca, sw, s);
     return ok ? MGRIT_OK : MGRIT_CUDA_ERROR;
   }
   if (launch_pdl(pack_rows_kernel, dim3(pgrid((i64)a.M * (a.H / 4))), dim3(kPT), 0, s, a.hin, a.hin_ks, a.B, a.H / 4, (i64)a.M,
@@ -719,6 +785,33 @@ int umma_fwd_step(const FwdStepArgs& a, UmmaFwdWs* w, cudaStream_t s) {
     return MGRIT_CUDA_ERROR;
   count_launch();
   ok = launch_gemm<192, true>(KC_FWD_STEP, w->Apack, a.H, w->W_hh, a.H, a.M, a.H, a.H, a.H, 3 * a.H, EpiFwd{a}, s);
+  return ok ? MGRIT_OK : MGRIT_CUDA_ERROR;
+}
+
+// MGRIT_GRU_SWEEP=0 in the environment launches every relaxation step on its own.
+static bool sweep_enabled() {
+  static int v = -1;
+  if (v < 0) { const char* e = getenv("MGRIT_GRU_SWEEP"); v = (e && e[0] == '0') ? 0 : 1; }
+  return v == 1;
+}
+
+int umma_fwd_sweep(const FwdSweepArgs& a, UmmaFwdWs* w, cudaStream_t s) {
+  if (!sweep_enabled() || 128 % a.B != 0 || !a.Ub || a.n < 1 || a.n > kMaxSweepSteps || a.n > kMaxFwdSweepSteps || !a.ctr)
+    return MGRIT_UNSUPPORTED;
+  const i64 BH = (i64)a.B * a.H;
+  CellArgs ca{};
+  ca.B = a.B; ca.H = a.H; ca.b_hh = a.b_hh; ca.gamma = a.gamma; ca.cell = a.cell; ca.mode = 0;
+  SweepArgs sw{};
+  sw.n_steps = a.n; sw.ctr = a.ctr;
+  for (int i = 0; i < a.n; ++i) {
+    sw.st[i].hout = a.st[i].out; sw.st[i].hout_ks = a.st[i].out_ks; sw.st[i].hout_b = a.st[i].out_b;
+    sw.st[i].in_s = a.st[i].in_s; sw.st[i].tgt_s = a.st[i].tgt_s; sw.st[i].dep = i == 0 ? 0 : a.st[i].dep;
+  }
+  CellFwdOperands o{};
+  o.A = a.Ub; o.hp = a.U; o.in_ss = BH; o.in_ks = (i64)a.cf * BH; o.in_slots = a.cf;
+  o.gi = a.gi; o.gi_ss = a.gi_ss; o.gi_ks = a.gi_ks; o.tgt_slots = a.cf;
+  o.g = a.g; o.g_ss = BH; o.g_ks = (i64)a.cf * BH;
+  const bool ok = a.g ? launch_fwd<true>(KC_FWD_STEP, o, a.nk, w->W_hh, ca, sw, s) : launch_fwd<false>(KC_FWD_STEP, o, a.nk, w->W_hh, ca, sw, s);
   return ok ? MGRIT_OK : MGRIT_CUDA_ERROR;
 }
 
@@ -734,15 +827,15 @@ int umma_linearise(const LinArgs& a, UmmaAdjWs* w, cudaStream_t s) {
     ca.a = a.a; ca.cr = a.crb; ca.cz = a.czb; ca.cn = a.cnb; ca.cnp = a.cnpb;
     int done = 0;
     if (a.t0 == 0) {   // step 1 starts from h_0 (its own array)
-      if (!launch_cell<true, false>(KC_LINEARISE, w->hb0, 0, gi0, 0, a.h0, 0, nullptr, 0, 1, w->W_hh, ca, s)) return MGRIT_CUDA_ERROR;
+      if (!launch_lin(KC_LINEARISE, w->hb0, 0, gi0, 0, a.h0, 0, 1, w->W_hh, ca, s)) return MGRIT_CUDA_ERROR;
       done = 1;
     }
     if (N > done) {
       const i64 off = (i64)done * BH;
       ca.a = a.a + off; ca.cr = a.crb + off; ca.cz = a.czb + off; ca.cn = a.cnb + off; ca.cnp = a.cnpb ? a.cnpb + off : nullptr;
       const i64 t1 = a.t0 + (i64)done * a.stride_t;                  // fine time the first of these steps leaves from (>= 1)
-      if (!launch_cell<true, false>(KC_LINEARISE, w->hb0 + t1 * BH, a.stride_t * BH, gi0 + (i64)done * a.stride_t * BH * 3,
-                                    a.stride_t * BH * 3, a.h + (t1 - 1) * BH, a.stride_t * BH, nullptr, 0, N - done, w->W_hh, ca, s))
+      if (!launch_lin(KC_LINEARISE, w->hb0 + t1 * BH, a.stride_t * BH, gi0 + (i64)done * a.stride_t * BH * 3, a.stride_t * BH * 3,
+                      a.h + (t1 - 1) * BH, a.stride_t * BH, N - done, w->W_hh, ca, s))
         return MGRIT_CUDA_ERROR;
     }
     return MGRIT_OK;

@@ -63,6 +63,9 @@ int umma_project_rows(const float* X, __nv_bfloat16* xb, const __nv_bfloat16* Wb
                       cudaStream_t s);
 int umma_adj_dx(const AdjStepArgs& a, const __nv_bfloat16* W_ihT, int C, float* out, UmmaAdjWs* w, cudaStream_t s);
 int umma_fwd_step(const FwdStepArgs& a, UmmaFwdWs* w, cudaStream_t s);
+// all steps of a relaxation sweep in one launch of the fused kernel (needs the bf16 state copies and 128 % B == 0);
+// MGRIT_UNSUPPORTED = not available for this shape (the caller launches the steps one by one)
+int umma_fwd_sweep(const FwdSweepArgs& a, UmmaFwdWs* w, cudaStream_t s);
 int umma_linearise(const LinArgs& a, UmmaAdjWs* w, cudaStream_t s);
 int umma_adj_step(const AdjStepArgs& a, UmmaAdjWs* w, cudaStream_t s);
 int umma_gradients(const mgrit_gru_cfg* c, const gru_params* p, const float* x, const float* h0, const float* h,

@@ -52,3 +52,51 @@ def test_pair_and_single_cta_products_agree(tmp_path):
         assert err <= 1e-5 * scale, (k, err, scale)
         differ += int(err > 0)
     print("outputs that differ at all:", differ, "of", len(a.files))
+
+
+CHILD_SWEEP = r"""
+import sys, numpy as np, torch
+from paper_2203_04738_b200 import binding as B
+from paper_2203_04738_b200.synthetic import Workload, make_inputs
+out = {}
+# (cf, levels, relax_fine, relax_coarse, B, T, flags): FCF and FCFCF sweeps with C-steps, pair and single-CTA geometry,
+# a row count that ends in a partial tile, F-cycles
+cases = [(4, 3, 0, 1, 32, 1024, 0), (4, 3, 1, 2, 16, 512, 0), (2, 4, 1, 1, 8, 272, 0), (8, 2, 1, 1, 32, 512, B.FLAG_F_CYCLE),
+         (4, 2, 2, 0, 4, 96, 0)]
+for i, (cf, L, rf, rc, Bz, T, fl) in enumerate(cases):
+    w = Workload("sweep", T=T, B=Bz, I=64, H=512, cf=cf, levels=L, iters_fwd=2, iters_adj=2, relax_fine=rf, relax_coarse=rc,
+                 operands=2, classes=8, relu=True, seed=40 + i)
+    d = make_inputs(w)
+    p = {n: torch.from_numpy(d["layers"][0][n]).cuda() for n in ("W_ih", "W_hh", "b_ih", "b_hh")}
+    x, h0 = torch.from_numpy(d["x"]).cuda(), torch.from_numpy(d["h0"]).cuda()
+    cfg = B.make_cfg(T, Bz, w.I, w.H, cf=cf, levels=L, iters=2, relax_fine=rf, relax_coarse=rc, operands=B.OPERANDS_BF16, flags=fl)
+    n0 = B.kernel_launches()
+    h, gi, rn = B.mgrit_gru_forward(cfg, p, x, h0, want_resnorm=True)
+    out[f"launches{i}"] = np.array([B.kernel_launches() - n0])
+    out[f"h{i}"] = h.cpu().numpy(); out[f"rn{i}"] = np.array(rn)
+torch.cuda.synchronize()
+assert B.last_device_status() == 0
+np.savez(sys.argv[1], **out)
+"""
+
+
+def test_relaxation_sweeps_in_one_launch_give_the_same_bits(tmp_path):
+    """A relaxation sweep F (CF)^n [+ the evaluation of v] as ONE launch of the fused kernel, tiles of later steps
+    waiting on the row tiles they read, against one launch per step: the arithmetic of every element is the same, so
+    the states must be bit-identical (the residual norms are sums of atomics and agree to rounding); and the sweeps
+    must really have replaced launches."""
+    root = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+    outs = []
+    for flag in ("1", "0"):
+        out = str(tmp_path / f"sweep{flag}.npz")
+        env = dict(os.environ, MGRIT_GRU_SWEEP=flag, PYTHONPATH=root)
+        subprocess.run([sys.executable, "-c", CHILD_SWEEP, out], check=True, env=env, cwd=root, timeout=600)
+        outs.append(np.load(out))
+    a, b = outs
+    for k in a.files:
+        if k.startswith("h"):
+            assert np.array_equal(a[k], b[k]), k
+        elif k.startswith("rn"):
+            assert np.allclose(a[k], b[k], rtol=1e-5), k
+        else:
+            assert a[k][0] < b[k][0], (k, a[k], b[k])
