@@ -308,18 +308,41 @@ def main():
     wall0 = datetime.datetime.now()
     e0.record()
     t_host = time.perf_counter()
+    marks = []                                  # one event after every step: median and best step beside the mean
     for _ in range(args.steps):
         loss = step()
+        marks.append(torch.cuda.Event(enable_timing=True))
+        marks[-1].record()
     host_ms = (time.perf_counter() - t_host) * 1e3 / args.steps     # CPU time to enqueue one step (no sync inside)
     e1.record()
     barrier()
     wall1 = datetime.datetime.now()
     ms = e0.elapsed_time(e1)
+    per_step = sorted(a.elapsed_time(b) for a, b in zip([e0] + marks[:-1], marks))
+    step_stats = {"median_ms": per_step[len(per_step) // 2], "best_ms": per_step[0], "worst_ms": per_step[-1],
+                  "what": "single steps of the timed region (this rank), from an event recorded after every step"}
     launches = graphed.launches * args.steps if graphed is not None else B.kernel_launches() - l0
     windows = {"headline": (wall0, wall1)}      # the clock sampler keeps running through the later legs
     ms = max_over_ranks(ms, dev)
     ms_step = ms / args.steps
     value = job_throughput(T * w.B, ms_step, world)
+
+    # the forward solves alone (projections + MGRIT forward of every layer), host launches
+    fwd_only = None
+    if world == 1 and not args.no_kernel_timing:
+        from paper_2203_04738_b200.train_step import forward_pass
+        for _ in range(3):
+            forward_pass(layers, x, h0, buf)
+        torch.cuda.synchronize()
+        nf = max(3, args.steps // 2)
+        e0.record()
+        for _ in range(nf):
+            forward_pass(layers, x, h0, buf)
+        e1.record()
+        torch.cuda.synchronize()
+        fms = e0.elapsed_time(e1) / nf
+        fwd_only = {"ms_per_step": fms, "value": T * w.B / (fms * 1e-3), "unit": UNIT, "steps": nf,
+                    "what": "input projections + forward solve of every layer only (no head, adjoint, gradients or update)"}
 
     # end to end: inputs start in pinned host memory, the loss is read back, every step
     e2e = None
@@ -488,7 +511,7 @@ def main():
            "ms_per_step": ms_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
            "dtype": OPERAND_DTYPES[w.operands], "data": "synthetic", "config": config, "clocks": clocks,
            "e2e": e2e, "gpu_launches": int(launches), "roofline": roofline, "cpu_baseline": cpu,
-           "gpu_serial": gpu_serial, "t_sweep": t_sweep, "stacked_state": stacked, "roofline_by_class": roofline_by_class,
+           "step_stats": step_stats, "forward_only": fwd_only, "gpu_serial": gpu_serial, "t_sweep": t_sweep, "stacked_state": stacked, "roofline_by_class": roofline_by_class,
            "paper_context": "the paper reports up to 6.5x over serial training on 288 Xeon cores (32 MPI ranks x 9 threads) for T=128; "
                             "another machine and workload: context, not a target",
            "host_enqueue_ms_per_step": host_ms, "kernel_breakdown": breakdown, "kernel_by_size": by_size, "loss": float(loss.item()), "device_status": status}

@@ -142,6 +142,7 @@ struct AdjWs {
   __nv_bfloat16 *crb[kMaxLevels], *czb[kMaxLevels], *cnb[kMaxLevels], *cnpb;       // ... tensor-core engine (bf16)
   float *dA_h, *dA_i, *lam_tmp; double* res_acc; UmmaAdjWs um; Tf32Ws tf;
   __nv_bfloat16* chain_dAb; unsigned* chain_bar; uint4* chain_xw; size_t chain_xw_bytes;
+  float* chain_dA32;        // fp32 chain: [2][B][3H] operand exchange
 };
 
 void plan_fwd(const mgrit_gru_cfg* c, const Hier& hr, Ws& w, FwdWs* o) {
@@ -163,6 +164,8 @@ void plan_fwd(const mgrit_gru_cfg* c, const Hier& hr, Ws& w, FwdWs* o) {
     o->chain_xw = reinterpret_cast<uint4*>(w.take<char>(o->chain_xw_bytes));
     o->sweep_ctr_n = 1 << 16;
     o->sweep_ctr = w.take<int>(o->sweep_ctr_n);
+  } else {
+    o->chain_bar = w.take<unsigned>((size_t)c->B / 16 + 64);
   }
   if (is_tf32(c)) tf32_plan_fwd(c, hr.N, hr.L, w.base, &w.off, &o->tf);
 }
@@ -191,12 +194,15 @@ void plan_adj(const mgrit_gru_cfg* c, const Hier& hr, Ws& w, AdjWs* o) {
   if (c->operands == MGRIT_OPERANDS_BF16) {
     o->dA_h = o->dA_i = o->lam_tmp = nullptr;
     umma_plan_adj(c, hr.N, hr.L, w.base, &w.off, &o->um);
+    o->chain_dA32 = nullptr;
     o->chain_dAb = w.take<__nv_bfloat16>(6 * BH);
     o->chain_bar = w.take<unsigned>(((size_t)c->B / 16 + 1) * ((size_t)c->H / 8) + 64);
     o->chain_xw_bytes = serial_xw_bytes(c->B, c->H, 3);
     o->chain_xw = reinterpret_cast<uint4*>(w.take<char>(o->chain_xw_bytes));
   } else {
-    o->chain_dAb = nullptr; o->chain_bar = nullptr; o->chain_xw = nullptr; o->chain_xw_bytes = 0;
+    o->chain_dAb = nullptr; o->chain_xw = nullptr; o->chain_xw_bytes = 0;
+    o->chain_bar = w.take<unsigned>((size_t)c->B / 16 + 64);
+    o->chain_dA32 = w.take<float>(6 * BH);
     o->dA_h = w.take<float>((size_t)c->T * BH * 3);
     o->dA_i = w.take<float>((size_t)c->T * BH * 3);
     o->lam_tmp = w.take<float>((size_t)c->T * BH);     // lambda in forward order when the caller wants no dh
@@ -307,7 +313,16 @@ struct Cycle {
 struct FwdCycle : Cycle {
   const gru_params* p; const float* gi; UmmaFwdWs* um; FwdWs* fw;
   bool chain(int l) override {
-    if (c->operands != MGRIT_OPERANDS_BF16 || !fw->chain_ub) return false;
+    if (c->operands != MGRIT_OPERANDS_BF16) {     // fp32 and tf32 modes: the chain in FFMA arithmetic
+      if (!fw->chain_bar) return false;
+      Serial32FwdArgs a;
+      a.B = c->B; a.H = c->H; a.nsteps = hr.N[l]; a.u = U[l];
+      const i64 st = hr.stride_t[l];
+      a.gi = gi + (st - 1) * (i64)BH * 3; a.gi_step = st * (i64)BH * 3;
+      a.g = G[l]; a.W = p->W_hh; a.b_hh = p->b_hh; a.gamma = hr.gamma[l]; a.cell = c->cell; a.bar = fw->chain_bar;
+      return serial32_fwd_solve(a, s);
+    }
+    if (!fw->chain_ub) return false;
     SerialFwdArgs a;
     a.B = c->B; a.H = c->H; a.nsteps = hr.N[l];
     a.u = U[l]; a.ub = fw->chain_ub;
@@ -374,7 +389,17 @@ struct FwdCycle : Cycle {
 struct AdjCycle : Cycle {
   const gru_params* p; AdjWs* w;
   bool chain(int l) override {
-    if (c->operands != MGRIT_OPERANDS_BF16 || !w->chain_dAb) return false;
+    if (c->operands != MGRIT_OPERANDS_BF16) {
+      if (!w->chain_bar || !w->chain_dA32) return false;
+      Serial32AdjArgs a;
+      a.B = c->B; a.H = c->H; a.nsteps = hr.N[l]; a.mu = U[l]; a.dA = w->chain_dA32;
+      const i64 row0 = (i64)(hr.N[l] - 1) * BH;    // step s = 1 applies forward step N_l, stored at row N_l - 1
+      a.a = w->a[l] + row0; a.cr = w->cr[l] + row0; a.cz = w->cz[l] + row0; a.cn = w->cn[l] + row0;
+      a.coef_step = -(i64)BH;
+      a.g = G[l]; a.W = p->W_hh; a.bar = w->chain_bar;
+      return serial32_adj_solve(a, s);
+    }
+    if (!w->chain_dAb) return false;
     SerialAdjArgs a;
     a.B = c->B; a.H = c->H; a.nsteps = hr.N[l];
     a.mu = U[l]; a.dAb = w->chain_dAb;

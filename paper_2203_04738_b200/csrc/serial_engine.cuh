@@ -32,6 +32,31 @@ struct SerialAdjArgs {
   uint4* xw; size_t xw_bytes;    // as in SerialFwdArgs (three gate blocks per producer)
 };
 
+// The same chains in fp32 arithmetic (FFMA, precise gate math) for the fp32 and tf32 operand modes: fp32 weights in
+// shared memory, the fp32 state itself crosses CTAs (counter barrier + reload).
+struct Serial32FwdArgs {
+  int B, H, nsteps;
+  float* u;                      // level state; slots 1..nsteps are written
+  const float* gi; i64 gi_step;
+  const float* g;
+  const float* W;                // [3H][H] fp32
+  const float* b_hh;
+  float gamma; int cell;
+  unsigned* bar;                 // [ceil(B/16)] barrier counters (scratch)
+};
+struct Serial32AdjArgs {
+  int B, H, nsteps;
+  float* mu;
+  float* dA;                     // [2][B][3H] scratch: [cr|cz|cn] of the next step times the newest mu
+  const float *a, *cr, *cz, *cn; // coefficient rows of step 1; step s at + (s-1)*coef_step
+  i64 coef_step;
+  const float* g;
+  const float* W;                // [3H][H] fp32 (W_hh as given)
+  unsigned* bar;
+};
+bool serial32_fwd_solve(const Serial32FwdArgs& a, cudaStream_t s);
+bool serial32_adj_solve(const Serial32AdjArgs& a, cudaStream_t s);
+
 // bytes of exchange words for a chain over B rows of H units carrying `gates` values per (row, unit)
 size_t serial_xw_bytes(int B, int H, int gates);
 

@@ -428,6 +428,220 @@ __global__ void __launch_bounds__(kThreads, 1) serial_adj_kernel(SerialAdjArgs a
   }
 }
 
+// ================================================================================================
+// fp32 chains: the same two recurrences in FFMA arithmetic with precise gate math.  K is split over the 8 warps; a
+// lane owns 4 rows x CPL columns of the 16 x (8 CPL) outputs (the 8 lanes of a quarter warp read the same A words --
+// a broadcast -- and W rows 3 CPL (H + 4) floats apart: conflict-free 16-byte loads).
+template <int CPL>
+__device__ __forceinline__ void warp_gemm32(const float* As, const float* Ws, int ldk, int kbeg, int kend, float (*acc)[CPL]) {
+  const int lane = threadIdx.x & 31, rq = lane >> 3, cq = lane & 7;
+  const float* ar = As + (rq * 4) * ldk;
+  const float* wr = Ws + (cq * CPL) * ldk;
+  for (int k = kbeg; k < kend; k += 4) {
+    float4 av[4], wv[CPL];
+#pragma unroll
+    for (int r = 0; r < 4; ++r) av[r] = *reinterpret_cast<const float4*>(ar + r * ldk + k);
+#pragma unroll
+    for (int c = 0; c < CPL; ++c) wv[c] = *reinterpret_cast<const float4*>(wr + c * ldk + k);
+#pragma unroll
+    for (int r = 0; r < 4; ++r)
+#pragma unroll
+      for (int c = 0; c < CPL; ++c)
+        acc[r][c] = fmaf(av[r].x, wv[c].x, fmaf(av[r].y, wv[c].y, fmaf(av[r].z, wv[c].z, fmaf(av[r].w, wv[c].w, acc[r][c]))));
+  }
+}
+// warp partial sums -> red[warp][row][col]   (col < 8 CPL)
+template <int CPL>
+__device__ __forceinline__ void store_partials32(float* red, float (*acc)[CPL]) {
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31, rq = lane >> 3, cq = lane & 7;
+  constexpr int NC = 8 * CPL;
+  float* base = red + warp * kRows * NC;
+#pragma unroll
+  for (int r = 0; r < 4; ++r)
+#pragma unroll
+    for (int c = 0; c < CPL; ++c) base[(rq * 4 + r) * NC + cq * CPL + c] = acc[r][c];
+}
+
+// forward:  u_j = Phi_gamma(gi_j, u_{j-1}) + g_j ;  the CTA owns UNC hidden units (3 UNC weight rows)
+template <int UNC>
+__global__ void __launch_bounds__(kThreads, 1) serial32_fwd_kernel(Serial32FwdArgs a, int* status) {
+  constexpr int NW = 3 * UNC, CPL = NW / 8, OPT = (kRows * UNC + kThreads - 1) / kThreads;
+  extern __shared__ __align__(16) uint8_t smem[];
+  const int H = a.H, ldk = H + 4;
+  float* Ws = reinterpret_cast<float*>(smem);   // [NW][ldk]
+  float* As = Ws + NW * ldk;                    // [16][ldk]
+  float* red = As + kRows * ldk;                // [8][16][NW]
+  __shared__ int ok_smem;
+  const int tid = threadIdx.x, warp = tid >> 5;
+  const int u0 = blockIdx.x * UNC, rg = blockIdx.y, row0 = rg * kRows;
+  const int nrows = min(kRows, a.B - row0);
+  const unsigned ncta_rg = gridDim.x;
+  const i64 BH = (i64)a.B * H;
+
+  for (int e = tid; e < NW * (H / 4); e += kThreads) {
+    int r = e / (H / 4), c = e % (H / 4);
+    int gate = r / UNC, i = r % UNC;
+    *reinterpret_cast<float4*>(Ws + r * ldk + c * 4) = __ldg(reinterpret_cast<const float4*>(a.W + ((i64)gate * H + u0 + i) * H + c * 4));
+  }
+  for (int e = tid; e < kRows * ldk; e += kThreads) As[e] = 0.f;     // rows beyond the batch stay zero
+  if (tid == 0) ok_smem = 1;
+  __syncthreads();
+  for (int e = tid; e < nrows * (H / 4); e += kThreads) {
+    int r = e / (H / 4), c = e % (H / 4);
+    *reinterpret_cast<float4*>(As + r * ldk + c * 4) = __ldcg(reinterpret_cast<const float4*>(a.u + (i64)(row0 + r) * H + c * 4));
+  }
+  float hp[OPT], pgr[OPT], pgz[OPT], pgn[OPT], pg[OPT], br[OPT], bz[OPT], bn[OPT];
+#pragma unroll
+  for (int o = 0; o < OPT; ++o) {
+    int idx = tid + o * kThreads, r = idx / UNC, i = idx % UNC;
+    bool v = idx < kRows * UNC && r < nrows;
+    hp[o] = v ? __ldcg(a.u + (i64)(row0 + r) * H + u0 + i) : 0.f;
+    br[o] = a.b_hh[u0 + i]; bz[o] = a.b_hh[H + u0 + i]; bn[o] = a.b_hh[2 * H + u0 + i];
+    const float* gi = a.gi + (i64)(row0 + r) * 3 * H + u0 + i;
+    pgr[o] = v ? gi[0] : 0.f; pgz[o] = v ? gi[H] : 0.f; pgn[o] = v ? gi[2 * H] : 0.f;
+    pg[o] = (v && a.g) ? a.g[BH + (i64)(row0 + r) * H + u0 + i] : 0.f;
+  }
+  __syncthreads();
+
+  const int kw = H / kWarps;
+  for (int j = 1; j <= a.nsteps; ++j) {
+    float acc[4][CPL];
+#pragma unroll
+    for (int r = 0; r < 4; ++r)
+#pragma unroll
+      for (int c = 0; c < CPL; ++c) acc[r][c] = 0.f;
+    warp_gemm32<CPL>(As, Ws, ldk, warp * kw, (warp + 1) * kw, acc);
+    store_partials32<CPL>(red, acc);
+    __syncthreads();
+#pragma unroll
+    for (int o = 0; o < OPT; ++o) {
+      int idx = tid + o * kThreads, r = idx / UNC, i = idx % UNC;
+      if (idx < kRows * UNC && r < nrows) {
+        float ghr = sum_partials<NW>(red, r, i) + br[o];
+        float ghz = sum_partials<NW>(red, r, UNC + i) + bz[o];
+        float ghn = sum_partials<NW>(red, r, 2 * UNC + i) + bn[o];
+        float val = cell_forward<false>(pgr[o], pgz[o], pgn[o], ghr, ghz, ghn, hp[o], a.gamma, a.cell) + pg[o];
+        hp[o] = val;
+        a.u[(i64)j * BH + (i64)(row0 + r) * H + u0 + i] = val;
+      }
+    }
+    if (j == a.nsteps) break;
+#pragma unroll
+    for (int o = 0; o < OPT; ++o) {   // operands of the next step that do not depend on other CTAs
+      int idx = tid + o * kThreads, r = idx / UNC, i = idx % UNC;
+      if (idx < kRows * UNC && r < nrows) {
+        const float* gi = a.gi + (i64)j * a.gi_step + (i64)(row0 + r) * 3 * H + u0 + i;
+        pgr[o] = gi[0]; pgz[o] = gi[H]; pgn[o] = gi[2 * H];
+        if (a.g) pg[o] = a.g[(i64)(j + 1) * BH + (i64)(row0 + r) * H + u0 + i];
+      }
+    }
+    if (!grid_barrier(a.bar + rg, (unsigned)j * ncta_rg, status, &ok_smem)) return;
+    const float* uj = a.u + (i64)j * BH;     // the full new state of this row group
+    for (int e = tid; e < nrows * (H / 4); e += kThreads) {
+      int r = e / (H / 4), c = e % (H / 4);
+      cp_async16(As + r * ldk + c * 4, uj + (i64)(row0 + r) * H + c * 4);
+    }
+    cp_async_wait_all();
+    __syncthreads();
+  }
+}
+
+// adjoint:  mu_s = a_s mu_{s-1} + ([cr|cz|cn]_s mu_{s-1}) W_hh + g_s ;  the CTA owns UNC output units (columns of W_hh)
+template <int UNC>
+__global__ void __launch_bounds__(kThreads, 1) serial32_adj_kernel(Serial32AdjArgs a, int* status) {
+  constexpr int CPL = UNC / 8, OPT = (kRows * UNC + kThreads - 1) / kThreads;
+  extern __shared__ __align__(16) uint8_t smem[];
+  const int H = a.H, K = 3 * H, ldk = K + 4;
+  float* Ws = reinterpret_cast<float*>(smem);   // [UNC][ldk]: Ws[n][k] = W_hh[k][u0 + n]
+  float* As = Ws + UNC * ldk;                   // [16][ldk]
+  float* red = As + kRows * ldk;                // [8][16][UNC]
+  __shared__ int ok_smem;
+  const int tid = threadIdx.x, warp = tid >> 5;
+  const int u0 = blockIdx.x * UNC, rg = blockIdx.y, row0 = rg * kRows;
+  const int nrows = min(kRows, a.B - row0);
+  const unsigned ncta_rg = gridDim.x;
+  const i64 BH = (i64)a.B * H;
+
+  for (int e = tid; e < K * UNC; e += kThreads) {
+    int k = e / UNC, n = e % UNC;
+    Ws[n * ldk + k] = __ldg(a.W + (i64)k * H + u0 + n);
+  }
+  for (int e = tid; e < kRows * ldk; e += kThreads) As[e] = 0.f;
+  if (tid == 0) ok_smem = 1;
+  __syncthreads();
+  for (int e = tid; e < nrows * H; e += kThreads) {     // step 1: dA_1 = c_1 * mu_0
+    int r = e / H, i = e % H;
+    i64 off = (i64)(row0 + r) * H + i;
+    float m = __ldcg(a.mu + off);
+    As[r * ldk + i] = a.cr[off] * m;
+    As[r * ldk + H + i] = a.cz[off] * m;
+    As[r * ldk + 2 * H + i] = a.cn[off] * m;
+  }
+  float mp[OPT], pa[OPT], pg[OPT], ncr[OPT], ncz[OPT], ncn[OPT];
+#pragma unroll
+  for (int o = 0; o < OPT; ++o) {
+    int idx = tid + o * kThreads, r = idx / UNC, i = idx % UNC;
+    bool v = idx < kRows * UNC && r < nrows;
+    i64 off = (i64)(row0 + r) * H + u0 + i;
+    mp[o] = v ? __ldcg(a.mu + off) : 0.f;
+    pa[o] = v ? a.a[off] : 0.f;
+    pg[o] = (v && a.g) ? a.g[BH + off] : 0.f;
+    bool more = v && a.nsteps > 1;
+    ncr[o] = more ? a.cr[a.coef_step + off] : 0.f;
+    ncz[o] = more ? a.cz[a.coef_step + off] : 0.f;
+    ncn[o] = more ? a.cn[a.coef_step + off] : 0.f;
+  }
+  __syncthreads();
+
+  const int kw = K / kWarps;
+  for (int s = 1; s <= a.nsteps; ++s) {
+    float acc[4][CPL];
+#pragma unroll
+    for (int r = 0; r < 4; ++r)
+#pragma unroll
+      for (int c = 0; c < CPL; ++c) acc[r][c] = 0.f;
+    warp_gemm32<CPL>(As, Ws, ldk, warp * kw, (warp + 1) * kw, acc);
+    store_partials32<CPL>(red, acc);
+    __syncthreads();
+    float* dA = a.dA + (i64)(s & 1) * 3 * BH;
+#pragma unroll
+    for (int o = 0; o < OPT; ++o) {
+      int idx = tid + o * kThreads, r = idx / UNC, i = idx % UNC;
+      if (idx < kRows * UNC && r < nrows) {
+        float val = pa[o] * mp[o] + sum_partials<UNC>(red, r, i) + pg[o];
+        mp[o] = val;
+        i64 off = (i64)(row0 + r) * H + u0 + i;
+        a.mu[(i64)s * BH + off] = val;
+        if (s < a.nsteps) {
+          float* d = dA + (i64)(row0 + r) * K + u0 + i;
+          d[0] = ncr[o] * val; d[H] = ncz[o] * val; d[2 * H] = ncn[o] * val;
+        }
+      }
+    }
+    if (s == a.nsteps) break;
+#pragma unroll
+    for (int o = 0; o < OPT; ++o) {
+      int idx = tid + o * kThreads, r = idx / UNC, i = idx % UNC;
+      if (idx < kRows * UNC && r < nrows) {
+        i64 off = (i64)(row0 + r) * H + u0 + i;
+        pa[o] = a.a[(i64)s * a.coef_step + off];
+        if (a.g) pg[o] = a.g[(i64)(s + 1) * BH + off];
+        if (s + 1 < a.nsteps) {
+          i64 co = (i64)(s + 1) * a.coef_step + off;
+          ncr[o] = a.cr[co]; ncz[o] = a.cz[co]; ncn[o] = a.cn[co];
+        }
+      }
+    }
+    if (!grid_barrier(a.bar + rg, (unsigned)s * ncta_rg, status, &ok_smem)) return;
+    for (int e = tid; e < nrows * (K / 4); e += kThreads) {
+      int r = e / (K / 4), c = e % (K / 4);
+      cp_async16(As + r * ldk + c * 4, dA + (i64)(row0 + r) * K + c * 4);
+    }
+    cp_async_wait_all();
+    __syncthreads();
+  }
+}
+
 int* status_ptr() {     // status word of the current device, nullptr on failure
   const int dev = current_device_slot();
   if (dev < 0) return nullptr;
@@ -501,6 +715,38 @@ bool launch_coop(Kern kern, const Args& a, int unc, size_t smem, bool ll, int ga
   return true;
 }
 
+// ---- fp32 chains
+size_t fwd32_smem(int unc, int H) { return ((size_t)(3 * unc + kRows) * (H + 4) + (size_t)kWarps * kRows * 3 * unc) * 4; }
+size_t adj32_smem(int unc, int H) { return ((size_t)(unc + kRows) * (3 * H + 4) + (size_t)kWarps * kRows * unc) * 4; }
+int pick_unc32(int B, int H, bool adj) {
+  if (H % 32 != 0) return 0;                   // K split over 8 warps in steps of four
+  const int rgs = (B + kRows - 1) / kRows;
+  const int cands[2] = {8, 16};
+  for (int c : cands) {
+    if (H % c != 0) continue;
+    if ((i64)(H / c) * rgs > sm_count()) continue;
+    if ((adj ? adj32_smem(c, H) : fwd32_smem(c, H)) > kSmemLimit) continue;
+    return c;
+  }
+  return 0;
+}
+template <class Args, class Kern>
+bool launch_coop32(Kern kern, const Args& a, int unc, size_t smem, cudaStream_t s) {
+  if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess) return false;
+  const int rgs = (a.B + kRows - 1) / kRows;
+  if (cudaMemsetAsync(a.bar, 0, sizeof(unsigned) * rgs, s) != cudaSuccess) return false;
+  Args args = a;
+  int* st = status_ptr();
+  if (!st) return false;
+  void* params[2] = {(void*)&args, (void*)&st};
+  if (cudaLaunchCooperativeKernel((const void*)kern, dim3(a.H / unc, rgs), dim3(kThreads), params, smem, s) != cudaSuccess) {
+    cudaGetLastError();
+    return false;
+  }
+  count_launch();
+  return true;
+}
+
 }  // namespace
 
 size_t serial_xw_bytes(int B, int H, int gates) {
@@ -540,6 +786,33 @@ bool serial_adj_solve(const SerialAdjArgs& a, cudaStream_t s) {
                : (unc == 8 ? launch_coop(serial_adj_kernel<8, false>, a, unc, smem, false, 3, s)
                   : unc == 16 ? launch_coop(serial_adj_kernel<16, false>, a, unc, smem, false, 3, s)
                               : launch_coop(serial_adj_kernel<32, false>, a, unc, smem, false, 3, s));
+  prof_end(s);
+  return ok;
+}
+
+// MGRIT_GRU_CHAIN32=0 in the environment advances the fp32 / tf32 modes' coarsest level step by step instead.
+static bool chain32_enabled() {
+  static int v = -1;
+  if (v < 0) { const char* e = getenv("MGRIT_GRU_CHAIN32"); v = (e && e[0] == '0') ? 0 : 1; }
+  return v == 1;
+}
+
+bool serial32_fwd_solve(const Serial32FwdArgs& a, cudaStream_t s) {
+  const int unc = chain32_enabled() ? pick_unc32(a.B, a.H, false) : 0;
+  if (unc == 0 || a.nsteps <= 0 || !a.bar || !status_ptr()) return false;
+  const size_t smem = fwd32_smem(unc, a.H);
+  prof_begin(KC_FWD_SERIAL, 2.0 * a.B * 3.0 * a.H * a.H * a.nsteps, s);
+  const bool ok = unc == 8 ? launch_coop32(serial32_fwd_kernel<8>, a, unc, smem, s) : launch_coop32(serial32_fwd_kernel<16>, a, unc, smem, s);
+  prof_end(s);
+  return ok;
+}
+
+bool serial32_adj_solve(const Serial32AdjArgs& a, cudaStream_t s) {
+  const int unc = chain32_enabled() ? pick_unc32(a.B, a.H, true) : 0;
+  if (unc == 0 || a.nsteps <= 0 || !a.bar || !a.dA || !status_ptr()) return false;
+  const size_t smem = adj32_smem(unc, a.H);
+  prof_begin(KC_ADJ_SERIAL, 2.0 * a.B * 3.0 * a.H * a.H * a.nsteps, s);
+  const bool ok = unc == 8 ? launch_coop32(serial32_adj_kernel<8>, a, unc, smem, s) : launch_coop32(serial32_adj_kernel<16>, a, unc, smem, s);
   prof_end(s);
   return ok;
 }

@@ -395,7 +395,8 @@ struct EpiStore {  // out[m, n] = acc            (weight / input gradients)
   }
 };
 
-struct EpiFwd {  // GRU cell on the r|z|n accumulator columns of 64 hidden units
+template <bool FAST = true>
+struct EpiFwd {  // GRU cell on the r|z|n accumulator columns of 64 hidden units (FAST: MUFU gate math of the bf16 mode)
   FwdStepArgs a;
   __device__ void operator()(uint32_t taddr, int row, int u0, int half) const {
     const bool valid = row < a.M;
@@ -432,7 +433,7 @@ struct EpiFwd {  // GRU cell on the r|z|n accumulator columns of 64 hidden units
           float o[4];
 #pragma unroll
           for (int e = 0; e < 4; ++e) {
-            float phi = cell_forward<true>(f4get(gr[i], e), f4get(gz[i], e), f4get(gn[i], e), r[4 * i + e] + f4get(br, e),
+            float phi = cell_forward<FAST>(f4get(gr[i], e), f4get(gz[i], e), f4get(gn[i], e), r[4 * i + e] + f4get(br, e),
                                      z[4 * i + e] + f4get(bz, e), n[4 * i + e] + f4get(bn, e), f4get(h4[i], e), a.gamma, a.cell);
             // mode 0: phi + g ;  mode 1: previous - phi
             o[e] = a.mode == 1 ? f4get(g4[i], e) - phi : phi + f4get(g4[i], e);
@@ -445,7 +446,8 @@ struct EpiFwd {  // GRU cell on the r|z|n accumulator columns of 64 hidden units
 };
 
 template <bool BF16C = true>
-struct EpiLin {  // adjoint coefficients of every step of a level (gate coefficients stored in bf16, or in fp32)
+struct EpiLin {  // adjoint coefficients of every step of a level: bf16 mode (MUFU gate math, gate coefficients stored in bf16)
+                 // or tf32 modes (precise gate math, fp32 coefficients)
   LinArgs a;
   __device__ void operator()(uint32_t taddr, int row, int u0, int half) const {
     const bool valid = row < a.M;
@@ -480,7 +482,7 @@ struct EpiLin {  // adjoint coefficients of every step of a level (gate coeffici
           float oa[4], ocr[4], ocz[4], ocn[4], ocp[4];
 #pragma unroll
           for (int e = 0; e < 4; ++e) {
-            CellLin L = cell_linearise<true>(f4get(gr[i], e), f4get(gz[i], e), f4get(gn[i], e), r[4 * i + e] + f4get(br, e),
+            CellLin L = cell_linearise<BF16C>(f4get(gr[i], e), f4get(gz[i], e), f4get(gn[i], e), r[4 * i + e] + f4get(br, e),
                                        z[4 * i + e] + f4get(bz, e), n[4 * i + e] + f4get(bn, e), f4get(h4[i], e), a.gamma, a.cell);
             oa[e] = L.a; ocr[e] = L.cr; ocz[e] = L.cz; ocn[e] = L.cn; ocp[e] = L.cnp;
           }
@@ -784,7 +786,7 @@ int umma_fwd_step(const FwdStepArgs& a, UmmaFwdWs* w, cudaStream_t s) {
                  reinterpret_cast<uint2*>(w->Apack)) != cudaSuccess)
     return MGRIT_CUDA_ERROR;
   count_launch();
-  ok = launch_gemm<192, true>(KC_FWD_STEP, w->Apack, a.H, w->W_hh, a.H, a.M, a.H, a.H, a.H, 3 * a.H, EpiFwd{a}, s);
+  ok = launch_gemm<192, true>(KC_FWD_STEP, w->Apack, a.H, w->W_hh, a.H, a.M, a.H, a.H, a.H, 3 * a.H, EpiFwd<true>{a}, s);
   return ok ? MGRIT_OK : MGRIT_CUDA_ERROR;
 }
 
@@ -1102,7 +1104,7 @@ int tf32_fwd_step(const FwdStepArgs& a, Tf32Ws* w, cudaStream_t s) {
   const int S = w->S;
   if (!split_rows(a.hin, a.hin_ks, a.B, a.H, a.M, S, false, w->Apack, s)) return MGRIT_CUDA_ERROR;
   return launch_gemm<192, true>(KC_FWD_STEP, (const float*)w->Apack, (i64)S * a.H, (const float*)w->W_hh, (i64)S * a.H, a.M, a.H, S * a.H, a.H,
-                                3 * a.H, EpiFwd{a}, s) ? MGRIT_OK : MGRIT_CUDA_ERROR;
+                                3 * a.H, EpiFwd<false>{a}, s) ? MGRIT_OK : MGRIT_CUDA_ERROR;
 }
 
 int tf32_prepare_adj(const mgrit_gru_cfg* c, const gru_params* p, Tf32Ws* w, cudaStream_t s) {

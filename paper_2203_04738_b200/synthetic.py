@@ -29,7 +29,7 @@ class Workload:
     iters_adj: int
     relax_fine: int          # 0 = F, 1 = FCF
     relax_coarse: int
-    operands: int            # 0 = fp32, 2 = bf16 tensor-core operands
+    operands: int            # 0 = fp32 FFMA, 1 = tf32 three-term split, 2 = bf16, 3 = tf32 single pass (tensor-core operands)
     classes: int
     relu: bool
     layers: int = 1
@@ -41,8 +41,9 @@ class Workload:
 WORKLOADS = {
     "tiny": Workload("tiny", T=64, B=2, I=16, H=32, cf=4, levels=2, iters_fwd=2, iters_adj=2,
                      relax_fine=0, relax_coarse=1, operands=0, classes=8, relu=False, seed=0),
+    # fp32 state at fp32 tolerances; the products run on the tensor cores as three-term tf32 splits (operands = 1)
     "clip": Workload("clip", T=128, B=16, I=512, H=256, cf=4, levels=2, iters_fwd=2, iters_adj=2,
-                     relax_fine=1, relax_coarse=1, operands=0, classes=51, relu=True, seed=1),
+                     relax_fine=1, relax_coarse=1, operands=1, classes=51, relu=True, seed=1),
     "medium": Workload("medium", T=1024, B=32, I=1024, H=512, cf=4, levels=3, iters_fwd=2, iters_adj=2,
                        relax_fine=0, relax_coarse=1, operands=2, classes=51, relu=True, seed=2),
     "long": Workload("long", T=4096, B=8, I=2048, H=1024, cf=8, levels=4, iters_fwd=3, iters_adj=3,

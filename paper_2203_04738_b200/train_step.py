@@ -107,17 +107,22 @@ def all_params(layers, W_c, b_c):
     return out + [W_c, b_c]
 
 
+def forward_pass(layers, x, h0, buf: StepBuffers):
+    """Input projection + forward solve of every layer (MGRIT, or the serial sweep when the buffers say so); returns
+    the top layer's states (device, owned by buf)."""
+    inp = x
+    for l, p in enumerate(layers):
+        fn = B.gru_serial_forward if buf.serial else B.mgrit_gru_forward
+        fn(buf.cfgs_fwd[l], p, inp, h0, gi=buf.gi[l], h=buf.h[l], ws=buf.ws_fwd)
+        inp = buf.h[l]
+    return inp
+
+
 def training_step(w: Workload, layers, W_c, b_c, x, h0, labels, buf: StepBuffers, lr: float = 1e-3, update: bool = True,
                   adam: AdamState | None = None):
     """Forward (all layers) -> loss head -> adjoint (top layer first) -> weight gradients -> SGD (or Adam when an
     AdamState is given).  layers: list of dicts W_ih, W_hh, b_ih, b_hh (device fp32).  Returns the loss (device)."""
-    inp = x
-    for l, p in enumerate(layers):
-        if buf.serial:
-            B.gru_serial_forward(buf.cfgs_fwd[l], p, inp, h0, gi=buf.gi[l], h=buf.h[l], ws=buf.ws_fwd)
-        else:
-            B.mgrit_gru_forward(buf.cfgs_fwd[l], p, inp, h0, gi=buf.gi[l], h=buf.h[l], ws=buf.ws_fwd)
-        inp = buf.h[l]
+    forward_pass(layers, x, h0, buf)
     loss, dhT, dWc, dbc = B.xent_head_fwd_bwd(buf.h[-1][-1], W_c, b_c, labels, ws=buf.ws_head)
     seed = None
     for l in range(len(layers) - 1, -1, -1):
