@@ -91,7 +91,8 @@ typedef struct {
                            fp32 accumulation and fp32 everything else: meets the fp32 tolerances;
                            MGRIT_OPERANDS_TF32_1PASS: operands rounded to tf32 once (10 mantissa bits).
                            The tf32 modes need H % 64 == 0, I % 16 == 0, (T*B) % 4 == 0 and serve the
-                           mgrit_gru_* / gru_serial_* / gru_input_projection calls of one layer. */
+                           mgrit_gru_* / gru_serial_* / gru_input_projection calls of one layer and the
+                           mgrit_lstm_* calls (not the stacked-state calls). */
   int32_t flags;        /* OR of MGRIT_FLAG_*.  MGRIT_FLAG_SKIP_DUPLICATE_FRELAX: a cycle after the first starts
                            from C-points whose F-points the previous cycle's final F-relaxation already filled;
                            skip re-doing it (results are identical) */
@@ -192,7 +193,8 @@ int mgrit_gru_stack_adjoint(const mgrit_gru_cfg* cfg, int32_t n_layers, const gr
  *   The state of a time point is (c, h): u0[2,B,H], u[T,2,B,H], du_seed / du likewise; gi[T,B,4H].
  *   dhT[B,H]: loss derivative w.r.t. the last HIDDEN state.  grads: one gru_grads with the 4H-row shapes.
  *   Everything else (cycles, relaxation, flags, resnorm, levels == 1 = serial sweep / exact BPTT) as for the GRU calls.
- *   Operand mode MGRIT_OPERANDS_FP32 only (others: MGRIT_UNSUPPORTED). */
+ *   Operand modes MGRIT_OPERANDS_FP32 (FFMA) and the tf32 modes (tcgen05 products on four-gate tiles of 64 hidden
+ *   units; same shape limits as for the GRU); MGRIT_OPERANDS_BF16: MGRIT_UNSUPPORTED. */
 int mgrit_lstm_workspace_bytes(const mgrit_gru_cfg* cfg, size_t* fwd_bytes, size_t* adj_bytes);
 int mgrit_lstm_forward(const mgrit_gru_cfg* cfg, const gru_params* p, const float* x, const float* u0, float* gi, float* u,
                        float* resnorm, void* ws, size_t ws_bytes, mgrit_stream_t stream);

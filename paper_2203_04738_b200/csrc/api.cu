@@ -946,11 +946,11 @@ int stack_adjoint_impl(const mgrit_gru_cfg* cfg, int nl, const gru_params* p, co
 // ======================================================================================================
 // Implicit LSTM: the state of a time point is (c, h); level arrays are [N_l + 1][2][B][H] (part 0 = c, part 1 = h) and
 // the same Cycle drives them.  fp32 engine only (four-gate FFMA products).
-struct LstmFwdWs { float* U[kMaxLevels]; float* G[kMaxLevels]; double* res_acc; float *tmpC, *tmpH; size_t maxM; };
+struct LstmFwdWs { float* U[kMaxLevels]; float* G[kMaxLevels]; double* res_acc; float *tmpC, *tmpH; size_t maxM; Tf32Ws tf; };
 struct LstmAdjWs {
   float* U[kMaxLevels]; float* G[kMaxLevels]; double* res_acc;
   float *a[kMaxLevels], *p[kMaxLevels], *ci[kMaxLevels], *cf[kMaxLevels], *cg[kMaxLevels], *co[kMaxLevels];
-  float *tmpC, *tmpH, *hk, *dA; size_t maxM;
+  float *tmpC, *tmpH, *hk, *dA; size_t maxM; Tf32Ws tf;
 };
 
 void plan_lstm_fwd(const mgrit_gru_cfg* c, const Hier& hr, Ws& w, LstmFwdWs* o) {
@@ -963,6 +963,7 @@ void plan_lstm_fwd(const mgrit_gru_cfg* c, const Hier& hr, Ws& w, LstmFwdWs* o) 
   o->maxM = stack_max_rows(c, hr);
   o->tmpC = w.take<float>(o->maxM * c->H);
   o->tmpH = w.take<float>(o->maxM * c->H);
+  if (is_tf32(c)) tf32_plan_fwd(c, hr.N, hr.L, w.base, &w.off, &o->tf, 4);
 }
 
 void plan_lstm_adj(const mgrit_gru_cfg* c, const Hier& hr, Ws& w, LstmAdjWs* o) {
@@ -980,6 +981,7 @@ void plan_lstm_adj(const mgrit_gru_cfg* c, const Hier& hr, Ws& w, LstmAdjWs* o) 
   o->tmpH = w.take<float>(o->maxM * c->H);
   o->hk = w.take<float>(TB * c->H);
   o->dA = w.take<float>(TB * 4 * c->H);
+  if (is_tf32(c)) tf32_plan_adj(c, hr.N, hr.L, w.base, &w.off, &o->tf, 4);
 }
 
 struct LstmFwdCycle : Cycle {
@@ -993,7 +995,8 @@ struct LstmFwdCycle : Cycle {
     a.cout = fw->tmpC; a.hout = fw->tmpH;
     a.gi = gi + ((i64)st * d.tgt_slot - 1) * (i64)bh * 4; a.gi_ks = st * d.tgt_stride * (i64)bh * 4;
     a.W_hh = p->W_hh; a.b_hh = p->b_hh; a.gamma = hr.gamma[d.l]; a.cell = c->cell;
-    simt_lstm_fwd_step(a, s);
+    if (is_tf32(c)) { int r = tf32_lstm_fwd_step(a, &fw->tf, s); if (r) return r; }
+    else simt_lstm_fwd_step(a, s);
     for (int part = 0; part < 2; ++part) {
       const float* g = d.gadd ? d.gadd + (size_t)d.gadd_slot * slot + part * bh : nullptr;
       stream_combine_rows(part == 0 ? fw->tmpC : fw->tmpH, g, (i64)d.gadd_stride * slot, d.out + (size_t)d.out_slot * slot + part * bh,
@@ -1015,7 +1018,8 @@ struct LstmAdjCycle : Cycle {
     a.a = w->a[d.l] + row0; a.p = w->p[d.l] + row0; a.ci = w->ci[d.l] + row0; a.cf = w->cf[d.l] + row0;
     a.cg = w->cg[d.l] + row0; a.co = w->co[d.l] + row0; a.coef_ks = -(i64)d.tgt_stride * (i64)bh;
     a.W_hh = p->W_hh;
-    simt_lstm_adj_step(a, s);
+    if (is_tf32(c)) { int r = tf32_lstm_adj_step(a, &w->tf, s); if (r) return r; }
+    else simt_lstm_adj_step(a, s);
     for (int part = 0; part < 2; ++part) {
       const float* g = d.gadd ? d.gadd + (size_t)d.gadd_slot * slot + part * bh : nullptr;
       stream_combine_rows(part == 0 ? w->tmpC : w->tmpH, g, (i64)d.gadd_stride * slot, d.out + (size_t)d.out_slot * slot + part * bh,
@@ -1027,7 +1031,7 @@ struct LstmAdjCycle : Cycle {
 
 int lstm_check(const mgrit_gru_cfg* cfg, Hier* hr) {
   if (!cfg) return MGRIT_INVALID_ARG;
-  if (cfg->operands != MGRIT_OPERANDS_FP32) return MGRIT_UNSUPPORTED;      // four-gate products run on the fp32 engine only
+  if (cfg->operands == MGRIT_OPERANDS_BF16) return MGRIT_UNSUPPORTED;      // four-gate products: fp32 engine or the tf32 modes
   return check_cfg(cfg, hr);
 }
 
@@ -1044,7 +1048,8 @@ int lstm_forward_impl(const mgrit_gru_cfg* cfg, const gru_params* p, const float
   plan_lstm_fwd(&c, hr, w, &fw);
   if (!w.fits()) return MGRIT_WORKSPACE_TOO_SMALL;
   const size_t slot = (size_t)2 * c.B * c.H;
-  simt_project(x, p->W_ih, p->b_ih, gi, c.T * c.B, c.I, 4 * c.H, s);
+  if (is_tf32(&c)) { rc = tf32_prepare_fwd(&c, p, x, gi, &fw.tf, s); if (rc) return rc; }
+  else simt_project(x, p->W_ih, p->b_ih, gi, c.T * c.B, c.I, 4 * c.H, s);
   cudaMemsetAsync(fw.U[0] + slot, 0, sizeof(float) * (size_t)c.T * slot, s);
   for (int l = 0; l < hr.L; ++l) cudaMemcpyAsync(fw.U[l], u0, sizeof(float) * slot, cudaMemcpyDeviceToDevice, s);
   LstmFwdCycle cy;
@@ -1079,12 +1084,15 @@ int lstm_adjoint_impl(const mgrit_gru_cfg* cfg, const gru_params* p, const float
   if (!w.fits()) return MGRIT_WORKSPACE_TOO_SMALL;
   const size_t bh = (size_t)c.B * c.H, slot = 2 * bh;
   const int T = c.T;
+  const bool tf32 = is_tf32(&c);
+  if (tf32) { rc = tf32_prepare_adj(&c, p, &aw.tf, s); if (rc) return rc; }
   for (int l = 0; l < hr.L; ++l) {
     LstmLinArgs a;
     a.M = hr.N[l] * c.B; a.B = c.B; a.H = c.H; a.c0 = u0; a.h0 = u0 + bh; a.c = u; a.h = u + bh; a.ts = (i64)slot;
     a.stride_t = hr.stride_t[l]; a.t0 = hr.rem[l]; a.gi = gi; a.W_hh = p->W_hh; a.b_hh = p->b_hh; a.gamma = hr.gamma[l]; a.cell = c.cell;
     a.a = aw.a[l]; a.p = aw.p[l]; a.ci = aw.ci[l]; a.cf = aw.cf[l]; a.cg = aw.cg[l]; a.co = aw.co[l];
-    simt_lstm_linearise(a, s);
+    if (tf32) { rc = tf32_lstm_linearise(a, &aw.tf, s); if (rc) return rc; }
+    else simt_lstm_linearise(a, s);
   }
   cudaMemsetAsync(aw.U[0], 0, sizeof(float) * (size_t)(T + 1) * slot, s);
   cudaMemsetAsync(aw.G[0], 0, sizeof(float) * (size_t)(T + 1) * slot, s);
@@ -1106,11 +1114,20 @@ int lstm_adjoint_impl(const mgrit_gru_cfg* cfg, const gru_params* p, const float
   const float* lam_c = aw.U[0] + (size_t)(T - 1) * slot;
   simt_lstm_form_dA(lam_c, lam_c + bh, -(i64)slot, c.B, aw.p[0], aw.ci[0], aw.cf[0], aw.cg[0], aw.co[0], aw.dA, M, c.H, s);
   stream_gather_rows(aw.hk, (i64)bh, u + bh, (i64)slot, T, (i64)bh, s);        // hidden states as their own [T, B, H] array
-  simt_wgrad(aw.dA, (int)M, 4 * c.H, u0 + bh, c.B, aw.hk, c.H, g->dW_hh, s);
-  simt_wgrad(aw.dA, (int)M, 4 * c.H, nullptr, 0, x, c.I, g->dW_ih, s);
+  if (tf32) {
+    rc = tf32_wgrad(aw.dA, (int)M, 4 * c.H, u0 + bh, c.B, aw.hk, c.H, g->dW_hh, &aw.tf, s);
+    if (!rc) rc = tf32_wgrad(aw.dA, (int)M, 4 * c.H, nullptr, 0, x, c.I, g->dW_ih, &aw.tf, s);
+    if (rc) return rc;
+  } else {
+    simt_wgrad(aw.dA, (int)M, 4 * c.H, u0 + bh, c.B, aw.hk, c.H, g->dW_hh, s);
+    simt_wgrad(aw.dA, (int)M, 4 * c.H, nullptr, 0, x, c.I, g->dW_ih, s);
+  }
   stream_colsum(aw.dA, M, 4 * c.H, g->db_hh, s);
   cudaMemcpyAsync(g->db_ih, g->db_hh, sizeof(float) * 4 * c.H, cudaMemcpyDeviceToDevice, s);
-  if (dx) simt_dgrad(aw.dA, (int)M, 4 * c.H, p->W_ih, c.I, dx, s);
+  if (dx) {
+    if (tf32) { rc = tf32_dgrad(aw.dA, (int)M, 4 * c.H, c.I, dx, &aw.tf, s); if (rc) return rc; }
+    else simt_dgrad(aw.dA, (int)M, 4 * c.H, p->W_ih, c.I, dx, s);
+  }
   if (resnorm && hr.L > 1 && c.iters > 0) {
     rc = fetch_resnorm(aw.res_acc, resnorm, c.iters, s);
     if (rc) return rc;

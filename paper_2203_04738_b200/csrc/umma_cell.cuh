@@ -83,6 +83,15 @@ __device__ __forceinline__ void tmem_ld_wait8x3(float* a, float* b, float* c) {
                :
                : "memory");
 }
+__device__ __forceinline__ void tmem_ld_wait8x4(float* a, float* b, float* c, float* d) {
+  asm volatile("tcgen05.wait::ld.sync.aligned;"
+               : "+f"(a[0]), "+f"(a[1]), "+f"(a[2]), "+f"(a[3]), "+f"(a[4]), "+f"(a[5]), "+f"(a[6]), "+f"(a[7]),
+                 "+f"(b[0]), "+f"(b[1]), "+f"(b[2]), "+f"(b[3]), "+f"(b[4]), "+f"(b[5]), "+f"(b[6]), "+f"(b[7]),
+                 "+f"(c[0]), "+f"(c[1]), "+f"(c[2]), "+f"(c[3]), "+f"(c[4]), "+f"(c[5]), "+f"(c[6]), "+f"(c[7]),
+                 "+f"(d[0]), "+f"(d[1]), "+f"(d[2]), "+f"(d[3]), "+f"(d[4]), "+f"(d[5]), "+f"(d[6]), "+f"(d[7])
+               :
+               : "memory");
+}
 // One 32-byte store per thread: a warp's lanes write 32 different rows, and two 16-byte stores per row would
 // reach L2 as two half-filled sector writes each.
 __device__ __forceinline__ void stg8(float* p, const float* v) {

@@ -77,27 +77,27 @@ bool make_map(CUtensorMap* m, const float* base, uint64_t inner, uint64_t rows, 
 }
 
 // ET = bf16, or float for operands that hold tf32 values.  splits > 1 (split-aware epilogues only) cuts the reduction.
-template <int BN, bool GATES, class Epi, class ET>
+template <int BN, int NG, class Epi, class ET>
 bool launch_gemm(int kc, const ET* A, i64 lda, const ET* Bm, i64 ldb, int M, int N, int K, int gate_rows, int b_rows, Epi epi,
                  cudaStream_t s, int splits = 1) {
-  using C = Cfg<BN, GATES>;
+  using C = Cfg<BN, NG>;
   constexpr bool TF32 = sizeof(ET) == 4;
   if (M <= 0 || N <= 0) return true;
   int* const status = status_ptr();
   if (!status) return false;
   static bool attr_set[kMaxDevices] = {false};
-  auto kern = umma_gemm_kernel<BN, GATES, Epi, false, TF32>;
+  auto kern = umma_gemm_kernel<BN, NG, Epi, false, TF32>;
   if (!set_smem_once(kern, C::kSmemBytes, attr_set)) return false;
   CUtensorMap ta, tb;
   if (!make_map(&ta, A, (uint64_t)K, (uint64_t)M, (uint64_t)lda, BM)) return false;
-  if (!make_map(&tb, Bm, (uint64_t)K, (uint64_t)b_rows, (uint64_t)ldb, GATES ? BN / 3 : BN)) return false;
+  if (!make_map(&tb, Bm, (uint64_t)K, (uint64_t)b_rows, (uint64_t)ldb, NG > 0 ? BN / NG : BN)) return false;
   const int k_blocks = (K + (TF32 ? BK / 2 : BK) - 1) / (TF32 ? BK / 2 : BK);
   if (splits < 1 || !EpiSplitAware<Epi>::value) splits = 1;
   GemmShape sh{M, N, K, gate_rows, splits, (k_blocks + splits - 1) / splits};
   int m_tiles = (M + BM - 1) / BM, n_tiles = (N + C::kNPerTile - 1) / C::kNPerTile;
   int tiles = m_tiles * n_tiles * splits;
   int grid = tiles < kSMs ? tiles : kSMs;
-  ProfScope prof_(kc, 2.0 * M * (GATES ? 3.0 * N : (double)N) * K, s);
+  ProfScope prof_(kc, 2.0 * M * (NG > 0 ? (double)NG * N : (double)N) * K, s);
   if (launch_pdl(kern, dim3(grid), dim3(kThreads), C::kSmemBytes, s, ta, tb, sh, epi, status) != cudaSuccess) return false;
   count_launch();
   return true;
@@ -138,12 +138,12 @@ bool launch_gemm_pair(int kc, const bf16* A, i64 lda, const bf16* Bm, i64 ldb, i
 template <class Epi>
 bool launch_gemm_mn(int kc, const bf16* A, i64 lda, int Mdim, const bf16* Bm, i64 ldb, int Ndim, int K, int splits, Epi epi,
                     cudaStream_t s) {
-  using C = Cfg<256, false>;
+  using C = Cfg<256, 0>;
   if (Mdim <= 0 || Ndim <= 0) return true;
   int* const status = status_ptr();
   if (!status) return false;
   static bool attr_set[kMaxDevices] = {false};
-  auto kern = umma_gemm_kernel<256, false, Epi, true>;
+  auto kern = umma_gemm_kernel<256, 0, Epi, true>;
   if (!set_smem_once(kern, C::kSmemBytes, attr_set)) return false;
   CUtensorMap ta, tb;
   if (!make_map(&ta, A, (uint64_t)Mdim, (uint64_t)K, (uint64_t)lda, 64)) return false;
@@ -745,7 +745,7 @@ int umma_prepare_fwd(const mgrit_gru_cfg* c, const gru_params* p, const float* x
   // gi = x W_ih^T + b_ih :  M = T*B, N = 3H, K = I
   if (gemm_pair_enabled((int)TB, 3 * H)
           ? !launch_gemm_pair(KC_PROJ, w->xb, I, w->W_ih, I, (int)TB, 3 * H, I, 3 * H, EpiBias{gi, 3 * H, p->b_ih, (int)TB, 3 * H}, s)
-          : !launch_gemm<256, false>(KC_PROJ, w->xb, I, w->W_ih, I, (int)TB, 3 * H, I, 0, 3 * H, EpiBias{gi, 3 * H, p->b_ih, (int)TB, 3 * H}, s))
+          : !launch_gemm<256, 0>(KC_PROJ, w->xb, I, w->W_ih, I, (int)TB, 3 * H, I, 0, 3 * H, EpiBias{gi, 3 * H, p->b_ih, (int)TB, 3 * H}, s))
     return MGRIT_CUDA_ERROR;
   return MGRIT_OK;
 }
@@ -786,7 +786,7 @@ int umma_fwd_step(const FwdStepArgs& a, UmmaFwdWs* w, cudaStream_t s) {
                  reinterpret_cast<uint2*>(w->Apack)) != cudaSuccess)
     return MGRIT_CUDA_ERROR;
   count_launch();
-  ok = launch_gemm<192, true>(KC_FWD_STEP, w->Apack, a.H, w->W_hh, a.H, a.M, a.H, a.H, a.H, 3 * a.H, EpiFwd<true>{a}, s);
+  ok = launch_gemm<192, 3>(KC_FWD_STEP, w->Apack, a.H, w->W_hh, a.H, a.M, a.H, a.H, a.H, 3 * a.H, EpiFwd<true>{a}, s);
   return ok ? MGRIT_OK : MGRIT_CUDA_ERROR;
 }
 
@@ -857,7 +857,7 @@ int umma_linearise(const LinArgs& a, UmmaAdjWs* w, cudaStream_t s) {
       return MGRIT_CUDA_ERROR;
     count_launch();
   }
-  return launch_gemm<192, true>(KC_LINEARISE, w->Apack, a.H, w->W_hh, a.H, a.M, a.H, a.H, a.H, 3 * a.H, EpiLin<true>{a}, s) ? MGRIT_OK
+  return launch_gemm<192, 3>(KC_LINEARISE, w->Apack, a.H, w->W_hh, a.H, a.M, a.H, a.H, a.H, 3 * a.H, EpiLin<true>{a}, s) ? MGRIT_OK
                                                                                                                       : MGRIT_CUDA_ERROR;
 }
 
@@ -872,11 +872,11 @@ int umma_adj_step(const AdjStepArgs& a, UmmaAdjWs* w, cudaStream_t s) {
   const int tiles256 = ((a.M + BM - 1) / BM) * ((a.H + 255) / 256);
   bool ok;
   if (tiles256 * 2 <= kSMs)
-    ok = launch_gemm<64, false>(KC_ADJ_STEP, w->Apack, 3 * a.H, w->W_hhT, 3 * a.H, a.M, a.H, 3 * a.H, 0, a.H, EpiAdj<64>{a}, s);
+    ok = launch_gemm<64, 0>(KC_ADJ_STEP, w->Apack, 3 * a.H, w->W_hhT, 3 * a.H, a.M, a.H, 3 * a.H, 0, a.H, EpiAdj<64>{a}, s);
   else if (gemm_pair_enabled(a.M, a.H))
     ok = launch_gemm_pair(KC_ADJ_STEP, w->Apack, 3 * a.H, w->W_hhT, 3 * a.H, a.M, a.H, 3 * a.H, a.H, EpiAdj<256>{a}, s);
   else
-    ok = launch_gemm<256, false>(KC_ADJ_STEP, w->Apack, 3 * a.H, w->W_hhT, 3 * a.H, a.M, a.H, 3 * a.H, 0, a.H, EpiAdj<256>{a}, s);
+    ok = launch_gemm<256, 0>(KC_ADJ_STEP, w->Apack, 3 * a.H, w->W_hhT, 3 * a.H, a.M, a.H, 3 * a.H, 0, a.H, EpiAdj<256>{a}, s);
   return ok ? MGRIT_OK : MGRIT_CUDA_ERROR;
 }
 
@@ -949,7 +949,7 @@ int umma_gradients(const mgrit_gru_cfg* c, const gru_params* p, const float* x, 
   if (dx)
     ok = ok && (gemm_pair_enabled((int)M, I)
                     ? launch_gemm_pair(KC_WGRAD, dAi, 3 * H, w->W_ihT, 3 * H, (int)M, I, 3 * H, I, EpiStore{dx, I, (int)M, I, 0}, s)
-                    : launch_gemm<256, false>(KC_WGRAD, dAi, 3 * H, w->W_ihT, 3 * H, (int)M, I, 3 * H, 0, I, EpiStore{dx, I, (int)M, I, 0}, s));
+                    : launch_gemm<256, 0>(KC_WGRAD, dAi, 3 * H, w->W_ihT, 3 * H, (int)M, I, 3 * H, 0, I, EpiStore{dx, I, (int)M, I, 0}, s));
   return ok ? MGRIT_OK : MGRIT_CUDA_ERROR;
 }
 
@@ -958,7 +958,7 @@ void umma_convert(const float* src, __nv_bfloat16* dst, i64 n, cudaStream_t s) {
 // out[M, 3H] = X[M, K] W^T + bias with X fp32 contiguous (converted into xb first) and W already bf16 [3H, K]
 int umma_project_rows(const float* X, bf16* xb, const bf16* Wb, const float* bias, float* out, int M, int K, int H3, cudaStream_t s) {
   convert(X, xb, (i64)M * K, s);
-  return launch_gemm<256, false>(KC_PROJ, xb, K, Wb, K, M, H3, K, 0, H3, EpiBias{out, H3, bias, M, H3}, s) ? MGRIT_OK : MGRIT_CUDA_ERROR;
+  return launch_gemm<256, 0>(KC_PROJ, xb, K, Wb, K, M, H3, K, 0, H3, EpiBias{out, H3, bias, M, H3}, s) ? MGRIT_OK : MGRIT_CUDA_ERROR;
 }
 
 // out[M, C] = ([cr|cz|cn]*lam of the step `a`) W_ihT^T: the sensitivity a cell sends to its input (a.cnb holding c_n')
@@ -967,7 +967,7 @@ int umma_adj_dx(const AdjStepArgs& a, const bf16* W_ihT, int C, float* out, Umma
                  a.B, a.H / 4, (i64)a.M, reinterpret_cast<uint2*>(w->Apack)) != cudaSuccess)
     return MGRIT_CUDA_ERROR;
   count_launch();
-  return launch_gemm<256, false>(KC_ADJ_STEP, w->Apack, 3 * a.H, W_ihT, 3 * a.H, a.M, C, 3 * a.H, 0, C, EpiStore{out, C, a.M, C, 0}, s)
+  return launch_gemm<256, 0>(KC_ADJ_STEP, w->Apack, 3 * a.H, W_ihT, 3 * a.H, a.M, C, 3 * a.H, 0, C, EpiStore{out, C, a.M, C, 0}, s)
              ? MGRIT_OK : MGRIT_CUDA_ERROR;
 }
 
@@ -1062,11 +1062,11 @@ int tf32_supported(const mgrit_gru_cfg* c) {
   return MGRIT_OK;
 }
 
-void tf32_plan_fwd(const mgrit_gru_cfg* c, const int* N, int L, char* base, size_t* off, Tf32Ws* o) {
+void tf32_plan_fwd(const mgrit_gru_cfg* c, const int* N, int L, char* base, size_t* off, Tf32Ws* o, int ng) {
   const size_t S = c->operands == MGRIT_OPERANDS_TF32 ? 3 : 1, H = c->H, I = c->I, TB = (size_t)c->T * c->B;
-  o->S = (int)S;
-  o->W_hh = take<float>(base, off, 3 * H * S * H);
-  o->W_ih = take<float>(base, off, 3 * H * S * I);
+  o->S = (int)S; o->ng = ng;
+  o->W_hh = take<float>(base, off, ng * H * S * H);
+  o->W_ih = take<float>(base, off, ng * H * S * I);
   o->W_hhT = o->W_ihT = o->dAT = o->RT = nullptr;
   size_t ap = max_step_rows(c, N, L) * S * H;
   if (TB * S * I > ap) ap = TB * S * I;
@@ -1074,45 +1074,46 @@ void tf32_plan_fwd(const mgrit_gru_cfg* c, const int* N, int L, char* base, size
   o->Apack = take<float>(base, off, ap);
 }
 
-void tf32_plan_adj(const mgrit_gru_cfg* c, const int* N, int L, char* base, size_t* off, Tf32Ws* o) {
+void tf32_plan_adj(const mgrit_gru_cfg* c, const int* N, int L, char* base, size_t* off, Tf32Ws* o, int ng) {
+  (void)N; (void)L;
   const size_t S = c->operands == MGRIT_OPERANDS_TF32 ? 3 : 1, H = c->H, I = c->I, TB = (size_t)c->T * c->B;
-  o->S = (int)S;
-  o->W_hh = take<float>(base, off, 3 * H * S * H);
+  o->S = (int)S; o->ng = ng;
+  o->W_hh = take<float>(base, off, ng * H * S * H);
   o->W_ih = nullptr;
-  o->W_hhT = take<float>(base, off, H * S * 3 * H);
-  o->W_ihT = take<float>(base, off, I * S * 3 * H);
-  o->apack_elems = TB * S * 3 * H;       // the input-gradient product packs all T*B rows of dA; every step needs less
+  o->W_hhT = take<float>(base, off, H * S * ng * H);
+  o->W_ihT = take<float>(base, off, I * S * ng * H);
+  o->apack_elems = TB * S * ng * H;       // the input-gradient product packs all T*B rows of dA; every step needs less
   o->Apack = take<float>(base, off, o->apack_elems);
-  o->dAT = take<float>(base, off, 3 * H * S * TB);
+  o->dAT = take<float>(base, off, ng * H * S * TB);
   o->RT = take<float>(base, off, (H > I ? H : I) * S * TB);
-  o->split_scratch = take<float>(base, off, 4 * 3 * H * (H > I ? H : I));
+  o->split_scratch = take<float>(base, off, 4 * ng * H * (H > I ? H : I));
 }
 
 int tf32_prepare_fwd(const mgrit_gru_cfg* c, const gru_params* p, const float* x, float* gi, Tf32Ws* w, cudaStream_t s) {
-  const int H = c->H, I = c->I, S = w->S;
+  const int H = c->H, I = c->I, S = w->S, GH = w->ng * H;
   const int TB = c->T * c->B;
   if (!status_ptr()) return MGRIT_CUDA_ERROR;
-  bool ok = split_rows(p->W_hh, 0, 3 * H, H, 3 * H, S, true, w->W_hh, s) && split_rows(p->W_ih, 0, 3 * H, I, 3 * H, S, true, w->W_ih, s) &&
+  bool ok = split_rows(p->W_hh, 0, GH, H, GH, S, true, w->W_hh, s) && split_rows(p->W_ih, 0, GH, I, GH, S, true, w->W_ih, s) &&
             split_rows(x, 0, TB, I, TB, S, false, w->Apack, s);
-  // gi = x W_ih^T + b_ih :  M = T*B, N = 3H, K = S*I
-  ok = ok && launch_gemm<256, false>(KC_PROJ, (const float*)w->Apack, (i64)S * I, (const float*)w->W_ih, (i64)S * I, TB, 3 * H, S * I, 0, 3 * H,
-                                     EpiBias{gi, 3 * H, p->b_ih, TB, 3 * H}, s);
+  // gi = x W_ih^T + b_ih :  M = T*B, N = (3 or 4) H, K = S*I
+  ok = ok && launch_gemm<256, 0>(KC_PROJ, (const float*)w->Apack, (i64)S * I, (const float*)w->W_ih, (i64)S * I, TB, GH, S * I, 0, GH,
+                                     EpiBias{gi, GH, p->b_ih, TB, GH}, s);
   return ok ? MGRIT_OK : MGRIT_CUDA_ERROR;
 }
 
 int tf32_fwd_step(const FwdStepArgs& a, Tf32Ws* w, cudaStream_t s) {
   const int S = w->S;
   if (!split_rows(a.hin, a.hin_ks, a.B, a.H, a.M, S, false, w->Apack, s)) return MGRIT_CUDA_ERROR;
-  return launch_gemm<192, true>(KC_FWD_STEP, (const float*)w->Apack, (i64)S * a.H, (const float*)w->W_hh, (i64)S * a.H, a.M, a.H, S * a.H, a.H,
+  return launch_gemm<192, 3>(KC_FWD_STEP, (const float*)w->Apack, (i64)S * a.H, (const float*)w->W_hh, (i64)S * a.H, a.M, a.H, S * a.H, a.H,
                                 3 * a.H, EpiFwd<false>{a}, s) ? MGRIT_OK : MGRIT_CUDA_ERROR;
 }
 
 int tf32_prepare_adj(const mgrit_gru_cfg* c, const gru_params* p, Tf32Ws* w, cudaStream_t s) {
-  const int H = c->H, I = c->I, S = w->S;
+  const int H = c->H, I = c->I, S = w->S, GH = w->ng * H;
   if (!status_ptr()) return MGRIT_CUDA_ERROR;
-  if (!split_rows(p->W_hh, 0, 3 * H, H, 3 * H, S, true, w->W_hh, s)) return MGRIT_CUDA_ERROR;
-  transpose_split(nullptr, 0, p->W_hh, 3 * H, H, S, true, w->W_hhT, s);   // [H, S*3H]
-  transpose_split(nullptr, 0, p->W_ih, 3 * H, I, S, true, w->W_ihT, s);   // [I, S*3H]
+  if (!split_rows(p->W_hh, 0, GH, H, GH, S, true, w->W_hh, s)) return MGRIT_CUDA_ERROR;
+  transpose_split(nullptr, 0, p->W_hh, GH, H, S, true, w->W_hhT, s);   // [H, S*GH]
+  transpose_split(nullptr, 0, p->W_ih, GH, I, S, true, w->W_ihT, s);   // [I, S*GH]
   return MGRIT_OK;
 }
 
@@ -1130,7 +1131,7 @@ int tf32_linearise(const LinArgs& a, Tf32Ws* w, cudaStream_t s) {
     if (!split_rows(a.h + (t1 - 1) * BH, a.stride_t * BH, a.B, a.H, (i64)(N - done) * a.B, S, false, w->Apack + (i64)done * BH * S, s))
       return MGRIT_CUDA_ERROR;
   }
-  return launch_gemm<192, true>(KC_LINEARISE, (const float*)w->Apack, (i64)S * a.H, (const float*)w->W_hh, (i64)S * a.H, a.M, a.H, S * a.H, a.H,
+  return launch_gemm<192, 3>(KC_LINEARISE, (const float*)w->Apack, (i64)S * a.H, (const float*)w->W_hh, (i64)S * a.H, a.M, a.H, S * a.H, a.H,
                                 3 * a.H, EpiLin<false>{a}, s) ? MGRIT_OK : MGRIT_CUDA_ERROR;
 }
 
@@ -1144,9 +1145,9 @@ int tf32_adj_step(const AdjStepArgs& a, Tf32Ws* w, cudaStream_t s) {
   const int tiles256 = ((a.M + BM - 1) / BM) * ((a.H + 255) / 256);
   bool ok;
   if (tiles256 * 2 <= kSMs)
-    ok = launch_gemm<64, false>(KC_ADJ_STEP, (const float*)w->Apack, (i64)K, (const float*)w->W_hhT, (i64)K, a.M, a.H, K, 0, a.H, EpiAdj<64>{a}, s);
+    ok = launch_gemm<64, 0>(KC_ADJ_STEP, (const float*)w->Apack, (i64)K, (const float*)w->W_hhT, (i64)K, a.M, a.H, K, 0, a.H, EpiAdj<64>{a}, s);
   else
-    ok = launch_gemm<256, false>(KC_ADJ_STEP, (const float*)w->Apack, (i64)K, (const float*)w->W_hhT, (i64)K, a.M, a.H, K, 0, a.H, EpiAdj<256>{a}, s);
+    ok = launch_gemm<256, 0>(KC_ADJ_STEP, (const float*)w->Apack, (i64)K, (const float*)w->W_hhT, (i64)K, a.M, a.H, K, 0, a.H, EpiAdj<256>{a}, s);
   return ok ? MGRIT_OK : MGRIT_CUDA_ERROR;
 }
 
@@ -1161,10 +1162,10 @@ int tf32_wgrad(const float* dA, int M, int H3, const float* first, int Bfirst, c
   const size_t scratch_bytes = (size_t)4 * H3 * C * sizeof(float);
   const int splits = (((i64)H3 * C) % 4 == 0) ? pick_splits(H3, C, K, scratch_bytes) : 1;
   if (splits == 1)
-    return launch_gemm<256, false>(KC_WGRAD, (const float*)w->dAT, (i64)K, (const float*)w->RT, (i64)K, H3, C, K, 0, C, EpiStore{dW, C, H3, C, 0}, s)
+    return launch_gemm<256, 0>(KC_WGRAD, (const float*)w->dAT, (i64)K, (const float*)w->RT, (i64)K, H3, C, K, 0, C, EpiStore{dW, C, H3, C, 0}, s)
                ? MGRIT_OK : MGRIT_CUDA_ERROR;
   const i64 n = (i64)H3 * C;
-  if (!launch_gemm<256, false>(KC_WGRAD, (const float*)w->dAT, (i64)K, (const float*)w->RT, (i64)K, H3, C, K, 0, C,
+  if (!launch_gemm<256, 0>(KC_WGRAD, (const float*)w->dAT, (i64)K, (const float*)w->RT, (i64)K, H3, C, K, 0, C,
                                EpiStore{w->split_scratch, C, H3, C, n}, s, splits))
     return MGRIT_CUDA_ERROR;
   sum_splits_kernel<<<pgrid(n / 4), kPT, 0, s>>>(reinterpret_cast<const float4*>(w->split_scratch), n / 4, splits, reinterpret_cast<float4*>(dW));
@@ -1177,8 +1178,127 @@ int tf32_dgrad(const float* dA, int M, int H3, int C, float* dx, Tf32Ws* w, cuda
   const int S = w->S, K = S * H3;
   if ((size_t)M * K > w->apack_elems) return MGRIT_UNSUPPORTED;
   if (!split_rows(dA, 0, M, H3, M, S, false, w->Apack, s)) return MGRIT_CUDA_ERROR;
-  return launch_gemm<256, false>(KC_WGRAD, (const float*)w->Apack, (i64)K, (const float*)w->W_ihT, (i64)K, M, C, K, 0, C, EpiStore{dx, C, M, C, 0}, s)
+  return launch_gemm<256, 0>(KC_WGRAD, (const float*)w->Apack, (i64)K, (const float*)w->W_ihT, (i64)K, M, C, K, 0, C, EpiStore{dx, C, M, C, 0}, s)
              ? MGRIT_OK : MGRIT_CUDA_ERROR;
+}
+
+// ---------------------------------------------------------------- Implicit LSTM on the tf32 products
+namespace {
+
+// LSTM cell / its transposed-Jacobian coefficients on the i | f | g | o accumulator columns of 64 hidden units, one
+// output row per thread, 8 units at a time (precise gate math)
+template <bool LIN>
+struct EpiLstm {
+  LstmFwdArgs f;      // !LIN
+  LstmLinArgs l;      // LIN
+  __device__ void operator()(uint32_t taddr, int row, int u0, int half) const {
+    const int M = LIN ? l.M : f.M, B = LIN ? l.B : f.B, H = LIN ? l.H : f.H;
+    const bool valid = row < M;
+    const int k = valid ? row / B : 0, b = valid ? row % B : 0;
+    const float* gi; const float* cpp; const float* bh = (LIN ? l.b_hh : f.b_hh) + u0;
+    if (LIN) {
+      const i64 t = l.t0 + (i64)k * l.stride_t;
+      gi = l.gi + ((t + l.stride_t - 1) * B + b) * 4 * H + u0;
+      cpp = (t == 0 ? l.c0 + (i64)b * H : l.c + (t - 1) * l.ts + (i64)b * H) + u0;
+    } else {
+      gi = f.gi + (i64)k * f.gi_ks + (i64)b * 4 * H + u0;
+      cpp = f.cin + (i64)k * f.in_ks + (i64)b * H + u0;
+    }
+    const i64 o = (i64)row * H + u0;
+    const float gamma = LIN ? l.gamma : f.gamma; const int cell = LIN ? l.cell : f.cell;
+#pragma unroll 1
+    for (int c0 = half * 32; c0 < half * 32 + 32; c0 += 8) {
+      float g4[4][8], cp[8], acc[4][8];
+      if (valid) {
+#pragma unroll
+        for (int g = 0; g < 4; ++g) ld8(gi + (i64)g * H + c0, g4[g]);
+        ld8(cpp + c0, cp);
+      }
+#pragma unroll
+      for (int g = 0; g < 4; ++g) tmem_ld8(taddr + g * 64 + c0, acc[g]);
+      tmem_ld_wait8x4(acc[0], acc[1], acc[2], acc[3]);
+      if (valid) {
+        float o0[8], o1[8], o2[8], o3[8], o4[8], o5[8];
+#pragma unroll
+        for (int e = 0; e < 8; ++e) {
+          const int n = c0 + e;
+          const float ai = acc[0][e] + __ldg(bh + n), af = acc[1][e] + __ldg(bh + H + n), ag = acc[2][e] + __ldg(bh + 2 * H + n),
+                      ao = acc[3][e] + __ldg(bh + 3 * H + n);
+          if (LIN) {
+            LstmLin L = lstm_linearise(g4[0][e], g4[1][e], g4[2][e], g4[3][e], ai, af, ag, ao, cp[e], gamma, cell);
+            o0[e] = L.a; o1[e] = L.p; o2[e] = L.ci; o3[e] = L.cf; o4[e] = L.cg; o5[e] = L.co;
+          } else {
+            LstmOut r = lstm_forward(g4[0][e], g4[1][e], g4[2][e], g4[3][e], ai, af, ag, ao, cp[e], gamma, cell);
+            o0[e] = r.c; o1[e] = r.h;
+          }
+        }
+        if (LIN) {
+          st8(l.a + o + c0, o0); st8(l.p + o + c0, o1); st8(l.ci + o + c0, o2); st8(l.cf + o + c0, o3); st8(l.cg + o + c0, o4);
+          st8(l.co + o + c0, o5);
+        } else {
+          st8(f.cout + o + c0, o0); st8(f.hout + o + c0, o1);
+        }
+      }
+    }
+  }
+};
+
+// dst[m, seg*4H + g*H + i] = split(coefficient_g * (g < 3 ? Lc + p*Lh : Lh))   (A side);  lc_out[m, i] = a * (Lc + p*Lh)
+__global__ void __launch_bounds__(kPT) split_lstm_adj_kernel(LstmAdjArgs a, int S, float* __restrict__ dst) {
+  pdl_wait();
+  pdl_trigger();
+  const i64 total = (i64)a.M * a.H;
+  for (i64 e = (i64)blockIdx.x * blockDim.x + threadIdx.x; e < total; e += (i64)gridDim.x * blockDim.x) {
+    const i64 m = e / a.H; const int i = (int)(e % a.H);
+    const i64 kk = m / a.B; const int b = (int)(m % a.B);
+    const i64 ci = kk * a.coef_ks + (i64)b * a.H + i, li = kk * a.in_ks + (i64)b * a.H + i;
+    const float lh = a.lh[li], dc = a.lc[li] + a.p[ci] * lh;
+    a.lc_out[e] = a.a[ci] * dc;
+    const float v[4] = {a.ci[ci] * dc, a.cf[ci] * dc, a.cg[ci] * dc, a.co[ci] * lh};
+    for (int seg = 0; seg < S; ++seg)
+#pragma unroll
+      for (int g = 0; g < 4; ++g) dst[m * S * 4 * a.H + (i64)seg * 4 * a.H + g * a.H + i] = split_part(v[g], seg, false);
+  }
+}
+
+}  // namespace
+
+int tf32_lstm_fwd_step(const LstmFwdArgs& a, Tf32Ws* w, cudaStream_t s) {
+  const int S = w->S;
+  if (!split_rows(a.hin, a.in_ks, a.B, a.H, a.M, S, false, w->Apack, s)) return MGRIT_CUDA_ERROR;
+  EpiLstm<false> epi{};
+  epi.f = a;
+  return launch_gemm<256, 4>(KC_FWD_STEP, (const float*)w->Apack, (i64)S * a.H, (const float*)w->W_hh, (i64)S * a.H, a.M, a.H, S * a.H, a.H,
+                             4 * a.H, epi, s) ? MGRIT_OK : MGRIT_CUDA_ERROR;
+}
+
+int tf32_lstm_linearise(const LstmLinArgs& a, Tf32Ws* w, cudaStream_t s) {
+  // rows (j-1, b): hidden state entering forward step j of the level = h at fine time t0 + stride*(j-1) (h_0 for time 0)
+  const int N = a.M / a.B, S = w->S;
+  const i64 BHS = (i64)a.B * a.H * S;
+  int done = 0;
+  if (a.t0 == 0) {
+    if (!split_rows(a.h0, 0, a.B, a.H, a.B, S, false, w->Apack, s)) return MGRIT_CUDA_ERROR;
+    done = 1;
+  }
+  if (N > done) {
+    const i64 t1 = a.t0 + (i64)done * a.stride_t;
+    if (!split_rows(a.h + (t1 - 1) * a.ts, a.stride_t * a.ts, a.B, a.H, (i64)(N - done) * a.B, S, false, w->Apack + (i64)done * BHS, s))
+      return MGRIT_CUDA_ERROR;
+  }
+  EpiLstm<true> epi{};
+  epi.l = a;
+  return launch_gemm<256, 4>(KC_LINEARISE, (const float*)w->Apack, (i64)S * a.H, (const float*)w->W_hh, (i64)S * a.H, a.M, a.H, S * a.H, a.H,
+                             4 * a.H, epi, s) ? MGRIT_OK : MGRIT_CUDA_ERROR;
+}
+
+int tf32_lstm_adj_step(const LstmAdjArgs& a, Tf32Ws* w, cudaStream_t s) {
+  const int S = w->S, K = S * 4 * a.H;
+  ProfScope prof(KC_ADJ_STEP, 2.0 * a.M * (double)K * a.H, s);
+  if (launch_pdl(split_lstm_adj_kernel, dim3(pgrid((i64)a.M * a.H)), dim3(kPT), 0, s, a, S, w->Apack) != cudaSuccess) return MGRIT_CUDA_ERROR;
+  count_launch();
+  return launch_gemm<256, 0>(KC_ADJ_STEP, (const float*)w->Apack, (i64)K, (const float*)w->W_hhT, (i64)K, a.M, a.H, K, 0, a.H,
+                             EpiStore{a.lh_out, a.H, a.M, a.H, 0}, s) ? MGRIT_OK : MGRIT_CUDA_ERROR;
 }
 
 int umma_device_status() {

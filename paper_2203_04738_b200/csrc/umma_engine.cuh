@@ -30,6 +30,7 @@ struct UmmaAdjWs {
 // along the reduction (MGRIT_OPERANDS_TF32) or rounded once (S = 1, MGRIT_OPERANDS_TF32_1PASS)
 struct Tf32Ws {
   int S;
+  int ng;         // gate blocks of the weights: 3 (GRU) or 4 (LSTM); "3H" below reads ng*H
   float* W_hh;    // [3H, S*H]   B side of the forward product
   float* W_ih;    // [3H, S*I]   forward call only
   float* W_hhT;   // [H, S*3H]   adjoint call: B side of the adjoint step
@@ -41,8 +42,12 @@ struct Tf32Ws {
   float* split_scratch;   // partial products of a split reduction
 };
 int tf32_supported(const mgrit_gru_cfg* c);
-void tf32_plan_fwd(const mgrit_gru_cfg* c, const int* N, int L, char* base, size_t* off, Tf32Ws* o);
-void tf32_plan_adj(const mgrit_gru_cfg* c, const int* N, int L, char* base, size_t* off, Tf32Ws* o);
+void tf32_plan_fwd(const mgrit_gru_cfg* c, const int* N, int L, char* base, size_t* off, Tf32Ws* o, int ng = 3);
+void tf32_plan_adj(const mgrit_gru_cfg* c, const int* N, int L, char* base, size_t* off, Tf32Ws* o, int ng = 3);
+// Implicit LSTM steps on the same products (raw results, contiguous [M, H], as the fp32 engine's)
+int tf32_lstm_fwd_step(const LstmFwdArgs& a, Tf32Ws* w, cudaStream_t s);
+int tf32_lstm_linearise(const LstmLinArgs& a, Tf32Ws* w, cudaStream_t s);
+int tf32_lstm_adj_step(const LstmAdjArgs& a, Tf32Ws* w, cudaStream_t s);
 int tf32_prepare_fwd(const mgrit_gru_cfg* c, const gru_params* p, const float* x, float* gi, Tf32Ws* w, cudaStream_t s);
 int tf32_prepare_adj(const mgrit_gru_cfg* c, const gru_params* p, Tf32Ws* w, cudaStream_t s);
 int tf32_fwd_step(const FwdStepArgs& a, Tf32Ws* w, cudaStream_t s);

@@ -5,9 +5,9 @@
 //
 //   D[m, n] = sum_k A[m, k] * B[n, k]      A: [M, K] bf16 row-major, B: [N, K] bf16 row-major
 //
-// Tile 128 x BN x 64.  With GATES the BN = 192 accumulator columns are the r | z | n
-// pre-activations of the same 64 hidden units (three 64-row boxes of the [3H, K] weight), so the
-// epilogue can apply the whole GRU cell without another pass over memory.
+// Tile 128 x BN x 64.  With NG = 3 (GRU) or 4 (LSTM) gates the BN = 64 NG accumulator columns are the
+// pre-activations of the same 64 hidden units (NG 64-row boxes of the [NG H, K] weight), so the
+// epilogue can apply the whole cell without another pass over memory.
 //
 // Every wait on an mbarrier is bounded: when it runs out the CTA records an error code in the
 // status word, stops issuing work, releases its tensor memory and returns.
@@ -152,7 +152,7 @@ __device__ __forceinline__ void tmem_ld_wait() { asm volatile("tcgen05.wait::ld.
 
 struct GemmShape {
   int M, N, K;          // row pitches must be multiples of 16 bytes (TMA stride rule); any M, N
-  int gate_rows;        // GATES: row distance between the r, z, n blocks of B (= H); else 0
+  int gate_rows;        // NG > 0: row distance between the gate blocks of B (= H); else 0
   int splits;           // split products (MN-major, or an epilogue with kSplitAware): the reduction is cut into `splits`
   int kb_per_split;     // ranges of kb_per_split k-blocks, each (tile, range) is one work item and the epilogue is told
                         // which range it finishes; 0 or 1 = the whole reduction in one item
@@ -163,29 +163,29 @@ struct GemmShape {
 template <class E, class = void> struct EpiSplitAware { static constexpr bool value = false; };
 template <class E> struct EpiSplitAware<E, decltype((void)E::kSplitAware)> { static constexpr bool value = E::kSplitAware; };
 
-template <int BN, bool GATES>
+template <int BN, int NG>
 struct Cfg {
-  static constexpr int kStages = GATES ? 5 : (BN <= 64 ? 8 : 4);
+  static constexpr int kStages = NG == 3 ? 5 : (BN <= 64 ? 8 : 4);
   static constexpr int kABytes = BM * BK * 2;
   static constexpr int kBBytes = BN * BK * 2;
   static constexpr int kStageBytes = kABytes + kBBytes;
   static constexpr int kTmemCols = 512;  // two accumulators of BN <= 256 columns
   static constexpr int kSmemBytes = kStages * kStageBytes + 1024 /*alignment*/ + 256 /*barriers*/;
-  static constexpr int kNPerTile = GATES ? BN / 3 : BN;  // output columns (hidden units) per tile
+  static constexpr int kNPerTile = NG > 0 ? BN / NG : BN;  // output columns (hidden units) per tile
 };
 
 // Epi: __device__ void operator()(uint32_t tmem_row_addr, int row, int n0, int half) const
 //   tmem_row_addr: address of (this thread's lane, first column of the accumulator)
 //   row: global output row of this thread (may be >= M: then only the tcgen05.ld's are executed)
-//   n0 : first output column (GATES: first hidden unit) of the tile
+//   n0 : first output column (NG > 0: first hidden unit) of the tile
 //   half: 0 or 1, the half of the tile's output columns this warp is responsible for
 // MNMAJ: D[m, n] = sum_k A[k, m] * B[k, n] with A stored [K, M] and B stored [K, N] (both row-major)
 // TF32: the operands are fp32 words holding tf32 values (K-major only); a k-block is 32 of them, again 128 bytes a row
-template <int BN, bool GATES, class Epi, bool MNMAJ = false, bool TF32 = false>
+template <int BN, int NG, class Epi, bool MNMAJ = false, bool TF32 = false>
 __global__ void __launch_bounds__(kThreads, 1)
 umma_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB, GemmShape sh, Epi epi,
                  int* status) {
-  using C = Cfg<BN, GATES>;
+  using C = Cfg<BN, NG>;
   extern __shared__ uint8_t smem_raw[];
   const uint32_t raw = smem_u32(smem_raw);
   const uint32_t tiles_base = (raw + 1023u) & ~1023u;
@@ -255,10 +255,10 @@ umma_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
             for (int i = 0; i < BN / 64; ++i) tma_load_2d(b_dst + i * 8192, &tmB, full_bar(stage), nt * BN + i * 64, kb * BK);
           } else {
           tma_load_2d(a_dst, &tmA, full_bar(stage), kb * kBK, mt * BM);
-          if (GATES) {
+          if (NG > 0) {
 #pragma unroll
-            for (int g = 0; g < 3; ++g)
-              tma_load_2d(b_dst + g * (C::kBBytes / 3), &tmB, full_bar(stage), kb * kBK, g * sh.gate_rows + nt * C::kNPerTile);
+            for (int g = 0; g < NG; ++g)
+              tma_load_2d(b_dst + g * (C::kBBytes / (NG > 0 ? NG : 1)), &tmB, full_bar(stage), kb * kBK, g * sh.gate_rows + nt * C::kNPerTile);
           } else {
             tma_load_2d(b_dst, &tmB, full_bar(stage), kb * kBK, nt * BN);
           }

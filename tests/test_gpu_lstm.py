@@ -1,5 +1,6 @@
-"""GPU parity of the Implicit LSTM solved by MGRIT (fp32 engine) against the fp64 oracle at the same cycle count:
-states (c, h), adjoint sensitivities, all gradients; cycle variants; the serial sweep and exact BPTT (levels = 1)."""
+"""GPU parity of the Implicit LSTM solved by MGRIT against the fp64 oracle at the same cycle count, on the fp32 engine
+and on the tensor cores (tf32 three-term split, four-gate tiles of 64 hidden units): states (c, h), adjoint
+sensitivities, all gradients; cycle variants; the serial sweep and exact BPTT (levels = 1)."""
 import numpy as np
 import pytest
 import torch
@@ -15,10 +16,14 @@ CASES = [
     dict(T=50, B=2, I=16, H=32, cf=3, levels=3, rf=0, rc=2, flags=2 | 4, cell=1),     # F-cycle, ragged T, FCFCF inside
     dict(T=32, B=2, I=16, H=32, cf=2, levels=2, rf=0, rc=1, flags=0, cell=0),         # explicit (classic) cell, gamma <= 2
     dict(T=40, B=4, I=16, H=32, cf=4, levels=1, rf=0, rc=0, flags=0, cell=1),         # serial sweep + exact BPTT
+    # tensor cores (operands = 1: tf32 split): H a multiple of 64, rows that end in a partial 128-row tile
+    dict(T=64, B=5, I=48, H=128, cf=4, levels=3, rf=0, rc=1, flags=0, cell=1, op=1),
+    dict(T=52, B=4, I=32, H=64, cf=4, levels=2, rf=1, rc=1, flags=2 | 4, cell=1, op=1),   # F-cycle, ragged T
+    dict(T=24, B=4, I=32, H=192, cf=4, levels=1, rf=0, rc=0, flags=0, cell=1, op=1),      # serial sweep + exact BPTT
 ]
 
 
-@pytest.mark.parametrize("c", CASES, ids=lambda c: "T{T}B{B}H{H}cf{cf}L{levels}r{rf}{rc}f{flags}c{cell}".format(**c))
+@pytest.mark.parametrize("c", CASES, ids=lambda c: "T{T}B{B}H{H}cf{cf}L{levels}r{rf}{rc}f{flags}c{cell}".format(**c) + f"o{c.get('op', 0)}")
 def test_lstm_solve(c):
     from paper_2203_04738_b200 import binding as B
     rng = np.random.default_rng(700 + c["T"])
@@ -30,7 +35,7 @@ def test_lstm_solve(c):
     P = [a.astype(np.float64) for a in P32]
     p = dict(zip(("W_ih", "W_hh", "b_ih", "b_hh"), [to_dev(a) for a in P32]))
     cfg = B.make_cfg(T, Bn, I, H, cf=c["cf"], levels=c["levels"], iters=2, cell=c["cell"], relax_fine=c["rf"], relax_coarse=c["rc"],
-                     operands=B.OPERANDS_FP32, flags=c["flags"])
+                     operands=c.get("op", B.OPERANDS_FP32), flags=c["flags"])
     kw = dict(cf=c["cf"], levels=c["levels"], iters=2, cell=c["cell"], relax_fine=c["rf"], relax_coarse=c["rc"],
               cycle=O.CYCLE_F if c["flags"] & 2 else O.CYCLE_V, ragged=bool(c["flags"] & 4))
     multi = c["levels"] > 1
