@@ -100,3 +100,15 @@ def test_unsupported_shapes_and_entry_points(B):
     with pytest.raises(B.MgritError) as e:
         B.stack_workspace_bytes(_cfg(B, w2, 1), 2)
     assert e.value.code == -4
+
+
+def test_medium_full_size_split_keeps_the_fp32_tolerances():
+    # third configuration's sizes (I = 1024, H = 512, B = 32, T = 1024, three levels) in the tf32 split mode: reductions of
+    # 1024 and 1536 products per output, 1024 time steps -- every element against the oracle, forward and adjoint
+    import dataclasses
+    from paper_2203_04738_b200 import binding as B
+    w = dataclasses.replace(WORKLOADS["medium"], operands=1)
+    cfg = _cfg(B, w, w.iters_fwd)
+    d, err = _forward_case(B, w, cfg)
+    print(f"medium forward max|dh| in the tf32 split mode: {err:.3e}")
+    _adjoint_case(B, w, d, cfg, w.iters_adj, seed_all=True)
