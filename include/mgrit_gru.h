@@ -120,6 +120,19 @@ typedef struct {
  * gru_serial_backward.  Either output may be NULL. */
 int mgrit_gru_workspace_bytes(const mgrit_gru_cfg* cfg, size_t* fwd_bytes, size_t* adj_bytes);
 
+/* Building blocks of a time-sharded solve (Fig. "Parallel distribution of work in parallel-in-time training": every
+ * device owns a contiguous piece of the time axis and advances its own points): one cell evaluation, or its adjoint,
+ * for n*B independent rows given as contiguous arrays.  fp32 engine (FFMA) whatever cfg->operands says; cfg supplies
+ * B, H and the cell.
+ *   gru_step_rows:          out[n,B,H] = Phi_gamma(gi_rows[n,B,3H], u_prev[n,B,H])               (Eq. "gru", "gru-imap")
+ *   gru_adjoint_step_rows:  out[n,B,H] = (dPhi_gamma/dh at (gi_rows, h_lin))^T mu[n,B,H]         (discrete adjoint of it)
+ * ws: gru_adjoint_step_rows needs 5*n*B*H floats of device workspace (ws_bytes checked); gru_step_rows none.
+ * Asynchronous on `stream`; all pointers device, 32-byte aligned. */
+int gru_step_rows(const mgrit_gru_cfg* cfg, const gru_params* p, int32_t n, float gamma, const float* gi_rows, const float* u_prev,
+                  float* out, mgrit_stream_t stream);
+int gru_adjoint_step_rows(const mgrit_gru_cfg* cfg, const gru_params* p, int32_t n, float gamma, const float* gi_rows,
+                          const float* h_lin, const float* mu, float* out, void* ws, size_t ws_bytes, mgrit_stream_t stream);
+
 /* Size in bytes of the gi buffer for this cfg: T*B*3H floats, more with MGRIT_FLAG_GI_CARRIES_COPIES (0 for a bad cfg). */
 size_t mgrit_gru_gi_bytes(const mgrit_gru_cfg* cfg);
 

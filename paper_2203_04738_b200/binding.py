@@ -61,6 +61,8 @@ lib.mgrit_lstm_workspace_bytes.argtypes = [ctypes.POINTER(Cfg), ctypes.POINTER(_
 lib.mgrit_lstm_forward.argtypes = [ctypes.POINTER(Cfg), ctypes.POINTER(_Params), _vp, _vp, _vp, _vp, ctypes.POINTER(ctypes.c_float), _vp, _sz, _vp]
 lib.mgrit_lstm_adjoint.argtypes = [ctypes.POINTER(Cfg), ctypes.POINTER(_Params), _vp, _vp, _vp, _vp, _vp, _vp, _vp, _vp, _vp,
                                    ctypes.POINTER(_Grads), ctypes.POINTER(ctypes.c_float), _vp, _sz, _vp]
+lib.gru_step_rows.argtypes = [ctypes.POINTER(Cfg), ctypes.POINTER(_Params), _i32, ctypes.c_float, _vp, _vp, _vp, _vp]
+lib.gru_adjoint_step_rows.argtypes = [ctypes.POINTER(Cfg), ctypes.POINTER(_Params), _i32, ctypes.c_float, _vp, _vp, _vp, _vp, _vp, _sz, _vp]
 lib.xent_head_workspace_bytes.argtypes = [_i32, _i32]
 lib.xent_head_workspace_bytes.restype = _sz
 lib.xent_head_fwd_bwd.argtypes = [_i32, _i32, _i32, _vp, _vp, _vp, _vp, _vp, _vp, _vp, _vp, _vp, _sz, _vp]
@@ -211,6 +213,25 @@ def mgrit_gru_adjoint(cfg, p, x, h0, gi, h, dh_seed=None, dhT=None, want_dx=True
 
 def gru_serial_backward(cfg, p, x, h0, gi, h, dh_seed=None, dhT=None, want_dx=True, ws=None, out=None, want_dh=True):
     return _adjoint(lib.gru_serial_backward, True, cfg, p, x, h0, gi, h, dh_seed, dhT, want_dx, False, ws, out, want_dh)
+
+
+def gru_step_rows(cfg, p, gamma, gi_rows, u_prev, out=None):
+    """out[n,B,H] = Phi_gamma(gi_rows[n,B,3H], u_prev[n,B,H]): one cell evaluation for n*B independent rows (fp32 engine)."""
+    n = u_prev.shape[0]
+    out = torch.empty_like(u_prev) if out is None else out
+    _check(lib.gru_step_rows(ctypes.byref(cfg), ctypes.byref(_params(p)), n, float(gamma), _f32(gi_rows), _f32(u_prev), _f32(out),
+                             _stream()))
+    return out
+
+
+def gru_adjoint_step_rows(cfg, p, gamma, gi_rows, h_lin, mu, out=None, ws=None):
+    """out[n,B,H] = (dPhi_gamma/dh at (gi_rows, h_lin))^T mu: the adjoint of gru_step_rows, row by row."""
+    n = mu.shape[0]
+    out = torch.empty_like(mu) if out is None else out
+    ws = _ws(5 * n * cfg.B * cfg.H * 4 + 5 * 256, ws, mu.device)
+    _check(lib.gru_adjoint_step_rows(ctypes.byref(cfg), ctypes.byref(_params(p)), n, float(gamma), _f32(gi_rows), _f32(h_lin),
+                                     _f32(mu), _f32(out), _ptr(ws), ws.numel(), _stream()))
+    return out
 
 
 def stack_workspace_bytes(cfg: Cfg, n_layers: int):

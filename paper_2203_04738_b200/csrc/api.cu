@@ -1165,6 +1165,58 @@ int mgrit_gru_workspace_bytes(const mgrit_gru_cfg* cfg, size_t* fwd_bytes, size_
   return MGRIT_OK;
 }
 
+int gru_step_rows(const mgrit_gru_cfg* cfg, const gru_params* p, int32_t n, float gamma, const float* gi_rows, const float* u_prev,
+                  float* out, mgrit_stream_t stream) {
+  if (!cfg || !p || !p->W_hh || !p->b_hh || !gi_rows || !u_prev || !out || n < 0) return MGRIT_INVALID_ARG;
+  if (cfg->B <= 0 || cfg->H <= 0 || cfg->H % 8 != 0 || !(gamma > 0.f)) return MGRIT_INVALID_ARG;
+  if (cfg->cell != MGRIT_CELL_CLASSIC && cfg->cell != MGRIT_CELL_IMPLICIT) return MGRIT_INVALID_ARG;
+  if (!aligned32(gi_rows, u_prev, out, p->W_hh, p->b_hh)) return MGRIT_INVALID_ARG;
+  if ((i64)n * cfg->B > (i64)INT_MAX - 1024) return MGRIT_UNSUPPORTED;
+  if (n == 0) return MGRIT_OK;
+  cudaStream_t s = (cudaStream_t)stream;
+  const i64 BH = (i64)cfg->B * cfg->H;
+  FwdStepArgs a{};
+  a.M = n * cfg->B; a.B = cfg->B; a.H = cfg->H;
+  a.hin = u_prev; a.hin_ks = BH; a.hout = out; a.hout_ks = BH;
+  a.gi = gi_rows; a.gi_ks = 3 * BH;
+  a.W_hh = p->W_hh; a.b_hh = p->b_hh; a.gamma = gamma; a.cell = cfg->cell; a.mode = 0;
+  simt_fwd_step(a, s);
+  return finish(s, false);
+}
+
+int gru_adjoint_step_rows(const mgrit_gru_cfg* cfg, const gru_params* p, int32_t n, float gamma, const float* gi_rows,
+                          const float* h_lin, const float* mu, float* out, void* ws, size_t ws_bytes, mgrit_stream_t stream) {
+  if (!cfg || !p || !p->W_hh || !p->b_hh || !gi_rows || !h_lin || !mu || !out || n < 0) return MGRIT_INVALID_ARG;
+  if (cfg->B <= 0 || cfg->H <= 0 || cfg->H % 8 != 0 || !(gamma > 0.f)) return MGRIT_INVALID_ARG;
+  if (cfg->cell != MGRIT_CELL_CLASSIC && cfg->cell != MGRIT_CELL_IMPLICIT) return MGRIT_INVALID_ARG;
+  if (!aligned32(gi_rows, h_lin, mu, out, ws, p->W_hh, p->b_hh)) return MGRIT_INVALID_ARG;
+  if ((i64)n * cfg->B > (i64)INT_MAX - 1024) return MGRIT_UNSUPPORTED;
+  if (n == 0) return MGRIT_OK;
+  const i64 BH = (i64)cfg->B * cfg->H;
+  const size_t rows = (size_t)n * BH;
+  if (!ws) return MGRIT_INVALID_ARG;
+  Ws w{(char*)ws, ws_bytes, 0};
+  float* ca = w.take<float>(rows); float* cr = w.take<float>(rows); float* cz = w.take<float>(rows);
+  float* cn = w.take<float>(rows); float* cnp = w.take<float>(rows);
+  if (!w.fits()) return MGRIT_WORKSPACE_TOO_SMALL;
+  cudaStream_t s = (cudaStream_t)stream;
+  // coefficients of the n*B steps: row (j, b) leaves the state h_lin[j] with the input projection gi_rows[j]
+  // (the level layout of the linearisation with unit stride: step j + 1 leaves fine time 1 + j)
+  LinArgs l{};
+  l.M = n * cfg->B; l.B = cfg->B; l.H = cfg->H; l.h0 = h_lin; l.h = h_lin; l.stride_t = 1; l.t0 = 1;
+  l.gi = gi_rows - 3 * BH;      // its row t + stride - 1 = j + 1 is gi_rows[j]; row 0 is never read
+  l.W_hh = p->W_hh; l.b_hh = p->b_hh; l.gamma = gamma; l.cell = cfg->cell;
+  l.a = ca; l.cr = cr; l.cz = cz; l.cn = cn; l.cnp = cnp;
+  simt_linearise(l, s);
+  AdjStepArgs a{};
+  a.M = n * cfg->B; a.B = cfg->B; a.H = cfg->H;
+  a.lin = mu; a.lin_ks = BH; a.lout = out; a.lout_ks = BH;
+  a.a = ca; a.cr = cr; a.cz = cz; a.cn = cn; a.coef_ks = BH;
+  a.W_hh = p->W_hh; a.mode = 0;
+  simt_adj_step(a, s);
+  return finish(s, false);
+}
+
 size_t mgrit_gru_gi_bytes(const mgrit_gru_cfg* cfg) {
   Hier hr;
   if (check_cfg(cfg, &hr) != MGRIT_OK) return 0;

@@ -9,9 +9,11 @@ one [B, H] slab crosses a rank boundary -- written over two injected callables:
   comm: an object with ``rank``, ``world``, ``send_right(tensor)``, ``recv_left(like)``  (torch.distributed
         send/recv in `TorchComm`; NCCL on GPUs, gloo on CPUs).
 
-No arithmetic of the method lives in this module.  On the GPUs of this build only one device is available per run,
-so the schedule is exercised with two CPU ranks over gloo (tests/test_time_shard_gloo.py); the single-GPU library
-calls (mgrit_gru_forward / mgrit_gru_adjoint) are the world = 1 case of it.
+No arithmetic of the method lives in this module.  `DeviceSteps` supplies the two callables on a GPU through the
+library's row-wise calls (gru_step_rows / gru_adjoint_step_rows), so that each rank advances its own points on its own
+device and `TorchComm` moves the slabs over NCCL.  Only one device is available per run here, so the schedule is
+exercised with two and three CPU ranks over gloo (tests/test_time_shard_gloo.py) and the device steps with one rank on
+one GPU against the library's own single-device solve (tests/test_gpu_time_shard.py).
 
 Ownership: level l has points 0..N_l and intervals of c_f points.  Rank r owns a contiguous block of whole intervals,
 i.e. the F-points of those intervals and the C-point that ENDS each of them; point 0 (the fixed end) and, for r > 0,
@@ -48,6 +50,40 @@ class TorchComm:
         buf = torch.empty_like(like)
         self.dist.recv(buf, src=self.rank - 1)
         return buf
+
+
+class LocalComm:
+    """world = 1: nothing to hand off."""
+    rank, world, slabs_sent = 0, 1, 0
+
+    def send_right(self, t):
+        pass
+
+    def recv_left(self, like):
+        return None
+
+
+class DeviceSteps:
+    """The two step callables of `sharded_cycle` on this rank's GPU (argument marshalling around the C-ABI calls).
+
+    gi: [T, B, 3H] input projection (device); hfull: [T + 1, B, H] = [h_0; h], the states the adjoint is linearised at
+    (needed for `adj` only).  Level l advances with gamma = cf^l * dt and uses the input of the fine step that arrives at
+    the same time."""
+
+    def __init__(self, binding, cfg, params, gi, hfull=None):
+        self.B, self.cfg, self.p, self.gi, self.hfull = binding, cfg, params, gi, hfull
+
+    def fwd(self, l, j, u_prev):
+        m = self.cfg.cf ** l
+        rows = self.gi[(m * j - 1).to(self.gi.device)].contiguous()
+        return self.B.gru_step_rows(self.cfg, self.p, float(m) * self.cfg.dt, rows, u_prev.contiguous())
+
+    def adj(self, l, s, mu_prev):
+        # reversed point s of level l: the forward step that arrives at fine time t = T - m (s - 1) and leaves t - m
+        m, T = self.cfg.cf ** l, self.cfg.T
+        t = (T - m * (s - 1)).to(self.gi.device)
+        return self.B.gru_adjoint_step_rows(self.cfg, self.p, float(m) * self.cfg.dt, self.gi[t - 1].contiguous(),
+                                            self.hfull[t - m].contiguous(), mu_prev.contiguous())
 
 
 @dataclass
