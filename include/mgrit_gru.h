@@ -66,9 +66,10 @@ enum {
    * t = 0, the adjoint's reversed grids at t = T (the paper always uses T = 128 = a multiple of cf^(levels-1)). */
   MGRIT_FLAG_RAGGED_T = 4,
   /* The gi buffer of mgrit_gru_forward / mgrit_gru_adjoint has mgrit_gru_gi_bytes(cfg) bytes: the projection
-   * gi[T,B,3H] followed by room for the bf16 copies of x and of [h_0; h] that the forward call makes anyway in the
-   * bf16 operand mode; the adjoint call, given the same buffer (and the h that forward call returned), reads them
-   * instead of converting x and h again.  Set it in the cfg of BOTH calls.  Ignored (and harmless) where no such
+   * gi[T,B,3H] followed by room for the bf16 copies of x, of [h_0; h] and of gi itself that the forward call makes
+   * anyway in the bf16 operand mode; the adjoint call, given the same buffer (and the h that forward call returned),
+   * reads them instead of converting x and h again, and linearises at the bf16 copy of gi (the values the forward
+   * solve used) instead of the fp32 one.  Set it in the cfg of BOTH calls.  Ignored (and harmless) where no such
    * copies exist: fp32 operands, B not dividing 128, levels == 1, the serial entry points. */
   MGRIT_FLAG_GI_CARRIES_COPIES = 8
 };

@@ -113,7 +113,7 @@ int check_cfg(const mgrit_gru_cfg* c, Hier* hr) {
 
 // With MGRIT_FLAG_GI_CARRIES_COPIES the caller's gi buffer is followed by the bf16 copies that the forward call makes
 // anyway and the adjoint call needs again: x as [T*B, I] and the level-0 state [h_0; h] as [(T+1)*B, H].
-struct GiTail { __nv_bfloat16* xb; __nv_bfloat16* hb0; size_t total_bytes; };
+struct GiTail { __nv_bfloat16* xb; __nv_bfloat16* hb0; __nv_bfloat16* gib; size_t total_bytes; };
 GiTail gi_tail(const mgrit_gru_cfg* c, float* gi) {
   const size_t TB = (size_t)c->T * c->B;
   size_t off = (TB * 3 * c->H * sizeof(float) + 255) & ~(size_t)255;
@@ -122,12 +122,21 @@ GiTail gi_tail(const mgrit_gru_cfg* c, float* gi) {
   off += (TB * c->I * sizeof(__nv_bfloat16) + 255) & ~(size_t)255;
   t.hb0 = gi ? reinterpret_cast<__nv_bfloat16*>(reinterpret_cast<char*>(gi) + off) : nullptr;
   off += ((TB + c->B) * c->H * sizeof(__nv_bfloat16) + 255) & ~(size_t)255;
+  t.gib = gi ? reinterpret_cast<__nv_bfloat16*>(reinterpret_cast<char*>(gi) + off) : nullptr;      // the projection itself as bf16
+  off += (TB * 3 * c->H * sizeof(__nv_bfloat16) + 255) & ~(size_t)255;
   t.total_bytes = off;
   return t;
 }
 // the copies exist when the tensor-core engine keeps bf16 shadows of the level states (B divides 128) in an MGRIT solve
 bool carries_copies(const mgrit_gru_cfg* c, bool serial) {
   return !serial && (c->flags & MGRIT_FLAG_GI_CARRIES_COPIES) && c->operands == MGRIT_OPERANDS_BF16 && 128 % c->B == 0 && c->levels > 1;
+}
+
+// MGRIT_GRU_GI_BF16=0 in the environment keeps the fused kernels on the fp32 input projection (A/B measurements).
+bool gi_bf16_enabled() {
+  static int v = -1;
+  if (v < 0) { const char* e = getenv("MGRIT_GRU_GI_BF16"); v = (e && e[0] == '0') ? 0 : 1; }
+  return v == 1;
 }
 
 struct FwdWs {
@@ -312,6 +321,7 @@ struct Cycle {
 
 struct FwdCycle : Cycle {
   const gru_params* p; const float* gi; UmmaFwdWs* um; FwdWs* fw;
+  const __nv_bfloat16* gib = nullptr;   // bf16 copy of gi: what every kernel of the solve reads when the state copies exist
   bool chain(int l) override {
     if (c->operands != MGRIT_OPERANDS_BF16) {     // fp32 and tf32 modes: the chain in FFMA arithmetic
       if (!fw->chain_bar) return false;
@@ -323,11 +333,12 @@ struct FwdCycle : Cycle {
       return serial32_fwd_solve(a, s);
     }
     if (!fw->chain_ub) return false;
-    SerialFwdArgs a;
+    SerialFwdArgs a{};
     a.B = c->B; a.H = c->H; a.nsteps = hr.N[l];
     a.u = U[l]; a.ub = fw->chain_ub;
     i64 st = hr.stride_t[l];
     a.gi = gi + (st - 1) * (i64)BH * 3; a.gi_step = st * (i64)BH * 3;
+    a.gi_b = gib ? gib + (st - 1) * (i64)BH * 3 : nullptr;
     a.g = G[l]; a.W = um->W_hh; a.b_hh = p->b_hh; a.gamma = hr.gamma[l]; a.cell = c->cell; a.bar = fw->chain_bar;
     a.xw = fw->chain_xw; a.xw_bytes = fw->chain_xw_bytes;
     return serial_fwd_solve(a, s);
@@ -335,13 +346,14 @@ struct FwdCycle : Cycle {
   bool launch_sweep(int l, const int* kinds, int n) override {
     const int cf = c->cf;
     if (c->operands != MGRIT_OPERANDS_BF16 || !Ub || hr.N[l] % cf != 0 || n > kMaxFwdSweepSteps) return false;
-    FwdSweepArgs a;
+    FwdSweepArgs a{};
     a.B = c->B; a.H = c->H; a.nk = hr.N[l] / cf; a.cf = cf; a.n = n;
     const size_t need = (size_t)n * (((size_t)a.nk * c->B + 127) / 128);
     if (!fw->sweep_ctr || fw->sweep_ctr_used + need > fw->sweep_ctr_n) return false;
     a.U = U[l]; a.Ub = Ub[l];
     const i64 st = hr.stride_t[l];
     a.gi = gi + (st - 1) * (i64)BH * 3; a.gi_ss = st * (i64)BH * 3; a.gi_ks = st * cf * (i64)BH * 3;
+    a.gi_b = gib ? gib + (st - 1) * (i64)BH * 3 : nullptr;
     a.g = G[l] ? G[l] + BH : nullptr;
     a.b_hh = p->b_hh; a.gamma = hr.gamma[l]; a.cell = c->cell;
     a.ctr = fw->sweep_ctr + fw->sweep_ctr_used;
@@ -369,7 +381,7 @@ struct FwdCycle : Cycle {
     return true;
   }
   int launch_step(const StepDesc& d) override {
-    FwdStepArgs a;
+    FwdStepArgs a{};
     a.M = d.nk * c->B; a.B = c->B; a.H = c->H;
     a.hin = U[d.l] + (size_t)d.in_slot * BH; a.hin_ks = (i64)d.in_stride * BH;
     a.hout = d.out + (size_t)d.out_slot * BH; a.hout_ks = (i64)d.out_stride * BH;
@@ -377,6 +389,7 @@ struct FwdCycle : Cycle {
     a.hout_b = (Ub && d.out == U[d.l]) ? Ub[d.l] + (size_t)d.out_slot * BH : nullptr;
     i64 st = hr.stride_t[d.l];
     a.gi = gi + ((i64)st * d.tgt_slot - 1) * (i64)BH * 3; a.gi_ks = st * d.tgt_stride * (i64)BH * 3;
+    a.gi_b = gib ? gib + ((i64)st * d.tgt_slot - 1) * (i64)BH * 3 : nullptr;
     a.gadd = d.gadd ? d.gadd + (size_t)d.gadd_slot * BH : nullptr; a.gadd_ks = (i64)d.gadd_stride * BH;
     a.W_hh = p->W_hh; a.b_hh = p->b_hh; a.gamma = hr.gamma[d.l]; a.cell = c->cell; a.mode = d.mode;
     if (c->operands == MGRIT_OPERANDS_BF16) return umma_fwd_step(a, um, s);
@@ -472,7 +485,9 @@ int forward_impl(const mgrit_gru_cfg* cfg_in, bool serial, const gru_params* p, 
     GiTail t = gi_tail(&c, gi);
     fw.um.xb = t.xb;
     fw.Ub[0] = t.hb0;
+    fw.um.gib = t.gib;
   }
+  if (!gi_bf16_enabled()) fw.um.gib = nullptr;
 
   if (c.operands == MGRIT_OPERANDS_BF16) {
     rc = umma_prepare_fwd(&c, p, x, gi, &fw.um, s);
@@ -496,6 +511,7 @@ int forward_impl(const mgrit_gru_cfg* cfg_in, bool serial, const gru_params* p, 
   cy.c = &c; cy.hr = hr; cy.s = s; cy.U = fw.U; cy.G = fw.G; cy.res_acc = fw.res_acc; cy.BH = BH;
   cy.p = p; cy.gi = gi; cy.um = &fw.um; cy.fw = &fw;
   cy.Ub = shadows ? fw.Ub : nullptr;
+  cy.gib = shadows ? fw.um.gib : nullptr;
   rc = cy.solve();
   if (rc) return rc;
   cudaMemcpyAsync(h, fw.U[0] + BH, sizeof(float) * (size_t)c.T * BH, cudaMemcpyDeviceToDevice, s);
@@ -534,6 +550,7 @@ int adjoint_impl(const mgrit_gru_cfg* cfg_in, bool serial, const gru_params* p, 
     aw.um.xb = t.xb;
     aw.um.hb0 = t.hb0;
     aw.um.hb = t.hb0 + BH;
+    aw.um.gib = gi_bf16_enabled() ? t.gib : nullptr;
   }
   if (bf16) {
     rc = umma_prepare_adj(&c, p, h0, h, &aw.um, copies, s);
@@ -546,12 +563,13 @@ int adjoint_impl(const mgrit_gru_cfg* cfg_in, bool serial, const gru_params* p, 
   }
   // adjoint coefficients of every level's steps at the given states (restricted by injection)
   for (int l = 0; l < hr.L; ++l) {
-    LinArgs a;
+    LinArgs a{};
     a.M = hr.N[l] * c.B; a.B = c.B; a.H = c.H; a.h0 = h0; a.h = h; a.stride_t = hr.stride_t[l]; a.gi = gi;
     a.t0 = hr.rem[l];     // the level's reversed grid is anchored at T: its forward steps arrive at t0 + stride * j
     a.W_hh = p->W_hh; a.b_hh = p->b_hh; a.gamma = hr.gamma[l]; a.cell = c.cell;
     a.a = aw.a[l]; a.cr = aw.cr[l]; a.cz = aw.cz[l]; a.cn = aw.cn[l]; a.cnp = l == 0 ? aw.cnp : nullptr;
     a.crb = aw.crb[l]; a.czb = aw.czb[l]; a.cnb = aw.cnb[l]; a.cnpb = l == 0 ? aw.cnpb : nullptr;
+    a.gi_b = (bf16 && copies) ? aw.um.gib : nullptr;
     if (bf16) {
       rc = umma_linearise(a, &aw.um, s);
       if (rc) return rc;
@@ -679,7 +697,7 @@ struct StackFwdCycle : Cycle {
     const bool bf16 = c->operands == MGRIT_OPERANDS_BF16;
     const i64 st = hr.stride_t[d.l];
     for (int k = 0; k < nl; ++k) {
-      FwdStepArgs a;
+      FwdStepArgs a{};
       a.M = M; a.B = c->B; a.H = c->H;
       a.hin = U[d.l] + ((size_t)d.in_slot * nl + k) * bh; a.hin_ks = (i64)d.in_stride * slot;
       a.hout = fw->tmpPhi; a.hout_ks = (i64)bh;            // the raw step result, rows (k, b) contiguous
@@ -896,7 +914,7 @@ int stack_adjoint_impl(const mgrit_gru_cfg* cfg, int nl, const gru_params* p, co
       }
     }
     for (int l = 0; l < hr.L; ++l) {
-      LinArgs a;
+      LinArgs a{};
       a.M = hr.N[l] * c.B; a.B = c.B; a.H = c.H; a.h0 = h0 + (size_t)k * bh; a.h = L.hk; a.stride_t = hr.stride_t[l];
       a.t0 = hr.rem[l]; a.gi = k == 0 ? gi0 : L.gik;
       a.W_hh = p[k].W_hh; a.b_hh = p[k].b_hh; a.gamma = hr.gamma[l]; a.cell = c.cell;

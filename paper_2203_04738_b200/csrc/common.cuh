@@ -93,6 +93,7 @@ struct FwdStepArgs {
   const __nv_bfloat16* hin_b;       // bf16 copy of the previous state rows (same indexing) or nullptr
   __nv_bfloat16* hout_b;            // where to write the bf16 copy of the result (same indexing) or nullptr
   const float* gi;   i64 gi_ks;     // input projection rows    gi   + k*gi_ks   + b*3H
+  const __nv_bfloat16* gi_b;        // bf16 copy of those rows (same indexing) or nullptr: what the fused tensor-core kernel stages
   const float* gadd; i64 gadd_ks;   // optional FAS term rows (same shape as hout) or nullptr
   const float* W_hh;                // [3H,H] fp32
   const float* b_hh;                // [3H]
@@ -116,6 +117,7 @@ struct FwdSweepArgs {
   int B, H, nk, cf, n;
   const float* U; const __nv_bfloat16* Ub;   // level state and its bf16 copy, from slot 0
   const float* gi; i64 gi_ss, gi_ks;         // input projection of target coordinate 0 of interval 0; element strides per slot / interval
+  const __nv_bfloat16* gi_b;                 // its bf16 copy (same indexing) or nullptr
   const float* g;                            // FAS term of target coordinate 0 of interval 0 (slots like U), or nullptr
   const float* b_hh; float gamma; int cell;
   int* ctr;                                  // n * ceil(nk*B / 128) zeroed ints
@@ -132,6 +134,7 @@ struct LinArgs {
   i64 stride_t;                     // fine steps per level step: cf^l
   i64 t0;                           // fine time the level's first step leaves from (0 unless T is ragged)
   const float* gi;                  // [T,B,3H]
+  const __nv_bfloat16* gi_b;        // its bf16 copy or nullptr (fused tensor-core kernel only)
   const float* W_hh; const float* b_hh;
   float gamma; int cell;
   float *a, *cr, *cz, *cn, *cnp;    // cnp may be nullptr (only level 0 needs it)

@@ -240,8 +240,13 @@ __global__ void __launch_bounds__(kThreads, 1) serial_fwd_kernel(SerialFwdArgs a
     bool v = idx < kRows * UNC && r < nrows;
     hp[o] = v ? __ldcg(a.u + (i64)(row0 + r) * H + u0 + i) : 0.f;
     br[o] = a.b_hh[u0 + i]; bz[o] = a.b_hh[H + u0 + i]; bn[o] = a.b_hh[2 * H + u0 + i];
-    const float* gi = a.gi + (i64)(row0 + r) * 3 * H + u0 + i;
-    pgr[o] = v ? gi[0] : 0.f; pgz[o] = v ? gi[H] : 0.f; pgn[o] = v ? gi[2 * H] : 0.f;
+    const i64 go = (i64)(row0 + r) * 3 * H + u0 + i;
+    if (a.gi_b) {
+      pgr[o] = v ? __bfloat162float(a.gi_b[go]) : 0.f; pgz[o] = v ? __bfloat162float(a.gi_b[go + H]) : 0.f;
+      pgn[o] = v ? __bfloat162float(a.gi_b[go + 2 * H]) : 0.f;
+    } else {
+      pgr[o] = v ? a.gi[go] : 0.f; pgz[o] = v ? a.gi[go + H] : 0.f; pgn[o] = v ? a.gi[go + 2 * H] : 0.f;
+    }
     pg[o] = (v && a.g) ? a.g[BH + (i64)(row0 + r) * H + u0 + i] : 0.f;
   }
   __syncthreads();
@@ -281,8 +286,12 @@ __global__ void __launch_bounds__(kThreads, 1) serial_fwd_kernel(SerialFwdArgs a
     for (int o = 0; o < OPT; ++o) {
       int idx = tid + o * kThreads, r = idx / UNC, i = idx % UNC;
       if (idx < kRows * UNC && r < nrows) {
-        const float* gi = a.gi + (i64)j * a.gi_step + (i64)(row0 + r) * 3 * H + u0 + i;
-        pgr[o] = gi[0]; pgz[o] = gi[H]; pgn[o] = gi[2 * H];
+        const i64 go = (i64)j * a.gi_step + (i64)(row0 + r) * 3 * H + u0 + i;
+        if (a.gi_b) {
+          pgr[o] = __bfloat162float(a.gi_b[go]); pgz[o] = __bfloat162float(a.gi_b[go + H]); pgn[o] = __bfloat162float(a.gi_b[go + 2 * H]);
+        } else {
+          pgr[o] = a.gi[go]; pgz[o] = a.gi[go + H]; pgn[o] = a.gi[go + 2 * H];
+        }
         if (a.g) pg[o] = a.g[(i64)(j + 1) * BH + (i64)(row0 + r) * H + u0 + i];
       }
     }

@@ -111,6 +111,16 @@ __device__ __forceinline__ void sts_bf8(uint32_t addr, const float* v) {
                "r"(*reinterpret_cast<uint32_t*>(&p1)), "r"(*reinterpret_cast<uint32_t*>(&p2)), "r"(*reinterpret_cast<uint32_t*>(&p3))
                : "memory");
 }
+// eight bf16 values from shared memory (one 16-byte load) as floats
+__device__ __forceinline__ void lds_bf8(uint32_t addr, float* v) {
+  uint32_t w[4];
+  asm volatile("ld.shared.v4.b32 {%0,%1,%2,%3}, [%4];" : "=r"(w[0]), "=r"(w[1]), "=r"(w[2]), "=r"(w[3]) : "r"(addr));
+#pragma unroll
+  for (int i = 0; i < 4; ++i) {
+    v[2 * i] = __uint_as_float(w[i] << 16);
+    v[2 * i + 1] = __uint_as_float(w[i] & 0xffff0000u);
+  }
+}
 __device__ __forceinline__ float4 lds4(uint32_t addr) {
   float4 v;
   asm volatile("ld.shared.v4.f32 {%0,%1,%2,%3}, [%4];" : "=f"(v.x), "=f"(v.y), "=f"(v.z), "=f"(v.w) : "r"(addr));
@@ -187,7 +197,10 @@ template <bool PAIR> struct Geo {
   static constexpr int kBBytes = (PAIR ? BN / 2 : BN) * BK * 2;   // weight bytes staged per CTA and k-block
   static constexpr int kStageBytes = kABytes + kBBytes;           // 31 KiB / 40 KiB (multiples of 1 KiB)
 };
-template <bool HAS_G, bool LIN = false, bool PAIR = false> struct CellCfg {
+// GIB: the input projection is staged from its bf16 copy (rows of 32 bytes, 32-byte swizzle) instead of fp32: 10 instead of
+// 16 bytes per element of epilogue operands, and a third operand buffer fits.  What hides the latency of those loads is
+// the bytes in flight, and shared memory bounds them: a tile needs 128 x UN x (bytes per element) per main-loop time.
+template <bool HAS_G, bool LIN = false, bool PAIR = false, bool GIB = false> struct CellCfg {
   using G = Geo<PAIR>;
 #ifndef CELL_PAIR_STAGES
 #define CELL_PAIR_STAGES ((HAS_G || LIN) ? 4 : 5)
@@ -196,16 +209,16 @@ template <bool HAS_G, bool LIN = false, bool PAIR = false> struct CellCfg {
 #define CELL_PAIR_EBUFS 2
 #endif
   static constexpr int kStages = PAIR ? CELL_PAIR_STAGES : ((HAS_G || LIN) ? 3 : 4);
-  static constexpr int kEpiBufs = PAIR ? CELL_PAIR_EBUFS : 2;     // epilogue-operand chunks in flight
-  static constexpr int kOps = HAS_G ? 5 : 4;
-  static constexpr int kEpiBytes = kOps * kOpBytes;
+  static constexpr int kEpiBufs = GIB ? 3 : (PAIR ? CELL_PAIR_EBUFS : 2);     // epilogue-operand chunks in flight
+  static constexpr int kGiBytes = GIB ? BM * CH * 2 : kOpBytes;   // one gate's chunk of the input projection
+  static constexpr int kEpiBytes = 3 * kGiBytes + (HAS_G ? 2 : 1) * kOpBytes;   // gi r | z | n, previous state, additive term
   static constexpr int kOutBytes = LIN ? 4 * kCoefBytes : 0;      // per buffer
   static constexpr int kSmemBytes = kStages * G::kStageBytes + kEpiBufs * kEpiBytes + 2 * kOutBytes + 1024 + 256;
   static_assert(kSmemBytes + 1536 <= 232448, "shared memory budget (dynamic + static <= 227 KiB)");
 };
 }  // namespace cellk
 
-template <bool LIN, bool HAS_G, bool PAIR>
+template <bool LIN, bool HAS_G, bool PAIR, bool GIB = false>
 __global__ void __launch_bounds__(cellk::kThreads, 1)
 umma_cell_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB,
                  const __grid_constant__ CUtensorMap tmGI, const __grid_constant__ CUtensorMap tmHP,
@@ -213,7 +226,8 @@ umma_cell_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
                  const __grid_constant__ CUtensorMap tmCZ, const __grid_constant__ CUtensorMap tmCN,
                  const __grid_constant__ CUtensorMap tmCP, CellArgs p, const __grid_constant__ SweepArgs swp, int* status) {
   using namespace cellk;
-  using C = CellCfg<HAS_G, LIN, PAIR>;
+  using C = CellCfg<HAS_G, LIN, PAIR, GIB>;
+  constexpr int kGi = C::kGiBytes;
   using G = Geo<PAIR>;
   constexpr int UN = G::UN, BN = G::BN, NCH = G::NCH, kStageBytes = G::kStageBytes;
   extern __shared__ uint8_t smem_raw[];
@@ -377,15 +391,15 @@ umma_cell_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
           mbar_expect_tx(efull_bar(eb), C::kEpiBytes);
           if (LIN) {
             tma_load_3d(dst, &tmGI, efull_bar(eb), u, 0, k0);
-            tma_load_3d(dst + kOpBytes, &tmGI, efull_bar(eb), H + u, 0, k0);
-            tma_load_3d(dst + 2 * kOpBytes, &tmGI, efull_bar(eb), 2 * H + u, 0, k0);
-            tma_load_3d(dst + 3 * kOpBytes, &tmHP, efull_bar(eb), u, 0, k0);
+            tma_load_3d(dst + kGi, &tmGI, efull_bar(eb), H + u, 0, k0);
+            tma_load_3d(dst + 2 * kGi, &tmGI, efull_bar(eb), 2 * H + u, 0, k0);
+            tma_load_3d(dst + 3 * kGi, &tmHP, efull_bar(eb), u, 0, k0);
           } else {
             tma_load_4d(dst, &tmGI, efull_bar(eb), u, 0, tgt_s, k0);
-            tma_load_4d(dst + kOpBytes, &tmGI, efull_bar(eb), H + u, 0, tgt_s, k0);
-            tma_load_4d(dst + 2 * kOpBytes, &tmGI, efull_bar(eb), 2 * H + u, 0, tgt_s, k0);
-            tma_load_4d(dst + 3 * kOpBytes, &tmHP, efull_bar(eb), u, 0, in_s, k0);
-            if (HAS_G) tma_load_4d(dst + 4 * kOpBytes, &tmG, efull_bar(eb), u, 0, tgt_s, k0);
+            tma_load_4d(dst + kGi, &tmGI, efull_bar(eb), H + u, 0, tgt_s, k0);
+            tma_load_4d(dst + 2 * kGi, &tmGI, efull_bar(eb), 2 * H + u, 0, tgt_s, k0);
+            tma_load_4d(dst + 3 * kGi, &tmHP, efull_bar(eb), u, 0, in_s, k0);
+            if (HAS_G) tma_load_4d(dst + 3 * kGi + kOpBytes, &tmG, efull_bar(eb), u, 0, tgt_s, k0);
           }
           if (++eb == C::kEpiBufs) { eb = 0; ephase ^= 1u; }
         }
@@ -425,12 +439,16 @@ umma_cell_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
         if (ok) {
         const uint32_t src = epi_base + eb * C::kEpiBytes;
         float gr[8], gz[8], gn[8], hp[8], gg[8];
-        *reinterpret_cast<float4*>(gr) = lds4(src + off0);                 *reinterpret_cast<float4*>(gr + 4) = lds4(src + off1);
-        *reinterpret_cast<float4*>(gz) = lds4(src + kOpBytes + off0);      *reinterpret_cast<float4*>(gz + 4) = lds4(src + kOpBytes + off1);
-        *reinterpret_cast<float4*>(gn) = lds4(src + 2 * kOpBytes + off0);  *reinterpret_cast<float4*>(gn + 4) = lds4(src + 2 * kOpBytes + off1);
-        *reinterpret_cast<float4*>(hp) = lds4(src + 3 * kOpBytes + off0);  *reinterpret_cast<float4*>(hp + 4) = lds4(src + 3 * kOpBytes + off1);
+        if (GIB) {       // eight bf16 values per gate: one 16-byte load each (32-byte rows, 32-byte swizzle)
+          lds_bf8(src + offb, gr); lds_bf8(src + kGi + offb, gz); lds_bf8(src + 2 * kGi + offb, gn);
+        } else {
+          *reinterpret_cast<float4*>(gr) = lds4(src + off0);            *reinterpret_cast<float4*>(gr + 4) = lds4(src + off1);
+          *reinterpret_cast<float4*>(gz) = lds4(src + kGi + off0);      *reinterpret_cast<float4*>(gz + 4) = lds4(src + kGi + off1);
+          *reinterpret_cast<float4*>(gn) = lds4(src + 2 * kGi + off0);  *reinterpret_cast<float4*>(gn + 4) = lds4(src + 2 * kGi + off1);
+        }
+        *reinterpret_cast<float4*>(hp) = lds4(src + 3 * kGi + off0);  *reinterpret_cast<float4*>(hp + 4) = lds4(src + 3 * kGi + off1);
         if (HAS_G) {
-          *reinterpret_cast<float4*>(gg) = lds4(src + 4 * kOpBytes + off0); *reinterpret_cast<float4*>(gg + 4) = lds4(src + 4 * kOpBytes + off1);
+          *reinterpret_cast<float4*>(gg) = lds4(src + 3 * kGi + kOpBytes + off0); *reinterpret_cast<float4*>(gg + 4) = lds4(src + 3 * kGi + kOpBytes + off1);
         }
         const int cu = c * CH + half * 8;       // first of this thread's 8 units inside the tile
         float ar[8], az[8], an[8];

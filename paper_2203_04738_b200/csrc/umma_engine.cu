@@ -212,23 +212,25 @@ bool make_map4(CUtensorMap* m, CUtensorMapDataType dt, size_t esize, const void*
 // Adjoint linearisation on the fused kernel, TMA-staged epilogue operands.
 // Rows (k, b), k = 0..nk-1: A rows at A + k*a_ks + b*H (bf16), gi rows at gi + k*gi_ks + b*3H,
 // previous state at hp + k*hp_ks + b*H.
-template <bool PAIR>
-bool launch_lin_geo(int kc, const bf16* A, i64 a_ks, const float* gi, i64 gi_ks, const float* hp, i64 hp_ks, int nk, const bf16* W,
+template <bool PAIR, bool GIB>
+bool launch_lin_geo(int kc, const bf16* A, i64 a_ks, const void* gi, i64 gi_ks, const float* hp, i64 hp_ks, int nk, const bf16* W,
                     CellArgs ca, cudaStream_t s) {
-  using C = cellk::CellCfg<false, true, PAIR>;
+  using C = cellk::CellCfg<false, true, PAIR, GIB>;
   using G = cellk::Geo<PAIR>;
   if (nk <= 0) return true;
   int* const status = status_ptr();
   if (!status) return false;
   static bool attr_set[kMaxDevices] = {false};
-  auto kern = umma_cell_kernel<true, false, PAIR>;
+  auto kern = umma_cell_kernel<true, false, PAIR, GIB>;
   if (!set_smem_once(kern, C::kSmemBytes, attr_set)) return false;
   const int B = ca.B, H = ca.H, kt = 128 / B;
   ca.kt = kt; ca.M = nk * B;
   CUtensorMap ta, tb, tgi, thp;
   if (!make_map3(&ta, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, A, H, B, nk, H, a_ks, BK, kt, CU_TENSOR_MAP_SWIZZLE_128B)) return false;
   if (!make_map(&tb, W, (uint64_t)H, (uint64_t)3 * H, (uint64_t)H, G::kBox)) return false;
-  if (!make_map3(&tgi, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 4, gi, 3 * H, B, nk, 3 * H, gi_ks, cellk::CH, kt, CU_TENSOR_MAP_SWIZZLE_64B)) return false;
+  if (GIB ? !make_map3(&tgi, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, gi, 3 * H, B, nk, 3 * H, gi_ks, cellk::CH, kt, CU_TENSOR_MAP_SWIZZLE_32B)
+          : !make_map3(&tgi, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 4, gi, 3 * H, B, nk, 3 * H, gi_ks, cellk::CH, kt, CU_TENSOR_MAP_SWIZZLE_64B))
+    return false;
   if (!make_map3(&thp, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 4, hp, H, B, nk, H, hp_ks, cellk::CH, kt, CU_TENSOR_MAP_SWIZZLE_64B)) return false;
   // the four bf16 coefficient arrays [M, H] are written by TMA stores of [128 x 16] tiles
   CUtensorMap tcr = thp, tcz = thp, tcn = thp, tcp = thp;
@@ -253,10 +255,14 @@ bool launch_lin_geo(int kc, const bf16* A, i64 a_ks, const float* gi, i64 gi_ks,
   count_launch();
   return true;
 }
-bool launch_lin(int kc, const bf16* A, i64 a_ks, const float* gi, i64 gi_ks, const float* hp, i64 hp_ks, int nk, const bf16* W, CellArgs ca,
-                cudaStream_t s) {
-  if (cell_pair_enabled(nk * ca.B, ca.H)) return launch_lin_geo<true>(kc, A, a_ks, gi, gi_ks, hp, hp_ks, nk, W, ca, s);
-  return launch_lin_geo<false>(kc, A, a_ks, gi, gi_ks, hp, hp_ks, nk, W, ca, s);
+// gi: fp32 rows, or (gib) their bf16 copy with the same element indexing
+bool launch_lin(int kc, const bf16* A, i64 a_ks, const void* gi, bool gib, i64 gi_ks, const float* hp, i64 hp_ks, int nk, const bf16* W,
+                CellArgs ca, cudaStream_t s) {
+  const bool pair = cell_pair_enabled(nk * ca.B, ca.H);
+  if (gib) return pair ? launch_lin_geo<true, true>(kc, A, a_ks, gi, gi_ks, hp, hp_ks, nk, W, ca, s)
+                       : launch_lin_geo<false, true>(kc, A, a_ks, gi, gi_ks, hp, hp_ks, nk, W, ca, s);
+  return pair ? launch_lin_geo<true, false>(kc, A, a_ks, gi, gi_ks, hp, hp_ks, nk, W, ca, s)
+              : launch_lin_geo<false, false>(kc, A, a_ks, gi, gi_ks, hp, hp_ks, nk, W, ca, s);
 }
 
 // Forward steps on the fused kernel: one launch runs sw.n_steps dependent steps over the same rows (k, b), k = 0..nk-1.
@@ -265,16 +271,17 @@ bool launch_lin(int kc, const bf16* A, i64 a_ks, const float* gi, i64 gi_ks, con
 struct CellFwdOperands {
   const bf16* A; const float* hp; i64 in_ss, in_ks; int in_slots;
   const float* gi; i64 gi_ss, gi_ks; const float* g; i64 g_ss, g_ks; int tgt_slots;
+  const bf16* gi_b;      // bf16 copy of gi (same element indexing) or nullptr: staged instead of the fp32 rows
 };
-template <bool HAS_G, bool PAIR>
+template <bool HAS_G, bool PAIR, bool GIB>
 bool launch_fwd_geo(int kc, const CellFwdOperands& o, int nk, const bf16* W, CellArgs ca, const SweepArgs& sw, cudaStream_t s) {
-  using C = cellk::CellCfg<HAS_G, false, PAIR>;
+  using C = cellk::CellCfg<HAS_G, false, PAIR, GIB>;
   using G = cellk::Geo<PAIR>;
   if (nk <= 0) return true;
   int* const status = status_ptr();
   if (!status) return false;
   static bool attr_set[kMaxDevices] = {false};
-  auto kern = umma_cell_kernel<false, HAS_G, PAIR>;
+  auto kern = umma_cell_kernel<false, HAS_G, PAIR, GIB>;
   if (!set_smem_once(kern, C::kSmemBytes, attr_set)) return false;
   const int B = ca.B, H = ca.H, kt = 128 / B;
   ca.kt = kt; ca.M = nk * B;
@@ -282,7 +289,10 @@ bool launch_fwd_geo(int kc, const CellFwdOperands& o, int nk, const bf16* W, Cel
   const auto f32 = CU_TENSOR_MAP_DATA_TYPE_FLOAT32;
   if (!make_map4(&ta, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, o.A, H, B, o.in_slots, nk, H, o.in_ss, o.in_ks, BK, kt, CU_TENSOR_MAP_SWIZZLE_128B)) return false;
   if (!make_map(&tb, W, (uint64_t)H, (uint64_t)3 * H, (uint64_t)H, G::kBox)) return false;
-  if (!make_map4(&tgi, f32, 4, o.gi, 3 * H, B, o.tgt_slots, nk, 3 * H, o.gi_ss, o.gi_ks, cellk::CH, kt, CU_TENSOR_MAP_SWIZZLE_64B)) return false;
+  if (GIB ? !make_map4(&tgi, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, o.gi_b, 3 * H, B, o.tgt_slots, nk, 3 * H, o.gi_ss, o.gi_ks, cellk::CH, kt,
+                       CU_TENSOR_MAP_SWIZZLE_32B)
+          : !make_map4(&tgi, f32, 4, o.gi, 3 * H, B, o.tgt_slots, nk, 3 * H, o.gi_ss, o.gi_ks, cellk::CH, kt, CU_TENSOR_MAP_SWIZZLE_64B))
+    return false;
   if (!make_map4(&thp, f32, 4, o.hp, H, B, o.in_slots, nk, H, o.in_ss, o.in_ks, cellk::CH, kt, CU_TENSOR_MAP_SWIZZLE_64B)) return false;
   if (HAS_G) {
     if (!make_map4(&tg, f32, 4, o.g, H, B, o.tgt_slots, nk, H, o.g_ss, o.g_ks, cellk::CH, kt, CU_TENSOR_MAP_SWIZZLE_64B)) return false;
@@ -307,8 +317,9 @@ bool launch_fwd_geo(int kc, const CellFwdOperands& o, int nk, const bf16* W, Cel
 }
 template <bool HAS_G>
 bool launch_fwd(int kc, const CellFwdOperands& o, int nk, const bf16* W, const CellArgs& ca, const SweepArgs& sw, cudaStream_t s) {
-  if (cell_pair_enabled(nk * ca.B, ca.H)) return launch_fwd_geo<HAS_G, true>(kc, o, nk, W, ca, sw, s);
-  return launch_fwd_geo<HAS_G, false>(kc, o, nk, W, ca, sw, s);
+  const bool pair = cell_pair_enabled(nk * ca.B, ca.H);
+  if (o.gi_b) return pair ? launch_fwd_geo<HAS_G, true, true>(kc, o, nk, W, ca, sw, s) : launch_fwd_geo<HAS_G, false, true>(kc, o, nk, W, ca, sw, s);
+  return pair ? launch_fwd_geo<HAS_G, true, false>(kc, o, nk, W, ca, sw, s) : launch_fwd_geo<HAS_G, false, false>(kc, o, nk, W, ca, sw, s);
 }
 
 // ---------------------------------------------------------------- epilogues (one output row per thread)
@@ -347,8 +358,8 @@ __device__ __forceinline__ void st4(float* p, float a, float b, float c, float d
 }
 __device__ __forceinline__ float f4get(const float4& v, int e) { return e == 0 ? v.x : (e == 1 ? v.y : (e == 2 ? v.z : v.w)); }
 
-struct EpiBias {  // out[m, n] = acc + bias[n]      (input projection)
-  float* out; i64 ld; const float* bias; int M, N;
+struct EpiBias {  // out[m, n] = acc + bias[n]      (input projection); outb: optional bf16 copy of the same values
+  float* out; i64 ld; const float* bias; int M, N; bf16* outb;
   __device__ void operator()(uint32_t taddr, int row, int n0, int half) const {
     const bool valid = row < M;
     float* o = out + (i64)row * ld + n0;
@@ -365,6 +376,14 @@ struct EpiBias {  // out[m, n] = acc + bias[n]      (input projection)
         }
         st8(o + c0, v);
         st8(o + c0 + 8, v + 8);
+        if (outb) {
+          const uint2 p0 = pack4(make_float4(v[0], v[1], v[2], v[3])), p1 = pack4(make_float4(v[4], v[5], v[6], v[7]));
+          const uint2 p2 = pack4(make_float4(v[8], v[9], v[10], v[11])), p3 = pack4(make_float4(v[12], v[13], v[14], v[15]));
+          // sixteen bf16 values = one 32-byte store (a whole sector of this thread's row)
+          asm volatile("st.global.v8.b32 [%0], {%1,%2,%3,%4,%5,%6,%7,%8};" ::"l"(outb + (i64)row * ld + n0 + c0), "r"(p0.x), "r"(p0.y), "r"(p1.x),
+                       "r"(p1.y), "r"(p2.x), "r"(p2.y), "r"(p3.x), "r"(p3.y)
+                       : "memory");
+        }
       }
     }
   }
@@ -717,6 +736,7 @@ void umma_plan_fwd(const mgrit_gru_cfg* c, const int* N, int L, char* base, size
   o->W_ih = take<bf16>(base, off, (size_t)3 * c->H * c->I);
   o->xb = take<bf16>(base, off, (size_t)c->T * c->B * c->I);
   o->Apack = take<bf16>(base, off, o->maxM * c->H);
+  o->gib = take<bf16>(base, off, (size_t)c->T * c->B * 3 * c->H);
 }
 
 void umma_plan_adj(const mgrit_gru_cfg* c, const int* N, int L, char* base, size_t* off, UmmaAdjWs* o) {
@@ -734,6 +754,7 @@ void umma_plan_adj(const mgrit_gru_cfg* c, const int* N, int L, char* base, size
   o->xb = take<bf16>(base, off, I * TB);
   o->hb0 = take<bf16>(base, off, (size_t)c->B * H + TB * H);   // [h_0; h] contiguous: rows (t, b) of h_{t-1} start at hb0
   o->hb = o->hb0 ? o->hb0 + (size_t)c->B * H : nullptr;
+  o->gib = nullptr;
 }
 
 int umma_prepare_fwd(const mgrit_gru_cfg* c, const gru_params* p, const float* x, float* gi, UmmaFwdWs* w, cudaStream_t s) {
@@ -744,8 +765,8 @@ int umma_prepare_fwd(const mgrit_gru_cfg* c, const gru_params* p, const float* x
   convert(x, w->xb, TB * I, s);
   // gi = x W_ih^T + b_ih :  M = T*B, N = 3H, K = I
   if (gemm_pair_enabled((int)TB, 3 * H)
-          ? !launch_gemm_pair(KC_PROJ, w->xb, I, w->W_ih, I, (int)TB, 3 * H, I, 3 * H, EpiBias{gi, 3 * H, p->b_ih, (int)TB, 3 * H}, s)
-          : !launch_gemm<256, 0>(KC_PROJ, w->xb, I, w->W_ih, I, (int)TB, 3 * H, I, 0, 3 * H, EpiBias{gi, 3 * H, p->b_ih, (int)TB, 3 * H}, s))
+          ? !launch_gemm_pair(KC_PROJ, w->xb, I, w->W_ih, I, (int)TB, 3 * H, I, 3 * H, EpiBias{gi, 3 * H, p->b_ih, (int)TB, 3 * H, w->gib}, s)
+          : !launch_gemm<256, 0>(KC_PROJ, w->xb, I, w->W_ih, I, (int)TB, 3 * H, I, 0, 3 * H, EpiBias{gi, 3 * H, p->b_ih, (int)TB, 3 * H, w->gib}, s))
     return MGRIT_CUDA_ERROR;
   return MGRIT_OK;
 }
@@ -775,7 +796,7 @@ int umma_fwd_step(const FwdStepArgs& a, UmmaFwdWs* w, cudaStream_t s) {
     sw.st[0].hout = a.hout; sw.st[0].hout_ks = a.hout_ks; sw.st[0].hout_b = a.hout_b;
     CellFwdOperands o{};
     o.A = a.hin_b; o.hp = a.hin; o.in_ks = a.hin_ks; o.in_slots = 1;
-    o.gi = a.gi; o.gi_ks = a.gi_ks; o.tgt_slots = 1;
+    o.gi = a.gi; o.gi_b = a.gi_b; o.gi_ks = a.gi_ks; o.tgt_slots = 1;
     // in mode 1 the previous content of the destination plays the role of the additive term
     if (a.mode == 1) { o.g = a.hout; o.g_ks = a.hout_ks; }
     else { o.g = a.gadd; o.g_ks = a.gadd_ks; }
@@ -811,7 +832,7 @@ int umma_fwd_sweep(const FwdSweepArgs& a, UmmaFwdWs* w, cudaStream_t s) {
   }
   CellFwdOperands o{};
   o.A = a.Ub; o.hp = a.U; o.in_ss = BH; o.in_ks = (i64)a.cf * BH; o.in_slots = a.cf;
-  o.gi = a.gi; o.gi_ss = a.gi_ss; o.gi_ks = a.gi_ks; o.tgt_slots = a.cf;
+  o.gi = a.gi; o.gi_b = a.gi_b; o.gi_ss = a.gi_ss; o.gi_ks = a.gi_ks; o.tgt_slots = a.cf;
   o.g = a.g; o.g_ss = BH; o.g_ks = (i64)a.cf * BH;
   const bool ok = a.g ? launch_fwd<true>(KC_FWD_STEP, o, a.nk, w->W_hh, ca, sw, s) : launch_fwd<false>(KC_FWD_STEP, o, a.nk, w->W_hh, ca, sw, s);
   return ok ? MGRIT_OK : MGRIT_CUDA_ERROR;
@@ -823,21 +844,24 @@ int umma_linearise(const LinArgs& a, UmmaAdjWs* w, cudaStream_t s) {
   const i64 BH = (i64)a.B * a.H;
   const int N = a.M / a.B;
   const float* gi0 = a.gi + (a.t0 + a.stride_t - 1) * BH * 3;       // input of the fine step that arrives with step 1
+  const bf16* gib0 = a.gi_b ? a.gi_b + (a.t0 + a.stride_t - 1) * BH * 3 : nullptr;   // ... in the bf16 copy
   if (128 % a.B == 0) {
     CellArgs ca{};
     ca.B = a.B; ca.H = a.H; ca.b_hh = a.b_hh; ca.gamma = a.gamma; ca.cell = a.cell;
     ca.a = a.a; ca.cr = a.crb; ca.cz = a.czb; ca.cn = a.cnb; ca.cnp = a.cnpb;
     int done = 0;
     if (a.t0 == 0) {   // step 1 starts from h_0 (its own array)
-      if (!launch_lin(KC_LINEARISE, w->hb0, 0, gi0, 0, a.h0, 0, 1, w->W_hh, ca, s)) return MGRIT_CUDA_ERROR;
+      if (!launch_lin(KC_LINEARISE, w->hb0, 0, gib0 ? (const void*)gib0 : (const void*)gi0, gib0 != nullptr, 0, a.h0, 0, 1, w->W_hh, ca, s))
+        return MGRIT_CUDA_ERROR;
       done = 1;
     }
     if (N > done) {
       const i64 off = (i64)done * BH;
       ca.a = a.a + off; ca.cr = a.crb + off; ca.cz = a.czb + off; ca.cn = a.cnb + off; ca.cnp = a.cnpb ? a.cnpb + off : nullptr;
       const i64 t1 = a.t0 + (i64)done * a.stride_t;                  // fine time the first of these steps leaves from (>= 1)
-      if (!launch_lin(KC_LINEARISE, w->hb0 + t1 * BH, a.stride_t * BH, gi0 + (i64)done * a.stride_t * BH * 3, a.stride_t * BH * 3,
-                      a.h + (t1 - 1) * BH, a.stride_t * BH, N - done, w->W_hh, ca, s))
+      const i64 goff = (i64)done * a.stride_t * BH * 3;
+      if (!launch_lin(KC_LINEARISE, w->hb0 + t1 * BH, a.stride_t * BH, gib0 ? (const void*)(gib0 + goff) : (const void*)(gi0 + goff),
+                      gib0 != nullptr, a.stride_t * BH * 3, a.h + (t1 - 1) * BH, a.stride_t * BH, N - done, w->W_hh, ca, s))
         return MGRIT_CUDA_ERROR;
     }
     return MGRIT_OK;

@@ -9,6 +9,7 @@ struct UmmaFwdWs {
   __nv_bfloat16* W_ih;   // [3H,I]
   __nv_bfloat16* xb;     // [T*B,I]
   __nv_bfloat16* Apack;  // [maxM,H]  A operand of one step (rows gathered from the level state)
+  __nv_bfloat16* gib;    // [T*B,3H]  bf16 copy of the input projection, written by the projection's epilogue
   size_t maxM;
 };
 
@@ -23,6 +24,7 @@ struct UmmaAdjWs {
   __nv_bfloat16* xb;      // [T*B,I]   bf16 copy of the layer input
   __nv_bfloat16* hb0;     // [(T+1)*B,H] bf16 copy of [h_0; h]: row (t,b) is h_{t-1} of step t
   __nv_bfloat16* hb;      // = hb0 + B*H: the given states
+  const __nv_bfloat16* gib;  // bf16 copy of the input projection left by the forward call, or nullptr
   size_t maxM;
 };
 

@@ -237,9 +237,11 @@ def test_run_to_run_bit_identical_and_workspace_content_irrelevant(B):
     assert B.last_device_status() == 0
 
 
-def test_copies_carried_behind_gi_give_the_same_bits(B):
-    # FLAG_GI_CARRIES_COPIES only moves where the bf16 copies of x and [h_0; h] live: every output must keep its bits,
-    # also with the larger buffer poisoned beforehand; a case without shadows (B does not divide 128) ignores the flag.
+def test_copies_carried_behind_gi_change_nothing_but_rounding(B):
+    # FLAG_GI_CARRIES_COPIES moves where the bf16 copies of x, [h_0; h] and gi live: the forward outputs keep their bits
+    # (also with the larger buffer poisoned beforehand); the adjoint then linearises at the bf16 copy of gi, the values the
+    # forward solve itself used, instead of the fp32 projection, so its outputs move by that rounding and no more.  A case
+    # without state copies (B does not divide 128) ignores the flag and keeps every bit.
     for Bsz in (32, 24):
         w = Workload("carry", T=256, B=Bsz, I=64, H=256, cf=4, levels=3, iters_fwd=2, iters_adj=2, relax_fine=0, relax_coarse=1,
                      operands=2, classes=8, relu=True, seed=11)
@@ -255,5 +257,11 @@ def test_copies_carried_behind_gi_give_the_same_bits(B):
         assert gi2 is buf and torch.equal(B.gi_view(carry, buf), gi) and torch.equal(h2, h)
         r2 = B.mgrit_gru_adjoint(carry, p, x, h0, buf, h2, dhT=h2[-1].contiguous())
         for k in ("dh", "dh0", "dx", "dW_ih", "dW_hh", "db_ih", "db_hh"):
-            assert torch.equal(getattr(r, k), getattr(r2, k)), k
+            a, b = getattr(r, k), getattr(r2, k)
+            if Bsz == 24:
+                assert torch.equal(a, b), k
+            else:
+                # (dh0 has decayed by orders of magnitude over the sequence: compared on the scale of dh)
+                scale = float(r.dh.abs().max()) if k == "dh0" else float(a.abs().max())
+                assert float((a - b).abs().max()) <= 5e-3 * scale, k
     assert B.last_device_status() == 0
