@@ -24,12 +24,11 @@ sys.path.insert(0, ROOT)
 METRIC = "MGRIT-GRU fwd+adjoint timesteps*batch/sec"
 UNIT = "timesteps*batch/s"
 # DRAM bytes (dram__bytes_read.sum + dram__bytes_write.sum) of the fused forward-step kernel per (row x hidden
-# unit).  These are constants taken from `ncu --set full --clock-control none` captures of two launches of that
-# kernel, NOT measured in a bench run: 23.2 B on the default workload's own 16384-row launches (389 MB per launch,
-# H = 1024) and 19.5 B on the smaller `medium` case (81.7 MB for 8192 rows x 512 units, where more of the previous
-# step's output is still in L2).  Traffic grows in proportion to rows x hidden units, so a workload's per-launch
-# traffic is its figure x its average rows x H.
-NCU_DRAM_BYTES_PER_ROW_UNIT = {"forward_step": {1024: 23.2, 512: 19.5}}
+# unit).  A constant taken from an `ncu --set full --clock-control none` capture of that kernel, NOT measured in a
+# bench run: 17.4 B on the default workload's own level-0 sweep (four dependent steps of 16384 rows in one launch,
+# H = 1024: 1166 MB).  Traffic grows in proportion to rows x hidden units, so a workload's per-launch traffic is this
+# figure x the rows x H its launches process.
+NCU_DRAM_BYTES_PER_ROW_UNIT = {"forward_step": {1024: 17.4}}
 NOMINAL_BF16_TFLOPS = 2250.0       # dense bf16, vendor figure (context only)
 
 
@@ -431,7 +430,8 @@ def main():
                         # 16H + 4H/(cf-1) bytes; this implementation also writes and reads a bf16 copy of the state
                         # and re-reads the fp32 state every step: 24H bytes
                         "algorithmic_bytes": (16.0 + 4.0 / (w.cf - 1)) * units if name == "forward_step" else None,
-                        "implementation_bytes": 24.0 * units if name == "forward_step" else None,
+                        # input projection 6 (bf16 copy), previous state 4 + 2 (its bf16 copy), new state 4 + 2
+                        "implementation_bytes": 18.0 * units if name == "forward_step" else None,
                         "avg_launch_us": tms / n * 1e3, "launches_per_step": n // nprof,
                         "share_of_gemm_time": tms / max(sum(v[0] for v in prof.values()), 1e-9), "peak_source": note}
         roofline_by_class = {k: {"tflops": v[2] / (v[0] * 1e-3) / 1e12, "frac_sustained": v[2] / (v[0] * 1e-3) / 1e12 / peak,

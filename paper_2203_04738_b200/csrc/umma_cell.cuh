@@ -202,14 +202,20 @@ template <bool PAIR> struct Geo {
 // the bytes in flight, and shared memory bounds them: a tile needs 128 x UN x (bytes per element) per main-loop time.
 template <bool HAS_G, bool LIN = false, bool PAIR = false, bool GIB = false> struct CellCfg {
   using G = Geo<PAIR>;
+#ifndef CELL_PAIR_STAGES_PLAIN
+#define CELL_PAIR_STAGES_PLAIN 5
+#endif
 #ifndef CELL_PAIR_STAGES
-#define CELL_PAIR_STAGES ((HAS_G || LIN) ? 4 : 5)
+#define CELL_PAIR_STAGES ((HAS_G || LIN) ? 4 : CELL_PAIR_STAGES_PLAIN)
 #endif
 #ifndef CELL_PAIR_EBUFS
 #define CELL_PAIR_EBUFS 2
 #endif
   static constexpr int kStages = PAIR ? CELL_PAIR_STAGES : ((HAS_G || LIN) ? 3 : 4);
-  static constexpr int kEpiBufs = GIB ? 3 : (PAIR ? CELL_PAIR_EBUFS : 2);     // epilogue-operand chunks in flight
+#ifndef CELL_GIB_EBUFS
+#define CELL_GIB_EBUFS 3
+#endif
+  static constexpr int kEpiBufs = GIB ? ((PAIR && !HAS_G && !LIN) ? CELL_GIB_EBUFS : 3) : (PAIR ? CELL_PAIR_EBUFS : 2);     // epilogue-operand chunks in flight
   static constexpr int kGiBytes = GIB ? BM * CH * 2 : kOpBytes;   // one gate's chunk of the input projection
   static constexpr int kEpiBytes = 3 * kGiBytes + (HAS_G ? 2 : 1) * kOpBytes;   // gi r | z | n, previous state, additive term
   static constexpr int kOutBytes = LIN ? 4 * kCoefBytes : 0;      // per buffer
