@@ -83,6 +83,12 @@ __device__ __forceinline__ void tmem_ld_wait8x3(float* a, float* b, float* c) {
                :
                : "memory");
 }
+__device__ __forceinline__ void tmem_ld_wait8(float* a) {
+  asm volatile("tcgen05.wait::ld.sync.aligned;"
+               : "+f"(a[0]), "+f"(a[1]), "+f"(a[2]), "+f"(a[3]), "+f"(a[4]), "+f"(a[5]), "+f"(a[6]), "+f"(a[7])
+               :
+               : "memory");
+}
 __device__ __forceinline__ void tmem_ld_wait8x4(float* a, float* b, float* c, float* d) {
   asm volatile("tcgen05.wait::ld.sync.aligned;"
                : "+f"(a[0]), "+f"(a[1]), "+f"(a[2]), "+f"(a[3]), "+f"(a[4]), "+f"(a[5]), "+f"(a[6]), "+f"(a[7]),

@@ -6,6 +6,7 @@
 #include "cell.cuh"
 #include "umma_engine.cuh"
 #include "umma_cell.cuh"
+#include "umma_adj.cuh"
 #include "umma_gemm.cuh"
 #include "umma_gemm_pair.cuh"
 
@@ -607,18 +608,24 @@ __global__ void __launch_bounds__(kPT) pack_adj_kernel(const float* __restrict__
   pdl_wait();
   pdl_trigger();
   i64 total = M * H4;
+  // L2 hints: the packed operand is read back at once by the product (keep it), the coefficients are dead after this pass
+  uint64_t keep, drop;
+  asm("createpolicy.fractional.L2::evict_last.b64 %0, 1.0;" : "=l"(keep));
+  asm("createpolicy.fractional.L2::evict_first.b64 %0, 1.0;" : "=l"(drop));
+  auto ldc = [&](const bf16* p) { uint2 v; asm volatile("ld.global.L2::cache_hint.v2.b32 {%0,%1}, [%2], %3;" : "=r"(v.x), "=r"(v.y) : "l"(p), "l"(drop)); return v; };
+  auto stk = [&](uint2* p, uint2 v) { asm volatile("st.global.L2::cache_hint.v2.b32 [%0], {%1,%2}, %3;" ::"l"(p), "r"(v.x), "r"(v.y), "l"(keep) : "memory"); };
   for (i64 e = (i64)blockIdx.x * blockDim.x + threadIdx.x; e < total; e += (i64)gridDim.x * blockDim.x) {
     i64 m = e / H4; int c = (int)(e % H4);
     i64 k = m / B; int b = (int)(m % B);
     i64 ro = ((i64)b * H4 + c) * 4;
     float4 l = *reinterpret_cast<const float4*>(lin + k * lin_ks + ro);
-    float4 r = unpack4(*reinterpret_cast<const uint2*>(cr + k * coef_ks + ro));
-    float4 z = unpack4(*reinterpret_cast<const uint2*>(cz + k * coef_ks + ro));
-    float4 n = unpack4(*reinterpret_cast<const uint2*>(cn + k * coef_ks + ro));
+    float4 r = unpack4(ldc(cr + k * coef_ks + ro));
+    float4 z = unpack4(ldc(cz + k * coef_ks + ro));
+    float4 n = unpack4(ldc(cn + k * coef_ks + ro));
     i64 o = m * 3 * H4 + c;
-    dst[o] = pack4(make_float4(r.x * l.x, r.y * l.y, r.z * l.z, r.w * l.w));
-    dst[o + H4] = pack4(make_float4(z.x * l.x, z.y * l.y, z.z * l.z, z.w * l.w));
-    dst[o + 2 * H4] = pack4(make_float4(n.x * l.x, n.y * l.y, n.z * l.z, n.w * l.w));
+    stk(dst + o, pack4(make_float4(r.x * l.x, r.y * l.y, r.z * l.z, r.w * l.w)));
+    stk(dst + o + H4, pack4(make_float4(z.x * l.x, z.y * l.y, z.z * l.z, z.w * l.w)));
+    stk(dst + o + 2 * H4, pack4(make_float4(n.x * l.x, n.y * l.y, n.z * l.z, n.w * l.w)));
   }
 }
 
@@ -885,6 +892,53 @@ int umma_linearise(const LinArgs& a, UmmaAdjWs* w, cudaStream_t s) {
                                                                                                                       : MGRIT_CUDA_ERROR;
 }
 
+// MGRIT_GRU_ADJ_STAGED=0 in the environment keeps every adjoint product on the plain GEMM with global-load epilogue.
+static bool adj_staged_enabled() {
+  static int v = -1;
+  if (v < 0) { const char* e = getenv("MGRIT_GRU_ADJ_STAGED"); v = (e && e[0] == '0') ? 0 : 1; }
+  return v == 1;
+}
+
+// The adjoint product with TMA-staged epilogue operands (rows (k, b), 128 % B == 0).
+template <bool HAS_G, bool PAIR>
+static bool launch_adj_staged(const AdjStepArgs& a, const bf16* Apack, const bf16* W_hhT, const float* g, i64 g_ks, cudaStream_t s) {
+  using C = adjk::ACfg<HAS_G, PAIR>;
+  int* const status = status_ptr();
+  if (!status) return false;
+  static bool attr_set[kMaxDevices] = {false};
+  auto kern = umma_adj_kernel<HAS_G, PAIR>;
+  if (!set_smem_once(kern, C::kSmemBytes, attr_set)) return false;
+  const int B = a.B, H = a.H, kt = 128 / B, nk = a.M / B, K = 3 * H;
+  AdjKArgs ka{};
+  ka.M = a.M; ka.B = B; ka.H = H; ka.kt = kt; ka.nk = nk; ka.lout = a.lout; ka.lout_ks = a.lout_ks; ka.mode = a.mode;
+  ka.a_rev = (a.coef_ks < 0 && nk > 1) ? 1 : 0;
+  CUtensorMap ta, tb, tl, tca, tg;
+  if (!make_map(&ta, Apack, (uint64_t)K, (uint64_t)a.M, (uint64_t)K, BM)) return false;
+  if (!make_map(&tb, W_hhT, (uint64_t)K, (uint64_t)H, (uint64_t)K, PAIR ? adjk::ABN / 2 : adjk::ABN)) return false;
+  const auto f32 = CU_TENSOR_MAP_DATA_TYPE_FLOAT32;
+  if (!make_map3(&tl, f32, 4, a.lin, H, B, nk, H, a.lin_ks, adjk::ACH, kt, CU_TENSOR_MAP_SWIZZLE_64B)) return false;
+  const float* abase = ka.a_rev ? a.a + (i64)(nk - 1) * a.coef_ks : a.a;      // lowest address when the rows run backwards
+  if (!make_map3(&tca, f32, 4, abase, H, B, nk, H, ka.a_rev ? -a.coef_ks : a.coef_ks, adjk::ACH, kt, CU_TENSOR_MAP_SWIZZLE_64B)) return false;
+  if (HAS_G) {
+    if (!make_map3(&tg, f32, 4, g, H, B, nk, H, g_ks, adjk::ACH, kt, CU_TENSOR_MAP_SWIZZLE_64B)) return false;
+  } else {
+    tg = tl;
+  }
+  constexpr int kTileRows = PAIR ? 2 * BM : BM;
+  const int tiles = ((a.M + kTileRows - 1) / kTileRows) * ((H + adjk::ABN - 1) / adjk::ABN);
+  cudaError_t e;
+  if (PAIR) {
+    const int grid = 2 * (tiles < kSMs / 2 ? tiles : kSMs / 2);
+    e = launch_pdl_cluster(kern, 2, dim3(grid), dim3(adjk::kAdjThreads), C::kSmemBytes, s, ta, tb, tl, tca, tg, ka, K, status);
+  } else {
+    const int grid = tiles < kSMs ? tiles : kSMs;
+    e = launch_pdl(kern, dim3(grid), dim3(adjk::kAdjThreads), C::kSmemBytes, s, ta, tb, tl, tca, tg, ka, K, status);
+  }
+  if (e != cudaSuccess) return false;
+  count_launch();
+  return true;
+}
+
 int umma_adj_step(const AdjStepArgs& a, UmmaAdjWs* w, cudaStream_t s) {
   ProfScope prof(KC_ADJ_STEP, 2.0 * a.M * 3.0 * a.H * a.H, s);     // operand packing + product, timed together
   if (launch_pdl(pack_adj_kernel, dim3(pgrid((i64)a.M * (a.H / 4))), dim3(kPT), 0, s, a.lin, a.lin_ks, a.crb, a.czb, a.cnb, a.coef_ks,
@@ -895,6 +949,17 @@ int umma_adj_step(const AdjStepArgs& a, UmmaAdjWs* w, cudaStream_t s) {
   // bound by one CTA streaming all of K; 64-column tiles spread that stream over four times the CTAs.
   const int tiles256 = ((a.M + BM - 1) / BM) * ((a.H + 255) / 256);
   bool ok;
+  // strides of the staged operands: positive for the sensitivities, any sign for the coefficient rows
+  const bool staged = adj_staged_enabled() && 128 % a.B == 0 && tiles256 * 2 > kSMs && a.lin_ks > 0 && a.lout_ks > 0 &&
+                      (a.mode == 1 || !a.gadd || a.gadd_ks > 0);
+  if (staged) {
+    const float* g = a.mode == 1 ? a.lout : a.gadd;
+    const i64 g_ks = a.mode == 1 ? a.lout_ks : a.gadd_ks;
+    const bool pair = gemm_pair_enabled(a.M, a.H);
+    if (g) ok = pair ? launch_adj_staged<true, true>(a, w->Apack, w->W_hhT, g, g_ks, s) : launch_adj_staged<true, false>(a, w->Apack, w->W_hhT, g, g_ks, s);
+    else ok = pair ? launch_adj_staged<false, true>(a, w->Apack, w->W_hhT, nullptr, 0, s) : launch_adj_staged<false, false>(a, w->Apack, w->W_hhT, nullptr, 0, s);
+    return ok ? MGRIT_OK : MGRIT_CUDA_ERROR;
+  }
   if (tiles256 * 2 <= kSMs)
     ok = launch_gemm<64, 0>(KC_ADJ_STEP, w->Apack, 3 * a.H, w->W_hhT, 3 * a.H, a.M, a.H, 3 * a.H, 0, a.H, EpiAdj<64>{a}, s);
   else if (gemm_pair_enabled(a.M, a.H))

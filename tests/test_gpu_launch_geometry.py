@@ -100,3 +100,20 @@ def test_relaxation_sweeps_in_one_launch_give_the_same_bits(tmp_path):
             assert np.allclose(a[k], b[k], rtol=1e-5), k
         else:
             assert a[k][0] < b[k][0], (k, a[k], b[k])
+
+
+def test_staged_and_global_load_adjoint_epilogues_agree(tmp_path):
+    """The adjoint product with TMA-staged epilogue operands (reversed coefficient rows, pair and single-CTA geometry,
+    with and without a source term) against the plain GEMM whose epilogue loads the same operands from global memory:
+    the same sums in the same order, up to how the compiler contracts one multiply-add."""
+    root = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+    outs = []
+    for flag in ("1", "0"):
+        out = str(tmp_path / f"adj{flag}.npz")
+        env = dict(os.environ, MGRIT_GRU_ADJ_STAGED=flag, PYTHONPATH=root)
+        subprocess.run([sys.executable, "-c", CHILD, out], check=True, env=env, cwd=root, timeout=600)
+        outs.append(np.load(out))
+    a, b = outs
+    for k in a.files:
+        scale = np.max(np.abs(a[k]))
+        assert np.max(np.abs(a[k] - b[k])) <= 1e-6 * scale, k
