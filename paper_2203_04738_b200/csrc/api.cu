@@ -338,8 +338,8 @@ struct FwdCycle : Cycle {
     a.u = U[l]; a.ub = fw->chain_ub;
     i64 st = hr.stride_t[l];
     a.gi = gi + (st - 1) * (i64)BH * 3; a.gi_step = st * (i64)BH * 3;
-    // (the plain serial sweep has no other level to stay consistent with: it reads the fp32 projection)
-    a.gi_b = (gib && hr.L > 1) ? gib + (st - 1) * (i64)BH * 3 : nullptr;
+    // (the plain serial sweep has no other level to stay consistent with: it uses the fp32 projection as it is)
+    a.gi_as_bf16 = (gib && hr.L > 1) ? 1 : 0;
     a.g = G[l]; a.W = um->W_hh; a.b_hh = p->b_hh; a.gamma = hr.gamma[l]; a.cell = c->cell; a.bar = fw->chain_bar;
     a.xw = fw->chain_xw; a.xw_bytes = fw->chain_xw_bytes;
     return serial_fwd_solve(a, s);

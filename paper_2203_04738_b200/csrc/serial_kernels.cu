@@ -39,6 +39,8 @@ __device__ __forceinline__ int ld_relaxed(const int* p) {
   return v;
 }
 
+__device__ __forceinline__ float bf16_round(float x) { return __bfloat162float(__float2bfloat16_rn(x)); }
+
 // All CTAs that share `ctr` have finished the step whose arrival count is `target`.
 __device__ __forceinline__ bool grid_barrier(unsigned* ctr, unsigned target, int* status, int* ok_smem) {
   __syncthreads();
@@ -241,12 +243,7 @@ __global__ void __launch_bounds__(kThreads, 1) serial_fwd_kernel(SerialFwdArgs a
     hp[o] = v ? __ldcg(a.u + (i64)(row0 + r) * H + u0 + i) : 0.f;
     br[o] = a.b_hh[u0 + i]; bz[o] = a.b_hh[H + u0 + i]; bn[o] = a.b_hh[2 * H + u0 + i];
     const i64 go = (i64)(row0 + r) * 3 * H + u0 + i;
-    if (a.gi_b) {
-      pgr[o] = v ? __bfloat162float(a.gi_b[go]) : 0.f; pgz[o] = v ? __bfloat162float(a.gi_b[go + H]) : 0.f;
-      pgn[o] = v ? __bfloat162float(a.gi_b[go + 2 * H]) : 0.f;
-    } else {
-      pgr[o] = v ? a.gi[go] : 0.f; pgz[o] = v ? a.gi[go + H] : 0.f; pgn[o] = v ? a.gi[go + 2 * H] : 0.f;
-    }
+    pgr[o] = v ? a.gi[go] : 0.f; pgz[o] = v ? a.gi[go + H] : 0.f; pgn[o] = v ? a.gi[go + 2 * H] : 0.f;
     pg[o] = (v && a.g) ? a.g[BH + (i64)(row0 + r) * H + u0 + i] : 0.f;
   }
   __syncthreads();
@@ -268,7 +265,9 @@ __global__ void __launch_bounds__(kThreads, 1) serial_fwd_kernel(SerialFwdArgs a
         float ghr = sum_partials<NW>(red, r, i) + br[o];
         float ghz = sum_partials<NW>(red, r, UNC + i) + bz[o];
         float ghn = sum_partials<NW>(red, r, 2 * UNC + i) + bn[o];
-        val = cell_forward<true>(pgr[o], pgz[o], pgn[o], ghr, ghz, ghn, hp[o], a.gamma, a.cell) + pg[o];
+        const float gir = a.gi_as_bf16 ? bf16_round(pgr[o]) : pgr[o], giz = a.gi_as_bf16 ? bf16_round(pgz[o]) : pgz[o];
+        const float gin = a.gi_as_bf16 ? bf16_round(pgn[o]) : pgn[o];
+        val = cell_forward<true>(gir, giz, gin, ghr, ghz, ghn, hp[o], a.gamma, a.cell) + pg[o];
         hp[o] = val;
         i64 off = (i64)(row0 + r) * H + u0 + i;
         a.u[(i64)j * BH + off] = val;
@@ -287,11 +286,9 @@ __global__ void __launch_bounds__(kThreads, 1) serial_fwd_kernel(SerialFwdArgs a
       int idx = tid + o * kThreads, r = idx / UNC, i = idx % UNC;
       if (idx < kRows * UNC && r < nrows) {
         const i64 go = (i64)j * a.gi_step + (i64)(row0 + r) * 3 * H + u0 + i;
-        if (a.gi_b) {
-          pgr[o] = __bfloat162float(a.gi_b[go]); pgz[o] = __bfloat162float(a.gi_b[go + H]); pgn[o] = __bfloat162float(a.gi_b[go + 2 * H]);
-        } else {
-          pgr[o] = a.gi[go]; pgz[o] = a.gi[go + H]; pgn[o] = a.gi[go + 2 * H];
-        }
+        // (loaded now, rounded where they are used: an instruction that depends on these loads here would wait for them
+        // in front of the exchange)
+        pgr[o] = a.gi[go]; pgz[o] = a.gi[go + H]; pgn[o] = a.gi[go + 2 * H];
         if (a.g) pg[o] = a.g[(i64)(j + 1) * BH + (i64)(row0 + r) * H + u0 + i];
       }
     }
