@@ -207,8 +207,8 @@ int mgrit_gru_stack_adjoint(const mgrit_gru_cfg* cfg, int32_t n_layers, const gr
  *   The state of a time point is (c, h): u0[2,B,H], u[T,2,B,H], du_seed / du likewise; gi[T,B,4H].
  *   dhT[B,H]: loss derivative w.r.t. the last HIDDEN state.  grads: one gru_grads with the 4H-row shapes.
  *   Everything else (cycles, relaxation, flags, resnorm, levels == 1 = serial sweep / exact BPTT) as for the GRU calls.
- *   Operand modes MGRIT_OPERANDS_FP32 (FFMA) and the tf32 modes (tcgen05 products on four-gate tiles of 64 hidden
- *   units; same shape limits as for the GRU); MGRIT_OPERANDS_BF16: MGRIT_UNSUPPORTED. */
+ *   Operand modes: MGRIT_OPERANDS_FP32 (FFMA), the tf32 modes and MGRIT_OPERANDS_BF16 (tcgen05 products on four-gate
+ *   tiles of 64 hidden units; same shape limits and tolerances as for the GRU). */
 int mgrit_lstm_workspace_bytes(const mgrit_gru_cfg* cfg, size_t* fwd_bytes, size_t* adj_bytes);
 int mgrit_lstm_forward(const mgrit_gru_cfg* cfg, const gru_params* p, const float* x, const float* u0, float* gi, float* u,
                        float* resnorm, void* ws, size_t ws_bytes, mgrit_stream_t stream);

@@ -965,11 +965,11 @@ int stack_adjoint_impl(const mgrit_gru_cfg* cfg, int nl, const gru_params* p, co
 // ======================================================================================================
 // Implicit LSTM: the state of a time point is (c, h); level arrays are [N_l + 1][2][B][H] (part 0 = c, part 1 = h) and
 // the same Cycle drives them.  fp32 engine only (four-gate FFMA products).
-struct LstmFwdWs { float* U[kMaxLevels]; float* G[kMaxLevels]; double* res_acc; float *tmpC, *tmpH; size_t maxM; Tf32Ws tf; };
+struct LstmFwdWs { float* U[kMaxLevels]; float* G[kMaxLevels]; double* res_acc; float *tmpC, *tmpH; size_t maxM; Tf32Ws tf; LstmBfWs bf; };
 struct LstmAdjWs {
   float* U[kMaxLevels]; float* G[kMaxLevels]; double* res_acc;
   float *a[kMaxLevels], *p[kMaxLevels], *ci[kMaxLevels], *cf[kMaxLevels], *cg[kMaxLevels], *co[kMaxLevels];
-  float *tmpC, *tmpH, *hk, *dA; size_t maxM; Tf32Ws tf;
+  float *tmpC, *tmpH, *hk, *dA; size_t maxM; Tf32Ws tf; LstmBfWs bf;
 };
 
 void plan_lstm_fwd(const mgrit_gru_cfg* c, const Hier& hr, Ws& w, LstmFwdWs* o) {
@@ -983,6 +983,7 @@ void plan_lstm_fwd(const mgrit_gru_cfg* c, const Hier& hr, Ws& w, LstmFwdWs* o) 
   o->tmpC = w.take<float>(o->maxM * c->H);
   o->tmpH = w.take<float>(o->maxM * c->H);
   if (is_tf32(c)) tf32_plan_fwd(c, hr.N, hr.L, w.base, &w.off, &o->tf, 4);
+  if (c->operands == MGRIT_OPERANDS_BF16) lstmbf_plan_fwd(c, o->maxM, w.base, &w.off, &o->bf);
 }
 
 void plan_lstm_adj(const mgrit_gru_cfg* c, const Hier& hr, Ws& w, LstmAdjWs* o) {
@@ -1001,6 +1002,7 @@ void plan_lstm_adj(const mgrit_gru_cfg* c, const Hier& hr, Ws& w, LstmAdjWs* o) 
   o->hk = w.take<float>(TB * c->H);
   o->dA = w.take<float>(TB * 4 * c->H);
   if (is_tf32(c)) tf32_plan_adj(c, hr.N, hr.L, w.base, &w.off, &o->tf, 4);
+  if (c->operands == MGRIT_OPERANDS_BF16) lstmbf_plan_adj(c, o->maxM, w.base, &w.off, &o->bf);
 }
 
 struct LstmFwdCycle : Cycle {
@@ -1015,6 +1017,7 @@ struct LstmFwdCycle : Cycle {
     a.gi = gi + ((i64)st * d.tgt_slot - 1) * (i64)bh * 4; a.gi_ks = st * d.tgt_stride * (i64)bh * 4;
     a.W_hh = p->W_hh; a.b_hh = p->b_hh; a.gamma = hr.gamma[d.l]; a.cell = c->cell;
     if (is_tf32(c)) { int r = tf32_lstm_fwd_step(a, &fw->tf, s); if (r) return r; }
+    else if (c->operands == MGRIT_OPERANDS_BF16) { int r = lstmbf_fwd_step(a, &fw->bf, s); if (r) return r; }
     else simt_lstm_fwd_step(a, s);
     for (int part = 0; part < 2; ++part) {
       const float* g = d.gadd ? d.gadd + (size_t)d.gadd_slot * slot + part * bh : nullptr;
@@ -1038,6 +1041,7 @@ struct LstmAdjCycle : Cycle {
     a.cg = w->cg[d.l] + row0; a.co = w->co[d.l] + row0; a.coef_ks = -(i64)d.tgt_stride * (i64)bh;
     a.W_hh = p->W_hh;
     if (is_tf32(c)) { int r = tf32_lstm_adj_step(a, &w->tf, s); if (r) return r; }
+    else if (c->operands == MGRIT_OPERANDS_BF16) { int r = lstmbf_adj_step(a, &w->bf, s); if (r) return r; }
     else simt_lstm_adj_step(a, s);
     for (int part = 0; part < 2; ++part) {
       const float* g = d.gadd ? d.gadd + (size_t)d.gadd_slot * slot + part * bh : nullptr;
@@ -1050,8 +1054,7 @@ struct LstmAdjCycle : Cycle {
 
 int lstm_check(const mgrit_gru_cfg* cfg, Hier* hr) {
   if (!cfg) return MGRIT_INVALID_ARG;
-  if (cfg->operands == MGRIT_OPERANDS_BF16) return MGRIT_UNSUPPORTED;      // four-gate products: fp32 engine or the tf32 modes
-  return check_cfg(cfg, hr);
+  return check_cfg(cfg, hr);        // (bf16 and tf32 operands: check_cfg applies the tensor-core engines' shape limits)
 }
 
 int lstm_forward_impl(const mgrit_gru_cfg* cfg, const gru_params* p, const float* x, const float* u0, float* gi, float* u,
@@ -1068,6 +1071,7 @@ int lstm_forward_impl(const mgrit_gru_cfg* cfg, const gru_params* p, const float
   if (!w.fits()) return MGRIT_WORKSPACE_TOO_SMALL;
   const size_t slot = (size_t)2 * c.B * c.H;
   if (is_tf32(&c)) { rc = tf32_prepare_fwd(&c, p, x, gi, &fw.tf, s); if (rc) return rc; }
+  else if (c.operands == MGRIT_OPERANDS_BF16) { rc = lstmbf_prepare_fwd(&c, p, x, gi, &fw.bf, s); if (rc) return rc; }
   else simt_project(x, p->W_ih, p->b_ih, gi, c.T * c.B, c.I, 4 * c.H, s);
   cudaMemsetAsync(fw.U[0] + slot, 0, sizeof(float) * (size_t)c.T * slot, s);
   for (int l = 0; l < hr.L; ++l) cudaMemcpyAsync(fw.U[l], u0, sizeof(float) * slot, cudaMemcpyDeviceToDevice, s);
@@ -1103,14 +1107,16 @@ int lstm_adjoint_impl(const mgrit_gru_cfg* cfg, const gru_params* p, const float
   if (!w.fits()) return MGRIT_WORKSPACE_TOO_SMALL;
   const size_t bh = (size_t)c.B * c.H, slot = 2 * bh;
   const int T = c.T;
-  const bool tf32 = is_tf32(&c);
+  const bool tf32 = is_tf32(&c), bf = c.operands == MGRIT_OPERANDS_BF16;
   if (tf32) { rc = tf32_prepare_adj(&c, p, &aw.tf, s); if (rc) return rc; }
+  if (bf) { rc = lstmbf_prepare_adj(&c, p, &aw.bf, s); if (rc) return rc; }
   for (int l = 0; l < hr.L; ++l) {
     LstmLinArgs a;
     a.M = hr.N[l] * c.B; a.B = c.B; a.H = c.H; a.c0 = u0; a.h0 = u0 + bh; a.c = u; a.h = u + bh; a.ts = (i64)slot;
     a.stride_t = hr.stride_t[l]; a.t0 = hr.rem[l]; a.gi = gi; a.W_hh = p->W_hh; a.b_hh = p->b_hh; a.gamma = hr.gamma[l]; a.cell = c.cell;
     a.a = aw.a[l]; a.p = aw.p[l]; a.ci = aw.ci[l]; a.cf = aw.cf[l]; a.cg = aw.cg[l]; a.co = aw.co[l];
     if (tf32) { rc = tf32_lstm_linearise(a, &aw.tf, s); if (rc) return rc; }
+    else if (bf) { rc = lstmbf_linearise(a, &aw.bf, s); if (rc) return rc; }
     else simt_lstm_linearise(a, s);
   }
   cudaMemsetAsync(aw.U[0], 0, sizeof(float) * (size_t)(T + 1) * slot, s);
@@ -1137,13 +1143,16 @@ int lstm_adjoint_impl(const mgrit_gru_cfg* cfg, const gru_params* p, const float
     rc = tf32_wgrad(aw.dA, (int)M, 4 * c.H, u0 + bh, c.B, aw.hk, c.H, g->dW_hh, &aw.tf, s);
     if (!rc) rc = tf32_wgrad(aw.dA, (int)M, 4 * c.H, nullptr, 0, x, c.I, g->dW_ih, &aw.tf, s);
     if (rc) return rc;
+  } else if (bf) {
+    rc = lstmbf_gradients(&c, aw.dA, x, u0 + bh, aw.hk, g, dx, &aw.bf, s);
+    if (rc) return rc;
   } else {
     simt_wgrad(aw.dA, (int)M, 4 * c.H, u0 + bh, c.B, aw.hk, c.H, g->dW_hh, s);
     simt_wgrad(aw.dA, (int)M, 4 * c.H, nullptr, 0, x, c.I, g->dW_ih, s);
   }
   stream_colsum(aw.dA, M, 4 * c.H, g->db_hh, s);
   cudaMemcpyAsync(g->db_ih, g->db_hh, sizeof(float) * 4 * c.H, cudaMemcpyDeviceToDevice, s);
-  if (dx) {
+  if (dx && !bf) {
     if (tf32) { rc = tf32_dgrad(aw.dA, (int)M, 4 * c.H, c.I, dx, &aw.tf, s); if (rc) return rc; }
     else simt_dgrad(aw.dA, (int)M, 4 * c.H, p->W_ih, c.I, dx, s);
   }

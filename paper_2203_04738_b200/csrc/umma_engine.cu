@@ -1276,7 +1276,7 @@ namespace {
 
 // LSTM cell / its transposed-Jacobian coefficients on the i | f | g | o accumulator columns of 64 hidden units, one
 // output row per thread, 8 units at a time (precise gate math)
-template <bool LIN>
+template <bool LIN, bool FAST = false>
 struct EpiLstm {
   LstmFwdArgs f;      // !LIN
   LstmLinArgs l;      // LIN
@@ -1314,10 +1314,10 @@ struct EpiLstm {
           const float ai = acc[0][e] + __ldg(bh + n), af = acc[1][e] + __ldg(bh + H + n), ag = acc[2][e] + __ldg(bh + 2 * H + n),
                       ao = acc[3][e] + __ldg(bh + 3 * H + n);
           if (LIN) {
-            LstmLin L = lstm_linearise(g4[0][e], g4[1][e], g4[2][e], g4[3][e], ai, af, ag, ao, cp[e], gamma, cell);
+            LstmLin L = lstm_linearise<FAST>(g4[0][e], g4[1][e], g4[2][e], g4[3][e], ai, af, ag, ao, cp[e], gamma, cell);
             o0[e] = L.a; o1[e] = L.p; o2[e] = L.ci; o3[e] = L.cf; o4[e] = L.cg; o5[e] = L.co;
           } else {
-            LstmOut r = lstm_forward(g4[0][e], g4[1][e], g4[2][e], g4[3][e], ai, af, ag, ao, cp[e], gamma, cell);
+            LstmOut r = lstm_forward<FAST>(g4[0][e], g4[1][e], g4[2][e], g4[3][e], ai, af, ag, ao, cp[e], gamma, cell);
             o0[e] = r.c; o1[e] = r.h;
           }
         }
@@ -1388,6 +1388,126 @@ int tf32_lstm_adj_step(const LstmAdjArgs& a, Tf32Ws* w, cudaStream_t s) {
   count_launch();
   return launch_gemm<256, 0>(KC_ADJ_STEP, (const float*)w->Apack, (i64)K, (const float*)w->W_hhT, (i64)K, a.M, a.H, K, 0, a.H,
                              EpiStore{a.lh_out, a.H, a.M, a.H, 0}, s) ? MGRIT_OK : MGRIT_CUDA_ERROR;
+}
+
+// ---------------------------------------------------------------- Implicit LSTM, bf16 operands
+namespace {
+// dst[m, g*H + i] = bf16(coefficient_g * (g < 3 ? Lc + p*Lh : Lh));  lc_out[m, i] = a * (Lc + p*Lh)
+__global__ void __launch_bounds__(kPT) pack_lstm_adj_kernel(LstmAdjArgs a, bf16* __restrict__ dst) {
+  pdl_wait();
+  pdl_trigger();
+  const i64 total = (i64)a.M * a.H;
+  for (i64 e = (i64)blockIdx.x * blockDim.x + threadIdx.x; e < total; e += (i64)gridDim.x * blockDim.x) {
+    const i64 m = e / a.H; const int i = (int)(e % a.H);
+    const i64 kk = m / a.B; const int b = (int)(m % a.B);
+    const i64 ci = kk * a.coef_ks + (i64)b * a.H + i, li = kk * a.in_ks + (i64)b * a.H + i;
+    const float lh = a.lh[li], dc = a.lc[li] + a.p[ci] * lh;
+    a.lc_out[e] = a.a[ci] * dc;
+    bf16* d = dst + m * 4 * a.H + i;
+    d[0] = __float2bfloat16(a.ci[ci] * dc); d[a.H] = __float2bfloat16(a.cf[ci] * dc);
+    d[2 * a.H] = __float2bfloat16(a.cg[ci] * dc); d[3 * a.H] = __float2bfloat16(a.co[ci] * lh);
+  }
+}
+bool pack_rows(const float* src, i64 ks, int B, int H, i64 M, bf16* dst, cudaStream_t s) {
+  if (M <= 0) return true;
+  if (launch_pdl(pack_rows_kernel, dim3(pgrid(M * (H / 4))), dim3(kPT), 0, s, src, ks, B, H / 4, M, reinterpret_cast<uint2*>(dst)) != cudaSuccess)
+    return false;
+  count_launch();
+  return true;
+}
+}  // namespace
+
+void lstmbf_plan_fwd(const mgrit_gru_cfg* c, size_t max_rows, char* base, size_t* off, LstmBfWs* o) {
+  const size_t H = c->H, I = c->I, TB = (size_t)c->T * c->B;
+  *o = LstmBfWs{};
+  o->W_hh = take<bf16>(base, off, 4 * H * H);
+  o->W_ih = take<bf16>(base, off, 4 * H * I);
+  o->apack_elems = max_rows * H > TB * I ? max_rows * H : TB * I;      // a step's rows, or x for the projection
+  o->Apack = take<bf16>(base, off, o->apack_elems);
+}
+
+void lstmbf_plan_adj(const mgrit_gru_cfg* c, size_t max_rows, char* base, size_t* off, LstmBfWs* o) {
+  const size_t H = c->H, I = c->I, TB = (size_t)c->T * c->B;
+  *o = LstmBfWs{};
+  o->W_hh = take<bf16>(base, off, 4 * H * H);
+  o->W_hhT = take<bf16>(base, off, 4 * H * H);
+  o->W_ihT = take<bf16>(base, off, 4 * H * I);
+  size_t ap = max_rows * 4 * H;
+  if (TB * H > ap) ap = TB * H;        // the linearisation packs all T*B rows of a level at once
+  o->apack_elems = ap;
+  o->Apack = take<bf16>(base, off, ap);
+  o->xb = take<bf16>(base, off, TB * I);
+  o->hb0 = take<bf16>(base, off, (TB + c->B) * H);
+  o->dAb = take<bf16>(base, off, TB * 4 * H);
+  o->scratch_bytes = (size_t)4 * 4 * H * (H > I ? H : I) * sizeof(float);
+  o->scratch = take<float>(base, off, o->scratch_bytes / sizeof(float));
+}
+
+int lstmbf_prepare_fwd(const mgrit_gru_cfg* c, const gru_params* p, const float* x, float* gi, LstmBfWs* w, cudaStream_t s) {
+  const int H = c->H, I = c->I, TB = c->T * c->B;
+  if (!status_ptr()) return MGRIT_CUDA_ERROR;
+  convert(p->W_hh, w->W_hh, (i64)4 * H * H, s);
+  convert(p->W_ih, w->W_ih, (i64)4 * H * I, s);
+  convert(x, w->Apack, (i64)TB * I, s);
+  return launch_gemm<256, 0>(KC_PROJ, w->Apack, I, w->W_ih, I, TB, 4 * H, I, 0, 4 * H, EpiBias{gi, 4 * H, p->b_ih, TB, 4 * H}, s) ? MGRIT_OK
+                                                                                                                       : MGRIT_CUDA_ERROR;
+}
+
+int lstmbf_prepare_adj(const mgrit_gru_cfg* c, const gru_params* p, LstmBfWs* w, cudaStream_t s) {
+  const int H = c->H, I = c->I;
+  if (!status_ptr()) return MGRIT_CUDA_ERROR;
+  convert(p->W_hh, w->W_hh, (i64)4 * H * H, s);
+  transpose(p->W_hh, 4 * H, H, w->W_hhT, 4 * H, 0, s);   // [H, 4H]
+  transpose(p->W_ih, 4 * H, I, w->W_ihT, 4 * H, 0, s);   // [I, 4H]
+  return MGRIT_OK;
+}
+
+int lstmbf_fwd_step(const LstmFwdArgs& a, LstmBfWs* w, cudaStream_t s) {
+  if (!pack_rows(a.hin, a.in_ks, a.B, a.H, a.M, w->Apack, s)) return MGRIT_CUDA_ERROR;
+  EpiLstm<false, true> epi{};
+  epi.f = a;
+  return launch_gemm<256, 4>(KC_FWD_STEP, w->Apack, a.H, w->W_hh, a.H, a.M, a.H, a.H, a.H, 4 * a.H, epi, s) ? MGRIT_OK : MGRIT_CUDA_ERROR;
+}
+
+int lstmbf_linearise(const LstmLinArgs& a, LstmBfWs* w, cudaStream_t s) {
+  const int N = a.M / a.B;
+  const i64 BH = (i64)a.B * a.H;
+  int done = 0;
+  if (a.t0 == 0) {
+    if (!pack_rows(a.h0, 0, a.B, a.H, a.B, w->Apack, s)) return MGRIT_CUDA_ERROR;
+    done = 1;
+  }
+  if (N > done) {
+    const i64 t1 = a.t0 + (i64)done * a.stride_t;
+    if (!pack_rows(a.h + (t1 - 1) * a.ts, a.stride_t * a.ts, a.B, a.H, (i64)(N - done) * a.B, w->Apack + (i64)done * BH, s)) return MGRIT_CUDA_ERROR;
+  }
+  EpiLstm<true, true> epi{};
+  epi.l = a;
+  return launch_gemm<256, 4>(KC_LINEARISE, w->Apack, a.H, w->W_hh, a.H, a.M, a.H, a.H, a.H, 4 * a.H, epi, s) ? MGRIT_OK : MGRIT_CUDA_ERROR;
+}
+
+int lstmbf_adj_step(const LstmAdjArgs& a, LstmBfWs* w, cudaStream_t s) {
+  const int K = 4 * a.H;
+  ProfScope prof(KC_ADJ_STEP, 2.0 * a.M * (double)K * a.H, s);
+  if (launch_pdl(pack_lstm_adj_kernel, dim3(pgrid((i64)a.M * a.H)), dim3(kPT), 0, s, a, w->Apack) != cudaSuccess) return MGRIT_CUDA_ERROR;
+  count_launch();
+  return launch_gemm<256, 0>(KC_ADJ_STEP, w->Apack, K, w->W_hhT, K, a.M, a.H, K, 0, a.H, EpiStore{a.lh_out, a.H, a.M, a.H, 0}, s) ? MGRIT_OK
+                                                                                                                              : MGRIT_CUDA_ERROR;
+}
+
+int lstmbf_gradients(const mgrit_gru_cfg* c, const float* dA, const float* x, const float* h0, const float* hk, const gru_grads* g,
+                     float* dx, LstmBfWs* w, cudaStream_t s) {
+  const int H = c->H, I = c->I, B = c->B;
+  const i64 M = (i64)c->T * B;
+  ProfScope prof(KC_WGRAD, 2.0 * M * 4.0 * H * ((double)H + I + (dx ? I : 0)), s);
+  convert(dA, w->dAb, M * 4 * H, s);
+  convert(x, w->xb, M * I, s);
+  convert(h0, w->hb0, (i64)B * H, s);
+  convert(hk, w->hb0 + (i64)B * H, M * H, s);          // rows (t, b) of h_{t-1} start at hb0
+  bool ok = wgrad_gemm(w->dAb, 4 * H, w->hb0, H, (int)M, g->dW_hh, w->scratch, w->scratch_bytes, s);
+  ok = ok && wgrad_gemm(w->dAb, 4 * H, w->xb, I, (int)M, g->dW_ih, w->scratch, w->scratch_bytes, s);
+  if (dx) ok = ok && launch_gemm<256, 0>(KC_WGRAD, w->dAb, 4 * H, w->W_ihT, 4 * H, (int)M, I, 4 * H, 0, I, EpiStore{dx, I, (int)M, I, 0}, s);
+  return ok ? MGRIT_OK : MGRIT_CUDA_ERROR;
 }
 
 int umma_device_status() {

@@ -59,6 +59,26 @@ int tf32_wgrad(const float* dA, int M, int H3, const float* first, int Bfirst, c
                cudaStream_t s);
 int tf32_dgrad(const float* dA, int M, int H3, int C, float* dx, Tf32Ws* w, cudaStream_t s);
 
+// Implicit LSTM with bf16 operands: the plain GEMM with four-gate tiles, fp32 states and fp32 coefficients
+struct LstmBfWs {
+  __nv_bfloat16 *W_hh, *W_ih;     // [4H,H], [4H,I]
+  __nv_bfloat16 *W_hhT, *W_ihT;   // [H,4H], [I,4H]   (adjoint call)
+  __nv_bfloat16* Apack;           // A side of the current product
+  size_t apack_elems;
+  __nv_bfloat16 *xb, *hb0, *dAb;  // [T*B,I]; [(T+1)*B,H] = [h_0; h]; [T*B,4H]   (gradient pass)
+  float* scratch; size_t scratch_bytes;   // partial products of the split weight-gradient reductions
+};
+void lstmbf_plan_fwd(const mgrit_gru_cfg* c, size_t max_rows, char* base, size_t* off, LstmBfWs* o);
+void lstmbf_plan_adj(const mgrit_gru_cfg* c, size_t max_rows, char* base, size_t* off, LstmBfWs* o);
+int lstmbf_prepare_fwd(const mgrit_gru_cfg* c, const gru_params* p, const float* x, float* gi, LstmBfWs* w, cudaStream_t s);
+int lstmbf_prepare_adj(const mgrit_gru_cfg* c, const gru_params* p, LstmBfWs* w, cudaStream_t s);
+int lstmbf_fwd_step(const LstmFwdArgs& a, LstmBfWs* w, cudaStream_t s);
+int lstmbf_linearise(const LstmLinArgs& a, LstmBfWs* w, cudaStream_t s);
+int lstmbf_adj_step(const LstmAdjArgs& a, LstmBfWs* w, cudaStream_t s);
+// dW_hh, dW_ih (and dx) from dA[T*B,4H] fp32; hidden states h0 [B,H] and hk [T,B,H] fp32
+int lstmbf_gradients(const mgrit_gru_cfg* c, const float* dA, const float* x, const float* h0, const float* hk, const gru_grads* g,
+                     float* dx, LstmBfWs* w, cudaStream_t s);
+
 int umma_supported(const mgrit_gru_cfg* c);
 void umma_plan_fwd(const mgrit_gru_cfg* c, const int* N, int L, char* base, size_t* off, UmmaFwdWs* o);
 void umma_plan_adj(const mgrit_gru_cfg* c, const int* N, int L, char* base, size_t* off, UmmaAdjWs* o);
