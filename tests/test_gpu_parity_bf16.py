@@ -265,3 +265,21 @@ def test_copies_carried_behind_gi_change_nothing_but_rounding(B):
                 scale = float(r.dh.abs().max()) if k == "dh0" else float(a.abs().max())
                 assert float((a - b).abs().max()) <= 5e-3 * scale, k
     assert B.last_device_status() == 0
+
+
+def test_long_sweeps_repeat_bit_for_bit(B):
+    # Sixteen dependent steps per launch (cf = 8, FCF on both non-coarsest levels), single-CTA and pair geometry, tiles of a
+    # later step waiting on counters of the earlier one: a missed dependency would show as a run that differs.
+    for Bsz, T in ((8, 2048), (32, 1024)):
+        w = Workload("rep", T=T, B=Bsz, I=64, H=512, cf=8, levels=3, iters_fwd=2, iters_adj=2, relax_fine=1, relax_coarse=1,
+                     operands=2, classes=8, relu=True, seed=13)
+        d = make_inputs(w)
+        p, x, h0 = upload(d)
+        cfg = _cfg(B, w, 2)
+        first = None
+        for _ in range(12):
+            h, _, rn = B.mgrit_gru_forward(cfg, p, x, h0, want_resnorm=True)
+            if first is None:
+                first = h.clone()
+            assert torch.equal(h, first)
+    assert B.last_device_status() == 0
