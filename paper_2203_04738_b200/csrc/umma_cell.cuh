@@ -221,10 +221,11 @@ template <bool HAS_G, bool LIN = false, bool PAIR = false, bool GIB = false> str
 #ifndef CELL_GIB_EBUFS
 #define CELL_GIB_EBUFS 3
 #endif
-  static constexpr int kEpiBufs = GIB ? ((PAIR && !HAS_G && !LIN) ? CELL_GIB_EBUFS : 3) : (PAIR ? CELL_PAIR_EBUFS : 2);     // epilogue-operand chunks in flight
+  static constexpr int kEpiBufs = GIB ? ((PAIR && !HAS_G && !LIN) ? CELL_GIB_EBUFS : (LIN ? 2 : 3)) : (PAIR ? CELL_PAIR_EBUFS : 2);     // epilogue-operand chunks in flight
   static constexpr int kGiBytes = GIB ? BM * CH * 2 : kOpBytes;   // one gate's chunk of the input projection
   static constexpr int kEpiBytes = 3 * kGiBytes + (HAS_G ? 2 : 1) * kOpBytes;   // gi r | z | n, previous state, additive term
-  static constexpr int kOutBytes = LIN ? 4 * kCoefBytes : 0;      // per buffer
+  // per buffer: four bf16 coefficient tiles and (with GIB, where shared memory allows it) the fp32 tile of `a`
+  static constexpr int kOutBytes = LIN ? 4 * kCoefBytes + (GIB ? kOpBytes : 0) : 0;
   static constexpr int kSmemBytes = kStages * G::kStageBytes + kEpiBufs * kEpiBytes + 2 * kOutBytes + 1024 + 256;
   static_assert(kSmemBytes + 1536 <= 232448, "shared memory budget (dynamic + static <= 227 KiB)");
 };
@@ -515,7 +516,13 @@ umma_cell_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
               oa[e] = L.a; ocr[e] = L.cr; ocz[e] = L.cz; ocn[e] = L.cn; ocp[e] = L.cnp;
             }
             const i64 idx = (i64)row * H + u;
-            stg8(p.a + idx, oa);
+            if (GIB) {      // `a` leaves through shared memory like the coefficients (64-byte rows, 64-byte swizzle)
+              const uint32_t da = out_base + ob * C::kOutBytes + 4 * kCoefBytes;
+              asm volatile("st.shared.v4.f32 [%0], {%1,%2,%3,%4};" ::"r"(da + off0), "f"(oa[0]), "f"(oa[1]), "f"(oa[2]), "f"(oa[3]) : "memory");
+              asm volatile("st.shared.v4.f32 [%0], {%1,%2,%3,%4};" ::"r"(da + off1), "f"(oa[4]), "f"(oa[5]), "f"(oa[6]), "f"(oa[7]) : "memory");
+            } else {
+              stg8(p.a + idx, oa);
+            }
             const uint32_t dst = out_base + ob * C::kOutBytes + offb;
             sts_bf8(dst, ocr);
             sts_bf8(dst + kCoefBytes, ocz);
@@ -538,6 +545,7 @@ umma_cell_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
             tma_store_2d(&tmCZ, srcb + kCoefBytes, u, row0);
             tma_store_2d(&tmCN, srcb + 2 * kCoefBytes, u, row0);
             if (p.cnp) tma_store_2d(&tmCP, srcb + 3 * kCoefBytes, u, row0);
+            if (GIB) tma_store_2d(&tmG, srcb + 4 * kCoefBytes, u, row0);      // (the linearisation has no additive term: this map is `a`)
             asm volatile("cp.async.bulk.commit_group;" ::: "memory");
           }
           ob ^= 1;

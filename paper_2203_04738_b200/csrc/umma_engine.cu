@@ -239,6 +239,9 @@ bool launch_lin_geo(int kc, const bf16* A, i64 a_ks, const void* gi, i64 gi_ks, 
     return make_map2(m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, base, H, (uint64_t)ca.M, H, cellk::CH, BM, CU_TENSOR_MAP_SWIZZLE_32B);
   };
   if (!cmap(&tcr, ca.cr) || !cmap(&tcz, ca.cz) || !cmap(&tcn, ca.cn) || (ca.cnp && !cmap(&tcp, ca.cnp))) return false;
+  CUtensorMap taout = thp;      // with the bf16-staged projection `a` is written by TMA stores too ([128 x 16] fp32 tiles)
+  if (GIB && !make_map2(&taout, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 4, ca.a, H, (uint64_t)ca.M, H, cellk::CH, BM, CU_TENSOR_MAP_SWIZZLE_64B))
+    return false;
   constexpr int kTileRows = PAIR ? 2 * BM : BM;
   const int tiles = ((ca.M + kTileRows - 1) / kTileRows) * ((H + G::UN - 1) / G::UN);
   SweepArgs sw{};
@@ -247,10 +250,10 @@ bool launch_lin_geo(int kc, const bf16* A, i64 a_ks, const void* gi, i64 gi_ks, 
   cudaError_t e;
   if (PAIR) {
     const int grid = 2 * (tiles < kSMs / 2 ? tiles : kSMs / 2);
-    e = launch_pdl_cluster(kern, 2, dim3(grid), dim3(cellk::kThreads), C::kSmemBytes, s, ta, tb, tgi, thp, thp, tcr, tcz, tcn, tcp, ca, sw, status);
+    e = launch_pdl_cluster(kern, 2, dim3(grid), dim3(cellk::kThreads), C::kSmemBytes, s, ta, tb, tgi, thp, taout, tcr, tcz, tcn, tcp, ca, sw, status);
   } else {
     const int grid = tiles < kSMs ? tiles : kSMs;
-    e = launch_pdl(kern, dim3(grid), dim3(cellk::kThreads), C::kSmemBytes, s, ta, tb, tgi, thp, thp, tcr, tcz, tcn, tcp, ca, sw, status);
+    e = launch_pdl(kern, dim3(grid), dim3(cellk::kThreads), C::kSmemBytes, s, ta, tb, tgi, thp, taout, tcr, tcz, tcn, tcp, ca, sw, status);
   }
   if (e != cudaSuccess) return false;
   count_launch();
