@@ -250,3 +250,25 @@ def test_misaligned_pointer_is_rejected(B):
     assert B.lib.mgrit_gru_forward(*args(gi.data_ptr())) == 0
     assert B.lib.mgrit_gru_forward(*args(gi.data_ptr() + 16)) == -1      # 16-byte aligned only
     torch.cuda.synchronize()
+
+
+def test_workspace_content_is_irrelevant(B):
+    # only the C-points of the initial guess are cleared by the library: nothing else of the workspace may be read before it
+    # is written, whatever it held (NaN patterns here), forward and adjoint, V- and F-cycles, ragged T
+    w = WORKLOADS["tiny"]
+    d = make_inputs(w)
+    p, x, h0 = upload(d)
+    for flags, T, levels, cf in ((0, w.T, 2, 4), (B.FLAG_F_CYCLE, w.T, 3, 2), (B.FLAG_RAGGED_T, 61, 3, 4)):
+        d2 = make_inputs(w, T=T)
+        p, x, h0 = upload(d2)
+        cfg = _cfg(B, w, 2, levels=levels, cf=cf, T=T, flags=flags)
+        nf, na = B.workspace_bytes(cfg)
+        outs = []
+        for fill in (0x00, 0xFF):
+            ws = torch.full((nf,), fill, dtype=torch.uint8, device="cuda")
+            h, gi, _ = B.mgrit_gru_forward(cfg, p, x, h0, ws=ws)
+            wa = torch.full((na,), fill, dtype=torch.uint8, device="cuda")
+            r = B.mgrit_gru_adjoint(cfg, p, x, h0, gi, h, dhT=h[-1].contiguous(), ws=wa)
+            outs.append([t.clone() for t in (h, r.dh, r.dh0, r.dx, r.dW_hh, r.dW_ih)])
+        for a, b in zip(*outs):
+            assert torch.equal(a, b) and bool(torch.isfinite(a).all())
