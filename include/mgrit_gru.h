@@ -268,6 +268,13 @@ int mgrit_gru_last_device_status(void);
 /* Synchronises the current device and resets its status words to zero. */
 int mgrit_gru_clear_device_status(void);
 
+/* Self-test of the bounded device-side waits (no counterpart in the paper): launches one warp that waits, with the
+ * library's own wait routine and a limit of limit_ms (1..1000) instead of the 2 s of the real kernels, on a barrier
+ * that nothing signals.  The wait runs out, the kernel records it in the status word and returns normally; afterwards
+ * mgrit_gru_last_device_status() reports MGRIT_DEVICE_TIMEOUT until mgrit_gru_clear_device_status() is called.
+ * Asynchronous on `stream`. */
+int mgrit_gru_selftest_bounded_wait(int32_t limit_ms, mgrit_stream_t stream);
+
 /* Number of kernels this library has launched since it was loaded (all streams). */
 unsigned long long mgrit_gru_kernel_launches(void);
 

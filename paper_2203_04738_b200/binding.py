@@ -69,6 +69,7 @@ lib.xent_head_fwd_bwd.argtypes = [_i32, _i32, _i32, _vp, _vp, _vp, _vp, _vp, _vp
 lib.xent_head_fwd_bwd_noalloc.argtypes = [_i32, _i32, _i32, _vp, _vp, _vp, _vp, _vp, _vp, _vp, _vp, _vp]
 lib.sgd_update.argtypes = [_vp, _vp, _sz, ctypes.c_float, _vp]
 lib.adam_update.argtypes = [_vp, _vp, _vp, _vp, _sz, ctypes.c_float, ctypes.c_float, ctypes.c_float, ctypes.c_float, _i32, _vp]
+lib.mgrit_gru_selftest_bounded_wait.argtypes = [_i32, _vp]
 lib.mgrit_gru_last_device_status.restype = ctypes.c_int
 lib.mgrit_gru_clear_device_status.restype = ctypes.c_int
 lib.mgrit_gru_kernel_launches.restype = ctypes.c_ulonglong
@@ -363,6 +364,11 @@ def last_device_status() -> int:
 
 def clear_device_status() -> None:
     _check(lib.mgrit_gru_clear_device_status())
+
+
+def selftest_bounded_wait(limit_ms: int = 20) -> None:
+    """Launch the library's wait self-test: a bounded wait that runs out and records MGRIT_DEVICE_TIMEOUT."""
+    _check(lib.mgrit_gru_selftest_bounded_wait(limit_ms, _stream()))
 
 
 def kernel_launches() -> int:

@@ -1402,6 +1402,8 @@ int mgrit_gru_clear_device_status(void) {
   return (umma_clear_device_status() == 0 && serial_clear_device_status() == 0) ? MGRIT_OK : MGRIT_CUDA_ERROR;
 }
 
+int mgrit_gru_selftest_bounded_wait(int32_t limit_ms, mgrit_stream_t stream) { return umma_selftest_wait(limit_ms, (cudaStream_t)stream); }
+
 unsigned long long mgrit_gru_kernel_launches(void) { return g_kernel_launches.load(std::memory_order_relaxed); }
 
 int mgrit_gru_profile_enable(int on) {

@@ -1513,6 +1513,30 @@ int lstmbf_gradients(const mgrit_gru_cfg* c, const float* dA, const float* x, co
   return ok ? MGRIT_OK : MGRIT_CUDA_ERROR;
 }
 
+// Self-test of the bounded waits: one warp waits, with the library's own wait routine and a short limit, on a barrier
+// that nothing ever signals.  The wait runs out, records its code in the status word and the kernel returns normally.
+namespace {
+__global__ void __launch_bounds__(32) wait_probe_kernel(int* status, unsigned long long limit_ns) {
+  __shared__ __align__(8) unsigned long long bar;
+  __shared__ int abort_flag;
+  if (threadIdx.x == 0) {
+    abort_flag = 0;
+    mbar_init(smem_u32(&bar), 1);
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    mbar_wait(smem_u32(&bar), 0u, &abort_flag, status, 90, limit_ns);
+  }
+}
+}  // namespace
+
+int umma_selftest_wait(int limit_ms, cudaStream_t s) {
+  if (limit_ms < 1 || limit_ms > 1000) return MGRIT_INVALID_ARG;
+  int* const status = status_ptr();
+  if (!status) return MGRIT_CUDA_ERROR;
+  wait_probe_kernel<<<1, 32, 0, s>>>(status, (unsigned long long)limit_ms * 1000000ull);
+  count_launch();
+  return cudaGetLastError() == cudaSuccess ? MGRIT_OK : MGRIT_CUDA_ERROR;
+}
+
 int umma_device_status() {
   const int dev = current_device_slot();
   if (dev < 0) return -1;

@@ -101,6 +101,7 @@ int umma_gradients(const mgrit_gru_cfg* c, const gru_params* p, const float* x, 
                    const gru_grads* g, UmmaAdjWs* w, bool have_xb, cudaStream_t s);
 // the three step functions return MGRIT_OK or MGRIT_CUDA_ERROR (a tensor map could not be encoded, a launch failed)
 int umma_device_status();
+int umma_selftest_wait(int limit_ms, cudaStream_t s);
 int umma_clear_device_status();
 
 }  // namespace mg

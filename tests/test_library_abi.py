@@ -69,6 +69,8 @@ def test_status_calls_answer_without_a_device(lib):
         assert lib.mgrit_gru_clear_device_status() == 0 and lib.mgrit_gru_last_device_status() == 0
     else:
         assert lib.mgrit_gru_last_device_status() == -5 and lib.mgrit_gru_clear_device_status() == -5
+        assert lib.mgrit_gru_selftest_bounded_wait(20, None) == -5        # no device to run the self-test on
+    assert lib.mgrit_gru_selftest_bounded_wait(0, None) == -1 and lib.mgrit_gru_selftest_bounded_wait(5000, None) == -1
 
 
 def test_cycle_variant_flags_are_validated_on_the_host(lib):
