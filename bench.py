@@ -200,6 +200,66 @@ def time_gpu_step(w, T, serial, steps, warmup, dev, use_graph=True):
 
 
 # ------------------------------------------------------------------------------------------ main
+def time_lstm(w, T, dev):
+    """One Implicit-LSTM layer of the workload's shape: MGRIT forward (the workload's forward cycles), adjoint cycles
+    seeded at the last step, all gradients and dx; next to it the serial sweep + exact BPTT (levels = 1).  Host launches."""
+    import numpy as np
+    import torch
+    from paper_2203_04738_b200 import binding as B
+    rng = np.random.default_rng(w.seed + 17)
+    k = 1.0 / np.sqrt(w.H)
+    shapes = dict(W_ih=(4 * w.H, w.I), W_hh=(4 * w.H, w.H), b_ih=(4 * w.H,), b_hh=(4 * w.H,))
+    p = {n: torch.from_numpy(rng.uniform(-k, k, sh).astype(np.float32)).to(dev) for n, sh in shapes.items()}
+    x = torch.from_numpy(np.maximum(rng.standard_normal((T, w.B, w.I)), 0).astype(np.float32)).to(dev)
+    u0 = torch.zeros(2, w.B, w.H, device=dev)
+    dhT = torch.from_numpy(rng.standard_normal((w.B, w.H)).astype(np.float32)).to(dev)
+    out = {}
+    for leg, levels in (("mgrit", w.levels), ("serial", 1)):
+        kw = dict(cf=w.cf, levels=levels, relax_fine=w.relax_fine, relax_coarse=w.relax_coarse, operands=w.operands)
+        cf_ = B.make_cfg(T, w.B, w.I, w.H, iters=w.iters_fwd if levels > 1 else 1, **kw)
+        ca_ = B.make_cfg(T, w.B, w.I, w.H, iters=w.iters_adj if levels > 1 else 1, **kw)
+        nf, na = B.lstm_workspace_bytes(cf_)[0], B.lstm_workspace_bytes(ca_)[1]
+        wsf, wsa = torch.empty(nf, dtype=torch.uint8, device=dev), torch.empty(na, dtype=torch.uint8, device=dev)
+
+        def step():
+            u, gi, _ = B.mgrit_lstm_forward(cf_, p, x, u0, ws=wsf)
+            return B.mgrit_lstm_adjoint(ca_, p, x, u0, gi, u, dhT=dhT, want_du=False, ws=wsa)
+
+        for _ in range(2):
+            step()
+        torch.cuda.synchronize()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        for _ in range(3):
+            step()
+        e1.record()
+        torch.cuda.synchronize()
+        ms = e0.elapsed_time(e1) / 3
+        out[f"{leg}_ms"] = ms
+        if leg == "mgrit":
+            B.profile_enable(True)
+            step()
+            prof = B.profile_read()
+            by_size = {}
+            for name, tms_, fl_ in B.profile_records():
+                e = by_size.setdefault(f"{name}@{fl_ / 1e9:.2f}GF", [0, 0.0])
+                e[0] += 1
+                e[1] += tms_
+            out["kernel_by_size"] = {kk: {"launches_per_step": v[0], "avg_us": v[1] / v[0] * 1e3, "ms_per_step": v[1],
+                                          "tflops": float(kk.split("@")[1][:-2]) * 1e9 / (v[1] / v[0] * 1e-3) / 1e12}
+                                     for kk, v in by_size.items()}
+            B.profile_enable(False)
+            out["kernel_breakdown"] = {kk: {"ms_per_step": v[0], "launches_per_step": v[1],
+                                            "tflops": (v[2] / (v[0] * 1e-3) / 1e12) if v[0] > 0 else None} for kk, v in prof.items()}
+        del wsf, wsa
+        torch.cuda.empty_cache()
+    out.update({"value": T * w.B / (out["mgrit_ms"] * 1e-3), "unit": UNIT, "steps": 3, "launch": "host launches",
+                "speedup_vs_serial": out["serial_ms"] / out["mgrit_ms"],
+                "what": f"one Implicit-LSTM layer, T={T}, B={w.B}, I={w.I}, H={w.H}, operands {OPERAND_NAMES[w.operands]}: "
+                        f"{w.iters_fwd} forward / {w.iters_adj} adjoint cycles + gradients; serial = sweep + exact BPTT"})
+    return out
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -217,6 +277,7 @@ def main():
     ap.add_argument("--no-sweep", action="store_true", help="skip the sequence-length sweep (t_sweep)")
     ap.add_argument("--operands", default=None, choices=["fp32", "tf32", "bf16", "tf32_1pass"],
                     help="override the workload's operand mode (tf32: three-term split on the tensor cores, fp32-level accuracy)")
+    ap.add_argument("--lstm", action="store_true", help="also time one Implicit-LSTM layer of the workload's shape (key lstm)")
     ap.add_argument("--stacked", action="store_true", help="also time the step with all layers in one state (one MGRIT cycle for the stack)")
     args = ap.parse_args()
 
@@ -484,6 +545,9 @@ def main():
         stacked = {"ms_per_step": ms_st, "value": T * w.B / (ms_st * 1e-3), "unit": UNIT, "steps": 3, "launch": "host launches",
                    "what": "all layers in one time-step state, one MGRIT cycle for the stack (generic step kernels: not tuned)"}
         del wsf, wsa
+    lstm = None
+    if rank == 0 and world == 1 and args.lstm:
+        lstm = time_lstm(w, T, dev)
     clocks = None
     if sampler:
         clocks = sampler.stop(*windows["headline"])
@@ -511,7 +575,7 @@ def main():
            "ms_per_step": ms_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
            "dtype": OPERAND_DTYPES[w.operands], "data": "synthetic", "config": config, "clocks": clocks,
            "e2e": e2e, "gpu_launches": int(launches), "roofline": roofline, "cpu_baseline": cpu,
-           "step_stats": step_stats, "forward_only": fwd_only, "gpu_serial": gpu_serial, "t_sweep": t_sweep, "stacked_state": stacked, "roofline_by_class": roofline_by_class,
+           "step_stats": step_stats, "forward_only": fwd_only, "gpu_serial": gpu_serial, "t_sweep": t_sweep, "stacked_state": stacked, "lstm": lstm, "roofline_by_class": roofline_by_class,
            "paper_context": "the paper reports up to 6.5x over serial training on 288 Xeon cores (32 MPI ranks x 9 threads) for T=128; "
                             "another machine and workload: context, not a target",
            "host_enqueue_ms_per_step": host_ms, "kernel_breakdown": breakdown, "kernel_by_size": by_size, "loss": float(loss.item()), "device_status": status}

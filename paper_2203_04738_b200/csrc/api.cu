@@ -1029,10 +1029,16 @@ struct LstmFwdCycle : Cycle {
     a.cout = fw->tmpC; a.hout = fw->tmpH;
     a.gi = gi + ((i64)st * d.tgt_slot - 1) * (i64)bh * 4; a.gi_ks = st * d.tgt_stride * (i64)bh * 4;
     a.W_hh = p->W_hh; a.b_hh = p->b_hh; a.gamma = hr.gamma[d.l]; a.cell = c->cell;
+    // the tensor-core engines write the level array from their epilogue; the FFMA engine leaves raw results to combine
+    const bool fused = c->operands != MGRIT_OPERANDS_FP32;
+    a.up = LstmUpdate{};
+    if (fused)
+      a.up = LstmUpdate{d.out + (size_t)d.out_slot * slot, (i64)d.out_stride * (i64)slot, d.gadd ? d.gadd + (size_t)d.gadd_slot * slot : nullptr,
+                        (i64)d.gadd_stride * (i64)slot, (i64)bh, d.mode};
     if (is_tf32(c)) { int r = tf32_lstm_fwd_step(a, &fw->tf, s); if (r) return r; }
     else if (c->operands == MGRIT_OPERANDS_BF16) { int r = lstmbf_fwd_step(a, &fw->bf, s); if (r) return r; }
     else simt_lstm_fwd_step(a, s);
-    for (int part = 0; part < 2; ++part) {
+    for (int part = 0; part < 2 && !fused; ++part) {
       const float* g = d.gadd ? d.gadd + (size_t)d.gadd_slot * slot + part * bh : nullptr;
       stream_combine_rows(part == 0 ? fw->tmpC : fw->tmpH, g, (i64)d.gadd_stride * slot, d.out + (size_t)d.out_slot * slot + part * bh,
                           (i64)d.out_stride * slot, c->B, c->H, (i64)a.M, d.mode, s);
@@ -1053,10 +1059,15 @@ struct LstmAdjCycle : Cycle {
     a.a = w->a[d.l] + row0; a.p = w->p[d.l] + row0; a.ci = w->ci[d.l] + row0; a.cf = w->cf[d.l] + row0;
     a.cg = w->cg[d.l] + row0; a.co = w->co[d.l] + row0; a.coef_ks = -(i64)d.tgt_stride * (i64)bh;
     a.W_hh = p->W_hh;
+    const bool fused = c->operands != MGRIT_OPERANDS_FP32;
+    a.up = LstmUpdate{};
+    if (fused)
+      a.up = LstmUpdate{d.out + (size_t)d.out_slot * slot, (i64)d.out_stride * (i64)slot, d.gadd ? d.gadd + (size_t)d.gadd_slot * slot : nullptr,
+                        (i64)d.gadd_stride * (i64)slot, (i64)bh, d.mode};
     if (is_tf32(c)) { int r = tf32_lstm_adj_step(a, &w->tf, s); if (r) return r; }
     else if (c->operands == MGRIT_OPERANDS_BF16) { int r = lstmbf_adj_step(a, &w->bf, s); if (r) return r; }
     else simt_lstm_adj_step(a, s);
-    for (int part = 0; part < 2; ++part) {
+    for (int part = 0; part < 2 && !fused; ++part) {
       const float* g = d.gadd ? d.gadd + (size_t)d.gadd_slot * slot + part * bh : nullptr;
       stream_combine_rows(part == 0 ? w->tmpC : w->tmpH, g, (i64)d.gadd_stride * slot, d.out + (size_t)d.out_slot * slot + part * bh,
                           (i64)d.out_stride * slot, c->B, c->H, (i64)a.M, d.mode, s);

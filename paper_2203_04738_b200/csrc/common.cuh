@@ -156,6 +156,11 @@ struct AdjStepArgs {
 };
 
 // ---- Implicit LSTM steps (state of a point = (c, h), 4H gate rows i | f | g | o); rows m = (k, b) as above ----
+// Level-array update formed by the step kernel itself (tensor-core engines): the raw result of row (k, b) goes to
+// out + k*out_ks + b*H (cell part; hidden part at + part) as raw + g (mode 0; g optional, same indexing with g_ks) or as
+// (previous content) - raw (mode 1, FAS right-hand side).  out == nullptr: the raw results go to the contiguous
+// [M, H] arrays of the step instead and the caller combines them.
+struct LstmUpdate { float* out; i64 out_ks; const float* g; i64 g_ks; i64 part; int mode; };
 struct LstmFwdArgs {
   int M, B, H;
   const float* cin; const float* hin; i64 in_ks;    // previous cell / hidden state rows (+ k*in_ks + b*H)
@@ -163,6 +168,7 @@ struct LstmFwdArgs {
   const float* gi; i64 gi_ks;                       // input projection rows (+ k*gi_ks + b*4H)
   const float* W_hh; const float* b_hh;             // [4H, H], [4H]
   float gamma; int cell;
+  LstmUpdate up;
 };
 // coefficients of every step of one level: step j = 1..N leaves fine time t0 + stride_t*(j-1); the given states are
 // c/h[t] at c + (t-1)*ts / h + (t-1)*ts for t >= 1 and c0/h0 for t = 0; outputs [N*B, H] each
@@ -181,6 +187,7 @@ struct LstmAdjArgs {
   float* lc_out; float* lh_out;
   const float *a, *p, *ci, *cf, *cg, *co; i64 coef_ks;
   const float* W_hh;
+  LstmUpdate up;
 };
 void simt_lstm_fwd_step(const LstmFwdArgs& a, cudaStream_t s);
 void simt_lstm_linearise(const LstmLinArgs& a, cudaStream_t s);

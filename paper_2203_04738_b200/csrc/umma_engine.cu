@@ -1298,13 +1298,21 @@ struct EpiLstm {
     }
     const i64 o = (i64)row * H + u0;
     const float gamma = LIN ? l.gamma : f.gamma; const int cell = LIN ? l.cell : f.cell;
+    // the kernel forms the level-array update itself: destination rows, and what is combined with the raw result
+    // (the additive term, or in mode 1 the previous content of the destination)
+    float* udst = nullptr; const float* usrc = nullptr;
+    if (!LIN && f.up.out) {
+      udst = f.up.out + (i64)k * f.up.out_ks + (i64)b * H + u0;
+      usrc = f.up.mode == 1 ? udst : (f.up.g ? f.up.g + (i64)k * f.up.g_ks + (i64)b * H + u0 : nullptr);
+    }
 #pragma unroll 1
     for (int c0 = half * 32; c0 < half * 32 + 32; c0 += 8) {
-      float g4[4][8], cp[8], acc[4][8];
+      float g4[4][8], cp[8], acc[4][8], tc[8], th[8];
       if (valid) {
 #pragma unroll
         for (int g = 0; g < 4; ++g) ld8(gi + (i64)g * H + c0, g4[g]);
         ld8(cpp + c0, cp);
+        if (!LIN && usrc) { ld8(usrc + c0, tc); ld8(usrc + f.up.part + c0, th); }
       }
 #pragma unroll
       for (int g = 0; g < 4; ++g) tmem_ld8(taddr + g * 64 + c0, acc[g]);
@@ -1327,9 +1335,53 @@ struct EpiLstm {
         if (LIN) {
           st8(l.a + o + c0, o0); st8(l.p + o + c0, o1); st8(l.ci + o + c0, o2); st8(l.cf + o + c0, o3); st8(l.cg + o + c0, o4);
           st8(l.co + o + c0, o5);
+        } else if (udst) {
+          if (usrc) {
+#pragma unroll
+            for (int e = 0; e < 8; ++e) {
+              o0[e] = f.up.mode == 1 ? tc[e] - o0[e] : o0[e] + tc[e];
+              o1[e] = f.up.mode == 1 ? th[e] - o1[e] : o1[e] + th[e];
+            }
+          }
+          st8(udst + c0, o0); st8(udst + f.up.part + c0, o1);
         } else {
           st8(f.cout + o + c0, o0); st8(f.hout + o + c0, o1);
         }
+      }
+    }
+  }
+};
+
+// cell-part result of an adjoint step: raw to lc_out, or straight into the level array (see LstmUpdate)
+__device__ __forceinline__ void lstm_store_lc(const LstmAdjArgs& a, i64 e, i64 kk, int b, int i, float v) {
+  if (!a.up.out) { a.lc_out[e] = v; return; }
+  float* d = a.up.out + kk * a.up.out_ks + (i64)b * a.H + i;
+  if (a.up.mode == 1) *d = *d - v;
+  else *d = a.up.g ? v + a.up.g[kk * a.up.g_ks + (i64)b * a.H + i] : v;
+}
+
+// hidden-part result of an adjoint step written into the level array: out = acc + g, or (previous content) - acc
+template <int BN>
+struct EpiUpdate {
+  LstmUpdate u; int M, N, B;
+  __device__ void operator()(uint32_t taddr, int row, int n0, int half) const {
+    const bool valid = row < M;
+    const int k = valid ? row / B : 0, b = valid ? row % B : 0;
+    float* o = u.out + u.part + (i64)k * u.out_ks + (i64)b * N + n0;
+    const float* g = u.mode == 1 ? o : (u.g ? u.g + u.part + (i64)k * u.g_ks + (i64)b * N + n0 : nullptr);
+    const int cbeg = half * (BN / 2);
+    for (int c0 = cbeg; c0 < cbeg + BN / 2 && n0 + c0 < N; c0 += 16) {
+      float v[16], t[16];
+      if (valid && g) { ld8(g + c0, t); ld8(g + c0 + 8, t + 8); }
+      tmem_ld16(taddr + c0, v);
+      tmem_ld_wait();
+      if (valid) {
+        if (g) {
+#pragma unroll
+          for (int e = 0; e < 16; ++e) v[e] = u.mode == 1 ? t[e] - v[e] : v[e] + t[e];
+        }
+        st8(o + c0, v);
+        st8(o + c0 + 8, v + 8);
       }
     }
   }
@@ -1345,7 +1397,7 @@ __global__ void __launch_bounds__(kPT) split_lstm_adj_kernel(LstmAdjArgs a, int 
     const i64 kk = m / a.B; const int b = (int)(m % a.B);
     const i64 ci = kk * a.coef_ks + (i64)b * a.H + i, li = kk * a.in_ks + (i64)b * a.H + i;
     const float lh = a.lh[li], dc = a.lc[li] + a.p[ci] * lh;
-    a.lc_out[e] = a.a[ci] * dc;
+    lstm_store_lc(a, e, kk, b, i, a.a[ci] * dc);
     const float v[4] = {a.ci[ci] * dc, a.cf[ci] * dc, a.cg[ci] * dc, a.co[ci] * lh};
     for (int seg = 0; seg < S; ++seg)
 #pragma unroll
@@ -1389,8 +1441,11 @@ int tf32_lstm_adj_step(const LstmAdjArgs& a, Tf32Ws* w, cudaStream_t s) {
   ProfScope prof(KC_ADJ_STEP, 2.0 * a.M * (double)K * a.H, s);
   if (launch_pdl(split_lstm_adj_kernel, dim3(pgrid((i64)a.M * a.H)), dim3(kPT), 0, s, a, S, w->Apack) != cudaSuccess) return MGRIT_CUDA_ERROR;
   count_launch();
-  return launch_gemm<256, 0>(KC_ADJ_STEP, (const float*)w->Apack, (i64)K, (const float*)w->W_hhT, (i64)K, a.M, a.H, K, 0, a.H,
-                             EpiStore{a.lh_out, a.H, a.M, a.H, 0}, s) ? MGRIT_OK : MGRIT_CUDA_ERROR;
+  const bool ok = a.up.out ? launch_gemm<256, 0>(KC_ADJ_STEP, (const float*)w->Apack, (i64)K, (const float*)w->W_hhT, (i64)K, a.M, a.H, K, 0, a.H,
+                                                 EpiUpdate<256>{a.up, a.M, a.H, a.B}, s)
+                           : launch_gemm<256, 0>(KC_ADJ_STEP, (const float*)w->Apack, (i64)K, (const float*)w->W_hhT, (i64)K, a.M, a.H, K, 0, a.H,
+                                                 EpiStore{a.lh_out, a.H, a.M, a.H, 0}, s);
+  return ok ? MGRIT_OK : MGRIT_CUDA_ERROR;
 }
 
 // ---------------------------------------------------------------- Implicit LSTM, bf16 operands
@@ -1405,7 +1460,7 @@ __global__ void __launch_bounds__(kPT) pack_lstm_adj_kernel(LstmAdjArgs a, bf16*
     const i64 kk = m / a.B; const int b = (int)(m % a.B);
     const i64 ci = kk * a.coef_ks + (i64)b * a.H + i, li = kk * a.in_ks + (i64)b * a.H + i;
     const float lh = a.lh[li], dc = a.lc[li] + a.p[ci] * lh;
-    a.lc_out[e] = a.a[ci] * dc;
+    lstm_store_lc(a, e, kk, b, i, a.a[ci] * dc);
     bf16* d = dst + m * 4 * a.H + i;
     d[0] = __float2bfloat16(a.ci[ci] * dc); d[a.H] = __float2bfloat16(a.cf[ci] * dc);
     d[2 * a.H] = __float2bfloat16(a.cg[ci] * dc); d[3 * a.H] = __float2bfloat16(a.co[ci] * lh);
@@ -1494,8 +1549,14 @@ int lstmbf_adj_step(const LstmAdjArgs& a, LstmBfWs* w, cudaStream_t s) {
   ProfScope prof(KC_ADJ_STEP, 2.0 * a.M * (double)K * a.H, s);
   if (launch_pdl(pack_lstm_adj_kernel, dim3(pgrid((i64)a.M * a.H)), dim3(kPT), 0, s, a, w->Apack) != cudaSuccess) return MGRIT_CUDA_ERROR;
   count_launch();
-  return launch_gemm<256, 0>(KC_ADJ_STEP, w->Apack, K, w->W_hhT, K, a.M, a.H, K, 0, a.H, EpiStore{a.lh_out, a.H, a.M, a.H, 0}, s) ? MGRIT_OK
-                                                                                                                              : MGRIT_CUDA_ERROR;
+  // few-row steps (coarse levels, the serial sweep): 64-column tiles spread the stream over K over four times the CTAs
+  const bool few = ((a.M + BM - 1) / BM) * ((a.H + 255) / 256) * 2 <= kSMs;
+  const bool ok = !a.up.out ? launch_gemm<256, 0>(KC_ADJ_STEP, w->Apack, K, w->W_hhT, K, a.M, a.H, K, 0, a.H, EpiStore{a.lh_out, a.H, a.M, a.H, 0}, s)
+                  : few     ? launch_gemm<64, 0>(KC_ADJ_STEP, w->Apack, K, w->W_hhT, K, a.M, a.H, K, 0, a.H, EpiUpdate<64>{a.up, a.M, a.H, a.B}, s)
+                  : gemm_pair_enabled(a.M, a.H)
+                            ? launch_gemm_pair(KC_ADJ_STEP, w->Apack, K, w->W_hhT, K, a.M, a.H, K, a.H, EpiUpdate<256>{a.up, a.M, a.H, a.B}, s)
+                            : launch_gemm<256, 0>(KC_ADJ_STEP, w->Apack, K, w->W_hhT, K, a.M, a.H, K, 0, a.H, EpiUpdate<256>{a.up, a.M, a.H, a.B}, s);
+  return ok ? MGRIT_OK : MGRIT_CUDA_ERROR;
 }
 
 int lstmbf_gradients(const mgrit_gru_cfg* c, const float* dA, const float* x, const float* h0, const float* hk, const gru_grads* g,
