@@ -978,11 +978,15 @@ int stack_adjoint_impl(const mgrit_gru_cfg* cfg, int nl, const gru_params* p, co
 // ======================================================================================================
 // Implicit LSTM: the state of a time point is (c, h); level arrays are [N_l + 1][2][B][H] (part 0 = c, part 1 = h) and
 // the same Cycle drives them.  fp32 engine only (four-gate FFMA products).
-struct LstmFwdWs { float* U[kMaxLevels]; float* G[kMaxLevels]; double* res_acc; float *tmpC, *tmpH; size_t maxM; Tf32Ws tf; LstmBfWs bf; };
+struct LstmFwdWs {
+  float* U[kMaxLevels]; float* G[kMaxLevels]; double* res_acc; float *tmpC, *tmpH; size_t maxM; Tf32Ws tf; LstmBfWs bf;
+  uint4* chain_xw; size_t chain_xw_bytes;      // exchange words of the persistent chain kernel (bf16 operands)
+};
 struct LstmAdjWs {
   float* U[kMaxLevels]; float* G[kMaxLevels]; double* res_acc;
   float *a[kMaxLevels], *p[kMaxLevels], *ci[kMaxLevels], *cf[kMaxLevels], *cg[kMaxLevels], *co[kMaxLevels];
   float *tmpC, *tmpH, *hk, *dA; size_t maxM; Tf32Ws tf; LstmBfWs bf;
+  uint4* chain_xw; size_t chain_xw_bytes;
 };
 
 void plan_lstm_fwd(const mgrit_gru_cfg* c, const Hier& hr, Ws& w, LstmFwdWs* o) {
@@ -997,6 +1001,11 @@ void plan_lstm_fwd(const mgrit_gru_cfg* c, const Hier& hr, Ws& w, LstmFwdWs* o) 
   o->tmpH = w.take<float>(o->maxM * c->H);
   if (is_tf32(c)) tf32_plan_fwd(c, hr.N, hr.L, w.base, &w.off, &o->tf, 4);
   if (c->operands == MGRIT_OPERANDS_BF16) lstmbf_plan_fwd(c, o->maxM, w.base, &w.off, &o->bf);
+  o->chain_xw = nullptr; o->chain_xw_bytes = 0;
+  if (c->operands == MGRIT_OPERANDS_BF16 && c->H % 128 == 0) {
+    o->chain_xw_bytes = serial_xw_bytes(c->B, c->H, 1);
+    o->chain_xw = reinterpret_cast<uint4*>(w.take<char>(o->chain_xw_bytes));
+  }
 }
 
 void plan_lstm_adj(const mgrit_gru_cfg* c, const Hier& hr, Ws& w, LstmAdjWs* o) {
@@ -1016,10 +1025,25 @@ void plan_lstm_adj(const mgrit_gru_cfg* c, const Hier& hr, Ws& w, LstmAdjWs* o) 
   o->dA = w.take<float>(TB * 4 * c->H);
   if (is_tf32(c)) tf32_plan_adj(c, hr.N, hr.L, w.base, &w.off, &o->tf, 4);
   if (c->operands == MGRIT_OPERANDS_BF16) lstmbf_plan_adj(c, o->maxM, w.base, &w.off, &o->bf);
+  o->chain_xw = nullptr; o->chain_xw_bytes = 0;
+  if (c->operands == MGRIT_OPERANDS_BF16 && c->H % 128 == 0) {
+    o->chain_xw_bytes = serial_xw_bytes(c->B, c->H, 4);
+    o->chain_xw = reinterpret_cast<uint4*>(w.take<char>(o->chain_xw_bytes));
+  }
 }
 
 struct LstmFwdCycle : Cycle {
   const gru_params* p; const float* gi; LstmFwdWs* fw;
+  bool chain(int l) override {
+    if (c->operands != MGRIT_OPERANDS_BF16 || !fw->chain_xw) return false;
+    const i64 bh = (i64)c->B * c->H, st = hr.stride_t[l];
+    LstmChainFwdArgs a{};
+    a.B = c->B; a.H = c->H; a.nsteps = hr.N[l]; a.u = U[l];
+    a.gi = gi + (st - 1) * bh * 4; a.gi_step = st * bh * 4;
+    a.g = G[l]; a.W = fw->bf.W_hh; a.b_hh = p->b_hh; a.gamma = hr.gamma[l]; a.cell = c->cell;
+    a.xw = fw->chain_xw; a.xw_bytes = fw->chain_xw_bytes;
+    return lstm_chain_fwd_solve(a, s);
+  }
   int launch_step(const StepDesc& d) override {
     const size_t bh = (size_t)c->B * c->H, slot = 2 * bh;
     const i64 st = hr.stride_t[d.l];
@@ -1049,6 +1073,18 @@ struct LstmFwdCycle : Cycle {
 
 struct LstmAdjCycle : Cycle {
   const gru_params* p; LstmAdjWs* w;
+  bool chain(int l) override {
+    if (c->operands != MGRIT_OPERANDS_BF16 || !w->chain_xw) return false;
+    const i64 bh = (i64)c->B * c->H;
+    const i64 row0 = (i64)(hr.N[l] - 1) * bh;     // step s = 1 applies forward step N_l, stored at row N_l - 1
+    LstmChainAdjArgs a{};
+    a.B = c->B; a.H = c->H; a.nsteps = hr.N[l]; a.mu = U[l];
+    a.a = w->a[l] + row0; a.p = w->p[l] + row0; a.ci = w->ci[l] + row0; a.cf = w->cf[l] + row0; a.cg = w->cg[l] + row0;
+    a.co = w->co[l] + row0; a.coef_step = -bh;
+    a.g = G[l]; a.WT = w->bf.W_hhT;
+    a.xw = w->chain_xw; a.xw_bytes = w->chain_xw_bytes;
+    return lstm_chain_adj_solve(a, s);
+  }
   int launch_step(const StepDesc& d) override {
     const size_t bh = (size_t)c->B * c->H, slot = 2 * bh;
     const i64 row0 = (i64)(hr.N[d.l] - d.tgt_slot) * (i64)bh;

@@ -67,6 +67,32 @@ bool serial_adj_supported(int B, int H);
 // false: shape not supported or the cooperative launch failed (the caller then advances step by step)
 bool serial_fwd_solve(const SerialFwdArgs& a, cudaStream_t s);
 bool serial_adj_solve(const SerialAdjArgs& a, cudaStream_t s);
+// Implicit LSTM chains, bf16 operands.  A state slot is (c, h): arrays [nsteps+1][2][B][H], slot 0 given.
+//   forward:  (c, h)_j = Phi_gamma(gi_j, (c, h)_{j-1}) + g_j
+//   adjoint:  dc = Lc + p*Lh;  (Lc, Lh)_s = (a*dc, [ci*dc | cf*dc | cg*dc | co*Lh] W_hh) + g_s   (coefficients of step s)
+struct LstmChainFwdArgs {
+  int B, H, nsteps;
+  float* u;
+  const float* gi; i64 gi_step;  // projection rows of step 1 (+ (j-1)*gi_step for step j), row b at + b*4H
+  const float* g;                // [nsteps+1][2][B][H] additive term, or nullptr
+  const __nv_bfloat16* W;        // [4H][H]
+  const float* b_hh;
+  float gamma; int cell;
+  uint4* xw; size_t xw_bytes;    // exchange words, serial_xw_bytes(B, H, 1)
+};
+struct LstmChainAdjArgs {
+  int B, H, nsteps;
+  float* mu;
+  const float *a, *p, *ci, *cf, *cg, *co;   // coefficient rows of step 1; step s at + (s-1)*coef_step
+  i64 coef_step;
+  const float* g;
+  const __nv_bfloat16* WT;       // [H][4H] = W_hh^T
+  uint4* xw; size_t xw_bytes;    // exchange words, serial_xw_bytes(B, H, 4)
+};
+bool lstm_chain_fwd_supported(int B, int H);
+bool lstm_chain_adj_supported(int B, int H);
+bool lstm_chain_fwd_solve(const LstmChainFwdArgs& a, cudaStream_t s);
+bool lstm_chain_adj_solve(const LstmChainAdjArgs& a, cudaStream_t s);
 int serial_device_status();
 int serial_clear_device_status();
 

@@ -435,6 +435,235 @@ __global__ void __launch_bounds__(kThreads, 1) serial_adj_kernel(SerialAdjArgs a
 }
 
 // ================================================================================================
+// Implicit LSTM chains (bf16 operands, flag-in-data exchange).  The structure is that of the GRU chains above; a
+// time point's state is (c, h): the cell state never leaves the thread that owns its (row, unit), only h crosses CTAs.
+//
+// forward:  gates from gi_j and h_{j-1} W_hh^T (four gate rows per unit in shared memory), (c, h)_j = cell + g_j
+template <int UNC>
+__global__ void __launch_bounds__(kThreads, 1) lstm_fwd_chain_kernel(LstmChainFwdArgs a, int* status) {
+  constexpr int NW = 4 * UNC, NT = NW / 8, OPT = (kRows * UNC + kThreads - 1) / kThreads;
+  constexpr int kBlockVals = kRows * UNC, kBlockWords = (kBlockVals + kValsPerWord - 1) / kValsPerWord;
+  __shared__ __align__(16) bf16 xstage[kRows * 32];
+  extern __shared__ __align__(16) uint8_t smem[];
+  const int H = a.H, ldk = H + 8;
+  bf16* Ws = reinterpret_cast<bf16*>(smem);                 // [NW][ldk]
+  bf16* As = Ws + NW * ldk;                                 // [16][ldk]
+  float* red = reinterpret_cast<float*>(As + kRows * ldk);  // [8][16][NW]
+  __shared__ int ok_smem;
+  const int tid = threadIdx.x, warp = tid >> 5;
+  const int u0 = blockIdx.x * UNC, rg = blockIdx.y, row0 = rg * kRows;
+  const int nrows = min(kRows, a.B - row0);
+  const i64 BH = (i64)a.B * H, slot = 2 * BH;
+
+  for (int e = tid; e < NW * (H / 8); e += kThreads) {      // weight rows gate*H + u0 + i, resident for the whole chain
+    int r = e / (H / 8), c = e % (H / 8);
+    int gate = r / UNC, i = r % UNC;
+    *reinterpret_cast<uint4*>(Ws + r * ldk + c * 8) =
+        __ldg(reinterpret_cast<const uint4*>(a.W + ((i64)gate * H + u0 + i) * H + c * 8));
+  }
+  for (int e = tid; e < kRows * ldk / 2; e += kThreads) reinterpret_cast<uint32_t*>(As)[e] = 0u;     // rows beyond the batch stay zero
+  if (tid == 0) ok_smem = 1;
+  __syncthreads();
+  for (int e = tid; e < nrows * (H / 4); e += kThreads) {   // step 1 reads the fp32 initial hidden state
+    int r = e / (H / 4), c = e % (H / 4);
+    float4 v = __ldcg(reinterpret_cast<const float4*>(a.u + BH + (i64)(row0 + r) * H + c * 4));
+    __nv_bfloat162 lo = __floats2bfloat162_rn(v.x, v.y), hi = __floats2bfloat162_rn(v.z, v.w);
+    uint2 o; o.x = *reinterpret_cast<uint32_t*>(&lo); o.y = *reinterpret_cast<uint32_t*>(&hi);
+    *reinterpret_cast<uint2*>(As + r * ldk + c * 4) = o;
+  }
+  float cp[OPT], pgi[OPT][4], bia[OPT][4], pgc[OPT], pgh[OPT];
+#pragma unroll
+  for (int o = 0; o < OPT; ++o) {
+    int idx = tid + o * kThreads, r = idx / UNC, i = idx % UNC;
+    bool v = idx < kRows * UNC && r < nrows;
+    const i64 off = (i64)(row0 + r) * H + u0 + i;
+    cp[o] = v ? __ldcg(a.u + off) : 0.f;
+#pragma unroll
+    for (int g = 0; g < 4; ++g) {
+      bia[o][g] = a.b_hh[g * H + u0 + i];
+      pgi[o][g] = v ? a.gi[(i64)(row0 + r) * 4 * H + g * H + u0 + i] : 0.f;
+    }
+    pgc[o] = (v && a.g) ? a.g[slot + off] : 0.f;
+    pgh[o] = (v && a.g) ? a.g[slot + BH + off] : 0.f;
+  }
+  __syncthreads();
+
+  const int kw = H / kWarps;
+  for (int j = 1; j <= a.nsteps; ++j) {
+    float acc[NT][4];
+#pragma unroll
+    for (int nt = 0; nt < NT; ++nt) acc[nt][0] = acc[nt][1] = acc[nt][2] = acc[nt][3] = 0.f;
+    warp_gemm<NT>(As, Ws, ldk, warp * kw, (warp + 1) * kw, acc);
+    store_partials<NT>(red, acc);
+    __syncthreads();
+#pragma unroll
+    for (int o = 0; o < OPT; ++o) {
+      int idx = tid + o * kThreads, r = idx / UNC, i = idx % UNC;
+      float hv = 0.f;
+      if (idx < kRows * UNC && r < nrows) {
+        float gh[4];
+#pragma unroll
+        for (int g = 0; g < 4; ++g) gh[g] = sum_partials<NW>(red, r, g * UNC + i) + bia[o][g];
+        LstmOut q = lstm_forward<true>(pgi[o][0], pgi[o][1], pgi[o][2], pgi[o][3], gh[0], gh[1], gh[2], gh[3], cp[o], a.gamma, a.cell);
+        const float cv = q.c + pgc[o];
+        hv = q.h + pgh[o];
+        cp[o] = cv;
+        const i64 off = (i64)(row0 + r) * H + u0 + i;
+        a.u[(i64)j * slot + off] = cv;
+        a.u[(i64)j * slot + BH + off] = hv;
+      }
+      if (idx < kRows * UNC) xstage[idx] = __float2bfloat16(hv);      // rows beyond the batch travel as zeros
+    }
+    if (j == a.nsteps) break;
+    __syncthreads();
+    publish_block(xstage, kBlockVals, a.xw + ((i64)(rg * 2 + (j & 1)) * gridDim.x + blockIdx.x) * kBlockWords, (unsigned)j);
+    // operands of the next step that do not depend on other CTAs (nothing may depend on these loads before the exchange)
+#pragma unroll
+    for (int o = 0; o < OPT; ++o) {
+      int idx = tid + o * kThreads, r = idx / UNC, i = idx % UNC;
+      if (idx < kRows * UNC && r < nrows) {
+        const float* gi = a.gi + (i64)j * a.gi_step + (i64)(row0 + r) * 4 * H + u0 + i;
+#pragma unroll
+        for (int g = 0; g < 4; ++g) pgi[o][g] = gi[g * H];
+        if (a.g) {
+          const i64 off = (i64)(j + 1) * slot + (i64)(row0 + r) * H + u0 + i;
+          pgc[o] = a.g[off]; pgh[o] = a.g[off + BH];
+        }
+      }
+    }
+    const bool ok = gather_blocks<UNC, 1>(a.xw + (i64)(rg * 2 + (j & 1)) * gridDim.x * kBlockWords, (int)gridDim.x, (unsigned)j, As, ldk, H,
+                                          status);
+    if (!ok) ok_smem = 0;
+    __syncthreads();
+    if (ok_smem == 0) return;
+  }
+}
+
+// adjoint:  the CTA owns UNC output units (columns of W_hh) over all K = 4H reduction indices.  Its slice of W_hh^T
+// (UNC x 4H bf16, up to 128 KB) does not fit shared memory next to the 16 x 4H operand rows, so it lives in REGISTERS
+// for the whole chain: warp w reduces k in [w*K/8, (w+1)*K/8) and a lane keeps exactly the B fragments of its
+// m16n8k16 products there (KS k-steps x UNC/8 column tiles x 2 words; 128 registers at H = 1024, UNC = 16).
+// The bf16 operand [ci*dc | cf*dc | cg*dc | co*Lh] of the NEXT step is formed by the CTA that produced (Lc, Lh).
+template <int UNC, int KS>
+__global__ void __launch_bounds__(kThreads, 1) lstm_adj_chain_kernel(LstmChainAdjArgs a, int* status) {
+  constexpr int NT = UNC / 8, OPT = (kRows * UNC + kThreads - 1) / kThreads;
+  constexpr int kBlockVals = 4 * kRows * UNC, kBlockWords = (kBlockVals + kValsPerWord - 1) / kValsPerWord;
+  __shared__ __align__(16) bf16 xstage[4 * kRows * 16];
+  extern __shared__ __align__(16) uint8_t smem[];
+  const int H = a.H, K = 4 * H, ldk = K + 8;
+  bf16* As = reinterpret_cast<bf16*>(smem);                 // [16][ldk]
+  float* red = reinterpret_cast<float*>(As + kRows * ldk);  // [8][16][UNC]
+  __shared__ int ok_smem;
+  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31, lg = lane >> 2, lt = lane & 3;
+  const int u0 = blockIdx.x * UNC, rg = blockIdx.y, row0 = rg * kRows;
+  const int nrows = min(kRows, a.B - row0);
+  const i64 BH = (i64)a.B * H, slot = 2 * BH;
+  const int kbeg = warp * (K / kWarps);                     // K / 8 = 16 KS
+
+  uint32_t wreg[KS][NT][2];
+#pragma unroll
+  for (int ks = 0; ks < KS; ++ks)
+#pragma unroll
+    for (int nt = 0; nt < NT; ++nt) {
+      const bf16* wp = a.WT + (i64)(u0 + nt * 8 + lg) * K + kbeg + 16 * ks + 2 * lt;
+      wreg[ks][nt][0] = __ldg(reinterpret_cast<const uint32_t*>(wp));
+      wreg[ks][nt][1] = __ldg(reinterpret_cast<const uint32_t*>(wp + 8));
+    }
+  for (int e = tid; e < kRows * ldk / 2; e += kThreads) reinterpret_cast<uint32_t*>(As)[e] = 0u;
+  if (tid == 0) ok_smem = 1;
+  __syncthreads();
+  // step 1: operand from the given sensitivities (slot 0) and the coefficients of step 1, all 4H columns of this row group
+  for (int e = tid; e < nrows * H; e += kThreads) {
+    int r = e / H, i = e % H;
+    const i64 off = (i64)(row0 + r) * H + i;
+    const float lh = __ldcg(a.mu + BH + off), dc = __ldcg(a.mu + off) + a.p[off] * lh;
+    As[r * ldk + i] = __float2bfloat16(a.ci[off] * dc);
+    As[r * ldk + H + i] = __float2bfloat16(a.cf[off] * dc);
+    As[r * ldk + 2 * H + i] = __float2bfloat16(a.cg[off] * dc);
+    As[r * ldk + 3 * H + i] = __float2bfloat16(a.co[off] * lh);
+  }
+  // per owned (row, unit): dc of the step in flight, its a and source terms; the coefficients of the step after it
+  float dcur[OPT], pa[OPT], pgc[OPT], pgh[OPT], np_[OPT], nci[OPT], ncf[OPT], ncg[OPT], nco[OPT];
+#pragma unroll
+  for (int o = 0; o < OPT; ++o) {
+    int idx = tid + o * kThreads, r = idx / UNC, i = idx % UNC;
+    bool v = idx < kRows * UNC && r < nrows;
+    const i64 off = (i64)(row0 + r) * H + u0 + i;
+    dcur[o] = v ? __ldcg(a.mu + off) + a.p[off] * __ldcg(a.mu + BH + off) : 0.f;
+    pa[o] = v ? a.a[off] : 0.f;
+    pgc[o] = (v && a.g) ? a.g[slot + off] : 0.f;
+    pgh[o] = (v && a.g) ? a.g[slot + BH + off] : 0.f;
+    const bool more = v && a.nsteps > 1;
+    const i64 co = a.coef_step + off;
+    np_[o] = more ? a.p[co] : 0.f; nci[o] = more ? a.ci[co] : 0.f; ncf[o] = more ? a.cf[co] : 0.f;
+    ncg[o] = more ? a.cg[co] : 0.f; nco[o] = more ? a.co[co] : 0.f;
+  }
+  __syncthreads();
+
+  for (int s = 1; s <= a.nsteps; ++s) {
+    float acc[NT][4];
+#pragma unroll
+    for (int nt = 0; nt < NT; ++nt) acc[nt][0] = acc[nt][1] = acc[nt][2] = acc[nt][3] = 0.f;
+#pragma unroll
+    for (int ks = 0; ks < KS; ++ks) {
+      const int k0 = kbeg + 16 * ks;
+      uint32_t af[4];
+      af[0] = *reinterpret_cast<const uint32_t*>(As + lg * ldk + k0 + 2 * lt);
+      af[1] = *reinterpret_cast<const uint32_t*>(As + (lg + 8) * ldk + k0 + 2 * lt);
+      af[2] = *reinterpret_cast<const uint32_t*>(As + lg * ldk + k0 + 2 * lt + 8);
+      af[3] = *reinterpret_cast<const uint32_t*>(As + (lg + 8) * ldk + k0 + 2 * lt + 8);
+#pragma unroll
+      for (int nt = 0; nt < NT; ++nt) mma16816(acc[nt], af, wreg[ks][nt][0], wreg[ks][nt][1]);
+    }
+    store_partials<NT>(red, acc);
+    __syncthreads();
+#pragma unroll
+    for (int o = 0; o < OPT; ++o) {
+      int idx = tid + o * kThreads, r = idx / UNC, i = idx % UNC;
+      const bool live = idx < kRows * UNC && r < nrows;
+      float x4[4] = {0.f, 0.f, 0.f, 0.f};
+      if (live) {
+        const float lc = pa[o] * dcur[o] + pgc[o];
+        const float lh = sum_partials<UNC>(red, r, i) + pgh[o];
+        const i64 off = (i64)(row0 + r) * H + u0 + i;
+        a.mu[(i64)s * slot + off] = lc;
+        a.mu[(i64)s * slot + BH + off] = lh;
+        const float dn = lc + np_[o] * lh;      // the next step's dc (its coefficients are zero behind the last step)
+        dcur[o] = dn;
+        x4[0] = nci[o] * dn; x4[1] = ncf[o] * dn; x4[2] = ncg[o] * dn; x4[3] = nco[o] * lh;
+      }
+      if (idx < kRows * UNC) {                  // block order [gate][row][unit]; rows beyond the batch travel as zeros
+#pragma unroll
+        for (int g = 0; g < 4; ++g) xstage[g * kRows * UNC + idx] = __float2bfloat16(x4[g]);
+      }
+    }
+    if (s == a.nsteps) break;
+    __syncthreads();
+    publish_block(xstage, kBlockVals, a.xw + ((i64)(rg * 2 + (s & 1)) * gridDim.x + blockIdx.x) * kBlockWords, (unsigned)s);
+#pragma unroll
+    for (int o = 0; o < OPT; ++o) {             // operands of the steps to come that do not depend on other CTAs
+      int idx = tid + o * kThreads, r = idx / UNC, i = idx % UNC;
+      if (idx < kRows * UNC && r < nrows) {
+        const i64 off = (i64)(row0 + r) * H + u0 + i;
+        pa[o] = a.a[(i64)s * a.coef_step + off];
+        if (a.g) { pgc[o] = a.g[(i64)(s + 1) * slot + off]; pgh[o] = a.g[(i64)(s + 1) * slot + BH + off]; }
+        if (s + 1 < a.nsteps) {
+          const i64 co = (i64)(s + 1) * a.coef_step + off;
+          np_[o] = a.p[co]; nci[o] = a.ci[co]; ncf[o] = a.cf[co]; ncg[o] = a.cg[co]; nco[o] = a.co[co];
+        } else {
+          np_[o] = nci[o] = ncf[o] = ncg[o] = nco[o] = 0.f;
+        }
+      }
+    }
+    const bool ok = gather_blocks<UNC, 4>(a.xw + (i64)(rg * 2 + (s & 1)) * gridDim.x * kBlockWords, (int)gridDim.x, (unsigned)s, As, ldk, H,
+                                          status);
+    if (!ok) ok_smem = 0;
+    __syncthreads();
+    if (ok_smem == 0) return;
+  }
+}
+
+// ================================================================================================
 // fp32 chains: the same two recurrences in FFMA arithmetic with precise gate math.  K is split over the 8 warps; a
 // lane owns 4 rows x CPL columns of the 16 x (8 CPL) outputs (the 8 lanes of a quarter warp read the same A words --
 // a broadcast -- and W rows 3 CPL (H + 4) floats apart: conflict-free 16-byte loads).
@@ -792,6 +1021,78 @@ bool serial_adj_solve(const SerialAdjArgs& a, cudaStream_t s) {
                : (unc == 8 ? launch_coop(serial_adj_kernel<8, false>, a, unc, smem, false, 3, s)
                   : unc == 16 ? launch_coop(serial_adj_kernel<16, false>, a, unc, smem, false, 3, s)
                               : launch_coop(serial_adj_kernel<32, false>, a, unc, smem, false, 3, s));
+  prof_end(s);
+  return ok;
+}
+
+// ---- Implicit LSTM chains
+namespace {
+size_t lstm_fwd_smem(int unc, int H) { return (size_t)(4 * unc + kRows) * (H + 8) * 2 + (size_t)kWarps * kRows * 4 * unc * 4; }
+size_t lstm_adj_smem(int unc, int H) { return (size_t)kRows * (4 * H + 8) * 2 + (size_t)kWarps * kRows * unc * 4; }
+int lstm_pick_unc(int B, int H, bool adj) {
+  if (adj ? !(H == 128 || H == 256 || H == 512 || H == 1024) : H % 128 != 0) return 0;
+  const int rgs = (B + kRows - 1) / kRows;
+  const int cands[3] = {8, 16, 32};
+  for (int c : cands) {
+    if (H % c != 0 || (adj && c > 16)) continue;
+    if ((i64)(H / c) * rgs > sm_count()) continue;
+    if ((adj ? lstm_adj_smem(c, H) : lstm_fwd_smem(c, H)) > kSmemLimit) continue;
+    return c;
+  }
+  return 0;
+}
+template <class Args, class Kern>
+bool launch_lstm_chain(Kern kern, const Args& a, int unc, size_t smem, int gates, cudaStream_t s) {
+  if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess) return false;
+  const int rgs = (a.B + kRows - 1) / kRows;
+  // no exchange word may carry a step number of an earlier launch
+  const size_t words = (size_t)rgs * 2 * (a.H / unc) * ((size_t)(gates * kRows * unc + kValsPerWord - 1) / kValsPerWord);
+  if (words * sizeof(uint4) > a.xw_bytes) return false;
+  if (cudaMemsetAsync(a.xw, 0, words * sizeof(uint4), s) != cudaSuccess) return false;
+  Args args = a;
+  int* st = status_ptr();
+  if (!st) return false;
+  void* params[2] = {(void*)&args, (void*)&st};
+  if (cudaLaunchCooperativeKernel((const void*)kern, dim3(a.H / unc, rgs), dim3(kThreads), params, smem, s) != cudaSuccess) {
+    cudaGetLastError();
+    return false;
+  }
+  count_launch();
+  return true;
+}
+template <int UNC>
+bool launch_lstm_adj(const LstmChainAdjArgs& a, size_t smem, cudaStream_t s) {
+  switch (a.H) {
+    case 128: return launch_lstm_chain(lstm_adj_chain_kernel<UNC, 4>, a, UNC, smem, 4, s);
+    case 256: return launch_lstm_chain(lstm_adj_chain_kernel<UNC, 8>, a, UNC, smem, 4, s);
+    case 512: return launch_lstm_chain(lstm_adj_chain_kernel<UNC, 16>, a, UNC, smem, 4, s);
+    case 1024: return launch_lstm_chain(lstm_adj_chain_kernel<UNC, 32>, a, UNC, smem, 4, s);
+    default: return false;
+  }
+}
+}  // namespace
+
+bool lstm_chain_fwd_supported(int B, int H) { return chain_ll_enabled() && lstm_pick_unc(B, H, false) != 0; }
+bool lstm_chain_adj_supported(int B, int H) { return chain_ll_enabled() && lstm_pick_unc(B, H, true) != 0; }
+
+bool lstm_chain_fwd_solve(const LstmChainFwdArgs& a, cudaStream_t s) {
+  const int unc = chain_ll_enabled() ? lstm_pick_unc(a.B, a.H, false) : 0;
+  if (unc == 0 || a.nsteps <= 0 || !a.xw || !status_ptr()) return false;
+  const size_t smem = lstm_fwd_smem(unc, a.H);
+  prof_begin(KC_FWD_SERIAL, 2.0 * a.B * 4.0 * a.H * a.H * a.nsteps, s);
+  const bool ok = unc == 8    ? launch_lstm_chain(lstm_fwd_chain_kernel<8>, a, unc, smem, 1, s)
+                  : unc == 16 ? launch_lstm_chain(lstm_fwd_chain_kernel<16>, a, unc, smem, 1, s)
+                              : launch_lstm_chain(lstm_fwd_chain_kernel<32>, a, unc, smem, 1, s);
+  prof_end(s);
+  return ok;
+}
+
+bool lstm_chain_adj_solve(const LstmChainAdjArgs& a, cudaStream_t s) {
+  const int unc = chain_ll_enabled() ? lstm_pick_unc(a.B, a.H, true) : 0;
+  if (unc == 0 || a.nsteps <= 0 || !a.xw || !status_ptr()) return false;
+  const size_t smem = lstm_adj_smem(unc, a.H);
+  prof_begin(KC_ADJ_SERIAL, 2.0 * a.B * 4.0 * a.H * a.H * a.nsteps, s);
+  const bool ok = unc == 8 ? launch_lstm_adj<8>(a, smem, s) : launch_lstm_adj<16>(a, smem, s);
   prof_end(s);
   return ok;
 }

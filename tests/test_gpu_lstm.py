@@ -25,6 +25,12 @@ CASES = [
     dict(T=64, B=5, I=48, H=128, cf=4, levels=3, rf=0, rc=1, flags=0, cell=1, op=2),
     dict(T=256, B=16, I=64, H=256, cf=4, levels=3, rf=1, rc=1, flags=0, cell=1, op=2),
     dict(T=24, B=8, I=32, H=64, cf=4, levels=1, rf=0, rc=0, flags=0, cell=1, op=2),       # serial sweep + exact BPTT
+    # bf16 operands on the persistent chain kernels (H a multiple of 128): the whole serial sweep / the coarsest level in
+    # one launch; two row groups with a partial one; the widest shapes (weights of the adjoint chain held in registers)
+    dict(T=48, B=20, I=32, H=128, cf=4, levels=1, rf=0, rc=0, flags=0, cell=1, op=2),
+    dict(T=64, B=32, I=64, H=512, cf=4, levels=2, rf=0, rc=1, flags=0, cell=1, op=2),
+    dict(T=32, B=32, I=64, H=1024, cf=4, levels=2, rf=0, rc=1, flags=0, cell=1, op=2),
+    dict(T=24, B=16, I=64, H=1024, cf=4, levels=1, rf=0, rc=0, flags=0, cell=0, op=2),    # classic cell, serial sweep
 ]
 
 
