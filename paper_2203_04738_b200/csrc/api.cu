@@ -1197,24 +1197,28 @@ int lstm_adjoint_impl(const mgrit_gru_cfg* cfg, const gru_params* p, const float
   // gradient pass over all fine steps at once: dA_t from the step-output sensitivities (read in place, reversed in time)
   const i64 M = (i64)T * c.B;
   const float* lam_c = aw.U[0] + (size_t)(T - 1) * slot;
-  simt_lstm_form_dA(lam_c, lam_c + bh, -(i64)slot, c.B, aw.p[0], aw.ci[0], aw.cf[0], aw.cg[0], aw.co[0], aw.dA, M, c.H, s);
-  stream_gather_rows(aw.hk, (i64)bh, u + bh, (i64)slot, T, (i64)bh, s);        // hidden states as their own [T, B, H] array
-  if (tf32) {
-    rc = tf32_wgrad(aw.dA, (int)M, 4 * c.H, u0 + bh, c.B, aw.hk, c.H, g->dW_hh, &aw.tf, s);
-    if (!rc) rc = tf32_wgrad(aw.dA, (int)M, 4 * c.H, nullptr, 0, x, c.I, g->dW_ih, &aw.tf, s);
-    if (rc) return rc;
-  } else if (bf) {
-    rc = lstmbf_gradients(&c, aw.dA, x, u0 + bh, aw.hk, g, dx, &aw.bf, s);
+  if (bf) {
+    // bf16 operands: dA is formed as bf16 together with the bias sums, the hidden states are packed straight from u
+    rc = lstmbf_gradients(&c, lam_c, lam_c + bh, -(i64)slot, aw.p[0], aw.ci[0], aw.cf[0], aw.cg[0], aw.co[0], x, u0 + bh, u + bh, (i64)slot, g,
+                          dx, &aw.bf, s);
     if (rc) return rc;
   } else {
-    simt_wgrad(aw.dA, (int)M, 4 * c.H, u0 + bh, c.B, aw.hk, c.H, g->dW_hh, s);
-    simt_wgrad(aw.dA, (int)M, 4 * c.H, nullptr, 0, x, c.I, g->dW_ih, s);
-  }
-  stream_colsum(aw.dA, M, 4 * c.H, g->db_hh, s);
-  cudaMemcpyAsync(g->db_ih, g->db_hh, sizeof(float) * 4 * c.H, cudaMemcpyDeviceToDevice, s);
-  if (dx && !bf) {
-    if (tf32) { rc = tf32_dgrad(aw.dA, (int)M, 4 * c.H, c.I, dx, &aw.tf, s); if (rc) return rc; }
-    else simt_dgrad(aw.dA, (int)M, 4 * c.H, p->W_ih, c.I, dx, s);
+    simt_lstm_form_dA(lam_c, lam_c + bh, -(i64)slot, c.B, aw.p[0], aw.ci[0], aw.cf[0], aw.cg[0], aw.co[0], aw.dA, M, c.H, s);
+    stream_gather_rows(aw.hk, (i64)bh, u + bh, (i64)slot, T, (i64)bh, s);        // hidden states as their own [T, B, H] array
+    if (tf32) {
+      rc = tf32_wgrad(aw.dA, (int)M, 4 * c.H, u0 + bh, c.B, aw.hk, c.H, g->dW_hh, &aw.tf, s);
+      if (!rc) rc = tf32_wgrad(aw.dA, (int)M, 4 * c.H, nullptr, 0, x, c.I, g->dW_ih, &aw.tf, s);
+      if (rc) return rc;
+    } else {
+      simt_wgrad(aw.dA, (int)M, 4 * c.H, u0 + bh, c.B, aw.hk, c.H, g->dW_hh, s);
+      simt_wgrad(aw.dA, (int)M, 4 * c.H, nullptr, 0, x, c.I, g->dW_ih, s);
+    }
+    stream_colsum(aw.dA, M, 4 * c.H, g->db_hh, s);
+    cudaMemcpyAsync(g->db_ih, g->db_hh, sizeof(float) * 4 * c.H, cudaMemcpyDeviceToDevice, s);
+    if (dx) {
+      if (tf32) { rc = tf32_dgrad(aw.dA, (int)M, 4 * c.H, c.I, dx, &aw.tf, s); if (rc) return rc; }
+      else simt_dgrad(aw.dA, (int)M, 4 * c.H, p->W_ih, c.I, dx, s);
+    }
   }
   if (resnorm && hr.L > 1 && c.iters > 0) {
     rc = fetch_resnorm(aw.res_acc, resnorm, c.iters, s);

@@ -1454,16 +1454,34 @@ namespace {
 __global__ void __launch_bounds__(kPT) pack_lstm_adj_kernel(LstmAdjArgs a, bf16* __restrict__ dst) {
   pdl_wait();
   pdl_trigger();
-  const i64 total = (i64)a.M * a.H;
-  for (i64 e = (i64)blockIdx.x * blockDim.x + threadIdx.x; e < total; e += (i64)gridDim.x * blockDim.x) {
-    const i64 m = e / a.H; const int i = (int)(e % a.H);
+  const int H4 = a.H / 4;
+  const i64 total = (i64)a.M * H4;
+  for (i64 e = (i64)blockIdx.x * blockDim.x + threadIdx.x; e < total; e += (i64)gridDim.x * blockDim.x) {     // four units per thread
+    const i64 m = e / H4; const int i = (int)(e % H4) * 4;
     const i64 kk = m / a.B; const int b = (int)(m % a.B);
     const i64 ci = kk * a.coef_ks + (i64)b * a.H + i, li = kk * a.in_ks + (i64)b * a.H + i;
-    const float lh = a.lh[li], dc = a.lc[li] + a.p[ci] * lh;
-    lstm_store_lc(a, e, kk, b, i, a.a[ci] * dc);
-    bf16* d = dst + m * 4 * a.H + i;
-    d[0] = __float2bfloat16(a.ci[ci] * dc); d[a.H] = __float2bfloat16(a.cf[ci] * dc);
-    d[2 * a.H] = __float2bfloat16(a.cg[ci] * dc); d[3 * a.H] = __float2bfloat16(a.co[ci] * lh);
+    const float4 lh = ld4(a.lh + li), lc = ld4(a.lc + li), pp = ld4(a.p + ci), aa = ld4(a.a + ci);
+    const float4 c0 = ld4(a.ci + ci), c1 = ld4(a.cf + ci), c2 = ld4(a.cg + ci), c3 = ld4(a.co + ci);
+    const float4 dc = make_float4(lc.x + pp.x * lh.x, lc.y + pp.y * lh.y, lc.z + pp.z * lh.z, lc.w + pp.w * lh.w);
+    float4 v = make_float4(aa.x * dc.x, aa.y * dc.y, aa.z * dc.z, aa.w * dc.w);
+    if (!a.up.out) {
+      *reinterpret_cast<float4*>(a.lc_out + m * a.H + i) = v;
+    } else {           // cell-part result straight into the level array (see LstmUpdate)
+      float* d = a.up.out + kk * a.up.out_ks + (i64)b * a.H + i;
+      if (a.up.mode == 1) {
+        const float4 o = ld4(d);
+        v = make_float4(o.x - v.x, o.y - v.y, o.z - v.z, o.w - v.w);
+      } else if (a.up.g) {
+        const float4 g = ld4(a.up.g + kk * a.up.g_ks + (i64)b * a.H + i);
+        v = make_float4(v.x + g.x, v.y + g.y, v.z + g.z, v.w + g.w);
+      }
+      *reinterpret_cast<float4*>(d) = v;
+    }
+    uint2* q = reinterpret_cast<uint2*>(dst + m * 4 * a.H + i);
+    q[0] = pack4(make_float4(c0.x * dc.x, c0.y * dc.y, c0.z * dc.z, c0.w * dc.w));
+    q[H4] = pack4(make_float4(c1.x * dc.x, c1.y * dc.y, c1.z * dc.z, c1.w * dc.w));
+    q[2 * H4] = pack4(make_float4(c2.x * dc.x, c2.y * dc.y, c2.z * dc.z, c2.w * dc.w));
+    q[3 * H4] = pack4(make_float4(c3.x * lh.x, c3.y * lh.y, c3.z * lh.z, c3.w * lh.w));
   }
 }
 bool pack_rows(const float* src, i64 ks, int B, int H, i64 M, bf16* dst, cudaStream_t s) {
@@ -1547,7 +1565,7 @@ int lstmbf_linearise(const LstmLinArgs& a, LstmBfWs* w, cudaStream_t s) {
 int lstmbf_adj_step(const LstmAdjArgs& a, LstmBfWs* w, cudaStream_t s) {
   const int K = 4 * a.H;
   ProfScope prof(KC_ADJ_STEP, 2.0 * a.M * (double)K * a.H, s);
-  if (launch_pdl(pack_lstm_adj_kernel, dim3(pgrid((i64)a.M * a.H)), dim3(kPT), 0, s, a, w->Apack) != cudaSuccess) return MGRIT_CUDA_ERROR;
+  if (launch_pdl(pack_lstm_adj_kernel, dim3(pgrid((i64)a.M * (a.H / 4))), dim3(kPT), 0, s, a, w->Apack) != cudaSuccess) return MGRIT_CUDA_ERROR;
   count_launch();
   // few-row steps (coarse levels, the serial sweep): 64-column tiles spread the stream over K over four times the CTAs
   const bool few = ((a.M + BM - 1) / BM) * ((a.H + 255) / 256) * 2 <= kSMs;
@@ -1559,15 +1577,85 @@ int lstmbf_adj_step(const LstmAdjArgs& a, LstmBfWs* w, cudaStream_t s) {
   return ok ? MGRIT_OK : MGRIT_CUDA_ERROR;
 }
 
-int lstmbf_gradients(const mgrit_gru_cfg* c, const float* dA, const float* x, const float* h0, const float* hk, const gru_grads* g,
+namespace {
+// Gradient-pass operand of the LSTM as bf16, row-major: dA[m, :] = [ci*dc | cf*dc | cg*dc | co*Lh] with dc = Lc + p*Lh, plus
+// this block's fp32 column sums of the four products (bias-gradient partials) to part[blockIdx.x][4][H].  Row m = (t, b):
+// sensitivities at lc / lh + t*lam_ts + b*H (lam_ts may be negative: the adjoint keeps its unknowns in reversed time
+// order).  Block = 32 float4 columns (128 units) x 8 rows at a time.
+__global__ void __launch_bounds__(256) lstm_form_dA_rows_kernel(const float* __restrict__ lc, const float* __restrict__ lh, i64 lam_ts, int B,
+                                                                const float* __restrict__ p, const float* __restrict__ ci,
+                                                                const float* __restrict__ cf, const float* __restrict__ cg,
+                                                                const float* __restrict__ co, i64 M, int H, uint2* __restrict__ dA,
+                                                                float* __restrict__ part, int rows_per_block) {
+  __shared__ float red[4][8][128];
+  const int tx = threadIdx.x & 31, ty = threadIdx.x >> 5;
+  const int H4 = H / 4, c4 = blockIdx.y * 32 + tx;
+  const i64 m0 = (i64)blockIdx.x * rows_per_block;
+  float4 s[4];
+#pragma unroll
+  for (int g = 0; g < 4; ++g) s[g] = make_float4(0.f, 0.f, 0.f, 0.f);
+  if (c4 < H4) {
+    for (i64 m = m0 + ty; m < m0 + rows_per_block && m < M; m += 8) {
+      const i64 e = (m * H4 + c4) * 4;
+      const int t = (int)m / B, bb = (int)m - t * B;       // row counts fit 32 bits (checked by the host)
+      const i64 li = (i64)t * lam_ts + ((i64)bb * H4 + c4) * 4;
+      const float4 h = ld4(lh + li), c = ld4(lc + li), pp = ld4(p + e);
+      const float4 k0 = ld4(ci + e), k1 = ld4(cf + e), k2 = ld4(cg + e), k3 = ld4(co + e);
+      const float4 dc = make_float4(c.x + pp.x * h.x, c.y + pp.y * h.y, c.z + pp.z * h.z, c.w + pp.w * h.w);
+      const float4 v[4] = {make_float4(k0.x * dc.x, k0.y * dc.y, k0.z * dc.z, k0.w * dc.w), make_float4(k1.x * dc.x, k1.y * dc.y, k1.z * dc.z, k1.w * dc.w),
+                           make_float4(k2.x * dc.x, k2.y * dc.y, k2.z * dc.z, k2.w * dc.w), make_float4(k3.x * h.x, k3.y * h.y, k3.z * h.z, k3.w * h.w)};
+      const i64 o = m * 4 * H4 + c4;
+#pragma unroll
+      for (int g = 0; g < 4; ++g) {
+        dA[o + g * H4] = pack4(v[g]);
+        s[g].x += v[g].x; s[g].y += v[g].y; s[g].z += v[g].z; s[g].w += v[g].w;
+      }
+    }
+  }
+#pragma unroll
+  for (int g = 0; g < 4; ++g) {
+    red[g][ty][tx * 4] = s[g].x; red[g][ty][tx * 4 + 1] = s[g].y; red[g][ty][tx * 4 + 2] = s[g].z; red[g][ty][tx * 4 + 3] = s[g].w;
+  }
+  __syncthreads();
+  for (int e = threadIdx.x; e < 4 * 128; e += 256) {
+    int g = e / 128, u = e % 128, col = blockIdx.y * 128 + u;
+    if (col >= H) continue;
+    float acc = 0.f;
+#pragma unroll
+    for (int r = 0; r < 8; ++r) acc += red[g][r][u];
+    part[((i64)blockIdx.x * 4 + g) * H + col] = acc;
+  }
+}
+// db_hh = db_ih = the per-block partials summed in block order (the same bits on every run)
+__global__ void __launch_bounds__(kPT) lstm_sum_db_kernel(const float* __restrict__ part, int nblk, int H, float* __restrict__ db_hh,
+                                                          float* __restrict__ db_ih) {
+  for (int e = blockIdx.x * blockDim.x + threadIdx.x; e < 4 * H; e += gridDim.x * blockDim.x) {
+    float acc = 0.f;
+    for (int k = 0; k < nblk; ++k) acc += part[(i64)k * 4 * H + e];
+    db_hh[e] = acc; db_ih[e] = acc;
+  }
+}
+}  // namespace
+
+// All gradients of the LSTM parameters (and dx) from the step-output sensitivities (lc, lh; rows (t, b) at + t*lam_ts + b*H),
+// the level-0 coefficients and the hidden states entering each step (h0, then h_rows + (t-1)*h_ts).
+int lstmbf_gradients(const mgrit_gru_cfg* c, const float* lc, const float* lh, i64 lam_ts, const float* p, const float* ci, const float* cf,
+                     const float* cg, const float* co, const float* x, const float* h0, const float* h_rows, i64 h_ts, const gru_grads* g,
                      float* dx, LstmBfWs* w, cudaStream_t s) {
   const int H = c->H, I = c->I, B = c->B;
   const i64 M = (i64)c->T * B;
   ProfScope prof(KC_WGRAD, 2.0 * M * 4.0 * H * ((double)H + I + (dx ? I : 0)), s);
-  convert(dA, w->dAb, M * 4 * H, s);
+  const int rows_per_block = 256;
+  dim3 grid((unsigned)((M + rows_per_block - 1) / rows_per_block), (H / 4 + 31) / 32);
+  if ((size_t)grid.x * 4 * H * sizeof(float) > w->scratch_bytes) return MGRIT_UNSUPPORTED;
+  // (the bias partials use the split-product scratch before the weight-gradient products need it)
+  lstm_form_dA_rows_kernel<<<grid, 256, 0, s>>>(lc, lh, lam_ts, B, p, ci, cf, cg, co, M, H, reinterpret_cast<uint2*>(w->dAb), w->scratch,
+                                                rows_per_block);
+  lstm_sum_db_kernel<<<pgrid(4 * H), kPT, 0, s>>>(w->scratch, (int)grid.x, H, g->db_hh, g->db_ih);
+  count_launch(2);
   convert(x, w->xb, M * I, s);
   convert(h0, w->hb0, (i64)B * H, s);
-  convert(hk, w->hb0 + (i64)B * H, M * H, s);          // rows (t, b) of h_{t-1} start at hb0
+  if (c->T > 1 && !pack_rows(h_rows, h_ts, B, H, M - B, w->hb0 + (i64)B * H, s)) return MGRIT_CUDA_ERROR;   // rows (t, b) of h_{t-1} start at hb0
   bool ok = wgrad_gemm(w->dAb, 4 * H, w->hb0, H, (int)M, g->dW_hh, w->scratch, w->scratch_bytes, s);
   ok = ok && wgrad_gemm(w->dAb, 4 * H, w->xb, I, (int)M, g->dW_ih, w->scratch, w->scratch_bytes, s);
   if (dx) ok = ok && launch_gemm<256, 0>(KC_WGRAD, w->dAb, 4 * H, w->W_ihT, 4 * H, (int)M, I, 4 * H, 0, I, EpiStore{dx, I, (int)M, I, 0}, s);

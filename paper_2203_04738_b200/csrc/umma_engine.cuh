@@ -76,7 +76,8 @@ int lstmbf_fwd_step(const LstmFwdArgs& a, LstmBfWs* w, cudaStream_t s);
 int lstmbf_linearise(const LstmLinArgs& a, LstmBfWs* w, cudaStream_t s);
 int lstmbf_adj_step(const LstmAdjArgs& a, LstmBfWs* w, cudaStream_t s);
 // dW_hh, dW_ih (and dx) from dA[T*B,4H] fp32; hidden states h0 [B,H] and hk [T,B,H] fp32
-int lstmbf_gradients(const mgrit_gru_cfg* c, const float* dA, const float* x, const float* h0, const float* hk, const gru_grads* g,
+int lstmbf_gradients(const mgrit_gru_cfg* c, const float* lc, const float* lh, i64 lam_ts, const float* p, const float* ci, const float* cf,
+                     const float* cg, const float* co, const float* x, const float* h0, const float* h_rows, i64 h_ts, const gru_grads* g,
                      float* dx, LstmBfWs* w, cudaStream_t s);
 
 int umma_supported(const mgrit_gru_cfg* c);
