@@ -173,6 +173,37 @@ __device__ __forceinline__ void warp_gemm(const bf16* As, const bf16* Ws, int ld
   }
 }
 
+// The same product with the B fragments (the CTA's weight slice, constant for the whole chain) held in registers:
+// w[ks][nt] = the two words a lane feeds to the product of k-step ks and column tile nt.  Same instructions in the same
+// order as warp_gemm, so the results are bit-identical; the shared-memory reads of the weights disappear.
+template <int NT, int KS>
+__device__ __forceinline__ void load_wregs(const bf16* Ws, int ldk, int kbeg, uint32_t (&w)[KS][NT][2]) {
+  const int lane = threadIdx.x & 31, g = lane >> 2, t = lane & 3;
+#pragma unroll
+  for (int ks = 0; ks < KS; ++ks)
+#pragma unroll
+    for (int nt = 0; nt < NT; ++nt) {
+      const bf16* wr = Ws + (nt * 8 + g) * ldk + kbeg + 16 * ks + 2 * t;
+      w[ks][nt][0] = *reinterpret_cast<const uint32_t*>(wr);
+      w[ks][nt][1] = *reinterpret_cast<const uint32_t*>(wr + 8);
+    }
+}
+template <int NT, int KS>
+__device__ __forceinline__ void warp_gemm_regs(const bf16* As, int ldk, int kbeg, const uint32_t (&w)[KS][NT][2], float (*acc)[4]) {
+  const int lane = threadIdx.x & 31, g = lane >> 2, t = lane & 3;
+#pragma unroll
+  for (int ks = 0; ks < KS; ++ks) {
+    const int k0 = kbeg + 16 * ks;
+    uint32_t a[4];
+    a[0] = *reinterpret_cast<const uint32_t*>(As + g * ldk + k0 + 2 * t);
+    a[1] = *reinterpret_cast<const uint32_t*>(As + (g + 8) * ldk + k0 + 2 * t);
+    a[2] = *reinterpret_cast<const uint32_t*>(As + g * ldk + k0 + 2 * t + 8);
+    a[3] = *reinterpret_cast<const uint32_t*>(As + (g + 8) * ldk + k0 + 2 * t + 8);
+#pragma unroll
+    for (int nt = 0; nt < NT; ++nt) mma16816(acc[nt], a, w[ks][nt][0], w[ks][nt][1]);
+  }
+}
+
 // warp partial sums -> red[warp][row][col]   (col < NT*8)
 template <int NT>
 __device__ __forceinline__ void store_partials(float* red, float (*acc)[4]) {
@@ -197,7 +228,8 @@ __device__ __forceinline__ float sum_partials(const float* red, int row, int col
 
 // ------------------------------------------------------------------------------------------------
 // forward chain:  u_j = Phi_gamma(gi_j, u_{j-1}) + g_j ,  j = 1..nsteps
-template <int UNC, bool LL>
+// KS > 0: the weight fragments live in registers (KS = k-steps of 16 per warp = H / 128; see warp_gemm_regs).
+template <int UNC, bool LL, int KS = 0>
 __global__ void __launch_bounds__(kThreads, 1) serial_fwd_kernel(SerialFwdArgs a, int* status) {
   constexpr int NW = 3 * UNC, NT = NW / 8, OPT = (kRows * UNC + kThreads - 1) / kThreads;
   constexpr int kBlockVals = kRows * UNC, kBlockWords = (kBlockVals + kValsPerWord - 1) / kValsPerWord;
@@ -249,11 +281,14 @@ __global__ void __launch_bounds__(kThreads, 1) serial_fwd_kernel(SerialFwdArgs a
   __syncthreads();
 
   const int kw = H / kWarps;
+  uint32_t wreg[KS > 0 ? KS : 1][NT][2];
+  if (KS > 0) load_wregs<NT, (KS > 0 ? KS : 1)>(Ws, ldk, warp * kw, wreg);
   for (int j = 1; j <= a.nsteps; ++j) {
     float acc[NT][4];
 #pragma unroll
     for (int nt = 0; nt < NT; ++nt) acc[nt][0] = acc[nt][1] = acc[nt][2] = acc[nt][3] = 0.f;
-    warp_gemm<NT>(As, Ws, ldk, warp * kw, (warp + 1) * kw, acc);
+    if (KS > 0) warp_gemm_regs<NT, (KS > 0 ? KS : 1)>(As, ldk, warp * kw, wreg, acc);
+    else warp_gemm<NT>(As, Ws, ldk, warp * kw, (warp + 1) * kw, acc);
     store_partials<NT>(red, acc);
     __syncthreads();
     bf16* ub = a.ub + (i64)(j & 1) * BH;
@@ -315,7 +350,7 @@ __global__ void __launch_bounds__(kThreads, 1) serial_fwd_kernel(SerialFwdArgs a
 // ------------------------------------------------------------------------------------------------
 // adjoint chain:  mu_s = a_s * mu_{s-1} + [cr_s|cz_s|cn_s]*mu_{s-1} W_hh + g_s ,  s = 1..nsteps
 // The bf16 operand copy carries dA_{s+1} = [cr|cz|cn]_{s+1} * mu_s, formed by the CTA that produced mu_s.
-template <int UNC, bool LL>
+template <int UNC, bool LL, int KS = 0>     // KS > 0: weight fragments in registers, KS = 3H / 128
 __global__ void __launch_bounds__(kThreads, 1) serial_adj_kernel(SerialAdjArgs a, int* status) {
   constexpr int NT = UNC / 8, OPT = (kRows * UNC + kThreads - 1) / kThreads;
   constexpr int kBlockVals = 3 * kRows * UNC, kBlockWords = (kBlockVals + kValsPerWord - 1) / kValsPerWord;
@@ -367,11 +402,14 @@ __global__ void __launch_bounds__(kThreads, 1) serial_adj_kernel(SerialAdjArgs a
   __syncthreads();
 
   const int kw = K / kWarps;
+  uint32_t wreg[KS > 0 ? KS : 1][NT][2];
+  if (KS > 0) load_wregs<NT, (KS > 0 ? KS : 1)>(Ws, ldk, warp * kw, wreg);
   for (int s = 1; s <= a.nsteps; ++s) {
     float acc[NT][4];
 #pragma unroll
     for (int nt = 0; nt < NT; ++nt) acc[nt][0] = acc[nt][1] = acc[nt][2] = acc[nt][3] = 0.f;
-    warp_gemm<NT>(As, Ws, ldk, warp * kw, (warp + 1) * kw, acc);
+    if (KS > 0) warp_gemm_regs<NT, (KS > 0 ? KS : 1)>(As, ldk, warp * kw, wreg, acc);
+    else warp_gemm<NT>(As, Ws, ldk, warp * kw, (warp + 1) * kw, acc);
     store_partials<NT>(red, acc);
     __syncthreads();
     bf16* dAb = a.dAb + (i64)(s & 1) * 3 * BH;
@@ -993,12 +1031,28 @@ size_t serial_xw_bytes(int B, int H, int gates) {
 bool serial_fwd_supported(int B, int H) { return pick_unc(B, H, false) != 0; }
 bool serial_adj_supported(int B, int H) { return pick_unc(B, H, true) != 0; }
 
+// MGRIT_GRU_CHAIN_WREG=0 in the environment keeps the chains' weight fragments in shared memory (same results).
+static bool chain_wreg_enabled() {
+  static int v = -1;
+  if (v < 0) { const char* e = getenv("MGRIT_GRU_CHAIN_WREG"); v = (e && e[0] == '0') ? 0 : 1; }
+  return v == 1;
+}
+
 bool serial_fwd_solve(const SerialFwdArgs& a, cudaStream_t s) {
   int unc = pick_unc(a.B, a.H, false);
   if (unc == 0 || a.nsteps <= 0 || !status_ptr()) return false;
   size_t smem = fwd_smem(unc, a.H);
   prof_begin(KC_FWD_SERIAL, 2.0 * a.B * 3.0 * a.H * a.H * a.nsteps, s);
   const bool ll = chain_ll_enabled() && a.xw != nullptr;
+  if (ll && chain_wreg_enabled() && (unc == 8 || unc == 16) && (a.H == 512 || a.H == 1024)) {
+    bool okr;
+    if (a.H == 1024) okr = unc == 8 ? launch_coop(serial_fwd_kernel<8, true, 8>, a, unc, smem, true, 1, s)
+                                    : launch_coop(serial_fwd_kernel<16, true, 8>, a, unc, smem, true, 1, s);
+    else okr = unc == 8 ? launch_coop(serial_fwd_kernel<8, true, 4>, a, unc, smem, true, 1, s)
+                        : launch_coop(serial_fwd_kernel<16, true, 4>, a, unc, smem, true, 1, s);
+    prof_end(s);
+    return okr;
+  }
   bool ok = ll ? (unc == 8 ? launch_coop(serial_fwd_kernel<8, true>, a, unc, smem, true, 1, s)
                   : unc == 16 ? launch_coop(serial_fwd_kernel<16, true>, a, unc, smem, true, 1, s)
                               : launch_coop(serial_fwd_kernel<32, true>, a, unc, smem, true, 1, s))
@@ -1015,6 +1069,15 @@ bool serial_adj_solve(const SerialAdjArgs& a, cudaStream_t s) {
   size_t smem = adj_smem(unc, a.H);
   prof_begin(KC_ADJ_SERIAL, 2.0 * a.B * 3.0 * a.H * a.H * a.nsteps, s);
   const bool ll = chain_ll_enabled() && a.xw != nullptr;
+  if (ll && chain_wreg_enabled() && (unc == 8 || unc == 16) && (a.H == 512 || a.H == 1024)) {
+    bool okr;
+    if (a.H == 1024) okr = unc == 8 ? launch_coop(serial_adj_kernel<8, true, 24>, a, unc, smem, true, 3, s)
+                                    : launch_coop(serial_adj_kernel<16, true, 24>, a, unc, smem, true, 3, s);
+    else okr = unc == 8 ? launch_coop(serial_adj_kernel<8, true, 12>, a, unc, smem, true, 3, s)
+                        : launch_coop(serial_adj_kernel<16, true, 12>, a, unc, smem, true, 3, s);
+    prof_end(s);
+    return okr;
+  }
   bool ok = ll ? (unc == 8 ? launch_coop(serial_adj_kernel<8, true>, a, unc, smem, true, 3, s)
                   : unc == 16 ? launch_coop(serial_adj_kernel<16, true>, a, unc, smem, true, 3, s)
                               : launch_coop(serial_adj_kernel<32, true>, a, unc, smem, true, 3, s))

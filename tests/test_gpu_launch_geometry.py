@@ -117,3 +117,45 @@ def test_staged_and_global_load_adjoint_epilogues_agree(tmp_path):
     for k in a.files:
         scale = np.max(np.abs(a[k]))
         assert np.max(np.abs(a[k] - b[k])) <= 1e-6 * scale, k
+
+
+CHILD_CHAIN = r"""
+import sys, numpy as np, torch
+from paper_2203_04738_b200 import binding as B
+from paper_2203_04738_b200.synthetic import Workload, make_inputs
+out = {}
+# (T, B, H, levels): the serial sweep as one chain (8 units per CTA), and a coarsest level of 16 steps at the widest shape
+# (16 units per CTA, two row groups, one of them partial)
+for i, (T, Bz, H, L) in enumerate([(48, 8, 512, 1), (64, 24, 1024, 2)]):
+    w = Workload("chainw", T=T, B=Bz, I=64, H=H, cf=4, levels=L, iters_fwd=2, iters_adj=2, relax_fine=0, relax_coarse=1,
+                 operands=2, classes=8, relu=True, seed=70 + i)
+    d = make_inputs(w)
+    p = {n: torch.from_numpy(d["layers"][0][n]).cuda() for n in ("W_ih", "W_hh", "b_ih", "b_hh")}
+    x, h0 = torch.from_numpy(d["x"]).cuda(), torch.from_numpy(d["h0"]).cuda()
+    cfg = B.make_cfg(T, Bz, w.I, H, cf=4, levels=L, iters=2, operands=B.OPERANDS_BF16)
+    if L == 1:
+        h, gi = B.gru_serial_forward(cfg, p, x, h0)
+    else:
+        h, gi, _ = B.mgrit_gru_forward(cfg, p, x, h0)
+    seed = torch.from_numpy(np.random.default_rng(5 + i).standard_normal(tuple(h.shape)).astype(np.float32)).cuda()
+    r = B.gru_serial_backward(cfg, p, x, h0, gi, h, dh_seed=seed) if L == 1 else B.mgrit_gru_adjoint(cfg, p, x, h0, gi, h, dh_seed=seed)
+    out[f"h{i}"] = h.cpu().numpy(); out[f"dh{i}"] = r.dh.cpu().numpy(); out[f"dW_hh{i}"] = r.dW_hh.cpu().numpy()
+torch.cuda.synchronize()
+assert B.last_device_status() == 0
+np.savez(sys.argv[1], **out)
+"""
+
+
+def test_chain_weights_in_registers_give_the_same_bits(tmp_path):
+    """The persistent chain kernels with their weight fragments in registers issue the same products in the same order
+    as with the weights in shared memory: every output must be bit-identical."""
+    root = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+    outs = []
+    for flag in ("1", "0"):
+        out = str(tmp_path / f"chainw{flag}.npz")
+        env = dict(os.environ, MGRIT_GRU_CHAIN_WREG=flag, PYTHONPATH=root)
+        subprocess.run([sys.executable, "-c", CHILD_CHAIN, out], check=True, env=env, cwd=root, timeout=600)
+        outs.append(np.load(out))
+    a, b = outs
+    for k in a.files:
+        assert np.array_equal(a[k], b[k]), k
