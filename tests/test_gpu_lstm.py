@@ -87,3 +87,51 @@ def test_lstm_tensor_core_modes_reject_unsupported_shapes():
             B.lstm_workspace_bytes(B.make_cfg(64, 8, 64, 32, cf=4, levels=2, operands=op))       # H = 32 is not a multiple of 64
         assert e.value.code == -4
         assert B.lstm_workspace_bytes(B.make_cfg(64, 8, 64, 128, cf=4, levels=2, operands=op))[0] > 0
+
+
+def test_lstm_full_size_sampled_row_and_gradients():
+    """One Implicit-LSTM layer at the shape and in the launch configuration that `bench.py --lstm` times (the default
+    workload's T, B, I, H, levels and cycle counts; bf16 operands; chain kernels on the coarsest level).  Batch rows do
+    not interact in the recurrence, so the oracle solves the full-length problem for one sampled row (states, adjoint
+    sensitivities, dx); the weight gradients sum over ALL (t, b): one time-parallel fp64 pass of the oracle over the
+    full batch, fed the GPU's states and sensitivities, checks exactly the gradient kernels."""
+    from paper_2203_04738_b200 import binding as B
+    from paper_2203_04738_b200.synthetic import WORKLOADS
+    w = WORKLOADS["train"]
+    T, Bn, I, H = w.T, w.B, w.I, w.H
+    rng = np.random.default_rng(811)
+    k = 1.0 / np.sqrt(H)
+    P32 = [rng.uniform(-k, k, s).astype(np.float32) for s in ((4 * H, I), (4 * H, H), (4 * H,), (4 * H,))]
+    x32 = np.maximum(rng.standard_normal((T, Bn, I)), 0).astype(np.float32)
+    u032 = (rng.standard_normal((2, Bn, H)) * 0.3).astype(np.float32)
+    dhT = rng.standard_normal((Bn, H)).astype(np.float32)
+    p = dict(zip(("W_ih", "W_hh", "b_ih", "b_hh"), [to_dev(a) for a in P32]))
+    kwc = dict(cf=w.cf, levels=w.levels, relax_fine=w.relax_fine, relax_coarse=w.relax_coarse, operands=B.OPERANDS_BF16)
+    cfg_f = B.make_cfg(T, Bn, I, H, iters=w.iters_fwd, **kwc)
+    cfg_a = B.make_cfg(T, Bn, I, H, iters=w.iters_adj, **kwc)
+    xd, u0d = to_dev(x32), to_dev(u032)
+    n0 = B.kernel_launches()
+    u, gi, rn = B.mgrit_lstm_forward(cfg_f, p, xd, u0d, want_resnorm=True)
+    du, du0, r, rna = B.mgrit_lstm_adjoint(cfg_a, p, xd, u0d, gi, u, dhT=to_dev(dhT), want_resnorm=True)
+    # the coarsest level ran as chains: far fewer launches than one per dependent step (128 steps, 4 cycles in all)
+    assert B.kernel_launches() - n0 < 400
+    assert B.last_device_status() == 0
+    assert all(a > b for a, b in zip(rn, rn[1:])) and all(a > b for a, b in zip(rna, rna[1:]))
+    P = [a.astype(np.float64) for a in P32]
+    kw = dict(cf=w.cf, levels=w.levels, cell=1, relax_fine=w.relax_fine, relax_coarse=w.relax_coarse)
+    rows = [11]
+    xr, u0r = x32[:, rows].astype(np.float64), u032[:, rows].astype(np.float64)
+    uref, _ = O.lstm_mgrit_forward(*P, xr, u0r, iters=w.iters_fwd, **kw)
+    ug = u[:, :, rows].cpu().numpy().astype(np.float64)
+    assert rel_inf(ug, uref) < 2e-2
+    seed = np.zeros_like(ug)
+    seed[-1, 1] = dhT[rows]
+    lam, lam0, g, _ = O.lstm_mgrit_adjoint(*P, xr, u0r, ug, seed, iters=w.iters_adj, **kw)
+    assert rel_inf(du[:, :, rows].cpu().numpy(), lam) < 2e-2
+    assert max_abs(du0[:, rows].cpu().numpy(), lam0) / np.max(np.abs(lam)) < 2e-2
+    assert rel_inf(r.dx[:, rows].cpu().numpy(), g["dx"]) < 2e-2
+    del g, lam, uref
+    gw = O.lstm_weight_gradients(*P, x32.astype(np.float64), u032.astype(np.float64), u.cpu().numpy().astype(np.float64),
+                                 du.cpu().numpy().astype(np.float64), want_dx=False)
+    for key in ("dW_ih", "dW_hh", "db_ih", "db_hh"):
+        assert rel_inf(getattr(r, key).cpu().numpy(), gw[key]) < 2e-2, key
