@@ -89,8 +89,8 @@ struct LstmChainAdjArgs {
   const __nv_bfloat16* WT;       // [H][4H] = W_hh^T
   uint4* xw; size_t xw_bytes;    // exchange words, serial_xw_bytes(B, H, 4)
 };
-bool lstm_chain_fwd_supported(int B, int H);
-bool lstm_chain_adj_supported(int B, int H);
+// false: shape not supported (forward: H % 128 != 0; adjoint: H not in {128, 256, 512, 1024}; too many CTAs for one wave)
+// or the cooperative launch failed: the caller then advances step by step
 bool lstm_chain_fwd_solve(const LstmChainFwdArgs& a, cudaStream_t s);
 bool lstm_chain_adj_solve(const LstmChainAdjArgs& a, cudaStream_t s);
 int serial_device_status();

@@ -1135,9 +1135,6 @@ bool launch_lstm_adj(const LstmChainAdjArgs& a, size_t smem, cudaStream_t s) {
 }
 }  // namespace
 
-bool lstm_chain_fwd_supported(int B, int H) { return chain_ll_enabled() && lstm_pick_unc(B, H, false) != 0; }
-bool lstm_chain_adj_supported(int B, int H) { return chain_ll_enabled() && lstm_pick_unc(B, H, true) != 0; }
-
 bool lstm_chain_fwd_solve(const LstmChainFwdArgs& a, cudaStream_t s) {
   const int unc = chain_ll_enabled() ? lstm_pick_unc(a.B, a.H, false) : 0;
   if (unc == 0 || a.nsteps <= 0 || !a.xw || !status_ptr()) return false;
