@@ -75,7 +75,10 @@ umma_adj_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
   constexpr int kTileRows = PAIR ? 2 * BM : BM;
   const int m_tiles = (p.M + kTileRows - 1) / kTileRows, n_tiles = (H + BNa - 1) / BNa, tiles = m_tiles * n_tiles;
   const int k_blocks = (K + BK - 1) / BK;
-  auto row_tile = [&](int t) { return PAIR ? 2 * (t / n_tiles) + (int)rank : t / n_tiles; };
+  // Row tiles from the last to the first: the packing kernel writes the operand rows in ascending order and most of the
+  // 100 MB of a 16384-row step have left L2 by the time it ends, except the rows written last (and this kernel's
+  // results of the first rows are the newest when the next packing kernel starts there).
+  auto row_tile = [&](int t) { const int q = m_tiles - 1 - t / n_tiles; return PAIR ? 2 * q + (int)rank : q; };
 
   if (threadIdx.x == 0) {
     abort_flag = 0;

@@ -80,7 +80,7 @@ bool make_map(CUtensorMap* m, const float* base, uint64_t inner, uint64_t rows, 
 // ET = bf16, or float for operands that hold tf32 values.  splits > 1 (split-aware epilogues only) cuts the reduction.
 template <int BN, int NG, class Epi, class ET>
 bool launch_gemm(int kc, const ET* A, i64 lda, const ET* Bm, i64 ldb, int M, int N, int K, int gate_rows, int b_rows, Epi epi,
-                 cudaStream_t s, int splits = 1) {
+                 cudaStream_t s, int splits = 1, bool desc = false) {
   using C = Cfg<BN, NG>;
   constexpr bool TF32 = sizeof(ET) == 4;
   if (M <= 0 || N <= 0) return true;
@@ -94,7 +94,7 @@ bool launch_gemm(int kc, const ET* A, i64 lda, const ET* Bm, i64 ldb, int M, int
   if (!make_map(&tb, Bm, (uint64_t)K, (uint64_t)b_rows, (uint64_t)ldb, NG > 0 ? BN / NG : BN)) return false;
   const int k_blocks = (K + (TF32 ? BK / 2 : BK) - 1) / (TF32 ? BK / 2 : BK);
   if (splits < 1 || !EpiSplitAware<Epi>::value) splits = 1;
-  GemmShape sh{M, N, K, gate_rows, splits, (k_blocks + splits - 1) / splits};
+  GemmShape sh{M, N, K, gate_rows, splits, (k_blocks + splits - 1) / splits, desc ? 1 : 0};
   int m_tiles = (M + BM - 1) / BM, n_tiles = (N + C::kNPerTile - 1) / C::kNPerTile;
   int tiles = m_tiles * n_tiles * splits;
   int grid = tiles < kSMs ? tiles : kSMs;
@@ -113,7 +113,8 @@ static bool gemm_pair_enabled(int M, int N) {
   return v == 1 && (i64)((M + BM - 1) / BM) * ((N + 255) / 256) > kSMs;
 }
 template <class Epi>
-bool launch_gemm_pair(int kc, const bf16* A, i64 lda, const bf16* Bm, i64 ldb, int M, int N, int K, int b_rows, Epi epi, cudaStream_t s) {
+bool launch_gemm_pair(int kc, const bf16* A, i64 lda, const bf16* Bm, i64 ldb, int M, int N, int K, int b_rows, Epi epi, cudaStream_t s,
+                      bool desc = false) {
   if (M <= 0 || N <= 0) return true;
   int* const status = status_ptr();
   if (!status) return false;
@@ -123,7 +124,7 @@ bool launch_gemm_pair(int kc, const bf16* A, i64 lda, const bf16* Bm, i64 ldb, i
   CUtensorMap ta, tb;
   if (!make_map(&ta, A, (uint64_t)K, (uint64_t)M, (uint64_t)lda, BM)) return false;
   if (!make_map(&tb, Bm, (uint64_t)K, (uint64_t)b_rows, (uint64_t)ldb, pairk::BN / 2)) return false;
-  GemmShape sh{M, N, K, 0};
+  GemmShape sh{M, N, K, 0, 1, 0, desc ? 1 : 0};
   int tiles = ((M + 2 * BM - 1) / (2 * BM)) * ((N + pairk::BN - 1) / pairk::BN);
   int grid = 2 * (tiles < kSMs / 2 ? tiles : kSMs / 2);
   ProfScope prof_(kc, 2.0 * M * (double)N * K, s);
@@ -1571,9 +1572,11 @@ int lstmbf_adj_step(const LstmAdjArgs& a, LstmBfWs* w, cudaStream_t s) {
   const bool few = ((a.M + BM - 1) / BM) * ((a.H + 255) / 256) * 2 <= kSMs;
   const bool ok = !a.up.out ? launch_gemm<256, 0>(KC_ADJ_STEP, w->Apack, K, w->W_hhT, K, a.M, a.H, K, 0, a.H, EpiStore{a.lh_out, a.H, a.M, a.H, 0}, s)
                   : few     ? launch_gemm<64, 0>(KC_ADJ_STEP, w->Apack, K, w->W_hhT, K, a.M, a.H, K, 0, a.H, EpiUpdate<64>{a.up, a.M, a.H, a.B}, s)
+                  // (row tiles in descending order: the operand rows packed last are still in L2)
                   : gemm_pair_enabled(a.M, a.H)
-                            ? launch_gemm_pair(KC_ADJ_STEP, w->Apack, K, w->W_hhT, K, a.M, a.H, K, a.H, EpiUpdate<256>{a.up, a.M, a.H, a.B}, s)
-                            : launch_gemm<256, 0>(KC_ADJ_STEP, w->Apack, K, w->W_hhT, K, a.M, a.H, K, 0, a.H, EpiUpdate<256>{a.up, a.M, a.H, a.B}, s);
+                            ? launch_gemm_pair(KC_ADJ_STEP, w->Apack, K, w->W_hhT, K, a.M, a.H, K, a.H, EpiUpdate<256>{a.up, a.M, a.H, a.B}, s, true)
+                            : launch_gemm<256, 0>(KC_ADJ_STEP, w->Apack, K, w->W_hhT, K, a.M, a.H, K, 0, a.H, EpiUpdate<256>{a.up, a.M, a.H, a.B}, s,
+                                                  1, true);
   return ok ? MGRIT_OK : MGRIT_CUDA_ERROR;
 }
 

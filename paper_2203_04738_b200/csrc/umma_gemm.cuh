@@ -157,6 +157,8 @@ struct GemmShape {
   int splits;           // split products (MN-major, or an epilogue with kSplitAware): the reduction is cut into `splits`
   int kb_per_split;     // ranges of kb_per_split k-blocks, each (tile, range) is one work item and the epilogue is told
                         // which range it finishes; 0 or 1 = the whole reduction in one item
+  int desc;             // 1: row tiles from the last to the first (a producer kernel wrote the A rows in ascending order:
+                        // the rows written last are the ones still in L2)
 };
 
 // An epilogue that can finish one range of a split reduction declares `static constexpr bool kSplitAware = true`
@@ -243,7 +245,7 @@ umma_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
       int stage = 0; uint32_t phase = 0;
       bool ok = true;
       for (int t = blockIdx.x; t < tiles && ok; t += gridDim.x) {
-        const int mt = (t % mn_tiles) / n_tiles, nt = t % n_tiles;
+        const int mq = (t % mn_tiles) / n_tiles, mt = sh.desc ? m_tiles - 1 - mq : mq, nt = t % n_tiles;
         for (int kb = kb_begin(t), kbe = kb_end(t); kb < kbe; ++kb) {
           if (!mbar_wait(empty_bar(stage), phase ^ 1u, abortp, status, 1)) { ok = false; break; }
           const uint32_t a_dst = tiles_base + stage * C::kStageBytes;
@@ -307,7 +309,7 @@ umma_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
     const int half = (warp - 2) >> 2;   // which half of the tile's columns this warp handles
     int it = 0;
     for (int t = blockIdx.x; t < tiles; t += gridDim.x, ++it) {
-      const int mt = (t % mn_tiles) / n_tiles, nt = t % n_tiles;
+      const int mq = (t % mn_tiles) / n_tiles, mt = sh.desc ? m_tiles - 1 - mq : mq, nt = t % n_tiles;
       const int as = it & 1;
       const uint32_t aphase = (uint32_t)(it >> 1) & 1u;
       if (!mbar_wait(tfull_bar(as), aphase, abortp, status, 4)) break;

@@ -109,7 +109,7 @@ umma_gemm_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_cons
     if (lane == 0) {
       int stage = 0; uint32_t phase = 0; bool ok = true;
       for (int t = cta; t < tiles && ok; t += ncta) {
-        const int mt = 2 * (t / n_tiles) + (int)rank, nt = t % n_tiles;
+        const int mq = t / n_tiles, mt = 2 * (sh.desc ? m_tiles - 1 - mq : mq) + (int)rank, nt = t % n_tiles;
         for (int kb = 0; kb < k_blocks; ++kb) {
           if (!mbar_wait(empty_bar(stage), phase ^ 1u, abortp, status, 21)) { ok = false; break; }
           const uint32_t a_dst = tiles_base + stage * kStageBytes, b_dst = a_dst + kABytes;
@@ -154,7 +154,7 @@ umma_gemm_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_cons
     const int half = (warp - 2) >> 2;
     int it = 0;
     for (int t = cta; t < tiles; t += ncta, ++it) {
-      const int mt = 2 * (t / n_tiles) + (int)rank, nt = t % n_tiles;
+      const int mq = t / n_tiles, mt = 2 * (sh.desc ? m_tiles - 1 - mq : mq) + (int)rank, nt = t % n_tiles;
       const int as = it & 1;
       const uint32_t aphase = (uint32_t)(it >> 1) & 1u;
       if (!mbar_wait(tfull_bar(as), aphase, abortp, status, 24)) break;
