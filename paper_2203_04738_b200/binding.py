@@ -23,7 +23,7 @@ OK = 0
 CELL_CLASSIC, CELL_IMPLICIT = 0, 1
 RELAX_F, RELAX_FCF, RELAX_FCFCF = 0, 1, 2
 OPERANDS_FP32, OPERANDS_TF32, OPERANDS_BF16, OPERANDS_TF32_1PASS = 0, 1, 2, 3
-FLAG_SKIP_DUPLICATE_FRELAX, FLAG_F_CYCLE, FLAG_RAGGED_T, FLAG_GI_CARRIES_COPIES = 1, 2, 4, 8
+FLAG_SKIP_DUPLICATE_FRELAX, FLAG_F_CYCLE, FLAG_RAGGED_T, FLAG_GI_CARRIES_COPIES, FLAG_GI_F32_UNUSED = 1, 2, 4, 8, 16
 
 
 class Cfg(ctypes.Structure):

@@ -322,6 +322,7 @@ struct Cycle {
 struct FwdCycle : Cycle {
   const gru_params* p; const float* gi; UmmaFwdWs* um; FwdWs* fw;
   const __nv_bfloat16* gib = nullptr;   // bf16 copy of gi: what every kernel of the solve reads when the state copies exist
+  bool gi_f32 = true;                   // false: the fp32 projection was not written (MGRIT_FLAG_GI_F32_UNUSED); gib is set
 
   bool chain(int l) override {
     if (c->operands != MGRIT_OPERANDS_BF16) {     // fp32 and tf32 modes: the chain in FFMA arithmetic
@@ -341,6 +342,7 @@ struct FwdCycle : Cycle {
     a.gi = gi + (st - 1) * (i64)BH * 3; a.gi_step = st * (i64)BH * 3;
     // (the plain serial sweep has no other level to stay consistent with: it uses the fp32 projection as it is)
     a.gi_as_bf16 = (gib && hr.L > 1) ? 1 : 0;
+    if (!gi_f32) { a.gi_b = gib + (st - 1) * (i64)BH * 3; a.gi = nullptr; }
     a.g = G[l]; a.W = um->W_hh; a.b_hh = p->b_hh; a.gamma = hr.gamma[l]; a.cell = c->cell; a.bar = fw->chain_bar;
     a.xw = fw->chain_xw; a.xw_bytes = fw->chain_xw_bytes;
     return serial_fwd_solve(a, s);
@@ -502,9 +504,11 @@ int forward_impl(const mgrit_gru_cfg* cfg_in, bool serial, const gru_params* p, 
     fw.um.gib = t.gib;
   }
   if (!gi_bf16_enabled()) fw.um.gib = nullptr;
+  // the caller does not read the fp32 projection and every kernel of this solve reads its bf16 copy: do not write it
+  const bool gi_f32 = !((c.flags & MGRIT_FLAG_GI_F32_UNUSED) && carries_copies(&c, serial) && fw.um.gib);
 
   if (c.operands == MGRIT_OPERANDS_BF16) {
-    rc = umma_prepare_fwd(&c, p, x, gi, &fw.um, s);
+    rc = umma_prepare_fwd(&c, p, x, gi_f32 ? gi : nullptr, &fw.um, s);
     if (rc) return rc;
   } else if (is_tf32(&c)) {
     rc = tf32_prepare_fwd(&c, p, x, gi, &fw.tf, s);
@@ -526,6 +530,7 @@ int forward_impl(const mgrit_gru_cfg* cfg_in, bool serial, const gru_params* p, 
   cy.p = p; cy.gi = gi; cy.um = &fw.um; cy.fw = &fw;
   cy.Ub = shadows ? fw.Ub : nullptr;
   cy.gib = shadows ? fw.um.gib : nullptr;
+  cy.gi_f32 = gi_f32;
   rc = cy.solve();
   if (rc) return rc;
   cudaMemcpyAsync(h, fw.U[0] + BH, sizeof(float) * (size_t)c.T * BH, cudaMemcpyDeviceToDevice, s);

@@ -10,6 +10,7 @@ struct SerialFwdArgs {
   float* u;                      // level state; slots 1..nsteps are written
   __nv_bfloat16* ub;             // [2][B][H] scratch: bf16 copy of the newest state
   const float* gi; i64 gi_step;  // projection rows of step 1 (+ (j-1)*gi_step for step j), row b at + b*3H
+  const __nv_bfloat16* gi_b;     // the projection as bf16 (same indexing as gi), or nullptr; when given, gi is not read
   int gi_as_bf16;                // 1: round every projection value to bf16 after loading it, so that the chain sees the same
                                  // values as the relaxation kernels of the other levels, which stage the projection's bf16 copy
   const float* g;                // [nsteps+1][B][H] additive term, or nullptr

@@ -226,6 +226,19 @@ __device__ __forceinline__ float sum_partials(const float* red, int row, int col
   return s;
 }
 
+// A projection value as the chain's prefetch loads it and as the cell uses it.  Nothing may depend on the load before the
+// exchange (a dependent instruction would wait for DRAM there), so a bf16 source is kept as its raw 16 bits in the
+// register and widened only at the use; an fp32 source is rounded to bf16 at the use when the solve's other levels read
+// the bf16 copy.
+__device__ __forceinline__ float ld_gi(const SerialFwdArgs& a, i64 idx) {
+  if (a.gi_b) return __uint_as_float((uint32_t)reinterpret_cast<const unsigned short*>(a.gi_b)[idx]);
+  return a.gi[idx];
+}
+__device__ __forceinline__ float use_gi(const SerialFwdArgs& a, float raw) {
+  if (a.gi_b) return __uint_as_float(__float_as_uint(raw) << 16);
+  return a.gi_as_bf16 ? bf16_round(raw) : raw;
+}
+
 // ------------------------------------------------------------------------------------------------
 // forward chain:  u_j = Phi_gamma(gi_j, u_{j-1}) + g_j ,  j = 1..nsteps
 // KS > 0: the weight fragments live in registers (KS = k-steps of 16 per warp = H / 128; see warp_gemm_regs).
@@ -275,7 +288,7 @@ __global__ void __launch_bounds__(kThreads, 1) serial_fwd_kernel(SerialFwdArgs a
     hp[o] = v ? __ldcg(a.u + (i64)(row0 + r) * H + u0 + i) : 0.f;
     br[o] = a.b_hh[u0 + i]; bz[o] = a.b_hh[H + u0 + i]; bn[o] = a.b_hh[2 * H + u0 + i];
     const i64 go = (i64)(row0 + r) * 3 * H + u0 + i;
-    pgr[o] = v ? a.gi[go] : 0.f; pgz[o] = v ? a.gi[go + H] : 0.f; pgn[o] = v ? a.gi[go + 2 * H] : 0.f;
+    pgr[o] = v ? ld_gi(a, go) : 0.f; pgz[o] = v ? ld_gi(a, go + H) : 0.f; pgn[o] = v ? ld_gi(a, go + 2 * H) : 0.f;
     pg[o] = (v && a.g) ? a.g[BH + (i64)(row0 + r) * H + u0 + i] : 0.f;
   }
   __syncthreads();
@@ -300,8 +313,7 @@ __global__ void __launch_bounds__(kThreads, 1) serial_fwd_kernel(SerialFwdArgs a
         float ghr = sum_partials<NW>(red, r, i) + br[o];
         float ghz = sum_partials<NW>(red, r, UNC + i) + bz[o];
         float ghn = sum_partials<NW>(red, r, 2 * UNC + i) + bn[o];
-        const float gir = a.gi_as_bf16 ? bf16_round(pgr[o]) : pgr[o], giz = a.gi_as_bf16 ? bf16_round(pgz[o]) : pgz[o];
-        const float gin = a.gi_as_bf16 ? bf16_round(pgn[o]) : pgn[o];
+        const float gir = use_gi(a, pgr[o]), giz = use_gi(a, pgz[o]), gin = use_gi(a, pgn[o]);
         val = cell_forward<true>(gir, giz, gin, ghr, ghz, ghn, hp[o], a.gamma, a.cell) + pg[o];
         hp[o] = val;
         i64 off = (i64)(row0 + r) * H + u0 + i;
@@ -323,7 +335,7 @@ __global__ void __launch_bounds__(kThreads, 1) serial_fwd_kernel(SerialFwdArgs a
         const i64 go = (i64)j * a.gi_step + (i64)(row0 + r) * 3 * H + u0 + i;
         // (loaded now, rounded where they are used: an instruction that depends on these loads here would wait for them
         // in front of the exchange)
-        pgr[o] = a.gi[go]; pgz[o] = a.gi[go + H]; pgn[o] = a.gi[go + 2 * H];
+        pgr[o] = ld_gi(a, go); pgz[o] = ld_gi(a, go + H); pgn[o] = ld_gi(a, go + 2 * H);
         if (a.g) pg[o] = a.g[(i64)(j + 1) * BH + (i64)(row0 + r) * H + u0 + i];
       }
     }

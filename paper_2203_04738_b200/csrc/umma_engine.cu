@@ -363,7 +363,7 @@ __device__ __forceinline__ void st4(float* p, float a, float b, float c, float d
 }
 __device__ __forceinline__ float f4get(const float4& v, int e) { return e == 0 ? v.x : (e == 1 ? v.y : (e == 2 ? v.z : v.w)); }
 
-struct EpiBias {  // out[m, n] = acc + bias[n]      (input projection); outb: optional bf16 copy of the same values
+struct EpiBias {  // out[m, n] = acc + bias[n]      (input projection); outb: optional bf16 copy of the same values; out may be null then
   float* out; i64 ld; const float* bias; int M, N; bf16* outb;
   __device__ void operator()(uint32_t taddr, int row, int n0, int half) const {
     const bool valid = row < M;
@@ -379,8 +379,10 @@ struct EpiBias {  // out[m, n] = acc + bias[n]      (input projection); outb: op
           float4 b = ldg4(bias + n0 + c0 + i);
           v[i] += b.x; v[i + 1] += b.y; v[i + 2] += b.z; v[i + 3] += b.w;
         }
-        st8(o + c0, v);
-        st8(o + c0 + 8, v + 8);
+        if (out) {
+          st8(o + c0, v);
+          st8(o + c0 + 8, v + 8);
+        }
         if (outb) {
           const uint2 p0 = pack4(make_float4(v[0], v[1], v[2], v[3])), p1 = pack4(make_float4(v[4], v[5], v[6], v[7]));
           const uint2 p2 = pack4(make_float4(v[8], v[9], v[10], v[11])), p3 = pack4(make_float4(v[12], v[13], v[14], v[15]));

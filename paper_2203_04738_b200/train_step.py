@@ -30,7 +30,7 @@ def make_cfgs(w: Workload, T: int, Bsz: int, serial: bool = False, flags: int = 
     for l in range(w.layers):
         I = w.I if l == 0 else w.H
         kw = dict(cf=w.cf, levels=1 if serial else w.levels, cell=w.cell, relax_fine=w.relax_fine,
-                  relax_coarse=w.relax_coarse, operands=w.operands, flags=flags | B.FLAG_GI_CARRIES_COPIES)
+                  relax_coarse=w.relax_coarse, operands=w.operands, flags=flags | B.FLAG_GI_CARRIES_COPIES | B.FLAG_GI_F32_UNUSED)      # (nothing here reads the fp32 projection)
         fw.append(B.make_cfg(T, Bsz, I, w.H, iters=w.iters_fwd, **kw))
         ad.append(B.make_cfg(T, Bsz, I, w.H, iters=w.iters_adj, **kw))
     return fw, ad

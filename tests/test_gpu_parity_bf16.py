@@ -267,6 +267,35 @@ def test_copies_carried_behind_gi_change_nothing_but_rounding(B):
     assert B.last_device_status() == 0
 
 
+def test_unwritten_fp32_projection_changes_no_bit(B):
+    # FLAG_GI_F32_UNUSED: the forward call writes only the bf16 copy of the projection (the chain of the coarsest level
+    # then reads that copy instead of rounding the fp32 values itself) and leaves the fp32 part of the buffer alone --
+    # every output of the forward and of the adjoint call must keep its bits, and the poison must still be there.
+    # Where the copies do not exist (B does not divide 128) the flag is ignored and the projection is written.
+    for Bsz in (32, 8, 24):
+        w = Workload("nof32", T=256, B=Bsz, I=64, H=256, cf=4, levels=3, iters_fwd=2, iters_adj=2, relax_fine=0, relax_coarse=1,
+                     operands=2, classes=8, relu=True, seed=17)
+        d = make_inputs(w)
+        p, x, h0 = upload(d)
+        carry = _cfg(B, w, 2, flags=B.FLAG_GI_CARRIES_COPIES)
+        skip = _cfg(B, w, 2, flags=B.FLAG_GI_CARRIES_COPIES | B.FLAG_GI_F32_UNUSED)
+        b1, b2 = B.alloc_gi(carry, x.device), B.alloc_gi(skip, x.device)
+        assert b1.numel() == b2.numel()
+        b2.fill_(float("nan"))
+        h, _, rn = B.mgrit_gru_forward(carry, p, x, h0, gi=b1, want_resnorm=True)
+        h2, _, rn2 = B.mgrit_gru_forward(skip, p, x, h0, gi=b2, want_resnorm=True)
+        assert torch.equal(h, h2) and rn == rn2
+        written = not bool(torch.isnan(B.gi_view(skip, b2)).all())
+        assert written == (Bsz == 24)
+        if written:
+            assert torch.equal(B.gi_view(skip, b2), B.gi_view(carry, b1))
+        r = B.mgrit_gru_adjoint(carry, p, x, h0, b1, h, dhT=h[-1].contiguous())
+        r2 = B.mgrit_gru_adjoint(skip, p, x, h0, b2, h2, dhT=h2[-1].contiguous())
+        for k in ("dh", "dh0", "dx", "dW_ih", "dW_hh", "db_ih", "db_hh"):
+            assert torch.equal(getattr(r, k), getattr(r2, k)), k
+    assert B.last_device_status() == 0
+
+
 def test_long_sweeps_repeat_bit_for_bit(B):
     # Sixteen dependent steps per launch (cf = 8, FCF on both non-coarsest levels), single-CTA and pair geometry, tiles of a
     # later step waiting on counters of the earlier one: a missed dependency would show as a run that differs.
