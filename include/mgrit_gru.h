@@ -77,7 +77,11 @@ enum {
    * projection -- every kernel of the solve and of the adjoint reads that copy anyway -- and leaves the T*B*3H floats
    * at the start of the buffer untouched (0.8 GB of stores per layer of the default workload).  All outputs are
    * bit-identical with and without it.  Set it in the cfg of BOTH calls; ignored where the copies do not exist. */
-  MGRIT_FLAG_GI_F32_UNUSED = 16
+  MGRIT_FLAG_GI_F32_UNUSED = 16,
+  /* mgrit_gru_forward / gru_serial_forward only: h points to T + 1 slots [T+1,B,H] instead of T.  The call writes h_0
+   * to slot 0 and h_t to slot t: the level-0 unknowns of the solve live in the caller's array itself and the copy of
+   * T*B*H floats that otherwise ends the call is saved (same bits).  The adjoint calls take h + B*H as their h. */
+  MGRIT_FLAG_H_LEADS_WITH_H0 = 32
 };
 
 /* Problem and cycle description (Algorithm "MGProp", remark "Beyond Two-Level", Section

@@ -24,6 +24,7 @@ CELL_CLASSIC, CELL_IMPLICIT = 0, 1
 RELAX_F, RELAX_FCF, RELAX_FCFCF = 0, 1, 2
 OPERANDS_FP32, OPERANDS_TF32, OPERANDS_BF16, OPERANDS_TF32_1PASS = 0, 1, 2, 3
 FLAG_SKIP_DUPLICATE_FRELAX, FLAG_F_CYCLE, FLAG_RAGGED_T, FLAG_GI_CARRIES_COPIES, FLAG_GI_F32_UNUSED = 1, 2, 4, 8, 16
+FLAG_H_LEADS_WITH_H0 = 32
 
 
 class Cfg(ctypes.Structure):
@@ -150,28 +151,38 @@ def gru_input_projection(cfg, p, x, gi=None, ws=None):
     return gi
 
 
+def _h_array(cfg, h, dev):
+    """The state array of a forward call and the number of leading slots that are not part of h[T,B,H]."""
+    lead = 1 if cfg.flags & FLAG_H_LEADS_WITH_H0 else 0
+    if h is None:
+        h = torch.empty(cfg.T + lead, cfg.B, cfg.H, device=dev)
+    assert h.shape[0] == cfg.T + lead and h.is_contiguous()
+    return h, lead
+
+
 def mgrit_gru_forward(cfg, p, x, h0, want_resnorm=False, gi=None, h=None, ws=None):
-    """-> (h[T,B,H], gi[T,B,3H], resnorm list or None)"""
+    """-> (h[T,B,H], gi[T,B,3H], resnorm list or None).  With FLAG_H_LEADS_WITH_H0 the array passed as `h` (or allocated
+    here) has T + 1 slots, slot 0 receives h_0, and the returned h is the view of its slots 1..T."""
     dev = x.device
     gi = alloc_gi(cfg, dev) if gi is None else gi       # (a flat buffer when the copies flag is set, else viewed as [T,B,3H])
     if gi.dim() == 1 and not (cfg.flags & FLAG_GI_CARRIES_COPIES):
         gi = gi_view(cfg, gi)
-    h = torch.empty(cfg.T, cfg.B, cfg.H, device=dev) if h is None else h
+    h, lead = _h_array(cfg, h, dev)
     ws = _ws(workspace_bytes(cfg)[0], ws, dev)
     rn = (ctypes.c_float * max(cfg.iters, 1))() if want_resnorm else None
     _check(lib.mgrit_gru_forward(ctypes.byref(cfg), ctypes.byref(_params(p)), _f32(x), _f32(h0), _f32(gi), _f32(h), rn,
                                  _ptr(ws), ws.numel(), _stream()))
-    return h, gi, (list(rn)[:cfg.iters] if want_resnorm else None)
+    return h[lead:], gi, (list(rn)[:cfg.iters] if want_resnorm else None)
 
 
 def gru_serial_forward(cfg, p, x, h0, gi=None, h=None, ws=None):
     dev = x.device
     gi = torch.empty(cfg.T, cfg.B, 3 * cfg.H, device=dev) if gi is None else gi
-    h = torch.empty(cfg.T, cfg.B, cfg.H, device=dev) if h is None else h
+    h, lead = _h_array(cfg, h, dev)
     ws = _ws(workspace_bytes(cfg)[0], ws, dev)
     _check(lib.gru_serial_forward(ctypes.byref(cfg), ctypes.byref(_params(p)), _f32(x), _f32(h0), _f32(gi), _f32(h),
                                   _ptr(ws), ws.numel(), _stream()))
-    return h, gi
+    return h[lead:], gi
 
 
 @dataclass

@@ -497,6 +497,9 @@ int forward_impl(const mgrit_gru_cfg* cfg_in, bool serial, const gru_params* p, 
   plan_fwd(&c, hr, w, &fw);
   if (!w.fits()) return MGRIT_WORKSPACE_TOO_SMALL;
   size_t BH = (size_t)c.B * c.H;
+  // the caller's array has a leading slot for h_0: the level-0 unknowns live there and nothing is copied at the end
+  const bool h_in_place = (c.flags & MGRIT_FLAG_H_LEADS_WITH_H0) != 0;
+  if (h_in_place) fw.U[0] = h;
   if (carries_copies(&c, serial)) {      // make the copies where the adjoint call will look for them
     GiTail t = gi_tail(&c, gi);
     fw.um.xb = t.xb;
@@ -533,7 +536,7 @@ int forward_impl(const mgrit_gru_cfg* cfg_in, bool serial, const gru_params* p, 
   cy.gi_f32 = gi_f32;
   rc = cy.solve();
   if (rc) return rc;
-  cudaMemcpyAsync(h, fw.U[0] + BH, sizeof(float) * (size_t)c.T * BH, cudaMemcpyDeviceToDevice, s);
+  if (!h_in_place) cudaMemcpyAsync(h, fw.U[0] + BH, sizeof(float) * (size_t)c.T * BH, cudaMemcpyDeviceToDevice, s);
   if (resnorm && hr.L > 1 && c.iters > 0) {
     rc = fetch_resnorm(fw.res_acc, resnorm, c.iters, s);
     if (rc) return rc;

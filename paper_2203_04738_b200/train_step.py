@@ -20,9 +20,10 @@ class StepBuffers:
     ws_adj: torch.Tensor
     ws_head: torch.Tensor
     gi: list
-    h: list
+    h: list            # h[l]: [T,B,H] view of slots 1..T of h_full[l]
     adj: list
     serial: bool = False
+    h_full: list = None    # h_full[l]: [T+1,B,H], slot 0 = h_0 (written by the forward call: MGRIT_FLAG_H_LEADS_WITH_H0)
 
 
 def make_cfgs(w: Workload, T: int, Bsz: int, serial: bool = False, flags: int = 0):
@@ -31,7 +32,8 @@ def make_cfgs(w: Workload, T: int, Bsz: int, serial: bool = False, flags: int = 
         I = w.I if l == 0 else w.H
         kw = dict(cf=w.cf, levels=1 if serial else w.levels, cell=w.cell, relax_fine=w.relax_fine,
                   relax_coarse=w.relax_coarse, operands=w.operands, flags=flags | B.FLAG_GI_CARRIES_COPIES | B.FLAG_GI_F32_UNUSED)      # (nothing here reads the fp32 projection)
-        fw.append(B.make_cfg(T, Bsz, I, w.H, iters=w.iters_fwd, **kw))
+        # the forward calls write the level-0 unknowns straight into the buffers' state arrays (one leading slot for h_0)
+        fw.append(B.make_cfg(T, Bsz, I, w.H, iters=w.iters_fwd, **dict(kw, flags=kw["flags"] | B.FLAG_H_LEADS_WITH_H0)))
         ad.append(B.make_cfg(T, Bsz, I, w.H, iters=w.iters_adj, **kw))
     return fw, ad
 
@@ -46,9 +48,10 @@ def alloc_buffers(w: Workload, T: int, Bsz: int, device, serial: bool = False, f
         # dh (dL/dh_t for every t) is not an input of anything in a training step: only written when asked for
         adj.append(B.AdjointResult(dh=mk(T, Bsz, w.H) if want_dh else None, dh0=mk(Bsz, w.H), dx=mk(T, Bsz, c.I) if l > 0 else None,
                                    dW_ih=mk(3 * w.H, c.I), dW_hh=mk(3 * w.H, w.H), db_ih=mk(3 * w.H), db_hh=mk(3 * w.H)))
+    h_full = [mk(T + 1, Bsz, w.H) for _ in fw]
     return StepBuffers(fw, ad, torch.empty(nf, dtype=torch.uint8, device=device), torch.empty(na, dtype=torch.uint8, device=device),
                        torch.empty(B.lib.xent_head_workspace_bytes(Bsz, w.classes), dtype=torch.uint8, device=device),
-                       [B.alloc_gi(c, device) for c in fw], [mk(T, Bsz, w.H) for _ in fw], adj, serial)
+                       [B.alloc_gi(c, device) for c in fw], [t[1:] for t in h_full], adj, serial, h_full)
 
 
 class HostInputPipeline:
@@ -113,7 +116,7 @@ def forward_pass(layers, x, h0, buf: StepBuffers):
     inp = x
     for l, p in enumerate(layers):
         fn = B.gru_serial_forward if buf.serial else B.mgrit_gru_forward
-        fn(buf.cfgs_fwd[l], p, inp, h0, gi=buf.gi[l], h=buf.h[l], ws=buf.ws_fwd)
+        fn(buf.cfgs_fwd[l], p, inp, h0, gi=buf.gi[l], h=buf.h_full[l], ws=buf.ws_fwd)
         inp = buf.h[l]
     return inp
 

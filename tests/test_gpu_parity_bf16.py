@@ -296,6 +296,29 @@ def test_unwritten_fp32_projection_changes_no_bit(B):
     assert B.last_device_status() == 0
 
 
+def test_state_array_with_a_leading_slot_keeps_every_bit(B):
+    # FLAG_H_LEADS_WITH_H0: the level-0 unknowns live in the caller's [T+1,B,H] array (slot 0 = h_0) and the final copy is
+    # saved; h must keep its bits, for the multigrid solve and the serial sweep, on the tensor-core and the FFMA engine.
+    for operands in (B.OPERANDS_BF16, B.OPERANDS_FP32):
+        w = Workload("lead", T=128, B=16, I=64, H=128, cf=4, levels=3, iters_fwd=2, iters_adj=2, relax_fine=0, relax_coarse=1,
+                     operands=operands, classes=8, relu=True, seed=19)
+        d = make_inputs(w)
+        d["h0"] = (np.random.default_rng(3).standard_normal(d["h0"].shape) * 0.3).astype(np.float32)
+        p, x, h0 = upload(d)
+        kw = dict(cf=w.cf, levels=w.levels, iters=2, relax_fine=w.relax_fine, relax_coarse=w.relax_coarse, operands=operands)
+        plain = B.make_cfg(w.T, w.B, w.I, w.H, **kw)
+        lead = B.make_cfg(w.T, w.B, w.I, w.H, flags=B.FLAG_H_LEADS_WITH_H0, **kw)
+        h, _, _ = B.mgrit_gru_forward(plain, p, x, h0)
+        full = torch.full((w.T + 1, w.B, w.H), float("nan"), device="cuda")
+        h2, _, _ = B.mgrit_gru_forward(lead, p, x, h0, h=full)
+        assert h2.data_ptr() == full[1:].data_ptr() and torch.equal(h2, h) and torch.equal(full[0], h0)
+        hs, _ = B.gru_serial_forward(plain, p, x, h0)
+        full.fill_(float("nan"))
+        hs2, _ = B.gru_serial_forward(lead, p, x, h0, h=full)
+        assert torch.equal(hs2, hs) and torch.equal(full[0], h0)
+    assert B.last_device_status() == 0
+
+
 def test_long_sweeps_repeat_bit_for_bit(B):
     # Sixteen dependent steps per launch (cf = 8, FCF on both non-coarsest levels), single-CTA and pair geometry, tiles of a
     # later step waiting on counters of the earlier one: a missed dependency would show as a run that differs.
