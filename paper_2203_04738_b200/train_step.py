@@ -160,18 +160,19 @@ class GraphedTrainingStep:
     tensors passed here must stay alive and keep their addresses; new data is copied INTO them.  ``launches`` is
     the number of library kernels one replay runs."""
 
-    def __init__(self, w: Workload, layers, W_c, b_c, x, h0, labels, buf: StepBuffers, **kw):
+    def __init__(self, w: Workload, layers, W_c, b_c, x, h0, labels, buf: StepBuffers, step_fn=None, **kw):
         args = (w, layers, W_c, b_c, x, h0, labels, buf)
+        fn = (lambda: training_step(*args, **kw)) if step_fn is None else step_fn     # step_fn: any fixed sequence of library calls
         side = torch.cuda.Stream()
         side.wait_stream(torch.cuda.current_stream())
         with torch.cuda.stream(side):               # first use of every kernel outside the capture (attribute set-up)
-            training_step(*args, **kw)
+            fn()
         torch.cuda.current_stream().wait_stream(side)
         torch.cuda.synchronize()
         n0 = B.kernel_launches()
         self.graph = torch.cuda.CUDAGraph()
         with torch.cuda.graph(self.graph):
-            self.loss = training_step(*args, **kw)
+            self.loss = fn()
         self.launches = B.kernel_launches() - n0
         self._keep = args
 
