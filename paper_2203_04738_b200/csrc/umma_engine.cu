@@ -863,7 +863,9 @@ int umma_linearise(const LinArgs& a, UmmaAdjWs* w, cudaStream_t s) {
     ca.B = a.B; ca.H = a.H; ca.b_hh = a.b_hh; ca.gamma = a.gamma; ca.cell = a.cell;
     ca.a = a.a; ca.cr = a.crb; ca.cz = a.czb; ca.cn = a.cnb; ca.cnp = a.cnpb;
     int done = 0;
-    if (a.t0 == 0) {   // step 1 starts from h_0 (its own array)
+    // step 1 starts from h_0: a launch of its own, unless the caller keeps h_0 in the slot in front of h (the layout
+    // of MGRIT_FLAG_H_LEADS_WITH_H0) -- then rows (t - 1) of h are valid for t = 0 as well
+    if (a.t0 == 0 && a.h0 + BH != a.h) {
       if (!launch_lin(KC_LINEARISE, w->hb0, 0, gib0 ? (const void*)gib0 : (const void*)gi0, gib0 != nullptr, 0, a.h0, 0, 1, w->W_hh, ca, s))
         return MGRIT_CUDA_ERROR;
       done = 1;

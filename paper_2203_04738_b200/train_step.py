@@ -131,7 +131,8 @@ def training_step(w: Workload, layers, W_c, b_c, x, h0, labels, buf: StepBuffers
     for l in range(len(layers) - 1, -1, -1):
         inp = x if l == 0 else buf.h[l - 1]
         fn = B.gru_serial_backward if buf.serial else B.mgrit_gru_adjoint
-        fn(buf.cfgs_adj[l], layers[l], inp, h0, buf.gi[l], buf.h[l], dh_seed=seed, dhT=dhT if seed is None else None,
+        # (h_0 as the forward call left it in slot 0 of the state array: contiguous with h, one linearisation launch per level)
+        fn(buf.cfgs_adj[l], layers[l], inp, buf.h_full[l][0], buf.gi[l], buf.h[l], dh_seed=seed, dhT=dhT if seed is None else None,
            want_dx=l > 0, ws=buf.ws_adj, out=buf.adj[l])
         seed = buf.adj[l].dx
     if update and adam is not None:

@@ -308,10 +308,23 @@ def test_state_array_with_a_leading_slot_keeps_every_bit(B):
         kw = dict(cf=w.cf, levels=w.levels, iters=2, relax_fine=w.relax_fine, relax_coarse=w.relax_coarse, operands=operands)
         plain = B.make_cfg(w.T, w.B, w.I, w.H, **kw)
         lead = B.make_cfg(w.T, w.B, w.I, w.H, flags=B.FLAG_H_LEADS_WITH_H0, **kw)
-        h, _, _ = B.mgrit_gru_forward(plain, p, x, h0)
+        h, gi, _ = B.mgrit_gru_forward(plain, p, x, h0)
         full = torch.full((w.T + 1, w.B, w.H), float("nan"), device="cuda")
         h2, _, _ = B.mgrit_gru_forward(lead, p, x, h0, h=full)
         assert h2.data_ptr() == full[1:].data_ptr() and torch.equal(h2, h) and torch.equal(full[0], h0)
+        # the adjoint given h_0 in the slot in front of h (one linearisation launch per level instead of two) changes no bit
+        seed = to_dev((np.random.default_rng(4).standard_normal((w.T, w.B, w.H)) * 0.1).astype(np.float32))
+        pad = torch.zeros(3, w.B, w.H, device="cuda")      # an h_0 that certainly does not sit in front of h
+        pad[1].copy_(h0)
+        n0 = B.kernel_launches()
+        r = B.mgrit_gru_adjoint(plain, p, x, pad[1], gi, h, dh_seed=seed)
+        n1 = B.kernel_launches()
+        r2 = B.mgrit_gru_adjoint(plain, p, x, full[0], gi, h2, dh_seed=seed)
+        n2 = B.kernel_launches()
+        for k in ("dh", "dh0", "dx", "dW_ih", "dW_hh", "db_ih", "db_hh"):
+            assert torch.equal(getattr(r, k), getattr(r2, k)), k
+        if operands == B.OPERANDS_BF16:
+            assert n2 - n1 < n1 - n0
         hs, _ = B.gru_serial_forward(plain, p, x, h0)
         full.fill_(float("nan"))
         hs2, _ = B.gru_serial_forward(lead, p, x, h0, h=full)
