@@ -79,8 +79,9 @@ bool make_map(CUtensorMap* m, const float* base, uint64_t inner, uint64_t rows, 
 
 // ET = bf16, or float for operands that hold tf32 values.  splits > 1 (split-aware epilogues only) cuts the reduction.
 template <int BN, int NG, class Epi, class ET>
+// a_ext / a_from / a_add: the A operand skips a column block of its array (see GemmShape); a_ext = columns of the array.
 bool launch_gemm(int kc, const ET* A, i64 lda, const ET* Bm, i64 ldb, int M, int N, int K, int gate_rows, int b_rows, Epi epi,
-                 cudaStream_t s, int splits = 1, bool desc = false) {
+                 cudaStream_t s, int splits = 1, bool desc = false, int a_ext = 0, int a_from = 0, int a_add = 0) {
   using C = Cfg<BN, NG>;
   constexpr bool TF32 = sizeof(ET) == 4;
   if (M <= 0 || N <= 0) return true;
@@ -90,11 +91,11 @@ bool launch_gemm(int kc, const ET* A, i64 lda, const ET* Bm, i64 ldb, int M, int
   auto kern = umma_gemm_kernel<BN, NG, Epi, false, TF32>;
   if (!set_smem_once(kern, C::kSmemBytes, attr_set)) return false;
   CUtensorMap ta, tb;
-  if (!make_map(&ta, A, (uint64_t)K, (uint64_t)M, (uint64_t)lda, BM)) return false;
+  if (!make_map(&ta, A, (uint64_t)(a_ext > 0 ? a_ext : K), (uint64_t)M, (uint64_t)lda, BM)) return false;
   if (!make_map(&tb, Bm, (uint64_t)K, (uint64_t)b_rows, (uint64_t)ldb, NG > 0 ? BN / NG : BN)) return false;
   const int k_blocks = (K + (TF32 ? BK / 2 : BK) - 1) / (TF32 ? BK / 2 : BK);
   if (splits < 1 || !EpiSplitAware<Epi>::value) splits = 1;
-  GemmShape sh{M, N, K, gate_rows, splits, (k_blocks + splits - 1) / splits, desc ? 1 : 0};
+  GemmShape sh{M, N, K, gate_rows, splits, (k_blocks + splits - 1) / splits, desc ? 1 : 0, a_from, a_add};
   int m_tiles = (M + BM - 1) / BM, n_tiles = (N + C::kNPerTile - 1) / C::kNPerTile;
   int tiles = m_tiles * n_tiles * splits;
   int grid = tiles < kSMs ? tiles : kSMs;
@@ -114,7 +115,7 @@ static bool gemm_pair_enabled(int M, int N) {
 }
 template <class Epi>
 bool launch_gemm_pair(int kc, const bf16* A, i64 lda, const bf16* Bm, i64 ldb, int M, int N, int K, int b_rows, Epi epi, cudaStream_t s,
-                      bool desc = false) {
+                      bool desc = false, int a_ext = 0, int a_from = 0, int a_add = 0) {
   if (M <= 0 || N <= 0) return true;
   int* const status = status_ptr();
   if (!status) return false;
@@ -122,9 +123,9 @@ bool launch_gemm_pair(int kc, const bf16* A, i64 lda, const bf16* Bm, i64 ldb, i
   auto kern = umma_gemm_pair_kernel<Epi>;
   if (!set_smem_once(kern, pairk::kSmemBytes, attr_set)) return false;
   CUtensorMap ta, tb;
-  if (!make_map(&ta, A, (uint64_t)K, (uint64_t)M, (uint64_t)lda, BM)) return false;
+  if (!make_map(&ta, A, (uint64_t)(a_ext > 0 ? a_ext : K), (uint64_t)M, (uint64_t)lda, BM)) return false;
   if (!make_map(&tb, Bm, (uint64_t)K, (uint64_t)b_rows, (uint64_t)ldb, pairk::BN / 2)) return false;
-  GemmShape sh{M, N, K, 0, 1, 0, desc ? 1 : 0};
+  GemmShape sh{M, N, K, 0, 1, 0, desc ? 1 : 0, a_from, a_add};
   int tiles = ((M + 2 * BM - 1) / (2 * BM)) * ((N + pairk::BN - 1) / pairk::BN);
   int grid = 2 * (tiles < kSMs / 2 ? tiles : kSMs / 2);
   ProfScope prof_(kc, 2.0 * M * (double)N * K, s);
@@ -139,7 +140,7 @@ bool launch_gemm_pair(int kc, const bf16* A, i64 lda, const bf16* Bm, i64 ldb, i
 // weight-gradient reductions dW = dA^T h, which therefore need no transposed copies.
 template <class Epi>
 bool launch_gemm_mn(int kc, const bf16* A, i64 lda, int Mdim, const bf16* Bm, i64 ldb, int Ndim, int K, int splits, Epi epi,
-                    cudaStream_t s) {
+                    cudaStream_t s, int a_ext = 0, int a_from = 0, int a_add = 0) {
   using C = Cfg<256, 0>;
   if (Mdim <= 0 || Ndim <= 0) return true;
   int* const status = status_ptr();
@@ -148,11 +149,11 @@ bool launch_gemm_mn(int kc, const bf16* A, i64 lda, int Mdim, const bf16* Bm, i6
   auto kern = umma_gemm_kernel<256, 0, Epi, true>;
   if (!set_smem_once(kern, C::kSmemBytes, attr_set)) return false;
   CUtensorMap ta, tb;
-  if (!make_map(&ta, A, (uint64_t)Mdim, (uint64_t)K, (uint64_t)lda, 64)) return false;
+  if (!make_map(&ta, A, (uint64_t)(a_ext > 0 ? a_ext : Mdim), (uint64_t)K, (uint64_t)lda, 64)) return false;
   if (!make_map(&tb, Bm, (uint64_t)Ndim, (uint64_t)K, (uint64_t)ldb, 64)) return false;
   const int k_blocks = (K + BK - 1) / BK;
   if (splits < 1) splits = 1;
-  GemmShape sh{Mdim, Ndim, K, 0, splits, (k_blocks + splits - 1) / splits};
+  GemmShape sh{Mdim, Ndim, K, 0, splits, (k_blocks + splits - 1) / splits, 0, a_from, a_add};
   int tiles = ((Mdim + BM - 1) / BM) * ((Ndim + 255) / 256) * splits;
   int grid = tiles < kSMs ? tiles : kSMs;
   ProfScope prof_(kc, 2.0 * Mdim * (double)Ndim * K, s);
@@ -653,8 +654,8 @@ __global__ void __launch_bounds__(1024) transpose_kernel(const float* __restrict
 // reversed time order).  Block = 32 float4 columns (128 units) x 8 rows at a time.
 __global__ void __launch_bounds__(256) form_dA_rows_kernel(const float* __restrict__ lam, i64 lam_ts, int B, const bf16* __restrict__ cr,
                                                            const bf16* __restrict__ cz, const bf16* __restrict__ cn,
-                                                           const bf16* __restrict__ cnp, i64 M, int H, uint2* __restrict__ dAh,
-                                                           uint2* __restrict__ dAi, float* __restrict__ part, int rows_per_block) {
+                                                           const bf16* __restrict__ cnp, i64 M, int H, uint2* __restrict__ dA4,
+                                                           float* __restrict__ part, int rows_per_block) {
   __shared__ float red[4][8][128];
   const int tx = threadIdx.x & 31, ty = threadIdx.x >> 5;
   const int H4 = H / 4, c4 = blockIdx.y * 32 + tx;
@@ -671,12 +672,9 @@ __global__ void __launch_bounds__(256) form_dA_rows_kernel(const float* __restri
       float4 n = unpack4(reinterpret_cast<const uint2*>(cn)[e]), q = unpack4(reinterpret_cast<const uint2*>(cnp)[e]);
       float4 v[4] = {make_float4(r.x * l.x, r.y * l.y, r.z * l.z, r.w * l.w), make_float4(z.x * l.x, z.y * l.y, z.z * l.z, z.w * l.w),
                      make_float4(n.x * l.x, n.y * l.y, n.z * l.z, n.w * l.w), make_float4(q.x * l.x, q.y * l.y, q.z * l.z, q.w * l.w)};
-      i64 o = m * 3 * H4 + c4;
-      uint2 pr = pack4(v[0]), pz = pack4(v[1]);
-      dAh[o] = pr; dAi[o] = pr;
-      dAh[o + H4] = pz; dAi[o + H4] = pz;
-      dAh[o + 2 * H4] = pack4(v[2]);
-      dAi[o + 2 * H4] = pack4(v[3]);
+      i64 o = m * 4 * H4 + c4;
+#pragma unroll
+      for (int g = 0; g < 4; ++g) dA4[o + g * H4] = pack4(v[g]);
 #pragma unroll
       for (int g = 0; g < 4; ++g) { s[g].x += v[g].x; s[g].y += v[g].y; s[g].z += v[g].z; s[g].w += v[g].w; }
     }
@@ -762,8 +760,7 @@ void umma_plan_adj(const mgrit_gru_cfg* c, const int* N, int L, char* base, size
   if (TB * H > apack) apack = TB * H;     // the linearisation packs all T*B rows of a level at once
   o->Apack = take<bf16>(base, off, apack);
   o->apack_elems = apack;
-  o->dAh = take<bf16>(base, off, 3 * H * TB);
-  o->dAi = take<bf16>(base, off, 3 * H * TB);
+  o->dA4 = take<bf16>(base, off, 4 * H * TB);
   o->xb = take<bf16>(base, off, I * TB);
   o->hb0 = take<bf16>(base, off, (size_t)c->B * H + TB * H);   // [h_0; h] contiguous: rows (t, b) of h_{t-1} start at hb0
   o->hb = o->hb0 ? o->hb0 + (size_t)c->B * H : nullptr;
@@ -1005,12 +1002,16 @@ static int pick_splits(int Mdim, int Ndim, int K, size_t scratch_bytes) {
 }
 
 template <class OutT>
+// (a_ld > 0: dA is a column selection of a wider array with a_ld columns -- the first a_from columns and, when a_add != 0,
+// the columns behind a gap of a_add)
 static bool wgrad_gemm(const bf16* dA, int H3, const bf16* R, int cols, int K, OutT* out, float* scratch, size_t scratch_bytes,
-                       cudaStream_t s) {
+                       cudaStream_t s, int a_ld = 0, int a_from = 0, int a_add = 0) {
   const int splits = (((i64)H3 * cols) % 4 == 0) ? pick_splits(H3, cols, K, scratch_bytes) : 1;
-  if (splits == 1) return launch_gemm_mn(KC_WGRAD, dA, H3, H3, R, cols, cols, K, 1, EpiStore{out, cols, H3, cols, 0}, s);
+  const i64 lda = a_ld > 0 ? a_ld : H3;
+  if (splits == 1)
+    return launch_gemm_mn(KC_WGRAD, dA, lda, H3, R, cols, cols, K, 1, EpiStore{out, cols, H3, cols, 0}, s, a_ld, a_from, a_add);
   const i64 n = (i64)H3 * cols;
-  if (!launch_gemm_mn(KC_WGRAD, dA, H3, H3, R, cols, cols, K, splits, EpiStore{scratch, cols, H3, cols, n}, s)) return false;
+  if (!launch_gemm_mn(KC_WGRAD, dA, lda, H3, R, cols, cols, K, splits, EpiStore{scratch, cols, H3, cols, n}, s, a_ld, a_from, a_add)) return false;
   sum_splits_kernel<<<pgrid(n / 4), kPT, 0, s>>>(reinterpret_cast<const float4*>(scratch), n / 4, splits, reinterpret_cast<float4*>(out));
   count_launch();
   return true;
@@ -1025,7 +1026,9 @@ int umma_gradients(const mgrit_gru_cfg* c, const gru_params* p, const float* x, 
   // one timing record for the whole pass: operand forming, bias sums, the three products and their split sums
   ProfScope prof(KC_WGRAD, 2.0 * M * 3.0 * H * ((double)H + I + (dx ? I : 0)), s);
   // operands of the three gradient GEMMs, all row-major (the reduction index t,b is the row index)
-  bf16* dAh = w->dAh; bf16* dAi = w->dAi;        // [M, 3H] each
+  // dA4 [M, 4H] = [cr | cz | cn | cn'] * lambda: the operand of the recurrent-weight gradient is its first three column
+  // blocks, that of the input-weight gradient and of dx its blocks 0, 1 and 3 (the products skip block 2)
+  bf16* dA4 = w->dA4;
   const int rows_per_block = 256;
   // (the step operand buffer is free during the gradient pass: scratch for the bias partials, then for the split
   // partial products of the weight-gradient GEMMs; M >= 8 makes nblk*16H <= 2MH bytes)
@@ -1033,20 +1036,21 @@ int umma_gradients(const mgrit_gru_cfg* c, const gru_params* p, const float* x, 
   const size_t scratch_bytes = w->apack_elems * sizeof(bf16);
   dim3 grid((unsigned)((M + rows_per_block - 1) / rows_per_block), (H / 4 + 31) / 32);
   if ((size_t)grid.x * 4 * H * sizeof(float) > scratch_bytes) return MGRIT_UNSUPPORTED;
-  form_dA_rows_kernel<<<grid, 256, 0, s>>>(lam, lam_ts, B, cr, cz, cn, cnp, M, H, reinterpret_cast<uint2*>(dAh),
-                                           reinterpret_cast<uint2*>(dAi), scratch, rows_per_block);
+  form_dA_rows_kernel<<<grid, 256, 0, s>>>(lam, lam_ts, B, cr, cz, cn, cnp, M, H, reinterpret_cast<uint2*>(dA4), scratch, rows_per_block);
   sum_db_kernel<<<pgrid(4 * H), kPT, 0, s>>>(scratch, (int)grid.x, H, g->db_hh, g->db_ih);
   count_launch(2);
   if (!have_xb) convert(x, w->xb, M * I, s);     // x as bf16 [M, I]; h_{t-1} as bf16 = [h_0; h] without its last slot (w->hb0)
   bool ok = true;
   // dW_hh[3H, H] = dA_h^T h_prev ;  dW_ih[3H, I] = dA_i^T x    (K = T*B, MN-major operands)
-  ok = ok && wgrad_gemm(dAh, 3 * H, w->hb0, H, (int)M, g->dW_hh, scratch, scratch_bytes, s);
-  ok = ok && wgrad_gemm(dAi, 3 * H, w->xb, I, (int)M, g->dW_ih, scratch, scratch_bytes, s);
+  ok = ok && wgrad_gemm(dA4, 3 * H, w->hb0, H, (int)M, g->dW_hh, scratch, scratch_bytes, s, 4 * H, 3 * H, 0);
+  ok = ok && wgrad_gemm(dA4, 3 * H, w->xb, I, (int)M, g->dW_ih, scratch, scratch_bytes, s, 4 * H, 2 * H, H);
   // dx[T*B, I] = dA_i W_ih   (K = 3H, K-major operands)
   if (dx)
     ok = ok && (gemm_pair_enabled((int)M, I)
-                    ? launch_gemm_pair(KC_WGRAD, dAi, 3 * H, w->W_ihT, 3 * H, (int)M, I, 3 * H, I, EpiStore{dx, I, (int)M, I, 0}, s)
-                    : launch_gemm<256, 0>(KC_WGRAD, dAi, 3 * H, w->W_ihT, 3 * H, (int)M, I, 3 * H, 0, I, EpiStore{dx, I, (int)M, I, 0}, s));
+                    ? launch_gemm_pair(KC_WGRAD, dA4, 4 * H, w->W_ihT, 3 * H, (int)M, I, 3 * H, I, EpiStore{dx, I, (int)M, I, 0}, s, false, 4 * H,
+                                       2 * H, H)
+                    : launch_gemm<256, 0>(KC_WGRAD, dA4, 4 * H, w->W_ihT, 3 * H, (int)M, I, 3 * H, 0, I, EpiStore{dx, I, (int)M, I, 0}, s, 1,
+                                          false, 4 * H, 2 * H, H));
   return ok ? MGRIT_OK : MGRIT_CUDA_ERROR;
 }
 

@@ -19,8 +19,7 @@ struct UmmaAdjWs {
   __nv_bfloat16* W_ihT;   // [I,3H]   (dx = dA_i W_ih)
   __nv_bfloat16* Apack;   // [maxM,3H]
   size_t apack_elems;     // its size in elements
-  __nv_bfloat16* dAh;     // [T*B,3H]  gradient-pass operand [cr|cz|cn]*lambda
-  __nv_bfloat16* dAi;     // [T*B,3H]  gradient-pass operand [cr|cz|cn']*lambda
+  __nv_bfloat16* dA4;     // [T*B,4H]  gradient-pass operands [cr|cz|cn|cn']*lambda (recurrent weights: blocks 0-2; input side: 0, 1, 3)
   __nv_bfloat16* xb;      // [T*B,I]   bf16 copy of the layer input
   __nv_bfloat16* hb0;     // [(T+1)*B,H] bf16 copy of [h_0; h]: row (t,b) is h_{t-1} of step t
   __nv_bfloat16* hb;      // = hb0 + B*H: the given states

@@ -159,6 +159,8 @@ struct GemmShape {
                         // which range it finishes; 0 or 1 = the whole reduction in one item
   int desc;             // 1: row tiles from the last to the first (a producer kernel wrote the A rows in ascending order:
                         // the rows written last are the ones still in L2)
+  int a_from, a_add;    // a_add != 0: the A operand skips a column block of its array -- coordinates along the array's
+                        // contiguous dimension (K for K-major, M for MN-major operands) at or beyond a_from move up by a_add
 };
 
 // An epilogue that can finish one range of a split reduction declares `static constexpr bool kSplitAware = true`
@@ -253,11 +255,15 @@ umma_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
           mbar_expect_tx(full_bar(stage), C::kStageBytes);
           if (MNMAJ) {
 #pragma unroll
-            for (int i = 0; i < BM / 64; ++i) tma_load_2d(a_dst + i * 8192, &tmA, full_bar(stage), mt * BM + i * 64, kb * BK);
+            for (int i = 0; i < BM / 64; ++i) {
+              int xa = mt * BM + i * 64;
+              if (sh.a_add && xa >= sh.a_from) xa += sh.a_add;
+              tma_load_2d(a_dst + i * 8192, &tmA, full_bar(stage), xa, kb * BK);
+            }
 #pragma unroll
             for (int i = 0; i < BN / 64; ++i) tma_load_2d(b_dst + i * 8192, &tmB, full_bar(stage), nt * BN + i * 64, kb * BK);
           } else {
-          tma_load_2d(a_dst, &tmA, full_bar(stage), kb * kBK, mt * BM);
+          tma_load_2d(a_dst, &tmA, full_bar(stage), (sh.a_add && kb * kBK >= sh.a_from) ? kb * kBK + sh.a_add : kb * kBK, mt * BM);
           if (NG > 0) {
 #pragma unroll
             for (int g = 0; g < NG; ++g)

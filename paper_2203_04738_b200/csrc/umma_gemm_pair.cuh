@@ -115,7 +115,7 @@ umma_gemm_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_cons
           const uint32_t a_dst = tiles_base + stage * kStageBytes, b_dst = a_dst + kABytes;
           const uint32_t fullL = mapa_shared(full_bar(stage), 0);
           if (rank == 0) mbar_expect_tx(full_bar(stage), 2 * kStageBytes);
-          tma_load_2d_pair(a_dst, &tmA, fullL, kb * BK, mt * BM);
+          tma_load_2d_pair(a_dst, &tmA, fullL, (sh.a_add && kb * BK >= sh.a_from) ? kb * BK + sh.a_add : kb * BK, mt * BM);
           tma_load_2d_pair(b_dst, &tmB, fullL, kb * BK, nt * BN + (int)rank * (BN / 2));
           if (++stage == kStages) { stage = 0; phase ^= 1u; }
         }
