@@ -993,6 +993,7 @@ struct LstmFwdWs {
 struct LstmAdjWs {
   float* U[kMaxLevels]; float* G[kMaxLevels]; double* res_acc;
   float *a[kMaxLevels], *p[kMaxLevels], *ci[kMaxLevels], *cf[kMaxLevels], *cg[kMaxLevels], *co[kMaxLevels];
+  __nv_bfloat16 *cib[kMaxLevels], *cfb[kMaxLevels], *cgb[kMaxLevels], *cob[kMaxLevels];    // bf16 operands: the gate coefficients as bf16 instead
   float *tmpC, *tmpH, *hk, *dA; size_t maxM; Tf32Ws tf; LstmBfWs bf;
   uint4* chain_xw; size_t chain_xw_bytes;
 };
@@ -1022,8 +1023,15 @@ void plan_lstm_adj(const mgrit_gru_cfg* c, const Hier& hr, Ws& w, LstmAdjWs* o) 
     o->U[l] = w.take<float>((size_t)(hr.N[l] + 1) * slot);
     o->G[l] = w.take<float>((size_t)(hr.N[l] + 1) * slot);
     const size_t n = (size_t)hr.N[l] * bh;
-    o->a[l] = w.take<float>(n); o->p[l] = w.take<float>(n); o->ci[l] = w.take<float>(n);
-    o->cf[l] = w.take<float>(n); o->cg[l] = w.take<float>(n); o->co[l] = w.take<float>(n);
+    o->a[l] = w.take<float>(n); o->p[l] = w.take<float>(n);
+    if (c->operands == MGRIT_OPERANDS_BF16) {
+      o->ci[l] = o->cf[l] = o->cg[l] = o->co[l] = nullptr;
+      o->cib[l] = w.take<__nv_bfloat16>(n); o->cfb[l] = w.take<__nv_bfloat16>(n);
+      o->cgb[l] = w.take<__nv_bfloat16>(n); o->cob[l] = w.take<__nv_bfloat16>(n);
+    } else {
+      o->ci[l] = w.take<float>(n); o->cf[l] = w.take<float>(n); o->cg[l] = w.take<float>(n); o->co[l] = w.take<float>(n);
+      o->cib[l] = o->cfb[l] = o->cgb[l] = o->cob[l] = nullptr;
+    }
   }
   o->res_acc = w.take<double>((size_t)(c->iters > 0 ? c->iters : 1));
   o->maxM = stack_max_rows(c, hr);
@@ -1087,8 +1095,8 @@ struct LstmAdjCycle : Cycle {
     const i64 row0 = (i64)(hr.N[l] - 1) * bh;     // step s = 1 applies forward step N_l, stored at row N_l - 1
     LstmChainAdjArgs a{};
     a.B = c->B; a.H = c->H; a.nsteps = hr.N[l]; a.mu = U[l];
-    a.a = w->a[l] + row0; a.p = w->p[l] + row0; a.ci = w->ci[l] + row0; a.cf = w->cf[l] + row0; a.cg = w->cg[l] + row0;
-    a.co = w->co[l] + row0; a.coef_step = -bh;
+    a.a = w->a[l] + row0; a.p = w->p[l] + row0; a.ci = w->cib[l] + row0; a.cf = w->cfb[l] + row0; a.cg = w->cgb[l] + row0;
+    a.co = w->cob[l] + row0; a.coef_step = -bh;
     a.g = G[l]; a.WT = w->bf.W_hhT;
     a.xw = w->chain_xw; a.xw_bytes = w->chain_xw_bytes;
     return lstm_chain_adj_solve(a, s);
@@ -1100,8 +1108,12 @@ struct LstmAdjCycle : Cycle {
     a.M = d.nk * c->B; a.B = c->B; a.H = c->H;
     a.lc = U[d.l] + (size_t)d.in_slot * slot; a.lh = a.lc + bh; a.in_ks = (i64)d.in_stride * slot;
     a.lc_out = w->tmpC; a.lh_out = w->tmpH;
-    a.a = w->a[d.l] + row0; a.p = w->p[d.l] + row0; a.ci = w->ci[d.l] + row0; a.cf = w->cf[d.l] + row0;
-    a.cg = w->cg[d.l] + row0; a.co = w->co[d.l] + row0; a.coef_ks = -(i64)d.tgt_stride * (i64)bh;
+    a.a = w->a[d.l] + row0; a.p = w->p[d.l] + row0; a.coef_ks = -(i64)d.tgt_stride * (i64)bh;
+    const bool cb = w->cib[d.l] != nullptr;      // (the four gate coefficients: bf16 arrays on the bf16 engine, fp32 arrays otherwise)
+    a.ci = cb ? nullptr : w->ci[d.l] + row0; a.cf = cb ? nullptr : w->cf[d.l] + row0;
+    a.cg = cb ? nullptr : w->cg[d.l] + row0; a.co = cb ? nullptr : w->co[d.l] + row0;
+    a.cib = cb ? w->cib[d.l] + row0 : nullptr; a.cfb = cb ? w->cfb[d.l] + row0 : nullptr;
+    a.cgb = cb ? w->cgb[d.l] + row0 : nullptr; a.cob = cb ? w->cob[d.l] + row0 : nullptr;
     a.W_hh = p->W_hh;
     const bool fused = c->operands != MGRIT_OPERANDS_FP32;
     a.up = LstmUpdate{};
@@ -1183,6 +1195,7 @@ int lstm_adjoint_impl(const mgrit_gru_cfg* cfg, const gru_params* p, const float
     a.M = hr.N[l] * c.B; a.B = c.B; a.H = c.H; a.c0 = u0; a.h0 = u0 + bh; a.c = u; a.h = u + bh; a.ts = (i64)slot;
     a.stride_t = hr.stride_t[l]; a.t0 = hr.rem[l]; a.gi = gi; a.W_hh = p->W_hh; a.b_hh = p->b_hh; a.gamma = hr.gamma[l]; a.cell = c.cell;
     a.a = aw.a[l]; a.p = aw.p[l]; a.ci = aw.ci[l]; a.cf = aw.cf[l]; a.cg = aw.cg[l]; a.co = aw.co[l];
+    a.cib = aw.cib[l]; a.cfb = aw.cfb[l]; a.cgb = aw.cgb[l]; a.cob = aw.cob[l];
     if (tf32) { rc = tf32_lstm_linearise(a, &aw.tf, s); if (rc) return rc; }
     else if (bf) { rc = lstmbf_linearise(a, &aw.bf, s); if (rc) return rc; }
     else simt_lstm_linearise(a, s);
@@ -1207,7 +1220,7 @@ int lstm_adjoint_impl(const mgrit_gru_cfg* cfg, const gru_params* p, const float
   const float* lam_c = aw.U[0] + (size_t)(T - 1) * slot;
   if (bf) {
     // bf16 operands: dA is formed as bf16 together with the bias sums, the hidden states are packed straight from u
-    rc = lstmbf_gradients(&c, lam_c, lam_c + bh, -(i64)slot, aw.p[0], aw.ci[0], aw.cf[0], aw.cg[0], aw.co[0], x, u0 + bh, u + bh, (i64)slot, g,
+    rc = lstmbf_gradients(&c, lam_c, lam_c + bh, -(i64)slot, aw.p[0], aw.cib[0], aw.cfb[0], aw.cgb[0], aw.cob[0], x, u0 + bh, u + bh, (i64)slot, g,
                           dx, &aw.bf, s);
     if (rc) return rc;
   } else {

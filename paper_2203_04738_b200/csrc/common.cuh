@@ -179,6 +179,7 @@ struct LstmLinArgs {
   const float* gi;                                  // [T, B, 4H]
   const float* W_hh; const float* b_hh; float gamma; int cell;
   float *a, *p, *ci, *cf, *cg, *co;
+  __nv_bfloat16 *cib, *cfb, *cgb, *cob;             // bf16 engine: the four gate coefficients as bf16 instead (ci..co unused)
 };
 // one adjoint step: dc = Lc + p*Lh; lc_out = a*dc; lh_out = [ci*dc | cf*dc | cg*dc | co*Lh] W_hh   (raw, contiguous [M, H] each)
 struct LstmAdjArgs {
@@ -186,6 +187,7 @@ struct LstmAdjArgs {
   const float* lc; const float* lh; i64 in_ks;      // incoming sensitivities rows
   float* lc_out; float* lh_out;
   const float *a, *p, *ci, *cf, *cg, *co; i64 coef_ks;
+  const __nv_bfloat16 *cib, *cfb, *cgb, *cob;       // bf16 engine: the four gate coefficients as bf16 instead (ci..co unused)
   const float* W_hh;
   LstmUpdate up;
 };

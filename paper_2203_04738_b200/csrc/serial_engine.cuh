@@ -84,7 +84,8 @@ struct LstmChainFwdArgs {
 struct LstmChainAdjArgs {
   int B, H, nsteps;
   float* mu;
-  const float *a, *p, *ci, *cf, *cg, *co;   // coefficient rows of step 1; step s at + (s-1)*coef_step
+  const float *a, *p;                       // coefficient rows of step 1; step s at + (s-1)*coef_step
+  const __nv_bfloat16 *ci, *cf, *cg, *co;   // the four gate coefficients (bf16), same indexing
   i64 coef_step;
   const float* g;
   const __nv_bfloat16* WT;       // [H][4H] = W_hh^T

@@ -627,13 +627,17 @@ __global__ void __launch_bounds__(kThreads, 1) lstm_adj_chain_kernel(LstmChainAd
     int r = e / H, i = e % H;
     const i64 off = (i64)(row0 + r) * H + i;
     const float lh = __ldcg(a.mu + BH + off), dc = __ldcg(a.mu + off) + a.p[off] * lh;
-    As[r * ldk + i] = __float2bfloat16(a.ci[off] * dc);
-    As[r * ldk + H + i] = __float2bfloat16(a.cf[off] * dc);
-    As[r * ldk + 2 * H + i] = __float2bfloat16(a.cg[off] * dc);
-    As[r * ldk + 3 * H + i] = __float2bfloat16(a.co[off] * lh);
+    As[r * ldk + i] = __float2bfloat16(__bfloat162float(a.ci[off]) * dc);
+    As[r * ldk + H + i] = __float2bfloat16(__bfloat162float(a.cf[off]) * dc);
+    As[r * ldk + 2 * H + i] = __float2bfloat16(__bfloat162float(a.cg[off]) * dc);
+    As[r * ldk + 3 * H + i] = __float2bfloat16(__bfloat162float(a.co[off]) * lh);
   }
   // per owned (row, unit): dc of the step in flight, its a and source terms; the coefficients of the step after it
-  float dcur[OPT], pa[OPT], pgc[OPT], pgh[OPT], np_[OPT], nci[OPT], ncf[OPT], ncg[OPT], nco[OPT];
+  // (the bf16 gate coefficients stay raw in their registers until they are used: a conversion behind the load would wait
+  // for it in front of the exchange)
+  float dcur[OPT], pa[OPT], pgc[OPT], pgh[OPT], np_[OPT];
+  bf16 nci[OPT], ncf[OPT], ncg[OPT], nco[OPT];
+  const bf16 bzero = __float2bfloat16(0.f);
 #pragma unroll
   for (int o = 0; o < OPT; ++o) {
     int idx = tid + o * kThreads, r = idx / UNC, i = idx % UNC;
@@ -645,8 +649,8 @@ __global__ void __launch_bounds__(kThreads, 1) lstm_adj_chain_kernel(LstmChainAd
     pgh[o] = (v && a.g) ? a.g[slot + BH + off] : 0.f;
     const bool more = v && a.nsteps > 1;
     const i64 co = a.coef_step + off;
-    np_[o] = more ? a.p[co] : 0.f; nci[o] = more ? a.ci[co] : 0.f; ncf[o] = more ? a.cf[co] : 0.f;
-    ncg[o] = more ? a.cg[co] : 0.f; nco[o] = more ? a.co[co] : 0.f;
+    np_[o] = more ? a.p[co] : 0.f; nci[o] = more ? a.ci[co] : bzero; ncf[o] = more ? a.cf[co] : bzero;
+    ncg[o] = more ? a.cg[co] : bzero; nco[o] = more ? a.co[co] : bzero;
   }
   __syncthreads();
 
@@ -680,7 +684,8 @@ __global__ void __launch_bounds__(kThreads, 1) lstm_adj_chain_kernel(LstmChainAd
         a.mu[(i64)s * slot + BH + off] = lh;
         const float dn = lc + np_[o] * lh;      // the next step's dc (its coefficients are zero behind the last step)
         dcur[o] = dn;
-        x4[0] = nci[o] * dn; x4[1] = ncf[o] * dn; x4[2] = ncg[o] * dn; x4[3] = nco[o] * lh;
+        x4[0] = __bfloat162float(nci[o]) * dn; x4[1] = __bfloat162float(ncf[o]) * dn; x4[2] = __bfloat162float(ncg[o]) * dn;
+        x4[3] = __bfloat162float(nco[o]) * lh;
       }
       if (idx < kRows * UNC) {                  // block order [gate][row][unit]; rows beyond the batch travel as zeros
 #pragma unroll
@@ -701,7 +706,7 @@ __global__ void __launch_bounds__(kThreads, 1) lstm_adj_chain_kernel(LstmChainAd
           const i64 co = (i64)(s + 1) * a.coef_step + off;
           np_[o] = a.p[co]; nci[o] = a.ci[co]; ncf[o] = a.cf[co]; ncg[o] = a.cg[co]; nco[o] = a.co[co];
         } else {
-          np_[o] = nci[o] = ncf[o] = ncg[o] = nco[o] = 0.f;
+          np_[o] = 0.f; nci[o] = ncf[o] = ncg[o] = nco[o] = bzero;
         }
       }
     }

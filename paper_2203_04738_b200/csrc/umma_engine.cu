@@ -1342,8 +1342,16 @@ struct EpiLstm {
           }
         }
         if (LIN) {
-          st8(l.a + o + c0, o0); st8(l.p + o + c0, o1); st8(l.ci + o + c0, o2); st8(l.cf + o + c0, o3); st8(l.cg + o + c0, o4);
-          st8(l.co + o + c0, o5);
+          st8(l.a + o + c0, o0); st8(l.p + o + c0, o1);
+          if (l.cib) {      // gate coefficients as bf16: eight values = one 16-byte store each
+            auto stb = [&](bf16* dst, const float* v) {
+              const uint2 q0 = pack4(make_float4(v[0], v[1], v[2], v[3])), q1 = pack4(make_float4(v[4], v[5], v[6], v[7]));
+              *reinterpret_cast<uint4*>(dst + o + c0) = make_uint4(q0.x, q0.y, q1.x, q1.y);
+            };
+            stb(l.cib, o2); stb(l.cfb, o3); stb(l.cgb, o4); stb(l.cob, o5);
+          } else {
+            st8(l.ci + o + c0, o2); st8(l.cf + o + c0, o3); st8(l.cg + o + c0, o4); st8(l.co + o + c0, o5);
+          }
         } else if (udst) {
           if (usrc) {
 #pragma unroll
@@ -1470,7 +1478,13 @@ __global__ void __launch_bounds__(kPT) pack_lstm_adj_kernel(LstmAdjArgs a, bf16*
     const i64 kk = m / a.B; const int b = (int)(m % a.B);
     const i64 ci = kk * a.coef_ks + (i64)b * a.H + i, li = kk * a.in_ks + (i64)b * a.H + i;
     const float4 lh = ld4(a.lh + li), lc = ld4(a.lc + li), pp = ld4(a.p + ci), aa = ld4(a.a + ci);
-    const float4 c0 = ld4(a.ci + ci), c1 = ld4(a.cf + ci), c2 = ld4(a.cg + ci), c3 = ld4(a.co + ci);
+    float4 c0, c1, c2, c3;
+    if (a.cib) {
+      c0 = unpack4(*reinterpret_cast<const uint2*>(a.cib + ci)); c1 = unpack4(*reinterpret_cast<const uint2*>(a.cfb + ci));
+      c2 = unpack4(*reinterpret_cast<const uint2*>(a.cgb + ci)); c3 = unpack4(*reinterpret_cast<const uint2*>(a.cob + ci));
+    } else {
+      c0 = ld4(a.ci + ci); c1 = ld4(a.cf + ci); c2 = ld4(a.cg + ci); c3 = ld4(a.co + ci);
+    }
     const float4 dc = make_float4(lc.x + pp.x * lh.x, lc.y + pp.y * lh.y, lc.z + pp.z * lh.z, lc.w + pp.w * lh.w);
     float4 v = make_float4(aa.x * dc.x, aa.y * dc.y, aa.z * dc.z, aa.w * dc.w);
     if (!a.up.out) {
@@ -1594,9 +1608,9 @@ namespace {
 // sensitivities at lc / lh + t*lam_ts + b*H (lam_ts may be negative: the adjoint keeps its unknowns in reversed time
 // order).  Block = 32 float4 columns (128 units) x 8 rows at a time.
 __global__ void __launch_bounds__(256) lstm_form_dA_rows_kernel(const float* __restrict__ lc, const float* __restrict__ lh, i64 lam_ts, int B,
-                                                                const float* __restrict__ p, const float* __restrict__ ci,
-                                                                const float* __restrict__ cf, const float* __restrict__ cg,
-                                                                const float* __restrict__ co, i64 M, int H, uint2* __restrict__ dA,
+                                                                const float* __restrict__ p, const bf16* __restrict__ ci,
+                                                                const bf16* __restrict__ cf, const bf16* __restrict__ cg,
+                                                                const bf16* __restrict__ co, i64 M, int H, uint2* __restrict__ dA,
                                                                 float* __restrict__ part, int rows_per_block) {
   __shared__ float red[4][8][128];
   const int tx = threadIdx.x & 31, ty = threadIdx.x >> 5;
@@ -1611,7 +1625,8 @@ __global__ void __launch_bounds__(256) lstm_form_dA_rows_kernel(const float* __r
       const int t = (int)m / B, bb = (int)m - t * B;       // row counts fit 32 bits (checked by the host)
       const i64 li = (i64)t * lam_ts + ((i64)bb * H4 + c4) * 4;
       const float4 h = ld4(lh + li), c = ld4(lc + li), pp = ld4(p + e);
-      const float4 k0 = ld4(ci + e), k1 = ld4(cf + e), k2 = ld4(cg + e), k3 = ld4(co + e);
+      const float4 k0 = unpack4(*reinterpret_cast<const uint2*>(ci + e)), k1 = unpack4(*reinterpret_cast<const uint2*>(cf + e));
+      const float4 k2 = unpack4(*reinterpret_cast<const uint2*>(cg + e)), k3 = unpack4(*reinterpret_cast<const uint2*>(co + e));
       const float4 dc = make_float4(c.x + pp.x * h.x, c.y + pp.y * h.y, c.z + pp.z * h.z, c.w + pp.w * h.w);
       const float4 v[4] = {make_float4(k0.x * dc.x, k0.y * dc.y, k0.z * dc.z, k0.w * dc.w), make_float4(k1.x * dc.x, k1.y * dc.y, k1.z * dc.z, k1.w * dc.w),
                            make_float4(k2.x * dc.x, k2.y * dc.y, k2.z * dc.z, k2.w * dc.w), make_float4(k3.x * h.x, k3.y * h.y, k3.z * h.z, k3.w * h.w)};
@@ -1650,8 +1665,8 @@ __global__ void __launch_bounds__(kPT) lstm_sum_db_kernel(const float* __restric
 
 // All gradients of the LSTM parameters (and dx) from the step-output sensitivities (lc, lh; rows (t, b) at + t*lam_ts + b*H),
 // the level-0 coefficients and the hidden states entering each step (h0, then h_rows + (t-1)*h_ts).
-int lstmbf_gradients(const mgrit_gru_cfg* c, const float* lc, const float* lh, i64 lam_ts, const float* p, const float* ci, const float* cf,
-                     const float* cg, const float* co, const float* x, const float* h0, const float* h_rows, i64 h_ts, const gru_grads* g,
+int lstmbf_gradients(const mgrit_gru_cfg* c, const float* lc, const float* lh, i64 lam_ts, const float* p, const bf16* ci, const bf16* cf,
+                     const bf16* cg, const bf16* co, const float* x, const float* h0, const float* h_rows, i64 h_ts, const gru_grads* g,
                      float* dx, LstmBfWs* w, cudaStream_t s) {
   const int H = c->H, I = c->I, B = c->B;
   const i64 M = (i64)c->T * B;

@@ -75,9 +75,9 @@ int lstmbf_fwd_step(const LstmFwdArgs& a, LstmBfWs* w, cudaStream_t s);
 int lstmbf_linearise(const LstmLinArgs& a, LstmBfWs* w, cudaStream_t s);
 int lstmbf_adj_step(const LstmAdjArgs& a, LstmBfWs* w, cudaStream_t s);
 // dW_hh, dW_ih (and dx) from dA[T*B,4H] fp32; hidden states h0 [B,H] and hk [T,B,H] fp32
-int lstmbf_gradients(const mgrit_gru_cfg* c, const float* lc, const float* lh, i64 lam_ts, const float* p, const float* ci, const float* cf,
-                     const float* cg, const float* co, const float* x, const float* h0, const float* h_rows, i64 h_ts, const gru_grads* g,
-                     float* dx, LstmBfWs* w, cudaStream_t s);
+int lstmbf_gradients(const mgrit_gru_cfg* c, const float* lc, const float* lh, i64 lam_ts, const float* p, const __nv_bfloat16* ci,
+                     const __nv_bfloat16* cf, const __nv_bfloat16* cg, const __nv_bfloat16* co, const float* x, const float* h0,
+                     const float* h_rows, i64 h_ts, const gru_grads* g, float* dx, LstmBfWs* w, cudaStream_t s);
 
 int umma_supported(const mgrit_gru_cfg* c);
 void umma_plan_fwd(const mgrit_gru_cfg* c, const int* N, int L, char* base, size_t* off, UmmaFwdWs* o);
