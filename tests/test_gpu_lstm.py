@@ -114,7 +114,9 @@ def test_lstm_full_size_sampled_row_and_gradients():
     u, gi, rn = B.mgrit_lstm_forward(cfg_f, p, xd, u0d, want_resnorm=True)
     du, du0, r, rna = B.mgrit_lstm_adjoint(cfg_a, p, xd, u0d, gi, u, dhT=to_dev(dhT), want_resnorm=True)
     # the coarsest level ran as chains: far fewer launches than one per dependent step (128 steps, 4 cycles in all)
-    assert B.kernel_launches() - n0 < 400
+    # (MGRIT_GRU_CHAIN_LL=0, an A/B switch of the library, turns those kernels off)
+    import os
+    assert B.kernel_launches() - n0 < 400 or os.environ.get("MGRIT_GRU_CHAIN_LL") == "0"
     assert B.last_device_status() == 0
     assert all(a > b for a, b in zip(rn, rn[1:])) and all(a > b for a, b in zip(rna, rna[1:]))
     P = [a.astype(np.float64) for a in P32]

@@ -286,7 +286,8 @@ def test_unwritten_fp32_projection_changes_no_bit(B):
         h2, _, rn2 = B.mgrit_gru_forward(skip, p, x, h0, gi=b2, want_resnorm=True)
         assert torch.equal(h, h2) and rn == rn2
         written = not bool(torch.isnan(B.gi_view(skip, b2)).all())
-        assert written == (Bsz == 24)
+        import os
+        assert written == (Bsz == 24 or os.environ.get("MGRIT_GRU_GI_BF16") == "0")      # (that A/B switch removes the bf16 copy)
         if written:
             assert torch.equal(B.gi_view(skip, b2), B.gi_view(carry, b1))
         r = B.mgrit_gru_adjoint(carry, p, x, h0, b1, h, dhT=h[-1].contiguous())
